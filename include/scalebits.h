@@ -1,0 +1,173 @@
+/*
+ * scalebits.h -- C ABI of the B200 (sm_100a) hot path of ScaleBITS' bitwidth search
+ * (arxiv 2602.17698): score every hardware-aligned weight block at every candidate
+ * bitwidth, then allocate bits globally under a memory budget.
+ *
+ * Conventions (all entry points):
+ *   - Every tensor pointer is CALLER-OWNED DEVICE memory on the context's device,
+ *     valid until the context's stream has passed the call.  The only host pointers
+ *     are `bits` arrays (read during the call), `sb_alloc_report*` and out-params of
+ *     sb_create / sb_kernel_launches.
+ *   - Calls enqueue work on the context's stream and return without waiting, except
+ *     sb_allocate_bits and sb_sync, which synchronise that stream.
+ *   - Return value: SB_OK, or an argument / shape / budget error detected on the host
+ *     (nothing was enqueued).  Conditions detected on the device (non-finite input,
+ *     packed capacity exceeded, a bounded wait that ran out) are latched in a device
+ *     status word and returned by the next sb_sync / sb_allocate_bits.
+ *   - bf16 matrices are row-major with a leading dimension in elements; the base
+ *     must be 16-byte aligned and the leading dimension a multiple of 8.
+ *   - A permutation is int32 perm[new] = old.  NULL means identity.
+ *   - The library owns one scratch arena per context, grown on demand (a growth
+ *     synchronises the stream); after the first call of each shape nothing allocates.
+ *   - No call falls back to the CPU.
+ */
+#ifndef SCALEBITS_H_
+#define SCALEBITS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sb_ctx sb_ctx;
+
+typedef enum {
+    SB_OK = 0,
+    SB_ERR_INVALID = 1,     /* NULL / out-of-range argument, bad bit list            */
+    SB_ERR_SHAPE = 2,       /* sizes not divisible as required, misaligned pointer   */
+    SB_ERR_BUDGET = 3,      /* budget below the smallest candidate bitwidth          */
+    SB_ERR_SCRATCH = 4,     /* scratch allocation failed / capacity too small        */
+    SB_ERR_CUDA = 5,        /* a CUDA runtime call failed (see sb_last_error)        */
+    SB_ERR_NOCONVERGE = 6,  /* Algorithm 2 hit the iteration cap (4096)              */
+    SB_ERR_NONFINITE = 7,   /* a non-finite score or error was produced on device    */
+    SB_ERR_TIMEOUT = 8      /* a bounded device-side wait (scan look-back) ran out   */
+} sb_status;
+
+enum { SB_ALLOC_SCALEBITS = 0, SB_ALLOC_GREEDY = 1 };
+enum { SB_ACC_ROW = 1, SB_ACC_COL = 2 };
+
+/* Context: device, stream (a cudaStream_t passed as void*, NULL = default stream),
+ * scratch arena, device status word.  One context per stream; not thread-safe.      */
+sb_status sb_create(sb_ctx** ctx, int device, void* cuda_stream);
+sb_status sb_destroy(sb_ctx* ctx);
+/* Waits for the stream, returns and clears the latched device status.               */
+sb_status sb_sync(sb_ctx* ctx);
+/* Static / context-owned string describing the last host-side error.                */
+const char* sb_last_error(const sb_ctx* ctx);
+/* Number of kernels this context has launched so far (for launch accounting).       */
+int64_t sb_kernel_launches(const sb_ctx* ctx);
+
+/* Calibration second moments -- the column factor |x_j| of the element sensitivity
+ * (Section 3.2, the equation after Eq. 3), aggregated over tokens as a second moment:
+ *     sumsq[j] = (accumulate ? sumsq[j] : 0) + scale * sum_t X[t][j]^2
+ * X: bf16 [T][K], leading dimension ldx.  sumsq: fp32 [K].  K % 8 == 0.
+ * fp32 accumulation in a fixed order (run-to-run deterministic).                    */
+sb_status sb_calib_moments(sb_ctx* ctx, const void* X_bf16, int64_t T, int64_t K, int64_t ldx,
+                           float* sumsq, int accumulate, float scale);
+
+/* Bi-directional channel reordering (Section 4.1; coupling rules of Appendix D).
+ * Phase 1 (W != NULL): fake-quantise W on its ORIGINAL layout at ref_bits (round to
+ * nearest, asymmetric min-max, groups of `group` consecutive columns; Section 5
+ * "Implementation"), element sensitivity s_rj = a_r c_j (W_rj - Q(W)_rj)^2, and
+ *     row_score[r] (+)= sum_j s_rj,   col_score[j] (+)= sum_r s_rj
+ * (accumulate is a bit mask: SB_ACC_ROW adds to what row_score holds, SB_ACC_COL to what
+ * col_score holds, otherwise the buffer is overwritten; matrices that must share a
+ * permutation pass the same buffer).  Either score pointer may be NULL.
+ * Phase 2 (per axis, when *_segment > 0 and *_perm != NULL): sort the channels of the
+ * score buffer by score, descending, ties to the lower index, independently inside
+ * each run of *_segment channels (*_segment = axis length: whole axis; head_dim: within
+ * each attention head).  Phase 2 sees the scores after phase 1.
+ * W == NULL skips phase 1 ("sort only"); R / C still give the axis lengths.
+ * C % group == 0, group in {16,32,64,128}.  col_moment: fp32 [C]; row_weight: fp32
+ * [R] or NULL (= 1).                                                                 */
+sb_status sb_reorder_channels(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_t C, int64_t ldw,
+                              const float* col_moment, const float* row_weight,
+                              int ref_bits, int group,
+                              float* row_score, float* col_score, int accumulate,
+                              int64_t row_segment, int64_t col_segment,
+                              int32_t* row_perm, int32_t* col_perm);
+
+/* Helpers for grouped-query attention (Appendix D: value / output projections are
+ * reordered inside each head; query heads that read one value head share its order):
+ *   fold:   dst[h*seg + d] += sum_{u<reps} src[(h*reps + u)*seg + d],  n_dst = len(dst)
+ *   expand: out[(h*reps + u)*seg + d] = (h*reps + u)*seg + (perm[h*seg + d] - h*seg)   */
+sb_status sb_fold_segment_scores(sb_ctx* ctx, float* dst, const float* src, int64_t n_dst,
+                                 int reps, int64_t seg);
+sb_status sb_expand_segment_perm(sb_ctx* ctx, int32_t* out, const int32_t* perm, int64_t n_src,
+                                 int reps, int64_t seg);
+
+/* Block scores -- the hot loop (block partition: Section 4.1; marginal gains of one
+ * precision step: Section 4.2, Eq. 6).  On the permuted layout
+ * W'[r][j] = W[row_perm[r]][col_perm[j]], for every block i of block_rows x block_cols
+ * (row-major over the block grid) and every candidate b_l = bits[l]:
+ *     err[i][l]  = sum_{(r,j) in block i} a_r c_j (W'_rj - Q_{b_l}(W')_rj)^2
+ *     gain[i][l] = (err[i][l] - err[i][l+1]) / ((b_{l+1} - b_l) * block_rows*block_cols)
+ * with the same quantizer as above on groups of `group` consecutive columns of W'.
+ * col_moment / row_weight are indexed by ORIGINAL column / row.  All candidates are
+ * evaluated from registers in one pass over W; fp32 arithmetic, fixed summation order.
+ * bits: host array, strictly ascending, each in 1..8, 1 <= n_bits <= 8.
+ * R % block_rows == 0, C % block_cols == 0, block_cols % group == 0, block_rows even,
+ * block_cols in {32,64} or a multiple of 128.
+ * err: fp32 [(R/br)*(C/bc)][n_bits]; gain: fp32 [..][n_bits-1] or NULL;
+ * W_perm_out: bf16 [R][C] (ld = C) receives W' or NULL.                              */
+sb_status sb_block_scores(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_t C, int64_t ldw,
+                          const int32_t* row_perm, const int32_t* col_perm,
+                          const float* col_moment, const float* row_weight,
+                          int block_rows, int block_cols, int group,
+                          const int* bits, int n_bits,
+                          float* err, float* gain, void* W_perm_out_bf16);
+
+typedef struct {
+    int64_t cap_bits;            /* floor(budget * sum M_i), code bits only            */
+    int64_t used_bits;           /* sum M_i * bits[level_i] of the result              */
+    int32_t iterations;          /* Algorithm 2 loop iterations (greedy: steps taken)  */
+    int32_t accepted;            /* accepted exchange steps                            */
+    int32_t rejected;            /* rejected exchange steps (each halves k)            */
+    int32_t expansions;          /* expansion steps                                    */
+    double proxy_loss_init;      /* sum_i err[i][warm start]                           */
+    double proxy_loss_final;     /* sum_i err[i][level_i]                              */
+    int64_t level_hist[8];       /* blocks per level                                   */
+} sb_alloc_report;
+
+/* Global allocation (Eq. 1 with blocks weighted by their sizes M_i) on the separable
+ * proxy loss L(level) = sum_i err[i][level_i].
+ *   SB_ALLOC_SCALEBITS: Algorithm 2 -- warm start at the largest candidate <= budget,
+ *     batches of k = floor(gamma N) blocks ranked by the gain of their next step up /
+ *     down, expansion while the budget is slack (truncated so it is never exceeded),
+ *     balanced exchange when it is active, accepted only if the proxy loss strictly
+ *     falls, else k halves; stops when k < floor(gammaT N).
+ *   SB_ALLOC_GREEDY: Algorithm 1 from the lowest candidate along each block's lower
+ *     convex hull: all hull steps sorted by gain per bit, longest affordable prefix.
+ * Ranking keys are IEEE binary64 quotients of the fp32 table entries; ties go to the
+ * lower block index.  err: fp32 [N][n_bits].  block_elems: int64 [N] or NULL (then every
+ * block has uniform_block_elems weights).  level: uint8 [N], index into bits[].
+ * report: HOST struct, filled before return (the call synchronises the stream).        */
+sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
+                           const int64_t* block_elems, int64_t uniform_block_elems,
+                           const int* bits, int n_bits, double budget_avg_bits,
+                           int mode, double gamma0, double gammaT,
+                           uint8_t* level, sb_alloc_report* report);
+
+/* Pack (Section 5.3: one bitwidth per tile).  Quantise each block of W' at
+ * bits[level[block]] with the same quantizer, evaluated in IEEE binary64 so that the
+ * integer codes are reproducible: lo = min, range = max - min, inv = qmax / range,
+ * q = clamp(rint((v - lo) * inv), 0, qmax) (round half to even), scale = range / qmax.
+ * Layout: blocks in grid row-major order; inside a block the codes in block-row-major
+ * order, code k in bits [k*b, (k+1)*b) of a little-endian stream of 32-bit words;
+ * block_off_words[i] = first word of block i (exclusive prefix sum, [nb+1] entries);
+ * meta[(r*(C/group) + g)] = {(float)scale, (float)lo} for group g of permuted row r.
+ * If block_off_words[nb] > packed_capacity_words nothing beyond the capacity is written
+ * and SB_ERR_SCRATCH is latched.  block_rows*block_cols*bits % 32 == 0 is required,
+ * group % 4 == 0, block_cols % 32 == 0.                                              */
+sb_status sb_pack_blocks(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_t C, int64_t ldw,
+                         const int32_t* row_perm, const int32_t* col_perm,
+                         int block_rows, int block_cols, int group,
+                         const int* bits, int n_bits, const uint8_t* level,
+                         uint32_t* packed, int64_t packed_capacity_words,
+                         int64_t* block_off_words, float* meta);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SCALEBITS_H_ */

@@ -1,0 +1,112 @@
+// Context management of the C-ABI library: device, stream, scratch arena, status word.
+#include <stdarg.h>
+#include <string.h>
+
+#include "common.cuh"
+
+sb_status sb_fail(sb_ctx* ctx, sb_status st, const char* fmt, ...) {
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof ctx->err, fmt, ap);
+        va_end(ap);
+    }
+    return st;
+}
+
+bool sb_check_bits(const int* bits, int n_bits) {
+    if (!bits || n_bits < 1 || n_bits > 8) return false;
+    for (int l = 0; l < n_bits; ++l) {
+        if (bits[l] < 1 || bits[l] > 8) return false;
+        if (l > 0 && bits[l] <= bits[l - 1]) return false;
+    }
+    return true;
+}
+
+sb_status sb_scratch(sb_ctx* ctx, size_t bytes, void** out) {
+    if (bytes > ctx->scratch_bytes) {
+        // growth is rare (first call of a shape): wait for work that may use the old arena
+        SB_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+        if (ctx->scratch) SB_CUDA(ctx, cudaFree(ctx->scratch));
+        ctx->scratch = nullptr;
+        ctx->scratch_bytes = 0;
+        size_t want = bytes + bytes / 8 + (1u << 20);
+        cudaError_t e = cudaMalloc(&ctx->scratch, want);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            return sb_fail(ctx, SB_ERR_SCRATCH, "scratch arena of %zu bytes: %s", want,
+                           cudaGetErrorString(e));
+        }
+        ctx->scratch_bytes = want;
+    }
+    *out = ctx->scratch;
+    return SB_OK;
+}
+
+extern "C" {
+
+sb_status sb_create(sb_ctx** out, int device, void* cuda_stream) {
+    if (!out) return SB_ERR_INVALID;
+    *out = nullptr;
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) {
+        (void)cudaGetLastError();
+        return SB_ERR_CUDA;   // no usable CUDA device: this library has no CPU path
+    }
+    sb_ctx* ctx = new sb_ctx();
+    ctx->device = device;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaDeviceProp prop;
+    if (cudaSetDevice(device) != cudaSuccess ||
+        cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
+        delete ctx;
+        return SB_ERR_CUDA;
+    }
+    if (prop.major != 10) {   // built for sm_100a only
+        delete ctx;
+        return SB_ERR_CUDA;
+    }
+    ctx->sm_count = prop.multiProcessorCount;
+    if (cudaMalloc(&ctx->dstate, sizeof(SbDeviceState)) != cudaSuccess ||
+        cudaMemset(ctx->dstate, 0, sizeof(SbDeviceState)) != cudaSuccess ||
+        cudaMallocHost(&ctx->pinned, 4096) != cudaSuccess) {
+        delete ctx;
+        return SB_ERR_CUDA;
+    }
+    ctx->pinned_bytes = 4096;
+    *out = ctx;
+    return SB_OK;
+}
+
+sb_status sb_destroy(sb_ctx* ctx) {
+    if (!ctx) return SB_OK;
+    cudaSetDevice(ctx->device);
+    cudaStreamSynchronize(ctx->stream);
+    if (ctx->scratch) cudaFree(ctx->scratch);
+    if (ctx->dstate) cudaFree(ctx->dstate);
+    if (ctx->lb_mem) cudaFree(ctx->lb_mem);
+    if (ctx->pinned) cudaFreeHost(ctx->pinned);
+    delete ctx;
+    return SB_OK;
+}
+
+sb_status sb_sync(sb_ctx* ctx) {
+    if (!ctx) return SB_ERR_INVALID;
+    SbDeviceState* h = static_cast<SbDeviceState*>(ctx->pinned);
+    SB_CUDA(ctx, cudaMemcpyAsync(h, ctx->dstate, sizeof(SbDeviceState), cudaMemcpyDeviceToHost,
+                                 ctx->stream));
+    SB_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (h->status != 0) {
+        sb_status st = static_cast<sb_status>(h->status);
+        int where = h->where;
+        SB_CUDA(ctx, cudaMemsetAsync(ctx->dstate, 0, 2 * sizeof(int), ctx->stream));
+        return sb_fail(ctx, st, "device-side status %d latched by kernel family %d", (int)st, where);
+    }
+    return SB_OK;
+}
+
+const char* sb_last_error(const sb_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+int64_t sb_kernel_launches(const sb_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

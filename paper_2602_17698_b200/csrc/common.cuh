@@ -1,0 +1,118 @@
+// Shared host/device helpers of the CUDA library (sm_100a only).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "scalebits.h"
+
+// ---- context ---------------------------------------------------------------------
+struct SbDeviceState {           // lives in device memory, one per context
+    int status;                  // latched sb_status detected on the device
+    int where;                   // kernel id that latched it
+    unsigned int ticket;         // dynamic tile ids of the look-back scans
+    unsigned int pad;
+};
+
+struct sb_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    int sm_count = 148;
+    void* scratch = nullptr;     // arena, grown on demand
+    size_t scratch_bytes = 0;
+    SbDeviceState* dstate = nullptr;
+    void* pinned = nullptr;      // small pinned host buffer for read-backs
+    size_t pinned_bytes = 0;
+    unsigned int scan_epoch = 0; // tags look-back descriptors so they need no clearing
+    void* lb_mem = nullptr;      // look-back descriptors (context-owned, never in the arena)
+    unsigned int lb_max_tiles = 0;
+    int64_t launches = 0;
+    char err[256] = {0};
+};
+
+sb_status sb_fail(sb_ctx* ctx, sb_status st, const char* fmt, ...);
+sb_status sb_scratch(sb_ctx* ctx, size_t bytes, void** out);   // whole arena, >= bytes
+
+#define SB_CUDA(ctx, call)                                                              \
+    do {                                                                                \
+        cudaError_t e__ = (call);                                                       \
+        if (e__ != cudaSuccess)                                                         \
+            return sb_fail((ctx), SB_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e__)); \
+    } while (0)
+
+#define SB_LAUNCHED(ctx)                                                                \
+    do {                                                                                \
+        (ctx)->launches++;                                                              \
+        cudaError_t e__ = cudaGetLastError();                                           \
+        if (e__ != cudaSuccess)                                                         \
+            return sb_fail((ctx), SB_ERR_CUDA, "launch failed at %s:%d: %s", __FILE__,  \
+                           __LINE__, cudaGetErrorString(e__));                          \
+    } while (0)
+
+// carve aligned sub-buffers out of the arena
+struct Carver {
+    char* base; size_t off = 0;
+    explicit Carver(void* p) : base(static_cast<char*>(p)) {}
+    template <typename T> T* take(size_t n) {
+        off = (off + 255) & ~size_t(255);
+        T* p = reinterpret_cast<T*>(base + off);
+        off += n * sizeof(T);
+        return p;
+    }
+    static size_t need(std::initializer_list<size_t> bytes) {
+        size_t t = 0;
+        for (size_t b : bytes) t = ((t + 255) & ~size_t(255)) + b;
+        return t + 256;
+    }
+};
+
+bool sb_check_bits(const int* bits, int n_bits);
+
+enum SbKernelId { SBK_MOMENTS = 1, SBK_STATS, SBK_SCORES, SBK_GATHER, SBK_ARGSORT, SBK_SCAN,
+                  SBK_SORT, SBK_ALLOC, SBK_PACK };
+
+// ---- device helpers ----------------------------------------------------------------
+#ifdef __CUDACC__
+__device__ __forceinline__ void sb_latch(SbDeviceState* st, int status, int where) {
+    if (atomicCAS(&st->status, 0, status) == 0) st->where = where;
+}
+
+// two bf16 packed in a 32-bit word -> two fp32 (exact)
+__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// 128-bit read-only streaming load (weights / activations are read exactly once)
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint2 ld_stream8(const void* p) {
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];"
+                 : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_u32(unsigned* p, unsigned v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+#endif

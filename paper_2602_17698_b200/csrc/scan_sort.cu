@@ -1,0 +1,207 @@
+// Hand-written device-wide primitives: exclusive scans (decoupled look-back) and a stable
+// LSD radix sort of 64-bit keys with 32-bit payloads (8-bit digits: per-tile histogram,
+// one scan over the digit-major histogram, stable scatter).
+#include "lookback.cuh"
+
+namespace {
+
+constexpr int SCAN_THREADS = 256;
+constexpr int SCAN_ITEMS = 8;
+constexpr int SCAN_TILE = SCAN_THREADS * SCAN_ITEMS;
+
+template <typename T>
+__global__ void __launch_bounds__(SCAN_THREADS)
+scan_exclusive_kernel(const T* __restrict__ in, T* __restrict__ out, int64_t n, int write_total,
+                      LookbackBuf lb, unsigned epoch, SbDeviceState* st) {
+    const unsigned tile = lookback_tile_id(st);
+    const int64_t base = (int64_t)tile * SCAN_TILE + (int64_t)threadIdx.x * SCAN_ITEMS;
+    T v[SCAN_ITEMS];
+    T sum = t_zero((T*)nullptr);
+#pragma unroll
+    for (int k = 0; k < SCAN_ITEMS; ++k) {
+        v[k] = (base + k < n) ? in[base + k] : t_zero((T*)nullptr);
+        sum = t_add(sum, v[k]);
+    }
+    T tile_total;
+    T ex = block_exclusive_scan<T, SCAN_THREADS>(sum, tile_total);
+    const T prefix = lookback_prefix<T>(tile_total, tile, lb, epoch, st);
+    T run = t_add(prefix, ex);
+#pragma unroll
+    for (int k = 0; k < SCAN_ITEMS; ++k) {
+        if (base + k < n) out[base + k] = run;
+        run = t_add(run, v[k]);
+    }
+    if (write_total && tile == gridDim.x - 1 && threadIdx.x == SCAN_THREADS - 1) out[n] = run;
+}
+
+// ---- radix sort ---------------------------------------------------------------------------
+constexpr int SORT_THREADS = 256;
+constexpr int SORT_ITEMS = 8;                       // consecutive 32-item warp steps
+constexpr int SORT_TILE = SORT_THREADS * SORT_ITEMS;   // 2048 keys per CTA
+constexpr int RADIX = 256;
+
+// hist[digit * tiles + tile] = number of keys of the tile with that digit
+__global__ void __launch_bounds__(SORT_THREADS)
+radix_hist_kernel(const unsigned long long* __restrict__ keys, int64_t n, int shift, int tiles,
+                  unsigned* __restrict__ hist) {
+    __shared__ unsigned h[RADIX];
+    h[threadIdx.x] = 0;
+    __syncthreads();
+    const int64_t base = (int64_t)blockIdx.x * SORT_TILE;
+    for (int k = 0; k < SORT_ITEMS; ++k) {
+        const int64_t i = base + k * SORT_THREADS + threadIdx.x;
+        if (i < n) atomicAdd(&h[(unsigned)(keys[i] >> shift) & 0xffu], 1u);
+    }
+    __syncthreads();
+    hist[(int64_t)threadIdx.x * tiles + blockIdx.x] = h[threadIdx.x];
+}
+
+// Stable scatter.  Warp w of the CTA owns the contiguous keys [w*256, (w+1)*256) of the tile
+// and walks them 32 at a time; within a step equal digits are ranked by lane
+// (__match_any_sync), across steps by a per-warp running count, across warps by a prefix
+// over the warps' digit counts, across tiles by the scanned histogram.
+__global__ void __launch_bounds__(SORT_THREADS)
+radix_scatter_kernel(const unsigned long long* __restrict__ keys_in, const unsigned* __restrict__ vals_in,
+                     unsigned long long* __restrict__ keys_out, unsigned* __restrict__ vals_out,
+                     int64_t n, int shift, int tiles, const unsigned* __restrict__ hist_scanned) {
+    constexpr int WARPS = SORT_THREADS / 32;
+    __shared__ unsigned cnt[WARPS][RADIX];          // running count per warp and digit
+    __shared__ unsigned basepos[RADIX];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int d = lane; d < RADIX; d += 32) cnt[warp][d] = 0;
+    __syncwarp();
+    const int64_t wbase = (int64_t)blockIdx.x * SORT_TILE + (int64_t)warp * (32 * SORT_ITEMS);
+    unsigned long long key[SORT_ITEMS];
+    unsigned val[SORT_ITEMS], rank[SORT_ITEMS];
+#pragma unroll
+    for (int k = 0; k < SORT_ITEMS; ++k) {
+        const int64_t i = wbase + k * 32 + lane;
+        const bool ok = i < n;
+        key[k] = ok ? keys_in[i] : 0ull;
+        val[k] = ok ? vals_in[i] : 0u;
+        const unsigned d = (unsigned)(key[k] >> shift) & 0xffu;
+        // lanes past the end vote in a digit of their own (256) so they never disturb ranks
+        const unsigned peers = __match_any_sync(0xffffffffu, ok ? d : 256u);
+        const unsigned before = __popc(peers & ((1u << lane) - 1u));
+        unsigned prior = 0;
+        if (ok) prior = cnt[warp][d];
+        __syncwarp();
+        if (ok && before == 0) cnt[warp][d] = prior + __popc(peers);
+        __syncwarp();
+        rank[k] = prior + before;
+    }
+    __syncthreads();
+    // prefix over warps for every digit (thread d handles digit d), plus the tile's base
+    {
+        const int d = threadIdx.x;
+        unsigned run = 0;
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) {
+            const unsigned c = cnt[w][d];
+            cnt[w][d] = run;
+            run += c;
+        }
+        basepos[d] = hist_scanned[(int64_t)d * tiles + blockIdx.x];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < SORT_ITEMS; ++k) {
+        const int64_t i = wbase + k * 32 + lane;
+        if (i < n) {
+            const unsigned d = (unsigned)(key[k] >> shift) & 0xffu;
+            const int64_t pos = (int64_t)basepos[d] + cnt[warp][d] + rank[k];
+            keys_out[pos] = key[k];
+            vals_out[pos] = val[k];
+        }
+    }
+}
+
+}  // namespace
+
+// A fresh tag for the next look-back launch, and descriptors for `tiles` tiles.  The
+// descriptors are recognised by their tag, so they are zeroed only when the buffer is
+// (re)allocated or the 30-bit tag wraps.
+LookbackBuf sb_lookback(sb_ctx* ctx, unsigned tiles, unsigned* epoch_out, sb_status* st) {
+    *st = SB_OK;
+    ctx->scan_epoch++;
+    bool rezero = false;
+    if (ctx->scan_epoch >= (1u << 30)) { ctx->scan_epoch = 1; rezero = true; }
+    if (tiles > ctx->lb_max_tiles) {
+        unsigned want = 1u << 14;
+        while (want < tiles) want <<= 1;
+        cudaStreamSynchronize(ctx->stream);
+        if (ctx->lb_mem) cudaFree(ctx->lb_mem);
+        ctx->lb_mem = nullptr;
+        ctx->lb_max_tiles = 0;
+        if (cudaMalloc(&ctx->lb_mem, (size_t)want * 36) != cudaSuccess) {
+            (void)cudaGetLastError();
+            *st = sb_fail(ctx, SB_ERR_SCRATCH, "look-back descriptors for %u tiles", want);
+            return LookbackBuf{};
+        }
+        ctx->lb_max_tiles = want;
+        rezero = true;
+    }
+    if (rezero) cudaMemsetAsync(ctx->lb_mem, 0, (size_t)ctx->lb_max_tiles * 36, ctx->stream);
+    LookbackBuf lb;
+    unsigned char* p = static_cast<unsigned char*>(ctx->lb_mem);
+    lb.agg = p;
+    lb.inc = p + (size_t)ctx->lb_max_tiles * 16;
+    lb.flags = reinterpret_cast<unsigned*>(p + (size_t)ctx->lb_max_tiles * 32);
+    lb.max_tiles = ctx->lb_max_tiles;
+    *epoch_out = ctx->scan_epoch;
+    return lb;
+}
+
+template <typename T>
+static sb_status scan_launch(sb_ctx* ctx, const T* in, T* out, int64_t n, int write_total) {
+    if (n <= 0) {
+        if (write_total) SB_CUDA(ctx, cudaMemsetAsync(out, 0, sizeof(T), ctx->stream));
+        return SB_OK;
+    }
+    const unsigned tiles = (unsigned)((n + SCAN_TILE - 1) / SCAN_TILE);
+    sb_status st;
+    unsigned epoch;
+    LookbackBuf lb = sb_lookback(ctx, tiles, &epoch, &st);
+    if (st != SB_OK) return st;
+    scan_exclusive_kernel<T><<<tiles, SCAN_THREADS, 0, ctx->stream>>>(
+        in, out, n, write_total, lb, epoch, ctx->dstate);
+    SB_LAUNCHED(ctx);
+    return SB_OK;
+}
+
+sb_status sb_scan_exclusive_u32(sb_ctx* ctx, const unsigned* in, unsigned* out, int64_t n) {
+    return scan_launch<unsigned>(ctx, in, out, n, 0);
+}
+sb_status sb_scan_exclusive_u64(sb_ctx* ctx, const unsigned long long* in, unsigned long long* out,
+                                int64_t n) {
+    return scan_launch<unsigned long long>(ctx, in, out, n, 1);
+}
+
+size_t sb_radix_sort_scratch_bytes(int64_t n) {
+    const int64_t tiles = (n + SORT_TILE - 1) / SORT_TILE;
+    return (size_t)tiles * RADIX * sizeof(unsigned) * 2 + 512;
+}
+
+sb_status sb_radix_sort_u64(sb_ctx* ctx, unsigned long long* keys, unsigned long long* keys_tmp,
+                            unsigned* vals, unsigned* vals_tmp, int64_t n, void* scratch) {
+    if (n <= 0) return SB_OK;
+    const int tiles = (int)((n + SORT_TILE - 1) / SORT_TILE);
+    Carver cv(scratch);
+    unsigned* hist = cv.take<unsigned>((size_t)tiles * RADIX);
+    unsigned* hist_scanned = cv.take<unsigned>((size_t)tiles * RADIX);
+    unsigned long long* kin = keys; unsigned long long* kout = keys_tmp;
+    unsigned* vin = vals; unsigned* vout = vals_tmp;
+    for (int pass = 0; pass < 8; ++pass) {
+        const int shift = pass * 8;
+        radix_hist_kernel<<<tiles, SORT_THREADS, 0, ctx->stream>>>(kin, n, shift, tiles, hist);
+        SB_LAUNCHED(ctx);
+        sb_status st = sb_scan_exclusive_u32(ctx, hist, hist_scanned, (int64_t)tiles * RADIX);
+        if (st != SB_OK) return st;
+        radix_scatter_kernel<<<tiles, SORT_THREADS, 0, ctx->stream>>>(kin, vin, kout, vout, n, shift,
+                                                                      tiles, hist_scanned);
+        SB_LAUNCHED(ctx);
+        unsigned long long* tk = kin; kin = kout; kout = tk;
+        unsigned* tv = vin; vin = vout; vout = tv;
+    }
+    return SB_OK;
+}

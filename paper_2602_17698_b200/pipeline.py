@@ -1,0 +1,192 @@
+"""Sequences the C-ABI calls for one Llama-shaped decoder layer (harness, not hot path).
+
+Only bookkeeping lives here: which matrices share a channel permutation (Appendix D of
+the paper) and where each matrix's rows of the global error table start.  Every number
+is produced by the library's kernels.
+
+Coupling (Appendix D):
+  * residual stream: the columns of q/k/v/gate/up and the rows of o/down share one
+    permutation of the hidden dimension (scores summed over all of them);
+  * MLP: rows of gate/up and columns of down share one permutation of the intermediate
+    dimension;
+  * attention: only v (rows) and o (columns) are reordered, inside each head; with
+    grouped-query attention the query heads that read one value head share its order;
+    the output order of q and k is kept.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, Optional, Sequence
+
+import torch
+
+from .binding import Context, SB_ALLOC_SCALEBITS
+from .synth import LayerShape
+
+
+@dataclass
+class SearchConfig:
+    bits: Sequence[int] = (2, 3, 4, 8)
+    budget: float = 2.5
+    block_rows: int = 128
+    block_cols: int = 128
+    group: int = 128
+    gamma0: float = 0.05
+    gammaT: float = 0.02
+    mode: int = SB_ALLOC_SCALEBITS
+    reorder: bool = True
+
+    @property
+    def ref_bits(self) -> int:
+        """Reorder statistics are taken at the warm-start precision (Algorithm 2, line 2)."""
+        ok = [b for b in self.bits if b <= self.budget]
+        return max(ok) if ok else min(self.bits)
+
+
+# (row permutation, column permutation) of each linear, by name of the coupled channel set
+COUPLING = {
+    "q_proj": (None, "hidden"), "k_proj": (None, "hidden"), "v_proj": ("v_heads", "hidden"),
+    "o_proj": ("hidden", "o_heads"), "gate_proj": ("intermediate", "hidden"),
+    "up_proj": ("intermediate", "hidden"), "down_proj": ("hidden", "intermediate"),
+}
+
+
+@dataclass
+class LayerResult:
+    moments: Dict[str, torch.Tensor]
+    perms: Dict[str, Optional[torch.Tensor]]
+    scores: Dict[str, torch.Tensor]
+    err: torch.Tensor                 # [N, L] global table, matrices in shape.linears order
+    gain: Optional[torch.Tensor]
+    block_start: Dict[str, int]
+    n_blocks: int
+    level: Optional[torch.Tensor] = None
+    report: Optional[dict] = None
+    packed: Dict[str, tuple] = field(default_factory=dict)
+
+    def row_perm(self, name):
+        return self.perms[COUPLING[name][0]] if COUPLING[name][0] else None
+
+    def col_perm(self, name):
+        return self.perms[COUPLING[name][1]] if COUPLING[name][1] else None
+
+
+class LayerWorkspace:
+    """Device buffers for one layer, allocated once so a timed step allocates nothing."""
+
+    def __init__(self, shape: LayerShape, cfg: SearchConfig, device, keep_permuted: bool = True):
+        self.shape, self.cfg = shape, cfg
+        f32 = dict(dtype=torch.float32, device=device)
+        i32 = dict(dtype=torch.int32, device=device)
+        L = len(cfg.bits)
+        kv = shape.n_kv_heads * shape.head_dim
+        qd = shape.n_heads * shape.head_dim
+        self.moments = {n: torch.empty(k, **f32) for n, k in shape.act_dims.items()}
+        self.hid_score = torch.empty(shape.hidden, **f32)
+        self.mid_score = torch.empty(shape.intermediate, **f32)
+        self.vo_score = torch.empty(kv, **f32)
+        self.o_col_score = torch.empty(qd, **f32)
+        self.p_hid = torch.empty(shape.hidden, **i32)
+        self.p_mid = torch.empty(shape.intermediate, **i32)
+        self.p_v = torch.empty(kv, **i32)
+        self.p_o = torch.empty(qd, **i32)
+        self.block_start, n = {}, 0
+        for lin in shape.linears:
+            self.block_start[lin.name] = n
+            n += (lin.rows // cfg.block_rows) * (lin.cols // cfg.block_cols)
+        self.n_blocks = n
+        self.err = torch.empty((n, L), **f32)
+        self.gain = torch.empty((n, max(L - 1, 1)), **f32)   # [N, L-1] per-bit marginal gains
+        self.level = torch.empty(n, dtype=torch.uint8, device=device)
+        self.w_perm = ({lin.name: torch.empty((lin.rows, lin.cols), dtype=torch.bfloat16, device=device)
+                        for lin in shape.linears} if keep_permuted else None)
+        self.packed = {}
+        for lin in shape.linears:
+            nb = (lin.rows // cfg.block_rows) * (lin.cols // cfg.block_cols)
+            self.packed[lin.name] = (
+                torch.empty(lin.rows * lin.cols * max(cfg.bits) // 32, dtype=torch.int32, device=device),
+                torch.empty(nb + 1, dtype=torch.int64, device=device),
+                torch.empty((lin.rows * lin.cols // cfg.group, 2), **f32))
+
+
+def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str, torch.Tensor],
+                 ws: LayerWorkspace, allocate: bool = True, pack: bool = True) -> LayerResult:
+    """moments -> reorder statistics -> permutations -> block scores -> allocation -> pack."""
+    shape, cfg = ws.shape, ws.cfg
+    lin = {l.name: l for l in shape.linears}
+    g, rb = cfg.group, cfg.ref_bits
+    reps = shape.n_heads // shape.n_kv_heads
+    hd = shape.head_dim
+    W = weights
+
+    # a1: calibration second moments, one per distinct linear input
+    for name, X in acts.items():
+        ctx.calib_moments(X, ws.moments[name])
+    c = {n: ws.moments[l.act] for n, l in lin.items()}
+
+    perms = {"hidden": None, "intermediate": None, "v_heads": None, "o_heads": None}
+    if cfg.reorder:
+        # a2: reorder statistics, accumulated into the buffer of each coupled channel set
+        ctx.reorder_channels(W["q_proj"], c["q_proj"], rb, g, col_score=ws.hid_score)
+        ctx.reorder_channels(W["k_proj"], c["k_proj"], rb, g, col_score=ws.hid_score, accumulate_col=True)
+        ctx.reorder_channels(W["v_proj"], c["v_proj"], rb, g, row_score=ws.vo_score,
+                             col_score=ws.hid_score, accumulate_col=True)
+        ctx.reorder_channels(W["o_proj"], c["o_proj"], rb, g, row_score=ws.hid_score,
+                             col_score=ws.o_col_score, accumulate_row=True)
+        ctx.reorder_channels(W["gate_proj"], c["gate_proj"], rb, g, row_score=ws.mid_score,
+                             col_score=ws.hid_score, accumulate_col=True)
+        ctx.reorder_channels(W["up_proj"], c["up_proj"], rb, g, row_score=ws.mid_score,
+                             col_score=ws.hid_score, accumulate_row=True, accumulate_col=True)
+        ctx.reorder_channels(W["down_proj"], c["down_proj"], rb, g, row_score=ws.hid_score,
+                             col_score=ws.mid_score, accumulate_row=True, accumulate_col=True)
+        ctx.fold_segment_scores(ws.vo_score, ws.o_col_score, reps, hd)
+        # a3: one sort per coupled channel set ("sort only" calls: W = NULL)
+        ctx.reorder_channels(None, None, rb, g, row_score=ws.hid_score, row_segment=shape.hidden,
+                             row_perm=ws.p_hid, shape=(shape.hidden, g))
+        ctx.reorder_channels(None, None, rb, g, row_score=ws.mid_score, row_segment=shape.intermediate,
+                             row_perm=ws.p_mid, shape=(shape.intermediate, g))
+        ctx.reorder_channels(None, None, rb, g, row_score=ws.vo_score, row_segment=hd,
+                             row_perm=ws.p_v, shape=(ws.vo_score.numel(), g))
+        ctx.expand_segment_perm(ws.p_v, reps, hd, out=ws.p_o)
+        perms = {"hidden": ws.p_hid, "intermediate": ws.p_mid, "v_heads": ws.p_v, "o_heads": ws.p_o}
+
+    res = LayerResult(moments=ws.moments, perms=perms,
+                      scores={"hidden": ws.hid_score, "intermediate": ws.mid_score,
+                              "v_heads": ws.vo_score, "o_cols": ws.o_col_score},
+                      err=ws.err, gain=ws.gain if len(cfg.bits) > 1 else None,
+                      block_start=ws.block_start, n_blocks=ws.n_blocks)
+
+    # a4: block scores of every matrix into its rows of the global table
+    L = len(cfg.bits)
+    for name, l in lin.items():
+        nb = (l.rows // cfg.block_rows) * (l.cols // cfg.block_cols)
+        s = ws.block_start[name]
+        ctx.block_scores(W[name], c[name], cfg.bits, cfg.block_rows, cfg.block_cols, g,
+                         row_perm=res.row_perm(name), col_perm=res.col_perm(name),
+                         err=ws.err[s:s + nb], gain=ws.gain[s:s + nb] if L > 1 else None,
+                         want_gain=L > 1,
+                         W_perm_out=ws.w_perm[name] if ws.w_perm is not None else None)
+    if not allocate:
+        return res
+
+    # a5: one global allocation over all blocks of the layer
+    res.level, res.report = ctx.allocate_bits(
+        ws.err, cfg.bits, cfg.budget, cfg.mode, cfg.gamma0, cfg.gammaT,
+        uniform_block_elems=cfg.block_rows * cfg.block_cols, level=ws.level)
+    if not pack:
+        return res
+
+    # a6: pack every matrix at its blocks' levels (from the permuted copy when it was kept)
+    for name, l in lin.items():
+        nb = (l.rows // cfg.block_rows) * (l.cols // cfg.block_cols)
+        s = ws.block_start[name]
+        packed, off, meta = ws.packed[name]
+        if ws.w_perm is not None:
+            ctx.pack_blocks(ws.w_perm[name], cfg.bits, ws.level[s:s + nb], cfg.block_rows,
+                            cfg.block_cols, g, packed=packed, block_off=off, meta=meta)
+        else:
+            ctx.pack_blocks(W[name], cfg.bits, ws.level[s:s + nb], cfg.block_rows, cfg.block_cols, g,
+                            row_perm=res.row_perm(name), col_perm=res.col_perm(name),
+                            packed=packed, block_off=off, meta=meta)
+        res.packed[name] = (packed, off, meta)
+    return res

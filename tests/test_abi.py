@@ -1,0 +1,62 @@
+"""The C-ABI library builds, loads, and exports every symbol its header declares (no GPU)."""
+import ctypes
+import os
+import re
+
+import pytest
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(sb_[a-z0-9_]+)\s*\(", text))
+    return names
+
+
+def test_library_builds_and_exports_every_declared_symbol():
+    from paper_2602_17698_b200 import build, binding
+    path = build.build()
+    assert os.path.exists(path)
+    lib = ctypes.CDLL(path)
+    declared = _declared()
+    assert {"sb_calib_moments", "sb_reorder_channels", "sb_block_scores", "sb_allocate_bits",
+            "sb_pack_blocks"} <= declared
+    for name in declared:
+        assert hasattr(lib, name), f"{name} declared in include/ but not exported"
+    assert set(binding.EXPORTS) <= declared
+
+
+def test_binding_has_a_method_per_entry_point():
+    from paper_2602_17698_b200 import binding
+    for name in _declared():
+        short = name[3:]
+        if short in ("create", "destroy", "last_error"):
+            continue
+        assert hasattr(binding.Context, short), short
+
+
+@pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU failure mode")
+def test_no_cpu_fallback():
+    """Without a CUDA device the product path fails loudly instead of computing on the CPU."""
+    from paper_2602_17698_b200 import binding
+    with pytest.raises(RuntimeError):
+        binding.Context()
+    h = ctypes.c_void_p()
+    assert binding.lib().sb_create(ctypes.byref(h), 0, None) == binding.SB_ERR_CUDA
+    assert not h.value
+
+
+def test_product_code_never_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2602_17698_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for fn in files:
+            if fn.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, fn)).read()
+                assert not re.search(r"^\s*(from|import)\s+oracle\b", text, flags=re.M), fn
+                assert "libsbo" not in text and "scalebits_oracle" not in text, fn
