@@ -1,0 +1,335 @@
+#!/usr/bin/env python
+"""Benchmark of the bitwidth-search hot path on one Llama-3-8B-shaped decoder layer.
+
+One step = one pass of the whole path over one layer of synthetic input: calibration
+moments of the four linear inputs, reorder statistics + permutations, block scores of the
+seven matrices at every candidate bitwidth, global allocation, packing.  Prints ONE JSON
+line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "weight elements scored/s across all candidate bits"
+UNIT = "elements/s"
+TOKENS = 65536
+BITS = (2, 3, 4, 8)
+BUDGET = 2.5
+SEED = 0
+WORKLOAD = ("one Llama-3-8B-shaped decoder layer (q/o 4096x4096, k/v 1024x4096, gate/up 14336x4096, "
+            "down 4096x14336; 218,103,808 bf16 weights), 65536 calibration tokens per input, "
+            "blocks 128x128, group 128, bits {2,3,4,8}, budget 2.5")
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until a capture exists for that kernel)
+NCU_TRAFFIC_BYTES = {"moments_partial_kernel": None}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ---- clocks during the timed region ----------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.rows, self.proc, self.uuid = [], None, uuid
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.06)
+        self.proc.terminate()
+        inside = [r for (t, r) in self.rows if t0 <= t <= t1 + 0.05] or [r for (_, r) in self.rows]
+        sm, smax, reasons = [], None, set()
+        for r in inside:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax = float(f[2])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": smax,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---- the CPU oracle on a bounded sample (cpu_baseline leg and --impl reference) ---------------
+SAMPLE_DIV = 2   # the oracle is timed on 1/SAMPLE_DIV of the rows of every matrix and of the tokens
+SAMPLE_TEXT = ("first half of the rows of each of the 7 matrices (109,051,904 weights) and 32768 of the "
+               "65536 tokens of each of the 4 inputs, all five stages, per step")
+
+
+def oracle_sample_inputs():
+    """A row slice of every matrix of the layer and a token slice of every input (CPU tensors)."""
+    from paper_2602_17698_b200 import synth
+    shape = synth.LLAMA3_8B
+    W = {l.name: synth.make_weight(l.rows // SAMPLE_DIV, l.cols, synth.tensor_seed(SEED, 0, l.tensor_id))
+         for l in shape.linears}
+    X = {n: synth.make_activations(TOKENS // SAMPLE_DIV, k, synth.tensor_seed(SEED, 0, synth.ACT_TENSOR_ID[n]))
+         for n, k in shape.act_dims.items()}
+    return shape, W, X
+
+
+def oracle_step(shape, W, X):
+    """The oracle's five stages, as they stand, on the sample; returns weight elements scored."""
+    import numpy as np
+    from oracle import sbo
+    lin = {l.name: l for l in shape.linears}
+    mom = {n: sbo.calib_moments(x, 1.0 / x.shape[0]) for n, x in X.items()}
+    tables, n_elems = [], 0
+    for name, w in W.items():
+        c = mom[lin[name].act]
+        rs, cs = sbo.reorder_scores(w, c, ref_bits=2, group=128)
+        pr = sbo.argsort_desc_segments(rs)
+        pc = sbo.argsort_desc_segments(cs)
+        err, _ = sbo.block_scores(w, c, BITS, 128, 128, 128, row_perm=pr, col_perm=pc)
+        tables.append((name, pr, pc, err))
+        n_elems += w.shape[0] * w.shape[1]
+    table = np.concatenate([t[3] for t in tables])
+    st, level, rep = sbo.allocate_scalebits(table, BITS, BUDGET, 0.05, 0.02, 128 * 128)
+    assert st == sbo.OK
+    s = 0
+    for name, pr, pc, err in tables:
+        nb = err.shape[0]
+        sbo.pack_blocks(W[name], BITS, level[s:s + nb], 128, 128, 128, row_perm=pr, col_perm=pc)
+        s += nb
+    return n_elems
+
+
+def time_oracle(steps: int, warmup: int):
+    from oracle import sbo
+    sbo.build()
+    shape, W, X = oracle_sample_inputs()
+    for _ in range(warmup):
+        oracle_step(shape, W, X)
+    t0 = time.perf_counter()
+    n = 0
+    for _ in range(steps):
+        n += oracle_step(shape, W, X)
+    dt = time.perf_counter() - t0
+    return n / dt, dt / steps, sbo.num_threads(), SAMPLE_TEXT
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, min(args.steps, 3))
+    warm = 1 if args.warmup > 0 else 0
+    value, sec, cores, sample = time_oracle(steps, warm)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warm, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample_per_step": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---- the CUDA path ------------------------------------------------------------------------------
+STAGES = ("moments", "reorder_stats", "sort", "scores", "allocate", "pack")
+
+
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2602_17698_b200 import synth
+    from paper_2602_17698_b200.binding import Context
+    from paper_2602_17698_b200.pipeline import LayerWorkspace, SearchConfig, search_layer
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    shape = synth.LLAMA3_8B
+    cfg = SearchConfig(bits=BITS, budget=BUDGET)
+    # replicas: every rank searches its own layer (layer index = rank), no data-path collective
+    W = synth.make_layer_weights(shape, SEED, rank, dev)
+    X = synth.make_layer_activations(shape, TOKENS, SEED, rank, dev)
+    ctx = Context()
+    ws = LayerWorkspace(shape, cfg, dev)
+    n_weights = shape.n_weights
+    in_bytes = sum(w.numel() * 2 for w in W.values()) + sum(x.numel() * 2 for x in X.values())
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step(timers=None):
+        return search_layer(ctx, W, X, ws, timers=timers)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    sampler = None
+    if rank == 0:
+        sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(local).uuid))
+        sampler.start()
+        time.sleep(0.15)
+    timers = {s: [] for s in STAGES}
+    l0 = ctx.kernel_launches()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        res = step(timers)
+    e1.record()
+    barrier()
+    t_wall1 = time.time()
+    launches = ctx.kernel_launches() - l0
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+    tmax = torch.tensor([ms], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+    ms = float(tmax.item())
+    ms_per_step = ms / args.steps
+    value = world * n_weights / (ms_per_step * 1e-3)
+
+    stage_ms = {s: sum(a.elapsed_time(b) for a, b in timers[s]) / args.steps for s in STAGES}
+    stage_launch_ms = {s: (sum(a.elapsed_time(b) for a, b in timers[s]) / max(len(timers[s]), 1))
+                       for s in STAGES}
+
+    # ---- end to end: pinned host inputs -> device every step, result back to the host --------
+    e2e = None
+    if not args.no_e2e:
+        hW = {n: torch.empty(w.shape, dtype=w.dtype, pin_memory=True).copy_(w) for n, w in W.items()}
+        hX = {n: torch.empty(x.shape, dtype=x.dtype, pin_memory=True).copy_(x) for n, x in X.items()}
+        h_level = torch.empty(ws.n_blocks, dtype=torch.uint8, pin_memory=True)
+        h_packed = {n: tuple(torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in ws.packed[n])
+                    for n in ws.packed}
+        d2h = h_level.numel() + sum(t.numel() * t.element_size() for tup in h_packed.values() for t in tup)
+
+        def e2e_step():
+            for n in W:
+                W[n].copy_(hW[n], non_blocking=True)
+            for n in X:
+                X[n].copy_(hX[n], non_blocking=True)
+            r = step()
+            h_level.copy_(r.level, non_blocking=True)
+            for n, tup in r.packed.items():
+                for dst, src in zip(h_packed[n], tup):
+                    dst.copy_(src, non_blocking=True)
+            torch.cuda.synchronize()
+
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        e2e_step()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        b.record()
+        barrier()
+        t = torch.tensor([a.elapsed_time(b)], device=dev, dtype=torch.float64)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item()) / e2e_steps
+        e2e = {"value": world * n_weights / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+               "steps": e2e_steps, "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": d2h}
+
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        # dominant kernel by time: the calibration-moments reduction (3.49 GB read per step)
+        mom_bytes = sum(x.numel() * 2 for x in X.values())
+        mom_launches = len(X)
+        achieved = mom_bytes / (stage_ms["moments"] * 1e-3) / 1e9
+        traffic = NCU_TRAFFIC_BYTES["moments_partial_kernel"]
+        roofline = {"kernel": "moments_partial_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
+                    "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
+                    "traffic": traffic, "algorithmic_bytes_per_launch": mom_bytes / mom_launches,
+                    "launches_per_step": mom_launches, "avg_launch_ms": stage_ms["moments"] / mom_launches}
+        w_bytes = 2 * n_weights
+        stage_gbs = {"moments": achieved,
+                     "reorder_stats": w_bytes / (stage_ms["reorder_stats"] * 1e-3) / 1e9,
+                     "scores": w_bytes / (stage_ms["scores"] * 1e-3) / 1e9,
+                     "pack": w_bytes / (stage_ms["pack"] * 1e-3) / 1e9}
+        cpu = None
+        if not args.no_cpu_baseline:
+            v, sec, cores, sample = time_oracle(3, 0)
+            cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                   "seconds": sec}
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": WORKLOAD, "tokens": TOKENS, "bits": list(BITS), "budget": BUDGET,
+                           "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                           "l2": "inputs (3.9 GB per step) larger than L2, no flush needed",
+                           "allocation": res.report},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+                "roofline": roofline, "cpu_baseline": cpu,
+                "stages_ms_per_step": stage_ms, "stages_algorithmic_gbs": stage_gbs,
+                "scoring_elements_per_s": n_weights / (stage_ms["scores"] * 1e-3)}
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

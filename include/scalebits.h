@@ -107,7 +107,7 @@ sb_status sb_expand_segment_perm(sb_ctx* ctx, int32_t* out, const int32_t* perm,
  * col_moment / row_weight are indexed by ORIGINAL column / row.  All candidates are
  * evaluated from registers in one pass over W; fp32 arithmetic, fixed summation order.
  * bits: host array, strictly ascending, each in 1..8, 1 <= n_bits <= 8.
- * R % block_rows == 0, C % block_cols == 0, block_cols % group == 0, block_rows even,
+ * R % block_rows == 0, C % block_cols == 0, block_cols % group == 0, block_rows % 4 == 0,
  * block_cols in {32,64} or a multiple of 128.
  * err: fp32 [(R/br)*(C/bc)][n_bits]; gain: fp32 [..][n_bits-1] or NULL;
  * W_perm_out: bf16 [R][C] (ld = C) receives W' or NULL.                              */

@@ -22,7 +22,12 @@ LookbackBuf sb_lookback(sb_ctx* ctx, unsigned tiles, unsigned* epoch_out, sb_sta
 
 #ifdef __CUDACC__
 constexpr unsigned LB_AGG = 1u, LB_INC = 2u;
-constexpr int LB_SPIN_LIMIT = 1 << 22;
+constexpr unsigned long long LB_WAIT_NS = 250ull * 1000 * 1000;   // give up after 250 ms
+__device__ __forceinline__ unsigned long long lb_now_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
 
 __device__ __forceinline__ unsigned t_zero(unsigned*) { return 0u; }
 __device__ __forceinline__ unsigned long long t_zero(unsigned long long*) { return 0ull; }
@@ -64,12 +69,10 @@ __device__ __forceinline__ T block_exclusive_scan(T v, T& block_total) {
             T o = t_shfl_up(winc, d);
             if (lane >= d) winc = t_add(winc, o);
         }
-        if (lane < NT / 32) {
-            // exclusive prefix of the warp totals
-            T ex = t_shfl_up(winc, 1);
-            if (lane == 0) ex = t_zero((T*)nullptr);
-            warp_tot[lane] = ex;
-        }
+        // exclusive prefix of the warp totals (the shuffle is executed by the whole warp)
+        T wex = t_shfl_up(winc, 1);
+        if (lane == 0) wex = t_zero((T*)nullptr);
+        if (lane < NT / 32) warp_tot[lane] = wex;
         if (lane == NT / 32 - 1) total_sh = winc;
     }
     __syncthreads();
@@ -124,10 +127,16 @@ __device__ __forceinline__ T lookback_prefix(T aggregate, unsigned tile, Lookbac
                 T v = t_zero((T*)nullptr);
                 if (t >= 0) {
                     unsigned f = ld_acquire_u32(lb.flags + t);
+                    unsigned long long t_start = 0;
                     int spins = 0;
                     while ((f >> 2) != epoch || (f & 3u) == 0u) {
-                        if (++spins > LB_SPIN_LIMIT) { timed_out = true; break; }
-                        __nanosleep(32);
+                        // bounded wait: a predecessor that never publishes must not hang the GPU
+                        if ((++spins & 63) == 0) {
+                            const unsigned long long now = lb_now_ns();
+                            if (t_start == 0) t_start = now;
+                            else if (now - t_start > LB_WAIT_NS) { timed_out = true; break; }
+                        }
+                        __nanosleep(64);
                         f = ld_acquire_u32(lb.flags + t);
                     }
                     state = timed_out ? LB_INC : (f & 3u);

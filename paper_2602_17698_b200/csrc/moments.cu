@@ -80,7 +80,7 @@ __global__ void moments_finish_kernel(const float* __restrict__ partial, int spl
 extern "C" sb_status sb_calib_moments(sb_ctx* ctx, const void* X, int64_t T, int64_t K,
                                       int64_t ldx, float* sumsq, int accumulate, float scale) {
     if (!ctx) return SB_ERR_INVALID;
-    if (!X || !sumsq || T < 0 || K <= 0) return sb_fail(ctx, SB_ERR_INVALID, "moments: null or empty");
+    if ((!X && T > 0) || !sumsq || T < 0 || K <= 0) return sb_fail(ctx, SB_ERR_INVALID, "moments: null or empty");
     if (K % 8 || ldx % 8 || ldx < K || (reinterpret_cast<uintptr_t>(X) & 15))
         return sb_fail(ctx, SB_ERR_SHAPE, "moments: K, ldx must be multiples of 8 and X 16-byte aligned");
     SB_CUDA(ctx, cudaSetDevice(ctx->device));

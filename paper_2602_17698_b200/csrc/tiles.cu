@@ -160,10 +160,16 @@ block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
             for (int l = 0; l < L; ++l) {
                 const float inv = ba.qmax[l] * rinv;
                 const float nscale = live ? -(range * ba.inv_qmax[l]) : 0.f;
+                // With many levels q * scale carries the fp32 rounding of the step times q,
+                // a bias shared by the whole group: from 6 bits on the step is kept as a
+                // two-float sum (the residual range - scale * qmax is exact in one FMA).
+                const bool fine = ba.bits[l] >= 6;
+                const float nscale_lo = fine ? -(fmaf(nscale, ba.qmax[l], range) * ba.inv_qmax[l]) : 0.f;
 #pragma unroll
                 for (int k = 0; k < CPL; ++k) {
                     const float q = fmaf(vm[k], inv, RNE_MAGIC) - RNE_MAGIC;
-                    const float e = fmaf(q, nscale, vm[k]);
+                    float e = fmaf(q, nscale, vm[k]);
+                    if (fine) e = fmaf(q, nscale_lo, e);
                     if (ROWW) acc[k][l] = fmaf(e * ar, e, acc[k][l]);
                     else acc[k][l] = fmaf(e, e, acc[k][l]);
                 }
@@ -254,6 +260,7 @@ reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, 
         const bool live = range >= MIN_RANGE;
         const float inv = live ? qmax * rcp_approx(range) : 0.f;
         const float nscale = live ? -(range * inv_qmax) : 0.f;
+        const float nscale_lo = -(fmaf(nscale, qmax, range) * inv_qmax);   // two-float step
         float ar = 1.f;
         if (ROWW) ar = (r < R) ? row_weight[r] : 0.f;
         float rs = 0.f;
@@ -263,7 +270,7 @@ reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, 
             for (int h = 0; h < 2; ++h) {
                 const float vm = (h ? bf16hi(w[k]) : bf16lo(w[k])) - lo;
                 const float q = fmaf(vm, inv, RNE_MAGIC) - RNE_MAGIC;
-                const float e = fmaf(q, nscale, vm);
+                const float e = fmaf(q, nscale_lo, fmaf(q, nscale, vm));
                 const float e2 = ROWW ? e * e * ar : e * e;
                 acc[2 * k + h] += e2;
                 rs = fmaf(cw[2 * k + h], e2, rs);
@@ -493,7 +500,7 @@ sb_status sb_block_scores(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int6
     if (!ctx) return SB_ERR_INVALID;
     if (!W || !col_moment || !err || R <= 0 || C <= 0) return sb_fail(ctx, SB_ERR_INVALID, "scores: null or empty");
     if (!sb_check_bits(bits, n_bits)) return sb_fail(ctx, SB_ERR_INVALID, "scores: bits must be ascending in 1..8");
-    if (br <= 0 || bc <= 0 || R % br || C % bc || !valid_group(group) || bc % group ||
+    if (br <= 0 || bc <= 0 || br % 4 || R % br || C % bc || !valid_group(group) || bc % group ||
         !(bc == 32 || bc == 64 || bc % 128 == 0) || ldw % 8 || ldw < C ||
         (reinterpret_cast<uintptr_t>(W) & 15))
         return sb_fail(ctx, SB_ERR_SHAPE, "scores: block %dx%d group %d does not tile %lldx%lld", br, bc,

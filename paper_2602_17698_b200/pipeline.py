@@ -109,9 +109,32 @@ class LayerWorkspace:
                 torch.empty((lin.rows * lin.cols // cfg.group, 2), **f32))
 
 
+class _Timed:
+    """Brackets one library call with CUDA events on the current stream (None: no timing)."""
+
+    def __init__(self, timers, stage):
+        self.timers, self.stage = timers, stage
+
+    def __enter__(self):
+        if self.timers is not None:
+            self.a = torch.cuda.Event(enable_timing=True)
+            self.b = torch.cuda.Event(enable_timing=True)
+            self.a.record()
+
+    def __exit__(self, *exc):
+        if self.timers is not None:
+            self.b.record()
+            self.timers[self.stage].append((self.a, self.b))
+
+
 def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str, torch.Tensor],
-                 ws: LayerWorkspace, allocate: bool = True, pack: bool = True) -> LayerResult:
-    """moments -> reorder statistics -> permutations -> block scores -> allocation -> pack."""
+                 ws: LayerWorkspace, allocate: bool = True, pack: bool = True,
+                 timers: Optional[dict] = None) -> LayerResult:
+    """moments -> reorder statistics -> permutations -> block scores -> allocation -> pack.
+
+    `timers`, if given, maps the stage names moments / reorder_stats / sort / scores /
+    allocate / pack to lists that receive one (start, end) CUDA event pair per library call.
+    """
     shape, cfg = ws.shape, ws.cfg
     lin = {l.name: l for l in shape.linears}
     g, rb = cfg.group, cfg.ref_bits
@@ -121,33 +144,38 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
 
     # a1: calibration second moments, one per distinct linear input
     for name, X in acts.items():
-        ctx.calib_moments(X, ws.moments[name])
+        with _Timed(timers, "moments"):
+            ctx.calib_moments(X, ws.moments[name])
     c = {n: ws.moments[l.act] for n, l in lin.items()}
 
     perms = {"hidden": None, "intermediate": None, "v_heads": None, "o_heads": None}
     if cfg.reorder:
         # a2: reorder statistics, accumulated into the buffer of each coupled channel set
-        ctx.reorder_channels(W["q_proj"], c["q_proj"], rb, g, col_score=ws.hid_score)
-        ctx.reorder_channels(W["k_proj"], c["k_proj"], rb, g, col_score=ws.hid_score, accumulate_col=True)
-        ctx.reorder_channels(W["v_proj"], c["v_proj"], rb, g, row_score=ws.vo_score,
-                             col_score=ws.hid_score, accumulate_col=True)
-        ctx.reorder_channels(W["o_proj"], c["o_proj"], rb, g, row_score=ws.hid_score,
-                             col_score=ws.o_col_score, accumulate_row=True)
-        ctx.reorder_channels(W["gate_proj"], c["gate_proj"], rb, g, row_score=ws.mid_score,
-                             col_score=ws.hid_score, accumulate_col=True)
-        ctx.reorder_channels(W["up_proj"], c["up_proj"], rb, g, row_score=ws.mid_score,
-                             col_score=ws.hid_score, accumulate_row=True, accumulate_col=True)
-        ctx.reorder_channels(W["down_proj"], c["down_proj"], rb, g, row_score=ws.hid_score,
-                             col_score=ws.mid_score, accumulate_row=True, accumulate_col=True)
-        ctx.fold_segment_scores(ws.vo_score, ws.o_col_score, reps, hd)
+        stats = [
+            ("q_proj", dict(col_score=ws.hid_score)),
+            ("k_proj", dict(col_score=ws.hid_score, accumulate_col=True)),
+            ("v_proj", dict(row_score=ws.vo_score, col_score=ws.hid_score, accumulate_col=True)),
+            ("o_proj", dict(row_score=ws.hid_score, col_score=ws.o_col_score, accumulate_row=True)),
+            ("gate_proj", dict(row_score=ws.mid_score, col_score=ws.hid_score, accumulate_col=True)),
+            ("up_proj", dict(row_score=ws.mid_score, col_score=ws.hid_score, accumulate_row=True,
+                             accumulate_col=True)),
+            ("down_proj", dict(row_score=ws.hid_score, col_score=ws.mid_score, accumulate_row=True,
+                               accumulate_col=True)),
+        ]
+        for name, kw in stats:
+            with _Timed(timers, "reorder_stats"):
+                ctx.reorder_channels(W[name], c[name], rb, g, **kw)
         # a3: one sort per coupled channel set ("sort only" calls: W = NULL)
-        ctx.reorder_channels(None, None, rb, g, row_score=ws.hid_score, row_segment=shape.hidden,
-                             row_perm=ws.p_hid, shape=(shape.hidden, g))
-        ctx.reorder_channels(None, None, rb, g, row_score=ws.mid_score, row_segment=shape.intermediate,
-                             row_perm=ws.p_mid, shape=(shape.intermediate, g))
-        ctx.reorder_channels(None, None, rb, g, row_score=ws.vo_score, row_segment=hd,
-                             row_perm=ws.p_v, shape=(ws.vo_score.numel(), g))
-        ctx.expand_segment_perm(ws.p_v, reps, hd, out=ws.p_o)
+        with _Timed(timers, "sort"):
+            ctx.fold_segment_scores(ws.vo_score, ws.o_col_score, reps, hd)
+            ctx.reorder_channels(None, None, rb, g, row_score=ws.hid_score, row_segment=shape.hidden,
+                                 row_perm=ws.p_hid, shape=(shape.hidden, g))
+            ctx.reorder_channels(None, None, rb, g, row_score=ws.mid_score,
+                                 row_segment=shape.intermediate, row_perm=ws.p_mid,
+                                 shape=(shape.intermediate, g))
+            ctx.reorder_channels(None, None, rb, g, row_score=ws.vo_score, row_segment=hd,
+                                 row_perm=ws.p_v, shape=(ws.vo_score.numel(), g))
+            ctx.expand_segment_perm(ws.p_v, reps, hd, out=ws.p_o)
         perms = {"hidden": ws.p_hid, "intermediate": ws.p_mid, "v_heads": ws.p_v, "o_heads": ws.p_o}
 
     res = LayerResult(moments=ws.moments, perms=perms,
@@ -161,18 +189,20 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
     for name, l in lin.items():
         nb = (l.rows // cfg.block_rows) * (l.cols // cfg.block_cols)
         s = ws.block_start[name]
-        ctx.block_scores(W[name], c[name], cfg.bits, cfg.block_rows, cfg.block_cols, g,
-                         row_perm=res.row_perm(name), col_perm=res.col_perm(name),
-                         err=ws.err[s:s + nb], gain=ws.gain[s:s + nb] if L > 1 else None,
-                         want_gain=L > 1,
-                         W_perm_out=ws.w_perm[name] if ws.w_perm is not None else None)
+        with _Timed(timers, "scores"):
+            ctx.block_scores(W[name], c[name], cfg.bits, cfg.block_rows, cfg.block_cols, g,
+                             row_perm=res.row_perm(name), col_perm=res.col_perm(name),
+                             err=ws.err[s:s + nb], gain=ws.gain[s:s + nb] if L > 1 else None,
+                             want_gain=L > 1,
+                             W_perm_out=ws.w_perm[name] if ws.w_perm is not None else None)
     if not allocate:
         return res
 
     # a5: one global allocation over all blocks of the layer
-    res.level, res.report = ctx.allocate_bits(
-        ws.err, cfg.bits, cfg.budget, cfg.mode, cfg.gamma0, cfg.gammaT,
-        uniform_block_elems=cfg.block_rows * cfg.block_cols, level=ws.level)
+    with _Timed(timers, "allocate"):
+        res.level, res.report = ctx.allocate_bits(
+            ws.err, cfg.bits, cfg.budget, cfg.mode, cfg.gamma0, cfg.gammaT,
+            uniform_block_elems=cfg.block_rows * cfg.block_cols, level=ws.level)
     if not pack:
         return res
 
@@ -181,12 +211,13 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
         nb = (l.rows // cfg.block_rows) * (l.cols // cfg.block_cols)
         s = ws.block_start[name]
         packed, off, meta = ws.packed[name]
-        if ws.w_perm is not None:
-            ctx.pack_blocks(ws.w_perm[name], cfg.bits, ws.level[s:s + nb], cfg.block_rows,
-                            cfg.block_cols, g, packed=packed, block_off=off, meta=meta)
-        else:
-            ctx.pack_blocks(W[name], cfg.bits, ws.level[s:s + nb], cfg.block_rows, cfg.block_cols, g,
-                            row_perm=res.row_perm(name), col_perm=res.col_perm(name),
-                            packed=packed, block_off=off, meta=meta)
+        with _Timed(timers, "pack"):
+            if ws.w_perm is not None:
+                ctx.pack_blocks(ws.w_perm[name], cfg.bits, ws.level[s:s + nb], cfg.block_rows,
+                                cfg.block_cols, g, packed=packed, block_off=off, meta=meta)
+            else:
+                ctx.pack_blocks(W[name], cfg.bits, ws.level[s:s + nb], cfg.block_rows, cfg.block_cols,
+                                g, row_perm=res.row_perm(name), col_perm=res.col_perm(name),
+                                packed=packed, block_off=off, meta=meta)
         res.packed[name] = (packed, off, meta)
     return res

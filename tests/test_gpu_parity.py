@@ -202,9 +202,11 @@ def test_block_scores_degenerate_groups(ctx):
     err, _ = ctx.block_scores(W, c, bits, 64, 128, 128)
     ctx.sync()
     oerr, _ = sbo.block_scores(W.cpu(), np.ones(C), bits, 64, 128, 128)
-    assert_close(err.cpu().numpy(), oerr, REL, abs_floor=1e-12)
+    # on-grid data has zero error in exact arithmetic; fp32 leaves the rounding of the grid
+    # step: floor 1e-12 * sum W^2 of a block (~3e3 here)
+    assert_close(err.cpu().numpy(), oerr, REL, abs_floor=3e-9)
     assert torch.count_nonzero(err[:2]) == 0         # block row 0: constant groups
-    assert torch.count_nonzero(err[2:4, 0]) == 0     # block row 1 at 2 bits: on-grid
+    assert float(err[2:4].max()) < 3e-9              # block row 1: on the 2- and 4-bit grids
     Wz = torch.zeros_like(W)
     ez, _ = ctx.block_scores(Wz, c, bits, 64, 128, 128)
     ctx.sync()
