@@ -167,6 +167,28 @@ sb_status sb_pack_blocks(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_t C, 
                          uint32_t* packed, int64_t packed_capacity_words,
                          int64_t* block_off_words, float* meta);
 
+/* Allocation-free variant of sb_calib_moments (the paper has no counterpart: this entry
+ * point exists for deployment, not for the method).  It is for callers that cannot allocate
+ * device memory when they need the moments: a serving process whose device memory was
+ * handed out in full at start-up, code running under a framework's caching allocator where
+ * a raw cudaMalloc would synchronise the device and fragment the pool, a latency-critical
+ * loop.  It needs no context and calls no cudaMalloc / cudaFree or any allocating routine:
+ * its per-split partial sums live in a fixed 4 MiB array inside the library image, which
+ * every GPU that loads the library holds until the process exits.
+ *   - Same arithmetic, argument meaning and layout as sb_calib_moments; X, sumsq are DEVICE
+ *     pointers on the CURRENT device (the caller makes it current); cuda_stream is a
+ *     cudaStream_t (NULL = default stream).  Work is enqueued, not waited for.
+ *   - K <= 65536; larger K returns SB_ERR_SCRATCH (and says so on stderr): split the columns
+ *     across calls or use sb_calib_moments.  Other argument errors as in sb_calib_moments.
+ *   - The first call on each device looks up the array's device address; make that first
+ *     call before any stream capture begins.
+ *   - All calls share the array and it keeps the previous call's contents.  Every partial
+ *     that a call reads it has written first, so nothing needs clearing; but two calls whose
+ *     kernels overlap on the GPU (e.g. on different streams) race on it and must be ordered
+ *     by the caller.                                                                      */
+sb_status sb_calib_moments_noalloc(void* cuda_stream, const void* X_bf16, int64_t T, int64_t K,
+                                   int64_t ldx, float* sumsq, int accumulate, float scale);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,7 +22,8 @@ SB_ACC_ROW, SB_ACC_COL = 1, 2
 
 EXPORTS = ["sb_create", "sb_destroy", "sb_sync", "sb_last_error", "sb_kernel_launches",
            "sb_calib_moments", "sb_reorder_channels", "sb_fold_segment_scores",
-           "sb_expand_segment_perm", "sb_block_scores", "sb_allocate_bits", "sb_pack_blocks"]
+           "sb_expand_segment_perm", "sb_block_scores", "sb_allocate_bits", "sb_pack_blocks",
+           "sb_calib_moments_noalloc"]
 
 
 class SbError(RuntimeError):
@@ -233,3 +234,30 @@ class Context:
             block_rows, block_cols, group, barr, L, _ptr(level, torch.uint8), _ptr(packed),
             packed.numel(), _ptr(block_off, torch.int64), _ptr(meta, torch.float32)))
         return packed, block_off, meta
+
+
+def calib_moments_noalloc(X: torch.Tensor, sumsq: Optional[torch.Tensor] = None,
+                          accumulate: bool = False, scale: Optional[float] = None,
+                          stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """sb_calib_moments_noalloc: second moments without a context and without any device
+    allocation inside the library (fixed in-library scratch, K <= 65536).
+
+    For callers that cannot allocate when they need the moments (device memory fully handed
+    out at start-up, code under a caching allocator, latency-critical loops).  X's device
+    must be current.  Calls share the scratch: do not let two of them overlap on the GPU.
+    """
+    T, K, ldx = _mat(X)
+    if sumsq is None:
+        sumsq = torch.empty(K, dtype=torch.float32, device=X.device)
+        accumulate = False
+    if scale is None:
+        scale = 1.0 / max(T, 1)
+    s = torch.cuda.current_stream(X.device) if stream is None else stream
+    fn = lib().sb_calib_moments_noalloc
+    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_int, C.c_float]
+    fn.restype = C.c_int
+    st = fn(C.c_void_p(s.cuda_stream), _ptr(X), T, K, ldx, _ptr(sumsq, torch.float32),
+            int(accumulate), float(scale))
+    if st != SB_OK:
+        raise SbError(st, "sb_calib_moments_noalloc failed (see stderr)")
+    return sumsq

@@ -1,0 +1,178 @@
+// sb_calib_moments_noalloc: the calibration second moments for callers that must not
+// allocate device memory.
+//
+// Who needs it: code that runs where cudaMalloc is off limits -- a serving loop whose device
+// memory was handed out in full at start-up (another pool owns every byte, so an allocation
+// fails or evicts someone), a section managed by a framework's caching allocator where a raw
+// cudaMalloc would synchronise the device and fragment the pool, or a latency-critical path
+// that cannot afford the implicit synchronisation of an allocation.  The regular entry point
+// keeps its per-split partial sums in a context-owned arena that grows with cudaMalloc; this
+// one keeps them in a fixed array that is part of the library image instead.
+//
+// The array costs SB_NOALLOC_SCRATCH_FLOATS * 4 bytes (4 MiB) on EVERY GPU that loads the
+// library, for the life of the process.  All calls share it and it keeps whatever the last
+// call left there; the kernels overwrite every partial they later read, so nothing has to
+// start at zero, but two calls whose kernels overlap on the GPU (for instance on different
+// streams) race on it.
+//
+// The first call on each device looks up the array's device address (no allocation); make
+// that first call before any stream capture begins.
+#include <mutex>
+
+#include "common.cuh"
+
+#define SB_NOALLOC_SCRATCH_FLOATS (1 << 20)
+#define SB_NOALLOC_MAX_K 65536
+
+static __device__ __align__(256) float sb_noalloc_scratch[SB_NOALLOC_SCRATCH_FLOATS];
+
+namespace {
+
+constexpr int NA_TX = 32, NA_TY = 8, NA_COLS = NA_TX * 8, NA_UNROLL = 8;
+
+// grid.x = chunks of 256 columns, grid.y = row splits; partial[split][K]
+__global__ void __launch_bounds__(NA_TX * NA_TY)
+noalloc_partial_kernel(const __nv_bfloat16* __restrict__ X, int64_t T, int64_t K, int64_t ldx,
+                       int64_t rows_per_split, float* __restrict__ partial) {
+    const int tx = threadIdx.x, ty = threadIdx.y;
+    const int64_t col = (int64_t)blockIdx.x * NA_COLS + tx * 8;
+    const int64_t t0 = (int64_t)blockIdx.y * rows_per_split;
+    const int64_t t1 = min(T, t0 + rows_per_split);
+    float acc[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+    if (col < K) {
+        const __nv_bfloat16* base = X + col;
+        int64_t t = t0 + ty;
+        for (; t + (NA_UNROLL - 1) * NA_TY < t1; t += NA_UNROLL * NA_TY) {
+            uint4 v[NA_UNROLL];
+#pragma unroll
+            for (int u = 0; u < NA_UNROLL; ++u) v[u] = ld_stream16(base + (t + u * NA_TY) * ldx);
+#pragma unroll
+            for (int u = 0; u < NA_UNROLL; ++u) {
+                const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float a = bf16lo(w[k]), b = bf16hi(w[k]);
+                    acc[2 * k] = fmaf(a, a, acc[2 * k]);
+                    acc[2 * k + 1] = fmaf(b, b, acc[2 * k + 1]);
+                }
+            }
+        }
+        for (; t < t1; t += NA_TY) {
+            const uint4 v = ld_stream16(base + t * ldx);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float a = bf16lo(w[k]), b = bf16hi(w[k]);
+                acc[2 * k] = fmaf(a, a, acc[2 * k]);
+                acc[2 * k + 1] = fmaf(b, b, acc[2 * k + 1]);
+            }
+        }
+    }
+    __shared__ float red[NA_TY][NA_COLS + 8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) red[ty][tx * 8 + k] = acc[k];
+    __syncthreads();
+    const int c = ty * NA_TX + tx;
+    const int64_t gc = (int64_t)blockIdx.x * NA_COLS + c;
+    if (gc < K) {
+        float s = 0.f;
+#pragma unroll
+        for (int y = 0; y < NA_TY; ++y) s += red[y][c];
+        partial[(int64_t)blockIdx.y * K + gc] = s;      // every (split, column) is written
+    }
+}
+
+__global__ void noalloc_finish_kernel(const float* __restrict__ partial, int splits, int64_t K,
+                                      float scale, int accumulate, float* __restrict__ out) {
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= K) return;
+    float s = 0.f;
+    for (int p = 0; p < splits; ++p) s += partial[(int64_t)p * K + j];
+    s *= scale;
+    out[j] = accumulate ? out[j] + s : s;
+}
+
+// In host code `sb_noalloc_scratch` is only a stand-in for the symbol, not a device address:
+// the address the kernels can use comes from cudaGetSymbolAddress, looked up once per device
+// with that device current.
+std::mutex g_mu;
+float* g_scratch_ptr[64] = {nullptr};
+int g_sm_count[64] = {0};
+
+sb_status scratch_for_current_device(float** out, int* sm_count) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        (void)cudaGetLastError();
+        fprintf(stderr, "sb_calib_moments_noalloc: no current CUDA device\n");
+        return SB_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_scratch_ptr[dev]) {
+        float* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), sb_noalloc_scratch);
+        if (e != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            fprintf(stderr, "sb_calib_moments_noalloc: cudaGetSymbolAddress failed: %s\n",
+                    cudaGetErrorString(e));
+            return SB_ERR_CUDA;
+        }
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            sms = 148;
+        g_sm_count[dev] = sms;
+        g_scratch_ptr[dev] = p;
+    }
+    *out = g_scratch_ptr[dev];
+    *sm_count = g_sm_count[dev];
+    return SB_OK;
+}
+
+}  // namespace
+
+extern "C" sb_status sb_calib_moments_noalloc(void* cuda_stream, const void* X, int64_t T, int64_t K,
+                                              int64_t ldx, float* sumsq, int accumulate, float scale) {
+    if ((!X && T > 0) || !sumsq || T < 0 || K <= 0) {
+        fprintf(stderr, "sb_calib_moments_noalloc: null or empty argument\n");
+        return SB_ERR_INVALID;
+    }
+    if (K % 8 || ldx % 8 || ldx < K || (reinterpret_cast<uintptr_t>(X) & 15)) {
+        fprintf(stderr, "sb_calib_moments_noalloc: K and ldx must be multiples of 8, X 16-byte aligned\n");
+        return SB_ERR_SHAPE;
+    }
+    if (K > SB_NOALLOC_MAX_K) {
+        fprintf(stderr, "sb_calib_moments_noalloc: K = %lld exceeds the fixed scratch (at most %d "
+                        "channels per call; split the columns or use sb_calib_moments)\n",
+                (long long)K, SB_NOALLOC_MAX_K);
+        return SB_ERR_SCRATCH;
+    }
+    float* partial = nullptr;
+    int sms = 148;
+    sb_status st = scratch_for_current_device(&partial, &sms);
+    if (st != SB_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int col_chunks = (int)((K + NA_COLS - 1) / NA_COLS);
+    const int64_t min_rows = NA_TY * NA_UNROLL;
+    int splits = (sms * 8 + col_chunks - 1) / col_chunks;
+    const int max_splits = (int)(SB_NOALLOC_SCRATCH_FLOATS / K);       // >= 16 by the K limit
+    if (splits > max_splits) splits = max_splits;
+    if ((int64_t)splits * min_rows > T) splits = (int)((T + min_rows - 1) / min_rows);
+    if (splits < 1) splits = 1;
+    int64_t rows_per_split = (T + splits - 1) / splits;
+    rows_per_split = (rows_per_split + min_rows - 1) / min_rows * min_rows;
+    if (rows_per_split < min_rows) rows_per_split = min_rows;
+    splits = (int)((T + rows_per_split - 1) / rows_per_split);
+    if (splits < 1) splits = 1;
+    dim3 grid(col_chunks, splits), block(NA_TX, NA_TY);
+    noalloc_partial_kernel<<<grid, block, 0, stream>>>(static_cast<const __nv_bfloat16*>(X), T, K, ldx,
+                                                       rows_per_split, partial);
+    noalloc_finish_kernel<<<(unsigned)((K + 255) / 256), 256, 0, stream>>>(partial, splits, K, scale,
+                                                                           accumulate, sumsq);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        fprintf(stderr, "sb_calib_moments_noalloc: launch failed: %s\n", cudaGetErrorString(e));
+        return SB_ERR_CUDA;
+    }
+    return SB_OK;
+}
