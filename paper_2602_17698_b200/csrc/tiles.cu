@@ -17,9 +17,11 @@ constexpr int CTA_WARPS = CTA_THREADS / 32;
 constexpr float RNE_MAGIC = 12582912.f;        // 1.5 * 2^23: fma(x, s, MAGIC) - MAGIC = rint(x*s)
 constexpr float MIN_RANGE = 7.52316385e-37f;   // 2^-120: below this a group counts as constant
 
-struct BitsArg {
-    float qmax[8];       // 2^b - 1
-    float inv_qmax[8];   // 1 / (2^b - 1)
+struct __align__(8) BitsArg {
+    float2 q2[8];        // (qmax, qmax), qmax = 2^b - 1, as a packed fp32 pair
+    float2 niq2[8];      // (-1/qmax, -1/qmax)
+    float qmax[8];
+    float inv_qmax[8];
     int bits[8];
 };
 
@@ -29,7 +31,7 @@ __device__ __forceinline__ __nv_bfloat162 b162(uint32_t v) { return *reinterpret
 // min and max of a group: NW packed words per lane, `team` lanes (a power of two, aligned)
 // per group.  Exact: bf16 min/max, the pair (min, -max) rides one register through the
 // shuffles.
-template <int NW>
+template <int NW, int TEAM = 0>
 __device__ __forceinline__ void group_minmax(const uint32_t (&w)[NW], int team, float& lo, float& hi) {
     __nv_bfloat162 mn = b162(w[0]), mx = mn;
 #pragma unroll
@@ -41,8 +43,14 @@ __device__ __forceinline__ void group_minmax(const uint32_t (&w)[NW], int team, 
     const uint32_t a = u32(__hmin2(mn, b162(__byte_perm(mnu, mnu, 0x1032))));
     const uint32_t b = u32(__hmax2(mx, b162(__byte_perm(mxu, mxu, 0x1032)))) ^ 0x80008000u;
     uint32_t p = (a & 0x0000ffffu) | (b & 0xffff0000u);
-    for (int o = team >> 1; o > 0; o >>= 1)
-        p = u32(__hmin2(b162(p), b162(__shfl_xor_sync(0xffffffffu, p, o))));
+    if (TEAM > 0) {
+#pragma unroll
+        for (int o = TEAM >> 1; o > 0; o >>= 1)
+            p = u32(__hmin2(b162(p), b162(__shfl_xor_sync(0xffffffffu, p, o))));
+    } else {
+        for (int o = team >> 1; o > 0; o >>= 1)
+            p = u32(__hmin2(b162(p), b162(__shfl_xor_sync(0xffffffffu, p, o))));
+    }
     lo = bf16lo(p);
     hi = -bf16hi(p);
 }
@@ -101,129 +109,256 @@ __device__ __forceinline__ void load_cols(const __nv_bfloat16* p, bool ok, uint3
     }
 }
 
+// ---- packed fp32 pairs --------------------------------------------------------------------
+// sm_100a executes fma / add / mul on two fp32 values held in one 64-bit register.  The FP32
+// pipe does the same number of lane-operations per clock either way, but the packed form needs
+// half the issue slots, which leaves room for the integer, shuffle and load instructions.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pk2(float a, float b) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void upk2(f32x2 v, float& a, float& b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// ---- asynchronous 16-byte copies global -> shared (L2 only, no register staging) -----------
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 // ---- block scores ------------------------------------------------------------------------
-// CTA = 8 warps.  A lane owns CPL consecutive columns of a 128-column chunk; 128/CPL lanes
-// cover a row of the chunk and a warp covers 32*CPL/128 rows per step.  grid.x = column
-// tiles (one block when block_cols >= 128, else 128/block_cols blocks side by side),
-// grid.y = block rows.
-template <int L, int CPL, bool ROWW>
-__global__ void __launch_bounds__(CTA_THREADS)
+// Every WARP is autonomous: it walks its own units (a block, or a 32-row part of one), stages
+// its own 16-row slabs of the 128-column chunk in its own shared-memory ring with asynchronous
+// 16-byte copies (two slabs per warp, 64 KB in flight per SM), and synchronises with nobody
+// but itself.  Without CTA barriers the warps of an SM drift apart, so the integer/shuffle
+// phase of one warp (group min/max, unpacking) overlaps the FP32 phase of another.  A lane
+// owns CPL consecutive columns of the chunk; 128/CPL lanes cover a row, a warp covers
+// 32*CPL/128 rows per step.  The 16-byte pieces of a row are laid out in shared memory so
+// that a quarter-warp reads 128 contiguous bytes (no bank conflicts).  Everything inside the
+// candidate loop is packed fp32 pairs (fma/add/mul.f32x2), including the per-group constants,
+// which come from packed pairs in the kernel parameters.  Each unit writes its partial block
+// errors; a second tiny kernel adds the parts of a block in a fixed order.
+//
+// NFINE = how many of the L candidates (the last ones: bits ascend) keep the grid step as a
+// two-float sum: with many levels q * scale carries the fp32 rounding of the step times q, a
+// bias shared by the whole group; the residual range - scale * qmax is exact in one FMA.
+// A row weight a_r enters as sqrt(a_r) on (v - lo), on the range and, inverted, on the
+// reciprocal, so that the accumulated square carries a_r without any per-candidate work.
+constexpr int SLAB_ROWS = 16;
+constexpr int SLAB_BYTES = SLAB_ROWS * 256;
+
+template <int L, int CPL, int NFINE, bool FULLG, bool ROWW>
+__global__ void __launch_bounds__(CTA_THREADS, 2)
 block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
                     const int32_t* __restrict__ load_row_perm,   // rows gathered at load time
                     const int32_t* __restrict__ c_perm,          // original column of permuted j
                     const int32_t* __restrict__ a_perm,          // original row of permuted r
                     const float* __restrict__ col_moment, const float* __restrict__ row_weight,
                     int br, int bc, int group, BitsArg ba, int64_t n_block_cols,
-                    float* __restrict__ err, float* __restrict__ gain, SbDeviceState* dstate) {
+                    int64_t n_tile_cols, int parts, int part_rows, int64_t n_units, int64_t n_blocks,
+                    float* __restrict__ part_out) {
     constexpr int LANE_COLS = TILE_COLS / CPL;      // lanes across a chunk row
     constexpr int ROW_SLOTS = 32 / LANE_COLS;       // rows per warp step
     constexpr int NW = CPL / 2;
+    constexpr int PIECES = CPL / 8;                 // 16-byte pieces per lane and row
+    extern __shared__ __align__(16) unsigned char tile_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int cl = lane % LANE_COLS, slot = lane / LANE_COLS;
     const int team = group / CPL > 0 ? group / CPL : 1;
     const int chunks = bc >= TILE_COLS ? bc / TILE_COLS : 1;
     const int tile_w = bc >= TILE_COLS ? bc : TILE_COLS;
-    const int64_t row0 = (int64_t)blockIdx.y * br;
-    const int64_t colT = (int64_t)blockIdx.x * tile_w;
-
-    float tot[L];
-#pragma unroll
-    for (int l = 0; l < L; ++l) tot[l] = 0.f;
-
-    for (int ch = 0; ch < chunks; ++ch) {
-        const int64_t col = colT + (int64_t)ch * TILE_COLS + cl * CPL;
-        float acc[CPL][L];
-#pragma unroll
-        for (int k = 0; k < CPL; ++k)
-#pragma unroll
-            for (int l = 0; l < L; ++l) acc[k][l] = 0.f;
-
-        for (int rr = warp * ROW_SLOTS + slot; rr < br; rr += CTA_WARPS * ROW_SLOTS) {
-            const int64_t r = row0 + rr;
-            const int64_t rs = load_row_perm ? load_row_perm[r] : r;
-            uint32_t w[NW];
-            load_cols<CPL>(W + rs * ldw + col, true, w);
-            float lo, hi;
-            group_minmax<NW>(w, team, lo, hi);
-            const float range = hi - lo;
-            const bool live = range >= MIN_RANGE;
-            const float rinv = live ? rcp_approx(range) : 0.f;
-            float ar = 1.f;
-            if (ROWW) ar = row_weight[a_perm ? a_perm[r] : r];
-            float vm[CPL];
-#pragma unroll
-            for (int k = 0; k < NW; ++k) {
-                vm[2 * k] = bf16lo(w[k]) - lo;
-                vm[2 * k + 1] = bf16hi(w[k]) - lo;
-            }
-#pragma unroll
-            for (int l = 0; l < L; ++l) {
-                const float inv = ba.qmax[l] * rinv;
-                const float nscale = live ? -(range * ba.inv_qmax[l]) : 0.f;
-                // With many levels q * scale carries the fp32 rounding of the step times q,
-                // a bias shared by the whole group: from 6 bits on the step is kept as a
-                // two-float sum (the residual range - scale * qmax is exact in one FMA).
-                const bool fine = ba.bits[l] >= 6;
-                const float nscale_lo = fine ? -(fmaf(nscale, ba.qmax[l], range) * ba.inv_qmax[l]) : 0.f;
-#pragma unroll
-                for (int k = 0; k < CPL; ++k) {
-                    const float q = fmaf(vm[k], inv, RNE_MAGIC) - RNE_MAGIC;
-                    float e = fmaf(q, nscale, vm[k]);
-                    if (fine) e = fmaf(q, nscale_lo, e);
-                    if (ROWW) acc[k][l] = fmaf(e * ar, e, acc[k][l]);
-                    else acc[k][l] = fmaf(e, e, acc[k][l]);
-                }
-            }
-        }
-        // column factors once per chunk
-#pragma unroll
-        for (int k = 0; k < CPL; ++k) {
-            const int64_t j = col + k;
-            const float cw = col_moment[c_perm ? c_perm[j] : j];
-#pragma unroll
-            for (int l = 0; l < L; ++l) tot[l] = fmaf(cw, acc[k][l], tot[l]);
-        }
-    }
-
-    // reduce: lanes of the same block (sub-block when bc < 128), then warps, fixed order
+    const f32x2 magic2 = pk2(RNE_MAGIC, RNE_MAGIC), nmagic2 = pk2(-RNE_MAGIC, -RNE_MAGIC);
     const int lanes_per_sub = bc >= TILE_COLS ? LANE_COLS : bc / CPL;    // lanes across one block
     const int nsub = bc >= TILE_COLS ? 1 : TILE_COLS / bc;
+    const int slabs = (part_rows + SLAB_ROWS - 1) / SLAB_ROWS;           // per chunk of a unit
+    unsigned char* ring = tile_smem + (size_t)warp * (2 * SLAB_BYTES);
+    // this lane's share of a slab: 16-byte piece g of rows g_row, g_row + 2, ...
+    const int g = lane & 15, g_row = lane >> 4;
+    const int g_dst = g_row * 256 + (g % PIECES) * (LANE_COLS * 16) + (g / PIECES) * 16;
+    const int my_off = slot * 256 + cl * 16;
+    const int64_t warp_id = (int64_t)blockIdx.x * CTA_WARPS + warp;
+    const int64_t warp_stride = (int64_t)gridDim.x * CTA_WARPS;
+
+    // stage slab `sl` of chunk `ch` of unit `u` (rows beyond the part are skipped)
+    auto issue = [&](int64_t u, int ch, int sl, int stage) {
+        const int64_t t = u / parts;
+        const int64_t row0 = t / n_tile_cols * br + (int64_t)(u % parts) * part_rows + sl * SLAB_ROWS;
+        const int rows_here = min(SLAB_ROWS, part_rows - sl * SLAB_ROWS);
+        const __nv_bfloat16* src = W + t % n_tile_cols * tile_w + (int64_t)ch * TILE_COLS + g * 8;
+        unsigned char* dst = ring + stage * SLAB_BYTES + g_dst;
+        if (load_row_perm) {
+            const int32_t* rp = load_row_perm + row0;
+            for (int row = g_row; row < rows_here; row += 2, dst += 2 * 256)
+                cp_async16(dst, src + (int64_t)rp[row] * ldw);
+        } else {
+            src += (row0 + g_row) * ldw;
+            for (int row = g_row; row < rows_here; row += 2, dst += 2 * 256, src += 2 * ldw)
+                cp_async16(dst, src);
+        }
+        cp_async_commit();
+    };
+
+    int stage = 0;
+    int64_t unit = warp_id;
+    if (unit < n_units) issue(unit, 0, 0, 0);
+    for (; unit < n_units; unit += warp_stride) {
+        const int64_t t = unit / parts;
+        const int p = (int)(unit % parts);
+        const int64_t row_base = t / n_tile_cols * br + (int64_t)p * part_rows;
+        const int64_t colT = t % n_tile_cols * tile_w;
+        f32x2 tot2[L];
 #pragma unroll
-    for (int l = 0; l < L; ++l) {
-        float v = tot[l];
-        for (int o = lanes_per_sub >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        for (int o = LANE_COLS; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        tot[l] = v;
-    }
-    __shared__ float red[CTA_WARPS][4][8];
-    if (slot == 0 && (cl % lanes_per_sub) == 0) {
-        const int sb = cl / lanes_per_sub;
+        for (int l = 0; l < L; ++l) tot2[l] = 0ull;
+
+        for (int ch = 0; ch < chunks; ++ch) {
+            f32x2 acc[NW][L];
 #pragma unroll
-        for (int l = 0; l < L; ++l) red[warp][sb][l] = tot[l];
-    }
-    __syncthreads();
-    if (threadIdx.x < nsub) {
-        const int sb = threadIdx.x;
-        const int64_t blk = (int64_t)blockIdx.y * n_block_cols + (int64_t)blockIdx.x * nsub + sb;
-        float e[L];
-        bool finite = true;
+            for (int k = 0; k < NW; ++k)
+#pragma unroll
+                for (int l = 0; l < L; ++l) acc[k][l] = 0ull;
+
+            for (int sl = 0; sl < slabs; ++sl, stage ^= 1) {
+                // keep the next slab in flight, then wait for this one
+                if (sl + 1 < slabs) issue(unit, ch, sl + 1, stage ^ 1);
+                else if (ch + 1 < chunks) issue(unit, ch + 1, 0, stage ^ 1);
+                else if (unit + warp_stride < n_units) issue(unit + warp_stride, 0, 0, stage ^ 1);
+                else cp_async_commit();
+                cp_async_wait<1>();
+                __syncwarp();
+                const unsigned char* src = ring + stage * SLAB_BYTES + my_off;
+                const int rows_here = min(SLAB_ROWS, part_rows - sl * SLAB_ROWS);
+#pragma unroll 1
+                for (int rr = slot; rr < rows_here; rr += ROW_SLOTS, src += ROW_SLOTS * 256) {
+                    uint32_t w[NW];
+#pragma unroll
+                    for (int h = 0; h < PIECES; ++h) {
+                        const uint4 x = *reinterpret_cast<const uint4*>(src + h * (LANE_COLS * 16));
+                        w[4 * h] = x.x; w[4 * h + 1] = x.y; w[4 * h + 2] = x.z; w[4 * h + 3] = x.w;
+                    }
+                    float lo, hi;
+                    group_minmax<NW, FULLG ? LANE_COLS : 0>(w, team, lo, hi);
+                    float range = hi - lo;
+                    const bool live = range >= MIN_RANGE;
+                    float rinv = rcp_approx(range);
+                    float sa = 1.f;
+                    if (ROWW) {
+                        const int64_t r = row_base + sl * SLAB_ROWS + rr;
+                        const float a = row_weight[a_perm ? a_perm[r] : r];
+                        sa = sqrtf(a);
+                        rinv = a > 0.f ? rinv * rcp_approx(sa) : 0.f;
+                        range *= sa;
+                    }
+                    if (!live) { rinv = 0.f; range = 0.f; }
+                    const f32x2 rinv2 = pk2(rinv, rinv), range2 = pk2(range, range);
+                    const f32x2 nlo2 = pk2(-lo, -lo);
+                    f32x2 vm[NW];
+#pragma unroll
+                    for (int k = 0; k < NW; ++k) vm[k] = add2(pk2(bf16lo(w[k]), bf16hi(w[k])), nlo2);
+                    if (ROWW) {
+                        const f32x2 sa2 = pk2(sa, sa);
+#pragma unroll
+                        for (int k = 0; k < NW; ++k) vm[k] = mul2(vm[k], sa2);
+                    }
+#pragma unroll
+                    for (int l = 0; l < L; ++l) {
+                        const f32x2 q2 = *reinterpret_cast<const f32x2*>(&ba.q2[l]);
+                        const f32x2 niq2 = *reinterpret_cast<const f32x2*>(&ba.niq2[l]);
+                        const f32x2 inv2 = mul2(q2, rinv2);
+                        const f32x2 ns2 = mul2(niq2, range2);                   // -(range / qmax)
+                        if (l >= L - NFINE) {
+                            const f32x2 nslo2 = mul2(fma2(ns2, q2, range2), niq2);   // -(residual / qmax)
+#pragma unroll
+                            for (int k = 0; k < NW; ++k) {
+                                const f32x2 qq = add2(fma2(vm[k], inv2, magic2), nmagic2);
+                                const f32x2 e = fma2(qq, nslo2, fma2(qq, ns2, vm[k]));
+                                acc[k][l] = fma2(e, e, acc[k][l]);
+                            }
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < NW; ++k) {
+                                const f32x2 qq = add2(fma2(vm[k], inv2, magic2), nmagic2);
+                                const f32x2 e = fma2(qq, ns2, vm[k]);
+                                acc[k][l] = fma2(e, e, acc[k][l]);
+                            }
+                        }
+                    }
+                }
+                __syncwarp();             // the slab is consumed before its stage is refilled
+            }
+            // column factors once per chunk of the unit
+            const int64_t col = colT + (int64_t)ch * TILE_COLS + cl * CPL;
+#pragma unroll
+            for (int k = 0; k < NW; ++k) {
+                const int64_t j = col + 2 * k;
+                const f32x2 c2 = pk2(__ldg(col_moment + (c_perm ? c_perm[j] : j)),
+                                     __ldg(col_moment + (c_perm ? c_perm[j + 1] : j + 1)));
+#pragma unroll
+                for (int l = 0; l < L; ++l) tot2[l] = fma2(c2, acc[k][l], tot2[l]);
+            }
+        }
+
+        // lanes of the same block (sub-block when bc < 128), fixed order
+        float tot[L];
 #pragma unroll
         for (int l = 0; l < L; ++l) {
-            float s = 0.f;
-#pragma unroll
-            for (int wv = 0; wv < CTA_WARPS; ++wv) s += red[wv][sb][l];
-            e[l] = s;
-            err[blk * L + l] = s;
-            finite = finite && isfinite(s);
+            float a0, a1;
+            upk2(tot2[l], a0, a1);
+            float v = a0 + a1;
+            for (int o = lanes_per_sub >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            for (int o = LANE_COLS; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            tot[l] = v;
         }
-        if (!finite) sb_latch(dstate, SB_ERR_NONFINITE, SBK_SCORES);
-        if (gain) {
-            const float M = (float)br * (float)bc;
+        if (slot == 0 && (cl % lanes_per_sub) == 0) {
+            const int sb = cl / lanes_per_sub;
+            const int64_t blk = t / n_tile_cols * n_block_cols + t % n_tile_cols * nsub + sb;
+            float* dst = part_out + ((int64_t)p * n_blocks + blk) * L;
 #pragma unroll
-            for (int l = 0; l + 1 < L; ++l)
-                gain[blk * (L - 1) + l] = (e[l] - e[l + 1]) / ((float)(ba.bits[l + 1] - ba.bits[l]) * M);
+            for (int l = 0; l < L; ++l) dst[l] = tot[l];
         }
     }
+    cp_async_wait<0>();
+}
+
+// err[blk][l] = sum over the row parts of a block, in order; gains; non-finite check
+__global__ void scores_finish_kernel(const float* __restrict__ part, int parts, int64_t n_blocks, int L,
+                                     BitsArg ba, float M, float* __restrict__ err,
+                                     float* __restrict__ gain, SbDeviceState* dstate) {
+    const int64_t blk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (blk >= n_blocks) return;
+    float e[8];
+    bool finite = true;
+    for (int l = 0; l < L; ++l) {
+        float s = 0.f;
+        for (int p = 0; p < parts; ++p) s += part[((int64_t)p * n_blocks + blk) * L + l];
+        e[l] = s;
+        err[blk * L + l] = s;
+        finite = finite && isfinite(s);
+    }
+    if (!finite) sb_latch(dstate, SB_ERR_NONFINITE, SBK_SCORES);
+    if (gain)
+        for (int l = 0; l + 1 < L; ++l)
+            gain[blk * (L - 1) + l] = (e[l] - e[l + 1]) / ((float)(ba.bits[l + 1] - ba.bits[l]) * M);
 }
 
 // ---- reorder statistics --------------------------------------------------------------------
@@ -320,8 +455,9 @@ __global__ void rank_count_kernel(const float* __restrict__ score, int64_t K, in
     const int64_t j1 = min(s0 + seg, j0 + span);
     const uint32_t ki = order_key(score[i]);
     int cnt = 0;
+#pragma unroll 8
     for (int64_t j = j0; j < j1; ++j) {
-        const uint32_t kj = order_key(__ldg(score + j));
+        const uint32_t kj = order_key(__ldg(score + j));     // same j across the warp: broadcast
         cnt += (kj > ki) || (kj == ki && j < i);
     }
     if (cnt) atomicAdd(rank + i, cnt);
@@ -358,6 +494,8 @@ BitsArg make_bits(const int* bits, int n) {
         ba.bits[l] = b;
         ba.qmax[l] = (float)((1 << b) - 1);
         ba.inv_qmax[l] = 1.0f / (float)((1 << b) - 1);
+        ba.q2[l] = make_float2(ba.qmax[l], ba.qmax[l]);
+        ba.niq2[l] = make_float2(-ba.inv_qmax[l], -ba.inv_qmax[l]);
     }
     return ba;
 }
@@ -366,8 +504,9 @@ bool valid_group(int g) { return g == 16 || g == 32 || g == 64 || g == 128; }
 
 sb_status argsort_axis(sb_ctx* ctx, const float* score, int64_t K, int64_t seg, int32_t* perm, int* rank) {
     SB_CUDA(ctx, cudaMemsetAsync(rank, 0, sizeof(int) * K, ctx->stream));
-    int splits = (int)((seg + 2047) / 2048);
-    if (splits > 64) splits = 64;
+    // short comparison loops (<= 256 per thread): the counting is latency-bound otherwise
+    int splits = (int)((seg + 255) / 256);
+    if (splits > 1024) splits = 1024;
     const int64_t span = (seg + splits - 1) / splits;
     dim3 grid((unsigned)((K + 255) / 256), splits);
     rank_count_kernel<<<grid, 256, 0, ctx->stream>>>(score, K, seg, span, rank);
@@ -377,17 +516,62 @@ sb_status argsort_axis(sb_ctx* ctx, const float* score, int64_t K, int64_t seg, 
     return SB_OK;
 }
 
-template <int L, int CPL>
-void launch_scores(sb_ctx* ctx, dim3 grid, bool roww, const __nv_bfloat16* W, int64_t ldw,
-                   const int32_t* lrp, const int32_t* cperm, const int32_t* aperm, const float* cm,
-                   const float* rw, int br, int bc, int group, const BitsArg& ba, int64_t nbc,
-                   float* err, float* gain) {
-    if (roww)
-        block_scores_kernel<L, CPL, true><<<grid, CTA_THREADS, 0, ctx->stream>>>(
-            W, ldw, lrp, cperm, aperm, cm, rw, br, bc, group, ba, nbc, err, gain, ctx->dstate);
-    else
-        block_scores_kernel<L, CPL, false><<<grid, CTA_THREADS, 0, ctx->stream>>>(
-            W, ldw, lrp, cperm, aperm, cm, rw, br, bc, group, ba, nbc, err, gain, ctx->dstate);
+template <int L, int CPL, int NFINE, bool FULLG, bool ROWW>
+sb_status launch_scores_k(sb_ctx* ctx, const __nv_bfloat16* W, int64_t ldw, const int32_t* lrp,
+                          const int32_t* cperm, const int32_t* aperm, const float* cm, const float* rw,
+                          int br, int bc, int group, const BitsArg& ba, int64_t R, int64_t C, float* err,
+                          float* gain, float* part_buf) {
+    const int tile_w = bc >= 128 ? bc : 128;
+    const int64_t n_tile_cols = C / tile_w, nbc = C / bc, n_blocks = (R / br) * nbc;
+    // a unit is a 32-row part of a tile when the block height allows it, else the whole tile
+    const int part_rows = br % 32 == 0 ? 32 : br;
+    const int parts = br / part_rows;
+    const int64_t n_units = (R / br) * n_tile_cols * parts;
+    const size_t smem = (size_t)CTA_WARPS * 2 * SLAB_BYTES;
+    auto kern = block_scores_kernel<L, CPL, NFINE, FULLG, ROWW>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        SB_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr_done = true;
+    }
+    int64_t grid = (int64_t)ctx->sm_count * 2;      // persistent: two CTAs per SM
+    const int64_t need = (n_units + CTA_WARPS - 1) / CTA_WARPS;
+    if (grid > need) grid = need;
+    kern<<<(unsigned)grid, CTA_THREADS, smem, ctx->stream>>>(
+        W, ldw, lrp, cperm, aperm, cm, rw, br, bc, group, ba, nbc, n_tile_cols, parts, part_rows, n_units,
+        n_blocks, part_buf);
+    SB_LAUNCHED(ctx);
+    scores_finish_kernel<<<(unsigned)((n_blocks + 255) / 256), 256, 0, ctx->stream>>>(
+        part_buf, parts, n_blocks, L, ba, (float)br * (float)bc, err, gain, ctx->dstate);
+    SB_LAUNCHED(ctx);
+    return SB_OK;
+}
+
+// the common case (group = 128 columns, no row weights) gets its own instance with the
+// group reduction unrolled; everything else shares the general one
+template <int L, int CPL, int NFINE>
+sb_status launch_scores_n(sb_ctx* ctx, const __nv_bfloat16* W, int64_t ldw, const int32_t* lrp,
+                          const int32_t* cperm, const int32_t* aperm, const float* cm, const float* rw,
+                          int br, int bc, int group, const BitsArg& ba, int64_t R, int64_t C, float* err,
+                          float* gain, float* part_buf) {
+    if (group == 128 && !rw)
+        return launch_scores_k<L, CPL, NFINE, true, false>(ctx, W, ldw, lrp, cperm, aperm, cm, rw, br, bc,
+                                                           group, ba, R, C, err, gain, part_buf);
+    if (!rw)
+        return launch_scores_k<L, CPL, NFINE, false, false>(ctx, W, ldw, lrp, cperm, aperm, cm, rw, br, bc,
+                                                            group, ba, R, C, err, gain, part_buf);
+    return launch_scores_k<L, CPL, NFINE, false, true>(ctx, W, ldw, lrp, cperm, aperm, cm, rw, br, bc,
+                                                       group, ba, R, C, err, gain, part_buf);
+}
+
+// candidates with >= 6 bits keep a two-float grid step; they are the last `nfine` of the list.
+// Compiled for 0..2 such candidates and for "all of them" (always correct, a little slower).
+template <int L, int CPL, typename... A>
+sb_status launch_scores(int nfine, A... args) {
+    if (nfine == 0) return launch_scores_n<L, CPL, 0>(args...);
+    if (nfine == 1 && L >= 1) return launch_scores_n<L, CPL, (L >= 1 ? 1 : L)>(args...);
+    if (nfine == 2 && L >= 2) return launch_scores_n<L, CPL, (L >= 2 ? 2 : L)>(args...);
+    return launch_scores_n<L, CPL, L>(args...);
 }
 
 }  // namespace
@@ -509,12 +693,17 @@ sb_status sb_block_scores(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int6
     const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(W);
     int64_t ld = ldw;
     const int32_t* load_rp = row_perm;
-    if (col_perm || W_perm_out) {
-        void* dst = W_perm_out;
-        if (!dst) {
-            sb_status st = sb_scratch(ctx, (size_t)R * C * 2 + 256, &dst);
-            if (st != SB_OK) return st;
-        }
+    const int parts_max = br % 32 == 0 ? br / 32 : 1;
+    const size_t part_bytes = (size_t)parts_max * (R / br) * (C / bc) * n_bits * sizeof(float);
+    const bool need_copy = col_perm || W_perm_out;
+    void* arena;
+    sb_status sst = sb_scratch(ctx, Carver::need({part_bytes, (need_copy && !W_perm_out) ? (size_t)R * C * 2 : 0}),
+                               &arena);
+    if (sst != SB_OK) return sst;
+    Carver cv(arena);
+    float* part_buf = cv.take<float>(part_bytes / sizeof(float));
+    if (need_copy) {
+        void* dst = W_perm_out ? W_perm_out : static_cast<void*>(cv.take<unsigned char>((size_t)R * C * 2));
         sb_status st = sb_gather_bf16(ctx, W, R, C, ldw, row_perm, col_perm, dst);
         if (st != SB_OK) return st;
         src = static_cast<const __nv_bfloat16*>(dst);
@@ -524,12 +713,12 @@ sb_status sb_block_scores(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int6
     const BitsArg ba = make_bits(bits, n_bits);
     const int tile_w = bc >= 128 ? bc : 128;
     if (C % tile_w) return sb_fail(ctx, SB_ERR_SHAPE, "scores: C must be a multiple of 128");
-    dim3 grid((unsigned)(C / tile_w), (unsigned)(R / br));
-    const int64_t nbc = C / bc;
-    const bool roww = row_weight != nullptr;
-#define SB_SCORES(Lv, CPLv)                                                                       \
-    launch_scores<Lv, CPLv>(ctx, grid, roww, src, ld, load_rp, col_perm, row_perm, col_moment,     \
-                            row_weight, br, bc, group, ba, nbc, err, gain)
+    sb_status st = SB_OK;
+    int nfine = 0;
+    for (int l = 0; l < n_bits; ++l) nfine += bits[l] >= 6;
+#define SB_SCORES(Lv, CPLv)                                                                        \
+    st = launch_scores<Lv, CPLv>(nfine, ctx, src, ld, load_rp, col_perm, row_perm, col_moment,     \
+                                 row_weight, br, bc, group, ba, R, C, err, gain, part_buf)
     switch (n_bits) {
         case 1: SB_SCORES(1, 16); break;
         case 2: SB_SCORES(2, 16); break;
@@ -541,8 +730,7 @@ sb_status sb_block_scores(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int6
         default: SB_SCORES(8, 8); break;
     }
 #undef SB_SCORES
-    SB_LAUNCHED(ctx);
-    return SB_OK;
+    return st;
 }
 
 }  // extern "C"
