@@ -159,7 +159,7 @@ sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
  * meta[(r*(C/group) + g)] = {(float)scale, (float)lo} for group g of permuted row r.
  * If block_off_words[nb] > packed_capacity_words nothing beyond the capacity is written
  * and SB_ERR_SCRATCH is latched.  block_rows*block_cols*bits % 32 == 0 is required,
- * group % 4 == 0, block_cols % 32 == 0.                                              */
+ * group in {16,32,64,128}, block_rows % 4 == 0.                                           */
 sb_status sb_pack_blocks(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_t C, int64_t ldw,
                          const int32_t* row_perm, const int32_t* col_perm,
                          int block_rows, int block_cols, int group,

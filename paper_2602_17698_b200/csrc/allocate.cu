@@ -9,7 +9,11 @@
 // device-wide prefix sum of (count, cost) over the flagged entries -- a single look-back
 // scan per direction and iteration instead of a sort.  Algorithm 1 (greedy along each
 // block's convex hull) is one sort, one scan of the step costs and a threshold.
+#include <cooperative_groups.h>
+
 #include "lookback.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -17,6 +21,9 @@ constexpr int AT = 256;             // threads of the scan-select kernels
 constexpr int AI = 8;               // entries per thread
 constexpr int ATILE = AT * AI;
 constexpr int BT = 256;             // threads of the per-block kernels
+constexpr int LT = 256;             // threads of the persistent loop kernel
+constexpr int LT_WARPS_MAX = LT / 32;
+constexpr int LOOP_MAX_CTAS = 4096;
 
 struct AllocState {
     long long cap, used;
@@ -124,190 +131,257 @@ __global__ void init_finish_kernel(AllocArgs a, int nparts) {
     a.st->loss_init = s;
 }
 
-// ---- one iteration of Algorithm 2 ---------------------------------------------------------
-// Step 1: walk the up list; entries whose step starts at the block's level and gains > 0 are
-// candidates.  Candidate number p (0-based) with p < k records its rank and the cumulative
-// cost of candidates 0..p.
-__global__ void __launch_bounds__(AT)
-select_up_kernel(AllocArgs a, const unsigned* __restrict__ list, long long n, LookbackBuf lb,
-                 unsigned epoch, SbDeviceState* ds) {
-    const unsigned tile = lookback_tile_id(ds);
-    const AllocState s = *a.st;
-    if (s.done) return;   // every tile sees the same state: nobody waits on anybody
-    const long long base = (long long)tile * ATILE + (long long)threadIdx.x * AI;
-    unsigned blk[AI]; unsigned long long cost[AI]; bool flag[AI];
-    CntCost sum{0ull, 0u, 0u};
+// ---- the Algorithm 2 loop, one persistent cooperative kernel ----------------------------------
+// All iterations run inside one launch; the phases of an iteration are separated by grid-wide
+// barriers (cooperative launch: every CTA is resident).  CTA c owns a contiguous slice of both
+// sorted lists.  A "select" is two passes over the slice: (1) count the candidates and add up
+// their costs, publish the CTA total; (2) after the barrier, the exclusive prefix over the
+// lower CTAs gives every candidate its global rank p and cumulative cost.  The loop state
+// (k, used, loss, counters) is replicated: every CTA derives it from the same published
+// totals, added in the same order, so no CTA has to wait for a single writer.
+//   expansion iteration: up-count | up-rank + U | apply            (3 barriers)
+//   exchange  iteration: up-count | up-rank | down-count | down-rank + D | U | apply   (6)
+// Data written by other CTAs during the kernel is read through L2 (__ldcg): L1 is not
+// coherent across SMs inside one launch.
+struct LoopWork {
+    CntCost* up_tot; long long* up_first; CntCost* dn_tot;
+    double* dD; unsigned long long* freed; unsigned* nD;
+    double* dU; unsigned long long* costU; unsigned* nU;
+};
+
+__device__ __forceinline__ CntCost ldcg_cc(const CntCost* p) {
+    const ulonglong2 v = __ldcg(reinterpret_cast<const ulonglong2*>(p));
+    CntCost c; c.cost = v.x; c.cnt = (unsigned)v.y; c.pad = 0u;
+    return c;
+}
+
+// sum of one value per thread over the CTA, valid in every thread (fixed order)
+template <typename T>
+__device__ __forceinline__ T cta_total_u(T v) {
+    __shared__ T sh[LT_WARPS_MAX];
+    __shared__ T tot;
 #pragma unroll
-    for (int j = 0; j < AI; ++j) {
-        flag[j] = false; cost[j] = 0; blk[j] = 0;
-        if (base + j < n) {
-            const unsigned e = list[base + j];
-            const long long i = e / (unsigned)(a.L - 1);
-            const int l = (int)(e % (unsigned)(a.L - 1));
-            if (a.level[i] == l && a.err[i * a.L + l] > a.err[i * a.L + l + 1]) {
-                flag[j] = true;
-                blk[j] = (unsigned)i;
-                cost[j] = (unsigned long long)(elems_of(a, i) * (a.bits[l + 1] - a.bits[l]));
-                sum.cnt += 1; sum.cost += cost[j];
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        T s = 0;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += sh[w];
+        tot = s;
+    }
+    __syncthreads();
+    const T r = tot;
+    __syncthreads();
+    return r;
+}
+
+__global__ void __launch_bounds__(LT)
+scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
+                      const unsigned* __restrict__ dn_list, long long ne, LoopWork w) {
+    cg::grid_group grid = cg::this_grid();
+    const int G = gridDim.x, c = blockIdx.x, tid = threadIdx.x;
+    const long long per_cta = (ne + G - 1) / G;
+    const long long ipt = (per_cta + LT - 1) / LT;                    // entries per thread
+    const long long cta_hi = min(ne, (long long)(c + 1) * per_cta);
+    const long long t_lo = min(cta_hi, (long long)c * per_cta + (long long)tid * ipt);
+    const long long t_hi = min(cta_hi, t_lo + ipt);
+    const unsigned Lm1 = (unsigned)(a.L - 1);
+
+    const AllocState s0 = *a.st;                    // written before the launch
+    const long long cap = s0.cap, kT = s0.kT;
+    long long k = s0.k, used = s0.used;
+    double loss = s0.loss;
+    int iter = 0, accepted = 0, rejected = 0, expansions = 0, status = 0;
+
+    // candidate test of one list entry; returns the block or -1
+    auto up_entry = [&](long long p, unsigned long long& cost, double& de) -> long long {
+        const unsigned e = up_list[p];
+        const long long i = e / Lm1;
+        const int l = (int)(e % Lm1);
+        if ((int)__ldcg(a.level + i) != l) return -1;
+        const float e0 = a.err[i * a.L + l], e1 = a.err[i * a.L + l + 1];
+        if (!(e0 > e1)) return -1;
+        cost = (unsigned long long)(elems_of(a, i) * (a.bits[l + 1] - a.bits[l]));
+        de = __dsub_rn((double)e0, (double)e1);
+        return i;
+    };
+
+    while (k >= kT) {
+        if (iter >= 4096) { status = SB_ERR_NOCONVERGE; break; }
+        const unsigned stamp = (unsigned)iter + 1u;
+        const long long slack = cap - used;
+        const long long h = k / 2 > 0 ? k / 2 : 1;
+
+        // ---- up-count -------------------------------------------------------------------------
+        CntCost mine{0ull, 0u, 0u};
+        long long my_first = -1;
+        for (long long p = t_lo; p < t_hi; ++p) {
+            unsigned long long cost; double de;
+            if (up_entry(p, cost, de) >= 0) {
+                if (mine.cnt == 0) my_first = (long long)cost;
+                mine.cnt += 1; mine.cost += cost;
             }
         }
-    }
-    CntCost tile_total;
-    CntCost ex = block_exclusive_scan<CntCost, AT>(sum, tile_total);
-    const CntCost prefix = lookback_prefix<CntCost>(tile_total, tile, lb, epoch, ds);
-    CntCost run = t_add(prefix, ex);
-    if ((long long)run.cnt >= s.k) return;
-#pragma unroll
-    for (int j = 0; j < AI; ++j) {
-        if (!flag[j]) continue;
-        const unsigned p = run.cnt;
-        run.cnt += 1; run.cost += cost[j];
-        if ((long long)p < s.k) {
-            a.uprank[blk[j]] = p;
-            a.upcum[blk[j]] = run.cost;
-            a.upstamp[blk[j]] = (unsigned)s.iter + 1u;
-            if (p == 0 && s.used < s.cap && (long long)cost[j] <= s.cap - s.used) a.st->expand_ok = 1;
+        CntCost cta_tot;
+        const CntCost ex = block_exclusive_scan<CntCost, LT>(mine, cta_tot);
+        if (ex.cnt == 0 && mine.cnt > 0) w.up_first[c] = my_first;      // the CTA's first candidate
+        if (tid == 0) {
+            w.up_tot[c] = cta_tot;
+            if (cta_tot.cnt == 0) w.up_first[c] = -1;
         }
-    }
-}
+        grid.sync();
 
-// Step 2 (exchange stage only): walk the down list; entries whose step ends at the block's
-// level, outside the first h up-candidates, are down-candidates; the first h of them form D.
-__global__ void __launch_bounds__(AT)
-select_down_kernel(AllocArgs a, const unsigned* __restrict__ list, long long n, LookbackBuf lb,
-                   unsigned epoch, SbDeviceState* ds) {
-    const unsigned tile = lookback_tile_id(ds);
-    const AllocState s = *a.st;
-    if (s.done || s.expand_ok) return;   // uniform over the grid (set before this launch)
-    const long long h = s.k / 2 > 0 ? s.k / 2 : 1;
-    const unsigned stamp = (unsigned)s.iter + 1u;
-    const long long base = (long long)tile * ATILE + (long long)threadIdx.x * AI;
-    unsigned blk[AI]; unsigned long long cost[AI]; double de[AI]; bool flag[AI];
-    CntCost sum{0ull, 0u, 0u};
-#pragma unroll
-    for (int j = 0; j < AI; ++j) {
-        flag[j] = false; cost[j] = 0; blk[j] = 0; de[j] = 0.0;
-        if (base + j < n) {
-            const unsigned e = list[base + j];
-            const long long i = e / (unsigned)(a.L - 1);
-            const int l = (int)(e % (unsigned)(a.L - 1));
-            const bool in_u0 = a.upstamp[i] == stamp && (long long)a.uprank[i] < h;
-            if (a.level[i] == l + 1 && !in_u0) {
-                flag[j] = true;
-                blk[j] = (unsigned)i;
-                cost[j] = (unsigned long long)(elems_of(a, i) * (a.bits[l + 1] - a.bits[l]));
-                de[j] = __dsub_rn((double)a.err[i * a.L + l], (double)a.err[i * a.L + l + 1]);
-                sum.cnt += 1; sum.cost += cost[j];
+        // ---- prefix over the lower CTAs, cost of the globally first candidate ------------------
+        unsigned long long pre_cost = 0; unsigned pre_cnt = 0; int first_cta = 0x7fffffff;
+        for (int j = tid; j < G; j += LT) {
+            const CntCost t = ldcg_cc(w.up_tot + j);
+            if (j < c) { pre_cost += t.cost; pre_cnt += t.cnt; }
+            if (t.cnt > 0 && j < first_cta) first_cta = j;
+        }
+        pre_cost = cta_total_u<unsigned long long>(pre_cost);
+        pre_cnt = cta_total_u<unsigned>(pre_cnt);
+        {
+            __shared__ int fc;
+            if (tid == 0) fc = 0x7fffffff;
+            __syncthreads();
+            if (first_cta != 0x7fffffff) atomicMin(&fc, first_cta);
+            __syncthreads();
+            first_cta = fc;
+            __syncthreads();
+        }
+        const long long first_cost = first_cta != 0x7fffffff ? __ldcg(w.up_first + first_cta) : -1;
+        const bool expand = used < cap && first_cost >= 0 && first_cost <= slack;
+        const long long lim_rank = expand ? k : h;
+
+        // ---- up-rank (and, in an expansion, the set U itself) -----------------------------------
+        double dU_mine = 0.0; unsigned long long costU_mine = 0; unsigned nU_mine = 0;
+        if ((long long)pre_cnt + ex.cnt < lim_rank) {
+            unsigned long long run_cost = pre_cost + ex.cost;
+            long long run_cnt = (long long)pre_cnt + ex.cnt;
+            for (long long p = t_lo; p < t_hi && run_cnt < lim_rank; ++p) {
+                unsigned long long cost; double de;
+                const long long i = up_entry(p, cost, de);
+                if (i < 0) continue;
+                run_cost += cost;
+                a.uprank[i] = (unsigned)run_cnt;
+                a.upcum[i] = run_cost;
+                a.upstamp[i] = stamp;
+                if (expand && (long long)run_cost <= slack) {
+                    a.ustamp[i] = stamp;
+                    dU_mine += de; costU_mine += cost; nU_mine += 1;
+                }
+                run_cnt += 1;
             }
         }
-    }
-    CntCost tile_total;
-    CntCost ex = block_exclusive_scan<CntCost, AT>(sum, tile_total);
-    const CntCost prefix = lookback_prefix<CntCost>(tile_total, tile, lb, epoch, ds);
-    CntCost run = t_add(prefix, ex);
-    double dsum = 0.0; unsigned long long fsum = 0; unsigned cnt = 0;
-#pragma unroll
-    for (int j = 0; j < AI; ++j) {
-        if (!flag[j]) continue;
-        const unsigned p = run.cnt;
-        run.cnt += 1;
-        if ((long long)p < h) {
-            a.dnstamp[blk[j]] = stamp;
-            dsum += de[j]; fsum += cost[j]; cnt += 1;
+        if (expand) {
+            const double d = cta_sum<LT>(dU_mine);
+            const unsigned long long cu = cta_total_u<unsigned long long>(costU_mine);
+            const unsigned nu = cta_total_u<unsigned>(nU_mine);
+            if (tid == 0) { w.dU[c] = d; w.costU[c] = cu; w.nU[c] = nu; }
         }
-    }
-    const double tsum = cta_sum<AT>(dsum);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        fsum += __shfl_xor_sync(0xffffffffu, fsum, o);
-        cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-    }
-    if ((threadIdx.x & 31) == 0 && cnt) {
-        atomicAdd(&a.st->freed, fsum);
-        atomicAdd(&a.st->nD, cnt);
-    }
-    if (threadIdx.x == 0) a.part[tile] = tsum;
-    if (cta_is_last(&a.st->done_down) && threadIdx.x == 0) {
-        double t = 0.0;
-        for (unsigned p = 0; p < gridDim.x; ++p) t += ((volatile double*)a.part)[p];
-        a.st->dD = t;
-    }
-}
+        grid.sync();
 
-// Step 3: the up-set U.  Expansion: candidates 0..k-1 whose cumulative cost fits the slack.
-// Exchange: candidates 0..h-1 whose cumulative cost fits slack + what D frees.  The last CTA
-// adds the partial gains in a fixed order and takes the accept decision.
-__global__ void __launch_bounds__(BT) decide_kernel(AllocArgs a, double* part) {
-    const AllocState s = *a.st;
-    if (s.done) return;
-    const long long i = (long long)blockIdx.x * BT + threadIdx.x;
-    const unsigned stamp = (unsigned)s.iter + 1u;
-    const bool expand = s.expand_ok != 0;
-    const long long h = s.k / 2 > 0 ? s.k / 2 : 1;
-    const long long lim_rank = expand ? s.k : h;
-    const long long lim_cost = (s.cap - s.used) + (expand ? 0ll : (long long)s.freed);
-    double de = 0.0; unsigned long long c = 0; unsigned cnt = 0;
-    if (i < a.N && a.upstamp[i] == stamp && (long long)a.uprank[i] < lim_rank &&
-        (long long)a.upcum[i] <= lim_cost) {
-        const int l = a.level[i];
-        a.ustamp[i] = stamp;
-        de = __dsub_rn((double)a.err[i * a.L + l], (double)a.err[i * a.L + l + 1]);
-        c = (unsigned long long)(elems_of(a, i) * (a.bits[l + 1] - a.bits[l]));
-        cnt = 1;
-    }
-    const double tsum = cta_sum<BT>(de);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        c += __shfl_xor_sync(0xffffffffu, c, o);
-        cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-    }
-    if ((threadIdx.x & 31) == 0 && cnt) {
-        atomicAdd(&a.st->costU, c);
-        atomicAdd(&a.st->nU, cnt);
-    }
-    if (threadIdx.x == 0) part[blockIdx.x] = tsum;
-    if (cta_is_last(&a.st->done_decide) && threadIdx.x == 0) {
-        double t = 0.0;
-        for (unsigned p = 0; p < gridDim.x; ++p) t += ((volatile double*)part)[p];
-        a.st->dU = t;
-        const unsigned nU = *(volatile unsigned*)&a.st->nU, nD = *(volatile unsigned*)&a.st->nD;
-        const double dD = *(volatile double*)&a.st->dD;
-        a.st->accept = expand ? (nU > 0) : (nU > 0 && nD > 0 && t > dD);
-    }
-}
+        if (!expand) {
+            // ---- down-count ----------------------------------------------------------------------
+            auto dn_entry = [&](long long p, unsigned long long& cost, double& de) -> long long {
+                const unsigned e = dn_list[p];
+                const long long i = e / Lm1;
+                const int l = (int)(e % Lm1);
+                if ((int)__ldcg(a.level + i) != l + 1) return -1;
+                if (__ldcg(a.upstamp + i) == stamp && (long long)__ldcg(a.uprank + i) < h) return -1;
+                cost = (unsigned long long)(elems_of(a, i) * (a.bits[l + 1] - a.bits[l]));
+                de = __dsub_rn((double)a.err[i * a.L + l], (double)a.err[i * a.L + l + 1]);
+                return i;
+            };
+            CntCost dm{0ull, 0u, 0u};
+            for (long long p = t_lo; p < t_hi; ++p) {
+                unsigned long long cost; double de;
+                if (dn_entry(p, cost, de) >= 0) { dm.cnt += 1; dm.cost += cost; }
+            }
+            CntCost dn_cta;
+            const CntCost dex = block_exclusive_scan<CntCost, LT>(dm, dn_cta);
+            if (tid == 0) w.dn_tot[c] = dn_cta;
+            grid.sync();
+            unsigned dpre = 0;
+            for (int j = tid; j < c; j += LT) dpre += ldcg_cc(w.dn_tot + j).cnt;
+            dpre = cta_total_u<unsigned>(dpre);
+            // ---- down-rank: the first h candidates form D -----------------------------------------
+            double dD_mine = 0.0; unsigned long long freed_mine = 0; unsigned nD_mine = 0;
+            long long run_cnt = (long long)dpre + dex.cnt;
+            for (long long p = t_lo; p < t_hi && run_cnt < h; ++p) {
+                unsigned long long cost; double de;
+                const long long i = dn_entry(p, cost, de);
+                if (i < 0) continue;
+                a.dnstamp[i] = stamp;
+                dD_mine += de; freed_mine += cost; nD_mine += 1;
+                run_cnt += 1;
+            }
+            {
+                const double d = cta_sum<LT>(dD_mine);
+                const unsigned long long f = cta_total_u<unsigned long long>(freed_mine);
+                const unsigned nd = cta_total_u<unsigned>(nD_mine);
+                if (tid == 0) { w.dD[c] = d; w.freed[c] = f; w.nD[c] = nd; }
+            }
+            grid.sync();
+            // ---- U: up-candidates 0..h-1 whose cumulative cost fits slack + what D frees ------------
+            unsigned long long freed_tot = 0;
+            for (int j = tid; j < G; j += LT) freed_tot += __ldcg(w.freed + j);
+            freed_tot = cta_total_u<unsigned long long>(freed_tot);
+            const long long lim_cost = slack + (long long)freed_tot;
+            for (long long i = (long long)c * LT + tid; i < a.N; i += (long long)G * LT) {
+                if (__ldcg(a.upstamp + i) == stamp && (long long)__ldcg(a.uprank + i) < h &&
+                    (long long)__ldcg(a.upcum + i) <= lim_cost) {
+                    const int l = (int)__ldcg(a.level + i);
+                    a.ustamp[i] = stamp;
+                    dU_mine += __dsub_rn((double)a.err[i * a.L + l], (double)a.err[i * a.L + l + 1]);
+                    costU_mine += (unsigned long long)(elems_of(a, i) * (a.bits[l + 1] - a.bits[l]));
+                    nU_mine += 1;
+                }
+            }
+            const double d = cta_sum<LT>(dU_mine);
+            const unsigned long long cu = cta_total_u<unsigned long long>(costU_mine);
+            const unsigned nu = cta_total_u<unsigned>(nU_mine);
+            if (tid == 0) { w.dU[c] = d; w.costU[c] = cu; w.nU[c] = nu; }
+            grid.sync();
+        }
 
-// Step 4: apply the move, then (last CTA) advance the loop state.
-__global__ void __launch_bounds__(BT) apply_kernel(AllocArgs a) {
-    const AllocState s = *a.st;
-    if (s.done) return;
-    const long long i = (long long)blockIdx.x * BT + threadIdx.x;
-    const unsigned stamp = (unsigned)s.iter + 1u;
-    const bool expand = s.expand_ok != 0;
-    if (i < a.N && s.accept) {
-        if (a.ustamp[i] == stamp) a.level[i] += 1;
-        else if (!expand && a.dnstamp[i] == stamp) a.level[i] -= 1;
+        // ---- totals (same order in every CTA), decision, apply, replicated state update -----------
+        __shared__ double sh_dU, sh_dD;
+        if (tid == 0) {
+            double u = 0.0, dsum = 0.0;
+            for (int j = 0; j < G; ++j) u += __ldcg(w.dU + j);
+            if (!expand) for (int j = 0; j < G; ++j) dsum += __ldcg(w.dD + j);
+            sh_dU = u; sh_dD = dsum;
+        }
+        unsigned long long costU = 0, freed = 0; unsigned nU = 0, nD = 0;
+        for (int j = tid; j < G; j += LT) {
+            costU += __ldcg(w.costU + j); nU += __ldcg(w.nU + j);
+            if (!expand) { freed += __ldcg(w.freed + j); nD += __ldcg(w.nD + j); }
+        }
+        costU = cta_total_u<unsigned long long>(costU);
+        freed = cta_total_u<unsigned long long>(freed);
+        nU = cta_total_u<unsigned>(nU);
+        nD = cta_total_u<unsigned>(nD);
+        __syncthreads();
+        const double dU = sh_dU, dD = sh_dD;
+        const bool accept = expand ? (nU > 0) : (nU > 0 && nD > 0 && dU > dD);
+        if (accept) {
+            for (long long i = (long long)c * LT + tid; i < a.N; i += (long long)G * LT) {
+                if (__ldcg(a.ustamp + i) == stamp) a.level[i] = (unsigned char)(__ldcg(a.level + i) + 1);
+                else if (!expand && __ldcg(a.dnstamp + i) == stamp)
+                    a.level[i] = (unsigned char)(__ldcg(a.level + i) - 1);
+            }
+        }
+        if (expand && accept) { used += (long long)costU; loss -= dU; expansions += 1; }
+        else if (accept) { used += (long long)costU - (long long)freed; loss += dD - dU; accepted += 1; }
+        else { k /= 2; rejected += 1; }
+        iter += 1;
+        grid.sync();                                  // the new levels are visible to the next up-count
     }
-    if (cta_is_last(&a.st->done_apply) && threadIdx.x == 0) {
+    if (c == 0 && tid == 0) {
         AllocState* st = a.st;
-        if (expand && s.accept) {
-            st->used = s.used + (long long)s.costU;
-            st->loss = s.loss - s.dU;
-            st->expansions = s.expansions + 1;
-        } else if (s.accept) {
-            st->used = s.used + (long long)s.costU - (long long)s.freed;
-            st->loss = s.loss + (s.dD - s.dU);
-            st->accepted = s.accepted + 1;
-        } else {
-            st->k = s.k / 2;
-            st->rejected = s.rejected + 1;
-        }
-        st->iter = s.iter + 1;
-        if (st->k < s.kT) st->done = 1;
-        else if (st->iter >= 4096) { st->done = 1; st->status = SB_ERR_NOCONVERGE; }
-        st->expand_ok = 0; st->accept = 0; st->nU = 0; st->nD = 0; st->freed = 0; st->costU = 0;
-        st->dU = 0.0; st->dD = 0.0;
-        st->done_down = 0; st->done_decide = 0; st->done_apply = 0;
-        __threadfence();
+        st->k = k; st->used = used; st->loss = loss; st->iter = iter; st->accepted = accepted;
+        st->rejected = rejected; st->expansions = expansions; st->done = 1; st->status = status;
     }
 }
 
@@ -429,7 +503,8 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
                                                    ns * 4, ns * 4, ns * 4, ns * 4,
                                                    (size_t)N * 4, (size_t)N * 4, (size_t)N * 8,
                                                    (size_t)N * 4, (size_t)N * 4, nparts * 8,
-                                                   nparts * 8, sort_bytes, (size_t)(N + 1) * 8}), &arena);
+                                                   nparts * 8, sort_bytes, (size_t)(N + 1) * 8,
+                                                   (size_t)LOOP_MAX_CTAS * 128}), &arena);
     if (stt != SB_OK) return stt;
     Carver cv(arena);
     AllocState* dst = cv.take<AllocState>(1);
@@ -450,6 +525,11 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
     double* part2 = cv.take<double>(nparts);
     void* sort_scratch = cv.take<unsigned char>(sort_bytes);
     unsigned long long* totals = cv.take<unsigned long long>((size_t)N + 1);
+    CntCost* loop_cc = cv.take<CntCost>(2 * LOOP_MAX_CTAS);
+    long long* loop_ll = cv.take<long long>(LOOP_MAX_CTAS);
+    double* loop_d = cv.take<double>(2 * LOOP_MAX_CTAS);
+    unsigned long long* loop_u64 = cv.take<unsigned long long>(2 * LOOP_MAX_CTAS);
+    unsigned* loop_u32 = cv.take<unsigned>(2 * LOOP_MAX_CTAS);
 
     long long total_elems = 0;
     AllocState* hst = static_cast<AllocState*>(ctx->pinned);
@@ -546,28 +626,27 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
             if (stt != SB_OK) return stt;
             stt = sb_radix_sort_u64(ctx, kC, kD, vC, vD, nsteps, sort_scratch);
             if (stt != SB_OK) return stt;
-            bool done = false;
-            int chunk = 8;
-            while (!done) {
-                for (int it = 0; it < chunk; ++it) {
-                    unsigned epoch; sb_status s2;
-                    LookbackBuf lb = sb_lookback(ctx, (unsigned)ntiles, &epoch, &s2);
-                    if (s2 != SB_OK) return s2;
-                    select_up_kernel<<<(unsigned)ntiles, AT, 0, ctx->stream>>>(a, vA, nsteps, lb, epoch, ctx->dstate);
-                    SB_LAUNCHED(ctx);
-                    lb = sb_lookback(ctx, (unsigned)ntiles, &epoch, &s2);
-                    if (s2 != SB_OK) return s2;
-                    select_down_kernel<<<(unsigned)ntiles, AT, 0, ctx->stream>>>(a, vC, nsteps, lb, epoch, ctx->dstate);
-                    SB_LAUNCHED(ctx);
-                    decide_kernel<<<nblkB, BT, 0, ctx->stream>>>(a, part2);
-                    SB_LAUNCHED(ctx);
-                    apply_kernel<<<nblkB, BT, 0, ctx->stream>>>(a);
-                    SB_LAUNCHED(ctx);
-                }
-                stt = read_state(&fin);
-                if (stt != SB_OK) return stt;
-                done = fin.done != 0;
-            }
+            // the whole loop in one cooperative launch
+            int occ = 0;
+            SB_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scalebits_loop_kernel, LT, 0));
+            long long G = (long long)occ * ctx->sm_count;
+            const long long want = (nsteps + 4 * LT - 1) / (4 * LT) > (N + 4 * LT - 1) / (4 * LT)
+                                       ? (nsteps + 4 * LT - 1) / (4 * LT) : (N + 4 * LT - 1) / (4 * LT);
+            if (G > want) G = want;
+            if (G > LOOP_MAX_CTAS) G = LOOP_MAX_CTAS;
+            if (G < 1) G = 1;
+            LoopWork lw;
+            lw.up_tot = loop_cc; lw.dn_tot = loop_cc + LOOP_MAX_CTAS;
+            lw.up_first = loop_ll;
+            lw.dD = loop_d; lw.dU = loop_d + LOOP_MAX_CTAS;
+            lw.freed = loop_u64; lw.costU = loop_u64 + LOOP_MAX_CTAS;
+            lw.nD = loop_u32; lw.nU = loop_u32 + LOOP_MAX_CTAS;
+            const unsigned* up_list = vA; const unsigned* dn_list = vC;
+            long long ne = nsteps;
+            void* kargs[] = {&a, &up_list, &dn_list, &ne, &lw};
+            SB_CUDA(ctx, cudaLaunchCooperativeKernel((const void*)scalebits_loop_kernel, dim3((unsigned)G),
+                                                     dim3(LT), kargs, 0, ctx->stream));
+            ctx->launches++;
         }
         // single candidate (or finished): histogram of the final levels
         eval_kernel<<<nblkB, BT, 0, ctx->stream>>>(a, part2, 0);

@@ -12,43 +12,94 @@ namespace {
 constexpr int PK_THREADS = 256;
 constexpr int PK_WARPS = PK_THREADS / 32;
 
-__global__ void block_words_kernel(const unsigned char* __restrict__ level, int64_t nb, int n_bits,
-                                   long long words_per_bit, const int* __restrict__ bits_dev,
-                                   unsigned long long* __restrict__ words, SbDeviceState* ds) {
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= nb) return;
-    int l = level[i];
-    if (l >= n_bits) { sb_latch(ds, SB_ERR_INVALID, SBK_PACK); l = n_bits - 1; }
-    words[i] = (unsigned long long)(words_per_bit * bits_dev[l]);
-}
-
 struct PackBits { int bits[8]; };
 
-constexpr float PK_MAGIC = 12582912.f;          // 1.5 * 2^23
-constexpr float PK_TIE_BAND = 0.5f - 1.0f / 4096.0f;
+// block_off[i] = first 32-bit word of block i = exclusive prefix sum of the block sizes
+// (block_rows*block_cols*bits[level] / 32), block_off[nb] = total; one look-back scan.
+constexpr int PO_THREADS = 256, PO_ITEMS = 8, PO_TILE = PO_THREADS * PO_ITEMS;
+__global__ void __launch_bounds__(PO_THREADS)
+pack_offsets_kernel(const unsigned char* __restrict__ level, int64_t nb, int n_bits, PackBits pb,
+                    unsigned long long words_per_bit, unsigned long long* __restrict__ block_off,
+                    LookbackBuf lb, unsigned epoch, SbDeviceState* ds) {
+    const unsigned tile = lookback_tile_id(ds);
+    const int64_t base = (int64_t)tile * PO_TILE + (int64_t)threadIdx.x * PO_ITEMS;
+    unsigned long long v[PO_ITEMS], sum = 0ull;
+#pragma unroll
+    for (int k = 0; k < PO_ITEMS; ++k) {
+        v[k] = 0ull;
+        if (base + k < nb) {
+            int l = level[base + k];
+            if (l >= n_bits) { sb_latch(ds, SB_ERR_INVALID, SBK_PACK); l = n_bits - 1; }
+            int b = pb.bits[0];
+#pragma unroll
+            for (int j = 1; j < 8; ++j) b = (l == j) ? pb.bits[j] : b;
+            v[k] = words_per_bit * (unsigned long long)b;
+        }
+        sum += v[k];
+    }
+    unsigned long long tile_total;
+    const unsigned long long ex = block_exclusive_scan<unsigned long long, PO_THREADS>(sum, tile_total);
+    const unsigned long long prefix = lookback_prefix<unsigned long long>(tile_total, tile, lb, epoch, ds);
+    unsigned long long run = prefix + ex;
+#pragma unroll
+    for (int k = 0; k < PO_ITEMS; ++k) {
+        if (base + k < nb) block_off[base + k] = run;
+        run += v[k];
+    }
+    if (tile == gridDim.x - 1 && threadIdx.x == PO_THREADS - 1) block_off[nb] = run;
+}
 
-// CTA = one block row x one 128-column chunk; a warp takes one row of the chunk at a time, a
-// lane 4 consecutive columns.  Codes are DEFINED by the binary64 sequence
+
+
+constexpr float PK_MAGIC = 12582912.f;          // 1.5 * 2^23
+
+// 16 codes of B bits -> 16*B bits in w[0..3] (little-endian bit stream)
+template <int B>
+__device__ __forceinline__ void pack16(const unsigned (&code)[16], unsigned (&w)[4]) {
+    unsigned long long acc = 0ull;
+    int have = 0, out = 0;
+    w[0] = w[1] = w[2] = w[3] = 0u;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        acc |= (unsigned long long)code[k] << have;
+        have += B;
+        if (have >= 32) {
+            w[out++] = (unsigned)acc;
+            acc >>= 32;
+            have -= 32;
+        }
+    }
+    if (have > 0) w[out] = (unsigned)acc;
+}
+
+// CTA = one block row x one 128-column chunk.  A lane owns 16 consecutive columns (two
+// 16-byte loads), 8 lanes cover a row of the chunk, a warp covers 4 rows per step; the next
+// step's loads are issued before the current rows are encoded.
+//
+// Codes are DEFINED by the binary64 sequence
 //   range = hi - lo; inv = qmax / range; q = rint((v - lo) * inv)
 // but computed in fp32 wherever that provably gives the same integer: the fp32 value of t is
-// within 2^-13 of the fp64 one (t <= 255), so an element farther than 2^-12 from a rounding
+// within 1.8e-7 * qmax of the fp64 one, so an element farther than twice that from a rounding
 // tie keeps its fp32 code, and only rows that contain an element inside that band (exact
 // ties are common with bf16 data) redo those elements in fp64.  The stored scale is
 // fl32(range / qmax): with range exact in fp32 (checked) one correctly rounded fp32 division
 // equals the rounded fp64 quotient (a 24-bit integer over 2^b - 1 has a binary expansion of
 // period <= 8, never within 2^-53 of an fp32 rounding boundary).
+//
+// A lane's 16 codes are 16*b bits: whole words for even b, and for odd b a pair of lanes
+// makes whole words (the even lane also takes the low half-word of its neighbour).
 __global__ void __launch_bounds__(PK_THREADS)
 pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const int32_t* __restrict__ rp,
             int br, int bc, int group, PackBits pb, int n_bits,
             const unsigned char* __restrict__ level, const unsigned long long* __restrict__ off,
             unsigned* __restrict__ packed, long long capacity, float2* __restrict__ meta,
             int64_t n_block_cols, int64_t groups_per_row, SbDeviceState* ds) {
-    __shared__ unsigned stage[PK_WARPS][32];
     __shared__ int s_bits[4];
     __shared__ long long s_base[4];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int cl = lane & 7, slot = lane >> 3;
     const int piece = bc < 128 ? bc : 128;               // columns of one block inside the chunk
-    const int lpp = piece >> 2;                           // lanes (and stage words) per piece
+    const int lpp = piece >> 4;                           // lanes per piece
     const int64_t bi = blockIdx.y;
     const int64_t col0 = (int64_t)blockIdx.x * 128;
     if (threadIdx.x < 128 / piece) {
@@ -62,34 +113,40 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const int32_t* __r
         s_base[threadIdx.x] = (long long)off[blk] + ((c0 - bj * bc) * b) / 32;
     }
     __syncthreads();
-    const int pc = lane / lpp, lp = lane - pc * lpp;
+    const int pc = cl / lpp, lp = cl - pc * lpp;
     const int b = s_bits[pc];
-    const long long base = s_base[pc];
     const long long row_words = (long long)bc * b / 32;
+    // word offset of this lane's bits inside its row piece; odd b: the odd lane starts 16 bits in
+    const long long lane_base = s_base[pc] + (lp * 16 * b) / 32;
+    const bool odd_b = b & 1, odd_lane = lp & 1;
     const float qmaxf = (float)((1 << b) - 1);
-    const int team = group >> 2;                          // lanes per quantisation group
-    const int64_t gcol = (col0 + lane * 4) / group;
-    const bool meta_lane = (lane % team) == 0;
-    const int words = piece * b / 32;                     // words per row of one piece
-    const int bit0 = lp * 4 * b;
-    unsigned* st = &stage[warp][pc * lpp];
+    // |t32 - t64| <= 3 * 2^-24 * t <= 1.8e-7 * qmax: twice that keeps the fp32 code safe
+    const float tie_band = 0.5f - 4.0e-7f * qmaxf - 1.0e-7f;
+    const int team = group >> 4;                          // lanes per quantisation group
+    const int64_t gcol = (col0 + cl * 16) / group;
+    const bool meta_lane = (cl % team) == 0;
+    const __nv_bfloat16* colp = W + col0 + cl * 16;
 
-    int rr = warp;
-    uint2 raw = make_uint2(0u, 0u);
-    if (rr < br) {
+    auto row_ptr = [&](int rr) {
         const int64_t r = bi * br + rr;
-        raw = ld_stream8(W + (rp ? (int64_t)rp[r] : r) * ldw + col0 + lane * 4);
-    }
-    for (; rr < br; rr += PK_WARPS) {
+        return colp + (rp ? (int64_t)rp[r] : r) * ldw;
+    };
+    int rr = warp * 4 + slot;
+    uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0;
+    if (rr < br) { const __nv_bfloat16* p = row_ptr(rr); n0 = ld_stream16(p); n1 = ld_stream16(p + 8); }
+    for (; rr < br; rr += PK_WARPS * 4) {          // br % 4 == 0: a warp step is all or nothing
         const int64_t r = bi * br + rr;
-        const uint2 cur = raw;
-        if (rr + PK_WARPS < br) {                         // prefetch the next row of this warp
-            const int64_t rn = r + PK_WARPS;
-            raw = ld_stream8(W + (rp ? (int64_t)rp[rn] : rn) * ldw + col0 + lane * 4);
+        const uint32_t wv[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
+        if (rr + PK_WARPS * 4 < br) {
+            const __nv_bfloat16* p = row_ptr(rr + PK_WARPS * 4);
+            n0 = ld_stream16(p); n1 = ld_stream16(p + 8);
         }
-        const float v[4] = {bf16lo(cur.x), bf16hi(cur.x), bf16lo(cur.y), bf16hi(cur.y)};
-        float lo = fminf(fminf(v[0], v[1]), fminf(v[2], v[3]));
-        float hi = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3]));
+        float v[16];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { v[2 * k] = bf16lo(wv[k]); v[2 * k + 1] = bf16hi(wv[k]); }
+        float lo = v[0], hi = v[0];
+#pragma unroll
+        for (int k = 1; k < 16; ++k) { lo = fminf(lo, v[k]); hi = fmaxf(hi, v[k]); }
         for (int o = team >> 1; o > 0; o >>= 1) {
             lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
             hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
@@ -97,23 +154,28 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const int32_t* __r
         const double range64 = __dsub_rn((double)hi, (double)lo);     // exact
         const float range = (float)range64;
         const bool exact = (double)range == range64;
-        unsigned code[4] = {0u, 0u, 0u, 0u};
+        unsigned code[16];
         float scale = 0.f;
-        bool redo = false;
         unsigned near = 0u;
+        bool redo = false;
         if (range64 != 0.0) {
             // fp32 fast path (a denormal range overflows the reciprocal: let fp64 handle it)
             const bool fast = range >= 1e-30f;
-            const float inv = fast ? qmaxf / range : 0.f;
+            const float inv = fast ? __fdiv_rn(qmaxf, range) : 0.f;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
+            for (int k = 0; k < 16; ++k) {
                 const float t = (v[k] - lo) * inv;
-                const float q = (t + PK_MAGIC) - PK_MAGIC;
-                code[k] = (unsigned)fminf(fmaxf(q, 0.f), qmaxf);
-                if (!fast || fabsf(t - q) >= PK_TIE_BAND) near |= 1u << k;
+                const float m = t + PK_MAGIC;                 // integer in the low mantissa bits
+                const float q = m - PK_MAGIC;
+                code[k] = __float_as_uint(m) & 0xffu;
+                if (!(fabsf(t - q) < tie_band)) near |= 1u << k;
             }
+            if (!fast) near = 0xffffu;
             scale = __fdiv_rn(range, qmaxf);
             redo = near != 0u || !exact;
+        } else {
+#pragma unroll
+            for (int k = 0; k < 16; ++k) code[k] = 0u;
         }
         if (__any_sync(0xffffffffu, redo)) {
             if (redo) {
@@ -121,7 +183,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const int32_t* __r
                 const double inv = __ddiv_rn(qmax, range64);
                 if (!exact) scale = (float)__ddiv_rn(range64, qmax);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
+                for (int k = 0; k < 16; ++k) {
                     if (near & (1u << k)) {
                         const double t = __dmul_rn(__dsub_rn((double)v[k], dlo), inv);
                         double q = rint(t);                          // round half to even
@@ -132,22 +194,42 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const int32_t* __r
             }
         }
         if (meta_lane) meta[r * groups_per_row + gcol] = make_float2(scale, lo);
-        // a lane's 4 codes go to bit lp*4*b of its piece of the warp's stage
-        stage[warp][lane] = 0;
-        __syncwarp();
-        const unsigned long long chunk = (unsigned long long)code[0] | ((unsigned long long)code[1] << b) |
-                                         ((unsigned long long)code[2] << (2 * b)) |
-                                         ((unsigned long long)code[3] << (3 * b));
-        const unsigned long long sh = chunk << (bit0 & 31);
-        atomicOr(&st[bit0 >> 5], (unsigned)sh);
-        if ((unsigned)(sh >> 32)) atomicOr(&st[(bit0 >> 5) + 1], (unsigned)(sh >> 32));
-        __syncwarp();
-        if (lp < words) {
-            const long long dst = base + (long long)rr * row_words + lp;
-            if (dst < capacity) packed[dst] = st[lp];
-            else sb_latch(ds, SB_ERR_SCRATCH, SBK_PACK);
+        unsigned w[4];
+        switch (b) {
+            case 1: pack16<1>(code, w); break;
+            case 2: pack16<2>(code, w); break;
+            case 3: pack16<3>(code, w); break;
+            case 4: pack16<4>(code, w); break;
+            case 5: pack16<5>(code, w); break;
+            case 6: pack16<6>(code, w); break;
+            case 7: pack16<7>(code, w); break;
+            default: pack16<8>(code, w); break;
         }
-        __syncwarp();
+        // odd b: the pair (even lane, odd lane) holds 32*b bits; the even lane completes its last
+        // word with the neighbour's low half-word, the odd lane drops that half-word
+        const unsigned nb_low = __shfl_down_sync(0xffffffffu, w[0], 1);
+        int nwords = b >> 1;                                  // even b: b/2 whole words
+        if (odd_b) {
+            if (!odd_lane) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (i == (b >> 1)) w[i] |= nb_low << 16;
+                nwords = (b >> 1) + 1;
+            } else {
+#pragma unroll
+                for (int i = 0; i < 3; ++i) w[i] = (w[i] >> 16) | (w[i + 1] << 16);
+                w[3] >>= 16;
+                nwords = b >> 1;
+            }
+        }
+        const long long dst = lane_base + (odd_b && odd_lane ? 1 : 0) + (long long)rr * row_words;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (i < nwords) {
+                if (dst + i < capacity) packed[dst + i] = w[i];
+                else sb_latch(ds, SB_ERR_SCRATCH, SBK_PACK);
+            }
+        }
     }
 }
 
@@ -162,8 +244,8 @@ extern "C" sb_status sb_pack_blocks(sb_ctx* ctx, const void* W, int64_t R, int64
     if (!W || !level || !packed || !block_off_words || !meta || R <= 0 || C <= 0 || capacity_words < 0)
         return sb_fail(ctx, SB_ERR_INVALID, "pack: null or empty");
     if (!sb_check_bits(bits, n_bits)) return sb_fail(ctx, SB_ERR_INVALID, "pack: bits must be ascending in 1..8");
-    const bool g_ok = group == 4 || group == 8 || group == 16 || group == 32 || group == 64 || group == 128;
-    if (br <= 0 || bc <= 0 || R % br || C % bc || !g_ok || bc % group || bc % 32 || C % 128 ||
+    const bool g_ok = group == 16 || group == 32 || group == 64 || group == 128;
+    if (br <= 0 || bc <= 0 || br % 4 || R % br || C % bc || !g_ok || bc % group || bc % 32 || C % 128 ||
         !(bc == 32 || bc == 64 || bc % 128 == 0) || ldw % 8 || ldw < C ||
         (reinterpret_cast<uintptr_t>(W) & 15) || (reinterpret_cast<uintptr_t>(meta) & 7))
         return sb_fail(ctx, SB_ERR_SHAPE, "pack: block %dx%d group %d does not tile %lldx%lld", br, bc,
@@ -173,16 +255,14 @@ extern "C" sb_status sb_pack_blocks(sb_ctx* ctx, const void* W, int64_t R, int64
     SB_CUDA(ctx, cudaSetDevice(ctx->device));
     const int64_t nb = (R / br) * (C / bc);
     const size_t gather_bytes = col_perm ? (size_t)R * C * 2 : 0;
-    void* arena;
-    sb_status st = sb_scratch(ctx, Carver::need({(size_t)nb * 8, 64, gather_bytes}), &arena);
-    if (st != SB_OK) return st;
-    Carver cv(arena);
-    unsigned long long* words = cv.take<unsigned long long>((size_t)nb);
-    int* bits_dev = cv.take<int>(8);
     const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(W);
     int64_t ld = ldw;
     const int32_t* load_rp = row_perm;
     if (col_perm) {
+        void* arena;
+        sb_status st = sb_scratch(ctx, Carver::need({gather_bytes}), &arena);
+        if (st != SB_OK) return st;
+        Carver cv(arena);
         void* g = cv.take<unsigned char>(gather_bytes);
         st = sb_gather_bf16(ctx, W, R, C, ldw, row_perm, col_perm, g);
         if (st != SB_OK) return st;
@@ -192,14 +272,17 @@ extern "C" sb_status sb_pack_blocks(sb_ctx* ctx, const void* W, int64_t R, int64
     }
     PackBits pb{};
     for (int l = 0; l < 8; ++l) pb.bits[l] = l < n_bits ? bits[l] : bits[n_bits - 1];
-    int* hb = reinterpret_cast<int*>(static_cast<char*>(ctx->pinned) + 3072);
-    for (int l = 0; l < 8; ++l) hb[l] = pb.bits[l];
-    SB_CUDA(ctx, cudaMemcpyAsync(bits_dev, hb, 8 * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
-    block_words_kernel<<<(unsigned)((nb + 255) / 256), 256, 0, ctx->stream>>>(
-        level, nb, n_bits, (long long)br * bc / 32, bits_dev, words, ctx->dstate);
-    SB_LAUNCHED(ctx);
-    st = sb_scan_exclusive_u64(ctx, words, reinterpret_cast<unsigned long long*>(block_off_words), nb);
-    if (st != SB_OK) return st;
+    {
+        const unsigned tiles = (unsigned)((nb + PO_TILE - 1) / PO_TILE);
+        unsigned epoch;
+        sb_status st;
+        LookbackBuf lb = sb_lookback(ctx, tiles, &epoch, &st);
+        if (st != SB_OK) return st;
+        pack_offsets_kernel<<<tiles, PO_THREADS, 0, ctx->stream>>>(
+            level, nb, n_bits, pb, (unsigned long long)br * bc / 32,
+            reinterpret_cast<unsigned long long*>(block_off_words), lb, epoch, ctx->dstate);
+        SB_LAUNCHED(ctx);
+    }
     dim3 grid((unsigned)(C / 128), (unsigned)(R / br));
     pack_kernel<<<grid, PK_THREADS, 0, ctx->stream>>>(
         src, ld, load_rp, br, bc, group, pb, n_bits, level,
