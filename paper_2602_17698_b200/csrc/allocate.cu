@@ -92,17 +92,40 @@ __device__ __forceinline__ bool cta_is_last(unsigned* counter) {
 }
 
 // ---- set-up -----------------------------------------------------------------------------
-// keys of all steps e = i (L-1) + l; up list sorts descending (key = ~order), down ascending
-__global__ void step_keys_kernel(AllocArgs a, unsigned long long* kup, unsigned long long* kdn,
-                                 unsigned* vup, unsigned* vdn) {
+// keys of all steps e = i (L-1) + l; the up list sorts by gain descending (key = ~order)
+__global__ void step_keys_kernel(AllocArgs a, unsigned long long* kup, unsigned* vup) {
     const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long n = a.N * (a.L - 1);
     if (e >= n) return;
     const long long i = e / (a.L - 1);
     const int l = (int)(e % (a.L - 1));
     const unsigned long long o = order_key64(gain64(a, i, l, l + 1));
-    kup[e] = ~o; kdn[e] = o;
-    vup[e] = (unsigned)e; vdn[e] = (unsigned)e;
+    kup[e] = ~o;
+    vup[e] = (unsigned)e;
+}
+
+// The down list (gain ascending, ties to the lower step id) is the up list (gain descending,
+// ties to the lower step id) read backwards, except that runs of equal keys keep their order.
+__global__ void tie_heads_kernel(const unsigned long long* __restrict__ keys, long long n,
+                                 unsigned* __restrict__ head) {
+    const long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p < n) head[p] = (p == 0 || keys[p] != keys[p - 1]) ? 1u : 0u;
+}
+__global__ void run_starts_kernel(const unsigned* __restrict__ head, const unsigned* __restrict__ excl,
+                                  long long n, unsigned* __restrict__ start) {
+    const long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= n) return;
+    if (head[p]) start[excl[p]] = (unsigned)p;                    // run id = excl[p]
+    if (p == n - 1) start[excl[p] + head[p]] = (unsigned)n;       // one past the last run
+}
+__global__ void reverse_runs_kernel(const unsigned* __restrict__ up_list, const unsigned* __restrict__ head,
+                                    const unsigned* __restrict__ excl, const unsigned* __restrict__ start,
+                                    long long n, unsigned* __restrict__ dn_list) {
+    const long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= n) return;
+    const unsigned r = excl[p] + head[p] - 1u;
+    const long long a = start[r], b = start[r + 1];
+    dn_list[(n - b) + (p - a)] = up_list[p];
 }
 
 // level = l0 everywhere; loss / used partial sums; also clears the per-block stamps
@@ -620,12 +643,20 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
         report->proxy_loss_init = 0.0;
         if (nsteps > 0) {
             const unsigned g = (unsigned)((nsteps + 255) / 256);
-            step_keys_kernel<<<g, 256, 0, ctx->stream>>>(a, kA, kC, vA, vC);
+            step_keys_kernel<<<g, 256, 0, ctx->stream>>>(a, kA, vA);
             SB_LAUNCHED(ctx);
             stt = sb_radix_sort_u64(ctx, kA, kB, vA, vB, nsteps, sort_scratch);
             if (stt != SB_OK) return stt;
-            stt = sb_radix_sort_u64(ctx, kC, kD, vC, vD, nsteps, sort_scratch);
+            // down list = up list reversed run by run (vB: heads, vD: their prefix, kB: run starts)
+            unsigned* run_start = reinterpret_cast<unsigned*>(kB);
+            tie_heads_kernel<<<g, 256, 0, ctx->stream>>>(kA, nsteps, vB);
+            SB_LAUNCHED(ctx);
+            stt = sb_scan_exclusive_u32(ctx, vB, vD, nsteps);
             if (stt != SB_OK) return stt;
+            run_starts_kernel<<<g, 256, 0, ctx->stream>>>(vB, vD, nsteps, run_start);
+            SB_LAUNCHED(ctx);
+            reverse_runs_kernel<<<g, 256, 0, ctx->stream>>>(vA, vB, vD, run_start, nsteps, vC);
+            SB_LAUNCHED(ctx);
             // the whole loop in one cooperative launch
             int occ = 0;
             SB_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scalebits_loop_kernel, LT, 0));

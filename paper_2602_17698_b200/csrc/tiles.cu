@@ -150,7 +150,7 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // ---- block scores ------------------------------------------------------------------------
 // Every WARP is autonomous: it walks its own units (a block, or a 32-row part of one), stages
 // its own 16-row slabs of the 128-column chunk in its own shared-memory ring with asynchronous
-// 16-byte copies (two slabs per warp, 64 KB in flight per SM), and synchronises with nobody
+// 16-byte copies (three slabs per warp, two of them in flight: 128 KB per SM), and synchronises with nobody
 // but itself.  Without CTA barriers the warps of an SM drift apart, so the integer/shuffle
 // phase of one warp (group min/max, unpacking) overlaps the FP32 phase of another.  A lane
 // owns CPL consecutive columns of the chunk; 128/CPL lanes cover a row, a warp covers
@@ -167,9 +167,12 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // reciprocal, so that the accumulated square carries a_r without any per-candidate work.
 constexpr int SLAB_ROWS = 16;
 constexpr int SLAB_BYTES = SLAB_ROWS * 256;
+constexpr int SC_THREADS = 512;                 // one CTA of 16 warps per SM
+constexpr int SC_WARPS = SC_THREADS / 32;
+constexpr int RING = 3;                         // slabs per warp: one being read, two in flight
 
 template <int L, int CPL, int NFINE, bool FULLG, bool ROWW>
-__global__ void __launch_bounds__(CTA_THREADS, 2)
+__global__ void __launch_bounds__(SC_THREADS, 1)
 block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
                     const int32_t* __restrict__ load_row_perm,   // rows gathered at load time
                     const int32_t* __restrict__ c_perm,          // original column of permuted j
@@ -192,20 +195,22 @@ block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
     const int lanes_per_sub = bc >= TILE_COLS ? LANE_COLS : bc / CPL;    // lanes across one block
     const int nsub = bc >= TILE_COLS ? 1 : TILE_COLS / bc;
     const int slabs = (part_rows + SLAB_ROWS - 1) / SLAB_ROWS;           // per chunk of a unit
-    unsigned char* ring = tile_smem + (size_t)warp * (2 * SLAB_BYTES);
+    unsigned char* ring = tile_smem + (size_t)warp * (RING * SLAB_BYTES);
     // this lane's share of a slab: 16-byte piece g of rows g_row, g_row + 2, ...
     const int g = lane & 15, g_row = lane >> 4;
     const int g_dst = g_row * 256 + (g % PIECES) * (LANE_COLS * 16) + (g / PIECES) * 16;
     const int my_off = slot * 256 + cl * 16;
-    const int64_t warp_id = (int64_t)blockIdx.x * CTA_WARPS + warp;
-    const int64_t warp_stride = (int64_t)gridDim.x * CTA_WARPS;
+    const int64_t warp_id = (int64_t)blockIdx.x * SC_WARPS + warp;
+    const int64_t warp_stride = (int64_t)gridDim.x * SC_WARPS;
 
     // stage slab `sl` of chunk `ch` of unit `u` (rows beyond the part are skipped)
-    auto issue = [&](int64_t u, int ch, int sl, int stage) {
-        const int64_t t = u / parts;
-        const int64_t row0 = t / n_tile_cols * br + (int64_t)(u % parts) * part_rows + sl * SLAB_ROWS;
+    // (all index arithmetic is 32-bit: units, tiles and rows are far below 2^31)
+    const unsigned u_parts = (unsigned)parts, u_tcols = (unsigned)n_tile_cols;
+    auto issue = [&](unsigned u, int ch, int sl, int stage) {
+        const unsigned t = u / u_parts, by = t / u_tcols;
+        const int64_t row0 = (int64_t)(by * (unsigned)br + (u - t * u_parts) * (unsigned)part_rows + sl * SLAB_ROWS);
         const int rows_here = min(SLAB_ROWS, part_rows - sl * SLAB_ROWS);
-        const __nv_bfloat16* src = W + t % n_tile_cols * tile_w + (int64_t)ch * TILE_COLS + g * 8;
+        const __nv_bfloat16* src = W + (int64_t)((t - by * u_tcols) * (unsigned)tile_w + ch * TILE_COLS + g * 8);
         unsigned char* dst = ring + stage * SLAB_BYTES + g_dst;
         if (load_row_perm) {
             const int32_t* rp = load_row_perm + row0;
@@ -219,14 +224,27 @@ block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
         cp_async_commit();
     };
 
+    // issue cursor: RING - 1 slabs ahead of the slab being evaluated
+    int64_t i_unit = warp_id;
+    int i_ch = 0, i_sl = 0, i_stage = 0;
+    auto issue_next = [&]() {
+        if (i_unit < n_units) {
+            issue((unsigned)i_unit, i_ch, i_sl, i_stage);
+            if (++i_sl == slabs) { i_sl = 0; if (++i_ch == chunks) { i_ch = 0; i_unit += warp_stride; } }
+        } else {
+            cp_async_commit();            // keep one group per step so the wait count stays fixed
+        }
+        i_stage = i_stage + 1 == RING ? 0 : i_stage + 1;
+    };
+#pragma unroll
+    for (int i = 0; i < RING - 1; ++i) issue_next();
+
     int stage = 0;
-    int64_t unit = warp_id;
-    if (unit < n_units) issue(unit, 0, 0, 0);
-    for (; unit < n_units; unit += warp_stride) {
-        const int64_t t = unit / parts;
-        const int p = (int)(unit % parts);
-        const int64_t row_base = t / n_tile_cols * br + (int64_t)p * part_rows;
-        const int64_t colT = t % n_tile_cols * tile_w;
+    for (int64_t unit = warp_id; unit < n_units; unit += warp_stride) {
+        const unsigned t = (unsigned)unit / u_parts, by = t / u_tcols, bx = t - by * u_tcols;
+        const int p = (int)((unsigned)unit - t * u_parts);
+        const int64_t row_base = (int64_t)(by * (unsigned)br + (unsigned)p * (unsigned)part_rows);
+        const int64_t colT = (int64_t)(bx * (unsigned)tile_w);
         f32x2 tot2[L];
 #pragma unroll
         for (int l = 0; l < L; ++l) tot2[l] = 0ull;
@@ -238,13 +256,10 @@ block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
 #pragma unroll
                 for (int l = 0; l < L; ++l) acc[k][l] = 0ull;
 
-            for (int sl = 0; sl < slabs; ++sl, stage ^= 1) {
-                // keep the next slab in flight, then wait for this one
-                if (sl + 1 < slabs) issue(unit, ch, sl + 1, stage ^ 1);
-                else if (ch + 1 < chunks) issue(unit, ch + 1, 0, stage ^ 1);
-                else if (unit + warp_stride < n_units) issue(unit + warp_stride, 0, 0, stage ^ 1);
-                else cp_async_commit();
-                cp_async_wait<1>();
+            for (int sl = 0; sl < slabs; ++sl, stage = stage + 1 == RING ? 0 : stage + 1) {
+                // refill the stage read in the previous step, then wait for this slab
+                issue_next();
+                cp_async_wait<RING - 1>();
                 __syncwarp();
                 const unsigned char* src = ring + stage * SLAB_BYTES + my_off;
                 const int rows_here = min(SLAB_ROWS, part_rows - sl * SLAB_ROWS);
@@ -331,7 +346,7 @@ block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
         }
         if (slot == 0 && (cl % lanes_per_sub) == 0) {
             const int sb = cl / lanes_per_sub;
-            const int64_t blk = t / n_tile_cols * n_block_cols + t % n_tile_cols * nsub + sb;
+            const int64_t blk = (int64_t)by * n_block_cols + (int64_t)(bx * (unsigned)nsub + (unsigned)sb);
             float* dst = part_out + ((int64_t)p * n_blocks + blk) * L;
 #pragma unroll
             for (int l = 0; l < L; ++l) dst[l] = tot[l];
@@ -527,17 +542,17 @@ sb_status launch_scores_k(sb_ctx* ctx, const __nv_bfloat16* W, int64_t ldw, cons
     const int part_rows = br % 32 == 0 ? 32 : br;
     const int parts = br / part_rows;
     const int64_t n_units = (R / br) * n_tile_cols * parts;
-    const size_t smem = (size_t)CTA_WARPS * 2 * SLAB_BYTES;
+    const size_t smem = (size_t)SC_WARPS * RING * SLAB_BYTES;
     auto kern = block_scores_kernel<L, CPL, NFINE, FULLG, ROWW>;
     static bool attr_done = false;
     if (!attr_done) {
         SB_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attr_done = true;
     }
-    int64_t grid = (int64_t)ctx->sm_count * 2;      // persistent: two CTAs per SM
-    const int64_t need = (n_units + CTA_WARPS - 1) / CTA_WARPS;
+    int64_t grid = ctx->sm_count;                   // persistent: one 16-warp CTA per SM
+    const int64_t need = (n_units + SC_WARPS - 1) / SC_WARPS;
     if (grid > need) grid = need;
-    kern<<<(unsigned)grid, CTA_THREADS, smem, ctx->stream>>>(
+    kern<<<(unsigned)grid, SC_THREADS, smem, ctx->stream>>>(
         W, ldw, lrp, cperm, aperm, cm, rw, br, bc, group, ba, nbc, n_tile_cols, parts, part_rows, n_units,
         n_blocks, part_buf);
     SB_LAUNCHED(ctx);
