@@ -166,6 +166,23 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ---- multi-rank plumbing (replicas: every rank searches its own layer, no data-path collective) --
+def max_over_ranks(x: float, world: int, device=None) -> float:
+    """The slowest rank's time: what the whole job waits for."""
+    if world <= 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(units_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job units per second: all ranks' units over the slowest rank's step time."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
+
+
 # ---- the CUDA path ------------------------------------------------------------------------------
 STAGES = ("moments", "reorder_stats", "sort", "scores", "allocate", "pack")
 
@@ -175,7 +192,7 @@ def run_cuda(args):
     import torch.distributed as dist
     from paper_2602_17698_b200 import synth
     from paper_2602_17698_b200.binding import Context
-    from paper_2602_17698_b200.pipeline import LayerWorkspace, SearchConfig, search_layer
+    from paper_2602_17698_b200.pipeline import LayerWorkspace, SearchConfig, StageGraphs, search_layer
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -192,8 +209,14 @@ def run_cuda(args):
     # replicas: every rank searches its own layer (layer index = rank), no data-path collective
     W = synth.make_layer_weights(shape, SEED, rank, dev)
     X = synth.make_layer_activations(shape, TOKENS, SEED, rank, dev)
+    # the library works on one non-default stream, so that its stages can be captured into
+    # CUDA graphs (fixed pointers: the workspace and the inputs) and replayed without host gaps
+    stream = torch.cuda.Stream(device=dev)
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(stream)
     ctx = Context()
     ws = LayerWorkspace(shape, cfg, dev)
+    graphs = None if args.no_graphs else StageGraphs(ctx)
     n_weights = shape.n_weights
     in_bytes = sum(w.numel() * 2 for w in W.values()) + sum(x.numel() * 2 for x in X.values())
 
@@ -203,7 +226,7 @@ def run_cuda(args):
         torch.cuda.synchronize()
 
     def step(timers=None):
-        return search_layer(ctx, W, X, ws, timers=timers)
+        return search_layer(ctx, W, X, ws, timers=timers, graphs=graphs)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -215,7 +238,7 @@ def run_cuda(args):
         sampler.start()
         time.sleep(0.15)
     timers = {s: [] for s in STAGES}
-    l0 = ctx.kernel_launches()
+    l0 = ctx.kernel_launches() + (graphs.replayed_kernels if graphs else 0)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     t_wall0 = time.time()
@@ -225,15 +248,12 @@ def run_cuda(args):
     e1.record()
     barrier()
     t_wall1 = time.time()
-    launches = ctx.kernel_launches() - l0
+    launches = ctx.kernel_launches() + (graphs.replayed_kernels if graphs else 0) - l0
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
-    tmax = torch.tensor([ms], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-    ms = float(tmax.item())
+    ms = max_over_ranks(ms, world, dev)
     ms_per_step = ms / args.steps
-    value = world * n_weights / (ms_per_step * 1e-3)
+    value = job_throughput(n_weights, world, ms_per_step)
 
     stage_ms = {s: sum(a.elapsed_time(b) for a, b in timers[s]) / args.steps for s in STAGES}
     stage_launch_ms = {s: (sum(a.elapsed_time(b) for a, b in timers[s]) / max(len(timers[s]), 1))
@@ -270,11 +290,8 @@ def run_cuda(args):
             e2e_step()
         b.record()
         barrier()
-        t = torch.tensor([a.elapsed_time(b)], device=dev, dtype=torch.float64)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item()) / e2e_steps
-        e2e = {"value": world * n_weights / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+        e2e_ms = max_over_ranks(a.elapsed_time(b), world, dev) / e2e_steps
+        e2e = {"value": job_throughput(n_weights, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                "steps": e2e_steps, "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": d2h}
 
     if rank == 0:
@@ -304,6 +321,7 @@ def run_cuda(args):
                 "config": {"workload": WORKLOAD, "tokens": TOKENS, "bits": list(BITS), "budget": BUDGET,
                            "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                            "l2": "inputs (3.9 GB per step) larger than L2, no flush needed",
+                           "launch": "eager" if graphs is None else "one CUDA graph per stage (allocation eager)",
                            "allocation": res.report},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
                 "roofline": roofline, "cpu_baseline": cpu,
@@ -324,6 +342,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graphs", action="store_true", help="launch every library call eagerly")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

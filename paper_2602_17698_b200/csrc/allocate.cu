@@ -24,6 +24,7 @@ constexpr int BT = 256;             // threads of the per-block kernels
 constexpr int LT = 256;             // threads of the persistent loop kernel
 constexpr int LT_WARPS_MAX = LT / 32;
 constexpr int LOOP_MAX_CTAS = 4096;
+constexpr int LC = 4;               // list entries a thread keeps in registers between passes
 
 struct AllocState {
     long long cap, used;
@@ -235,14 +236,28 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
         const long long slack = cap - used;
         const long long h = k / 2 > 0 ? k / 2 : 1;
 
-        // ---- up-count -------------------------------------------------------------------------
+        // ---- up-count (a thread with at most LC entries keeps them for the rank pass) -----------
         CntCost mine{0ull, 0u, 0u};
         long long my_first = -1;
-        for (long long p = t_lo; p < t_hi; ++p) {
-            unsigned long long cost; double de;
-            if (up_entry(p, cost, de) >= 0) {
-                if (mine.cnt == 0) my_first = (long long)cost;
-                mine.cnt += 1; mine.cost += cost;
+        long long c_blk[LC]; unsigned long long c_cost[LC]; double c_de[LC];
+        const bool cached = ipt <= LC;
+        if (cached) {
+#pragma unroll
+            for (int j = 0; j < LC; ++j) {
+                c_blk[j] = -1; c_cost[j] = 0; c_de[j] = 0.0;
+                if (t_lo + j < t_hi) c_blk[j] = up_entry(t_lo + j, c_cost[j], c_de[j]);
+                if (c_blk[j] >= 0) {
+                    if (mine.cnt == 0) my_first = (long long)c_cost[j];
+                    mine.cnt += 1; mine.cost += c_cost[j];
+                }
+            }
+        } else {
+            for (long long p = t_lo; p < t_hi; ++p) {
+                unsigned long long cost; double de;
+                if (up_entry(p, cost, de) >= 0) {
+                    if (mine.cnt == 0) my_first = (long long)cost;
+                    mine.cnt += 1; mine.cost += cost;
+                }
             }
         }
         CntCost cta_tot;
@@ -281,10 +296,7 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
         if ((long long)pre_cnt + ex.cnt < lim_rank) {
             unsigned long long run_cost = pre_cost + ex.cost;
             long long run_cnt = (long long)pre_cnt + ex.cnt;
-            for (long long p = t_lo; p < t_hi && run_cnt < lim_rank; ++p) {
-                unsigned long long cost; double de;
-                const long long i = up_entry(p, cost, de);
-                if (i < 0) continue;
+            auto take = [&](long long i, unsigned long long cost, double de) {
                 run_cost += cost;
                 a.uprank[i] = (unsigned)run_cnt;
                 a.upcum[i] = run_cost;
@@ -294,6 +306,17 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
                     dU_mine += de; costU_mine += cost; nU_mine += 1;
                 }
                 run_cnt += 1;
+            };
+            if (cached) {
+#pragma unroll
+                for (int j = 0; j < LC; ++j)
+                    if (c_blk[j] >= 0 && run_cnt < lim_rank) take(c_blk[j], c_cost[j], c_de[j]);
+            } else {
+                for (long long p = t_lo; p < t_hi && run_cnt < lim_rank; ++p) {
+                    unsigned long long cost; double de;
+                    const long long i = up_entry(p, cost, de);
+                    if (i >= 0) take(i, cost, de);
+                }
             }
         }
         if (expand) {
@@ -661,8 +684,9 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
             int occ = 0;
             SB_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scalebits_loop_kernel, LT, 0));
             long long G = (long long)occ * ctx->sm_count;
-            const long long want = (nsteps + 4 * LT - 1) / (4 * LT) > (N + 4 * LT - 1) / (4 * LT)
-                                       ? (nsteps + 4 * LT - 1) / (4 * LT) : (N + 4 * LT - 1) / (4 * LT);
+            // a few list entries per thread: grid barriers cost more with more CTAs than the
+            // short passes gain
+            const long long want = (nsteps + LC * LT - 1) / (LC * LT);
             if (G > want) G = want;
             if (G > LOOP_MAX_CTAS) G = LOOP_MAX_CTAS;
             if (G < 1) G = 1;

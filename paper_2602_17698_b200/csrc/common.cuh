@@ -12,7 +12,7 @@ struct SbDeviceState {           // lives in device memory, one per context
     int status;                  // latched sb_status detected on the device
     int where;                   // kernel id that latched it
     unsigned int ticket;         // dynamic tile ids of the look-back scans
-    unsigned int pad;
+    unsigned int pad;            // CTAs of the current look-back launch that have finished
 };
 
 struct sb_ctx {
@@ -24,7 +24,6 @@ struct sb_ctx {
     SbDeviceState* dstate = nullptr;
     void* pinned = nullptr;      // small pinned host buffer for read-backs
     size_t pinned_bytes = 0;
-    unsigned int scan_epoch = 0; // tags look-back descriptors so they need no clearing
     void* lb_mem = nullptr;      // look-back descriptors (context-owned, never in the arena)
     unsigned int lb_max_tiles = 0;
     int64_t launches = 0;

@@ -12,13 +12,13 @@ struct CntCost {                       // (how many selected before me, their su
     unsigned pad;
 };
 
-struct LookbackBuf {                   // context-owned, zeroed once, tagged by epoch afterwards
-    unsigned* flags;                   // [max_tiles]  (epoch << 2) | state
+struct LookbackBuf {                   // context-owned; all flags are zero between launches
+    unsigned* flags;                   // [max_tiles]  0 = empty, 1 = aggregate, 2 = inclusive
     unsigned char* agg;                // [max_tiles] * 16 bytes
     unsigned char* inc;                // [max_tiles] * 16 bytes
     unsigned max_tiles;
 };
-LookbackBuf sb_lookback(sb_ctx* ctx, unsigned tiles, unsigned* epoch_out, sb_status* st);
+LookbackBuf sb_lookback(sb_ctx* ctx, unsigned tiles, sb_status* st);
 
 #ifdef __CUDACC__
 constexpr unsigned LB_AGG = 1u, LB_INC = 2u;
@@ -88,35 +88,47 @@ __device__ __forceinline__ T block_exclusive_scan(T v, T& block_total) {
 __device__ __forceinline__ unsigned lookback_tile_id(SbDeviceState* st) {
     __shared__ unsigned tile_sh;
     if (threadIdx.x == 0) {
-        tile_sh = atomicAdd(&st->ticket, 1u);
-        if (tile_sh == gridDim.x - 1) st->ticket = 0u;   // every ticket has been drawn
+        tile_sh = atomicAdd(&st->ticket, 1u);             // reset by lookback_finish
     }
     __syncthreads();
     return tile_sh;
 }
 
+// Call from all threads at the very end of a look-back kernel: the last CTA to get here clears
+// the descriptors this launch used and the tile ticket, so the next launch (stream order)
+// starts from zeroed flags.  No host-side state is involved: a captured launch can be replayed.
+__device__ __forceinline__ void lookback_finish(SbDeviceState* st, LookbackBuf lb) {
+    __shared__ bool last_sh;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last_sh = atomicAdd(&st->pad, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (last_sh) {
+        for (unsigned t = threadIdx.x; t < gridDim.x; t += blockDim.x) lb.flags[t] = 0u;
+        if (threadIdx.x == 0) { st->pad = 0u; st->ticket = 0u; }
+    }
+}
+
 // exclusive prefix of this tile's aggregate over all earlier tiles; call from all threads
 template <typename T>
-__device__ __forceinline__ T lookback_prefix(T aggregate, unsigned tile, LookbackBuf lb, unsigned epoch,
-                                             SbDeviceState* st) {
+__device__ __forceinline__ T lookback_prefix(T aggregate, unsigned tile, LookbackBuf lb, SbDeviceState* st) {
     __shared__ T prefix_sh;
     T* aggs = reinterpret_cast<T*>(lb.agg);
     T* incs = reinterpret_cast<T*>(lb.inc);
-    const unsigned tag = epoch << 2;
     if (threadIdx.x < 32) {
         const int lane = threadIdx.x;
         if (tile == 0) {
             if (lane == 0) {
                 incs[0] = aggregate;
                 __threadfence();
-                st_release_u32(lb.flags, tag | LB_INC);
+                st_release_u32(lb.flags, LB_INC);
                 prefix_sh = t_zero((T*)nullptr);
             }
         } else {
             if (lane == 0) {
                 aggs[tile] = aggregate;
                 __threadfence();
-                st_release_u32(lb.flags + tile, tag | LB_AGG);
+                st_release_u32(lb.flags + tile, LB_AGG);
             }
             T running = t_zero((T*)nullptr);
             int base = (int)tile - 1;
@@ -129,7 +141,7 @@ __device__ __forceinline__ T lookback_prefix(T aggregate, unsigned tile, Lookbac
                     unsigned f = ld_acquire_u32(lb.flags + t);
                     unsigned long long t_start = 0;
                     int spins = 0;
-                    while ((f >> 2) != epoch || (f & 3u) == 0u) {
+                    while ((f & 3u) == 0u) {
                         // bounded wait: a predecessor that never publishes must not hang the GPU
                         if ((++spins & 63) == 0) {
                             const unsigned long long now = lb_now_ns();
@@ -155,7 +167,7 @@ __device__ __forceinline__ T lookback_prefix(T aggregate, unsigned tile, Lookbac
             if (lane == 0) {
                 incs[tile] = t_add(running, aggregate);
                 __threadfence();
-                st_release_u32(lb.flags + tile, tag | LB_INC);
+                st_release_u32(lb.flags + tile, LB_INC);
                 prefix_sh = running;
             }
         }

@@ -20,7 +20,7 @@ constexpr int PO_THREADS = 256, PO_ITEMS = 8, PO_TILE = PO_THREADS * PO_ITEMS;
 __global__ void __launch_bounds__(PO_THREADS)
 pack_offsets_kernel(const unsigned char* __restrict__ level, int64_t nb, int n_bits, PackBits pb,
                     unsigned long long words_per_bit, unsigned long long* __restrict__ block_off,
-                    LookbackBuf lb, unsigned epoch, SbDeviceState* ds) {
+                    LookbackBuf lb, SbDeviceState* ds) {
     const unsigned tile = lookback_tile_id(ds);
     const int64_t base = (int64_t)tile * PO_TILE + (int64_t)threadIdx.x * PO_ITEMS;
     unsigned long long v[PO_ITEMS], sum = 0ull;
@@ -39,7 +39,7 @@ pack_offsets_kernel(const unsigned char* __restrict__ level, int64_t nb, int n_b
     }
     unsigned long long tile_total;
     const unsigned long long ex = block_exclusive_scan<unsigned long long, PO_THREADS>(sum, tile_total);
-    const unsigned long long prefix = lookback_prefix<unsigned long long>(tile_total, tile, lb, epoch, ds);
+    const unsigned long long prefix = lookback_prefix<unsigned long long>(tile_total, tile, lb, ds);
     unsigned long long run = prefix + ex;
 #pragma unroll
     for (int k = 0; k < PO_ITEMS; ++k) {
@@ -47,6 +47,7 @@ pack_offsets_kernel(const unsigned char* __restrict__ level, int64_t nb, int n_b
         run += v[k];
     }
     if (tile == gridDim.x - 1 && threadIdx.x == PO_THREADS - 1) block_off[nb] = run;
+    lookback_finish(ds, lb);
 }
 
 
@@ -274,13 +275,12 @@ extern "C" sb_status sb_pack_blocks(sb_ctx* ctx, const void* W, int64_t R, int64
     for (int l = 0; l < 8; ++l) pb.bits[l] = l < n_bits ? bits[l] : bits[n_bits - 1];
     {
         const unsigned tiles = (unsigned)((nb + PO_TILE - 1) / PO_TILE);
-        unsigned epoch;
         sb_status st;
-        LookbackBuf lb = sb_lookback(ctx, tiles, &epoch, &st);
+        LookbackBuf lb = sb_lookback(ctx, tiles, &st);
         if (st != SB_OK) return st;
         pack_offsets_kernel<<<tiles, PO_THREADS, 0, ctx->stream>>>(
             level, nb, n_bits, pb, (unsigned long long)br * bc / 32,
-            reinterpret_cast<unsigned long long*>(block_off_words), lb, epoch, ctx->dstate);
+            reinterpret_cast<unsigned long long*>(block_off_words), lb, ctx->dstate);
         SB_LAUNCHED(ctx);
     }
     dim3 grid((unsigned)(C / 128), (unsigned)(R / br));

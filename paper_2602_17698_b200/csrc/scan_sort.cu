@@ -12,7 +12,7 @@ constexpr int SCAN_TILE = SCAN_THREADS * SCAN_ITEMS;
 template <typename T>
 __global__ void __launch_bounds__(SCAN_THREADS)
 scan_exclusive_kernel(const T* __restrict__ in, T* __restrict__ out, int64_t n, int write_total,
-                      LookbackBuf lb, unsigned epoch, SbDeviceState* st) {
+                      LookbackBuf lb, SbDeviceState* st) {
     const unsigned tile = lookback_tile_id(st);
     const int64_t base = (int64_t)tile * SCAN_TILE + (int64_t)threadIdx.x * SCAN_ITEMS;
     T v[SCAN_ITEMS];
@@ -24,7 +24,7 @@ scan_exclusive_kernel(const T* __restrict__ in, T* __restrict__ out, int64_t n, 
     }
     T tile_total;
     T ex = block_exclusive_scan<T, SCAN_THREADS>(sum, tile_total);
-    const T prefix = lookback_prefix<T>(tile_total, tile, lb, epoch, st);
+    const T prefix = lookback_prefix<T>(tile_total, tile, lb, st);
     T run = t_add(prefix, ex);
 #pragma unroll
     for (int k = 0; k < SCAN_ITEMS; ++k) {
@@ -32,6 +32,7 @@ scan_exclusive_kernel(const T* __restrict__ in, T* __restrict__ out, int64_t n, 
         run = t_add(run, v[k]);
     }
     if (write_total && tile == gridDim.x - 1 && threadIdx.x == SCAN_THREADS - 1) out[n] = run;
+    lookback_finish(st, lb);
 }
 
 // ---- radix sort ---------------------------------------------------------------------------
@@ -118,14 +119,10 @@ radix_scatter_kernel(const unsigned long long* __restrict__ keys_in, const unsig
 
 }  // namespace
 
-// A fresh tag for the next look-back launch, and descriptors for `tiles` tiles.  The
-// descriptors are recognised by their tag, so they are zeroed only when the buffer is
-// (re)allocated or the 30-bit tag wraps.
-LookbackBuf sb_lookback(sb_ctx* ctx, unsigned tiles, unsigned* epoch_out, sb_status* st) {
+// Descriptors for `tiles` tiles.  Every look-back kernel leaves its flags zeroed, so the
+// buffer is cleared only when it is (re)allocated.
+LookbackBuf sb_lookback(sb_ctx* ctx, unsigned tiles, sb_status* st) {
     *st = SB_OK;
-    ctx->scan_epoch++;
-    bool rezero = false;
-    if (ctx->scan_epoch >= (1u << 30)) { ctx->scan_epoch = 1; rezero = true; }
     if (tiles > ctx->lb_max_tiles) {
         unsigned want = 1u << 14;
         while (want < tiles) want <<= 1;
@@ -139,16 +136,14 @@ LookbackBuf sb_lookback(sb_ctx* ctx, unsigned tiles, unsigned* epoch_out, sb_sta
             return LookbackBuf{};
         }
         ctx->lb_max_tiles = want;
-        rezero = true;
+        cudaMemsetAsync(ctx->lb_mem, 0, (size_t)ctx->lb_max_tiles * 36, ctx->stream);
     }
-    if (rezero) cudaMemsetAsync(ctx->lb_mem, 0, (size_t)ctx->lb_max_tiles * 36, ctx->stream);
     LookbackBuf lb;
     unsigned char* p = static_cast<unsigned char*>(ctx->lb_mem);
     lb.agg = p;
     lb.inc = p + (size_t)ctx->lb_max_tiles * 16;
     lb.flags = reinterpret_cast<unsigned*>(p + (size_t)ctx->lb_max_tiles * 32);
     lb.max_tiles = ctx->lb_max_tiles;
-    *epoch_out = ctx->scan_epoch;
     return lb;
 }
 
@@ -160,11 +155,10 @@ static sb_status scan_launch(sb_ctx* ctx, const T* in, T* out, int64_t n, int wr
     }
     const unsigned tiles = (unsigned)((n + SCAN_TILE - 1) / SCAN_TILE);
     sb_status st;
-    unsigned epoch;
-    LookbackBuf lb = sb_lookback(ctx, tiles, &epoch, &st);
+    LookbackBuf lb = sb_lookback(ctx, tiles, &st);
     if (st != SB_OK) return st;
     scan_exclusive_kernel<T><<<tiles, SCAN_THREADS, 0, ctx->stream>>>(
-        in, out, n, write_total, lb, epoch, ctx->dstate);
+        in, out, n, write_total, lb, ctx->dstate);
     SB_LAUNCHED(ctx);
     return SB_OK;
 }

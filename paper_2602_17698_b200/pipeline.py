@@ -127,14 +127,51 @@ class _Timed:
             self.timers[self.stage].append((self.a, self.b))
 
 
+class StageGraphs:
+    """CUDA graphs of the stages of one (workspace, weights, activations) binding.
+
+    Every pointer a stage uses is fixed (the workspace and the input tensors), so the stage's
+    library calls can be captured once on the context's stream and replayed: the kernels then
+    run back to back without per-call host overhead.  The allocation stays eager (it reads its
+    report back to the host).  The context must live on a non-default stream.
+    """
+
+    def __init__(self, ctx: Context):
+        self.ctx, self.graphs, self.kernels = ctx, {}, {}
+        self.replayed_kernels = 0          # kernels launched through graph replays so far
+
+    def run(self, stage: str, fn):
+        g = self.graphs.get(stage)
+        if g is None:
+            fn()                                   # eager once: scratch growth, attributes
+            self.ctx.stream.synchronize()
+            g = torch.cuda.CUDAGraph()
+            n0 = self.ctx.kernel_launches()
+            with torch.cuda.graph(g, stream=self.ctx.stream):
+                fn()
+            self.kernels[stage] = self.ctx.kernel_launches() - n0
+            self.graphs[stage] = g
+        g.replay()
+        self.replayed_kernels += self.kernels[stage]
+
+
 def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str, torch.Tensor],
                  ws: LayerWorkspace, allocate: bool = True, pack: bool = True,
-                 timers: Optional[dict] = None) -> LayerResult:
+                 timers: Optional[dict] = None, graphs: Optional[StageGraphs] = None) -> LayerResult:
     """moments -> reorder statistics -> permutations -> block scores -> allocation -> pack.
 
     `timers`, if given, maps the stage names moments / reorder_stats / sort / scores /
-    allocate / pack to lists that receive one (start, end) CUDA event pair per library call.
+    allocate / pack to lists that receive one (start, end) CUDA event pair per stage (per
+    library call for the moments, whose launches the roofline accounting needs).
+    `graphs`, if given, replays each stage from a CUDA graph captured on first use.
     """
+    def stage(name, fn):
+        with _Timed(timers, name):
+            if graphs is not None:
+                graphs.run(name, fn)
+            else:
+                fn()
+
     shape, cfg = ws.shape, ws.cfg
     lin = {l.name: l for l in shape.linears}
     g, rb = cfg.group, cfg.ref_bits
@@ -144,8 +181,12 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
 
     # a1: calibration second moments, one per distinct linear input
     for name, X in acts.items():
-        with _Timed(timers, "moments"):
-            ctx.calib_moments(X, ws.moments[name])
+        if graphs is not None:
+            with _Timed(timers, "moments"):
+                graphs.run("moments:" + name, lambda X=X, name=name: ctx.calib_moments(X, ws.moments[name]))
+        else:
+            with _Timed(timers, "moments"):
+                ctx.calib_moments(X, ws.moments[name])
     c = {n: ws.moments[l.act] for n, l in lin.items()}
 
     perms = {"hidden": None, "intermediate": None, "v_heads": None, "o_heads": None}
@@ -162,11 +203,12 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
             ("down_proj", dict(row_score=ws.hid_score, col_score=ws.mid_score, accumulate_row=True,
                                accumulate_col=True)),
         ]
-        for name, kw in stats:
-            with _Timed(timers, "reorder_stats"):
+        def do_stats():
+            for name, kw in stats:
                 ctx.reorder_channels(W[name], c[name], rb, g, **kw)
+
         # a3: one sort per coupled channel set ("sort only" calls: W = NULL)
-        with _Timed(timers, "sort"):
+        def do_sort():
             ctx.fold_segment_scores(ws.vo_score, ws.o_col_score, reps, hd)
             ctx.reorder_channels(None, None, rb, g, row_score=ws.hid_score, row_segment=shape.hidden,
                                  row_perm=ws.p_hid, shape=(shape.hidden, g))
@@ -176,6 +218,9 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
             ctx.reorder_channels(None, None, rb, g, row_score=ws.vo_score, row_segment=hd,
                                  row_perm=ws.p_v, shape=(ws.vo_score.numel(), g))
             ctx.expand_segment_perm(ws.p_v, reps, hd, out=ws.p_o)
+
+        stage("reorder_stats", do_stats)
+        stage("sort", do_sort)
         perms = {"hidden": ws.p_hid, "intermediate": ws.p_mid, "v_heads": ws.p_v, "o_heads": ws.p_o}
 
     res = LayerResult(moments=ws.moments, perms=perms,
@@ -186,15 +231,18 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
 
     # a4: block scores of every matrix into its rows of the global table
     L = len(cfg.bits)
-    for name, l in lin.items():
-        nb = (l.rows // cfg.block_rows) * (l.cols // cfg.block_cols)
-        s = ws.block_start[name]
-        with _Timed(timers, "scores"):
+
+    def do_scores():
+        for name, l in lin.items():
+            nb = (l.rows // cfg.block_rows) * (l.cols // cfg.block_cols)
+            s = ws.block_start[name]
             ctx.block_scores(W[name], c[name], cfg.bits, cfg.block_rows, cfg.block_cols, g,
                              row_perm=res.row_perm(name), col_perm=res.col_perm(name),
                              err=ws.err[s:s + nb], gain=ws.gain[s:s + nb] if L > 1 else None,
                              want_gain=L > 1,
                              W_perm_out=ws.w_perm[name] if ws.w_perm is not None else None)
+
+    stage("scores", do_scores)
     if not allocate:
         return res
 
@@ -207,11 +255,11 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
         return res
 
     # a6: pack every matrix at its blocks' levels (from the permuted copy when it was kept)
-    for name, l in lin.items():
-        nb = (l.rows // cfg.block_rows) * (l.cols // cfg.block_cols)
-        s = ws.block_start[name]
-        packed, off, meta = ws.packed[name]
-        with _Timed(timers, "pack"):
+    def do_pack():
+        for name, l in lin.items():
+            nb = (l.rows // cfg.block_rows) * (l.cols // cfg.block_cols)
+            s = ws.block_start[name]
+            packed, off, meta = ws.packed[name]
             if ws.w_perm is not None:
                 ctx.pack_blocks(ws.w_perm[name], cfg.bits, ws.level[s:s + nb], cfg.block_rows,
                                 cfg.block_cols, g, packed=packed, block_off=off, meta=meta)
@@ -219,5 +267,7 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
                 ctx.pack_blocks(W[name], cfg.bits, ws.level[s:s + nb], cfg.block_rows, cfg.block_cols,
                                 g, row_perm=res.row_perm(name), col_perm=res.col_perm(name),
                                 packed=packed, block_off=off, meta=meta)
-        res.packed[name] = (packed, off, meta)
+
+    stage("pack", do_pack)
+    res.packed = dict(ws.packed)
     return res
