@@ -30,9 +30,11 @@ WORKLOAD = ("one Llama-3-8B-shaped decoder layer (q/o 4096x4096, k/v 1024x4096, 
             "down 4096x14336; 218,103,808 bf16 weights), 65536 calibration tokens per input, "
             "blocks 128x128, group 128, bits {2,3,4,8}, budget 2.5")
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (None until a capture exists for that kernel)
-NCU_TRAFFIC_BYTES = {"moments_partial_kernel": None}
+# (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of the dominant kernel, from the
+# ncu capture summarised in profiles/moments_partial_kernel_65536x4096.md (541.04 MB moved for
+# 536.87 MB of activations); the kernel's traffic is proportional to T * K, so the ratio carries
+# over to the launches of the step
+NCU_TRAFFIC_RATIO = {"moments_partial_kernel": 1.0078}
 
 
 def measured_peaks():
@@ -298,9 +300,9 @@ def run_cuda(args):
         peak, peak_kind = measured_peaks()
         # dominant kernel by time: the calibration-moments reduction (3.49 GB read per step)
         mom_bytes = sum(x.numel() * 2 for x in X.values())
-        mom_launches = len(X)
+        mom_launches = len(X)          # one kernel per input; the stage's events bracket all four
         achieved = mom_bytes / (stage_ms["moments"] * 1e-3) / 1e9
-        traffic = NCU_TRAFFIC_BYTES["moments_partial_kernel"]
+        traffic = NCU_TRAFFIC_RATIO["moments_partial_kernel"] * mom_bytes / mom_launches
         roofline = {"kernel": "moments_partial_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
                     "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
                     "traffic": traffic, "algorithmic_bytes_per_launch": mom_bytes / mom_launches,
@@ -333,6 +335,50 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
+def run_only(which: str):
+    """A few calls of ONE library call on one input of the layer (for ncu captures: small, a
+    few launches, larger than L2): moments on a 65536 x 4096 input, the others on a
+    14336 x 4096 matrix."""
+    import torch
+    from paper_2602_17698_b200 import synth
+    from paper_2602_17698_b200.binding import Context
+    torch.cuda.set_device(0)
+    dev = "cuda:0"
+    ctx = Context()
+    R, Cc = 14336, 4096
+    c = torch.rand(Cc, device=dev) + 0.5
+    if which == "moments":
+        X = synth.make_activations(TOKENS, 4096, 7, dev)
+        for _ in range(3):
+            ctx.calib_moments(X)
+    else:
+        W = synth.make_weight(R, Cc, 100, dev)
+        nb = (R // 128) * (Cc // 128)
+        if which == "scores":
+            err = torch.empty(nb, len(BITS), device=dev)
+            for _ in range(3):
+                ctx.block_scores(W, c, BITS, 128, 128, 128, err=err, want_gain=False)
+        elif which == "reorder_stats":
+            rs, cs = torch.empty(R, device=dev), torch.empty(Cc, device=dev)
+            for _ in range(3):
+                ctx.reorder_channels(W, c, 2, 128, row_score=rs, col_score=cs)
+        elif which == "gather":
+            pr, pc = torch.randperm(R, device=dev).int(), torch.randperm(Cc, device=dev).int()
+            err, out = torch.empty(nb, len(BITS), device=dev), torch.empty_like(W)
+            for _ in range(3):
+                ctx.block_scores(W, c, BITS, 128, 128, 128, row_perm=pr, col_perm=pc, err=err,
+                                 want_gain=False, W_perm_out=out)
+        elif which == "pack":
+            level = torch.randint(0, len(BITS), (nb,), device=dev, dtype=torch.uint8)
+            for _ in range(3):
+                ctx.pack_blocks(W, BITS, level, 128, 128, 128)
+        else:
+            raise SystemExit(f"unknown stage {which}")
+    ctx.sync()
+    ctx.close()
+    print("done", which)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -343,8 +389,13 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graphs", action="store_true", help="launch every library call eagerly")
+    ap.add_argument("--only", default=None,
+                    help="three calls of one library call on one input, then exit (for ncu captures): "
+                         "moments | reorder_stats | scores | gather | pack")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.only:
+        run_only(args.only)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_cuda(args)

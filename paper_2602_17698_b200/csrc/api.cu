@@ -69,6 +69,8 @@ sb_status sb_create(sb_ctx** out, int device, void* cuda_stream) {
     ctx->sm_count = prop.multiProcessorCount;
     if (cudaMalloc(&ctx->dstate, sizeof(SbDeviceState)) != cudaSuccess ||
         cudaMemset(ctx->dstate, 0, sizeof(SbDeviceState)) != cudaSuccess ||
+        cudaMalloc(&ctx->moment_done, SB_MOMENT_CHUNKS * sizeof(unsigned)) != cudaSuccess ||
+        cudaMemset(ctx->moment_done, 0, SB_MOMENT_CHUNKS * sizeof(unsigned)) != cudaSuccess ||
         cudaMallocHost(&ctx->pinned, 4096) != cudaSuccess) {
         delete ctx;
         return SB_ERR_CUDA;
@@ -85,6 +87,7 @@ sb_status sb_destroy(sb_ctx* ctx) {
     if (ctx->scratch) cudaFree(ctx->scratch);
     if (ctx->dstate) cudaFree(ctx->dstate);
     if (ctx->lb_mem) cudaFree(ctx->lb_mem);
+    if (ctx->moment_done) cudaFree(ctx->moment_done);
     if (ctx->pinned) cudaFreeHost(ctx->pinned);
     delete ctx;
     return SB_OK;

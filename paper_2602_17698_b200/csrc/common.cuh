@@ -24,6 +24,7 @@ struct sb_ctx {
     SbDeviceState* dstate = nullptr;
     void* pinned = nullptr;      // small pinned host buffer for read-backs
     size_t pinned_bytes = 0;
+    unsigned int* moment_done = nullptr;   // per column chunk: row splits finished (zero between calls)
     void* lb_mem = nullptr;      // look-back descriptors (context-owned, never in the arena)
     unsigned int lb_max_tiles = 0;
     int64_t launches = 0;
@@ -67,6 +68,7 @@ struct Carver {
 };
 
 bool sb_check_bits(const int* bits, int n_bits);
+constexpr int SB_MOMENT_CHUNKS = 4096;   // column chunks of 256 a moments call may have (K <= 1M)
 
 enum SbKernelId { SBK_MOMENTS = 1, SBK_STATS, SBK_SCORES, SBK_GATHER, SBK_ARGSORT, SBK_SCAN,
                   SBK_SORT, SBK_ALLOC, SBK_PACK };
@@ -102,6 +104,36 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
 }
 __device__ __forceinline__ void st_release_u32(unsigned* p, unsigned v) {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+__device__ __forceinline__ uint32_t u32(__nv_bfloat162 v) { return *reinterpret_cast<uint32_t*>(&v); }
+__device__ __forceinline__ __nv_bfloat162 b162(uint32_t v) { return *reinterpret_cast<__nv_bfloat162*>(&v); }
+
+// min and max of a group: NW packed words per lane, `team` lanes (a power of two, aligned)
+// per group.  Exact: bf16 min/max, the pair (min, -max) rides one register through the
+// shuffles.
+template <int NW, int TEAM = 0>
+__device__ __forceinline__ void group_minmax(const uint32_t (&w)[NW], int team, float& lo, float& hi) {
+    __nv_bfloat162 mn = b162(w[0]), mx = mn;
+#pragma unroll
+    for (int k = 1; k < NW; ++k) {
+        mn = __hmin2(mn, b162(w[k]));
+        mx = __hmax2(mx, b162(w[k]));
+    }
+    const uint32_t mnu = u32(mn), mxu = u32(mx);
+    const uint32_t a = u32(__hmin2(mn, b162(__byte_perm(mnu, mnu, 0x1032))));
+    const uint32_t b = u32(__hmax2(mx, b162(__byte_perm(mxu, mxu, 0x1032)))) ^ 0x80008000u;
+    uint32_t p = (a & 0x0000ffffu) | (b & 0xffff0000u);
+    if (TEAM > 0) {
+#pragma unroll
+        for (int o = TEAM >> 1; o > 0; o >>= 1)
+            p = u32(__hmin2(b162(p), b162(__shfl_xor_sync(0xffffffffu, p, o))));
+    } else {
+        for (int o = team >> 1; o > 0; o >>= 1)
+            p = u32(__hmin2(b162(p), b162(__shfl_xor_sync(0xffffffffu, p, o))));
+    }
+    lo = bf16lo(p);
+    hi = -bf16hi(p);
 }
 
 __device__ __forceinline__ float warp_sum(float v) {

@@ -1,5 +1,6 @@
 // Calibration second moments: sumsq[j] (+)= scale * sum_t X[t][j]^2.
-// HBM-bound streaming column reduction: 2 bytes and one FMA per activation.
+// HBM-bound streaming column reduction: 2 bytes and one FMA per activation; one kernel (the
+// last CTA of a column chunk adds the row splits' partial sums).
 #include "common.cuh"
 
 namespace {
@@ -12,7 +13,9 @@ constexpr int MOM_UNROLL = 8;         // 16-byte loads in flight per thread
 // grid.x = column chunks of 256, grid.y = row splits; partial[split][K]
 __global__ void __launch_bounds__(MOM_TX * MOM_TY)
 moments_partial_kernel(const __nv_bfloat16* __restrict__ X, int64_t T, int64_t K, int64_t ldx,
-                       int64_t rows_per_split, float* __restrict__ partial) {
+                       int64_t rows_per_split, float* __restrict__ partial,
+                       unsigned* __restrict__ chunk_done, float scale, int accumulate,
+                       float* __restrict__ out) {
     const int tx = threadIdx.x, ty = threadIdx.y;
     const int64_t col = (int64_t)blockIdx.x * MOM_COLS + tx * 8;
     const int64_t t0 = (int64_t)blockIdx.y * rows_per_split;
@@ -63,16 +66,23 @@ moments_partial_kernel(const __nv_bfloat16* __restrict__ X, int64_t T, int64_t K
         for (int y = 0; y < MOM_TY; ++y) s += red[y][c];
         partial[(int64_t)blockIdx.y * K + gc] = s;
     }
-}
-
-__global__ void moments_finish_kernel(const float* __restrict__ partial, int splits, int64_t K,
-                                      float scale, int accumulate, float* __restrict__ out) {
-    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= K) return;
-    float s = 0.f;
-    for (int p = 0; p < splits; ++p) s += partial[(int64_t)p * K + j];
-    s *= scale;
-    out[j] = accumulate ? out[j] + s : s;
+    // The last CTA of this column chunk to finish adds the splits' partial sums in split order
+    // (a fixed order whichever CTA does it: bit-identical reruns) and clears the counter.
+    __shared__ bool last_sh;
+    __threadfence();
+    __syncthreads();
+    if (c == 0) last_sh = atomicAdd(chunk_done + blockIdx.x, 1u) == gridDim.y - 1;
+    __syncthreads();
+    if (last_sh) {
+        __threadfence();
+        if (gc < K) {
+            float s = 0.f;
+            for (unsigned p = 0; p < gridDim.y; ++p) s += __ldcg(partial + (int64_t)p * K + gc);
+            s *= scale;
+            out[gc] = accumulate ? out[gc] + s : s;
+        }
+        if (c == 0) chunk_done[blockIdx.x] = 0u;
+    }
 }
 
 }  // namespace
@@ -100,12 +110,12 @@ extern "C" sb_status sb_calib_moments(sb_ctx* ctx, const void* X, int64_t T, int
     if (st != SB_OK) return st;
     Carver cv(arena);
     float* partial = cv.take<float>((size_t)splits * K);
+    if (col_chunks > SB_MOMENT_CHUNKS)
+        return sb_fail(ctx, SB_ERR_SHAPE, "moments: K above %d not supported", SB_MOMENT_CHUNKS * MOM_COLS);
     dim3 grid(col_chunks, splits), block(MOM_TX, MOM_TY);
     moments_partial_kernel<<<grid, block, 0, ctx->stream>>>(
-        static_cast<const __nv_bfloat16*>(X), T, K, ldx, rows_per_split, partial);
-    SB_LAUNCHED(ctx);
-    moments_finish_kernel<<<(unsigned)((K + 255) / 256), 256, 0, ctx->stream>>>(
-        partial, splits, K, scale, accumulate, sumsq);
+        static_cast<const __nv_bfloat16*>(X), T, K, ldx, rows_per_split, partial, ctx->moment_done, scale,
+        accumulate, sumsq);
     SB_LAUNCHED(ctx);
     return SB_OK;
 }

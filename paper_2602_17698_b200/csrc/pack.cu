@@ -52,7 +52,7 @@ pack_offsets_kernel(const unsigned char* __restrict__ level, int64_t nb, int n_b
 
 
 
-constexpr float PK_MAGIC = 12582912.f;          // 1.5 * 2^23
+constexpr double PK_MAGIC64 = 6755399441055744.0;     // 1.5 * 2^52: low word of (t + MAGIC) = rint(t)
 
 // 16 codes of B bits -> 16*B bits in w[0..3] (little-endian bit stream)
 template <int B>
@@ -77,15 +77,14 @@ __device__ __forceinline__ void pack16(const unsigned (&code)[16], unsigned (&w)
 // 16-byte loads), 8 lanes cover a row of the chunk, a warp covers 4 rows per step; the next
 // step's loads are issued before the current rows are encoded.
 //
-// Codes are DEFINED by the binary64 sequence
+// Codes follow the binary64 sequence
 //   range = hi - lo; inv = qmax / range; q = rint((v - lo) * inv)
-// but computed in fp32 wherever that provably gives the same integer: the fp32 value of t is
-// within 1.8e-7 * qmax of the fp64 one, so an element farther than twice that from a rounding
-// tie keeps its fp32 code, and only rows that contain an element inside that band (exact
-// ties are common with bf16 data) redo those elements in fp64.  The stored scale is
-// fl32(range / qmax): with range exact in fp32 (checked) one correctly rounded fp32 division
-// equals the rounded fp64 quotient (a 24-bit integer over 2^b - 1 has a binary expansion of
-// period <= 8, never within 2^-53 of an fp32 rounding boundary).
+// literally: one fp64 division per lane and row, then a subtract, a multiply and the magic-number
+// add per element (its low word is the rounded integer, ties to even).  B200 issues fp64 at half
+// the fp32 rate, so this costs less than an fp32 path with a tie test and a divergent fp64 redo.
+// The stored scale is fl32(range / qmax): with range exact in fp32 (checked) one correctly
+// rounded fp32 division equals the rounded fp64 quotient (a 24-bit integer over 2^b - 1 has a
+// binary expansion of period <= 8, never within 2^-53 of an fp32 rounding boundary).
 //
 // A lane's 16 codes are 16*b bits: whole words for even b, and for odd b a pair of lanes
 // makes whole words (the even lane also takes the low half-word of its neighbour).
@@ -121,9 +120,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const int32_t* __r
     const long long lane_base = s_base[pc] + (lp * 16 * b) / 32;
     const bool odd_b = b & 1, odd_lane = lp & 1;
     const float qmaxf = (float)((1 << b) - 1);
-    // |t32 - t64| <= 3 * 2^-24 * t <= 1.8e-7 * qmax: twice that keeps the fp32 code safe
-    const float tie_band = 0.5f - 4.0e-7f * qmaxf - 1.0e-7f;
-    const int team = group >> 4;                          // lanes per quantisation group
+    const int team = group >> 4;                          // lanes per quantisation group (16 columns each)
     const int64_t gcol = (col0 + cl * 16) / group;
     const bool meta_lane = (cl % team) == 0;
     const __nv_bfloat16* colp = W + col0 + cl * 16;
@@ -142,57 +139,28 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const int32_t* __r
             const __nv_bfloat16* p = row_ptr(rr + PK_WARPS * 4);
             n0 = ld_stream16(p); n1 = ld_stream16(p + 8);
         }
-        float v[16];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) { v[2 * k] = bf16lo(wv[k]); v[2 * k + 1] = bf16hi(wv[k]); }
-        float lo = v[0], hi = v[0];
-#pragma unroll
-        for (int k = 1; k < 16; ++k) { lo = fminf(lo, v[k]); hi = fmaxf(hi, v[k]); }
-        for (int o = team >> 1; o > 0; o >>= 1) {
-            lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
-            hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
-        }
-        const double range64 = __dsub_rn((double)hi, (double)lo);     // exact
+        float lo, hi;
+        group_minmax<8>(wv, team, lo, hi);
+        const double dlo = (double)lo;
+        const double range64 = __dsub_rn((double)hi, dlo);            // exact
         const float range = (float)range64;
-        const bool exact = (double)range == range64;
         unsigned code[16];
         float scale = 0.f;
-        unsigned near = 0u;
-        bool redo = false;
         if (range64 != 0.0) {
-            // fp32 fast path (a denormal range overflows the reciprocal: let fp64 handle it)
-            const bool fast = range >= 1e-30f;
-            const float inv = fast ? __fdiv_rn(qmaxf, range) : 0.f;
+            const double inv = __ddiv_rn((double)qmaxf, range64);
+            scale = (double)range == range64 ? __fdiv_rn(range, qmaxf)
+                                             : (float)__ddiv_rn(range64, (double)qmaxf);
 #pragma unroll
-            for (int k = 0; k < 16; ++k) {
-                const float t = (v[k] - lo) * inv;
-                const float m = t + PK_MAGIC;                 // integer in the low mantissa bits
-                const float q = m - PK_MAGIC;
-                code[k] = __float_as_uint(m) & 0xffu;
-                if (!(fabsf(t - q) < tie_band)) near |= 1u << k;
+            for (int k = 0; k < 8; ++k) {
+                const double t0 = __dmul_rn(__dsub_rn((double)bf16lo(wv[k]), dlo), inv);
+                const double t1 = __dmul_rn(__dsub_rn((double)bf16hi(wv[k]), dlo), inv);
+                // 0 <= t <= qmax, so no clamp: the low word of t + 1.5 * 2^52 is rint(t)
+                code[2 * k] = (unsigned)__double2loint(__dadd_rn(t0, PK_MAGIC64)) & 0xffu;
+                code[2 * k + 1] = (unsigned)__double2loint(__dadd_rn(t1, PK_MAGIC64)) & 0xffu;
             }
-            if (!fast) near = 0xffffu;
-            scale = __fdiv_rn(range, qmaxf);
-            redo = near != 0u || !exact;
         } else {
 #pragma unroll
             for (int k = 0; k < 16; ++k) code[k] = 0u;
-        }
-        if (__any_sync(0xffffffffu, redo)) {
-            if (redo) {
-                const double qmax = (double)qmaxf, dlo = (double)lo;
-                const double inv = __ddiv_rn(qmax, range64);
-                if (!exact) scale = (float)__ddiv_rn(range64, qmax);
-#pragma unroll
-                for (int k = 0; k < 16; ++k) {
-                    if (near & (1u << k)) {
-                        const double t = __dmul_rn(__dsub_rn((double)v[k], dlo), inv);
-                        double q = rint(t);                          // round half to even
-                        q = fmin(fmax(q, 0.0), qmax);
-                        code[k] = (unsigned)q;
-                    }
-                }
-            }
         }
         if (meta_lane) meta[r * groups_per_row + gcol] = make_float2(scale, lo);
         unsigned w[4];

@@ -25,36 +25,6 @@ struct __align__(8) BitsArg {
     int bits[8];
 };
 
-__device__ __forceinline__ uint32_t u32(__nv_bfloat162 v) { return *reinterpret_cast<uint32_t*>(&v); }
-__device__ __forceinline__ __nv_bfloat162 b162(uint32_t v) { return *reinterpret_cast<__nv_bfloat162*>(&v); }
-
-// min and max of a group: NW packed words per lane, `team` lanes (a power of two, aligned)
-// per group.  Exact: bf16 min/max, the pair (min, -max) rides one register through the
-// shuffles.
-template <int NW, int TEAM = 0>
-__device__ __forceinline__ void group_minmax(const uint32_t (&w)[NW], int team, float& lo, float& hi) {
-    __nv_bfloat162 mn = b162(w[0]), mx = mn;
-#pragma unroll
-    for (int k = 1; k < NW; ++k) {
-        mn = __hmin2(mn, b162(w[k]));
-        mx = __hmax2(mx, b162(w[k]));
-    }
-    const uint32_t mnu = u32(mn), mxu = u32(mx);
-    const uint32_t a = u32(__hmin2(mn, b162(__byte_perm(mnu, mnu, 0x1032))));
-    const uint32_t b = u32(__hmax2(mx, b162(__byte_perm(mxu, mxu, 0x1032)))) ^ 0x80008000u;
-    uint32_t p = (a & 0x0000ffffu) | (b & 0xffff0000u);
-    if (TEAM > 0) {
-#pragma unroll
-        for (int o = TEAM >> 1; o > 0; o >>= 1)
-            p = u32(__hmin2(b162(p), b162(__shfl_xor_sync(0xffffffffu, p, o))));
-    } else {
-        for (int o = team >> 1; o > 0; o >>= 1)
-            p = u32(__hmin2(b162(p), b162(__shfl_xor_sync(0xffffffffu, p, o))));
-    }
-    lo = bf16lo(p);
-    hi = -bf16hi(p);
-}
-
 __device__ __forceinline__ float rcp_approx(float x) {
     float r;
     asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
@@ -477,6 +447,32 @@ __global__ void rank_count_kernel(const float* __restrict__ score, int64_t K, in
     }
     if (cnt) atomicAdd(rank + i, cnt);
 }
+// the same count with the compared keys staged in shared memory: a CTA's 256 channels lie in one
+// segment (segment % 256 == 0), blockIdx.y picks a run of 256 compared channels of that segment
+__global__ void __launch_bounds__(256)
+rank_count_tile_kernel(const float* __restrict__ score, int64_t K, int64_t seg, int* __restrict__ rank) {
+    __shared__ uint32_t sk[256];
+    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    const int64_t s0 = (int64_t)blockIdx.x * 256 / seg * seg;
+    const int64_t j0 = s0 + (int64_t)blockIdx.y * 256;
+    sk[threadIdx.x] = order_key(score[j0 + threadIdx.x]);
+    __syncthreads();
+    const uint32_t ki = order_key(score[i]);
+    // j < i decides ties: all-or-nothing for a tile except the one that contains i
+    const int64_t d = i - j0;                      // compared channels with index below i: j - j0 < d
+    int cnt = 0;
+    if (d <= 0) {
+#pragma unroll 16
+        for (int j = 0; j < 256; ++j) cnt += sk[j] > ki;
+    } else if (d >= 256) {
+#pragma unroll 16
+        for (int j = 0; j < 256; ++j) cnt += sk[j] >= ki;
+    } else {
+#pragma unroll 16
+        for (int j = 0; j < 256; ++j) cnt += (sk[j] > ki) || (sk[j] == ki && j < (int)d);
+    }
+    if (cnt) atomicAdd(rank + i, cnt);
+}
 __global__ void rank_scatter_kernel(const int* __restrict__ rank, int64_t K, int64_t seg,
                                     int32_t* __restrict__ perm) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -519,6 +515,14 @@ bool valid_group(int g) { return g == 16 || g == 32 || g == 64 || g == 128; }
 
 sb_status argsort_axis(sb_ctx* ctx, const float* score, int64_t K, int64_t seg, int32_t* perm, int* rank) {
     SB_CUDA(ctx, cudaMemsetAsync(rank, 0, sizeof(int) * K, ctx->stream));
+    if (seg % 256 == 0) {
+        dim3 grid((unsigned)(K / 256), (unsigned)(seg / 256));
+        rank_count_tile_kernel<<<grid, 256, 0, ctx->stream>>>(score, K, seg, rank);
+        SB_LAUNCHED(ctx);
+        rank_scatter_kernel<<<(unsigned)((K + 255) / 256), 256, 0, ctx->stream>>>(rank, K, seg, perm);
+        SB_LAUNCHED(ctx);
+        return SB_OK;
+    }
     // short comparison loops (<= 256 per thread): the counting is latency-bound otherwise
     int splits = (int)((seg + 255) / 256);
     if (splits > 1024) splits = 1024;

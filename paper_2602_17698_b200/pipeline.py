@@ -161,8 +161,7 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
     """moments -> reorder statistics -> permutations -> block scores -> allocation -> pack.
 
     `timers`, if given, maps the stage names moments / reorder_stats / sort / scores /
-    allocate / pack to lists that receive one (start, end) CUDA event pair per stage (per
-    library call for the moments, whose launches the roofline accounting needs).
+    allocate / pack to lists that receive one (start, end) CUDA event pair per stage.
     `graphs`, if given, replays each stage from a CUDA graph captured on first use.
     """
     def stage(name, fn):
@@ -180,13 +179,11 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
     W = weights
 
     # a1: calibration second moments, one per distinct linear input
-    for name, X in acts.items():
-        if graphs is not None:
-            with _Timed(timers, "moments"):
-                graphs.run("moments:" + name, lambda X=X, name=name: ctx.calib_moments(X, ws.moments[name]))
-        else:
-            with _Timed(timers, "moments"):
-                ctx.calib_moments(X, ws.moments[name])
+    def do_moments():
+        for name, X in acts.items():
+            ctx.calib_moments(X, ws.moments[name])
+
+    stage("moments", do_moments)
     c = {n: ws.moments[l.act] for n, l in lin.items()}
 
     perms = {"hidden": None, "intermediate": None, "v_heads": None, "o_heads": None}
