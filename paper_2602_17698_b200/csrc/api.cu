@@ -71,6 +71,8 @@ sb_status sb_create(sb_ctx** out, int device, void* cuda_stream) {
         cudaMemset(ctx->dstate, 0, sizeof(SbDeviceState)) != cudaSuccess ||
         cudaMalloc(&ctx->moment_done, SB_MOMENT_CHUNKS * sizeof(unsigned)) != cudaSuccess ||
         cudaMemset(ctx->moment_done, 0, SB_MOMENT_CHUNKS * sizeof(unsigned)) != cudaSuccess ||
+        cudaMalloc(&ctx->stats_done, 2 * SB_STATS_TILES * sizeof(unsigned)) != cudaSuccess ||
+        cudaMemset(ctx->stats_done, 0, 2 * SB_STATS_TILES * sizeof(unsigned)) != cudaSuccess ||
         cudaMallocHost(&ctx->pinned, 4096) != cudaSuccess) {
         delete ctx;
         return SB_ERR_CUDA;
@@ -88,6 +90,7 @@ sb_status sb_destroy(sb_ctx* ctx) {
     if (ctx->dstate) cudaFree(ctx->dstate);
     if (ctx->lb_mem) cudaFree(ctx->lb_mem);
     if (ctx->moment_done) cudaFree(ctx->moment_done);
+    if (ctx->stats_done) cudaFree(ctx->stats_done);
     if (ctx->pinned) cudaFreeHost(ctx->pinned);
     delete ctx;
     return SB_OK;

@@ -25,6 +25,7 @@ struct sb_ctx {
     void* pinned = nullptr;      // small pinned host buffer for read-backs
     size_t pinned_bytes = 0;
     unsigned int* moment_done = nullptr;   // per column chunk: row splits finished (zero between calls)
+    unsigned int* stats_done = nullptr;    // per tile row / tile column: tiles finished (zero between calls)
     void* lb_mem = nullptr;      // look-back descriptors (context-owned, never in the arena)
     unsigned int lb_max_tiles = 0;
     int64_t launches = 0;
@@ -68,6 +69,7 @@ struct Carver {
 };
 
 bool sb_check_bits(const int* bits, int n_bits);
+constexpr int SB_STATS_TILES = 8192;     // 128-wide tiles per axis a reorder call may have
 constexpr int SB_MOMENT_CHUNKS = 4096;   // column chunks of 256 a moments call may have (K <= 1M)
 
 enum SbKernelId { SBK_MOMENTS = 1, SBK_STATS, SBK_SCORES, SBK_GATHER, SBK_ARGSORT, SBK_SCAN,

@@ -131,13 +131,16 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const int32_t* __r
     };
     int rr = warp * 4 + slot;
     uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0;
-    if (rr < br) { const __nv_bfloat16* p = row_ptr(rr); n0 = ld_stream16(p); n1 = ld_stream16(p + 8); }
+    if (rr < br) {
+        const uint4* p = reinterpret_cast<const uint4*>(row_ptr(rr));
+        n0 = __ldg(p); n1 = __ldg(p + 1);
+    }
     for (; rr < br; rr += PK_WARPS * 4) {          // br % 4 == 0: a warp step is all or nothing
         const int64_t r = bi * br + rr;
         const uint32_t wv[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
         if (rr + PK_WARPS * 4 < br) {
-            const __nv_bfloat16* p = row_ptr(rr + PK_WARPS * 4);
-            n0 = ld_stream16(p); n1 = ld_stream16(p + 8);
+            const uint4* p = reinterpret_cast<const uint4*>(row_ptr(rr + PK_WARPS * 4));
+            n0 = __ldg(p); n1 = __ldg(p + 1);
         }
         float lo, hi;
         group_minmax<8>(wv, team, lo, hi);

@@ -31,30 +31,47 @@ __device__ __forceinline__ float rcp_approx(float x) {
     return r;
 }
 
+// ---- asynchronous 16-byte copies global -> shared (L2 only, no register staging) -----------
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 // ---- permuted gather: out[r][j] = W[rp[r]][cp[j]] ---------------------------------------
-// One source row is staged in shared memory with coalesced 16-byte loads, then read in
-// permuted order; 2-byte scattered reads never reach HBM.
+// A source row is staged in shared memory with coalesced asynchronous 16-byte copies (the next
+// row is in flight while the current one is written out), then read in permuted order: 2-byte
+// scattered reads never reach HBM.
 __global__ void __launch_bounds__(CTA_THREADS)
 gather_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, int64_t ldw,
               const int32_t* __restrict__ rp, const int32_t* __restrict__ cp,
               __nv_bfloat16* __restrict__ out, int rows_per_cta) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    unsigned short* row = reinterpret_cast<unsigned short*>(smem_raw);
+    unsigned short* buf[2] = {reinterpret_cast<unsigned short*>(smem_raw),
+                              reinterpret_cast<unsigned short*>(smem_raw) + C};
     const int64_t r0 = (int64_t)blockIdx.x * rows_per_cta;
-    for (int rr = 0; rr < rows_per_cta; ++rr) {
+    const int nrows = (int)min((int64_t)rows_per_cta, R - r0);
+    auto stage = [&](int rr) {
         const int64_t r = r0 + rr;
-        if (r >= R) break;
-        const int64_t rs = rp ? rp[r] : r;
-        const __nv_bfloat16* src = W + rs * ldw;
-        for (int64_t j = (int64_t)threadIdx.x * 8; j < C; j += CTA_THREADS * 8)
-            *reinterpret_cast<uint4*>(row + j) = ld_stream16(src + j);
+        const __nv_bfloat16* src = W + (rp ? (int64_t)rp[r] : r) * ldw;
+        unsigned short* dst = buf[rr & 1];
+        for (int64_t j = (int64_t)threadIdx.x * 8; j < C; j += CTA_THREADS * 8) cp_async16(dst + j, src + j);
+        cp_async_commit();
+    };
+    if (nrows > 0) stage(0);
+    for (int rr = 0; rr < nrows; ++rr) {
+        if (rr + 1 < nrows) stage(rr + 1); else cp_async_commit();
+        cp_async_wait<1>();
         __syncthreads();
-        unsigned short* dst = reinterpret_cast<unsigned short*>(out + r * C);
+        const unsigned short* row = buf[rr & 1];
+        unsigned short* dst = reinterpret_cast<unsigned short*>(out + (r0 + rr) * C);
         for (int64_t j = (int64_t)threadIdx.x * 8; j < C; j += CTA_THREADS * 8) {
             uint32_t o[4];
             if (cp) {
-                const int4 p0 = *reinterpret_cast<const int4*>(cp + j);
-                const int4 p1 = *reinterpret_cast<const int4*>(cp + j + 4);
+                const int4 p0 = __ldg(reinterpret_cast<const int4*>(cp + j));
+                const int4 p1 = __ldg(reinterpret_cast<const int4*>(cp + j + 4));
                 o[0] = row[p0.x] | ((uint32_t)row[p0.y] << 16);
                 o[1] = row[p0.z] | ((uint32_t)row[p0.w] << 16);
                 o[2] = row[p1.x] | ((uint32_t)row[p1.y] << 16);
@@ -65,7 +82,7 @@ gather_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, int64_t
             }
             *reinterpret_cast<uint4*>(dst + j) = make_uint4(o[0], o[1], o[2], o[3]);
         }
-        __syncthreads();
+        __syncthreads();          // the buffer is free for the row after next
     }
 }
 
@@ -74,7 +91,9 @@ template <int CPL>
 __device__ __forceinline__ void load_cols(const __nv_bfloat16* p, bool ok, uint32_t (&w)[CPL / 2]) {
 #pragma unroll
     for (int v = 0; v < CPL / 8; ++v) {
-        uint4 x = ok ? ld_stream16(p + 8 * v) : make_uint4(0, 0, 0, 0);
+        // plain read-only loads: a lane's two 16-byte pieces share 32-byte sectors with its
+        // neighbours', so the second load of a row should hit L1
+        uint4 x = ok ? __ldg(reinterpret_cast<const uint4*>(p + 8 * v)) : make_uint4(0, 0, 0, 0);
         w[4 * v] = x.x; w[4 * v + 1] = x.y; w[4 * v + 2] = x.z; w[4 * v + 3] = x.w;
     }
 }
@@ -107,15 +126,6 @@ __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
     asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
-
-// ---- asynchronous 16-byte copies global -> shared (L2 only, no register staging) -----------
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
-    const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // ---- block scores ------------------------------------------------------------------------
 // Every WARP is autonomous: it walks its own units (a block, or a 32-row part of one), stages
@@ -347,83 +357,145 @@ __global__ void scores_finish_kernel(const float* __restrict__ part, int parts, 
 }
 
 // ---- reorder statistics --------------------------------------------------------------------
-// 128 x 128 tiles of the ORIGINAL layout, one candidate (ref_bits).  Writes per-tile partial
-// row sums rowpart[tile_col][r] and column sums colpart[tile_row][j]; a second kernel adds
-// them up in a fixed order (no floating-point atomics: run-to-run deterministic).
-template <bool ROWW>
+// 128 x 128 tiles of the ORIGINAL layout, one candidate (ref_bits).  Every tile writes its
+// partial row sums rowpart[tile_col][r] and column sums colpart[tile_row][j]; the last tile of
+// a tile row (tile column) to finish adds the partials of that row strip (column strip) in
+// tile order -- a fixed order whichever CTA does it, and no floating-point atomics, so reruns
+// are bit-identical -- and adds them to / stores them in the score vectors.
+template <bool ROWW, bool FINE, int TILE_ROWS>
 __global__ void __launch_bounds__(CTA_THREADS)
 reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, int64_t ldw,
                      const float* __restrict__ col_moment, const float* __restrict__ row_weight,
                      int group, float qmax, float inv_qmax,
-                     float* __restrict__ rowpart, float* __restrict__ colpart) {
-    constexpr int CPL = 16, NW = 8, LANE_COLS = 8, ROW_SLOTS = 4, TILE_ROWS = 128;
+                     float* __restrict__ rowpart, float* __restrict__ colpart,
+                     float* __restrict__ row_score, float* __restrict__ col_score, int accumulate,
+                     unsigned* __restrict__ done_row, unsigned* __restrict__ done_col,
+                     SbDeviceState* dstate) {
+    constexpr int CPL = 16, NW = 8, LANE_COLS = 8, ROW_SLOTS = 4;
+    constexpr int ITERS = TILE_ROWS / (CTA_WARPS * ROW_SLOTS);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int cl = lane % LANE_COLS, slot = lane / LANE_COLS;
     const int team = group / CPL > 0 ? group / CPL : 1;
     const int64_t col = (int64_t)blockIdx.x * TILE_COLS + cl * CPL;
     const bool col_ok = col < C;
     const int64_t row0 = (int64_t)blockIdx.y * TILE_ROWS;
-    float cw[CPL], acc[CPL];
+    const f32x2 magic2 = pk2(RNE_MAGIC, RNE_MAGIC), nmagic2 = pk2(-RNE_MAGIC, -RNE_MAGIC);
+    f32x2 cw[NW], acc[NW];
 #pragma unroll
-    for (int k = 0; k < CPL; ++k) {
-        cw[k] = col_ok ? col_moment[col + k] : 0.f;
-        acc[k] = 0.f;
+    for (int k = 0; k < NW; ++k) {
+        cw[k] = col_ok ? pk2(col_moment[col + 2 * k], col_moment[col + 2 * k + 1]) : 0ull;
+        acc[k] = 0ull;
     }
-    for (int rr = warp * ROW_SLOTS + slot; rr < TILE_ROWS; rr += CTA_WARPS * ROW_SLOTS) {
-        const int64_t r = row0 + rr;
+    // the next step's two 16-byte loads are in flight while this step is evaluated
+    uint32_t wn[NW];
+    {
+        const int64_t r = row0 + warp * ROW_SLOTS + slot;
         const bool ok = col_ok && r < R;
+        load_cols<CPL>(W + (ok ? r * ldw + col : 0), ok, wn);
+    }
+#pragma unroll 2
+    for (int it = 0; it < ITERS; ++it) {
+        const int rr = it * (CTA_WARPS * ROW_SLOTS) + warp * ROW_SLOTS + slot;
+        const int64_t r = row0 + rr;
         uint32_t w[NW];
-        load_cols<CPL>(W + (ok ? r * ldw + col : 0), ok, w);
+#pragma unroll
+        for (int k = 0; k < NW; ++k) w[k] = wn[k];
+        if (it + 1 < ITERS) {
+            const int64_t rn = r + CTA_WARPS * ROW_SLOTS;
+            const bool okn = col_ok && rn < R;
+            load_cols<CPL>(W + (okn ? rn * ldw + col : 0), okn, wn);
+        }
         float lo, hi;
         group_minmax<NW>(w, team, lo, hi);
         const float range = hi - lo;
         const bool live = range >= MIN_RANGE;
         const float inv = live ? qmax * rcp_approx(range) : 0.f;
         const float nscale = live ? -(range * inv_qmax) : 0.f;
-        const float nscale_lo = -(fmaf(nscale, qmax, range) * inv_qmax);   // two-float step
-        float ar = 1.f;
-        if (ROWW) ar = (r < R) ? row_weight[r] : 0.f;
-        float rs = 0.f;
+        const f32x2 inv2 = pk2(inv, inv), ns2 = pk2(nscale, nscale), nlo2 = pk2(-lo, -lo);
+        f32x2 nslo2 = 0ull;
+        if (FINE) {                                     // two-float step from 6 bits on
+            const float nscale_lo = -(fmaf(nscale, qmax, range) * inv_qmax);
+            nslo2 = pk2(nscale_lo, nscale_lo);
+        }
+        f32x2 ar2 = 0ull;
+        if (ROWW) {
+            const float ar = (r < R) ? row_weight[r] : 0.f;
+            ar2 = pk2(ar, ar);
+        }
+        f32x2 rs2 = 0ull;
 #pragma unroll
         for (int k = 0; k < NW; ++k) {
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const float vm = (h ? bf16hi(w[k]) : bf16lo(w[k])) - lo;
-                const float q = fmaf(vm, inv, RNE_MAGIC) - RNE_MAGIC;
-                const float e = fmaf(q, nscale_lo, fmaf(q, nscale, vm));
-                const float e2 = ROWW ? e * e * ar : e * e;
-                acc[2 * k + h] += e2;
-                rs = fmaf(cw[2 * k + h], e2, rs);
-            }
+            const f32x2 vm = add2(pk2(bf16lo(w[k]), bf16hi(w[k])), nlo2);
+            const f32x2 qq = add2(fma2(vm, inv2, magic2), nmagic2);
+            f32x2 e = fma2(qq, ns2, vm);
+            if (FINE) e = fma2(qq, nslo2, e);
+            f32x2 e2 = mul2(e, e);
+            if (ROWW) e2 = mul2(e2, ar2);
+            acc[k] = add2(acc[k], e2);
+            rs2 = fma2(cw[k], e2, rs2);
         }
+        float r0f, r1f;
+        upk2(rs2, r0f, r1f);
+        float rs = r0f + r1f;
 #pragma unroll
         for (int o = LANE_COLS >> 1; o > 0; o >>= 1) rs += __shfl_xor_sync(0xffffffffu, rs, o);
         if (rowpart && cl == 0 && r < R) rowpart[(int64_t)blockIdx.x * R + r] = rs;
     }
-    if (!colpart) return;
     __shared__ float red[CTA_WARPS * ROW_SLOTS][TILE_COLS + 4];
+    if (colpart) {
 #pragma unroll
-    for (int k = 0; k < CPL; ++k) red[warp * ROW_SLOTS + slot][cl * CPL + k] = acc[k] * cw[k];
-    __syncthreads();
-    if (threadIdx.x < TILE_COLS) {
-        const int64_t j = (int64_t)blockIdx.x * TILE_COLS + threadIdx.x;
-        if (j < C) {
-            float s = 0.f;
+        for (int k = 0; k < NW; ++k) {
+            float a0, a1, c0, c1;
+            upk2(acc[k], a0, a1);
+            upk2(cw[k], c0, c1);
+            red[warp * ROW_SLOTS + slot][cl * CPL + 2 * k] = a0 * c0;
+            red[warp * ROW_SLOTS + slot][cl * CPL + 2 * k + 1] = a1 * c1;
+        }
+        __syncthreads();
+        if (threadIdx.x < TILE_COLS) {
+            const int64_t j = (int64_t)blockIdx.x * TILE_COLS + threadIdx.x;
+            if (j < C) {
+                float s = 0.f;
 #pragma unroll
-            for (int p = 0; p < CTA_WARPS * ROW_SLOTS; ++p) s += red[p][threadIdx.x];
-            colpart[(int64_t)blockIdx.y * C + j] = s;
+                for (int p = 0; p < CTA_WARPS * ROW_SLOTS; ++p) s += red[p][threadIdx.x];
+                colpart[(int64_t)blockIdx.y * C + j] = s;
+            }
         }
     }
-}
-
-__global__ void sum_partials_kernel(const float* __restrict__ part, int nparts, int64_t n,
-                                    int accumulate, float* __restrict__ out, SbDeviceState* dstate) {
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    float s = 0.f;
-    for (int p = 0; p < nparts; ++p) s += part[(int64_t)p * n + i];
-    if (!isfinite(s)) sb_latch(dstate, SB_ERR_NONFINITE, SBK_STATS);
-    out[i] = accumulate ? out[i] + s : s;
+    // last tile of this tile row / tile column: add the strip's partials in tile order
+    __shared__ bool last_row, last_col;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        last_row = rowpart && atomicAdd(done_row + blockIdx.y, 1u) == gridDim.x - 1;
+        last_col = colpart && atomicAdd(done_col + blockIdx.x, 1u) == gridDim.y - 1;
+    }
+    __syncthreads();
+    if (!last_row && !last_col) return;
+    __threadfence();
+    if (last_row) {
+        for (int rr = threadIdx.x; rr < TILE_ROWS; rr += CTA_THREADS) {
+            const int64_t r = row0 + rr;
+            if (r < R) {
+                float s = 0.f;
+                for (unsigned t = 0; t < gridDim.x; ++t) s += __ldcg(rowpart + (int64_t)t * R + r);
+                if (!isfinite(s)) sb_latch(dstate, SB_ERR_NONFINITE, SBK_STATS);
+                row_score[r] = (accumulate & SB_ACC_ROW) ? row_score[r] + s : s;
+            }
+        }
+        if (threadIdx.x == 0) done_row[blockIdx.y] = 0u;
+    }
+    if (last_col && threadIdx.x >= CTA_THREADS - TILE_COLS) {
+        const int t0 = threadIdx.x - (CTA_THREADS - TILE_COLS);
+        const int64_t j = (int64_t)blockIdx.x * TILE_COLS + t0;
+        if (j < C) {
+            float s = 0.f;
+            for (unsigned t = 0; t < gridDim.y; ++t) s += __ldcg(colpart + (int64_t)t * C + j);
+            if (!isfinite(s)) sb_latch(dstate, SB_ERR_NONFINITE, SBK_STATS);
+            col_score[j] = (accumulate & SB_ACC_COL) ? col_score[j] + s : s;
+        }
+        if (t0 == 0) done_col[blockIdx.x] = 0u;
+    }
 }
 
 // ---- argsort by counting: rank_i = #{j in segment : s_j > s_i or (s_j == s_i and j < i)} ----
@@ -598,15 +670,15 @@ sb_status launch_scores(int nfine, A... args) {
 // used by pack.cu as well
 sb_status sb_gather_bf16(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw,
                          const int32_t* rp, const int32_t* cp, void* out) {
-    const size_t smem = (size_t)C * 2;
-    if (smem > 200 * 1024) return sb_fail(ctx, SB_ERR_SHAPE, "gather: rows longer than 102400 columns");
+    const size_t smem = (size_t)C * 2 * 2;          // two row buffers
+    if (smem > 200 * 1024) return sb_fail(ctx, SB_ERR_SHAPE, "gather: rows longer than 51200 columns");
     static bool attr_set = false;
     if (!attr_set) {
         SB_CUDA(ctx, cudaFuncSetAttribute(gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           200 * 1024));
         attr_set = true;
     }
-    int rows_per_cta = 4;
+    int rows_per_cta = 8;
     const unsigned grid = (unsigned)((R + rows_per_cta - 1) / rows_per_cta);
     gather_kernel<<<grid, CTA_THREADS, smem, ctx->stream>>>(
         static_cast<const __nv_bfloat16*>(W), R, C, ldw, rp, cp, static_cast<__nv_bfloat16*>(out),
@@ -635,7 +707,10 @@ sb_status sb_reorder_channels(sb_ctx* ctx, const void* W, int64_t R, int64_t C, 
             (reinterpret_cast<uintptr_t>(W) & 15))
             return sb_fail(ctx, SB_ERR_SHAPE, "reorder: group in {16,32,64,128} must divide C; ldw %% 8; 16-byte base");
     }
-    const int tiles_r = (int)((R + 127) / 128), tiles_c = (int)((C + 127) / 128);
+    const int tiles_c = (int)((C + 127) / 128);
+    // tall tiles (512 rows) amortise the per-CTA prologue and epilogue when they still fill the GPU
+    const int tile_rows = (R / 512) * tiles_c >= 2 * ctx->sm_count ? 512 : 128;
+    const int tiles_r = (int)((R + tile_rows - 1) / tile_rows);
     const int64_t maxK = R > C ? R : C;
     void* arena;
     sb_status st = sb_scratch(ctx, Carver::need({(size_t)tiles_c * R * 4, (size_t)tiles_r * C * 4,
@@ -647,27 +722,25 @@ sb_status sb_reorder_channels(sb_ctx* ctx, const void* W, int64_t R, int64_t C, 
     int* rank = cv.take<int>((size_t)maxK);
     if (W && (row_score || col_score)) {
         const float qmax = (float)((1 << ref_bits) - 1);
+        if (tiles_r > SB_STATS_TILES || tiles_c > SB_STATS_TILES)
+            return sb_fail(ctx, SB_ERR_SHAPE, "reorder: more than %d tiles on an axis", SB_STATS_TILES);
         dim3 grid(tiles_c, tiles_r);
         auto* Wb = static_cast<const __nv_bfloat16*>(W);
-        if (row_weight)
-            reorder_stats_kernel<true><<<grid, CTA_THREADS, 0, ctx->stream>>>(
-                Wb, R, C, ldw, col_moment, row_weight, group, qmax, 1.0f / qmax,
-                row_score ? rowpart : nullptr, col_score ? colpart : nullptr);
-        else
-            reorder_stats_kernel<false><<<grid, CTA_THREADS, 0, ctx->stream>>>(
-                Wb, R, C, ldw, col_moment, row_weight, group, qmax, 1.0f / qmax,
-                row_score ? rowpart : nullptr, col_score ? colpart : nullptr);
+        float* rpart = row_score ? rowpart : nullptr;
+        float* cpart = col_score ? colpart : nullptr;
+        unsigned* done_row = ctx->stats_done;
+        unsigned* done_col = ctx->stats_done + SB_STATS_TILES;
+#define SB_STATS2(RW, FN, TR)                                                                     \
+    reorder_stats_kernel<RW, FN, TR><<<grid, CTA_THREADS, 0, ctx->stream>>>(                      \
+        Wb, R, C, ldw, col_moment, row_weight, group, qmax, 1.0f / qmax, rpart, cpart, row_score, \
+        col_score, accumulate, done_row, done_col, ctx->dstate)
+#define SB_STATS(RW, FN) do { if (tile_rows == 512) SB_STATS2(RW, FN, 512); else SB_STATS2(RW, FN, 128); } while (0)
+        const bool fine = ref_bits >= 6;
+        if (row_weight) { if (fine) SB_STATS(true, true); else SB_STATS(true, false); }
+        else { if (fine) SB_STATS(false, true); else SB_STATS(false, false); }
+#undef SB_STATS
+#undef SB_STATS2
         SB_LAUNCHED(ctx);
-        if (row_score) {
-            sum_partials_kernel<<<(unsigned)((R + 255) / 256), 256, 0, ctx->stream>>>(
-                rowpart, tiles_c, R, accumulate & SB_ACC_ROW, row_score, ctx->dstate);
-            SB_LAUNCHED(ctx);
-        }
-        if (col_score) {
-            sum_partials_kernel<<<(unsigned)((C + 255) / 256), 256, 0, ctx->stream>>>(
-                colpart, tiles_r, C, accumulate & SB_ACC_COL, col_score, ctx->dstate);
-            SB_LAUNCHED(ctx);
-        }
     }
     if (sort_rows) { st = argsort_axis(ctx, row_score, R, row_segment, row_perm, rank); if (st) return st; }
     if (sort_cols) { st = argsort_axis(ctx, col_score, C, col_segment, col_perm, rank); if (st) return st; }
