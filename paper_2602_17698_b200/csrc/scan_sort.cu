@@ -36,42 +36,66 @@ scan_exclusive_kernel(const T* __restrict__ in, T* __restrict__ out, int64_t n, 
 }
 
 // ---- radix sort ---------------------------------------------------------------------------
+// Stable LSD sort, 8-bit digits, "one sweep" per digit: the digit histograms of all passes come
+// from one read of the keys; each pass then ranks its tile, publishes the tile's digit counts and
+// resolves its global offsets by decoupled look-back over the earlier tiles' descriptors (one
+// thread per digit), and scatters -- one launch per pass instead of histogram + scan + scatter.
 constexpr int SORT_THREADS = 256;
-constexpr int SORT_ITEMS = 8;                       // consecutive 32-item warp steps
+constexpr int SORT_ITEMS = 8;                          // consecutive 32-item warp steps
 constexpr int SORT_TILE = SORT_THREADS * SORT_ITEMS;   // 2048 keys per CTA
 constexpr int RADIX = 256;
+constexpr int SORT_PASSES = 8;
+constexpr unsigned OS_AGG = 1u << 30, OS_INC = 2u << 30, OS_MASK = (1u << 30) - 1u;
 
-// hist[digit * tiles + tile] = number of keys of the tile with that digit
+// ghist[pass][digit] += number of keys with that digit in that pass
 __global__ void __launch_bounds__(SORT_THREADS)
-radix_hist_kernel(const unsigned long long* __restrict__ keys, int64_t n, int shift, int tiles,
-                  unsigned* __restrict__ hist) {
-    __shared__ unsigned h[RADIX];
-    h[threadIdx.x] = 0;
+radix_hist_all_kernel(const unsigned long long* __restrict__ keys, int64_t n, unsigned* __restrict__ ghist) {
+    __shared__ unsigned h[SORT_PASSES][RADIX];
+    for (int i = threadIdx.x; i < SORT_PASSES * RADIX; i += SORT_THREADS) (&h[0][0])[i] = 0;
     __syncthreads();
     const int64_t base = (int64_t)blockIdx.x * SORT_TILE;
     for (int k = 0; k < SORT_ITEMS; ++k) {
         const int64_t i = base + k * SORT_THREADS + threadIdx.x;
-        if (i < n) atomicAdd(&h[(unsigned)(keys[i] >> shift) & 0xffu], 1u);
+        if (i < n) {
+            const unsigned long long key = keys[i];
+#pragma unroll
+            for (int p = 0; p < SORT_PASSES; ++p) atomicAdd(&h[p][(unsigned)(key >> (8 * p)) & 0xffu], 1u);
+        }
     }
     __syncthreads();
-    hist[(int64_t)threadIdx.x * tiles + blockIdx.x] = h[threadIdx.x];
+    for (int i = threadIdx.x; i < SORT_PASSES * RADIX; i += SORT_THREADS) {
+        const unsigned c = (&h[0][0])[i];
+        if (c) atomicAdd(ghist + i, c);
+    }
 }
 
-// Stable scatter.  Warp w of the CTA owns the contiguous keys [w*256, (w+1)*256) of the tile
-// and walks them 32 at a time; within a step equal digits are ranked by lane
-// (__match_any_sync), across steps by a per-warp running count, across warps by a prefix
-// over the warps' digit counts, across tiles by the scanned histogram.
+// gbase[pass][digit] = number of keys with a smaller digit in that pass (one CTA per pass)
+__global__ void __launch_bounds__(RADIX)
+radix_base_kernel(const unsigned* __restrict__ ghist, unsigned* __restrict__ gbase) {
+    unsigned total;
+    const unsigned v = ghist[blockIdx.x * RADIX + threadIdx.x];
+    gbase[blockIdx.x * RADIX + threadIdx.x] = block_exclusive_scan<unsigned, RADIX>(v, total);
+}
+
+// One pass.  Warp w of the CTA owns the contiguous keys [w*256, (w+1)*256) of the tile and walks
+// them 32 at a time; within a step equal digits are ranked by lane (__match_any_sync), across
+// steps by a per-warp running count, across warps by a prefix over the warps' digit counts,
+// across tiles by the look-back over desc[tile][digit] = flag | count.
 __global__ void __launch_bounds__(SORT_THREADS)
-radix_scatter_kernel(const unsigned long long* __restrict__ keys_in, const unsigned* __restrict__ vals_in,
+onesweep_pass_kernel(const unsigned long long* __restrict__ keys_in, const unsigned* __restrict__ vals_in,
                      unsigned long long* __restrict__ keys_out, unsigned* __restrict__ vals_out,
-                     int64_t n, int shift, int tiles, const unsigned* __restrict__ hist_scanned) {
+                     int64_t n, int shift, const unsigned* __restrict__ gbase, unsigned* __restrict__ desc,
+                     unsigned* __restrict__ ticket, SbDeviceState* st) {
     constexpr int WARPS = SORT_THREADS / 32;
     __shared__ unsigned cnt[WARPS][RADIX];          // running count per warp and digit
     __shared__ unsigned basepos[RADIX];
+    __shared__ unsigned tile_sh;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) tile_sh = atomicAdd(ticket, 1u);
     for (int d = lane; d < RADIX; d += 32) cnt[warp][d] = 0;
-    __syncwarp();
-    const int64_t wbase = (int64_t)blockIdx.x * SORT_TILE + (int64_t)warp * (32 * SORT_ITEMS);
+    __syncthreads();
+    const unsigned tile = tile_sh;
+    const int64_t wbase = (int64_t)tile * SORT_TILE + (int64_t)warp * (32 * SORT_ITEMS);
     unsigned long long key[SORT_ITEMS];
     unsigned val[SORT_ITEMS], rank[SORT_ITEMS];
 #pragma unroll
@@ -92,8 +116,8 @@ radix_scatter_kernel(const unsigned long long* __restrict__ keys_in, const unsig
         rank[k] = prior + before;
     }
     __syncthreads();
-    // prefix over warps for every digit (thread d handles digit d), plus the tile's base
     {
+        // thread d: prefix over the warps, publish the tile's count, look back for the offset
         const int d = threadIdx.x;
         unsigned run = 0;
 #pragma unroll
@@ -102,7 +126,36 @@ radix_scatter_kernel(const unsigned long long* __restrict__ keys_in, const unsig
             cnt[w][d] = run;
             run += c;
         }
-        basepos[d] = hist_scanned[(int64_t)d * tiles + blockIdx.x];
+        unsigned* mine = desc + (size_t)tile * RADIX + d;
+        unsigned excl = 0;
+        if (tile == 0) {
+            st_release_u32(mine, OS_INC | run);
+        } else {
+            st_release_u32(mine, OS_AGG | run);
+            bool timed_out = false;
+            for (int t = (int)tile - 1; t >= 0 && !timed_out; --t) {
+                const unsigned* p = desc + (size_t)t * RADIX + d;
+                unsigned v = ld_acquire_u32(p);
+                unsigned long long t_start = 0;
+                int spins = 0;
+                while ((v & ~OS_MASK) == 0u) {
+                    // bounded wait: a predecessor that never publishes must not hang the GPU
+                    if ((++spins & 63) == 0) {
+                        const unsigned long long now = lb_now_ns();
+                        if (t_start == 0) t_start = now;
+                        else if (now - t_start > LB_WAIT_NS) { timed_out = true; break; }
+                    }
+                    __nanosleep(64);
+                    v = ld_acquire_u32(p);
+                }
+                if (timed_out) break;
+                excl += v & OS_MASK;
+                if (v & OS_INC) break;
+            }
+            if (timed_out) sb_latch(st, SB_ERR_TIMEOUT, SBK_SORT);
+            st_release_u32(mine, OS_INC | ((excl + run) & OS_MASK));
+        }
+        basepos[d] = gbase[d] + excl;
     }
     __syncthreads();
 #pragma unroll
@@ -173,26 +226,34 @@ sb_status sb_scan_exclusive_u64(sb_ctx* ctx, const unsigned long long* in, unsig
 
 size_t sb_radix_sort_scratch_bytes(int64_t n) {
     const int64_t tiles = (n + SORT_TILE - 1) / SORT_TILE;
-    return (size_t)tiles * RADIX * sizeof(unsigned) * 2 + 512;
+    // histograms, bases, tickets, then the per-pass tile descriptors
+    return (size_t)(2 * SORT_PASSES * RADIX + 64) * sizeof(unsigned) +
+           (size_t)SORT_PASSES * tiles * RADIX * sizeof(unsigned) + 1024;
 }
 
 sb_status sb_radix_sort_u64(sb_ctx* ctx, unsigned long long* keys, unsigned long long* keys_tmp,
                             unsigned* vals, unsigned* vals_tmp, int64_t n, void* scratch) {
     if (n <= 0) return SB_OK;
+    if (n >= (1ll << 30)) return sb_fail(ctx, SB_ERR_SHAPE, "sort: more than 2^30 keys");
     const int tiles = (int)((n + SORT_TILE - 1) / SORT_TILE);
     Carver cv(scratch);
-    unsigned* hist = cv.take<unsigned>((size_t)tiles * RADIX);
-    unsigned* hist_scanned = cv.take<unsigned>((size_t)tiles * RADIX);
+    unsigned* ghist = cv.take<unsigned>(SORT_PASSES * RADIX);
+    unsigned* tickets = ghist + SORT_PASSES * RADIX;            // contiguous: one memset clears both
+    cv.take<unsigned>(64);
+    unsigned* gbase = cv.take<unsigned>(SORT_PASSES * RADIX);
+    unsigned* desc = cv.take<unsigned>((size_t)SORT_PASSES * tiles * RADIX);
+    SB_CUDA(ctx, cudaMemsetAsync(ghist, 0, (SORT_PASSES * RADIX + 64) * sizeof(unsigned), ctx->stream));
+    SB_CUDA(ctx, cudaMemsetAsync(desc, 0, (size_t)SORT_PASSES * tiles * RADIX * sizeof(unsigned), ctx->stream));
+    radix_hist_all_kernel<<<tiles, SORT_THREADS, 0, ctx->stream>>>(keys, n, ghist);
+    SB_LAUNCHED(ctx);
+    radix_base_kernel<<<SORT_PASSES, RADIX, 0, ctx->stream>>>(ghist, gbase);
+    SB_LAUNCHED(ctx);
     unsigned long long* kin = keys; unsigned long long* kout = keys_tmp;
     unsigned* vin = vals; unsigned* vout = vals_tmp;
-    for (int pass = 0; pass < 8; ++pass) {
-        const int shift = pass * 8;
-        radix_hist_kernel<<<tiles, SORT_THREADS, 0, ctx->stream>>>(kin, n, shift, tiles, hist);
-        SB_LAUNCHED(ctx);
-        sb_status st = sb_scan_exclusive_u32(ctx, hist, hist_scanned, (int64_t)tiles * RADIX);
-        if (st != SB_OK) return st;
-        radix_scatter_kernel<<<tiles, SORT_THREADS, 0, ctx->stream>>>(kin, vin, kout, vout, n, shift,
-                                                                      tiles, hist_scanned);
+    for (int pass = 0; pass < SORT_PASSES; ++pass) {
+        onesweep_pass_kernel<<<tiles, SORT_THREADS, 0, ctx->stream>>>(
+            kin, vin, kout, vout, n, pass * 8, gbase + pass * RADIX, desc + (size_t)pass * tiles * RADIX,
+            tickets + pass, ctx->dstate);
         SB_LAUNCHED(ctx);
         unsigned long long* tk = kin; kin = kout; kout = tk;
         unsigned* tv = vin; vin = vout; vout = tv;
