@@ -21,9 +21,10 @@ constexpr int AT = 256;             // threads of the scan-select kernels
 constexpr int AI = 8;               // entries per thread
 constexpr int ATILE = AT * AI;
 constexpr int BT = 256;             // threads of the per-block kernels
-constexpr int LT = 256;             // threads of the persistent loop kernel
-constexpr int LT_WARPS_MAX = LT / 32;
+constexpr int LT_WARPS_MAX = 32;
 constexpr int LOOP_MAX_CTAS = 4096;
+constexpr int GL_THREADS = 256;     // grid (cooperative) form of the loop kernel
+constexpr int CL_THREADS = 512, CL_CTAS = 16;   // cluster form
 constexpr int LC = 4;               // list entries a thread keeps in registers between passes
 
 struct AllocState {
@@ -199,10 +200,16 @@ __device__ __forceinline__ T cta_total_u(T v) {
     return r;
 }
 
+template <int LT, bool CLUSTER>
 __global__ void __launch_bounds__(LT)
 scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
                       const unsigned* __restrict__ dn_list, long long ne, LoopWork w) {
-    cg::grid_group grid = cg::this_grid();
+    // CLUSTER: the whole grid is one thread-block cluster and the phase barrier is the hardware
+    // cluster barrier; otherwise a cooperative launch and the grid-wide barrier
+    auto phase_barrier = [&]() {
+        if (CLUSTER) cg::this_cluster().sync();
+        else cg::this_grid().sync();
+    };
     const int G = gridDim.x, c = blockIdx.x, tid = threadIdx.x;
     const long long per_cta = (ne + G - 1) / G;
     const long long ipt = (per_cta + LT - 1) / LT;                    // entries per thread
@@ -267,7 +274,7 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
             w.up_tot[c] = cta_tot;
             if (cta_tot.cnt == 0) w.up_first[c] = -1;
         }
-        grid.sync();
+        phase_barrier();
 
         // ---- prefix over the lower CTAs, cost of the globally first candidate ------------------
         unsigned long long pre_cost = 0; unsigned pre_cnt = 0; int first_cta = 0x7fffffff;
@@ -325,7 +332,7 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
             const unsigned nu = cta_total_u<unsigned>(nU_mine);
             if (tid == 0) { w.dU[c] = d; w.costU[c] = cu; w.nU[c] = nu; }
         }
-        grid.sync();
+        phase_barrier();
 
         if (!expand) {
             // ---- down-count ----------------------------------------------------------------------
@@ -347,7 +354,7 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
             CntCost dn_cta;
             const CntCost dex = block_exclusive_scan<CntCost, LT>(dm, dn_cta);
             if (tid == 0) w.dn_tot[c] = dn_cta;
-            grid.sync();
+            phase_barrier();
             unsigned dpre = 0;
             for (int j = tid; j < c; j += LT) dpre += ldcg_cc(w.dn_tot + j).cnt;
             dpre = cta_total_u<unsigned>(dpre);
@@ -368,7 +375,7 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
                 const unsigned nd = cta_total_u<unsigned>(nD_mine);
                 if (tid == 0) { w.dD[c] = d; w.freed[c] = f; w.nD[c] = nd; }
             }
-            grid.sync();
+            phase_barrier();
             // ---- U: up-candidates 0..h-1 whose cumulative cost fits slack + what D frees ------------
             unsigned long long freed_tot = 0;
             for (int j = tid; j < G; j += LT) freed_tot += __ldcg(w.freed + j);
@@ -388,7 +395,7 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
             const unsigned long long cu = cta_total_u<unsigned long long>(costU_mine);
             const unsigned nu = cta_total_u<unsigned>(nU_mine);
             if (tid == 0) { w.dU[c] = d; w.costU[c] = cu; w.nU[c] = nu; }
-            grid.sync();
+            phase_barrier();
         }
 
         // ---- totals (same order in every CTA), decision, apply, replicated state update -----------
@@ -422,7 +429,7 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
         else if (accept) { used += (long long)costU - (long long)freed; loss += dD - dU; accepted += 1; }
         else { k /= 2; rejected += 1; }
         iter += 1;
-        grid.sync();                                  // the new levels are visible to the next up-count
+        phase_barrier();                                  // the new levels are visible to the next up-count
     }
     if (c == 0 && tid == 0) {
         AllocState* st = a.st;
@@ -680,16 +687,6 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
             SB_LAUNCHED(ctx);
             reverse_runs_kernel<<<g, 256, 0, ctx->stream>>>(vA, vB, vD, run_start, nsteps, vC);
             SB_LAUNCHED(ctx);
-            // the whole loop in one cooperative launch
-            int occ = 0;
-            SB_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scalebits_loop_kernel, LT, 0));
-            long long G = (long long)occ * ctx->sm_count;
-            // a few list entries per thread: grid barriers cost more with more CTAs than the
-            // short passes gain
-            const long long want = (nsteps + LC * LT - 1) / (LC * LT);
-            if (G > want) G = want;
-            if (G > LOOP_MAX_CTAS) G = LOOP_MAX_CTAS;
-            if (G < 1) G = 1;
             LoopWork lw;
             lw.up_tot = loop_cc; lw.dn_tot = loop_cc + LOOP_MAX_CTAS;
             lw.up_first = loop_ll;
@@ -699,8 +696,44 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
             const unsigned* up_list = vA; const unsigned* dn_list = vC;
             long long ne = nsteps;
             void* kargs[] = {&a, &up_list, &dn_list, &ne, &lw};
-            SB_CUDA(ctx, cudaLaunchCooperativeKernel((const void*)scalebits_loop_kernel, dim3((unsigned)G),
-                                                     dim3(LT), kargs, 0, ctx->stream));
+            bool launched = false;
+            // Small problems: one thread-block cluster of 16 CTAs x 512 threads; its hardware
+            // barrier is several times cheaper than a grid-wide one, and a handful of list
+            // entries per thread is all the parallelism the passes need.
+            if (nsteps <= (long long)CL_CTAS * CL_THREADS * 16) {
+                auto kern = scalebits_loop_kernel<CL_THREADS, true>;
+                static bool attr_done = false;
+                if (!attr_done) {
+                    SB_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+                    attr_done = true;
+                }
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(CL_CTAS);
+                cfg.blockDim = dim3(CL_THREADS);
+                cfg.stream = ctx->stream;
+                cudaLaunchAttribute at[1];
+                at[0].id = cudaLaunchAttributeClusterDimension;
+                at[0].val.clusterDim.x = CL_CTAS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+                cfg.attrs = at; cfg.numAttrs = 1;
+                cudaError_t e = cudaLaunchKernelExC(&cfg, (const void*)kern, kargs);
+                if (e == cudaSuccess) launched = true;
+                else (void)cudaGetLastError();        // no room for such a cluster: use the grid form
+            }
+            if (!launched) {
+                // the whole loop in one cooperative launch
+                auto kern = scalebits_loop_kernel<GL_THREADS, false>;
+                int occ = 0;
+                SB_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, GL_THREADS, 0));
+                long long G = (long long)occ * ctx->sm_count;
+                // a few list entries per thread: grid barriers cost more with more CTAs than the
+                // short passes gain
+                const long long want = (nsteps + LC * GL_THREADS - 1) / (LC * GL_THREADS);
+                if (G > want) G = want;
+                if (G > LOOP_MAX_CTAS) G = LOOP_MAX_CTAS;
+                if (G < 1) G = 1;
+                SB_CUDA(ctx, cudaLaunchCooperativeKernel((const void*)kern, dim3((unsigned)G), dim3(GL_THREADS),
+                                                         kargs, 0, ctx->stream));
+            }
             ctx->launches++;
         }
         // single candidate (or finished): histogram of the final levels
