@@ -25,7 +25,8 @@ constexpr int LT_WARPS_MAX = 32;
 constexpr int LOOP_MAX_CTAS = 4096;
 constexpr int GL_THREADS = 256;     // grid (cooperative) form of the loop kernel
 constexpr int CL_THREADS = 512, CL_CTAS = 16;   // cluster form
-constexpr int LC = 4;               // list entries a thread keeps in registers between passes
+constexpr int LC = 4;               // list entries a thread has in flight at a time
+constexpr unsigned ENT_NONE = 0xffffffffu;      // list entry that is never a candidate
 
 struct AllocState {
     long long cap, used;
@@ -48,8 +49,9 @@ struct AllocArgs {
     long long N; int L; int bits[8];
     unsigned char* level;
     AllocState* st;
-    unsigned* uprank; unsigned* upstamp; unsigned long long* upcum;   // per block
-    unsigned* dnstamp; unsigned* ustamp;                               // per block
+    // per block: (stamp << 32 | rank) of its up-candidate, the cumulative cost and the error
+    // difference of that candidate, and the move marked for the apply step (stamp << 1 | down)
+    unsigned long long* upsr; unsigned long long* upcum; double* upde; unsigned* mark;
     double* part;                                                      // partial sums
 };
 
@@ -120,14 +122,27 @@ __global__ void run_starts_kernel(const unsigned* __restrict__ head, const unsig
     if (head[p]) start[excl[p]] = (unsigned)p;                    // run id = excl[p]
     if (p == n - 1) start[excl[p] + head[p]] = (unsigned)n;       // one past the last run
 }
-__global__ void reverse_runs_kernel(const unsigned* __restrict__ up_list, const unsigned* __restrict__ head,
-                                    const unsigned* __restrict__ excl, const unsigned* __restrict__ start,
-                                    long long n, unsigned* __restrict__ dn_list) {
+// Both lists in the form the loop reads: entry = block << 3 | from-level, plus the error
+// difference of the step.  Up-steps that do not lower the error are never candidates.
+__global__ void entry_info_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
+                                  const unsigned* __restrict__ head, const unsigned* __restrict__ excl,
+                                  const unsigned* __restrict__ start, long long n,
+                                  unsigned* __restrict__ up_ent, double* __restrict__ up_de,
+                                  unsigned* __restrict__ dn_ent, double* __restrict__ dn_de) {
     const long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (p >= n) return;
+    const unsigned e = up_list[p], Lm1 = (unsigned)(a.L - 1);
+    const unsigned i = e / Lm1, l = e - i * Lm1;
+    const float e0 = a.err[(long long)i * a.L + l], e1 = a.err[(long long)i * a.L + l + 1];
+    const double de = __dsub_rn((double)e0, (double)e1);
+    const unsigned ent = (i << 3) | l;
+    up_ent[p] = e0 > e1 ? ent : ENT_NONE;
+    up_de[p] = de;
     const unsigned r = excl[p] + head[p] - 1u;
-    const long long a = start[r], b = start[r + 1];
-    dn_list[(n - b) + (p - a)] = up_list[p];
+    const long long ra = start[r], rb = start[r + 1];
+    const long long q = (n - rb) + (p - ra);
+    dn_ent[q] = ent;
+    dn_de[q] = de;
 }
 
 // level = l0 everywhere; loss / used partial sums; also clears the per-block stamps
@@ -139,7 +154,7 @@ __global__ void __launch_bounds__(BT) init_levels_kernel(AllocArgs a, int l0, in
         a.level[i] = (unsigned char)l0;
         e = (double)a.err[i * a.L + l0];
         u = elems_of(a, i) * a.bits[l0];
-        if (clear) { a.upstamp[i] = 0; a.dnstamp[i] = 0; a.ustamp[i] = 0; }
+        if (clear) { a.upsr[i] = 0ull; a.mark[i] = 0u; }
     }
     const double s = cta_sum<BT>(e);
     if (threadIdx.x == 0) a.part[blockIdx.x] = s;
@@ -156,17 +171,19 @@ __global__ void init_finish_kernel(AllocArgs a, int nparts) {
     a.st->loss_init = s;
 }
 
-// ---- the Algorithm 2 loop, one persistent cooperative kernel ----------------------------------
-// All iterations run inside one launch; the phases of an iteration are separated by grid-wide
-// barriers (cooperative launch: every CTA is resident).  CTA c owns a contiguous slice of both
-// sorted lists.  A "select" is two passes over the slice: (1) count the candidates and add up
-// their costs, publish the CTA total; (2) after the barrier, the exclusive prefix over the
-// lower CTAs gives every candidate its global rank p and cumulative cost.  The loop state
-// (k, used, loss, counters) is replicated: every CTA derives it from the same published
+// ---- the Algorithm 2 loop, one persistent kernel ----------------------------------------------
+// All iterations run inside one launch; the phases of an iteration are separated by barriers over
+// all CTAs (every CTA is resident: one thread-block cluster, or a cooperative launch).  CTA c owns
+// a contiguous slice of both sorted lists.  A "select" is two passes over the slice: (1) count the
+// candidates and add up their costs, publish the CTA total; (2) after the barrier, the exclusive
+// prefix over the lower CTAs gives every candidate its global rank and cumulative cost.  The loop
+// state (k, used, loss, counters) is replicated: every CTA derives it from the same published
 // totals, added in the same order, so no CTA has to wait for a single writer.
 //   expansion iteration: up-count | up-rank + U | apply            (3 barriers)
 //   exchange  iteration: up-count | up-rank | down-count | down-rank + D | U | apply   (6)
-// Data written by other CTAs during the kernel is read through L2 (__ldcg): L1 is not
+// The lists are static: entry p carries (block << 3 | from-level) and the error difference of its
+// step, so a pass costs one dependent load (the block's current level), issued for LC entries at a
+// time.  Data written by other CTAs during the kernel is read through L2 (__ldcg): L1 is not
 // coherent across SMs inside one launch.
 struct LoopWork {
     CntCost* up_tot; long long* up_first; CntCost* dn_tot;
@@ -180,30 +197,53 @@ __device__ __forceinline__ CntCost ldcg_cc(const CntCost* p) {
     return c;
 }
 
-// sum of one value per thread over the CTA, valid in every thread (fixed order)
-template <typename T>
-__device__ __forceinline__ T cta_total_u(T v) {
-    __shared__ T sh[LT_WARPS_MAX];
-    __shared__ T tot;
+// Reduction of K 64-bit values per thread over the CTA, result in every thread, fixed order.
+// OPS holds two bits per slot: 0 = sum, 1 = min, 2 = max.  One barrier per call: the buffer
+// alternates, and any later call's barrier separates a buffer's readers from its next writers.
+template <int OP>
+__device__ __forceinline__ unsigned long long red_op(unsigned long long x, unsigned long long y) {
+    if constexpr (OP == 0) return x + y;
+    else if constexpr (OP == 1) return x < y ? x : y;
+    else return x > y ? x : y;
+}
+template <int NT, int K, int OPS, int S = 0>
+__device__ __forceinline__ void allreduce_slot(unsigned long long (&v)[K], unsigned long long (*sh)[K]) {
+    if constexpr (S < K) {
+        constexpr int OP = (OPS >> (2 * S)) & 3;
+        unsigned long long r = sh[0][S];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        T s = 0;
-        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += sh[w];
-        tot = s;
+        for (int wq = 1; wq < NT / 32; ++wq) r = red_op<OP>(r, sh[wq][S]);
+        v[S] = r;
+        allreduce_slot<NT, K, OPS, S + 1>(v, sh);
+    }
+}
+template <int NT, int K, int OPS, int S = 0>
+__device__ __forceinline__ void warpreduce_slot(unsigned long long (&v)[K]) {
+    if constexpr (S < K) {
+        constexpr int OP = (OPS >> (2 * S)) & 3;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v[S] = red_op<OP>(v[S], __shfl_xor_sync(0xffffffffu, v[S], o));
+        warpreduce_slot<NT, K, OPS, S + 1>(v);
+    }
+}
+template <int NT, int K, int OPS>
+__device__ __forceinline__ void cta_allreduce(unsigned long long (&v)[K], unsigned& flip) {
+    __shared__ unsigned long long sh[2][NT / 32][K];
+    warpreduce_slot<NT, K, OPS>(v);
+    if ((threadIdx.x & 31) == 0) {
+#pragma unroll
+        for (int s = 0; s < K; ++s) sh[flip][threadIdx.x >> 5][s] = v[s];
     }
     __syncthreads();
-    const T r = tot;
-    __syncthreads();
-    return r;
+    allreduce_slot<NT, K, OPS>(v, sh[flip]);
+    flip ^= 1u;
 }
 
 template <int LT, bool CLUSTER>
 __global__ void __launch_bounds__(LT)
-scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
-                      const unsigned* __restrict__ dn_list, long long ne, LoopWork w) {
+scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, const double* __restrict__ up_de,
+                      const unsigned* __restrict__ dn_ent, const double* __restrict__ dn_de,
+                      long long ne, LoopWork w) {
     // CLUSTER: the whole grid is one thread-block cluster and the phase barrier is the hardware
     // cluster barrier; otherwise a cooperative launch and the grid-wide barrier
     auto phase_barrier = [&]() {
@@ -216,25 +256,59 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
     const long long cta_hi = min(ne, (long long)(c + 1) * per_cta);
     const long long t_lo = min(cta_hi, (long long)c * per_cta + (long long)tid * ipt);
     const long long t_hi = min(cta_hi, t_lo + ipt);
-    const unsigned Lm1 = (unsigned)(a.L - 1);
 
     const AllocState s0 = *a.st;                    // written before the launch
     const long long cap = s0.cap, kT = s0.kT;
     long long k = s0.k, used = s0.used;
     double loss = s0.loss;
     int iter = 0, accepted = 0, rejected = 0, expansions = 0, status = 0;
+    unsigned flip = 0;
 
-    // candidate test of one list entry; returns the block or -1
-    auto up_entry = [&](long long p, unsigned long long& cost, double& de) -> long long {
-        const unsigned e = up_list[p];
-        const long long i = e / Lm1;
-        const int l = (int)(e % Lm1);
-        if ((int)__ldcg(a.level + i) != l) return -1;
-        const float e0 = a.err[i * a.L + l], e1 = a.err[i * a.L + l + 1];
-        if (!(e0 > e1)) return -1;
-        cost = (unsigned long long)(elems_of(a, i) * (a.bits[l + 1] - a.bits[l]));
-        de = __dsub_rn((double)e0, (double)e1);
-        return i;
+    // bit difference of the step l -> l + 1 in nibble l (a table in registers, not in local memory)
+    unsigned dbits = 0;
+#pragma unroll
+    for (int l = 0; l < 7; ++l) dbits |= (unsigned)(a.bits[l + 1] > a.bits[l] ? a.bits[l + 1] - a.bits[l] : 0) << (4 * l);
+    const long long* const block_elems = a.block_elems;
+    const long long uniform = a.uniform;
+    auto cost_of = [&](unsigned e) -> unsigned long long {
+        const long long m = block_elems ? block_elems[e >> 3] : uniform;
+        return (unsigned long long)(m * (long long)((dbits >> (4u * (e & 7u))) & 15u));
+    };
+    // visit(p, e) for this thread's up-candidates in list order, until it returns false
+    auto for_up = [&](auto&& visit) {
+        for (long long base = t_lo; base < t_hi; base += LC) {
+            unsigned e[LC]; int lv[LC];
+#pragma unroll
+            for (int j = 0; j < LC; ++j) e[j] = base + j < t_hi ? __ldg(up_ent + base + j) : ENT_NONE;
+#pragma unroll
+            for (int j = 0; j < LC; ++j) lv[j] = e[j] != ENT_NONE ? (int)__ldcg(a.level + (e[j] >> 3)) : -1;
+#pragma unroll
+            for (int j = 0; j < LC; ++j)
+                if (lv[j] == (int)(e[j] & 7u)) { if (!visit(base + j, e[j])) return; }
+        }
+    };
+    // down-candidates: the step ends at the block's level and the block is not among the first
+    // h up-candidates of this iteration
+    auto for_dn = [&](unsigned stamp, long long h, auto&& visit) {
+        for (long long base = t_lo; base < t_hi; base += LC) {
+            unsigned e[LC]; int lv[LC]; unsigned long long sr[LC];
+#pragma unroll
+            for (int j = 0; j < LC; ++j) e[j] = base + j < t_hi ? __ldg(dn_ent + base + j) : ENT_NONE;
+#pragma unroll
+            for (int j = 0; j < LC; ++j) {
+                lv[j] = -1; sr[j] = 0ull;
+                if (e[j] != ENT_NONE) {
+                    lv[j] = (int)__ldcg(a.level + (e[j] >> 3));
+                    sr[j] = __ldcg(a.upsr + (e[j] >> 3));
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < LC; ++j) {
+                if (lv[j] != (int)(e[j] & 7u) + 1) continue;
+                if ((unsigned)(sr[j] >> 32) == stamp && (long long)(unsigned)sr[j] < h) continue;
+                if (!visit(base + j, e[j])) return;
+            }
+        }
     };
 
     while (k >= kT) {
@@ -243,30 +317,15 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
         const long long slack = cap - used;
         const long long h = k / 2 > 0 ? k / 2 : 1;
 
-        // ---- up-count (a thread with at most LC entries keeps them for the rank pass) -----------
+        // ---- up-count ---------------------------------------------------------------------------
         CntCost mine{0ull, 0u, 0u};
         long long my_first = -1;
-        long long c_blk[LC]; unsigned long long c_cost[LC]; double c_de[LC];
-        const bool cached = ipt <= LC;
-        if (cached) {
-#pragma unroll
-            for (int j = 0; j < LC; ++j) {
-                c_blk[j] = -1; c_cost[j] = 0; c_de[j] = 0.0;
-                if (t_lo + j < t_hi) c_blk[j] = up_entry(t_lo + j, c_cost[j], c_de[j]);
-                if (c_blk[j] >= 0) {
-                    if (mine.cnt == 0) my_first = (long long)c_cost[j];
-                    mine.cnt += 1; mine.cost += c_cost[j];
-                }
-            }
-        } else {
-            for (long long p = t_lo; p < t_hi; ++p) {
-                unsigned long long cost; double de;
-                if (up_entry(p, cost, de) >= 0) {
-                    if (mine.cnt == 0) my_first = (long long)cost;
-                    mine.cnt += 1; mine.cost += cost;
-                }
-            }
-        }
+        for_up([&](long long, unsigned e) {
+            const unsigned long long cost = cost_of(e);
+            if (mine.cnt == 0) my_first = (long long)cost;
+            mine.cnt += 1; mine.cost += cost;
+            return true;
+        });
         CntCost cta_tot;
         const CntCost ex = block_exclusive_scan<CntCost, LT>(mine, cta_tot);
         if (ex.cnt == 0 && mine.cnt > 0) w.up_first[c] = my_first;      // the CTA's first candidate
@@ -277,124 +336,93 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
         phase_barrier();
 
         // ---- prefix over the lower CTAs, cost of the globally first candidate ------------------
-        unsigned long long pre_cost = 0; unsigned pre_cnt = 0; int first_cta = 0x7fffffff;
+        unsigned long long pre[3] = {0ull, 0ull, 0x7fffffffull};      // cost, count, first CTA with one
         for (int j = tid; j < G; j += LT) {
             const CntCost t = ldcg_cc(w.up_tot + j);
-            if (j < c) { pre_cost += t.cost; pre_cnt += t.cnt; }
-            if (t.cnt > 0 && j < first_cta) first_cta = j;
+            if (j < c) { pre[0] += t.cost; pre[1] += t.cnt; }
+            if (t.cnt > 0 && (unsigned long long)j < pre[2]) pre[2] = (unsigned long long)j;
         }
-        pre_cost = cta_total_u<unsigned long long>(pre_cost);
-        pre_cnt = cta_total_u<unsigned>(pre_cnt);
-        {
-            __shared__ int fc;
-            if (tid == 0) fc = 0x7fffffff;
-            __syncthreads();
-            if (first_cta != 0x7fffffff) atomicMin(&fc, first_cta);
-            __syncthreads();
-            first_cta = fc;
-            __syncthreads();
-        }
-        const long long first_cost = first_cta != 0x7fffffff ? __ldcg(w.up_first + first_cta) : -1;
+        cta_allreduce<LT, 3, 0 | (0 << 2) | (1 << 4)>(pre, flip);
+        const long long first_cost = pre[2] != 0x7fffffffull ? __ldcg(w.up_first + pre[2]) : -1;
         const bool expand = used < cap && first_cost >= 0 && first_cost <= slack;
         const long long lim_rank = expand ? k : h;
 
         // ---- up-rank (and, in an expansion, the set U itself) -----------------------------------
+        // U is a prefix of the ranked candidates, so its cost is the largest cumulative cost in it
         double dU_mine = 0.0; unsigned long long costU_mine = 0; unsigned nU_mine = 0;
-        if ((long long)pre_cnt + ex.cnt < lim_rank) {
-            unsigned long long run_cost = pre_cost + ex.cost;
-            long long run_cnt = (long long)pre_cnt + ex.cnt;
-            auto take = [&](long long i, unsigned long long cost, double de) {
-                run_cost += cost;
-                a.uprank[i] = (unsigned)run_cnt;
+        if (mine.cnt > 0 && (long long)pre[1] + ex.cnt < lim_rank) {
+            unsigned long long run_cost = pre[0] + ex.cost;
+            long long run_cnt = (long long)pre[1] + ex.cnt;
+            for_up([&](long long p, unsigned e) {
+                const long long i = (long long)(e >> 3);
+                const double de = __ldg(up_de + p);
+                run_cost += cost_of(e);
+                a.upsr[i] = ((unsigned long long)stamp << 32) | (unsigned long long)(unsigned)run_cnt;
                 a.upcum[i] = run_cost;
-                a.upstamp[i] = stamp;
+                a.upde[i] = de;
                 if (expand && (long long)run_cost <= slack) {
-                    a.ustamp[i] = stamp;
-                    dU_mine += de; costU_mine += cost; nU_mine += 1;
+                    a.mark[i] = stamp << 1;
+                    dU_mine += de; costU_mine = run_cost; nU_mine += 1;
                 }
                 run_cnt += 1;
-            };
-            if (cached) {
-#pragma unroll
-                for (int j = 0; j < LC; ++j)
-                    if (c_blk[j] >= 0 && run_cnt < lim_rank) take(c_blk[j], c_cost[j], c_de[j]);
-            } else {
-                for (long long p = t_lo; p < t_hi && run_cnt < lim_rank; ++p) {
-                    unsigned long long cost; double de;
-                    const long long i = up_entry(p, cost, de);
-                    if (i >= 0) take(i, cost, de);
-                }
-            }
+                return run_cnt < lim_rank;
+            });
         }
         if (expand) {
             const double d = cta_sum<LT>(dU_mine);
-            const unsigned long long cu = cta_total_u<unsigned long long>(costU_mine);
-            const unsigned nu = cta_total_u<unsigned>(nU_mine);
-            if (tid == 0) { w.dU[c] = d; w.costU[c] = cu; w.nU[c] = nu; }
+            unsigned long long r2[2] = {costU_mine, nU_mine};
+            cta_allreduce<LT, 2, 2 | (0 << 2)>(r2, flip);
+            if (tid == 0) { w.dU[c] = d; w.costU[c] = r2[0]; w.nU[c] = (unsigned)r2[1]; }
         }
         phase_barrier();
 
         if (!expand) {
             // ---- down-count ----------------------------------------------------------------------
-            auto dn_entry = [&](long long p, unsigned long long& cost, double& de) -> long long {
-                const unsigned e = dn_list[p];
-                const long long i = e / Lm1;
-                const int l = (int)(e % Lm1);
-                if ((int)__ldcg(a.level + i) != l + 1) return -1;
-                if (__ldcg(a.upstamp + i) == stamp && (long long)__ldcg(a.uprank + i) < h) return -1;
-                cost = (unsigned long long)(elems_of(a, i) * (a.bits[l + 1] - a.bits[l]));
-                de = __dsub_rn((double)a.err[i * a.L + l], (double)a.err[i * a.L + l + 1]);
-                return i;
-            };
             CntCost dm{0ull, 0u, 0u};
-            for (long long p = t_lo; p < t_hi; ++p) {
-                unsigned long long cost; double de;
-                if (dn_entry(p, cost, de) >= 0) { dm.cnt += 1; dm.cost += cost; }
-            }
+            for_dn(stamp, h, [&](long long, unsigned e) { dm.cnt += 1; dm.cost += cost_of(e); return true; });
             CntCost dn_cta;
             const CntCost dex = block_exclusive_scan<CntCost, LT>(dm, dn_cta);
             if (tid == 0) w.dn_tot[c] = dn_cta;
             phase_barrier();
-            unsigned dpre = 0;
-            for (int j = tid; j < c; j += LT) dpre += ldcg_cc(w.dn_tot + j).cnt;
-            dpre = cta_total_u<unsigned>(dpre);
+            unsigned long long dpre[1] = {0ull};
+            for (int j = tid; j < c; j += LT) dpre[0] += ldcg_cc(w.dn_tot + j).cnt;
+            cta_allreduce<LT, 1, 0>(dpre, flip);
             // ---- down-rank: the first h candidates form D -----------------------------------------
             double dD_mine = 0.0; unsigned long long freed_mine = 0; unsigned nD_mine = 0;
-            long long run_cnt = (long long)dpre + dex.cnt;
-            for (long long p = t_lo; p < t_hi && run_cnt < h; ++p) {
-                unsigned long long cost; double de;
-                const long long i = dn_entry(p, cost, de);
-                if (i < 0) continue;
-                a.dnstamp[i] = stamp;
-                dD_mine += de; freed_mine += cost; nD_mine += 1;
-                run_cnt += 1;
+            if (dm.cnt > 0 && (long long)dpre[0] + dex.cnt < h) {
+                long long run_cnt = (long long)dpre[0] + dex.cnt;
+                for_dn(stamp, h, [&](long long p, unsigned e) {
+                    a.mark[e >> 3] = (stamp << 1) | 1u;
+                    dD_mine += __ldg(dn_de + p); freed_mine += cost_of(e); nD_mine += 1;
+                    run_cnt += 1;
+                    return run_cnt < h;
+                });
             }
             {
                 const double d = cta_sum<LT>(dD_mine);
-                const unsigned long long f = cta_total_u<unsigned long long>(freed_mine);
-                const unsigned nd = cta_total_u<unsigned>(nD_mine);
-                if (tid == 0) { w.dD[c] = d; w.freed[c] = f; w.nD[c] = nd; }
+                unsigned long long r2[2] = {freed_mine, nD_mine};
+                cta_allreduce<LT, 2, 0>(r2, flip);
+                if (tid == 0) { w.dD[c] = d; w.freed[c] = r2[0]; w.nD[c] = (unsigned)r2[1]; }
             }
             phase_barrier();
             // ---- U: up-candidates 0..h-1 whose cumulative cost fits slack + what D frees ------------
-            unsigned long long freed_tot = 0;
-            for (int j = tid; j < G; j += LT) freed_tot += __ldcg(w.freed + j);
-            freed_tot = cta_total_u<unsigned long long>(freed_tot);
-            const long long lim_cost = slack + (long long)freed_tot;
+            unsigned long long fr[1] = {0ull};
+            for (int j = tid; j < G; j += LT) fr[0] += __ldcg(w.freed + j);
+            cta_allreduce<LT, 1, 0>(fr, flip);
+            const long long lim_cost = slack + (long long)fr[0];
             for (long long i = (long long)c * LT + tid; i < a.N; i += (long long)G * LT) {
-                if (__ldcg(a.upstamp + i) == stamp && (long long)__ldcg(a.uprank + i) < h &&
-                    (long long)__ldcg(a.upcum + i) <= lim_cost) {
-                    const int l = (int)__ldcg(a.level + i);
-                    a.ustamp[i] = stamp;
-                    dU_mine += __dsub_rn((double)a.err[i * a.L + l], (double)a.err[i * a.L + l + 1]);
-                    costU_mine += (unsigned long long)(elems_of(a, i) * (a.bits[l + 1] - a.bits[l]));
-                    nU_mine += 1;
+                const unsigned long long sr = __ldcg(a.upsr + i), cum = __ldcg(a.upcum + i);
+                const double de = __ldcg(a.upde + i);
+                if ((unsigned)(sr >> 32) == stamp && (long long)(unsigned)sr < h && (long long)cum <= lim_cost) {
+                    a.mark[i] = stamp << 1;
+                    dU_mine += de; nU_mine += 1;
+                    if (cum > costU_mine) costU_mine = cum;
                 }
             }
             const double d = cta_sum<LT>(dU_mine);
-            const unsigned long long cu = cta_total_u<unsigned long long>(costU_mine);
-            const unsigned nu = cta_total_u<unsigned>(nU_mine);
-            if (tid == 0) { w.dU[c] = d; w.costU[c] = cu; w.nU[c] = nu; }
+            unsigned long long r2[2] = {costU_mine, nU_mine};
+            cta_allreduce<LT, 2, 2 | (0 << 2)>(r2, flip);
+            if (tid == 0) { w.dU[c] = d; w.costU[c] = r2[0]; w.nU[c] = (unsigned)r2[1]; }
             phase_barrier();
         }
 
@@ -406,23 +434,23 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_list,
             if (!expand) for (int j = 0; j < G; ++j) dsum += __ldcg(w.dD + j);
             sh_dU = u; sh_dD = dsum;
         }
-        unsigned long long costU = 0, freed = 0; unsigned nU = 0, nD = 0;
+        unsigned long long tot[4] = {0ull, 0ull, 0ull, 0ull};       // costU (max), nU, freed, nD
         for (int j = tid; j < G; j += LT) {
-            costU += __ldcg(w.costU + j); nU += __ldcg(w.nU + j);
-            if (!expand) { freed += __ldcg(w.freed + j); nD += __ldcg(w.nD + j); }
+            const unsigned long long cu = __ldcg(w.costU + j);
+            if (cu > tot[0]) tot[0] = cu;
+            tot[1] += __ldcg(w.nU + j);
+            if (!expand) { tot[2] += __ldcg(w.freed + j); tot[3] += __ldcg(w.nD + j); }
         }
-        costU = cta_total_u<unsigned long long>(costU);
-        freed = cta_total_u<unsigned long long>(freed);
-        nU = cta_total_u<unsigned>(nU);
-        nD = cta_total_u<unsigned>(nD);
-        __syncthreads();
+        cta_allreduce<LT, 4, 2 | (0 << 2) | (0 << 4) | (0 << 6)>(tot, flip);
+        const unsigned long long costU = tot[0], freed = tot[2];
+        const unsigned nU = (unsigned)tot[1], nD = (unsigned)tot[3];
         const double dU = sh_dU, dD = sh_dD;
         const bool accept = expand ? (nU > 0) : (nU > 0 && nD > 0 && dU > dD);
         if (accept) {
             for (long long i = (long long)c * LT + tid; i < a.N; i += (long long)G * LT) {
-                if (__ldcg(a.ustamp + i) == stamp) a.level[i] = (unsigned char)(__ldcg(a.level + i) + 1);
-                else if (!expand && __ldcg(a.dnstamp + i) == stamp)
-                    a.level[i] = (unsigned char)(__ldcg(a.level + i) - 1);
+                const unsigned m = __ldcg(a.mark + i);
+                if ((m >> 1) == stamp)
+                    a.level[i] = (unsigned char)((int)__ldcg(a.level + i) + ((m & 1u) ? -1 : 1));
             }
         }
         if (expand && accept) { used += (long long)costU; loss -= dU; expansions += 1; }
@@ -541,7 +569,8 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
         return sb_fail(ctx, SB_ERR_INVALID, "allocate: gamma0, gammaT must lie in (0, 1]");
     const int L = n_bits;
     const long long nsteps = (long long)N * (L - 1);
-    if (nsteps >= (1ll << 32)) return sb_fail(ctx, SB_ERR_SHAPE, "allocate: N * (n_bits - 1) must fit 32 bits");
+    if (nsteps >= (1ll << 32) || N >= (1ll << 29) - 1)
+        return sb_fail(ctx, SB_ERR_SHAPE, "allocate: N must be below 2^29 and N * (n_bits - 1) below 2^32");
     SB_CUDA(ctx, cudaSetDevice(ctx->device));
     memset(report, 0, sizeof *report);
 
@@ -554,8 +583,8 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
     void* arena;
     sb_status stt = sb_scratch(ctx, Carver::need({sizeof(AllocState), ns * 8, ns * 8, ns * 8, ns * 8,
                                                    ns * 4, ns * 4, ns * 4, ns * 4,
-                                                   (size_t)N * 4, (size_t)N * 4, (size_t)N * 8,
-                                                   (size_t)N * 4, (size_t)N * 4, nparts * 8,
+                                                   (size_t)N * 8, (size_t)N * 8, (size_t)N * 8,
+                                                   (size_t)N * 4, nparts * 8,
                                                    nparts * 8, sort_bytes, (size_t)(N + 1) * 8,
                                                    (size_t)LOOP_MAX_CTAS * 128}), &arena);
     if (stt != SB_OK) return stt;
@@ -569,11 +598,10 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
     unsigned* vB = cv.take<unsigned>(ns);
     unsigned* vC = cv.take<unsigned>(ns);
     unsigned* vD = cv.take<unsigned>(ns);
-    unsigned* uprank = cv.take<unsigned>((size_t)N);
-    unsigned* upstamp = cv.take<unsigned>((size_t)N);
+    unsigned long long* upsr = cv.take<unsigned long long>((size_t)N);
     unsigned long long* upcum = cv.take<unsigned long long>((size_t)N);
-    unsigned* dnstamp = cv.take<unsigned>((size_t)N);
-    unsigned* ustamp = cv.take<unsigned>((size_t)N);
+    double* upde = cv.take<double>((size_t)N);
+    unsigned* mark = cv.take<unsigned>((size_t)N);
     double* part = cv.take<double>(nparts);
     double* part2 = cv.take<double>(nparts);
     void* sort_scratch = cv.take<unsigned char>(sort_bytes);
@@ -603,7 +631,7 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
     a.uniform = uniform_block_elems; a.N = N; a.L = L;
     for (int l = 0; l < 8; ++l) a.bits[l] = l < L ? bits[l] : 0;
     a.level = level; a.st = dst;
-    a.uprank = uprank; a.upstamp = upstamp; a.upcum = upcum; a.dnstamp = dnstamp; a.ustamp = ustamp;
+    a.upsr = upsr; a.upcum = upcum; a.upde = upde; a.mark = mark;
     a.part = part;
 
     int l0 = 0;
@@ -641,8 +669,8 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
         report->used_bits = fin.used;
         if (fin.used > cap) return sb_fail(ctx, SB_ERR_BUDGET, "allocate: budget below the smallest candidate");
         if (nsteps > 0) {
-            int* level32 = reinterpret_cast<int*>(uprank);
-            int* steps = reinterpret_cast<int*>(upstamp);
+            int* level32 = reinterpret_cast<int*>(upsr);
+            int* steps = reinterpret_cast<int*>(mark);
             SB_CUDA(ctx, cudaMemsetAsync(level32, 0, sizeof(int) * N, ctx->stream));
             SB_CUDA(ctx, cudaMemsetAsync(steps, 0, sizeof(int), ctx->stream));
             hull_steps_kernel<<<nblkB, BT, 0, ctx->stream>>>(a, kA, vA, kC);
@@ -677,7 +705,8 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
             SB_LAUNCHED(ctx);
             stt = sb_radix_sort_u64(ctx, kA, kB, vA, vB, nsteps, sort_scratch);
             if (stt != SB_OK) return stt;
-            // down list = up list reversed run by run (vB: heads, vD: their prefix, kB: run starts)
+            // down list = up list reversed run by run (vB: heads, vD: their prefix, kB: run starts);
+            // the sorted keys in kA are dead after tie_heads_kernel and hold the down entries
             unsigned* run_start = reinterpret_cast<unsigned*>(kB);
             tie_heads_kernel<<<g, 256, 0, ctx->stream>>>(kA, nsteps, vB);
             SB_LAUNCHED(ctx);
@@ -685,7 +714,10 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
             if (stt != SB_OK) return stt;
             run_starts_kernel<<<g, 256, 0, ctx->stream>>>(vB, vD, nsteps, run_start);
             SB_LAUNCHED(ctx);
-            reverse_runs_kernel<<<g, 256, 0, ctx->stream>>>(vA, vB, vD, run_start, nsteps, vC);
+            unsigned* up_ent = vC; unsigned* dn_ent = reinterpret_cast<unsigned*>(kA);
+            double* up_de = reinterpret_cast<double*>(kC); double* dn_de = reinterpret_cast<double*>(kD);
+            entry_info_kernel<<<g, 256, 0, ctx->stream>>>(a, vA, vB, vD, run_start, nsteps, up_ent, up_de,
+                                                          dn_ent, dn_de);
             SB_LAUNCHED(ctx);
             LoopWork lw;
             lw.up_tot = loop_cc; lw.dn_tot = loop_cc + LOOP_MAX_CTAS;
@@ -693,9 +725,10 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
             lw.dD = loop_d; lw.dU = loop_d + LOOP_MAX_CTAS;
             lw.freed = loop_u64; lw.costU = loop_u64 + LOOP_MAX_CTAS;
             lw.nD = loop_u32; lw.nU = loop_u32 + LOOP_MAX_CTAS;
-            const unsigned* up_list = vA; const unsigned* dn_list = vC;
+            const unsigned* up_ent_c = up_ent; const unsigned* dn_ent_c = dn_ent;
+            const double* up_de_c = up_de; const double* dn_de_c = dn_de;
             long long ne = nsteps;
-            void* kargs[] = {&a, &up_list, &dn_list, &ne, &lw};
+            void* kargs[] = {&a, &up_ent_c, &up_de_c, &dn_ent_c, &dn_de_c, &ne, &lw};
             bool launched = false;
             // Small problems: one thread-block cluster of 16 CTAs x 512 threads; its hardware
             // barrier is several times cheaper than a grid-wide one, and a handful of list
