@@ -9,7 +9,7 @@ sb_status sb_gather_bf16(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64
 
 namespace {
 
-constexpr int PK_THREADS = 256;
+constexpr int PK_THREADS = 128;
 constexpr int PK_WARPS = PK_THREADS / 32;
 
 struct PackBits { int bits[8]; };
@@ -54,23 +54,154 @@ pack_offsets_kernel(const unsigned char* __restrict__ level, int64_t nb, int n_b
 
 constexpr double PK_MAGIC64 = 6755399441055744.0;     // 1.5 * 2^52: low word of (t + MAGIC) = rint(t)
 
-// 16 codes of B bits -> 16*B bits in w[0..3] (little-endian bit stream)
+// 16 codes of B bits -> 16*B bits in w[0..3] (little-endian bit stream).  All positions are
+// compile-time constants; the fields are disjoint, so adding is the same as or-ing.
 template <int B>
 __device__ __forceinline__ void pack16(const unsigned (&code)[16], unsigned (&w)[4]) {
-    unsigned long long acc = 0ull;
-    int have = 0, out = 0;
     w[0] = w[1] = w[2] = w[3] = 0u;
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
-        acc |= (unsigned long long)code[k] << have;
-        have += B;
-        if (have >= 32) {
-            w[out++] = (unsigned)acc;
-            acc >>= 32;
-            have -= 32;
+        const int bit = k * B, j = bit >> 5, sh = bit & 31;
+        w[j] += code[k] << sh;
+        if (sh + B > 32) w[j + 1] += code[k] >> (32 - sh);
+    }
+}
+
+// What a lane needs to know about its place in the CTA's chunk.
+struct PackLane {
+    const __nv_bfloat16* colp;   // W + first column of the lane
+    const int32_t* rp;           // row permutation applied at load time, or null
+    int64_t ldw, row0;           // leading dimension, first row of the block row
+    int br, team;                // block rows; lanes per quantisation group
+    float2* meta;                // metadata of the lane's group in row row0
+    int64_t meta_ld;             // groups per matrix row
+    unsigned* dst;               // first word of the lane in row row0 of its block
+    unsigned row_words;          // words per block row
+    bool meta_lane, odd_lane;
+};
+
+// One (row, 16 columns) per lane and step: binary64 codes of the lane's 16 weights.
+// Returns the stored scale; code[] is all zero for a constant group.
+template <typename QMAX>
+__device__ __forceinline__ float encode16(const uint32_t (&wv)[8], float lo, float hi, QMAX qmax,
+                                          unsigned (&code)[16]) {
+    const double dlo = (double)lo;
+    const double range64 = __dsub_rn((double)hi, dlo);            // exact
+    const float range = (float)range64;
+    float scale = 0.f;
+    if (range64 != 0.0) {
+        const float qmaxf = (float)qmax;
+        const double inv = __ddiv_rn((double)qmaxf, range64);
+        scale = (double)range == range64 ? __fdiv_rn(range, qmaxf)
+                                         : (float)__ddiv_rn(range64, (double)qmaxf);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const double t0 = __dmul_rn(__dsub_rn((double)bf16lo(wv[k]), dlo), inv);
+            const double t1 = __dmul_rn(__dsub_rn((double)bf16hi(wv[k]), dlo), inv);
+            // 0 <= t <= qmax, so no clamp and no mask: the low word of t + 1.5 * 2^52 is rint(t)
+            code[2 * k] = (unsigned)__double2loint(__dadd_rn(t0, PK_MAGIC64));
+            code[2 * k + 1] = (unsigned)__double2loint(__dadd_rn(t1, PK_MAGIC64));
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) code[k] = 0u;
+    }
+    return scale;
+}
+
+// The whole chunk has one bitwidth B and fits the packed buffer: no per-word checks, all bit
+// positions constant.  A lane's 16 codes are 16*B bits: whole words for even B; for odd B a
+// pair of lanes makes whole words (the even lane completes its last word with the low
+// half-word of its neighbour, the odd lane drops that half-word).
+template <int B>
+__device__ __forceinline__ void pack_rows(const PackLane& pl) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int rr = warp * 4 + (lane >> 3);
+    auto row_ptr = [&](int r_in) {
+        const int64_t r = pl.row0 + r_in;
+        return reinterpret_cast<const uint4*>(pl.colp + (pl.rp ? (int64_t)pl.rp[r] : r) * pl.ldw);
+    };
+    uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0;
+    if (rr < pl.br) { const uint4* p = row_ptr(rr); n0 = __ldg(p); n1 = __ldg(p + 1); }
+    unsigned* dst = pl.dst + (size_t)rr * pl.row_words;
+    float2* mp = pl.meta + (int64_t)rr * pl.meta_ld;
+    const unsigned dst_step = PK_WARPS * 4 * pl.row_words;
+    const int64_t meta_step = (int64_t)PK_WARPS * 4 * pl.meta_ld;
+    for (; rr < pl.br; rr += PK_WARPS * 4, dst += dst_step, mp += meta_step) {   // br % 4 == 0
+        const uint32_t wv[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
+        if (rr + PK_WARPS * 4 < pl.br) { const uint4* p = row_ptr(rr + PK_WARPS * 4); n0 = __ldg(p); n1 = __ldg(p + 1); }
+        float lo, hi;
+        group_minmax<8>(wv, pl.team, lo, hi);
+        unsigned code[16], w[4];
+        const float scale = encode16(wv, lo, hi, (1 << B) - 1, code);
+        if (pl.meta_lane) *mp = make_float2(scale, lo);
+        pack16<B>(code, w);
+        if constexpr (B & 1) {
+            const unsigned nb_low = __shfl_down_sync(0xffffffffu, w[0], 1);
+            if (!pl.odd_lane) {
+                w[B >> 1] |= nb_low << 16;
+#pragma unroll
+                for (int i = 0; i <= (B >> 1); ++i) dst[i] = w[i];
+            } else {
+#pragma unroll
+                for (int i = 0; i < (B >> 1); ++i) dst[i] = (w[i] >> 16) | (w[i + 1] << 16);
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < (B >> 1); ++i) dst[i] = w[i];
         }
     }
-    if (have > 0) w[out] = (unsigned)acc;
+}
+
+// Chunks that hold blocks of different bitwidths (blocks narrower than 128 columns) or that
+// reach past the packed buffer: bitwidth per lane at run time, every word checked.
+__device__ __noinline__ void pack_rows_generic(PackLane pl, int b, long long lane_word,
+                                               long long capacity, unsigned* packed, SbDeviceState* ds) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool odd_b = b & 1;
+    for (int rr = warp * 4 + (lane >> 3); rr < pl.br; rr += PK_WARPS * 4) {
+        const int64_t r = pl.row0 + rr;
+        const uint4* p = reinterpret_cast<const uint4*>(pl.colp + (pl.rp ? (int64_t)pl.rp[r] : r) * pl.ldw);
+        const uint4 n0 = __ldg(p), n1 = __ldg(p + 1);
+        const uint32_t wv[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
+        float lo, hi;
+        group_minmax<8>(wv, pl.team, lo, hi);
+        unsigned code[16], w[4];
+        const float scale = encode16(wv, lo, hi, (1 << b) - 1, code);
+        if (pl.meta_lane) pl.meta[(int64_t)rr * pl.meta_ld] = make_float2(scale, lo);
+        switch (b) {
+            case 1: pack16<1>(code, w); break;
+            case 2: pack16<2>(code, w); break;
+            case 3: pack16<3>(code, w); break;
+            case 4: pack16<4>(code, w); break;
+            case 5: pack16<5>(code, w); break;
+            case 6: pack16<6>(code, w); break;
+            case 7: pack16<7>(code, w); break;
+            default: pack16<8>(code, w); break;
+        }
+        const unsigned nb_low = __shfl_down_sync(0xffffffffu, w[0], 1);
+        int nwords = b >> 1;                                  // even b: b/2 whole words
+        if (odd_b) {
+            if (!pl.odd_lane) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (i == (b >> 1)) w[i] |= nb_low << 16;
+                nwords = (b >> 1) + 1;
+            } else {
+#pragma unroll
+                for (int i = 0; i < 3; ++i) w[i] = (w[i] >> 16) | (w[i + 1] << 16);
+                w[3] >>= 16;
+            }
+        }
+        const long long dst = lane_word + (long long)rr * pl.row_words;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (i < nwords) {
+                if (dst + i < capacity) packed[dst + i] = w[i];
+                else sb_latch(ds, SB_ERR_SCRATCH, SBK_PACK);
+            }
+        }
+    }
 }
 
 // CTA = one block row x one 128-column chunk.  A lane owns 16 consecutive columns (two
@@ -85,9 +216,6 @@ __device__ __forceinline__ void pack16(const unsigned (&code)[16], unsigned (&w)
 // The stored scale is fl32(range / qmax): with range exact in fp32 (checked) one correctly
 // rounded fp32 division equals the rounded fp64 quotient (a 24-bit integer over 2^b - 1 has a
 // binary expansion of period <= 8, never within 2^-53 of an fp32 rounding boundary).
-//
-// A lane's 16 codes are 16*b bits: whole words for even b, and for odd b a pair of lanes
-// makes whole words (the even lane also takes the low half-word of its neighbour).
 __global__ void __launch_bounds__(PK_THREADS)
 pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const int32_t* __restrict__ rp,
             int br, int bc, int group, PackBits pb, int n_bits,
@@ -96,12 +224,13 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const int32_t* __r
             int64_t n_block_cols, int64_t groups_per_row, SbDeviceState* ds) {
     __shared__ int s_bits[4];
     __shared__ long long s_base[4];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int cl = lane & 7, slot = lane >> 3;
+    const int lane = threadIdx.x & 31;
+    const int cl = lane & 7;
     const int piece = bc < 128 ? bc : 128;               // columns of one block inside the chunk
     const int lpp = piece >> 4;                           // lanes per piece
     const int64_t bi = blockIdx.y;
     const int64_t col0 = (int64_t)blockIdx.x * 128;
+    bool fits = true;
     if (threadIdx.x < 128 / piece) {
         const int64_t c0 = col0 + (int64_t)threadIdx.x * piece;
         const int64_t bj = c0 / bc;
@@ -109,99 +238,47 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const int32_t* __r
         int lv = level[blk];
         if (lv >= n_bits) { sb_latch(ds, SB_ERR_INVALID, SBK_PACK); lv = n_bits - 1; }
         const int b = pb.bits[lv];
+        const long long base = (long long)off[blk] + ((c0 - bj * bc) * b) / 32;
         s_bits[threadIdx.x] = b;
-        s_base[threadIdx.x] = (long long)off[blk] + ((c0 - bj * bc) * b) / 32;
+        s_base[threadIdx.x] = base;
+        // last word this piece writes
+        fits = base + (long long)(br - 1) * ((long long)bc * b / 32) + (long long)piece * b / 32 <= capacity;
     }
-    __syncthreads();
+    const bool all_fit = __syncthreads_and(fits);
     const int pc = cl / lpp, lp = cl - pc * lpp;
     const int b = s_bits[pc];
-    const long long row_words = (long long)bc * b / 32;
-    // word offset of this lane's bits inside its row piece; odd b: the odd lane starts 16 bits in
-    const long long lane_base = s_base[pc] + (lp * 16 * b) / 32;
-    const bool odd_b = b & 1, odd_lane = lp & 1;
-    const float qmaxf = (float)((1 << b) - 1);
-    const int team = group >> 4;                          // lanes per quantisation group (16 columns each)
-    const int64_t gcol = (col0 + cl * 16) / group;
-    const bool meta_lane = (cl % team) == 0;
-    const __nv_bfloat16* colp = W + col0 + cl * 16;
+    bool uniform = true;
+    for (int q = 1; q < 128 / piece; ++q) uniform = uniform && s_bits[q] == s_bits[0];
 
-    auto row_ptr = [&](int rr) {
-        const int64_t r = bi * br + rr;
-        return colp + (rp ? (int64_t)rp[r] : r) * ldw;
-    };
-    int rr = warp * 4 + slot;
-    uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0;
-    if (rr < br) {
-        const uint4* p = reinterpret_cast<const uint4*>(row_ptr(rr));
-        n0 = __ldg(p); n1 = __ldg(p + 1);
-    }
-    for (; rr < br; rr += PK_WARPS * 4) {          // br % 4 == 0: a warp step is all or nothing
-        const int64_t r = bi * br + rr;
-        const uint32_t wv[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
-        if (rr + PK_WARPS * 4 < br) {
-            const uint4* p = reinterpret_cast<const uint4*>(row_ptr(rr + PK_WARPS * 4));
-            n0 = __ldg(p); n1 = __ldg(p + 1);
-        }
-        float lo, hi;
-        group_minmax<8>(wv, team, lo, hi);
-        const double dlo = (double)lo;
-        const double range64 = __dsub_rn((double)hi, dlo);            // exact
-        const float range = (float)range64;
-        unsigned code[16];
-        float scale = 0.f;
-        if (range64 != 0.0) {
-            const double inv = __ddiv_rn((double)qmaxf, range64);
-            scale = (double)range == range64 ? __fdiv_rn(range, qmaxf)
-                                             : (float)__ddiv_rn(range64, (double)qmaxf);
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const double t0 = __dmul_rn(__dsub_rn((double)bf16lo(wv[k]), dlo), inv);
-                const double t1 = __dmul_rn(__dsub_rn((double)bf16hi(wv[k]), dlo), inv);
-                // 0 <= t <= qmax, so no clamp: the low word of t + 1.5 * 2^52 is rint(t)
-                code[2 * k] = (unsigned)__double2loint(__dadd_rn(t0, PK_MAGIC64)) & 0xffu;
-                code[2 * k + 1] = (unsigned)__double2loint(__dadd_rn(t1, PK_MAGIC64)) & 0xffu;
-            }
-        } else {
-#pragma unroll
-            for (int k = 0; k < 16; ++k) code[k] = 0u;
-        }
-        if (meta_lane) meta[r * groups_per_row + gcol] = make_float2(scale, lo);
-        unsigned w[4];
+    PackLane pl;
+    pl.colp = W + col0 + cl * 16;
+    pl.rp = rp;
+    pl.ldw = ldw;
+    pl.row0 = bi * br;
+    pl.br = br;
+    pl.team = group >> 4;                                 // lanes per quantisation group (16 columns each)
+    pl.meta_ld = groups_per_row;
+    pl.meta = meta + pl.row0 * groups_per_row + (col0 + cl * 16) / group;
+    pl.meta_lane = (cl % pl.team) == 0;
+    pl.odd_lane = lp & 1;
+    pl.row_words = (unsigned)((long long)bc * b / 32);
+    // word offset of this lane's bits inside its row piece; odd b: the odd lane starts 16 bits in
+    const long long lane_word = s_base[pc] + (lp * 16 * b) / 32 + (((b & 1) && pl.odd_lane) ? 1 : 0);
+    pl.dst = packed + lane_word;
+
+    if (uniform && all_fit) {
         switch (b) {
-            case 1: pack16<1>(code, w); break;
-            case 2: pack16<2>(code, w); break;
-            case 3: pack16<3>(code, w); break;
-            case 4: pack16<4>(code, w); break;
-            case 5: pack16<5>(code, w); break;
-            case 6: pack16<6>(code, w); break;
-            case 7: pack16<7>(code, w); break;
-            default: pack16<8>(code, w); break;
+            case 1: pack_rows<1>(pl); break;
+            case 2: pack_rows<2>(pl); break;
+            case 3: pack_rows<3>(pl); break;
+            case 4: pack_rows<4>(pl); break;
+            case 5: pack_rows<5>(pl); break;
+            case 6: pack_rows<6>(pl); break;
+            case 7: pack_rows<7>(pl); break;
+            default: pack_rows<8>(pl); break;
         }
-        // odd b: the pair (even lane, odd lane) holds 32*b bits; the even lane completes its last
-        // word with the neighbour's low half-word, the odd lane drops that half-word
-        const unsigned nb_low = __shfl_down_sync(0xffffffffu, w[0], 1);
-        int nwords = b >> 1;                                  // even b: b/2 whole words
-        if (odd_b) {
-            if (!odd_lane) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    if (i == (b >> 1)) w[i] |= nb_low << 16;
-                nwords = (b >> 1) + 1;
-            } else {
-#pragma unroll
-                for (int i = 0; i < 3; ++i) w[i] = (w[i] >> 16) | (w[i + 1] << 16);
-                w[3] >>= 16;
-                nwords = b >> 1;
-            }
-        }
-        const long long dst = lane_base + (odd_b && odd_lane ? 1 : 0) + (long long)rr * row_words;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            if (i < nwords) {
-                if (dst + i < capacity) packed[dst + i] = w[i];
-                else sb_latch(ds, SB_ERR_SCRATCH, SBK_PACK);
-            }
-        }
+    } else {
+        pack_rows_generic(pl, b, lane_word, capacity, packed, ds);
     }
 }
 

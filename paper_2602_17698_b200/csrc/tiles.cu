@@ -41,51 +41,118 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // ---- permuted gather: out[r][j] = W[rp[r]][cp[j]] ---------------------------------------
-// A source row is staged in shared memory with coalesced asynchronous 16-byte copies (the next
-// row is in flight while the current one is written out), then read in permuted order: 2-byte
-// scattered reads never reach HBM.
+// A source row is staged in shared memory with coalesced asynchronous 16-byte copies (a ring of
+// three rows: two are in flight while one is written out, one barrier per row), then read in
+// permuted order: 2-byte scattered reads never reach HBM.
+constexpr int GA_STAGES = 3;
 __global__ void __launch_bounds__(CTA_THREADS)
-gather_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, int64_t ldw,
+gather_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int C, int64_t ldw,
               const int32_t* __restrict__ rp, const int32_t* __restrict__ cp,
               __nv_bfloat16* __restrict__ out, int rows_per_cta) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    unsigned short* buf[2] = {reinterpret_cast<unsigned short*>(smem_raw),
-                              reinterpret_cast<unsigned short*>(smem_raw) + C};
+    const unsigned row_bytes = (unsigned)C * 2u;
     const int64_t r0 = (int64_t)blockIdx.x * rows_per_cta;
     const int nrows = (int)min((int64_t)rows_per_cta, R - r0);
-    auto stage = [&](int rr) {
-        const int64_t r = r0 + rr;
-        const __nv_bfloat16* src = W + (rp ? (int64_t)rp[r] : r) * ldw;
-        unsigned short* dst = buf[rr & 1];
-        for (int64_t j = (int64_t)threadIdx.x * 8; j < C; j += CTA_THREADS * 8) cp_async16(dst + j, src + j);
-        cp_async_commit();
+    const int j0 = (int)threadIdx.x * 8;
+    auto stage = [&](int rr, int st) {
+        if (rr < nrows) {
+            const int64_t r = r0 + rr;
+            const __nv_bfloat16* src = W + (rp ? (int64_t)rp[r] : r) * ldw;
+            unsigned char* dst = smem_raw + (unsigned)st * row_bytes;
+            for (int j = j0; j < C; j += CTA_THREADS * 8) cp_async16(dst + 2 * j, src + j);
+        }
+        cp_async_commit();                      // one group per row, empty past the end
     };
-    if (nrows > 0) stage(0);
-    for (int rr = 0; rr < nrows; ++rr) {
-        if (rr + 1 < nrows) stage(rr + 1); else cp_async_commit();
-        cp_async_wait<1>();
-        __syncthreads();
-        const unsigned short* row = buf[rr & 1];
-        unsigned short* dst = reinterpret_cast<unsigned short*>(out + (r0 + rr) * C);
-        for (int64_t j = (int64_t)threadIdx.x * 8; j < C; j += CTA_THREADS * 8) {
-            uint32_t o[4];
+    stage(0, 0);
+    stage(1, 1);
+    int st = 0;
+    for (int rr = 0; rr < nrows; ++rr, st = st + 1 == GA_STAGES ? 0 : st + 1) {
+        cp_async_wait<1>();                     // row rr has landed (row rr + 1 may be in flight)
+        __syncthreads();                        // ... for every thread; row rr - 1 is consumed
+        stage(rr + 2, st >= 1 ? st - 1 : GA_STAGES - 1);
+        const unsigned short* row = reinterpret_cast<const unsigned short*>(smem_raw + (unsigned)st * row_bytes);
+        unsigned short* dst = reinterpret_cast<unsigned short*>(out + (r0 + rr) * (int64_t)C);
+        for (int j = j0; j < C; j += CTA_THREADS * 8) {
+            uint4 o;
             if (cp) {
                 const int4 p0 = __ldg(reinterpret_cast<const int4*>(cp + j));
                 const int4 p1 = __ldg(reinterpret_cast<const int4*>(cp + j + 4));
-                o[0] = row[p0.x] | ((uint32_t)row[p0.y] << 16);
-                o[1] = row[p0.z] | ((uint32_t)row[p0.w] << 16);
-                o[2] = row[p1.x] | ((uint32_t)row[p1.y] << 16);
-                o[3] = row[p1.z] | ((uint32_t)row[p1.w] << 16);
+                o.x = row[p0.x] | ((uint32_t)row[p0.y] << 16);
+                o.y = row[p0.z] | ((uint32_t)row[p0.w] << 16);
+                o.z = row[p1.x] | ((uint32_t)row[p1.y] << 16);
+                o.w = row[p1.z] | ((uint32_t)row[p1.w] << 16);
             } else {
-                const uint4 v = *reinterpret_cast<const uint4*>(row + j);
-                o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+                o = *reinterpret_cast<const uint4*>(row + j);
             }
-            *reinterpret_cast<uint4*>(dst + j) = make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4*>(dst + j) = o;
         }
-        __syncthreads();          // the buffer is free for the row after next
     }
+    cp_async_wait<0>();
 }
 
+// The same with the column permutation held in registers: a thread writes the same output
+// columns in every row, so it reads its source columns once (as byte offsets, two per
+// register) instead of once per row.  NIT * 2048 >= C, C < 32768.
+template <int NIT>
+__global__ void __launch_bounds__(CTA_THREADS)
+gather_cols_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int C, int64_t ldw,
+                   const int32_t* __restrict__ rp, const int32_t* __restrict__ cp,
+                   __nv_bfloat16* __restrict__ out, int rows_per_cta) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const unsigned row_bytes = (unsigned)C * 2u;
+    const int64_t r0 = (int64_t)blockIdx.x * rows_per_cta;
+    const int nrows = (int)min((int64_t)rows_per_cta, R - r0);
+    const int j0 = (int)threadIdx.x * 8;
+    uint32_t off2[NIT][4];
+#pragma unroll
+    for (int it = 0; it < NIT; ++it) {
+        const int j = j0 + it * (CTA_THREADS * 8);
+        int4 p0 = make_int4(0, 0, 0, 0), p1 = p0;
+        if (j < C) {
+            p0 = __ldg(reinterpret_cast<const int4*>(cp + j));
+            p1 = __ldg(reinterpret_cast<const int4*>(cp + j + 4));
+        }
+        off2[it][0] = (uint32_t)(2 * p0.x) | ((uint32_t)(2 * p0.y) << 16);
+        off2[it][1] = (uint32_t)(2 * p0.z) | ((uint32_t)(2 * p0.w) << 16);
+        off2[it][2] = (uint32_t)(2 * p1.x) | ((uint32_t)(2 * p1.y) << 16);
+        off2[it][3] = (uint32_t)(2 * p1.z) | ((uint32_t)(2 * p1.w) << 16);
+    }
+    auto stage = [&](int rr, int st) {
+        if (rr < nrows) {
+            const int64_t r = r0 + rr;
+            const __nv_bfloat16* src = W + (rp ? (int64_t)rp[r] : r) * ldw;
+            unsigned char* dst = smem_raw + (unsigned)st * row_bytes;
+            for (int j = j0; j < C; j += CTA_THREADS * 8) cp_async16(dst + 2 * j, src + j);
+        }
+        cp_async_commit();
+    };
+    stage(0, 0);
+    stage(1, 1);
+    int st = 0;
+    for (int rr = 0; rr < nrows; ++rr, st = st + 1 == GA_STAGES ? 0 : st + 1) {
+        cp_async_wait<1>();
+        __syncthreads();
+        stage(rr + 2, st >= 1 ? st - 1 : GA_STAGES - 1);
+        const unsigned char* row = smem_raw + (unsigned)st * row_bytes;
+        unsigned short* dst = reinterpret_cast<unsigned short*>(out + (r0 + rr) * (int64_t)C);
+        auto pair = [&](uint32_t o2) -> uint32_t {
+            const uint32_t a = *reinterpret_cast<const unsigned short*>(row + (o2 & 0xffffu));
+            const uint32_t b = *reinterpret_cast<const unsigned short*>(row + (o2 >> 16));
+            return a | (b << 16);
+        };
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int j = j0 + it * (CTA_THREADS * 8);
+            if (j < C) {
+                uint4 o;
+                o.x = pair(off2[it][0]); o.y = pair(off2[it][1]);
+                o.z = pair(off2[it][2]); o.w = pair(off2[it][3]);
+                *reinterpret_cast<uint4*>(dst + j) = o;
+            }
+        }
+    }
+    cp_async_wait<0>();
+}
 // ---- shared inner step: one lane, CPL consecutive columns of one row ----------------------
 template <int CPL>
 __device__ __forceinline__ void load_cols(const __nv_bfloat16* p, bool ok, uint32_t (&w)[CPL / 2]) {
@@ -670,8 +737,8 @@ sb_status launch_scores(int nfine, A... args) {
 // used by pack.cu as well
 sb_status sb_gather_bf16(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw,
                          const int32_t* rp, const int32_t* cp, void* out) {
-    const size_t smem = (size_t)C * 2 * 2;          // two row buffers
-    if (smem > 200 * 1024) return sb_fail(ctx, SB_ERR_SHAPE, "gather: rows longer than 51200 columns");
+    const size_t smem = (size_t)C * 2 * GA_STAGES;  // a ring of row buffers
+    if (smem > 200 * 1024) return sb_fail(ctx, SB_ERR_SHAPE, "gather: rows longer than 34133 columns");
     static bool attr_set = false;
     if (!attr_set) {
         SB_CUDA(ctx, cudaFuncSetAttribute(gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -680,9 +747,24 @@ sb_status sb_gather_bf16(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64
     }
     int rows_per_cta = 8;
     const unsigned grid = (unsigned)((R + rows_per_cta - 1) / rows_per_cta);
-    gather_kernel<<<grid, CTA_THREADS, smem, ctx->stream>>>(
-        static_cast<const __nv_bfloat16*>(W), R, C, ldw, rp, cp, static_cast<__nv_bfloat16*>(out),
-        rows_per_cta);
+    auto* Wb = static_cast<const __nv_bfloat16*>(W);
+    auto* ob = static_cast<__nv_bfloat16*>(out);
+#define SB_GATHER_COLS(NIT)                                                                          \
+    do {                                                                                             \
+        static bool attr_cols = false;                                                               \
+        if (!attr_cols) {                                                                            \
+            SB_CUDA(ctx, cudaFuncSetAttribute(gather_cols_kernel<NIT>,                               \
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)); \
+            attr_cols = true;                                                                        \
+        }                                                                                            \
+        gather_cols_kernel<NIT><<<grid, CTA_THREADS, smem, ctx->stream>>>(Wb, R, (int)C, ldw, rp, cp, ob, \
+                                                                          rows_per_cta);            \
+    } while (0)
+    if (cp && C <= 4096) SB_GATHER_COLS(2);
+    else if (cp && C <= 8192) SB_GATHER_COLS(4);
+    else if (cp && C <= 16384) SB_GATHER_COLS(8);
+    else gather_kernel<<<grid, CTA_THREADS, smem, ctx->stream>>>(Wb, R, (int)C, ldw, rp, cp, ob, rows_per_cta);
+#undef SB_GATHER_COLS
     SB_LAUNCHED(ctx);
     return SB_OK;
 }
