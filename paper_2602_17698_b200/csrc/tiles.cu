@@ -195,17 +195,23 @@ __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
 }
 
 // ---- block scores ------------------------------------------------------------------------
-// Every WARP is autonomous: it walks its own units (a block, or a 32-row part of one), stages
-// its own 16-row slabs of the 128-column chunk in its own shared-memory ring with asynchronous
-// 16-byte copies (three slabs per warp, two of them in flight: 128 KB per SM), and synchronises with nobody
-// but itself.  Without CTA barriers the warps of an SM drift apart, so the integer/shuffle
-// phase of one warp (group min/max, unpacking) overlaps the FP32 phase of another.  A lane
-// owns CPL consecutive columns of the chunk; 128/CPL lanes cover a row, a warp covers
-// 32*CPL/128 rows per step.  The 16-byte pieces of a row are laid out in shared memory so
-// that a quarter-warp reads 128 contiguous bytes (no bank conflicts).  Everything inside the
-// candidate loop is packed fp32 pairs (fma/add/mul.f32x2), including the per-group constants,
-// which come from packed pairs in the kernel parameters.  Each unit writes its partial block
-// errors; a second tiny kernel adds the parts of a block in a fixed order.
+// Every WARP is autonomous.  The matrix is cut into slabs of 16 rows x 128 columns (4 KB),
+// numbered tile by tile, chunk column by chunk column, top to bottom; the slabs are dealt to
+// the warps of the grid in contiguous, equally long ranges, so a warp streams down the chunk
+// columns of consecutive blocks.  It stages its slabs in its own shared-memory ring with
+// asynchronous 16-byte copies (three slabs per warp, two of them in flight) and synchronises
+// with nobody but itself, so the warps of an SM drift apart and the integer/shuffle phase of
+// one warp overlaps the FP32 phase of another.  Inside a warp the two phases of consecutive
+// steps overlap as well: the loop body first reads the NEXT step's rows from shared memory and
+// reduces their group min/max (shuffles, reciprocal), then evaluates all candidates on the
+// CURRENT step's registers, and the compiler interleaves the two instruction streams.
+//
+// A lane owns 8 consecutive columns of the chunk (16 lanes cover a row) and RPL rows per step,
+// so c_j multiplies the per-column accumulators once per chunk instead of once per element.
+// Everything inside the candidate loop is packed fp32 pairs (fma/add/mul.f32x2).  When the
+// warp leaves a chunk column (or its range ends) it writes the partial block errors of that
+// stretch as record (chunk number + warp number) -- unique, because either number only grows
+// along the slab sequence -- and a second tiny kernel adds the records of a block in order.
 //
 // NFINE = how many of the L candidates (the last ones: bits ascend) keep the grid step as a
 // two-float sum: with many levels q * scale carries the fp32 rounding of the step times q, a
@@ -217,205 +223,275 @@ constexpr int SLAB_BYTES = SLAB_ROWS * 256;
 constexpr int SC_THREADS = 512;                 // one CTA of 16 warps per SM
 constexpr int SC_WARPS = SC_THREADS / 32;
 constexpr int RING = 3;                         // slabs per warp: one being read, two in flight
+constexpr int SC_CPL = 8;                       // columns per lane
+constexpr int SC_NW = SC_CPL / 2;               // packed pairs per lane and row
 
-template <int L, int CPL, int NFINE, bool FULLG, bool ROWW>
+struct ScoreGeom {
+    int br, bc, group;
+    int chunks, tile_w, spb;       // 128-column chunks per tile; tile width; slabs per chunk column
+    int nsub, lanes_per_sub;       // blocks side by side in a chunk (bc < 128); lanes across one block
+    unsigned n_tile_cols, n_slabs, n_warps;
+};
+
+// owner of slab s when warp w takes slabs [n_slabs * w / n_warps, n_slabs * (w + 1) / n_warps)
+__device__ __forceinline__ unsigned slab_owner(unsigned s, unsigned n_slabs, unsigned n_warps) {
+    return (unsigned)((((unsigned long long)s + 1ull) * n_warps - 1ull) / n_slabs);
+}
+
+struct SlabCursor { int sl, ch; unsigned bx, by; };
+
+template <int RPL>
+struct StepRegs {
+    uint32_t w[RPL][SC_NW];
+    float lo[RPL], rinv[RPL], range[RPL], sa[RPL];
+    unsigned q;          // chunk column (in slab-sequence order) the step belongs to
+    int col;             // first column of that chunk
+    bool flush;          // last step of the warp's stretch of this chunk column
+};
+
+template <int L, int RPL, int NFINE, bool FULLG, bool ROWW>
 __global__ void __launch_bounds__(SC_THREADS, 1)
 block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
                     const int32_t* __restrict__ load_row_perm,   // rows gathered at load time
                     const int32_t* __restrict__ c_perm,          // original column of permuted j
                     const int32_t* __restrict__ a_perm,          // original row of permuted r
                     const float* __restrict__ col_moment, const float* __restrict__ row_weight,
-                    int br, int bc, int group, BitsArg ba, int64_t n_block_cols,
-                    int64_t n_tile_cols, int parts, int part_rows, int64_t n_units, int64_t n_blocks,
-                    float* __restrict__ part_out) {
-    constexpr int LANE_COLS = TILE_COLS / CPL;      // lanes across a chunk row
-    constexpr int ROW_SLOTS = 32 / LANE_COLS;       // rows per warp step
-    constexpr int NW = CPL / 2;
-    constexpr int PIECES = CPL / 8;                 // 16-byte pieces per lane and row
+                    ScoreGeom g, BitsArg ba, float* __restrict__ rec) {
+    constexpr int STEP_ROWS = 2 * RPL;              // rows per warp step
     extern __shared__ __align__(16) unsigned char tile_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int cl = lane % LANE_COLS, slot = lane / LANE_COLS;
-    const int team = group / CPL > 0 ? group / CPL : 1;
-    const int chunks = bc >= TILE_COLS ? bc / TILE_COLS : 1;
-    const int tile_w = bc >= TILE_COLS ? bc : TILE_COLS;
-    const f32x2 magic2 = pk2(RNE_MAGIC, RNE_MAGIC), nmagic2 = pk2(-RNE_MAGIC, -RNE_MAGIC);
-    const int lanes_per_sub = bc >= TILE_COLS ? LANE_COLS : bc / CPL;    // lanes across one block
-    const int nsub = bc >= TILE_COLS ? 1 : TILE_COLS / bc;
-    const int slabs = (part_rows + SLAB_ROWS - 1) / SLAB_ROWS;           // per chunk of a unit
+    const int cl = lane & 15, slot = lane >> 4;
+    const int team = g.group / SC_CPL;
+    const unsigned gw = blockIdx.x * SC_WARPS + warp;
+    const unsigned s_lo = (unsigned)((unsigned long long)g.n_slabs * gw / g.n_warps);
+    const unsigned s_hi = (unsigned)((unsigned long long)g.n_slabs * (gw + 1) / g.n_warps);
+    if (s_lo >= s_hi) return;                       // no barriers in this kernel
     unsigned char* ring = tile_smem + (size_t)warp * (RING * SLAB_BYTES);
-    // this lane's share of a slab: 16-byte piece g of rows g_row, g_row + 2, ...
-    const int g = lane & 15, g_row = lane >> 4;
-    const int g_dst = g_row * 256 + (g % PIECES) * (LANE_COLS * 16) + (g / PIECES) * 16;
-    const int my_off = slot * 256 + cl * 16;
-    const int64_t warp_id = (int64_t)blockIdx.x * SC_WARPS + warp;
-    const int64_t warp_stride = (int64_t)gridDim.x * SC_WARPS;
+    const f32x2 magic2 = pk2(RNE_MAGIC, RNE_MAGIC), nmagic2 = pk2(-RNE_MAGIC, -RNE_MAGIC);
 
-    // stage slab `sl` of chunk `ch` of unit `u` (rows beyond the part are skipped)
-    // (all index arithmetic is 32-bit: units, tiles and rows are far below 2^31)
-    const unsigned u_parts = (unsigned)parts, u_tcols = (unsigned)n_tile_cols;
-    auto issue = [&](unsigned u, int ch, int sl, int stage) {
-        const unsigned t = u / u_parts, by = t / u_tcols;
-        const int64_t row0 = (int64_t)(by * (unsigned)br + (u - t * u_parts) * (unsigned)part_rows + sl * SLAB_ROWS);
-        const int rows_here = min(SLAB_ROWS, part_rows - sl * SLAB_ROWS);
-        const __nv_bfloat16* src = W + (int64_t)((t - by * u_tcols) * (unsigned)tile_w + ch * TILE_COLS + g * 8);
-        unsigned char* dst = ring + stage * SLAB_BYTES + g_dst;
-        if (load_row_perm) {
-            const int32_t* rp = load_row_perm + row0;
-            for (int row = g_row; row < rows_here; row += 2, dst += 2 * 256)
-                cp_async16(dst, src + (int64_t)rp[row] * ldw);
-        } else {
-            src += (row0 + g_row) * ldw;
-            for (int row = g_row; row < rows_here; row += 2, dst += 2 * 256, src += 2 * ldw)
-                cp_async16(dst, src);
+    auto advance = [&](SlabCursor& c) {
+        if (++c.sl == g.spb) {
+            c.sl = 0;
+            if (++c.ch == g.chunks) {
+                c.ch = 0;
+                if (++c.bx == g.n_tile_cols) { c.bx = 0; ++c.by; }
+            }
+        }
+    };
+    SlabCursor rc;                                   // read cursor
+    unsigned r_q = s_lo / (unsigned)g.spb;           // chunk column of the read cursor
+    {
+        rc.sl = (int)(s_lo - r_q * (unsigned)g.spb);
+        const unsigned t = r_q / (unsigned)g.chunks;
+        rc.ch = (int)(r_q - t * (unsigned)g.chunks);
+        rc.by = t / g.n_tile_cols;
+        rc.bx = t - rc.by * g.n_tile_cols;
+    }
+    SlabCursor ic = rc;                              // issue cursor, RING - 1 slabs ahead
+    unsigned i_s = s_lo;
+    int i_stage = 0;
+    // stage the next slab of the range (an empty group past its end keeps the wait count fixed)
+    auto issue_next = [&]() {
+        if (i_s < s_hi) {
+            const int rows_here = min(SLAB_ROWS, g.br - ic.sl * SLAB_ROWS);
+            const int64_t row0 = (int64_t)ic.by * g.br + ic.sl * SLAB_ROWS;
+            const __nv_bfloat16* src = W + ((int64_t)ic.bx * g.tile_w + ic.ch * TILE_COLS + cl * SC_CPL);
+            unsigned char* dst = ring + i_stage * SLAB_BYTES + slot * 256 + cl * 16;
+            if (load_row_perm) {
+                const int32_t* rp = load_row_perm + row0;
+                for (int row = slot; row < rows_here; row += 2, dst += 512)
+                    cp_async16(dst, src + (int64_t)rp[row] * ldw);
+            } else {
+                src += (row0 + slot) * ldw;
+                if (rows_here == SLAB_ROWS) {
+#pragma unroll
+                    for (int i = 0; i < SLAB_ROWS / 2; ++i) cp_async16(dst + i * 512, src + (int64_t)(2 * i) * ldw);
+                } else {
+                    for (int row = slot; row < rows_here; row += 2, dst += 512, src += 2 * ldw)
+                        cp_async16(dst, src);
+                }
+            }
+            advance(ic);
+            ++i_s;
         }
         cp_async_commit();
-    };
-
-    // issue cursor: RING - 1 slabs ahead of the slab being evaluated
-    int64_t i_unit = warp_id;
-    int i_ch = 0, i_sl = 0, i_stage = 0;
-    auto issue_next = [&]() {
-        if (i_unit < n_units) {
-            issue((unsigned)i_unit, i_ch, i_sl, i_stage);
-            if (++i_sl == slabs) { i_sl = 0; if (++i_ch == chunks) { i_ch = 0; i_unit += warp_stride; } }
-        } else {
-            cp_async_commit();            // keep one group per step so the wait count stays fixed
-        }
         i_stage = i_stage + 1 == RING ? 0 : i_stage + 1;
     };
-#pragma unroll
-    for (int i = 0; i < RING - 1; ++i) issue_next();
 
-    int stage = 0;
-    for (int64_t unit = warp_id; unit < n_units; unit += warp_stride) {
-        const unsigned t = (unsigned)unit / u_parts, by = t / u_tcols, bx = t - by * u_tcols;
-        const int p = (int)((unsigned)unit - t * u_parts);
-        const int64_t row_base = (int64_t)(by * (unsigned)br + (unsigned)p * (unsigned)part_rows);
-        const int64_t colT = (int64_t)(bx * (unsigned)tile_w);
-        f32x2 tot2[L];
+    unsigned r_s = s_lo;
+    int r_stage = 0, r_step = 0, r_steps = 0;
+    bool more = true;                                // a step remains to be loaded
+    // the slab at the read cursor becomes readable; the stage left behind is refilled
+    auto enter_slab = [&]() {
+        __syncwarp();
+        issue_next();
+        cp_async_wait<RING - 1>();
+        __syncwarp();
+        r_steps = min(SLAB_ROWS, g.br - rc.sl * SLAB_ROWS) / STEP_ROWS;
+        r_step = 0;
+    };
+    // rows of the step at the read cursor -> registers, group min/max and reciprocal; advance
+    auto load_step = [&](StepRegs<RPL>& n) {
+        const unsigned char* src = ring + r_stage * SLAB_BYTES + (r_step * STEP_ROWS + slot) * 256 + cl * 16;
 #pragma unroll
-        for (int l = 0; l < L; ++l) tot2[l] = 0ull;
+        for (int i = 0; i < RPL; ++i) {
+            const uint4 x = *reinterpret_cast<const uint4*>(src + i * 512);
+            n.w[i][0] = x.x; n.w[i][1] = x.y; n.w[i][2] = x.z; n.w[i][3] = x.w;
+        }
+#pragma unroll
+        for (int i = 0; i < RPL; ++i) {
+            float lo, hi;
+            group_minmax<SC_NW, FULLG ? 16 : 0>(n.w[i], team, lo, hi);
+            float range = hi - lo;
+            const bool live = range >= MIN_RANGE;
+            float rinv = rcp_approx(range);
+            float sa = 1.f;
+            if (ROWW) {
+                const int64_t r = (int64_t)rc.by * g.br + rc.sl * SLAB_ROWS + r_step * STEP_ROWS + 2 * i + slot;
+                const float a = row_weight[a_perm ? a_perm[r] : r];
+                sa = sqrtf(a);
+                rinv = a > 0.f ? rinv * rcp_approx(sa) : 0.f;
+                range *= sa;
+            }
+            n.lo[i] = lo;
+            n.rinv[i] = live ? rinv : 0.f;
+            n.range[i] = live ? range : 0.f;
+            n.sa[i] = sa;
+        }
+        n.q = r_q;
+        n.col = (int)(rc.bx * (unsigned)g.tile_w) + rc.ch * TILE_COLS;
+        n.flush = false;
+        if (++r_step == r_steps) {                   // the slab is in registers: move on
+            n.flush = rc.sl == g.spb - 1 || r_s + 1 == s_hi;
+            if (rc.sl == g.spb - 1) ++r_q;
+            advance(rc);
+            ++r_s;
+            r_stage = r_stage + 1 == RING ? 0 : r_stage + 1;
+            if (r_s < s_hi) enter_slab(); else more = false;
+        }
+    };
 
-        for (int ch = 0; ch < chunks; ++ch) {
-            f32x2 acc[NW][L];
+    f32x2 acc[SC_NW][L];
 #pragma unroll
-            for (int k = 0; k < NW; ++k)
+    for (int k = 0; k < SC_NW; ++k)
 #pragma unroll
-                for (int l = 0; l < L; ++l) acc[k][l] = 0ull;
+        for (int l = 0; l < L; ++l) acc[k][l] = 0ull;
 
-            for (int sl = 0; sl < slabs; ++sl, stage = stage + 1 == RING ? 0 : stage + 1) {
-                // refill the stage read in the previous step, then wait for this slab
-                issue_next();
-                cp_async_wait<RING - 1>();
-                __syncwarp();
-                const unsigned char* src = ring + stage * SLAB_BYTES + my_off;
-                const int rows_here = min(SLAB_ROWS, part_rows - sl * SLAB_ROWS);
-#pragma unroll 1
-                for (int rr = slot; rr < rows_here; rr += ROW_SLOTS, src += ROW_SLOTS * 256) {
-                    uint32_t w[NW];
+    // all candidates on one step's registers
+    auto burst = [&](const StepRegs<RPL>& s) {
 #pragma unroll
-                    for (int h = 0; h < PIECES; ++h) {
-                        const uint4 x = *reinterpret_cast<const uint4*>(src + h * (LANE_COLS * 16));
-                        w[4 * h] = x.x; w[4 * h + 1] = x.y; w[4 * h + 2] = x.z; w[4 * h + 3] = x.w;
+        for (int i = 0; i < RPL; ++i) {
+            const f32x2 rinv2 = pk2(s.rinv[i], s.rinv[i]), range2 = pk2(s.range[i], s.range[i]);
+            const f32x2 nlo2 = pk2(-s.lo[i], -s.lo[i]);
+            f32x2 vm[SC_NW];
+#pragma unroll
+            for (int k = 0; k < SC_NW; ++k) vm[k] = add2(pk2(bf16lo(s.w[i][k]), bf16hi(s.w[i][k])), nlo2);
+            if (ROWW) {
+                const f32x2 sa2 = pk2(s.sa[i], s.sa[i]);
+#pragma unroll
+                for (int k = 0; k < SC_NW; ++k) vm[k] = mul2(vm[k], sa2);
+            }
+#pragma unroll
+            for (int l = 0; l < L; ++l) {
+                const f32x2 q2 = *reinterpret_cast<const f32x2*>(&ba.q2[l]);
+                const f32x2 niq2 = *reinterpret_cast<const f32x2*>(&ba.niq2[l]);
+                const f32x2 inv2 = mul2(q2, rinv2);
+                const f32x2 ns2 = mul2(niq2, range2);                   // -(range / qmax)
+                if (l >= L - NFINE) {
+                    const f32x2 nslo2 = mul2(fma2(ns2, q2, range2), niq2);   // -(residual / qmax)
+#pragma unroll
+                    for (int k = 0; k < SC_NW; ++k) {
+                        const f32x2 qq = add2(fma2(vm[k], inv2, magic2), nmagic2);
+                        const f32x2 e = fma2(qq, nslo2, fma2(qq, ns2, vm[k]));
+                        acc[k][l] = fma2(e, e, acc[k][l]);
                     }
-                    float lo, hi;
-                    group_minmax<NW, FULLG ? LANE_COLS : 0>(w, team, lo, hi);
-                    float range = hi - lo;
-                    const bool live = range >= MIN_RANGE;
-                    float rinv = rcp_approx(range);
-                    float sa = 1.f;
-                    if (ROWW) {
-                        const int64_t r = row_base + sl * SLAB_ROWS + rr;
-                        const float a = row_weight[a_perm ? a_perm[r] : r];
-                        sa = sqrtf(a);
-                        rinv = a > 0.f ? rinv * rcp_approx(sa) : 0.f;
-                        range *= sa;
-                    }
-                    if (!live) { rinv = 0.f; range = 0.f; }
-                    const f32x2 rinv2 = pk2(rinv, rinv), range2 = pk2(range, range);
-                    const f32x2 nlo2 = pk2(-lo, -lo);
-                    f32x2 vm[NW];
+                } else {
 #pragma unroll
-                    for (int k = 0; k < NW; ++k) vm[k] = add2(pk2(bf16lo(w[k]), bf16hi(w[k])), nlo2);
-                    if (ROWW) {
-                        const f32x2 sa2 = pk2(sa, sa);
-#pragma unroll
-                        for (int k = 0; k < NW; ++k) vm[k] = mul2(vm[k], sa2);
-                    }
-#pragma unroll
-                    for (int l = 0; l < L; ++l) {
-                        const f32x2 q2 = *reinterpret_cast<const f32x2*>(&ba.q2[l]);
-                        const f32x2 niq2 = *reinterpret_cast<const f32x2*>(&ba.niq2[l]);
-                        const f32x2 inv2 = mul2(q2, rinv2);
-                        const f32x2 ns2 = mul2(niq2, range2);                   // -(range / qmax)
-                        if (l >= L - NFINE) {
-                            const f32x2 nslo2 = mul2(fma2(ns2, q2, range2), niq2);   // -(residual / qmax)
-#pragma unroll
-                            for (int k = 0; k < NW; ++k) {
-                                const f32x2 qq = add2(fma2(vm[k], inv2, magic2), nmagic2);
-                                const f32x2 e = fma2(qq, nslo2, fma2(qq, ns2, vm[k]));
-                                acc[k][l] = fma2(e, e, acc[k][l]);
-                            }
-                        } else {
-#pragma unroll
-                            for (int k = 0; k < NW; ++k) {
-                                const f32x2 qq = add2(fma2(vm[k], inv2, magic2), nmagic2);
-                                const f32x2 e = fma2(qq, ns2, vm[k]);
-                                acc[k][l] = fma2(e, e, acc[k][l]);
-                            }
-                        }
+                    for (int k = 0; k < SC_NW; ++k) {
+                        const f32x2 qq = add2(fma2(vm[k], inv2, magic2), nmagic2);
+                        const f32x2 e = fma2(qq, ns2, vm[k]);
+                        acc[k][l] = fma2(e, e, acc[k][l]);
                     }
                 }
-                __syncwarp();             // the slab is consumed before its stage is refilled
-            }
-            // column factors once per chunk of the unit
-            const int64_t col = colT + (int64_t)ch * TILE_COLS + cl * CPL;
-#pragma unroll
-            for (int k = 0; k < NW; ++k) {
-                const int64_t j = col + 2 * k;
-                const f32x2 c2 = pk2(__ldg(col_moment + (c_perm ? c_perm[j] : j)),
-                                     __ldg(col_moment + (c_perm ? c_perm[j + 1] : j + 1)));
-#pragma unroll
-                for (int l = 0; l < L; ++l) tot2[l] = fma2(c2, acc[k][l], tot2[l]);
             }
         }
-
-        // lanes of the same block (sub-block when bc < 128), fixed order
+    };
+    // column factors, lanes of the same block, record (chunk number + warp number)
+    auto flush = [&](const StepRegs<RPL>& s) {
+        const int col = s.col + cl * SC_CPL;
+        f32x2 c2[SC_NW];
+#pragma unroll
+        for (int k = 0; k < SC_NW; ++k) {
+            const int j = col + 2 * k;
+            c2[k] = pk2(__ldg(col_moment + (c_perm ? c_perm[j] : j)),
+                        __ldg(col_moment + (c_perm ? c_perm[j + 1] : j + 1)));
+        }
         float tot[L];
 #pragma unroll
         for (int l = 0; l < L; ++l) {
+            f32x2 t2 = 0ull;
+#pragma unroll
+            for (int k = 0; k < SC_NW; ++k) { t2 = fma2(c2[k], acc[k][l], t2); acc[k][l] = 0ull; }
             float a0, a1;
-            upk2(tot2[l], a0, a1);
+            upk2(t2, a0, a1);
             float v = a0 + a1;
-            for (int o = lanes_per_sub >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            for (int o = LANE_COLS; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            for (int o = g.lanes_per_sub >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            v += __shfl_xor_sync(0xffffffffu, v, 16);
             tot[l] = v;
         }
-        if (slot == 0 && (cl % lanes_per_sub) == 0) {
-            const int sb = cl / lanes_per_sub;
-            const int64_t blk = (int64_t)by * n_block_cols + (int64_t)(bx * (unsigned)nsub + (unsigned)sb);
-            float* dst = part_out + ((int64_t)p * n_blocks + blk) * L;
+        if (slot == 0 && (cl % g.lanes_per_sub) == 0) {
+            float* dst = rec + ((size_t)(s.q + gw) * g.nsub + cl / g.lanes_per_sub) * L;
 #pragma unroll
             for (int l = 0; l < L; ++l) dst[l] = tot[l];
         }
+    };
+
+#pragma unroll
+    for (int i = 0; i < RING - 1; ++i) issue_next();
+    enter_slab();
+    StepRegs<RPL> A, B;
+    load_step(A);
+    while (true) {
+        const bool haveB = more;
+        if (haveB) load_step(B);
+        burst(A);
+        if (A.flush) flush(A);
+        if (!haveB) break;
+        const bool haveA = more;
+        if (haveA) load_step(A);
+        burst(B);
+        if (B.flush) flush(B);
+        if (!haveA) break;
     }
     cp_async_wait<0>();
 }
 
-// err[blk][l] = sum over the row parts of a block, in order; gains; non-finite check
-__global__ void scores_finish_kernel(const float* __restrict__ part, int parts, int64_t n_blocks, int L,
-                                     BitsArg ba, float M, float* __restrict__ err,
-                                     float* __restrict__ gain, SbDeviceState* dstate) {
+// err[blk][l] = sum of the records of the block's chunk columns, in slab order; gains;
+// non-finite check
+__global__ void scores_finish_kernel(const float* __restrict__ rec, ScoreGeom g, int64_t n_blocks,
+                                     int64_t n_block_cols, int L, BitsArg ba, float M,
+                                     float* __restrict__ err, float* __restrict__ gain,
+                                     SbDeviceState* dstate) {
     const int64_t blk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (blk >= n_blocks) return;
+    const unsigned by = (unsigned)(blk / n_block_cols), bxb = (unsigned)(blk - (int64_t)by * n_block_cols);
+    const unsigned bx = bxb / (unsigned)g.nsub, sb = bxb - bx * (unsigned)g.nsub;
+    const unsigned t = by * g.n_tile_cols + bx;
     float e[8];
+    for (int l = 0; l < L; ++l) e[l] = 0.f;
+    for (int ch = 0; ch < g.chunks; ++ch) {
+        const unsigned q = t * (unsigned)g.chunks + (unsigned)ch;
+        const unsigned s0 = q * (unsigned)g.spb, s1 = s0 + (unsigned)g.spb - 1u;
+        const unsigned w0 = slab_owner(s0, g.n_slabs, g.n_warps), w1 = slab_owner(s1, g.n_slabs, g.n_warps);
+        for (unsigned w = w0; w <= w1; ++w) {
+            const float* src = rec + ((size_t)(q + w) * g.nsub + sb) * L;
+            for (int l = 0; l < L; ++l) e[l] += src[l];
+        }
+    }
     bool finite = true;
     for (int l = 0; l < L; ++l) {
-        float s = 0.f;
-        for (int p = 0; p < parts; ++p) s += part[((int64_t)p * n_blocks + blk) * L + l];
-        e[l] = s;
-        err[blk * L + l] = s;
-        finite = finite && isfinite(s);
+        err[blk * L + l] = e[l];
+        finite = finite && isfinite(e[l]);
     }
     if (!finite) sb_latch(dstate, SB_ERR_NONFINITE, SBK_SCORES);
     if (gain)
@@ -674,62 +750,43 @@ sb_status argsort_axis(sb_ctx* ctx, const float* score, int64_t K, int64_t seg, 
     return SB_OK;
 }
 
-template <int L, int CPL, int NFINE, bool FULLG, bool ROWW>
+template <int L, int RPL, int NFINE, bool FULLG, bool ROWW>
 sb_status launch_scores_k(sb_ctx* ctx, const __nv_bfloat16* W, int64_t ldw, const int32_t* lrp,
                           const int32_t* cperm, const int32_t* aperm, const float* cm, const float* rw,
-                          int br, int bc, int group, const BitsArg& ba, int64_t R, int64_t C, float* err,
-                          float* gain, float* part_buf) {
-    const int tile_w = bc >= 128 ? bc : 128;
-    const int64_t n_tile_cols = C / tile_w, nbc = C / bc, n_blocks = (R / br) * nbc;
-    // a unit is a 32-row part of a tile when the block height allows it, else the whole tile
-    const int part_rows = br % 32 == 0 ? 32 : br;
-    const int parts = br / part_rows;
-    const int64_t n_units = (R / br) * n_tile_cols * parts;
+                          const ScoreGeom& g, const BitsArg& ba, int64_t n_blocks, int64_t nbc, int grid,
+                          float* err, float* gain, float* rec) {
     const size_t smem = (size_t)SC_WARPS * RING * SLAB_BYTES;
-    auto kern = block_scores_kernel<L, CPL, NFINE, FULLG, ROWW>;
+    auto kern = block_scores_kernel<L, RPL, NFINE, FULLG, ROWW>;
     static bool attr_done = false;
     if (!attr_done) {
         SB_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attr_done = true;
     }
-    int64_t grid = ctx->sm_count;                   // persistent: one 16-warp CTA per SM
-    const int64_t need = (n_units + SC_WARPS - 1) / SC_WARPS;
-    if (grid > need) grid = need;
-    kern<<<(unsigned)grid, SC_THREADS, smem, ctx->stream>>>(
-        W, ldw, lrp, cperm, aperm, cm, rw, br, bc, group, ba, nbc, n_tile_cols, parts, part_rows, n_units,
-        n_blocks, part_buf);
+    kern<<<(unsigned)grid, SC_THREADS, smem, ctx->stream>>>(W, ldw, lrp, cperm, aperm, cm, rw, g, ba, rec);
     SB_LAUNCHED(ctx);
     scores_finish_kernel<<<(unsigned)((n_blocks + 255) / 256), 256, 0, ctx->stream>>>(
-        part_buf, parts, n_blocks, L, ba, (float)br * (float)bc, err, gain, ctx->dstate);
+        rec, g, n_blocks, nbc, L, ba, (float)g.br * (float)g.bc, err, gain, ctx->dstate);
     SB_LAUNCHED(ctx);
     return SB_OK;
 }
 
 // the common case (group = 128 columns, no row weights) gets its own instance with the
 // group reduction unrolled; everything else shares the general one
-template <int L, int CPL, int NFINE>
-sb_status launch_scores_n(sb_ctx* ctx, const __nv_bfloat16* W, int64_t ldw, const int32_t* lrp,
-                          const int32_t* cperm, const int32_t* aperm, const float* cm, const float* rw,
-                          int br, int bc, int group, const BitsArg& ba, int64_t R, int64_t C, float* err,
-                          float* gain, float* part_buf) {
-    if (group == 128 && !rw)
-        return launch_scores_k<L, CPL, NFINE, true, false>(ctx, W, ldw, lrp, cperm, aperm, cm, rw, br, bc,
-                                                           group, ba, R, C, err, gain, part_buf);
-    if (!rw)
-        return launch_scores_k<L, CPL, NFINE, false, false>(ctx, W, ldw, lrp, cperm, aperm, cm, rw, br, bc,
-                                                            group, ba, R, C, err, gain, part_buf);
-    return launch_scores_k<L, CPL, NFINE, false, true>(ctx, W, ldw, lrp, cperm, aperm, cm, rw, br, bc,
-                                                       group, ba, R, C, err, gain, part_buf);
+template <int L, int RPL, int NFINE, typename... A>
+sb_status launch_scores_n(int group, const float* rw, A... args) {
+    if (group == 128 && !rw) return launch_scores_k<L, RPL, NFINE, true, false>(args...);
+    if (!rw) return launch_scores_k<L, RPL, NFINE, false, false>(args...);
+    return launch_scores_k<L, RPL, NFINE, false, true>(args...);
 }
 
 // candidates with >= 6 bits keep a two-float grid step; they are the last `nfine` of the list.
 // Compiled for 0..2 such candidates and for "all of them" (always correct, a little slower).
-template <int L, int CPL, typename... A>
+template <int L, int RPL, typename... A>
 sb_status launch_scores(int nfine, A... args) {
-    if (nfine == 0) return launch_scores_n<L, CPL, 0>(args...);
-    if (nfine == 1 && L >= 1) return launch_scores_n<L, CPL, (L >= 1 ? 1 : L)>(args...);
-    if (nfine == 2 && L >= 2) return launch_scores_n<L, CPL, (L >= 2 ? 2 : L)>(args...);
-    return launch_scores_n<L, CPL, L>(args...);
+    if (nfine == 0) return launch_scores_n<L, RPL, 0>(args...);
+    if (nfine == 1 && L >= 1) return launch_scores_n<L, RPL, (L >= 1 ? 1 : L)>(args...);
+    if (nfine == 2 && L >= 2) return launch_scores_n<L, RPL, (L >= 2 ? 2 : L)>(args...);
+    return launch_scores_n<L, RPL, L>(args...);
 }
 
 }  // namespace
@@ -867,15 +924,32 @@ sb_status sb_block_scores(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int6
     const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(W);
     int64_t ld = ldw;
     const int32_t* load_rp = row_perm;
-    const int parts_max = br % 32 == 0 ? br / 32 : 1;
-    const size_t part_bytes = (size_t)parts_max * (R / br) * (C / bc) * n_bits * sizeof(float);
+    // geometry of the slab walk and the record buffer of the partial sums
+    ScoreGeom geo{};
+    geo.br = br; geo.bc = bc; geo.group = group;
+    geo.tile_w = bc >= TILE_COLS ? bc : TILE_COLS;
+    if (C % geo.tile_w) return sb_fail(ctx, SB_ERR_SHAPE, "scores: C must be a multiple of 128");
+    geo.chunks = geo.tile_w / TILE_COLS;
+    geo.spb = (br + SLAB_ROWS - 1) / SLAB_ROWS;
+    geo.nsub = bc >= TILE_COLS ? 1 : TILE_COLS / bc;
+    geo.lanes_per_sub = bc >= TILE_COLS ? TILE_COLS / SC_CPL : bc / SC_CPL;
+    geo.n_tile_cols = (unsigned)(C / geo.tile_w);
+    const int64_t n_chunk_cols = (R / br) * (int64_t)geo.n_tile_cols * geo.chunks;
+    const int64_t n_slabs = n_chunk_cols * geo.spb;
+    if (n_slabs >= (1ll << 31)) return sb_fail(ctx, SB_ERR_SHAPE, "scores: matrix too large");
+    geo.n_slabs = (unsigned)n_slabs;
+    int64_t grid = (n_slabs + SC_WARPS - 1) / SC_WARPS;       // persistent: one 16-warp CTA per SM
+    if (grid > ctx->sm_count) grid = ctx->sm_count;
+    geo.n_warps = (unsigned)(grid * SC_WARPS);
+    const int64_t nbc = C / bc, n_blocks = (R / br) * nbc;
+    const size_t rec_bytes = (size_t)(n_chunk_cols + geo.n_warps) * geo.nsub * n_bits * sizeof(float);
     const bool need_copy = col_perm || W_perm_out;
     void* arena;
-    sb_status sst = sb_scratch(ctx, Carver::need({part_bytes, (need_copy && !W_perm_out) ? (size_t)R * C * 2 : 0}),
+    sb_status sst = sb_scratch(ctx, Carver::need({rec_bytes, (need_copy && !W_perm_out) ? (size_t)R * C * 2 : 0}),
                                &arena);
     if (sst != SB_OK) return sst;
     Carver cv(arena);
-    float* part_buf = cv.take<float>(part_bytes / sizeof(float));
+    float* rec = cv.take<float>(rec_bytes / sizeof(float));
     if (need_copy) {
         void* dst = W_perm_out ? W_perm_out : static_cast<void*>(cv.take<unsigned char>((size_t)R * C * 2));
         sb_status st = sb_gather_bf16(ctx, W, R, C, ldw, row_perm, col_perm, dst);
@@ -885,23 +959,22 @@ sb_status sb_block_scores(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int6
         load_rp = nullptr;
     }
     const BitsArg ba = make_bits(bits, n_bits);
-    const int tile_w = bc >= 128 ? bc : 128;
-    if (C % tile_w) return sb_fail(ctx, SB_ERR_SHAPE, "scores: C must be a multiple of 128");
     sb_status st = SB_OK;
     int nfine = 0;
     for (int l = 0; l < n_bits; ++l) nfine += bits[l] >= 6;
-#define SB_SCORES(Lv, CPLv)                                                                        \
-    st = launch_scores<Lv, CPLv>(nfine, ctx, src, ld, load_rp, col_perm, row_perm, col_moment,     \
-                                 row_weight, br, bc, group, ba, R, C, err, gain, part_buf)
+    // up to four candidates: a lane takes two rows per step; more: one row (fewer accumulators)
+#define SB_SCORES(Lv, RPLv)                                                                        \
+    st = launch_scores<Lv, RPLv>(nfine, group, row_weight, ctx, src, ld, load_rp, col_perm, row_perm, \
+                                 col_moment, row_weight, geo, ba, n_blocks, nbc, (int)grid, err, gain, rec)
     switch (n_bits) {
-        case 1: SB_SCORES(1, 16); break;
-        case 2: SB_SCORES(2, 16); break;
-        case 3: SB_SCORES(3, 16); break;
-        case 4: SB_SCORES(4, 16); break;
-        case 5: SB_SCORES(5, 8); break;
-        case 6: SB_SCORES(6, 8); break;
-        case 7: SB_SCORES(7, 8); break;
-        default: SB_SCORES(8, 8); break;
+        case 1: SB_SCORES(1, 2); break;
+        case 2: SB_SCORES(2, 2); break;
+        case 3: SB_SCORES(3, 2); break;
+        case 4: SB_SCORES(4, 2); break;
+        case 5: SB_SCORES(5, 1); break;
+        case 6: SB_SCORES(6, 1); break;
+        case 7: SB_SCORES(7, 1); break;
+        default: SB_SCORES(8, 1); break;
     }
 #undef SB_SCORES
     return st;
