@@ -343,6 +343,7 @@ def run_only(which: str):
     from paper_2602_17698_b200 import synth
     from paper_2602_17698_b200.binding import Context
     torch.cuda.set_device(0)
+    torch.manual_seed(0)
     dev = "cuda:0"
     ctx = Context()
     R, Cc = 14336, 4096

@@ -50,6 +50,38 @@ pack_offsets_kernel(const unsigned char* __restrict__ level, int64_t nb, int n_b
     lookback_finish(ds, lb);
 }
 
+// The same for a matrix whose blocks fit one CTA (up to 1024 x PO1_ITEMS): a plain CTA scan,
+// no descriptors, no ticket.
+constexpr int PO1_THREADS = 1024, PO1_ITEMS = 8;
+__global__ void __launch_bounds__(PO1_THREADS)
+pack_offsets_small_kernel(const unsigned char* __restrict__ level, int nb, int n_bits, PackBits pb,
+                          unsigned long long words_per_bit, unsigned long long* __restrict__ block_off,
+                          SbDeviceState* ds) {
+    const int base = (int)threadIdx.x * PO1_ITEMS;
+    unsigned long long v[PO1_ITEMS], sum = 0ull;
+#pragma unroll
+    for (int k = 0; k < PO1_ITEMS; ++k) {
+        v[k] = 0ull;
+        if (base + k < nb) {
+            int l = level[base + k];
+            if (l >= n_bits) { sb_latch(ds, SB_ERR_INVALID, SBK_PACK); l = n_bits - 1; }
+            int b = pb.bits[0];
+#pragma unroll
+            for (int j = 1; j < 8; ++j) b = (l == j) ? pb.bits[j] : b;
+            v[k] = words_per_bit * (unsigned long long)b;
+        }
+        sum += v[k];
+    }
+    unsigned long long total;
+    unsigned long long run = block_exclusive_scan<unsigned long long, PO1_THREADS>(sum, total);
+#pragma unroll
+    for (int k = 0; k < PO1_ITEMS; ++k) {
+        if (base + k < nb) block_off[base + k] = run;
+        run += v[k];
+    }
+    if (threadIdx.x == 0) block_off[nb] = total;
+}
+
 
 
 constexpr double PK_MAGIC64 = 6755399441055744.0;     // 1.5 * 2^52: low word of (t + MAGIC) = rint(t)
@@ -321,7 +353,12 @@ extern "C" sb_status sb_pack_blocks(sb_ctx* ctx, const void* W, int64_t R, int64
     }
     PackBits pb{};
     for (int l = 0; l < 8; ++l) pb.bits[l] = l < n_bits ? bits[l] : bits[n_bits - 1];
-    {
+    if (nb <= PO1_THREADS * PO1_ITEMS) {
+        pack_offsets_small_kernel<<<1, PO1_THREADS, 0, ctx->stream>>>(
+            level, (int)nb, n_bits, pb, (unsigned long long)br * bc / 32,
+            reinterpret_cast<unsigned long long*>(block_off_words), ctx->dstate);
+        SB_LAUNCHED(ctx);
+    } else {
         const unsigned tiles = (unsigned)((nb + PO_TILE - 1) / PO_TILE);
         sb_status st;
         LookbackBuf lb = sb_lookback(ctx, tiles, &st);

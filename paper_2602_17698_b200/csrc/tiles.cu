@@ -216,8 +216,9 @@ __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
 // NFINE = how many of the L candidates (the last ones: bits ascend) keep the grid step as a
 // two-float sum: with many levels q * scale carries the fp32 rounding of the step times q, a
 // bias shared by the whole group; the residual range - scale * qmax is exact in one FMA.
-// A row weight a_r enters as sqrt(a_r) on (v - lo), on the range and, inverted, on the
-// reciprocal, so that the accumulated square carries a_r without any per-candidate work.
+// A row weight a_r multiplies the squared residual itself (one more multiply per pair and
+// candidate in the weighted instances): scaling v - lo by sqrt(a_r) instead would round an
+// otherwise exact difference and cost two digits of accuracy at 8 bits.
 constexpr int SLAB_ROWS = 16;
 constexpr int SLAB_BYTES = SLAB_ROWS * 256;
 constexpr int SC_THREADS = 512;                 // one CTA of 16 warps per SM
@@ -237,26 +238,32 @@ struct ScoreGeom {
 __device__ __forceinline__ unsigned slab_owner(unsigned s, unsigned n_slabs, unsigned n_warps) {
     return (unsigned)((((unsigned long long)s + 1ull) * n_warps - 1ull) / n_slabs);
 }
+// warps between two owners may have an empty range (more warps than slabs): they write no record
+__device__ __forceinline__ bool slab_range_empty(unsigned w, unsigned n_slabs, unsigned n_warps) {
+    return (unsigned long long)n_slabs * w / n_warps == (unsigned long long)n_slabs * (w + 1) / n_warps;
+}
 
 struct SlabCursor { int sl, ch; unsigned bx, by; };
 
 template <int RPL>
 struct StepRegs {
     uint32_t w[RPL][SC_NW];
-    float lo[RPL], rinv[RPL], range[RPL], sa[RPL];
+    float lo[RPL], rinv[RPL], range[RPL], ar[RPL];   // ar: row weight a_r (1 without weights)
     unsigned q;          // chunk column (in slab-sequence order) the step belongs to
     int col;             // first column of that chunk
+    int row;             // first row of the step (the lane's rows are row + slot + 2 i)
     bool flush;          // last step of the warp's stretch of this chunk column
 };
 
-template <int L, int RPL, int NFINE, bool FULLG, bool ROWW>
+// The walk itself.  P supplies what is done with a step (P::burst) and with the end of a
+// stretch (P::flush), and keeps its accumulators in registers.
+template <class P>
 __global__ void __launch_bounds__(SC_THREADS, 1)
-block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
-                    const int32_t* __restrict__ load_row_perm,   // rows gathered at load time
-                    const int32_t* __restrict__ c_perm,          // original column of permuted j
-                    const int32_t* __restrict__ a_perm,          // original row of permuted r
-                    const float* __restrict__ col_moment, const float* __restrict__ row_weight,
-                    ScoreGeom g, BitsArg ba, float* __restrict__ rec) {
+slab_walk_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
+                 const int32_t* __restrict__ load_row_perm,   // rows gathered at load time
+                 const int32_t* __restrict__ a_perm,          // original row of permuted r
+                 const float* __restrict__ row_weight, ScoreGeom g, typename P::Args pa) {
+    constexpr int RPL = P::RPL;
     constexpr int STEP_ROWS = 2 * RPL;              // rows per warp step
     extern __shared__ __align__(16) unsigned char tile_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -267,7 +274,6 @@ block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
     const unsigned s_hi = (unsigned)((unsigned long long)g.n_slabs * (gw + 1) / g.n_warps);
     if (s_lo >= s_hi) return;                       // no barriers in this kernel
     unsigned char* ring = tile_smem + (size_t)warp * (RING * SLAB_BYTES);
-    const f32x2 magic2 = pk2(RNE_MAGIC, RNE_MAGIC), nmagic2 = pk2(-RNE_MAGIC, -RNE_MAGIC);
 
     auto advance = [&](SlabCursor& c) {
         if (++c.sl == g.spb) {
@@ -338,25 +344,23 @@ block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
             const uint4 x = *reinterpret_cast<const uint4*>(src + i * 512);
             n.w[i][0] = x.x; n.w[i][1] = x.y; n.w[i][2] = x.z; n.w[i][3] = x.w;
         }
+        n.row = (int)(rc.by * (unsigned)g.br) + rc.sl * SLAB_ROWS + r_step * STEP_ROWS;
 #pragma unroll
         for (int i = 0; i < RPL; ++i) {
             float lo, hi;
-            group_minmax<SC_NW, FULLG ? 16 : 0>(n.w[i], team, lo, hi);
-            float range = hi - lo;
+            group_minmax<SC_NW, P::FULLG ? 16 : 0>(n.w[i], team, lo, hi);
+            const float range = hi - lo;
             const bool live = range >= MIN_RANGE;
-            float rinv = rcp_approx(range);
-            float sa = 1.f;
-            if (ROWW) {
-                const int64_t r = (int64_t)rc.by * g.br + rc.sl * SLAB_ROWS + r_step * STEP_ROWS + 2 * i + slot;
-                const float a = row_weight[a_perm ? a_perm[r] : r];
-                sa = sqrtf(a);
-                rinv = a > 0.f ? rinv * rcp_approx(sa) : 0.f;
-                range *= sa;
+            const float rinv = rcp_approx(range);
+            float ar = 1.f;
+            if (P::ROWW) {
+                const int r = n.row + 2 * i + slot;
+                ar = row_weight[a_perm ? a_perm[r] : r];
             }
             n.lo[i] = lo;
             n.rinv[i] = live ? rinv : 0.f;
             n.range[i] = live ? range : 0.f;
-            n.sa[i] = sa;
+            n.ar[i] = ar;
         }
         n.q = r_q;
         n.col = (int)(rc.bx * (unsigned)g.tile_w) + rc.ch * TILE_COLS;
@@ -371,30 +375,74 @@ block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
         }
     };
 
-    f32x2 acc[SC_NW][L];
+    P p(pa, g, gw, cl, slot);
 #pragma unroll
-    for (int k = 0; k < SC_NW; ++k)
-#pragma unroll
-        for (int l = 0; l < L; ++l) acc[k][l] = 0ull;
+    for (int i = 0; i < RING - 1; ++i) issue_next();
+    enter_slab();
+    StepRegs<RPL> A, B;
+    load_step(A);
+    while (true) {
+        const bool haveB = more;
+        if (haveB) load_step(B);
+        p.burst(A);
+        if (A.flush) p.flush(A);
+        if (!haveB) break;
+        const bool haveA = more;
+        if (haveA) load_step(A);
+        p.burst(B);
+        if (B.flush) p.flush(B);
+        if (!haveA) break;
+    }
+    cp_async_wait<0>();
+}
 
-    // all candidates on one step's registers
-    auto burst = [&](const StepRegs<RPL>& s) {
+// v - lo of a lane's 8 columns as packed pairs (exact: both are bf16 values of one group)
+template <int RPL>
+__device__ __forceinline__ void centred_pairs(const StepRegs<RPL>& s, int i, f32x2 (&vm)[SC_NW]) {
+    const f32x2 nlo2 = pk2(-s.lo[i], -s.lo[i]);
+#pragma unroll
+    for (int k = 0; k < SC_NW; ++k) {
+        // low half through the byte permuter: the shift would take a slot of the FP32 pipe
+        const float v0 = __uint_as_float(__byte_perm(s.w[i][k], 0u, 0x1044));
+        vm[k] = add2(pk2(v0, bf16hi(s.w[i][k])), nlo2);
+    }
+}
+
+// Block scores: all L candidates per step, per-column accumulators, one record per stretch.
+template <int L_, int RPL_, int NFINE, bool FULLG_, bool ROWW_>
+struct ScorePolicy {
+    static constexpr int L = L_, RPL = RPL_;
+    static constexpr bool FULLG = FULLG_, ROWW = ROWW_;
+    struct Args {
+        const int32_t* c_perm;           // original column of permuted j
+        const float* col_moment;
+        BitsArg ba;
+        float* rec;
+    };
+    const Args& a;
+    const ScoreGeom& g;
+    const unsigned gw;
+    const int cl, slot;
+    f32x2 acc[SC_NW][L];
+    __device__ __forceinline__ ScorePolicy(const Args& a_, const ScoreGeom& g_, unsigned gw_, int cl_, int slot_)
+        : a(a_), g(g_), gw(gw_), cl(cl_), slot(slot_) {
+#pragma unroll
+        for (int k = 0; k < SC_NW; ++k)
+#pragma unroll
+            for (int l = 0; l < L; ++l) acc[k][l] = 0ull;
+    }
+    __device__ __forceinline__ void burst(const StepRegs<RPL>& s) {
+        const f32x2 magic2 = pk2(RNE_MAGIC, RNE_MAGIC), nmagic2 = pk2(-RNE_MAGIC, -RNE_MAGIC);
 #pragma unroll
         for (int i = 0; i < RPL; ++i) {
             const f32x2 rinv2 = pk2(s.rinv[i], s.rinv[i]), range2 = pk2(s.range[i], s.range[i]);
-            const f32x2 nlo2 = pk2(-s.lo[i], -s.lo[i]);
+            const f32x2 ar2 = pk2(s.ar[i], s.ar[i]);
             f32x2 vm[SC_NW];
-#pragma unroll
-            for (int k = 0; k < SC_NW; ++k) vm[k] = add2(pk2(bf16lo(s.w[i][k]), bf16hi(s.w[i][k])), nlo2);
-            if (ROWW) {
-                const f32x2 sa2 = pk2(s.sa[i], s.sa[i]);
-#pragma unroll
-                for (int k = 0; k < SC_NW; ++k) vm[k] = mul2(vm[k], sa2);
-            }
+            centred_pairs<RPL>(s, i, vm);
 #pragma unroll
             for (int l = 0; l < L; ++l) {
-                const f32x2 q2 = *reinterpret_cast<const f32x2*>(&ba.q2[l]);
-                const f32x2 niq2 = *reinterpret_cast<const f32x2*>(&ba.niq2[l]);
+                const f32x2 q2 = *reinterpret_cast<const f32x2*>(&a.ba.q2[l]);
+                const f32x2 niq2 = *reinterpret_cast<const f32x2*>(&a.ba.niq2[l]);
                 const f32x2 inv2 = mul2(q2, rinv2);
                 const f32x2 ns2 = mul2(niq2, range2);                   // -(range / qmax)
                 if (l >= L - NFINE) {
@@ -403,28 +451,28 @@ block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
                     for (int k = 0; k < SC_NW; ++k) {
                         const f32x2 qq = add2(fma2(vm[k], inv2, magic2), nmagic2);
                         const f32x2 e = fma2(qq, nslo2, fma2(qq, ns2, vm[k]));
-                        acc[k][l] = fma2(e, e, acc[k][l]);
+                        acc[k][l] = fma2(ROWW ? mul2(e, ar2) : e, e, acc[k][l]);
                     }
                 } else {
 #pragma unroll
                     for (int k = 0; k < SC_NW; ++k) {
                         const f32x2 qq = add2(fma2(vm[k], inv2, magic2), nmagic2);
                         const f32x2 e = fma2(qq, ns2, vm[k]);
-                        acc[k][l] = fma2(e, e, acc[k][l]);
+                        acc[k][l] = fma2(ROWW ? mul2(e, ar2) : e, e, acc[k][l]);
                     }
                 }
             }
         }
-    };
+    }
     // column factors, lanes of the same block, record (chunk number + warp number)
-    auto flush = [&](const StepRegs<RPL>& s) {
+    __device__ __forceinline__ void flush(const StepRegs<RPL>& s) {
         const int col = s.col + cl * SC_CPL;
         f32x2 c2[SC_NW];
 #pragma unroll
         for (int k = 0; k < SC_NW; ++k) {
             const int j = col + 2 * k;
-            c2[k] = pk2(__ldg(col_moment + (c_perm ? c_perm[j] : j)),
-                        __ldg(col_moment + (c_perm ? c_perm[j + 1] : j + 1)));
+            c2[k] = pk2(__ldg(a.col_moment + (a.c_perm ? a.c_perm[j] : j)),
+                        __ldg(a.col_moment + (a.c_perm ? a.c_perm[j + 1] : j + 1)));
         }
         float tot[L];
 #pragma unroll
@@ -440,31 +488,12 @@ block_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
             tot[l] = v;
         }
         if (slot == 0 && (cl % g.lanes_per_sub) == 0) {
-            float* dst = rec + ((size_t)(s.q + gw) * g.nsub + cl / g.lanes_per_sub) * L;
+            float* dst = a.rec + ((size_t)(s.q + gw) * g.nsub + cl / g.lanes_per_sub) * L;
 #pragma unroll
             for (int l = 0; l < L; ++l) dst[l] = tot[l];
         }
-    };
-
-#pragma unroll
-    for (int i = 0; i < RING - 1; ++i) issue_next();
-    enter_slab();
-    StepRegs<RPL> A, B;
-    load_step(A);
-    while (true) {
-        const bool haveB = more;
-        if (haveB) load_step(B);
-        burst(A);
-        if (A.flush) flush(A);
-        if (!haveB) break;
-        const bool haveA = more;
-        if (haveA) load_step(A);
-        burst(B);
-        if (B.flush) flush(B);
-        if (!haveA) break;
     }
-    cp_async_wait<0>();
-}
+};
 
 // err[blk][l] = sum of the records of the block's chunk columns, in slab order; gains;
 // non-finite check
@@ -484,6 +513,7 @@ __global__ void scores_finish_kernel(const float* __restrict__ rec, ScoreGeom g,
         const unsigned s0 = q * (unsigned)g.spb, s1 = s0 + (unsigned)g.spb - 1u;
         const unsigned w0 = slab_owner(s0, g.n_slabs, g.n_warps), w1 = slab_owner(s1, g.n_slabs, g.n_warps);
         for (unsigned w = w0; w <= w1; ++w) {
+            if (slab_range_empty(w, g.n_slabs, g.n_warps)) continue;
             const float* src = rec + ((size_t)(q + w) * g.nsub + sb) * L;
             for (int l = 0; l < L; ++l) e[l] += src[l];
         }
@@ -756,13 +786,15 @@ sb_status launch_scores_k(sb_ctx* ctx, const __nv_bfloat16* W, int64_t ldw, cons
                           const ScoreGeom& g, const BitsArg& ba, int64_t n_blocks, int64_t nbc, int grid,
                           float* err, float* gain, float* rec) {
     const size_t smem = (size_t)SC_WARPS * RING * SLAB_BYTES;
-    auto kern = block_scores_kernel<L, RPL, NFINE, FULLG, ROWW>;
+    using P = ScorePolicy<L, RPL, NFINE, FULLG, ROWW>;
+    auto kern = slab_walk_kernel<P>;
     static bool attr_done = false;
     if (!attr_done) {
         SB_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attr_done = true;
     }
-    kern<<<(unsigned)grid, SC_THREADS, smem, ctx->stream>>>(W, ldw, lrp, cperm, aperm, cm, rw, g, ba, rec);
+    typename P::Args pa{cperm, cm, ba, rec};
+    kern<<<(unsigned)grid, SC_THREADS, smem, ctx->stream>>>(W, ldw, lrp, aperm, rw, g, pa);
     SB_LAUNCHED(ctx);
     scores_finish_kernel<<<(unsigned)((n_blocks + 255) / 256), 256, 0, ctx->stream>>>(
         rec, g, n_blocks, nbc, L, ba, (float)g.br * (float)g.bc, err, gain, ctx->dstate);

@@ -25,3 +25,16 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _seeded_generators():
+    """Every test draws from freshly seeded numpy / torch generators (CPU and CUDA)."""
+    import numpy as np
+    np.random.seed(20260217)
+    try:
+        import torch
+        torch.manual_seed(20260217)
+    except Exception:  # pragma: no cover
+        pass
+    yield

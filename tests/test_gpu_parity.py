@@ -362,6 +362,29 @@ def test_pack(ctx, br, bc, g):
     assert codes.max() <= 2 ** b - 1
 
 
+def test_pack_many_blocks_offsets_span_several_scan_tiles(ctx):
+    R, C, br, bc, g = 2048, 4096, 32, 32, 32          # 8192 blocks x 2 = 16384 > one CTA's scan
+    bits = [2, 3, 4]
+    W = synth.make_weight(2 * R, C, 77, DEV)
+    nb = (2 * R // br) * (C // bc)
+    rng = np.random.default_rng(5)
+    level = torch.from_numpy(rng.integers(0, len(bits), size=nb).astype(np.uint8)).to(DEV)
+    packed, off, meta = ctx.pack_blocks(W, bits, level, br, bc, g)
+    ctx.sync()
+    sizes = np.array(bits)[level.cpu().numpy()] * (br * bc // 32)
+    off_h = off.cpu().numpy()
+    assert off_h[0] == 0 and np.array_equal(np.diff(off_h), sizes)
+    # sampled blocks against the oracle
+    Wh = W.cpu()
+    nbc = C // bc
+    for blk in rng.choice(nb, 16, replace=False):
+        bi, bj = divmod(int(blk), nbc)
+        tile = Wh[bi * br:(bi + 1) * br, bj * bc:(bj + 1) * bc].contiguous()
+        op, _, ometa = sbo.pack_blocks(tile, bits, level[blk:blk + 1].cpu().numpy(), br, bc, g)
+        got = packed[int(off_h[blk]):int(off_h[blk + 1])].cpu().numpy().view(np.uint32)
+        assert np.array_equal(got, op)
+
+
 def test_pack_capacity_is_enforced(ctx):
     from paper_2602_17698_b200.binding import SbError, SB_ERR_SCRATCH
     W = synth.make_weight(256, 256, 3, DEV)
