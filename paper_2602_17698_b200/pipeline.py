@@ -268,3 +268,177 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
     stage("pack", do_pack)
     res.packed = dict(ws.packed)
     return res
+
+
+# ---- whole model: one global allocation over the blocks of all layers --------------------------------
+@dataclass
+class ModelResult:
+    """Outputs of `search_model`; `tables[ref_bits]` is the [N, L] table the budgets of that
+    warm-start precision were allocated on, blocks ordered layer by layer, matrices in
+    `shape.linears` order inside a layer."""
+    moments: list                                    # per layer: {input name: [K] fp32}
+    block_start: Dict[tuple, int]                    # (layer, matrix name) -> first table row
+    n_blocks: int
+    tables: Dict[int, torch.Tensor] = field(default_factory=dict)
+    perms: Dict[int, dict] = field(default_factory=dict)      # ref_bits -> {"hidden": p, (set, layer): p}
+    scores: Dict[int, dict] = field(default_factory=dict)     # ref_bits -> the sorted score vectors
+    levels: Dict[float, torch.Tensor] = field(default_factory=dict)
+    reports: Dict[float, dict] = field(default_factory=dict)
+    ms: Dict[str, float] = field(default_factory=dict)        # CUDA-event time of the library calls
+
+
+class _Clock:
+    """Sums CUDA-event time of bracketed regions per key (read after a synchronise)."""
+
+    def __init__(self):
+        self.pairs = {}
+
+    def __call__(self, key):
+        clock = self
+
+        class _R:
+            def __enter__(self_inner):
+                self_inner.a = torch.cuda.Event(enable_timing=True)
+                self_inner.b = torch.cuda.Event(enable_timing=True)
+                self_inner.a.record()
+
+            def __exit__(self_inner, *exc):
+                self_inner.b.record()
+                clock.pairs.setdefault(key, []).append((self_inner.a, self_inner.b))
+
+        return _R()
+
+    def totals(self):
+        return {k: sum(a.elapsed_time(b) for a, b in v) for k, v in self.pairs.items()}
+
+
+def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConfig,
+                 budgets: Sequence[float], make_weights, make_acts, device,
+                 keep_tables: bool = True) -> ModelResult:
+    """Two sweeps over a model of `n_layers` identical decoder layers, then one global
+    allocation per budget (Eq. 1 over ALL blocks of the model).
+
+    The residual-stream permutation is shared by every layer (Appendix D: the hidden dimension
+    runs through the whole network), so its score vector is accumulated over all layers before
+    it is sorted: sweep 1 takes moments and reorder statistics, sweep 2 scores the blocks of
+    the permuted matrices.  Reorder statistics are taken at the warm-start precision of the
+    budget, so budgets are grouped by that precision and the sweeps run once per group.
+
+    `make_weights(layer)` / `make_acts(layer)` return the layer's tensors on `device` (weights
+    are kept resident, activations are dropped after their moments).  Only library calls are
+    timed (`ModelResult.ms`, keys moments / stats@b / sort@b / scores@b / allocate@budget).
+    """
+    f32 = dict(dtype=torch.float32, device=device)
+    i32 = dict(dtype=torch.int32, device=device)
+    lin = {l.name: l for l in shape.linears}
+    g = cfg.group
+    L = len(cfg.bits)
+    reps = shape.n_heads // shape.n_kv_heads
+    hd = shape.head_dim
+    kv, qd = shape.n_kv_heads * hd, shape.n_heads * hd
+    clock = _Clock()
+    prev_stream = torch.cuda.current_stream()
+
+    block_start, n = {}, 0
+    for layer in range(n_layers):
+        for l in shape.linears:
+            block_start[(layer, l.name)] = n
+            n += (l.rows // cfg.block_rows) * (l.cols // cfg.block_cols)
+    res = ModelResult(moments=[], block_start=block_start, n_blocks=n)
+
+    with torch.cuda.stream(ctx.stream):
+        # a1 once: the moments do not depend on the budget
+        weights = []
+        for layer in range(n_layers):
+            X = make_acts(layer)
+            m = {name: torch.empty(k, **f32) for name, k in shape.act_dims.items()}
+            with clock("moments"):
+                for name, x in X.items():
+                    ctx.calib_moments(x, m[name])
+            ctx.stream.synchronize()               # X is dropped: its memory must not be reused early
+            del X
+            res.moments.append(m)
+            weights.append(make_weights(layer))
+
+        groups = {}
+        for b in budgets:
+            ok = [x for x in cfg.bits if x <= b]
+            groups.setdefault(max(ok) if ok else min(cfg.bits), []).append(b)
+
+        for rb, bs in sorted(groups.items()):
+            hid = torch.empty(shape.hidden, **f32)
+            mid = [torch.empty(shape.intermediate, **f32) for _ in range(n_layers)]
+            vo = [torch.empty(kv, **f32) for _ in range(n_layers)]
+            ocol = [torch.empty(qd, **f32) for _ in range(n_layers)]
+            # sweep 1: a2, hidden scores accumulated over all layers
+            with clock(f"stats@{rb}"):
+                for layer in range(n_layers):
+                    W, m = weights[layer], res.moments[layer]
+                    c = {nm: m[l.act] for nm, l in lin.items()}
+                    first = layer == 0
+                    ctx.reorder_channels(W["q_proj"], c["q_proj"], rb, g, col_score=hid, accumulate_col=not first)
+                    ctx.reorder_channels(W["k_proj"], c["k_proj"], rb, g, col_score=hid, accumulate_col=True)
+                    ctx.reorder_channels(W["v_proj"], c["v_proj"], rb, g, row_score=vo[layer], col_score=hid,
+                                         accumulate_col=True)
+                    ctx.reorder_channels(W["o_proj"], c["o_proj"], rb, g, row_score=hid, col_score=ocol[layer],
+                                         accumulate_row=True)
+                    ctx.reorder_channels(W["gate_proj"], c["gate_proj"], rb, g, row_score=mid[layer],
+                                         col_score=hid, accumulate_col=True)
+                    ctx.reorder_channels(W["up_proj"], c["up_proj"], rb, g, row_score=mid[layer], col_score=hid,
+                                         accumulate_row=True, accumulate_col=True)
+                    ctx.reorder_channels(W["down_proj"], c["down_proj"], rb, g, row_score=hid,
+                                         col_score=mid[layer], accumulate_row=True, accumulate_col=True)
+            # a3: one sort of the residual stream, per-layer sorts of the other sets
+            p_hid = torch.empty(shape.hidden, **i32)
+            p_mid = [torch.empty(shape.intermediate, **i32) for _ in range(n_layers)]
+            p_v = [torch.empty(kv, **i32) for _ in range(n_layers)]
+            p_o = [torch.empty(qd, **i32) for _ in range(n_layers)]
+            with clock(f"sort@{rb}"):
+                if cfg.reorder:
+                    ctx.reorder_channels(None, None, rb, g, row_score=hid, row_segment=shape.hidden,
+                                         row_perm=p_hid, shape=(shape.hidden, g))
+                    for layer in range(n_layers):
+                        ctx.fold_segment_scores(vo[layer], ocol[layer], reps, hd)
+                        ctx.reorder_channels(None, None, rb, g, row_score=mid[layer],
+                                             row_segment=shape.intermediate, row_perm=p_mid[layer],
+                                             shape=(shape.intermediate, g))
+                        ctx.reorder_channels(None, None, rb, g, row_score=vo[layer], row_segment=hd,
+                                             row_perm=p_v[layer], shape=(kv, g))
+                        ctx.expand_segment_perm(p_v[layer], reps, hd, out=p_o[layer])
+            perms = {"hidden": p_hid if cfg.reorder else None}
+            for layer in range(n_layers):
+                perms[("intermediate", layer)] = p_mid[layer] if cfg.reorder else None
+                perms[("v_heads", layer)] = p_v[layer] if cfg.reorder else None
+                perms[("o_heads", layer)] = p_o[layer] if cfg.reorder else None
+
+            def perm_of(key, layer):
+                if key is None:
+                    return None
+                return perms["hidden"] if key == "hidden" else perms[(key, layer)]
+
+            # sweep 2: a4 into the global table
+            err = torch.empty((n, L), **f32)
+            with clock(f"scores@{rb}"):
+                for layer in range(n_layers):
+                    W, m = weights[layer], res.moments[layer]
+                    for nm, l in lin.items():
+                        nb = (l.rows // cfg.block_rows) * (l.cols // cfg.block_cols)
+                        s = block_start[(layer, nm)]
+                        rp, cp = COUPLING[nm]
+                        ctx.block_scores(W[nm], m[l.act], cfg.bits, cfg.block_rows, cfg.block_cols, g,
+                                         row_perm=perm_of(rp, layer), col_perm=perm_of(cp, layer),
+                                         err=err[s:s + nb], want_gain=False)
+            # a5: one global allocation per budget of the group
+            for b in bs:
+                with clock(f"allocate@{b:g}"):
+                    level, report = ctx.allocate_bits(err, cfg.bits, b, cfg.mode, cfg.gamma0, cfg.gammaT,
+                                                      uniform_block_elems=cfg.block_rows * cfg.block_cols)
+                res.levels[b], res.reports[b] = level, report
+            if keep_tables:
+                res.tables[rb] = err
+                res.perms[rb] = perms
+                res.scores[rb] = {"hidden": hid, "intermediate": mid, "v_heads": vo, "o_cols": ocol}
+        ctx.stream.synchronize()
+    prev_stream.synchronize()
+    res.ms = clock.totals()
+    return res
