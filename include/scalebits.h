@@ -17,8 +17,11 @@
  *   - bf16 matrices are row-major with a leading dimension in elements; the base
  *     must be 16-byte aligned and the leading dimension a multiple of 8.
  *   - A permutation is int32 perm[new] = old.  NULL means identity.
- *   - The library owns one scratch arena per context, grown on demand (a growth
- *     synchronises the stream); after the first call of each shape nothing allocates.
+ *   - The library owns one scratch arena per context, grown on demand; after the
+ *     first call of each shape nothing allocates.  An outgrown arena stays allocated
+ *     until sb_destroy, so launches already enqueued, or captured in a CUDA graph by
+ *     the caller, keep valid scratch pointers (a growth cannot happen during capture:
+ *     run every captured call once eagerly first).
  *   - No call falls back to the CPU.
  */
 #ifndef SCALEBITS_H_

@@ -25,18 +25,20 @@ bool sb_check_bits(const int* bits, int n_bits) {
 
 sb_status sb_scratch(sb_ctx* ctx, size_t bytes, void** out) {
     if (bytes > ctx->scratch_bytes) {
-        // growth is rare (first call of a shape): wait for work that may use the old arena
-        SB_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
-        if (ctx->scratch) SB_CUDA(ctx, cudaFree(ctx->scratch));
-        ctx->scratch = nullptr;
-        ctx->scratch_bytes = 0;
+        // Growth is rare (first call of a shape).  The old arena is retired, not freed: launches
+        // already enqueued, or captured in a CUDA graph by the caller, keep valid pointers until
+        // the context is destroyed.  Doubling bounds the retired arenas by the live one.
         size_t want = bytes + bytes / 8 + (1u << 20);
-        cudaError_t e = cudaMalloc(&ctx->scratch, want);
+        if (want < 2 * ctx->scratch_bytes) want = 2 * ctx->scratch_bytes;
+        void* fresh = nullptr;
+        cudaError_t e = cudaMalloc(&fresh, want);
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
             return sb_fail(ctx, SB_ERR_SCRATCH, "scratch arena of %zu bytes: %s", want,
                            cudaGetErrorString(e));
         }
+        if (ctx->scratch) ctx->retired.push_back(ctx->scratch);
+        ctx->scratch = fresh;
         ctx->scratch_bytes = want;
     }
     *out = ctx->scratch;
@@ -87,6 +89,7 @@ sb_status sb_destroy(sb_ctx* ctx) {
     cudaSetDevice(ctx->device);
     cudaStreamSynchronize(ctx->stream);
     if (ctx->scratch) cudaFree(ctx->scratch);
+    for (void* p : ctx->retired) cudaFree(p);
     if (ctx->dstate) cudaFree(ctx->dstate);
     if (ctx->lb_mem) cudaFree(ctx->lb_mem);
     if (ctx->moment_done) cudaFree(ctx->moment_done);

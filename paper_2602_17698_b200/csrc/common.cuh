@@ -1,5 +1,6 @@
 // Shared host/device helpers of the CUDA library (sm_100a only).
 #pragma once
+#include <vector>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -21,6 +22,7 @@ struct sb_ctx {
     int sm_count = 148;
     void* scratch = nullptr;     // arena, grown on demand
     size_t scratch_bytes = 0;
+    std::vector<void*> retired;  // outgrown arenas and descriptor buffers, freed with the context
     SbDeviceState* dstate = nullptr;
     void* pinned = nullptr;      // small pinned host buffer for read-backs
     size_t pinned_bytes = 0;

@@ -179,15 +179,15 @@ LookbackBuf sb_lookback(sb_ctx* ctx, unsigned tiles, sb_status* st) {
     if (tiles > ctx->lb_max_tiles) {
         unsigned want = 1u << 14;
         while (want < tiles) want <<= 1;
-        cudaStreamSynchronize(ctx->stream);
-        if (ctx->lb_mem) cudaFree(ctx->lb_mem);
-        ctx->lb_mem = nullptr;
-        ctx->lb_max_tiles = 0;
-        if (cudaMalloc(&ctx->lb_mem, (size_t)want * 36) != cudaSuccess) {
+        // the outgrown buffer is retired, not freed: captured launches may still point at it
+        void* fresh = nullptr;
+        if (cudaMalloc(&fresh, (size_t)want * 36) != cudaSuccess) {
             (void)cudaGetLastError();
             *st = sb_fail(ctx, SB_ERR_SCRATCH, "look-back descriptors for %u tiles", want);
             return LookbackBuf{};
         }
+        if (ctx->lb_mem) ctx->retired.push_back(ctx->lb_mem);
+        ctx->lb_mem = fresh;
         ctx->lb_max_tiles = want;
         cudaMemsetAsync(ctx->lb_mem, 0, (size_t)ctx->lb_max_tiles * 36, ctx->stream);
     }

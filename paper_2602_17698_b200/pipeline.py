@@ -314,7 +314,7 @@ class _Clock:
 
 def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConfig,
                  budgets: Sequence[float], make_weights, make_acts, device,
-                 keep_tables: bool = True) -> ModelResult:
+                 keep_tables: bool = True, keep_weights: bool = True) -> ModelResult:
     """Two sweeps over a model of `n_layers` identical decoder layers, then one global
     allocation per budget (Eq. 1 over ALL blocks of the model).
 
@@ -324,8 +324,10 @@ def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConf
     the permuted matrices.  Reorder statistics are taken at the warm-start precision of the
     budget, so budgets are grouped by that precision and the sweeps run once per group.
 
-    `make_weights(layer)` / `make_acts(layer)` return the layer's tensors on `device` (weights
-    are kept resident, activations are dropped after their moments).  Only library calls are
+    `make_weights(layer)` / `make_acts(layer)` return the layer's tensors on `device`.
+    Activations are dropped after their moments; weights stay resident, or with
+    `keep_weights=False` are made again in every sweep (a model larger than the device's
+    memory is streamed layer by layer: only moments, permutations and tables persist).  Only library calls are
     timed (`ModelResult.ms`, keys moments / stats@b / sort@b / scores@b / allocate@budget).
     """
     f32 = dict(dtype=torch.float32, device=device)
@@ -358,7 +360,11 @@ def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConf
             ctx.stream.synchronize()               # X is dropped: its memory must not be reused early
             del X
             res.moments.append(m)
-            weights.append(make_weights(layer))
+            if keep_weights:
+                weights.append(make_weights(layer))
+
+        def layer_weights(layer):
+            return weights[layer] if keep_weights else make_weights(layer)
 
         groups = {}
         for b in budgets:
@@ -371,11 +377,11 @@ def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConf
             vo = [torch.empty(kv, **f32) for _ in range(n_layers)]
             ocol = [torch.empty(qd, **f32) for _ in range(n_layers)]
             # sweep 1: a2, hidden scores accumulated over all layers
-            with clock(f"stats@{rb}"):
-                for layer in range(n_layers):
-                    W, m = weights[layer], res.moments[layer]
-                    c = {nm: m[l.act] for nm, l in lin.items()}
-                    first = layer == 0
+            for layer in range(n_layers):
+                W, m = layer_weights(layer), res.moments[layer]
+                c = {nm: m[l.act] for nm, l in lin.items()}
+                first = layer == 0
+                with clock(f"stats@{rb}"):
                     ctx.reorder_channels(W["q_proj"], c["q_proj"], rb, g, col_score=hid, accumulate_col=not first)
                     ctx.reorder_channels(W["k_proj"], c["k_proj"], rb, g, col_score=hid, accumulate_col=True)
                     ctx.reorder_channels(W["v_proj"], c["v_proj"], rb, g, row_score=vo[layer], col_score=hid,
@@ -418,9 +424,9 @@ def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConf
 
             # sweep 2: a4 into the global table
             err = torch.empty((n, L), **f32)
-            with clock(f"scores@{rb}"):
-                for layer in range(n_layers):
-                    W, m = weights[layer], res.moments[layer]
+            for layer in range(n_layers):
+                W, m = layer_weights(layer), res.moments[layer]
+                with clock(f"scores@{rb}"):
                     for nm, l in lin.items():
                         nb = (l.rows // cfg.block_rows) * (l.cols // cfg.block_cols)
                         s = block_start[(layer, nm)]

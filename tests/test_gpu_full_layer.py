@@ -1,7 +1,8 @@
 """The benchmark's workload at full size (one Llama-3-8B-shaped layer, 65536 tokens) in the
-launch configuration bench.py times (non-default stream, one CUDA graph per stage), checked
-on sampled outputs the oracle can compute one by one, plus the exact stages (permutations
-given scores, levels given the table, budget accounting)."""
+launch configuration bench.py times (non-default stream, one CUDA graph per stage), and the
+corners of the stress sweep (block shapes, group sizes, seven candidates) on the same layer,
+checked on sampled outputs the oracle can compute one by one, plus the exact stages
+(permutations given scores, levels given the table, budget accounting)."""
 import numpy as np
 import pytest
 import torch
@@ -15,15 +16,24 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def test_llama3_8b_layer_full_size_sampled_parity():
+STRESS_BITS = [1, 2, 3, 4, 5, 6, 8]
+
+
+@pytest.mark.parametrize("bits,br,bc,g,budget,tokens", [
+    ([2, 3, 4, 8], 128, 128, 128, 2.5, 65536),        # configs[1], as bench.py times it
+    (STRESS_BITS, 32, 32, 32, 1.75, 4096),            # configs[4]: the stress sweep's corners
+    (STRESS_BITS, 64, 64, 64, 2.5, 4096),
+    (STRESS_BITS, 256, 128, 128, 3.5, 4096),
+    ([2, 3, 4], 128, 128, 64, 3.0, 4096),
+])
+def test_llama3_8b_layer_full_size_sampled_parity(bits, br, bc, g, budget, tokens):
     from paper_2602_17698_b200.binding import Context
     from paper_2602_17698_b200.pipeline import COUPLING, LayerWorkspace, SearchConfig, StageGraphs, search_layer
     torch.cuda.set_device(0)
     shape = synth.LLAMA3_8B
-    bits, br, bc, g = [2, 3, 4, 8], 128, 128, 128
-    cfg = SearchConfig(bits=bits, budget=2.5)
+    cfg = SearchConfig(bits=bits, budget=budget, block_rows=br, block_cols=bc, group=g)
     W = synth.make_layer_weights(shape, 0, 0, DEV)
-    X = synth.make_layer_activations(shape, 65536, 0, 0, DEV)
+    X = synth.make_layer_activations(shape, tokens, 0, 0, DEV)
     stream = torch.cuda.Stream()
     torch.cuda.synchronize()
     with torch.cuda.stream(stream):
@@ -82,7 +92,7 @@ def test_llama3_8b_layer_full_size_sampled_parity():
         assert np.array_equal(lv, olv)
         assert res.report["used_bits"] == orep["used_bits"]
         assert res.report["iterations"] == orep["iterations"]
-    assert res.report["used_bits"] <= res.report["cap_bits"] == int(2.5 * shape.n_weights)
+    assert res.report["used_bits"] <= res.report["cap_bits"] == int(np.floor(budget * shape.n_weights))
 
     # a6: sampled blocks of the packed stream and their metadata; exact budget accounting
     total_words = 0
@@ -106,7 +116,9 @@ def test_llama3_8b_layer_full_size_sampled_parity():
             op, _, ometa = sbo.pack_blocks(tile, bits, lv[s0 + blk:s0 + blk + 1], br, bc, g)
             got = packed[int(off_h[blk]):int(off_h[blk + 1])].cpu().numpy().view(np.uint32)
             assert np.array_equal(got, op), f"packed {name} block {blk}"
-            assert np.array_equal(meta_h[bi * br:(bi + 1) * br, bj].view(np.uint32),
-                                  ometa.view(np.uint32)), f"meta {name} block {blk}"
+            gpb = bc // g                                # quantisation groups across one block
+            got_meta = np.ascontiguousarray(meta_h[bi * br:(bi + 1) * br, bj * gpb:(bj + 1) * gpb])
+            assert np.array_equal(got_meta.view(np.uint32).reshape(-1),
+                                  ometa.view(np.uint32).reshape(-1)), f"meta {name} block {blk}"
     assert total_words * 32 == res.report["used_bits"]
     ctx.close()

@@ -146,8 +146,8 @@ def test_llama3_8b_full_model_allocation_matches_oracle():
             table = res.tables[rb]
             for name, l in lin.items():
                 rp, cp = COUPLING[name]
-                pr = op[rp] if rp not in (None, "hidden") else (op["hidden"] if rp == "hidden" else np.arange(l.rows))
-                pc = op[cp] if cp not in (None, "hidden") else (op["hidden"] if cp == "hidden" else np.arange(l.cols))
+                pr = op[rp] if rp else np.arange(l.rows)
+                pc = op[cp] if cp else np.arange(l.cols)
                 nbc = l.cols // bc
                 nb = (l.rows // br) * nbc
                 s0 = res.block_start[(layer, name)]
@@ -174,4 +174,71 @@ def test_llama3_8b_full_model_allocation_matches_oracle():
             assert np.array_equal(res.levels[b].cpu().numpy(), olv), b
             assert rep["used_bits"] == orep["used_bits"]
             assert rep["iterations"] == orep["iterations"]
+    ctx.close()
+
+
+def test_llama3_70b_streamed_allocation_matches_oracle():
+    """configs[3]: 80 layers of the 70B shape (N = 4,177,920 blocks of 128 x 128), bits {2,3,4},
+    budget 2.25, weights regenerated from their seeds in each sweep (never resident).  The oracle
+    allocates on the GPU's table; sampled blocks of one layer are re-scored."""
+    from paper_2602_17698_b200.binding import Context
+    from paper_2602_17698_b200.pipeline import COUPLING, SearchConfig, search_model
+    torch.cuda.set_device(0)
+    shape, n_layers, tokens = synth.LLAMA3_70B, 80, 2048
+    bits, br, bc, g = [2, 3, 4], 128, 128, 128
+    budget = 2.25
+    cfg = SearchConfig(bits=bits, block_rows=br, block_cols=bc, group=g)
+
+    def make_weights(layer):
+        return synth.make_layer_weights(shape, 0, layer, DEV)
+
+    def make_acts(layer):
+        return synth.make_layer_activations(shape, tokens, 0, layer, DEV)
+
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        ctx = Context()
+        res = search_model(ctx, shape, n_layers, cfg, [budget], make_weights, make_acts, DEV,
+                           keep_weights=False)
+    torch.cuda.synchronize()
+    assert res.n_blocks == 4177920
+    lin = {l.name: l for l in shape.linears}
+    rng = np.random.default_rng(2)
+    sc, pm = res.scores[2], res.perms[2]
+    hid = sc["hidden"].cpu().double().numpy()
+    assert np.array_equal(pm["hidden"].cpu().numpy(), sbo.argsort_desc_segments(hid))
+    layer = 41
+    gsc = {"hidden": hid, "intermediate": sc["intermediate"][layer].cpu().double().numpy(),
+           "v_heads": sc["v_heads"][layer].cpu().double().numpy()}
+    op = helpers.oracle_layer_perms(shape, gsc)
+    for key in ("intermediate", "v_heads", "o_heads"):
+        assert np.array_equal(pm[(key, layer)].cpu().numpy(), op[key]), key
+    W = make_weights(layer)
+    gm = {n: res.moments[layer][n].cpu().double().numpy() for n in shape.act_dims}
+    table = res.tables[2]
+    for name, l in lin.items():
+        rp, cp = COUPLING[name]
+        pr = op[rp] if rp else np.arange(l.rows)
+        pc = op[cp] if cp else np.arange(l.cols)
+        nbc = l.cols // bc
+        nb = (l.rows // br) * nbc
+        s0 = res.block_start[(layer, name)]
+        for blk in rng.choice(nb, 3, replace=False):
+            bi, bj = divmod(int(blk), nbc)
+            rows = torch.from_numpy(pr[bi * br:(bi + 1) * br].astype(np.int64)).to(DEV)
+            cols = pc[bj * bc:(bj + 1) * bc]
+            tile = W[name][rows][:, torch.from_numpy(cols.astype(np.int64)).to(DEV)].contiguous().cpu()
+            oerr, _ = sbo.block_scores(tile, gm[l.act][cols], bits, br, bc, g)
+            assert_close(table[s0 + blk:s0 + blk + 1].cpu().numpy(), oerr, REL, what=f"err {name} block {blk}")
+    del W
+    th = table.cpu().double().numpy()
+    st, olv, orep = sbo.allocate_scalebits(th, bits, budget, cfg.gamma0, cfg.gammaT, br * bc)
+    assert st == sbo.OK
+    rep = res.reports[budget]
+    assert rep["cap_bits"] == int(np.floor(budget * n_layers * shape.n_weights))
+    assert rep["used_bits"] <= rep["cap_bits"]
+    if orep["min_margin"] >= 1e-9:
+        assert np.array_equal(res.levels[budget].cpu().numpy(), olv)
+        assert rep["used_bits"] == orep["used_bits"]
+        assert rep["iterations"] == orep["iterations"]
     ctx.close()
