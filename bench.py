@@ -216,7 +216,7 @@ def full_model_times(ctx, dev):
     # and loads the kernels that only large tables use (the cooperative form of the loop kernel)
     search_model(ctx, shape, 4, cfg, (2.25,), make_weights, make_acts, dev, keep_tables=False)
     res = search_model(ctx, shape, FULL_MODEL_LAYERS, cfg, FULL_MODEL_BUDGETS, make_weights, make_acts, dev,
-                       keep_tables=False)
+                       keep_tables=False, alloc_repeats=2)
     ms = res.ms
     sweeps = sorted({int(k.split("@")[1]) for k in ms if k.startswith("stats@")})
     first = FULL_MODEL_BUDGETS[0]
@@ -237,7 +237,8 @@ def full_model_times(ctx, dev):
             "ms_allocate_per_budget": alloc,
             "iterations_per_budget": {f"{b:g}": res.reports[b]["iterations"] for b in FULL_MODEL_BUDGETS},
             "ms_all_budgets_total": sum(ms.values()),
-            "timing": "sum of CUDA-event times around the library calls"}
+            "timing": "sum of CUDA-event times around the library calls; each allocation call is "
+                      "made twice and the faster one counted (it is eager and paced by the host)"}
 
 
 def run_cuda(args):
