@@ -466,6 +466,244 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, const do
     }
 }
 
+// The same loop for lists of at most 32 entries per thread (every layer-sized and model-sized
+// table on a full grid): a thread remembers its candidates of an iteration as bit masks, so the
+// rank, the membership of U / D and the apply step walk those bits instead of re-reading the
+// blocks' levels, and nothing per block but the up-rank stamp (read by the down pass) is stored.
+// Dependent L2 round trips per expansion iteration: 3 instead of 8.
+template <int LT, bool CLUSTER>
+__global__ void __launch_bounds__(LT)
+scalebits_loop_masked_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, const double* __restrict__ up_de,
+                             const unsigned* __restrict__ dn_ent, const double* __restrict__ dn_de,
+                             long long ne, LoopWork w) {
+    auto phase_barrier = [&]() {
+        if (CLUSTER) cg::this_cluster().sync();
+        else cg::this_grid().sync();
+    };
+    const int G = gridDim.x, c = blockIdx.x, tid = threadIdx.x;
+    const long long per_cta = (ne + G - 1) / G;
+    const long long ipt = (per_cta + LT - 1) / LT;                    // entries per thread, <= 32
+    const long long cta_hi = min(ne, (long long)(c + 1) * per_cta);
+    const long long t_lo = min(cta_hi, (long long)c * per_cta + (long long)tid * ipt);
+    const long long t_hi = min(cta_hi, t_lo + ipt);
+    const int n_mine = (int)(t_hi - t_lo);
+
+    const AllocState s0 = *a.st;                    // written before the launch
+    const long long cap = s0.cap, kT = s0.kT;
+    long long k = s0.k, used = s0.used;
+    double loss = s0.loss;
+    int iter = 0, accepted = 0, rejected = 0, expansions = 0, status = 0;
+    unsigned flip = 0;
+
+    unsigned dbits = 0;
+#pragma unroll
+    for (int l = 0; l < 7; ++l) dbits |= (unsigned)(a.bits[l + 1] > a.bits[l] ? a.bits[l + 1] - a.bits[l] : 0) << (4 * l);
+    const long long* const block_elems = a.block_elems;
+    const long long uniform = a.uniform;
+    auto cost_of = [&](unsigned e) -> unsigned long long {
+        const long long m = block_elems ? block_elems[e >> 3] : uniform;
+        return (unsigned long long)(m * (long long)((dbits >> (4u * (e & 7u))) & 15u));
+    };
+    constexpr unsigned long long FIRST_NONE = ~0ull;
+
+    while (k >= kT) {
+        if (iter >= 4096) { status = SB_ERR_NOCONVERGE; break; }
+        const unsigned stamp = (unsigned)iter + 1u;
+        const long long slack = cap - used;
+        const long long h = k / 2 > 0 ? k / 2 : 1;
+
+        // ---- up-count: candidate mask, count, cost ----------------------------------------------
+        unsigned cm = 0;
+        CntCost mine{0ull, 0u, 0u};
+        unsigned long long my_first = 0;
+        for (int b0 = 0; b0 < n_mine; b0 += LC) {
+            unsigned e[LC]; int lv[LC];
+#pragma unroll
+            for (int j = 0; j < LC; ++j) e[j] = b0 + j < n_mine ? __ldg(up_ent + t_lo + b0 + j) : ENT_NONE;
+#pragma unroll
+            for (int j = 0; j < LC; ++j) lv[j] = e[j] != ENT_NONE ? (int)__ldcg(a.level + (e[j] >> 3)) : -1;
+#pragma unroll
+            for (int j = 0; j < LC; ++j) {
+                if (lv[j] == (int)(e[j] & 7u)) {
+                    const unsigned long long cost = cost_of(e[j]);
+                    if (mine.cnt == 0) my_first = cost;
+                    mine.cnt += 1; mine.cost += cost;
+                    cm |= 1u << (b0 + j);
+                }
+            }
+        }
+        CntCost cta_tot;
+        const CntCost ex = block_exclusive_scan<CntCost, LT>(mine, cta_tot);
+        if (ex.cnt == 0 && mine.cnt > 0) w.up_first[c] = (long long)my_first;   // the CTA's first candidate
+        if (tid == 0) {
+            w.up_tot[c] = cta_tot;
+            if (cta_tot.cnt == 0) w.up_first[c] = -1;
+        }
+        phase_barrier();
+
+        // ---- prefix over the lower CTAs; cost of the globally first candidate (key = CTA, cost) --
+        unsigned long long pre[3] = {0ull, 0ull, FIRST_NONE};
+        for (int j = tid; j < G; j += LT) {
+            const CntCost t = ldcg_cc(w.up_tot + j);
+            const long long fc = __ldcg(w.up_first + j);
+            if (j < c) { pre[0] += t.cost; pre[1] += t.cnt; }
+            if (t.cnt > 0) {
+                const unsigned long long key = ((unsigned long long)j << 48) | ((unsigned long long)fc & 0xffffffffffffull);
+                if (key < pre[2]) pre[2] = key;
+            }
+        }
+        cta_allreduce<LT, 3, 0 | (0 << 2) | (1 << 4)>(pre, flip);
+        const long long first_cost = pre[2] != FIRST_NONE ? (long long)(pre[2] & 0xffffffffffffull) : -1;
+        const bool expand = used < cap && first_cost >= 0 && first_cost <= slack;
+        const long long lim_rank = expand ? k : h;
+        const unsigned long long base_cost = pre[0] + ex.cost;
+        const long long base_cnt = (long long)pre[1] + ex.cnt;
+
+        // ---- up-rank: in an expansion the set U itself, else the stamps the down pass excludes ----
+        // U is a prefix of the ranked candidates, so its cost is the largest cumulative cost in it
+        double dU_mine = 0.0; unsigned long long costU_mine = 0; unsigned nU_mine = 0;
+        unsigned um = 0;
+        if (cm && base_cnt < lim_rank) {
+            unsigned long long run_cost = base_cost;
+            long long run_cnt = base_cnt;
+            for (unsigned m = cm; m && run_cnt < lim_rank; m &= m - 1) {
+                const int j = __ffs(m) - 1;
+                const unsigned e = __ldg(up_ent + t_lo + j);
+                run_cost += cost_of(e);
+                if (expand) {
+                    if ((long long)run_cost <= slack) {
+                        um |= 1u << j;
+                        dU_mine += __ldg(up_de + t_lo + j); costU_mine = run_cost; nU_mine += 1;
+                    }
+                } else {
+                    a.upsr[e >> 3] = ((unsigned long long)stamp << 32) | (unsigned long long)(unsigned)run_cnt;
+                }
+                run_cnt += 1;
+            }
+        }
+        if (expand) {
+            const double d = cta_sum<LT>(dU_mine);
+            unsigned long long r2[2] = {costU_mine, nU_mine};
+            cta_allreduce<LT, 2, 2 | (0 << 2)>(r2, flip);
+            if (tid == 0) { w.dU[c] = d; w.costU[c] = r2[0]; w.nU[c] = (unsigned)r2[1]; }
+        }
+        phase_barrier();
+
+        unsigned dsel = 0;
+        if (!expand) {
+            // ---- down-count: the step ends at the block's level, the block is not in the up set ----
+            unsigned dcm = 0;
+            CntCost dm{0ull, 0u, 0u};
+            for (int b0 = 0; b0 < n_mine; b0 += LC) {
+                unsigned e[LC]; int lv[LC]; unsigned long long sr[LC];
+#pragma unroll
+                for (int j = 0; j < LC; ++j) e[j] = b0 + j < n_mine ? __ldg(dn_ent + t_lo + b0 + j) : ENT_NONE;
+#pragma unroll
+                for (int j = 0; j < LC; ++j) {
+                    lv[j] = -1; sr[j] = 0ull;
+                    if (e[j] != ENT_NONE) {
+                        lv[j] = (int)__ldcg(a.level + (e[j] >> 3));
+                        sr[j] = __ldcg(a.upsr + (e[j] >> 3));
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < LC; ++j) {
+                    if (lv[j] != (int)(e[j] & 7u) + 1) continue;
+                    if ((unsigned)(sr[j] >> 32) == stamp && (long long)(unsigned)sr[j] < h) continue;
+                    dm.cnt += 1; dm.cost += cost_of(e[j]);
+                    dcm |= 1u << (b0 + j);
+                }
+            }
+            CntCost dn_cta;
+            const CntCost dex = block_exclusive_scan<CntCost, LT>(dm, dn_cta);
+            if (tid == 0) w.dn_tot[c] = dn_cta;
+            phase_barrier();
+            unsigned long long dpre[1] = {0ull};
+            for (int j = tid; j < c; j += LT) dpre[0] += ldcg_cc(w.dn_tot + j).cnt;
+            cta_allreduce<LT, 1, 0>(dpre, flip);
+            // ---- down-rank: the first h candidates form D -----------------------------------------
+            double dD_mine = 0.0; unsigned long long freed_mine = 0; unsigned nD_mine = 0;
+            long long run_cnt = (long long)dpre[0] + dex.cnt;
+            for (unsigned m = dcm; m && run_cnt < h; m &= m - 1, ++run_cnt) {
+                const int j = __ffs(m) - 1;
+                const unsigned e = __ldg(dn_ent + t_lo + j);
+                dsel |= 1u << j;
+                dD_mine += __ldg(dn_de + t_lo + j); freed_mine += cost_of(e); nD_mine += 1;
+            }
+            {
+                const double d = cta_sum<LT>(dD_mine);
+                unsigned long long r2[2] = {freed_mine, nD_mine};
+                cta_allreduce<LT, 2, 0>(r2, flip);
+                if (tid == 0) { w.dD[c] = d; w.freed[c] = r2[0]; w.nD[c] = (unsigned)r2[1]; }
+            }
+            phase_barrier();
+            // ---- U: up-candidates 0..h-1 whose cumulative cost fits slack + what D frees ------------
+            unsigned long long fr[1] = {0ull};
+            for (int j = tid; j < G; j += LT) fr[0] += __ldcg(w.freed + j);
+            cta_allreduce<LT, 1, 0>(fr, flip);
+            const long long lim_cost = slack + (long long)fr[0];
+            if (cm && base_cnt < h) {
+                unsigned long long run_cost = base_cost;
+                long long rank = base_cnt;
+                for (unsigned m = cm; m && rank < h; m &= m - 1, ++rank) {
+                    const int j = __ffs(m) - 1;
+                    run_cost += cost_of(__ldg(up_ent + t_lo + j));
+                    if ((long long)run_cost > lim_cost) break;      // cumulative costs only grow
+                    um |= 1u << j;
+                    dU_mine += __ldg(up_de + t_lo + j); costU_mine = run_cost; nU_mine += 1;
+                }
+            }
+            const double d = cta_sum<LT>(dU_mine);
+            unsigned long long r2[2] = {costU_mine, nU_mine};
+            cta_allreduce<LT, 2, 2 | (0 << 2)>(r2, flip);
+            if (tid == 0) { w.dU[c] = d; w.costU[c] = r2[0]; w.nU[c] = (unsigned)r2[1]; }
+            phase_barrier();
+        }
+
+        // ---- totals (same order in every CTA), decision, apply, replicated state update -----------
+        __shared__ double sh_dU, sh_dD;
+        if (tid == 0) {
+            double u = 0.0, dsum = 0.0;
+            for (int j = 0; j < G; ++j) u += __ldcg(w.dU + j);
+            if (!expand) for (int j = 0; j < G; ++j) dsum += __ldcg(w.dD + j);
+            sh_dU = u; sh_dD = dsum;
+        }
+        unsigned long long tot[4] = {0ull, 0ull, 0ull, 0ull};       // costU (max), nU, freed, nD
+        for (int j = tid; j < G; j += LT) {
+            const unsigned long long cu = __ldcg(w.costU + j);
+            if (cu > tot[0]) tot[0] = cu;
+            tot[1] += __ldcg(w.nU + j);
+            if (!expand) { tot[2] += __ldcg(w.freed + j); tot[3] += __ldcg(w.nD + j); }
+        }
+        cta_allreduce<LT, 4, 2 | (0 << 2) | (0 << 4) | (0 << 6)>(tot, flip);
+        const unsigned long long costU = tot[0], freed = tot[2];
+        const unsigned nU = (unsigned)tot[1], nD = (unsigned)tot[3];
+        const double dU = sh_dU, dD = sh_dD;
+        const bool accept = expand ? (nU > 0) : (nU > 0 && nD > 0 && dU > dD);
+        if (accept) {
+            // the owner of a list entry knows the block and its new level: no loads
+            for (unsigned m = um; m; m &= m - 1) {
+                const unsigned e = __ldg(up_ent + t_lo + (__ffs(m) - 1));
+                a.level[e >> 3] = (unsigned char)((e & 7u) + 1u);
+            }
+            for (unsigned m = dsel; m; m &= m - 1) {
+                const unsigned e = __ldg(dn_ent + t_lo + (__ffs(m) - 1));
+                a.level[e >> 3] = (unsigned char)(e & 7u);
+            }
+        }
+        if (expand && accept) { used += (long long)costU; loss -= dU; expansions += 1; }
+        else if (accept) { used += (long long)costU - (long long)freed; loss += dD - dU; accepted += 1; }
+        else { k /= 2; rejected += 1; }
+        iter += 1;
+        phase_barrier();                                  // the new levels are visible to the next up-count
+    }
+    if (c == 0 && tid == 0) {
+        AllocState* st = a.st;
+        st->k = k; st->used = used; st->loss = loss; st->iter = iter; st->accepted = accepted;
+        st->rejected = rejected; st->expansions = expansions; st->done = 1; st->status = status;
+    }
+}
+
 // ---- Algorithm 1 ---------------------------------------------------------------------------
 // Hull steps of block i from level 0: the next vertex is the level of strictly lower error with
 // the steepest slope (exact ties: the farthest).  Entry e = i (L-1) + (q-1) describes the step
@@ -734,12 +972,8 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
             // barrier is several times cheaper than a grid-wide one, and a handful of list
             // entries per thread is all the parallelism the passes need.
             if (nsteps <= (long long)CL_CTAS * CL_THREADS * 16) {
-                auto kern = scalebits_loop_kernel<CL_THREADS, true>;
-                static bool attr_done = false;
-                if (!attr_done) {
-                    SB_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-                    attr_done = true;
-                }
+                auto kern = scalebits_loop_masked_kernel<CL_THREADS, true>;       // <= 16 entries per thread
+                SB_FUNC_ATTR(ctx, kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
                 cudaLaunchConfig_t cfg = {};
                 cfg.gridDim = dim3(CL_CTAS);
                 cfg.blockDim = dim3(CL_THREADS);
@@ -755,17 +989,28 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
             if (!launched) {
                 // the whole loop in one cooperative launch
                 auto kern = scalebits_loop_kernel<GL_THREADS, false>;
-                int occ = 0;
+                auto kern_masked = scalebits_loop_masked_kernel<GL_THREADS, false>;
+                int occ = 0, occ_m = 0;
                 SB_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, GL_THREADS, 0));
-                long long G = (long long)occ * ctx->sm_count;
-                // a few list entries per thread: grid barriers cost more with more CTAs than the
-                // short passes gain
-                const long long want = (nsteps + LC * GL_THREADS - 1) / (LC * GL_THREADS);
-                if (G > want) G = want;
-                if (G > LOOP_MAX_CTAS) G = LOOP_MAX_CTAS;
-                if (G < 1) G = 1;
-                SB_CUDA(ctx, cudaLaunchCooperativeKernel((const void*)kern, dim3((unsigned)G), dim3(GL_THREADS),
-                                                         kargs, 0, ctx->stream));
+                SB_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_m, kern_masked, GL_THREADS, 0));
+                auto grid_for = [&](int o) {
+                    long long G = (long long)o * ctx->sm_count;
+                    // a few list entries per thread: grid barriers cost more with more CTAs than
+                    // the short passes gain
+                    const long long want = (nsteps + LC * GL_THREADS - 1) / (LC * GL_THREADS);
+                    if (G > want) G = want;
+                    if (G > LOOP_MAX_CTAS) G = LOOP_MAX_CTAS;
+                    if (G < 1) G = 1;
+                    return G;
+                };
+                // the masked form needs at most 32 list entries per thread
+                long long G = grid_for(occ_m);
+                const long long per_cta = (nsteps + G - 1) / G;
+                const bool masked = (per_cta + GL_THREADS - 1) / GL_THREADS <= 32;
+                if (!masked) G = grid_for(occ);
+                SB_CUDA(ctx, cudaLaunchCooperativeKernel(masked ? (const void*)kern_masked : (const void*)kern,
+                                                         dim3((unsigned)G), dim3(GL_THREADS), kargs, 0,
+                                                         ctx->stream));
             }
             ctx->launches++;
         }

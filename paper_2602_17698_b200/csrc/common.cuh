@@ -1,5 +1,6 @@
 // Shared host/device helpers of the CUDA library (sm_100a only).
 #pragma once
+#include <set>
 #include <vector>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -23,6 +24,7 @@ struct sb_ctx {
     void* scratch = nullptr;     // arena, grown on demand
     size_t scratch_bytes = 0;
     std::vector<void*> retired;  // outgrown arenas and descriptor buffers, freed with the context
+    std::set<const void*> configured;   // kernels whose launch attributes this context has set
     SbDeviceState* dstate = nullptr;
     void* pinned = nullptr;      // small pinned host buffer for read-backs
     size_t pinned_bytes = 0;
@@ -42,6 +44,16 @@ sb_status sb_scratch(sb_ctx* ctx, size_t bytes, void** out);   // whole arena, >
         cudaError_t e__ = (call);                                                       \
         if (e__ != cudaSuccess)                                                         \
             return sb_fail((ctx), SB_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e__)); \
+    } while (0)
+
+// one-time launch attribute of a kernel, per context (so per device), not per process
+#define SB_FUNC_ATTR(ctx, func, attr, value)                                            \
+    do {                                                                                \
+        const void* f__ = reinterpret_cast<const void*>(func);                          \
+        if (!(ctx)->configured.count(f__)) {                                            \
+            SB_CUDA((ctx), cudaFuncSetAttribute(f__, (attr), (value)));                 \
+            (ctx)->configured.insert(f__);                                              \
+        }                                                                               \
     } while (0)
 
 #define SB_LAUNCHED(ctx)                                                                \

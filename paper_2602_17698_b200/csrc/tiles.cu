@@ -788,11 +788,7 @@ sb_status launch_scores_k(sb_ctx* ctx, const __nv_bfloat16* W, int64_t ldw, cons
     const size_t smem = (size_t)SC_WARPS * RING * SLAB_BYTES;
     using P = ScorePolicy<L, RPL, NFINE, FULLG, ROWW>;
     auto kern = slab_walk_kernel<P>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        SB_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_done = true;
-    }
+    SB_FUNC_ATTR(ctx, kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     typename P::Args pa{cperm, cm, ba, rec};
     kern<<<(unsigned)grid, SC_THREADS, smem, ctx->stream>>>(W, ldw, lrp, aperm, rw, g, pa);
     SB_LAUNCHED(ctx);
@@ -828,24 +824,15 @@ sb_status sb_gather_bf16(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64
                          const int32_t* rp, const int32_t* cp, void* out) {
     const size_t smem = (size_t)C * 2 * GA_STAGES;  // a ring of row buffers
     if (smem > 200 * 1024) return sb_fail(ctx, SB_ERR_SHAPE, "gather: rows longer than 34133 columns");
-    static bool attr_set = false;
-    if (!attr_set) {
-        SB_CUDA(ctx, cudaFuncSetAttribute(gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          200 * 1024));
-        attr_set = true;
-    }
+    SB_FUNC_ATTR(ctx, gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     int rows_per_cta = 8;
     const unsigned grid = (unsigned)((R + rows_per_cta - 1) / rows_per_cta);
     auto* Wb = static_cast<const __nv_bfloat16*>(W);
     auto* ob = static_cast<__nv_bfloat16*>(out);
 #define SB_GATHER_COLS(NIT)                                                                          \
     do {                                                                                             \
-        static bool attr_cols = false;                                                               \
-        if (!attr_cols) {                                                                            \
-            SB_CUDA(ctx, cudaFuncSetAttribute(gather_cols_kernel<NIT>,                               \
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)); \
-            attr_cols = true;                                                                        \
-        }                                                                                            \
+        SB_FUNC_ATTR(ctx, gather_cols_kernel<NIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+                     200 * 1024);                                                                    \
         gather_cols_kernel<NIT><<<grid, CTA_THREADS, smem, ctx->stream>>>(Wb, R, (int)C, ldw, rp, cp, ob, \
                                                                           rows_per_cta);            \
     } while (0)
