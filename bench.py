@@ -192,6 +192,73 @@ FULL_MODEL_BUDGETS = tuple(2.0 + 0.25 * i for i in range(9))          # 2.0 ... 
 FULL_MODEL_SUPER = {3: 101, 12: 102, 20: 103, 29: 104}                # layer -> seed of its super weight
 
 
+def kernel_rooflines(ctx, W, moments, dev, peak_gbs, sm_mhz):
+    """The other kernels of the path, one library call at a time on 14336 x 4096 matrices (three
+    different ones in rotation, 352 MB > L2, so every call streams from HBM), CUDA events on the
+    context's stream.  HBM-bound kernels against the measured copy bandwidth; the score kernel
+    against the FP32 pipe: 148 SMs x 128 lanes x SM clock lane-operations per second, with
+    4 L + 1 + (candidates of >= 6 bits) algorithmic lane-operations per weight."""
+    import torch
+    mats = [W["gate_proj"], W["up_proj"], W["gate_proj"].clone()]
+    c = moments["mlp_in"]
+    R, Cc = mats[0].shape
+    n = R * Cc
+    nb = (R // 128) * (Cc // 128)
+    f32 = dict(dtype=torch.float32, device=dev)
+    rs, cs = torch.empty(R, **f32), torch.empty(Cc, **f32)
+    err = torch.empty(nb, len(BITS), **f32)
+    out = torch.empty_like(mats[0])
+    gen = torch.Generator(device=dev).manual_seed(SEED)
+    pr = torch.randperm(R, device=dev, generator=gen).int()
+    pc = torch.randperm(Cc, device=dev, generator=gen).int()
+    level = torch.randint(0, len(BITS), (nb,), device=dev, dtype=torch.uint8, generator=gen)
+    packed = torch.empty(n * max(BITS) // 32, dtype=torch.int32, device=dev)
+    off = torch.empty(nb + 1, dtype=torch.int64, device=dev)
+    meta = torch.empty((n // 128, 2), **f32)
+
+    def timed(fn, reps=9):
+        for i in range(3):
+            fn(mats[i % 3])
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(reps):
+            fn(mats[i % 3])
+        b.record()
+        b.synchronize()
+        return a.elapsed_time(b) / reps
+
+    t_stats = timed(lambda m: ctx.reorder_channels(m, c, 2, 128, row_score=rs, col_score=cs))
+    t_score = timed(lambda m: ctx.block_scores(m, c, BITS, 128, 128, 128, err=err, want_gain=False))
+    t_perm = timed(lambda m: ctx.block_scores(m, c, BITS, 128, 128, 128, row_perm=pr, col_perm=pc, err=err,
+                                              want_gain=False, W_perm_out=out))
+    t_pack = timed(lambda m: ctx.pack_blocks(m, BITS, level, 128, 128, 128, packed=packed, block_off=off,
+                                             meta=meta))
+    t_gather = max(t_perm - t_score, 1e-6)
+    avg_bits = sum(BITS) / len(BITS)
+
+    def hbm(name, bytes_, ms, note):
+        a = bytes_ / (ms * 1e-3) / 1e9
+        return {"kernel": name, "bound": "hbm", "achieved": a, "peak": peak_gbs, "unit": "GB/s",
+                "frac": a / peak_gbs, "ms_per_call": ms, "algorithmic_bytes": bytes_, "note": note}
+
+    fine = sum(1 for b in BITS if b >= 6)
+    ops = 4 * len(BITS) + 1 + fine
+    alu_peak = 148 * 128 * sm_mhz * 1e6 / 1e12
+    a_ops = n * ops / (t_score * 1e-3) / 1e12
+    return [
+        hbm("reorder_stats_kernel", 2 * n, t_stats, "one call of sb_reorder_channels (statistics only)"),
+        {"kernel": "slab_walk_kernel<ScorePolicy> (+ scores_finish_kernel)", "bound": "alu", "achieved": a_ops,
+         "peak": alu_peak, "unit": "T fp32 lane-ops/s", "frac": a_ops / alu_peak, "ms_per_call": t_score,
+         "lane_ops_per_weight": ops, "hbm_gbs": 2 * n / (t_score * 1e-3) / 1e9,
+         "hbm_frac": 2 * n / (t_score * 1e-3) / 1e9 / peak_gbs,
+         "note": "one call of sb_block_scores without permutations; peak = 148 SMs x 128 lanes x SM clock"},
+        hbm("gather_cols_kernel", 4 * n, t_gather,
+            "sb_block_scores with both permutations and W_perm_out minus the call without (2 B read + 2 B written)"),
+        hbm("pack_offsets_small_kernel + pack_kernel", int(2 * n + n * avg_bits / 8 + n / 128 * 8), t_pack,
+            "one call of sb_pack_blocks, uniformly random levels (2 B read + codes + metadata written)"),
+    ]
+
+
 def full_model_times(ctx, dev):
     """configs[2]: 32 layers of the 8B shape searched as ONE model (residual-stream permutation
     shared by all layers, one global allocation over N = 425,984 blocks per budget), budgets
@@ -365,6 +432,8 @@ def run_cuda(args):
                      "reorder_stats": w_bytes / (stage_ms["reorder_stats"] * 1e-3) / 1e9,
                      "scores": w_bytes / (stage_ms["scores"] * 1e-3) / 1e9,
                      "pack": w_bytes / (stage_ms["pack"] * 1e-3) / 1e9}
+        sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
+        kernels = kernel_rooflines(ctx, W, ws.moments, dev, peak, sm_mhz)
         full_model = None
         if world == 1 and not args.no_full_model:
             del hW, hX                                   # pinned copies of the layer, if any
@@ -386,7 +455,7 @@ def run_cuda(args):
                 "roofline": roofline, "cpu_baseline": cpu,
                 "stages_ms_per_step": stage_ms, "stages_algorithmic_gbs": stage_gbs,
                 "scoring_elements_per_s": n_weights / (stage_ms["scores"] * 1e-3),
-                "full_model": full_model}
+                "roofline_other_kernels": kernels, "full_model": full_model}
         print(json.dumps(line), flush=True)
     ctx.close()
     if world > 1:
