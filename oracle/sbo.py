@@ -241,3 +241,50 @@ def pack_blocks(W, bits: Sequence[int], level, block_rows=128, block_cols=128, g
     if st != OK:
         raise ValueError(f"sbo_pack_blocks status {st}")
     return packed[:off[nb]].copy(), off, meta
+
+
+class StepReport(C.Structure):
+    _fields_ = [("cap_bits", C.c_int64), ("used_in", C.c_int64), ("used_out", C.c_int64),
+                ("expansion", C.c_int32), ("moved", C.c_int32),
+                ("n_up", C.c_int64), ("n_down", C.c_int64),
+                ("sum_up", C.c_double), ("sum_down", C.c_double)]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+def first_order_scores(W, G, bits: Sequence[int], level, block_rows=128, block_cols=128, group=128,
+                       row_perm=None, col_perm=None):
+    """-> (s_up[nb], s_down[nb], s_l1[nb]) of every block at its current level (Appendix E.3)."""
+    W, G = _u16(W), _u16(G)
+    assert W.shape == G.shape
+    R, Cc = W.shape
+    rp, cp = _i32(row_perm), _i32(col_perm)
+    barr, L = _bits(bits)
+    level = np.ascontiguousarray(level, dtype=np.uint8)
+    nb = (R // block_rows) * (Cc // block_cols)
+    assert level.size == nb
+    up, down, l1 = (np.zeros(nb, dtype=np.float64) for _ in range(3))
+    st = lib().sbo_first_order_scores(_p(W), _p(G), C.c_int64(R), C.c_int64(Cc), C.c_int64(Cc), C.c_int64(Cc),
+                                      _p(rp), _p(cp), C.c_int(block_rows), C.c_int(block_cols),
+                                      C.c_int(group), barr, C.c_int(L), _p(level), _p(up), _p(down), _p(l1))
+    if st != OK:
+        raise ValueError(f"sbo_first_order_scores status {st}")
+    return up, down, l1
+
+
+def exchange_step(s_up, s_down, level, bits: Sequence[int], budget: float, k: int,
+                  uniform_block_elems=128 * 128, block_elems=None):
+    """One iteration of Algorithm 2 on given scores -> (status, level_out, report dict)."""
+    s_up, s_down = _f64(s_up), _f64(s_down)
+    level = np.ascontiguousarray(level, dtype=np.uint8)
+    N = level.size
+    assert s_up.size == N and s_down.size == N
+    barr, L = _bits(bits)
+    be = None if block_elems is None else np.ascontiguousarray(block_elems, dtype=np.int64)
+    out = np.zeros(N, dtype=np.uint8)
+    rep = StepReport()
+    st = lib().sbo_exchange_step(_p(s_up), _p(s_down), _p(level), C.c_int64(N), _p(be),
+                                 C.c_int64(uniform_block_elems), barr, C.c_int(L), C.c_double(budget),
+                                 C.c_int64(k), _p(out), C.byref(rep))
+    return int(st), out, rep.as_dict()

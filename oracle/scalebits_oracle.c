@@ -29,6 +29,9 @@
  *     round-half-to-even.
  *   - Algorithm 1 (classic greedy) and Algorithm 2 (scalable greedy) on the
  *     separable proxy loss L(b) = sum_i E[i][level_i].
+ *   - Appendix E.3: the paper's own first-order scores s_up / s_down from a caller's
+ *     gradient, and one iteration of Algorithm 2 on such scores
+ *     (sbo_first_order_scores, sbo_exchange_step).
  *
  * Parity pins: see tests/test_oracle_*.py.  The exact trajectory of
  * sbo_allocate_scalebits (tie rules, odd k, budget truncation) is a reading of
@@ -535,6 +538,171 @@ int sbo_allocate_scalebits(const double* err, int64_t N, const int64_t* block_el
     rep->used_bits = used; rep->proxy_loss_final = loss;
     fill_report(rep, level, N);
     return status;
+}
+
+/* ---- first-order statistics of the current allocation (Appendix E.3) --------- */
+/* The paper's own scores for Algorithm 2: with g = dL/dw evaluated at the current quantized
+ * model and every block i quantized at ITS current bitwidth b = bits[level[i]],
+ *   s_up[i]   = - sum over block i of G (W' - Q_b(W'))     (first-order loss decrease of moving
+ *                                                            the block back to full precision;
+ *                                                            the paper prints g^T (w - w^Q) and
+ *                                                            ranks the LARGEST first, so the gain
+ *                                                            is read with the minus sign)
+ *   s_down[i] = 2^-b * sum over block i of |G * Q_b(W')|   (expected magnitude of the increase)
+ *   s_l1[i]   = sum over block i of |G (W' - Q_b(W'))|     (the p = 1 element sensitivity of
+ *                                                            Section 3.2, summed: the scale the
+ *                                                            signed sum is compared at)
+ * on the permuted layout, W' = W[rp][:, cp], G' = G[rp][:, cp].                              */
+int sbo_first_order_scores(const uint16_t* W, const uint16_t* G, int64_t R, int64_t C, int64_t ldw,
+                           int64_t ldg, const int32_t* row_perm, const int32_t* col_perm,
+                           int br, int bc, int group, const int* bits, int L, const uint8_t* level,
+                           double* s_up, double* s_down, double* s_l1) {
+    if (!check_bits(bits, L)) return SBO_ERR_INVALID;
+    if (br <= 0 || bc <= 0 || group <= 0 || R % br || C % bc || bc % group) return SBO_ERR_SHAPE;
+    const int64_t nbr = R / br, nbc = C / bc;
+    for (int64_t blk = 0; blk < nbr * nbc; ++blk)
+        if (level[blk] >= L) return SBO_ERR_INVALID;
+    #pragma omp parallel
+    {
+        double* v = (double*)malloc(sizeof(double) * group);
+        double* vh = (double*)malloc(sizeof(double) * group);
+        #pragma omp for schedule(dynamic, 1)
+        for (int64_t blk = 0; blk < nbr * nbc; ++blk) {
+            const int64_t bi = blk / nbc, bj = blk % nbc;
+            const int b = bits[level[blk]];
+            double up = 0.0, down = 0.0, l1 = 0.0;
+            for (int rr = 0; rr < br; ++rr) {
+                const int64_t r = bi * br + rr;
+                const int64_t rs = row_perm ? row_perm[r] : r;
+                for (int g0 = 0; g0 < bc; g0 += group) {
+                    for (int k = 0; k < group; ++k) {
+                        const int64_t j = bj * bc + g0 + k;
+                        const int64_t js = col_perm ? col_perm[j] : j;
+                        v[k] = sbo_bf16_to_f64(W[rs * ldw + js]);
+                    }
+                    sbo_quantize_group(v, group, b, NULL, vh, NULL, NULL);
+                    for (int k = 0; k < group; ++k) {
+                        const int64_t j = bj * bc + g0 + k;
+                        const int64_t js = col_perm ? col_perm[j] : j;
+                        const double g = sbo_bf16_to_f64(G[rs * ldg + js]);
+                        const double t = g * (v[k] - vh[k]);
+                        up -= t;
+                        l1 += fabs(t);
+                        down += fabs(g * vh[k]);
+                    }
+                }
+            }
+            s_up[blk] = up;
+            s_down[blk] = ldexp(down, -b);
+            if (s_l1) s_l1[blk] = l1;
+        }
+        free(v); free(vh);
+    }
+    return SBO_OK;
+}
+
+/* ---- one iteration of Algorithm 2 on caller-supplied scores ------------------- */
+/* Lines 6-10 of Algorithm 2 with s_up / s_down given per block AT ITS CURRENT LEVEL (they change
+ * with the model, so the caller refreshes them and decides on acceptance, line 11, itself).
+ * Same readings as sbo_allocate_scalebits: one move = one level of the candidate list; ranking
+ * keys per stored bit, s / ((b' - b) M_i), ties to the lower block; up-eligible: not at the
+ * top level and s_up > 0; down-eligible: not at the bottom level; the expansion is truncated
+ * to the longest prefix that fits the budget and, if nothing fits, the exchange runs instead;
+ * the up set is chosen first and the down set excludes it; U is the longest prefix of the up
+ * set whose cost fits the slack plus what D frees.  An exchange with an empty U or D moves
+ * nothing.                                                                                    */
+typedef struct {
+    int64_t cap_bits, used_in, used_out;
+    int32_t expansion;          /* 1: expansion step, 0: exchange step                          */
+    int32_t moved;              /* 0: nothing fits / nothing eligible: level_out == level       */
+    int64_t n_up, n_down;
+    double sum_up, sum_down;    /* first-order change promised: -sum_up + sum_down              */
+} sbo_step_report;
+
+int sbo_exchange_step(const double* s_up, const double* s_down, const uint8_t* level, int64_t N,
+                      const int64_t* block_elems, int64_t uniform, const int* bits, int L,
+                      double budget, int64_t k, uint8_t* level_out, sbo_step_report* rep) {
+    if (!check_bits(bits, L) || N <= 0 || k < 1) return SBO_ERR_INVALID;
+    memset(rep, 0, sizeof *rep);
+    const int64_t cap = budget_cap(budget, block_elems, uniform, N);
+    int64_t used = 0;
+    for (int64_t i = 0; i < N; ++i) {
+        if (level[i] >= L) return SBO_ERR_INVALID;
+        used += blk_elems(block_elems, uniform, i) * bits[level[i]];
+        level_out[i] = level[i];
+    }
+    rep->cap_bits = cap; rep->used_in = used; rep->used_out = used;
+    rank_item* up = (rank_item*)malloc(sizeof(rank_item) * (size_t)N);
+    rank_item* dn = (rank_item*)malloc(sizeof(rank_item) * (size_t)N);
+    char* in_up = (char*)calloc((size_t)N, 1);
+    int64_t nu = 0, nd = 0;
+    for (int64_t i = 0; i < N; ++i) {
+        const int l = level[i];
+        const double M = (double)blk_elems(block_elems, uniform, i);
+        if (l + 1 < L && s_up[i] > 0.0) {
+            up[nu].key = s_up[i] / ((double)(bits[l + 1] - bits[l]) * M);
+            up[nu].i = i; ++nu;
+        }
+    }
+    qsort(up, (size_t)nu, sizeof(rank_item), cmp_key_desc);
+    const int64_t slack = cap - used;
+    if (used < cap) {                                   /* expansion stage */
+        int64_t cum = 0, taken = 0;
+        for (int64_t p = 0; p < nu && p < k; ++p) {
+            const int64_t i = up[p].i; const int l = level[i];
+            const int64_t cost = blk_elems(block_elems, uniform, i) * (bits[l + 1] - bits[l]);
+            if (cum + cost > slack) break;
+            cum += cost; ++taken;
+            level_out[i] = (uint8_t)(l + 1);
+            rep->sum_up += s_up[i];
+        }
+        if (taken > 0) {
+            rep->expansion = 1; rep->moved = 1; rep->n_up = taken; rep->used_out = used + cum;
+            free(up); free(dn); free(in_up);
+            return SBO_OK;
+        }
+    }
+    /* exchange stage */
+    const int64_t h = k / 2 > 0 ? k / 2 : 1;
+    const int64_t nu0 = nu < h ? nu : h;
+    for (int64_t p = 0; p < nu0; ++p) in_up[up[p].i] = 1;
+    for (int64_t i = 0; i < N; ++i) {
+        const int l = level[i];
+        if (l > 0 && !in_up[i]) {
+            const double M = (double)blk_elems(block_elems, uniform, i);
+            dn[nd].key = s_down[i] / ((double)(bits[l] - bits[l - 1]) * M);
+            dn[nd].i = i; ++nd;
+        }
+    }
+    qsort(dn, (size_t)nd, sizeof(rank_item), cmp_key_asc);
+    const int64_t nd0 = nd < h ? nd : h;
+    int64_t freed = 0;
+    for (int64_t p = 0; p < nd0; ++p) {
+        const int64_t i = dn[p].i; const int l = level[i];
+        freed += blk_elems(block_elems, uniform, i) * (bits[l] - bits[l - 1]);
+    }
+    int64_t cum = 0, taken = 0;
+    for (int64_t p = 0; p < nu0; ++p) {
+        const int64_t i = up[p].i; const int l = level[i];
+        const int64_t cost = blk_elems(block_elems, uniform, i) * (bits[l + 1] - bits[l]);
+        if (cum + cost > slack + freed) break;
+        cum += cost; ++taken;
+    }
+    if (taken > 0 && nd0 > 0) {
+        for (int64_t p = 0; p < taken; ++p) {
+            const int64_t i = up[p].i;
+            level_out[i] = (uint8_t)(level[i] + 1);
+            rep->sum_up += s_up[i];
+        }
+        for (int64_t p = 0; p < nd0; ++p) {
+            const int64_t i = dn[p].i;
+            level_out[i] = (uint8_t)(level[i] - 1);
+            rep->sum_down += s_down[i];
+        }
+        rep->moved = 1; rep->n_up = taken; rep->n_down = nd0; rep->used_out = used + cum - freed;
+    }
+    free(up); free(dn); free(in_up);
+    return SBO_OK;
 }
 
 /* ---- packing (Section 5.3: uniform bitwidth per tile) ----------------------- */
