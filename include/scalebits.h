@@ -170,6 +170,55 @@ sb_status sb_pack_blocks(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_t C, 
                          uint32_t* packed, int64_t packed_capacity_words,
                          int64_t* block_off_words, float* meta);
 
+/* First-order mode (Appendix E.3, "choice of sensitivity statistics"): the paper's own scores
+ * for Algorithm 2 from a caller-supplied gradient G = dL/dw taken at the current quantized
+ * model.  Every block is quantized at ITS current bitwidth b = bits[level[block]] on the
+ * permuted layout W' = W[row_perm][:, col_perm], G' likewise:
+ *     s_up[i]   = - sum over block i of G' (W' - Q_b(W'))      (gain of restoring the block; the
+ *                                                               paper prints g^T (w - w^Q) and
+ *                                                               ranks the largest first)
+ *     s_down[i] = 2^-b * sum over block i of |G' Q_b(W')|
+ *     s_l1[i]   = sum over block i of |G' (W' - Q_b(W'))|      (p = 1 element sensitivities of
+ *                                                               Section 3.2, summed; optional)
+ *   - W, G: device bf16 [R][C] row-major, leading dimensions ldw / ldg (multiples of 8,
+ *     16-byte aligned bases); level: device uint8 [(R/br)*(C/bc)], blocks row-major over the
+ *     grid; s_up, s_down, s_l1 (or NULL): device fp32 of the same length.
+ *   - Shapes as sb_block_scores (group in {16,32,64,128} dividing block_cols, block_rows % 4
+ *     == 0, block_cols in {32, 64} or a multiple of 128, C % 128 == 0).
+ *   - fp32 accumulation: compare the signed sum at the scale of s_l1.  Non-finite sums latch
+ *     SB_ERR_NONFINITE, a level >= n_bits latches SB_ERR_INVALID.  Asynchronous.             */
+sb_status sb_first_order_scores(sb_ctx* ctx, const void* W_bf16, const void* G_bf16, int64_t R,
+                                int64_t C, int64_t ldw, int64_t ldg, const int32_t* row_perm,
+                                const int32_t* col_perm, int block_rows, int block_cols, int group,
+                                const int* bits, int n_bits, const uint8_t* level, float* s_up,
+                                float* s_down, float* s_l1);
+
+/* One iteration of Algorithm 2 (lines 6-10) on per-block scores AT THE CURRENT LEVELS; the
+ * caller refreshes the scores, evaluates the loss of level_out and decides on acceptance
+ * (line 11) itself.  Rules as in sb_allocate_bits: one move = one level of the candidate list;
+ * ranking keys per stored bit, s / ((b' - b) M_i) as a binary64 quotient of the fp32 scores,
+ * ties to the lower block; up-eligible: not at the top level and s_up > 0; down-eligible:
+ * not at the bottom level.  If the budget is not used up, the first k up-candidates are
+ * raised, truncated to the longest prefix that fits (expansion); if nothing fits, or the
+ * budget is used up, the first h = max(1, k/2) up-candidates and the first h down-candidates
+ * outside that set are exchanged, the up set truncated to what the freed bits and the slack
+ * pay for; an exchange with an empty side moves nothing.
+ *   - s_up, s_down: device fp32 [N]; level, level_out: device uint8 [N] (may be the same
+ *     buffer); block_elems: device int64 [N] or NULL with uniform_block_elems; budget in
+ *     average code bits per weight; report: HOST memory, filled after an internal stream
+ *     synchronisation (this call is synchronous).                                          */
+typedef struct {
+    int64_t cap_bits, used_in, used_out;
+    int32_t expansion;      /* 1: expansion step, 0: exchange step                         */
+    int32_t moved;          /* 0: level_out == level (nothing eligible or nothing fits)    */
+    int64_t n_up, n_down;
+    double sum_up, sum_down;    /* first-order change promised: sum_down - sum_up          */
+} sb_step_report;
+sb_status sb_exchange_step(sb_ctx* ctx, const float* s_up, const float* s_down, const uint8_t* level,
+                           int64_t N, const int64_t* block_elems, int64_t uniform_block_elems,
+                           const int* bits, int n_bits, double budget_avg_bits, int64_t k,
+                           uint8_t* level_out, sb_step_report* report);
+
 /* Allocation-free variant of sb_calib_moments (the paper has no counterpart: this entry
  * point exists for deployment, not for the method).  It is for callers that cannot allocate
  * device memory when they need the moments: a serving process whose device memory was

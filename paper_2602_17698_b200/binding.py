@@ -23,7 +23,7 @@ SB_ACC_ROW, SB_ACC_COL = 1, 2
 EXPORTS = ["sb_create", "sb_destroy", "sb_sync", "sb_last_error", "sb_kernel_launches",
            "sb_calib_moments", "sb_reorder_channels", "sb_fold_segment_scores",
            "sb_expand_segment_perm", "sb_block_scores", "sb_allocate_bits", "sb_pack_blocks",
-           "sb_calib_moments_noalloc"]
+           "sb_calib_moments_noalloc", "sb_first_order_scores", "sb_exchange_step"]
 
 
 class SbError(RuntimeError):
@@ -46,6 +46,16 @@ class AllocReport(C.Structure):
                 "proxy_loss_init": self.proxy_loss_init,
                 "proxy_loss_final": self.proxy_loss_final,
                 "level_hist": list(self.level_hist)}
+
+
+class StepReport(C.Structure):
+    _fields_ = [("cap_bits", C.c_int64), ("used_in", C.c_int64), ("used_out", C.c_int64),
+                ("expansion", C.c_int32), ("moved", C.c_int32),
+                ("n_up", C.c_int64), ("n_down", C.c_int64),
+                ("sum_up", C.c_double), ("sum_down", C.c_double)]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
 
 
 _lib = None
@@ -79,6 +89,11 @@ def lib() -> C.CDLL:
                                        f64, f64, vp, C.POINTER(AllocReport)]
         L.sb_pack_blocks.argtypes = [vp, vp, i64, i64, i64, vp, vp, i32, i32, i32,
                                      C.POINTER(C.c_int), i32, vp, vp, i64, vp, vp]
+        L.sb_first_order_scores.argtypes = [vp, vp, vp, i64, i64, i64, i64, vp, vp, i32, i32, i32,
+                                            C.POINTER(C.c_int), i32, vp, vp, vp, vp]
+        L.sb_exchange_step.argtypes = [vp, vp, vp, vp, i64, vp, i64, C.POINTER(C.c_int), i32, f64, i64,
+                                       vp, C.POINTER(StepReport)]
+        L.sb_calib_moments_noalloc.argtypes = [vp, vp, i64, i64, i64, vp, i32, f32]
         for name in EXPORTS:
             if name not in ("sb_last_error", "sb_kernel_launches"):
                 getattr(L, name).restype = C.c_int
@@ -217,6 +232,43 @@ class Context:
         self._check(st)
         return level, rep.as_dict()
 
+    def first_order_scores(self, W: torch.Tensor, G: torch.Tensor, bits: Sequence[int], level: torch.Tensor,
+                           block_rows: int = 128, block_cols: int = 128, group: int = 128,
+                           row_perm=None, col_perm=None, s_up=None, s_down=None, s_l1=None,
+                           want_l1: bool = True):
+        R, Cc, ldw = _mat(W)
+        Rg, Cg, ldg = _mat(G)
+        assert (R, Cc) == (Rg, Cg)
+        barr, L = _bits(bits)
+        nb = (R // block_rows) * (Cc // block_cols)
+        f32 = dict(dtype=torch.float32, device=W.device)
+        if s_up is None:
+            s_up = torch.empty(nb, **f32)
+        if s_down is None:
+            s_down = torch.empty(nb, **f32)
+        if s_l1 is None and want_l1:
+            s_l1 = torch.empty(nb, **f32)
+        self._check(lib().sb_first_order_scores(
+            self._h, _ptr(W), _ptr(G), R, Cc, ldw, ldg, _ptr(row_perm, torch.int32),
+            _ptr(col_perm, torch.int32), block_rows, block_cols, group, barr, L, _ptr(level, torch.uint8),
+            _ptr(s_up, torch.float32), _ptr(s_down, torch.float32), _ptr(s_l1, torch.float32)))
+        return s_up, s_down, s_l1
+
+    def exchange_step(self, s_up: torch.Tensor, s_down: torch.Tensor, level: torch.Tensor,
+                      bits: Sequence[int], budget: float, k: int, uniform_block_elems: int = 128 * 128,
+                      block_elems=None, level_out=None):
+        N = level.numel()
+        barr, L = _bits(bits)
+        if level_out is None:
+            level_out = torch.empty_like(level)
+        rep = StepReport()
+        st = lib().sb_exchange_step(self._h, _ptr(s_up, torch.float32), _ptr(s_down, torch.float32),
+                                    _ptr(level, torch.uint8), N, _ptr(block_elems, torch.int64),
+                                    int(uniform_block_elems), barr, L, float(budget), int(k),
+                                    _ptr(level_out, torch.uint8), C.byref(rep))
+        self._check(st)
+        return level_out, rep.as_dict()
+
     def pack_blocks(self, W: torch.Tensor, bits: Sequence[int], level: torch.Tensor,
                     block_rows: int = 128, block_cols: int = 128, group: int = 128,
                     row_perm=None, col_perm=None, packed=None, block_off=None, meta=None):
@@ -254,8 +306,6 @@ def calib_moments_noalloc(X: torch.Tensor, sumsq: Optional[torch.Tensor] = None,
         scale = 1.0 / max(T, 1)
     s = torch.cuda.current_stream(X.device) if stream is None else stream
     fn = lib().sb_calib_moments_noalloc
-    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_int, C.c_float]
-    fn.restype = C.c_int
     st = fn(C.c_void_p(s.cuda_stream), _ptr(X), T, K, ldx, _ptr(sumsq, torch.float32),
             int(accumulate), float(scale))
     if st != SB_OK:

@@ -32,6 +32,22 @@ def test_library_builds_and_exports_every_declared_symbol():
     assert set(binding.EXPORTS) <= declared
 
 
+def test_every_export_has_its_argument_types_declared():
+    """Without argtypes ctypes passes Python ints as 32-bit C ints: the upper half of a 64-bit
+    parameter on the stack would be whatever was there."""
+    from paper_2602_17698_b200 import binding
+    lib = binding.lib()
+    header = open(os.path.join(ROOT, "include", "scalebits.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    for name in binding.EXPORTS:
+        fn = getattr(lib, name)
+        assert fn.argtypes is not None, name
+        m = re.search(r"\b" + name + r"\s*\(([^;]*?)\)\s*;", header, flags=re.S)
+        assert m, name
+        n_params = len([p for p in m.group(1).split(",") if p.strip()])
+        assert len(fn.argtypes) == n_params, (name, len(fn.argtypes), n_params)
+
+
 def test_binding_has_a_method_per_entry_point():
     from paper_2602_17698_b200 import binding
     for name in _declared():
