@@ -193,6 +193,18 @@ sb_status sb_first_order_scores(sb_ctx* ctx, const void* W_bf16, const void* G_b
                                 const int* bits, int n_bits, const uint8_t* level, float* s_up,
                                 float* s_down, float* s_l1);
 
+/* Reorder statistics in the first-order form (Section 3.2 with p = 1, l1 channel aggregation
+ * of Section 4.1): element sensitivity |G_rj (W_rj - Q(W)_rj)| at ref_bits on the ORIGINAL
+ * layout, summed per row and per column.  Everything else (accumulate mask, segments, "sort
+ * only" calls with W == NULL, permutations) as in sb_reorder_channels; G: device bf16 [R][C],
+ * leading dimension ldg (a multiple of 8, 16-byte aligned base).                           */
+sb_status sb_reorder_channels_first_order(sb_ctx* ctx, const void* W_bf16, const void* G_bf16,
+                                          int64_t R, int64_t C, int64_t ldw, int64_t ldg,
+                                          int ref_bits, int group,
+                                          float* row_score, float* col_score, int accumulate,
+                                          int64_t row_segment, int64_t col_segment,
+                                          int32_t* row_perm, int32_t* col_perm);
+
 /* One iteration of Algorithm 2 (lines 6-10) on per-block scores AT THE CURRENT LEVELS; the
  * caller refreshes the scores, evaluates the loss of level_out and decides on acceptance
  * (line 11) itself.  Rules as in sb_allocate_bits: one move = one level of the candidate list;

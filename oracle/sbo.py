@@ -288,3 +288,21 @@ def exchange_step(s_up, s_down, level, bits: Sequence[int], budget: float, k: in
                                  C.c_int64(uniform_block_elems), barr, C.c_int(L), C.c_double(budget),
                                  C.c_int64(k), _p(out), C.byref(rep))
     return int(st), out, rep.as_dict()
+
+
+def reorder_scores_first_order(W, G, ref_bits: int = 3, group: int = 128,
+                               row_score: Optional[np.ndarray] = None, col_score: Optional[np.ndarray] = None,
+                               accumulate: bool = False) -> Tuple[np.ndarray, np.ndarray]:
+    """Channel sums of |G (W - Q(W))| on the original layout (the p = 1 sensitivity)."""
+    W, G = _u16(W), _u16(G)
+    assert W.shape == G.shape
+    R, Cc = W.shape
+    if row_score is None:
+        row_score = np.zeros(R, dtype=np.float64)
+    if col_score is None:
+        col_score = np.zeros(Cc, dtype=np.float64)
+    st = lib().sbo_reorder_scores_first_order(_p(W), _p(G), C.c_int64(R), C.c_int64(Cc), C.c_int64(Cc),
+                                              C.c_int64(Cc), C.c_int(ref_bits), C.c_int(group),
+                                              _p(row_score), _p(col_score), C.c_int(int(accumulate)))
+    assert st == OK, st
+    return row_score, col_score

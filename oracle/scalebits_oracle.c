@@ -601,6 +601,37 @@ int sbo_first_order_scores(const uint16_t* W, const uint16_t* G, int64_t R, int6
     return SBO_OK;
 }
 
+/* ---- reorder statistics, first-order form (Section 3.2, p = 1) --------------- */
+/* The element sensitivity of Section 3.2 in the form the paper uses with gradients,
+ * sigma_rj = |G_rj (W_rj - Q(W)_rj)|, on the ORIGINAL layout at ref_bits, aggregated per channel
+ * with the l1 norm (Section 4.1): row_score[r] (+)= sum_j sigma_rj, col_score[j] (+)= sum_r.   */
+int sbo_reorder_scores_first_order(const uint16_t* W, const uint16_t* G, int64_t R, int64_t C,
+                                   int64_t ldw, int64_t ldg, int ref_bits, int group,
+                                   double* row_score, double* col_score, int accumulate) {
+    if (group <= 0 || C % group != 0 || ref_bits < 1 || ref_bits > 8) return SBO_ERR_SHAPE;
+    if (!accumulate) {
+        if (row_score) for (int64_t r = 0; r < R; ++r) row_score[r] = 0.0;
+        if (col_score) for (int64_t j = 0; j < C; ++j) col_score[j] = 0.0;
+    }
+    double* v = (double*)malloc(sizeof(double) * group);
+    double* vh = (double*)malloc(sizeof(double) * group);
+    for (int64_t r = 0; r < R; ++r) {
+        double rs = 0.0;
+        for (int64_t j0 = 0; j0 < C; j0 += group) {
+            for (int k = 0; k < group; ++k) v[k] = sbo_bf16_to_f64(W[r * ldw + j0 + k]);
+            sbo_quantize_group(v, group, ref_bits, NULL, vh, NULL, NULL);
+            for (int k = 0; k < group; ++k) {
+                const double sigma = fabs(sbo_bf16_to_f64(G[r * ldg + j0 + k]) * (v[k] - vh[k]));
+                rs += sigma;
+                if (col_score) col_score[j0 + k] += sigma;
+            }
+        }
+        if (row_score) row_score[r] += rs;
+    }
+    free(v); free(vh);
+    return SBO_OK;
+}
+
 /* ---- one iteration of Algorithm 2 on caller-supplied scores ------------------- */
 /* Lines 6-10 of Algorithm 2 with s_up / s_down given per block AT ITS CURRENT LEVEL (they change
  * with the model, so the caller refreshes them and decides on acceptance, line 11, itself).

@@ -23,7 +23,8 @@ SB_ACC_ROW, SB_ACC_COL = 1, 2
 EXPORTS = ["sb_create", "sb_destroy", "sb_sync", "sb_last_error", "sb_kernel_launches",
            "sb_calib_moments", "sb_reorder_channels", "sb_fold_segment_scores",
            "sb_expand_segment_perm", "sb_block_scores", "sb_allocate_bits", "sb_pack_blocks",
-           "sb_calib_moments_noalloc", "sb_first_order_scores", "sb_exchange_step"]
+           "sb_calib_moments_noalloc", "sb_first_order_scores", "sb_exchange_step",
+           "sb_reorder_channels_first_order"]
 
 
 class SbError(RuntimeError):
@@ -94,6 +95,8 @@ def lib() -> C.CDLL:
         L.sb_exchange_step.argtypes = [vp, vp, vp, vp, i64, vp, i64, C.POINTER(C.c_int), i32, f64, i64,
                                        vp, C.POINTER(StepReport)]
         L.sb_calib_moments_noalloc.argtypes = [vp, vp, i64, i64, i64, vp, i32, f32]
+        L.sb_reorder_channels_first_order.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, i32, vp, vp, i32,
+                                                      i64, i64, vp, vp]
         for name in EXPORTS:
             if name not in ("sb_last_error", "sb_kernel_launches"):
                 getattr(L, name).restype = C.c_int
@@ -231,6 +234,20 @@ class Context:
                                     float(gamma0), float(gammaT), _ptr(level, torch.uint8), C.byref(rep))
         self._check(st)
         return level, rep.as_dict()
+
+    def reorder_channels_first_order(self, W: torch.Tensor, G: torch.Tensor, ref_bits: int, group: int,
+                                     row_score=None, col_score=None, accumulate_row: bool = False,
+                                     accumulate_col: bool = False, row_segment: int = 0, col_segment: int = 0,
+                                     row_perm=None, col_perm=None):
+        R, Cc, ldw = _mat(W)
+        Rg, Cg, ldg = _mat(G)
+        assert (R, Cc) == (Rg, Cg)
+        acc = (SB_ACC_ROW if accumulate_row else 0) | (SB_ACC_COL if accumulate_col else 0)
+        self._check(lib().sb_reorder_channels_first_order(
+            self._h, _ptr(W), _ptr(G), R, Cc, ldw, ldg, int(ref_bits), int(group),
+            _ptr(row_score, torch.float32), _ptr(col_score, torch.float32), acc, int(row_segment),
+            int(col_segment), _ptr(row_perm, torch.int32), _ptr(col_perm, torch.int32)))
+        return row_score, col_score
 
     def first_order_scores(self, W: torch.Tensor, G: torch.Tensor, bits: Sequence[int], level: torch.Tensor,
                            block_rows: int = 128, block_cols: int = 128, group: int = 128,

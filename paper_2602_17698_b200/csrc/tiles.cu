@@ -535,9 +535,12 @@ __global__ void scores_finish_kernel(const float* __restrict__ rec, ScoreGeom g,
 // a tile row (tile column) to finish adds the partials of that row strip (column strip) in
 // tile order -- a fixed order whichever CTA does it, and no floating-point atomics, so reruns
 // are bit-identical -- and adds them to / stores them in the score vectors.
-template <bool ROWW, bool FINE, int TILE_ROWS>
+// FIRST: the first-order form of the element sensitivity, |G_rj (W_rj - Q(W)_rj)| (Section 3.2
+// with p = 1), from a caller's gradient G; no column or row factors.
+template <bool ROWW, bool FINE, int TILE_ROWS, bool FIRST>
 __global__ void __launch_bounds__(CTA_THREADS)
 reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, int64_t ldw,
+                     const __nv_bfloat16* __restrict__ G, int64_t ldg,
                      const float* __restrict__ col_moment, const float* __restrict__ row_weight,
                      int group, float qmax, float inv_qmax,
                      float* __restrict__ rowpart, float* __restrict__ colpart,
@@ -556,27 +559,34 @@ reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, 
     f32x2 cw[NW], acc[NW];
 #pragma unroll
     for (int k = 0; k < NW; ++k) {
-        cw[k] = col_ok ? pk2(col_moment[col + 2 * k], col_moment[col + 2 * k + 1]) : 0ull;
+        if (FIRST) cw[k] = pk2(1.f, 1.f);
+        else cw[k] = col_ok ? pk2(col_moment[col + 2 * k], col_moment[col + 2 * k + 1]) : 0ull;
         acc[k] = 0ull;
     }
     // the next step's two 16-byte loads are in flight while this step is evaluated
-    uint32_t wn[NW];
+    uint32_t wn[NW], gn[FIRST ? NW : 1];
     {
         const int64_t r = row0 + warp * ROW_SLOTS + slot;
         const bool ok = col_ok && r < R;
         load_cols<CPL>(W + (ok ? r * ldw + col : 0), ok, wn);
+        if constexpr (FIRST) load_cols<CPL>(G + (ok ? r * ldg + col : 0), ok, gn);
     }
 #pragma unroll 2
     for (int it = 0; it < ITERS; ++it) {
         const int rr = it * (CTA_WARPS * ROW_SLOTS) + warp * ROW_SLOTS + slot;
         const int64_t r = row0 + rr;
-        uint32_t w[NW];
+        uint32_t w[NW], gw[FIRST ? NW : 1];
 #pragma unroll
         for (int k = 0; k < NW; ++k) w[k] = wn[k];
+        if constexpr (FIRST) {
+#pragma unroll
+            for (int k = 0; k < NW; ++k) gw[k] = gn[k];
+        }
         if (it + 1 < ITERS) {
             const int64_t rn = r + CTA_WARPS * ROW_SLOTS;
             const bool okn = col_ok && rn < R;
             load_cols<CPL>(W + (okn ? rn * ldw + col : 0), okn, wn);
+            if constexpr (FIRST) load_cols<CPL>(G + (okn ? rn * ldg + col : 0), okn, gn);
         }
         float lo, hi;
         group_minmax<NW>(w, team, lo, hi);
@@ -602,7 +612,13 @@ reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, 
             const f32x2 qq = add2(fma2(vm, inv2, magic2), nmagic2);
             f32x2 e = fma2(qq, ns2, vm);
             if (FINE) e = fma2(qq, nslo2, e);
-            f32x2 e2 = mul2(e, e);
+            f32x2 e2;
+            if constexpr (FIRST) {
+                const f32x2 ge = mul2(pk2(bf16lo(gw[k]), bf16hi(gw[k])), e);
+                e2 = ge & 0x7fffffff7fffffffull;                // |g e| on both halves
+            } else {
+                e2 = mul2(e, e);
+            }
             if (ROWW) e2 = mul2(e2, ar2);
             acc[k] = add2(acc[k], e2);
             rs2 = fma2(cw[k], e2, rs2);
@@ -845,10 +861,9 @@ sb_status sb_gather_bf16(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64
     return SB_OK;
 }
 
-extern "C" {
-
-sb_status sb_reorder_channels(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw,
-                              const float* col_moment, const float* row_weight, int ref_bits,
+// both forms of the reorder statistics (G == NULL: second-moment form) and the sorts
+static sb_status reorder_impl(sb_ctx* ctx, const void* W, const void* G, int64_t R, int64_t C, int64_t ldw,
+                              int64_t ldg, const float* col_moment, const float* row_weight, int ref_bits,
                               int group, float* row_score, float* col_score, int accumulate,
                               int64_t row_segment, int64_t col_segment, int32_t* row_perm,
                               int32_t* col_perm) {
@@ -859,7 +874,9 @@ sb_status sb_reorder_channels(sb_ctx* ctx, const void* W, int64_t R, int64_t C, 
     if (sort_cols && (!col_score || C % col_segment)) return sb_fail(ctx, SB_ERR_SHAPE, "reorder: column segment");
     SB_CUDA(ctx, cudaSetDevice(ctx->device));
     if (W) {
-        if (!col_moment) return sb_fail(ctx, SB_ERR_INVALID, "reorder: col_moment is NULL");
+        if (!G && !col_moment) return sb_fail(ctx, SB_ERR_INVALID, "reorder: col_moment is NULL");
+        if (G && (ldg % 8 || ldg < C || (reinterpret_cast<uintptr_t>(G) & 15)))
+            return sb_fail(ctx, SB_ERR_SHAPE, "reorder: gradient needs ldg %% 8 == 0, ldg >= C, 16-byte base");
         if (ref_bits < 1 || ref_bits > 8) return sb_fail(ctx, SB_ERR_INVALID, "reorder: ref_bits");
         if (!valid_group(group) || C % group || C % 16 || ldw % 8 || ldw < C ||
             (reinterpret_cast<uintptr_t>(W) & 15))
@@ -888,14 +905,16 @@ sb_status sb_reorder_channels(sb_ctx* ctx, const void* W, int64_t R, int64_t C, 
         float* cpart = col_score ? colpart : nullptr;
         unsigned* done_row = ctx->stats_done;
         unsigned* done_col = ctx->stats_done + SB_STATS_TILES;
-#define SB_STATS2(RW, FN, TR)                                                                     \
-    reorder_stats_kernel<RW, FN, TR><<<grid, CTA_THREADS, 0, ctx->stream>>>(                      \
-        Wb, R, C, ldw, col_moment, row_weight, group, qmax, 1.0f / qmax, rpart, cpart, row_score, \
-        col_score, accumulate, done_row, done_col, ctx->dstate)
-#define SB_STATS(RW, FN) do { if (tile_rows == 512) SB_STATS2(RW, FN, 512); else SB_STATS2(RW, FN, 128); } while (0)
+#define SB_STATS2(RW, FN, TR, FO)                                                                 \
+    reorder_stats_kernel<RW, FN, TR, FO><<<grid, CTA_THREADS, 0, ctx->stream>>>(                  \
+        Wb, R, C, ldw, Gb, ldg, col_moment, row_weight, group, qmax, 1.0f / qmax, rpart, cpart,  \
+        row_score, col_score, accumulate, done_row, done_col, ctx->dstate)
+#define SB_STATS(RW, FN, FO) do { if (tile_rows == 512) SB_STATS2(RW, FN, 512, FO); else SB_STATS2(RW, FN, 128, FO); } while (0)
         const bool fine = ref_bits >= 6;
-        if (row_weight) { if (fine) SB_STATS(true, true); else SB_STATS(true, false); }
-        else { if (fine) SB_STATS(false, true); else SB_STATS(false, false); }
+        auto* Gb = static_cast<const __nv_bfloat16*>(G);
+        if (G) { if (fine) SB_STATS(false, true, true); else SB_STATS(false, false, true); }
+        else if (row_weight) { if (fine) SB_STATS(true, true, false); else SB_STATS(true, false, false); }
+        else { if (fine) SB_STATS(false, true, false); else SB_STATS(false, false, false); }
 #undef SB_STATS
 #undef SB_STATS2
         SB_LAUNCHED(ctx);
@@ -903,6 +922,27 @@ sb_status sb_reorder_channels(sb_ctx* ctx, const void* W, int64_t R, int64_t C, 
     if (sort_rows) { st = argsort_axis(ctx, row_score, R, row_segment, row_perm, rank); if (st) return st; }
     if (sort_cols) { st = argsort_axis(ctx, col_score, C, col_segment, col_perm, rank); if (st) return st; }
     return SB_OK;
+}
+
+extern "C" {
+
+sb_status sb_reorder_channels(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw,
+                              const float* col_moment, const float* row_weight, int ref_bits,
+                              int group, float* row_score, float* col_score, int accumulate,
+                              int64_t row_segment, int64_t col_segment, int32_t* row_perm,
+                              int32_t* col_perm) {
+    return reorder_impl(ctx, W, nullptr, R, C, ldw, 0, col_moment, row_weight, ref_bits, group, row_score,
+                        col_score, accumulate, row_segment, col_segment, row_perm, col_perm);
+}
+
+sb_status sb_reorder_channels_first_order(sb_ctx* ctx, const void* W, const void* G, int64_t R, int64_t C,
+                                          int64_t ldw, int64_t ldg, int ref_bits, int group,
+                                          float* row_score, float* col_score, int accumulate,
+                                          int64_t row_segment, int64_t col_segment, int32_t* row_perm,
+                                          int32_t* col_perm) {
+    if (ctx && W && !G) return sb_fail(ctx, SB_ERR_INVALID, "reorder (first order): G is NULL");
+    return reorder_impl(ctx, W, G, R, C, ldw, ldg, nullptr, nullptr, ref_bits, group, row_score, col_score,
+                        accumulate, row_segment, col_segment, row_perm, col_perm);
 }
 
 sb_status sb_fold_segment_scores(sb_ctx* ctx, float* dst, const float* src, int64_t n_dst, int reps,

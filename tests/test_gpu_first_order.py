@@ -165,3 +165,29 @@ def test_first_order_loop_on_a_layer_walks_the_oracle_trajectory(ctx):
     assert expansions > 0 and exchanges > 0, (expansions, exchanges)
     used = int((torch.tensor(bits, device=DEV)[level.long()] * (br * bc)).sum())
     assert used <= int(budget * R * C)
+
+
+@pytest.mark.parametrize("R,C,g,bits", [(2048, 2048, 128, 3), (200, 384, 64, 2), (130, 272, 16, 4),
+                                        (1024, 512, 32, 8)])
+def test_first_order_reorder_scores_and_sort(ctx, R, C, g, bits):
+    W = synth.make_weight(R, C, 7 + R, DEV)
+    G = _grad(R, C, 9 + C)
+    rs = torch.empty(R, dtype=torch.float32, device=DEV)
+    cs = torch.empty(C, dtype=torch.float32, device=DEV)
+    pr = torch.empty(R, dtype=torch.int32, device=DEV)
+    pc = torch.empty(C, dtype=torch.int32, device=DEV)
+    ctx.reorder_channels_first_order(W, G, bits, g, row_score=rs, col_score=cs, row_segment=R,
+                                     col_segment=C, row_perm=pr, col_perm=pc)
+    ctx.sync()
+    ors, ocs = sbo.reorder_scores_first_order(W.cpu(), G.cpu(), ref_bits=bits, group=g)
+    assert np.allclose(rs.cpu().numpy(), ors, rtol=REL, atol=0)
+    assert np.allclose(cs.cpu().numpy(), ocs, rtol=REL, atol=0)
+    # hand-off: the oracle's sort of the GPU's scores must equal the GPU's permutation exactly
+    assert np.array_equal(pr.cpu().numpy(), sbo.argsort_desc_segments(rs.cpu().double().numpy()))
+    assert np.array_equal(pc.cpu().numpy(), sbo.argsort_desc_segments(cs.cpu().double().numpy()))
+    # accumulation over coupled matrices
+    rs2 = rs.clone()
+    ctx.reorder_channels_first_order(W, G, bits, g, row_score=rs2, col_score=cs, accumulate_row=True)
+    ctx.sync()
+    assert np.allclose(rs2.cpu().numpy(), 2 * ors, rtol=REL)
+    assert np.allclose(cs.cpu().numpy(), ocs, rtol=REL)

@@ -140,6 +140,38 @@ def test_permutations_equal_an_explicitly_permuted_matrix():
         assert np.array_equal(x, y)
 
 
+# ---- channel sums of the p = 1 sensitivity ------------------------------------------------------------
+def test_first_order_channel_scores_agree_with_the_block_sums_and_plain_loops():
+    R, C, g, b = 32, 128, 32, 3
+    W = synth.make_weight(R, C, 17)
+    G = _grad(R, C, 19)
+    rs, cs = sbo.reorder_scores_first_order(W, G, b, g)
+    # the same element sensitivities summed three ways: by row, by column, by block
+    _, _, l1 = sbo.first_order_scores(W, G, [b], np.zeros(8, dtype=np.uint8), 16, 32, g)
+    assert rs.sum() == pytest.approx(cs.sum(), rel=1e-13)
+    assert rs.sum() == pytest.approx(l1.sum(), rel=1e-13)
+    assert rs[:16].sum() == pytest.approx(l1[:4].sum(), rel=1e-13)            # first block row
+    assert cs[32:64].sum() == pytest.approx(l1[1] + l1[5], rel=1e-13)        # second block column
+    # plain loops for two rows and two columns, through the pinned group quantizer
+    Wd, Gd = _f64(W), _f64(G)
+    sig = np.empty_like(Wd)
+    for r in range(R):
+        for c0 in range(0, C, g):
+            _, vh, _, _ = sbo.quantize_group(Wd[r, c0:c0 + g], b)
+            sig[r, c0:c0 + g] = np.abs(Gd[r, c0:c0 + g] * (Wd[r, c0:c0 + g] - vh))
+    assert np.allclose(rs, sig.sum(axis=1), rtol=1e-13) and np.allclose(cs, sig.sum(axis=0), rtol=1e-13)
+    # accumulation over coupled matrices
+    rs2, cs2 = sbo.reorder_scores_first_order(W, G, b, g, row_score=rs.copy(), col_score=cs.copy(),
+                                              accumulate=True)
+    assert np.allclose(rs2, 2 * rs, rtol=1e-15) and np.allclose(cs2, 2 * cs, rtol=1e-15)
+    # a gradient that vanishes on a channel makes that channel's score vanish
+    G0 = G.clone()
+    G0[:, 7] = 0
+    G0[5, :] = 0
+    rs0, cs0 = sbo.reorder_scores_first_order(W, G0, b, g)
+    assert cs0[7] == 0.0 and rs0[5] == 0.0
+
+
 # ---- one iteration of Algorithm 2 on given scores -------------------------------------------------
 def _table(N, L, seed, ragged):
     rng = np.random.default_rng(seed)
