@@ -233,6 +233,14 @@ def kernel_rooflines(ctx, W, moments, dev, peak_gbs, sm_mhz):
                                               want_gain=False, W_perm_out=out))
     t_pack = timed(lambda m: ctx.pack_blocks(m, BITS, level, 128, 128, 128, packed=packed, block_off=off,
                                              meta=meta))
+    Gm = [(m.float() * 1e-2).to(torch.bfloat16) for m in mats[:2]]       # stand-in gradients
+    Gm.append(Gm[0].clone())
+    s_up, s_dn = torch.empty(nb, **f32), torch.empty(nb, **f32)
+    idx = {id(m): i for i, m in enumerate(mats)}
+    t_first = timed(lambda m: ctx.first_order_scores(m, Gm[idx[id(m)]], BITS, level, 128, 128, 128,
+                                                     s_up=s_up, s_down=s_dn, want_l1=False))
+    t_fstats = timed(lambda m: ctx.reorder_channels_first_order(m, Gm[idx[id(m)]], 2, 128, row_score=rs,
+                                                                col_score=cs))
     t_gather = max(t_perm - t_score, 1e-6)
     avg_bits = sum(BITS) / len(BITS)
 
@@ -256,6 +264,10 @@ def kernel_rooflines(ctx, W, moments, dev, peak_gbs, sm_mhz):
             "sb_block_scores with both permutations and W_perm_out minus the call without (2 B read + 2 B written)"),
         hbm("pack_offsets_small_kernel + pack_kernel", int(2 * n + n * avg_bits / 8 + n / 128 * 8), t_pack,
             "one call of sb_pack_blocks, uniformly random levels (2 B read + codes + metadata written)"),
+        hbm("first_order_kernel", 4 * n, t_first,
+            "one call of sb_first_order_scores, uniformly random levels (weights and gradient, 2 B each)"),
+        hbm("reorder_stats_kernel (first-order form)", 4 * n, t_fstats,
+            "one call of sb_reorder_channels_first_order (weights and gradient, 2 B each)"),
     ]
 
 
