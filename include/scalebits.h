@@ -170,6 +170,17 @@ sb_status sb_pack_blocks(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_t C, 
                          uint32_t* packed, int64_t packed_capacity_words,
                          int64_t* block_off_words, float* meta);
 
+/* Full calibration second-moment matrix on the tensor cores (Section 3.2: sb_calib_moments
+ * returns the diagonal of this matrix; a sensitivity that keeps the cross terms between input
+ * channels needs all of it):
+ *     H[i][j] = (accumulate ? H[i][j] : 0) + scale * sum_t X[t][i] X[t][j]
+ * X: device bf16 [T][K], leading dimension ldx (K % 8 == 0, ldx % 8 == 0, 16-byte aligned
+ * base); H: device fp32 [K][K], row-major, both triangles written.  bf16 products are exact in
+ * fp32, the sum over tokens is accumulated in fp32 by the tensor cores.  A pipeline wait that
+ * does not complete within 2 s latches SB_ERR_TIMEOUT and the kernel returns.  Asynchronous. */
+sb_status sb_calib_gram(sb_ctx* ctx, const void* X_bf16, int64_t T, int64_t K, int64_t ldx,
+                        float* H, int accumulate, float scale);
+
 /* First-order mode (Appendix E.3, "choice of sensitivity statistics"): the paper's own scores
  * for Algorithm 2 from a caller-supplied gradient G = dL/dw taken at the current quantized
  * model.  Every block is quantized at ITS current bitwidth b = bits[level[block]] on the

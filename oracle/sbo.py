@@ -306,3 +306,13 @@ def reorder_scores_first_order(W, G, ref_bits: int = 3, group: int = 128,
                                               _p(row_score), _p(col_score), C.c_int(int(accumulate)))
     assert st == OK, st
     return row_score, col_score
+
+
+def calib_gram(X, scale: Optional[float] = None) -> np.ndarray:
+    """H = scale * X^T X in fp64 (scale defaults to 1 / T); [K, K]."""
+    X = _u16(X)
+    T, K = X.shape
+    H = np.zeros((K, K), dtype=np.float64)
+    lib().sbo_calib_gram(_p(X), C.c_int64(T), C.c_int64(K), C.c_int64(K),
+                         C.c_double(1.0 / max(T, 1) if scale is None else scale), _p(H))
+    return H

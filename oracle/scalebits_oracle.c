@@ -89,6 +89,24 @@ void sbo_calib_moments(const uint16_t* X, int64_t T, int64_t K, int64_t ldx,
     }
 }
 
+/* ---- full calibration second-moment matrix -------------------------------- */
+/* H[i][j] = scale * sum_t X[t][i] X[t][j]: the matrix whose diagonal sbo_calib_moments
+ * returns (Section 3.2: the sensitivity "needs more than its diagonal" when cross terms
+ * between input channels are kept).  Plain triple loop, upper triangle mirrored.          */
+void sbo_calib_gram(const uint16_t* X, int64_t T, int64_t K, int64_t ldx, double scale, double* H) {
+    #pragma omp parallel for schedule(dynamic, 4)
+    for (int64_t i = 0; i < K; ++i) {
+        for (int64_t j = i; j < K; ++j) {
+            double s = 0.0;
+            for (int64_t t = 0; t < T; ++t)
+                s += sbo_bf16_to_f64(X[t * ldx + i]) * sbo_bf16_to_f64(X[t * ldx + j]);
+            H[i * K + j] = s * scale;
+        }
+    }
+    for (int64_t i = 0; i < K; ++i)
+        for (int64_t j = 0; j < i; ++j) H[i * K + j] = H[j * K + i];
+}
+
 /* ---- the quantizer Q(., b) on one group (Section 5 "Implementation") ------ */
 /* asymmetric min-max RTN, min-anchored:
  *   lo = min v, hi = max v, range = hi - lo, qmax = 2^b - 1

@@ -24,7 +24,7 @@ EXPORTS = ["sb_create", "sb_destroy", "sb_sync", "sb_last_error", "sb_kernel_lau
            "sb_calib_moments", "sb_reorder_channels", "sb_fold_segment_scores",
            "sb_expand_segment_perm", "sb_block_scores", "sb_allocate_bits", "sb_pack_blocks",
            "sb_calib_moments_noalloc", "sb_first_order_scores", "sb_exchange_step",
-           "sb_reorder_channels_first_order"]
+           "sb_reorder_channels_first_order", "sb_calib_gram"]
 
 
 class SbError(RuntimeError):
@@ -95,6 +95,7 @@ def lib() -> C.CDLL:
         L.sb_exchange_step.argtypes = [vp, vp, vp, vp, i64, vp, i64, C.POINTER(C.c_int), i32, f64, i64,
                                        vp, C.POINTER(StepReport)]
         L.sb_calib_moments_noalloc.argtypes = [vp, vp, i64, i64, i64, vp, i32, f32]
+        L.sb_calib_gram.argtypes = [vp, vp, i64, i64, i64, vp, i32, f32]
         L.sb_reorder_channels_first_order.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, i32, vp, vp, i32,
                                                       i64, i64, vp, vp]
         for name in EXPORTS:
@@ -171,6 +172,18 @@ class Context:
         self._check(lib().sb_calib_moments(self._h, _ptr(X), T, K, ldx, _ptr(sumsq, torch.float32),
                                            int(accumulate), float(scale)))
         return sumsq
+
+    def calib_gram(self, X: torch.Tensor, H: Optional[torch.Tensor] = None, accumulate: bool = False,
+                   scale: Optional[float] = None) -> torch.Tensor:
+        T, K, ldx = _mat(X)
+        if H is None:
+            H = torch.empty((K, K), dtype=torch.float32, device=X.device)
+            accumulate = False
+        if scale is None:
+            scale = 1.0 / max(T, 1)
+        self._check(lib().sb_calib_gram(self._h, _ptr(X), T, K, ldx, _ptr(H, torch.float32), int(accumulate),
+                                        float(scale)))
+        return H
 
     def reorder_channels(self, W: Optional[torch.Tensor], col_moment: Optional[torch.Tensor],
                          ref_bits: int, group: int, row_score=None, col_score=None,

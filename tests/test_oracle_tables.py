@@ -199,3 +199,22 @@ def test_block_counts_quoted_by_the_paper():
     v, tol = rows["llama3_8b_classic_greedy_iterations"]
     assert abs(n_blocks * 3.5 / v - 1) <= tol
     assert synth.LLAMA3_8B.n_weights == 218_103_808
+
+
+def test_gram_matrix_pins():
+    """Diagonal = the pinned second moments; symmetric; positive semi-definite; equal to a
+    float64 matrix product; closed form for one-hot rows."""
+    import torch
+    X = synth.make_activations(300, 40, 5)
+    H = sbo.calib_gram(X)
+    assert np.array_equal(H, H.T)
+    assert np.allclose(np.diag(H), sbo.calib_moments(X, 1.0 / 300), rtol=1e-13)
+    Xd = X.double().numpy()
+    assert np.allclose(H, Xd.T @ Xd / 300, rtol=1e-12, atol=1e-14)
+    assert np.linalg.eigvalsh(H).min() >= -1e-9 * np.abs(H).max()
+    # one-hot rows: H = diag(counts) * value^2 / T
+    idx = np.arange(64) % 8
+    onehot = torch.zeros(64, 8)
+    onehot[np.arange(64), idx] = 3.0
+    Ho = sbo.calib_gram(onehot.to(torch.bfloat16))
+    assert np.allclose(Ho, np.eye(8) * 9.0 * 8 / 64, rtol=0, atol=1e-15)
