@@ -192,7 +192,16 @@ FULL_MODEL_BUDGETS = tuple(2.0 + 0.25 * i for i in range(9))          # 2.0 ... 
 FULL_MODEL_SUPER = {3: 101, 12: 102, 20: 103, 29: 104}                # layer -> seed of its super weight
 
 
-def kernel_rooflines(ctx, W, moments, dev, peak_gbs, sm_mhz):
+def measured_tensor_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["bf16_tflops"]), "measured cuBLAS bf16 burst"
+    return 1590.0, "fallback"
+
+
+def kernel_rooflines(ctx, W, X, moments, dev, peak_gbs, sm_mhz):
     """The other kernels of the path, one library call at a time on 14336 x 4096 matrices (three
     different ones in rotation, 352 MB > L2, so every call streams from HBM), CUDA events on the
     context's stream.  HBM-bound kernels against the measured copy bandwidth; the score kernel
@@ -243,6 +252,23 @@ def kernel_rooflines(ctx, W, moments, dev, peak_gbs, sm_mhz):
                                                                 col_score=cs))
     t_gather = max(t_perm - t_score, 1e-6)
     avg_bits = sum(BITS) / len(BITS)
+    # the one contraction: H = X^T X / T of the layer's MLP input (65536 x 4096) on the tensor cores
+    Xg = X["mlp_in"]
+    Tg, Kg = Xg.shape
+    Hg = torch.empty((Kg, Kg), **f32)
+    for _ in range(2):
+        ctx.calib_gram(Xg, H=Hg)
+    ga, gb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ga.record()
+    for _ in range(5):
+        ctx.calib_gram(Xg, H=Hg)
+    gb.record()
+    gb.synchronize()
+    t_gram = ga.elapsed_time(gb) / 5
+    nt = (Kg + 127) // 128
+    gram_flops = 2.0 * Tg * 128 * 128 * (nt * (nt + 1) // 2)          # the upper-triangular tiles it computes
+    tpeak, tkind = measured_tensor_peak()
+    del Hg
 
     def hbm(name, bytes_, ms, note):
         a = bytes_ / (ms * 1e-3) / 1e9
@@ -264,6 +290,12 @@ def kernel_rooflines(ctx, W, moments, dev, peak_gbs, sm_mhz):
             "sb_block_scores with both permutations and W_perm_out minus the call without (2 B read + 2 B written)"),
         hbm("pack_offsets_small_kernel + pack_kernel", int(2 * n + n * avg_bits / 8 + n / 128 * 8), t_pack,
             "one call of sb_pack_blocks, uniformly random levels (2 B read + codes + metadata written)"),
+        {"kernel": "gram_kernel (tcgen05, TMA)", "bound": "tensor", "achieved": gram_flops / (t_gram * 1e-3) / 1e12,
+         "peak": tpeak, "unit": "TFLOP/s", "frac": gram_flops / (t_gram * 1e-3) / 1e12 / tpeak,
+         "peak_source": tkind, "ms_per_call": t_gram,
+         "effective_tflops_of_full_product": 2.0 * Tg * Kg * Kg / (t_gram * 1e-3) / 1e12,
+         "note": f"one call of sb_calib_gram on the {Tg} x {Kg} MLP input; flops of the upper-triangular "
+                 "128 x 128 tiles it computes (the mirror image is copied)"},
         hbm("first_order_kernel", 4 * n, t_first,
             "one call of sb_first_order_scores, uniformly random levels (weights and gradient, 2 B each)"),
         hbm("reorder_stats_kernel (first-order form)", 4 * n, t_fstats,
@@ -445,7 +477,7 @@ def run_cuda(args):
                      "scores": w_bytes / (stage_ms["scores"] * 1e-3) / 1e9,
                      "pack": w_bytes / (stage_ms["pack"] * 1e-3) / 1e9}
         sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
-        kernels = kernel_rooflines(ctx, W, ws.moments, dev, peak, sm_mhz)
+        kernels = kernel_rooflines(ctx, W, X, ws.moments, dev, peak, sm_mhz)
         full_model = None
         if world == 1 and not args.no_full_model:
             del hW, hX                                   # pinned copies of the layer, if any
@@ -491,6 +523,11 @@ def run_only(which: str):
         X = synth.make_activations(TOKENS, 4096, 7, dev)
         for _ in range(3):
             ctx.calib_moments(X)
+    elif which == "gram":
+        X = synth.make_activations(32768, 2048, 7, dev)           # 134 MB, 136 tiles of 128 x 128
+        H = torch.empty((2048, 2048), device=dev)
+        for _ in range(3):
+            ctx.calib_gram(X, H=H)
     else:
         W = synth.make_weight(R, Cc, 100, dev)
         nb = (R // 128) * (Cc // 128)
@@ -533,7 +570,7 @@ def main():
     ap.add_argument("--no-graphs", action="store_true", help="launch every library call eagerly")
     ap.add_argument("--only", default=None,
                     help="three calls of one library call on one input, then exit (for ncu captures): "
-                         "moments | reorder_stats | scores | gather | pack")
+                         "moments | gram | reorder_stats | scores | gather | pack")
     args = ap.parse_args()
     if args.only:
         run_only(args.only)
