@@ -34,7 +34,7 @@ WORKLOAD = ("one Llama-3-8B-shaped decoder layer (q/o 4096x4096, k/v 1024x4096, 
 # ncu capture summarised in profiles/moments_partial_kernel_65536x4096.md (541.04 MB moved for
 # 536.87 MB of activations); the kernel's traffic is proportional to T * K, so the ratio carries
 # over to the launches of the step
-NCU_TRAFFIC_RATIO = {"moments_partial_kernel": 1.0078}
+NCU_TRAFFIC_RATIO = {"moments_partial_kernel": 1.0071}
 
 
 def measured_peaks():
@@ -503,6 +503,7 @@ def run_cuda(args):
         print(json.dumps(line), flush=True)
     ctx.close()
     if world > 1:
+        dist.barrier()              # rank 0 may still have been timing its extra legs
         dist.destroy_process_group()
 
 
