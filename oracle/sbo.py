@@ -316,3 +316,21 @@ def calib_gram(X, scale: Optional[float] = None) -> np.ndarray:
     lib().sbo_calib_gram(_p(X), C.c_int64(T), C.c_int64(K), C.c_int64(K),
                          C.c_double(1.0 / max(T, 1) if scale is None else scale), _p(H))
     return H
+
+
+def block_scores_full(W, H, bits: Sequence[int], block_rows=128, block_cols=128, group=128,
+                      row_perm=None, col_perm=None) -> np.ndarray:
+    """Block error table with the full second-moment matrix H [C, C] (original column order)."""
+    W = _u16(W)
+    R, Cc = W.shape
+    H = np.ascontiguousarray(_f64(H).reshape(Cc, Cc))
+    rp, cp = _i32(row_perm), _i32(col_perm)
+    barr, L = _bits(bits)
+    nb = (R // block_rows) * (Cc // block_cols)
+    err = np.zeros((nb, L), dtype=np.float64)
+    st = lib().sbo_block_scores_full(_p(W), C.c_int64(R), C.c_int64(Cc), C.c_int64(Cc), _p(rp), _p(cp),
+                                     _p(H), C.c_int(block_rows), C.c_int(block_cols), C.c_int(group),
+                                     barr, C.c_int(L), _p(err))
+    if st != OK:
+        raise ValueError(f"sbo_block_scores_full status {st}")
+    return err

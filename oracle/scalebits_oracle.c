@@ -284,6 +284,60 @@ int sbo_block_scores(const uint16_t* W, int64_t R, int64_t C, int64_t ldw,
     return SBO_OK;
 }
 
+/* ---- block error table with the full second-moment matrix ------------------- */
+/* The sensitivity of Section 3.2 with the cross terms between input channels kept: for block i
+ * with columns J (permuted layout) and candidate b_l,
+ *   E[i][l] = sum over rows r of block i of  d_r H'_JJ d_r^T,   d_r = (W' - Q_{b_l}(W'))_{r,J},
+ * where H' = H[cp][:, cp] is the calibration second-moment matrix (sbo_calib_gram) in the
+ * permuted column order.  With a diagonal H this is sbo_block_scores with c = diag(H).         */
+int sbo_block_scores_full(const uint16_t* W, int64_t R, int64_t C, int64_t ldw,
+                          const int32_t* row_perm, const int32_t* col_perm, const double* H,
+                          int br, int bc, int group, const int* bits, int L, double* err) {
+    if (!check_bits(bits, L)) return SBO_ERR_INVALID;
+    if (br <= 0 || bc <= 0 || group <= 0 || R % br || C % bc || bc % group) return SBO_ERR_SHAPE;
+    const int64_t nbr = R / br, nbc = C / bc;
+    #pragma omp parallel
+    {
+        double* v = (double*)malloc(sizeof(double) * group);
+        double* vh = (double*)malloc(sizeof(double) * group);
+        double* d = (double*)malloc(sizeof(double) * bc);
+        #pragma omp for schedule(dynamic, 1)
+        for (int64_t blk = 0; blk < nbr * nbc; ++blk) {
+            const int64_t bi = blk / nbc, bj = blk % nbc;
+            for (int l = 0; l < L; ++l) {
+                double e = 0.0;
+                for (int rr = 0; rr < br; ++rr) {
+                    const int64_t r = bi * br + rr;
+                    const int64_t rs = row_perm ? row_perm[r] : r;
+                    for (int g0 = 0; g0 < bc; g0 += group) {
+                        for (int k = 0; k < group; ++k) {
+                            const int64_t j = bj * bc + g0 + k;
+                            const int64_t js = col_perm ? col_perm[j] : j;
+                            v[k] = sbo_bf16_to_f64(W[rs * ldw + js]);
+                        }
+                        sbo_quantize_group(v, group, bits[l], NULL, vh, NULL, NULL);
+                        for (int k = 0; k < group; ++k) d[g0 + k] = v[k] - vh[k];
+                    }
+                    for (int a = 0; a < bc; ++a) {
+                        const int64_t ja = bj * bc + a;
+                        const int64_t jas = col_perm ? col_perm[ja] : ja;
+                        double s = 0.0;
+                        for (int b = 0; b < bc; ++b) {
+                            const int64_t jb = bj * bc + b;
+                            const int64_t jbs = col_perm ? col_perm[jb] : jb;
+                            s += H[jas * C + jbs] * d[b];
+                        }
+                        e += d[a] * s;
+                    }
+                }
+                err[blk * L + l] = e;
+            }
+        }
+        free(v); free(vh); free(d);
+    }
+    return SBO_OK;
+}
+
 /* ---- allocation ------------------------------------------------------------ */
 static inline int64_t blk_elems(const int64_t* block_elems, int64_t uniform, int64_t i) {
     return block_elems ? block_elems[i] : uniform;

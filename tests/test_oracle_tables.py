@@ -218,3 +218,43 @@ def test_gram_matrix_pins():
     onehot[np.arange(64), idx] = 3.0
     Ho = sbo.calib_gram(onehot.to(torch.bfloat16))
     assert np.allclose(Ho, np.eye(8) * 9.0 * 8 / 64, rtol=0, atol=1e-15)
+
+
+def test_full_second_moment_block_scores_pins():
+    """Diagonal H reduces to the pinned block table; H = u u^T gives sum_r (d_r . u)^2; a
+    positive semi-definite H gives non-negative errors; permutations equal an explicitly
+    permuted problem."""
+    import torch
+    R, C, br, bc, g = 64, 128, 32, 64, 32
+    bits = [2, 3, 4]
+    W = synth.make_weight(R, C, 21)
+    rng = np.random.default_rng(2)
+    c = rng.uniform(0.1, 2.0, size=C)
+    e_diag = sbo.block_scores_full(W, np.diag(c), bits, br, bc, g)
+    e_ref, _ = sbo.block_scores(W, c, bits, br, bc, g)
+    assert np.allclose(e_diag, e_ref, rtol=1e-12)
+    # rank one: E = sum over rows of (d_r . u_J)^2, through the pinned group quantizer
+    u = rng.normal(size=C)
+    e_rank1 = sbo.block_scores_full(W, np.outer(u, u), bits, br, bc, g)
+    Wd = W.double().numpy()
+    for l, b in enumerate(bits):
+        D = np.empty_like(Wd)
+        for r in range(R):
+            for c0 in range(0, C, g):
+                _, vh, _, _ = sbo.quantize_group(Wd[r, c0:c0 + g], b)
+                D[r, c0:c0 + g] = Wd[r, c0:c0 + g] - vh
+        for blk in range((R // br) * (C // bc)):
+            bi, bj = divmod(blk, C // bc)
+            proj = D[bi * br:(bi + 1) * br, bj * bc:(bj + 1) * bc] @ u[bj * bc:(bj + 1) * bc]
+            assert e_rank1[blk, l] == pytest.approx((proj ** 2).sum(), rel=1e-11)
+    # a Gram matrix is positive semi-definite: errors are non-negative and fall with the bits
+    X = synth.make_activations(256, C, 5)
+    H = sbo.calib_gram(X)
+    e_full = sbo.block_scores_full(W, H, bits, br, bc, g)
+    assert np.all(e_full >= 0)
+    # permutations
+    pr, pc = rng.permutation(R).astype(np.int32), rng.permutation(C).astype(np.int32)
+    e_perm = sbo.block_scores_full(W, H, bits, br, bc, g, row_perm=pr, col_perm=pc)
+    Wp = W[torch.from_numpy(pr).long()][:, torch.from_numpy(pc).long()].contiguous()
+    Hp = H[np.ix_(pc, pc)]
+    assert np.allclose(e_perm, sbo.block_scores_full(Wp, Hp, bits, br, bc, g), rtol=1e-12)
