@@ -181,6 +181,24 @@ sb_status sb_pack_blocks(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_t C, 
 sb_status sb_calib_gram(sb_ctx* ctx, const void* X_bf16, int64_t T, int64_t K, int64_t ldx,
                         float* H, int accumulate, float scale);
 
+/* Block error table with the full second-moment matrix (Section 3.2 with the cross terms
+ * between input channels kept), on the permuted layout W' = W[row_perm][:, col_perm]:
+ *     err[i][l]  = sum over rows r of block i of  d_r H'_JJ d_r^T,
+ *                  d_r = (W' - Q_{b_l}(W'))[r, J],  J = the block's 128 columns,
+ *                  H'_JJ[a][b] = H[col_perm[J0 + a]][col_perm[J0 + b]]
+ *     gain[i][l] = (err[i][l] - err[i][l+1]) / ((b_{l+1} - b_l) * 128 * 128)
+ * H: device fp32 [C][C] in the ORIGINAL column order (sb_calib_gram); symmetric.  With a
+ * diagonal H this is sb_block_scores with col_moment = diag(H).  Blocks are 128 x 128
+ * (block_rows = block_cols = 128 is required), group in {16,32,64,128}; no row weights.
+ * The 128 x 128 Gram matrix of every (block, candidate) residual is a tensor-core contraction
+ * of two bf16 terms of the residual (relative error about 2^-16).  err, gain (or NULL) and
+ * W_perm_out (or NULL) as in sb_block_scores.  A pipeline wait that does not complete within
+ * 2 s latches SB_ERR_TIMEOUT.  Asynchronous.                                                */
+sb_status sb_block_scores_full(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_t C, int64_t ldw,
+                               const int32_t* row_perm, const int32_t* col_perm, const float* H,
+                               int block_rows, int block_cols, int group, const int* bits, int n_bits,
+                               float* err, float* gain, void* W_perm_out_bf16);
+
 /* First-order mode (Appendix E.3, "choice of sensitivity statistics"): the paper's own scores
  * for Algorithm 2 from a caller-supplied gradient G = dL/dw taken at the current quantized
  * model.  Every block is quantized at ITS current bitwidth b = bits[level[block]] on the

@@ -24,7 +24,8 @@ EXPORTS = ["sb_create", "sb_destroy", "sb_sync", "sb_last_error", "sb_kernel_lau
            "sb_calib_moments", "sb_reorder_channels", "sb_fold_segment_scores",
            "sb_expand_segment_perm", "sb_block_scores", "sb_allocate_bits", "sb_pack_blocks",
            "sb_calib_moments_noalloc", "sb_first_order_scores", "sb_exchange_step",
-           "sb_reorder_channels_first_order", "sb_calib_gram"]
+           "sb_reorder_channels_first_order", "sb_calib_gram",
+           "sb_block_scores_full"]
 
 
 class SbError(RuntimeError):
@@ -96,6 +97,8 @@ def lib() -> C.CDLL:
                                        vp, C.POINTER(StepReport)]
         L.sb_calib_moments_noalloc.argtypes = [vp, vp, i64, i64, i64, vp, i32, f32]
         L.sb_calib_gram.argtypes = [vp, vp, i64, i64, i64, vp, i32, f32]
+        L.sb_block_scores_full.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp, i32, i32, i32,
+                                           C.POINTER(C.c_int), i32, vp, vp, vp]
         L.sb_reorder_channels_first_order.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, i32, vp, vp, i32,
                                                       i64, i64, vp, vp]
         for name in EXPORTS:
@@ -230,6 +233,24 @@ class Context:
             self._h, _ptr(W), R, Cc, ldw, _ptr(row_perm, torch.int32), _ptr(col_perm, torch.int32),
             _ptr(col_moment, torch.float32), _ptr(row_weight, torch.float32),
             block_rows, block_cols, group, barr, L, _ptr(err, torch.float32),
+            _ptr(gain, torch.float32), _ptr(W_perm_out, torch.bfloat16)))
+        return err, gain
+
+    def block_scores_full(self, W: torch.Tensor, H: torch.Tensor, bits: Sequence[int],
+                          block_rows: int = 128, block_cols: int = 128, group: int = 128,
+                          row_perm=None, col_perm=None, err=None, gain=None, want_gain: bool = True,
+                          W_perm_out=None):
+        R, Cc, ldw = _mat(W)
+        assert H.shape == (Cc, Cc) and H.is_contiguous()
+        barr, L = _bits(bits)
+        nb = (R // block_rows) * (Cc // block_cols)
+        if err is None:
+            err = torch.empty((nb, L), dtype=torch.float32, device=W.device)
+        if gain is None and want_gain and L > 1:
+            gain = torch.empty((nb, L - 1), dtype=torch.float32, device=W.device)
+        self._check(lib().sb_block_scores_full(
+            self._h, _ptr(W), R, Cc, ldw, _ptr(row_perm, torch.int32), _ptr(col_perm, torch.int32),
+            _ptr(H, torch.float32), block_rows, block_cols, group, barr, L, _ptr(err, torch.float32),
             _ptr(gain, torch.float32), _ptr(W_perm_out, torch.bfloat16)))
         return err, gain
 

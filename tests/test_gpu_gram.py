@@ -57,3 +57,43 @@ def test_gram_accumulate_strided_and_deterministic(ctx):
     assert torch.allclose(H2, 2 * H1, rtol=1e-6)
     ref = sbo.calib_gram(X.contiguous().cpu(), scale=1.0)
     _check(H1.cpu().double().numpy(), ref)
+
+
+# ---- block error table with the full second-moment matrix -------------------------------------------
+@pytest.mark.parametrize("R,C,g,bits,perm", [(128, 128, 128, [2, 3, 4, 8], False), (256, 256, 128, [2, 3, 4, 8], False),
+                                             (512, 384, 64, [2, 3, 4], True), (384, 512, 16, [1, 2, 3, 4, 5, 6, 8], True),
+                                             (2048, 1024, 32, [3, 4], False)])
+def test_block_scores_with_the_full_second_moment_matrix(ctx, R, C, g, bits, perm):
+    from tests.helpers import REL
+    W = synth.make_weight(R, C, 51 + R + C, DEV)
+    X = synth.make_activations(2048, C, 53 + C, DEV)
+    H = ctx.calib_gram(X)
+    rng = np.random.default_rng(R + C)
+    pr = torch.from_numpy(rng.permutation(R).astype(np.int32)).to(DEV) if perm else None
+    pc = torch.from_numpy(rng.permutation(C).astype(np.int32)).to(DEV) if perm else None
+    err, gain = ctx.block_scores_full(W, H, bits, 128, 128, g, row_perm=pr, col_perm=pc)
+    ctx.sync()
+    # hand-off: the oracle is fed the GPU's matrix
+    ref = sbo.block_scores_full(W.cpu(), H.cpu().double().numpy(), bits, 128, 128, g,
+                                row_perm=None if pr is None else pr.cpu().numpy(),
+                                col_perm=None if pc is None else pc.cpu().numpy())
+    got = err.cpu().double().numpy()
+    assert np.all(np.abs(got - ref) <= REL * np.abs(ref)), np.max(np.abs(got - ref) / np.abs(ref))
+    if len(bits) > 1:
+        gref = (ref[:, :-1] - ref[:, 1:]) / (np.diff(bits)[None, :] * 128 * 128)
+        tol = REL * (np.abs(ref[:, :-1]) + np.abs(ref[:, 1:])) / (np.diff(bits)[None, :] * 128 * 128)
+        assert np.all(np.abs(gain.cpu().double().numpy() - gref) <= tol)
+    e2, _ = ctx.block_scores_full(W, H, bits, 128, 128, g, row_perm=pr, col_perm=pc)
+    ctx.sync()
+    assert torch.equal(err, e2)                       # deterministic
+
+
+def test_full_scores_with_a_diagonal_matrix_equal_the_diagonal_path(ctx):
+    from tests.helpers import REL
+    R, C, g, bits = 256, 384, 128, [2, 3, 4, 8]
+    W = synth.make_weight(R, C, 61, DEV)
+    c = torch.rand(C, device=DEV) + 0.25
+    e_full, _ = ctx.block_scores_full(W, torch.diag(c).contiguous(), bits, 128, 128, g)
+    e_diag, _ = ctx.block_scores(W, c, bits, 128, 128, g)
+    ctx.sync()
+    assert torch.allclose(e_full, e_diag, rtol=REL, atol=0)
