@@ -268,6 +268,9 @@ def kernel_rooflines(ctx, W, X, moments, dev, peak_gbs, sm_mhz):
     nt = (Kg + 127) // 128
     gram_flops = 2.0 * Tg * 128 * 128 * (nt * (nt + 1) // 2)          # the upper-triangular tiles it computes
     tpeak, tkind = measured_tensor_peak()
+    # block scores with the full matrix (same 14336 x 4096 matrices, H of their input)
+    t_full = timed(lambda m: ctx.block_scores_full(m, Hg, BITS, 128, 128, 128, err=err, want_gain=False), reps=6)
+    full_flops = nb * len(BITS) * 2 * 2.0 * 128 ** 3            # two 128^3 contractions per block and candidate
     del Hg
 
     def hbm(name, bytes_, ms, note):
@@ -296,6 +299,11 @@ def kernel_rooflines(ctx, W, X, moments, dev, peak_gbs, sm_mhz):
          "effective_tflops_of_full_product": 2.0 * Tg * Kg * Kg / (t_gram * 1e-3) / 1e12,
          "note": f"one call of sb_calib_gram on the {Tg} x {Kg} MLP input; flops of the upper-triangular "
                  "128 x 128 tiles it computes (the mirror image is copied)"},
+        {"kernel": "full_scores_kernel (tcgen05)", "bound": "tensor", "achieved": full_flops / (t_full * 1e-3) / 1e12,
+         "peak": tpeak, "unit": "TFLOP/s", "frac": full_flops / (t_full * 1e-3) / 1e12 / tpeak,
+         "peak_source": tkind, "ms_per_call": t_full,
+         "note": "one call of sb_block_scores_full on a 14336 x 4096 matrix, 4 candidates; flops of the two "
+                 "128 x 128 x 128 contractions per block and candidate"},
         hbm("first_order_kernel", 4 * n, t_first,
             "one call of sb_first_order_scores, uniformly random levels (weights and gradient, 2 B each)"),
         hbm("reorder_stats_kernel (first-order form)", 4 * n, t_fstats,
