@@ -554,6 +554,12 @@ def run_only(which: str):
             for _ in range(3):
                 ctx.block_scores(W, c, BITS, 128, 128, 128, row_perm=pr, col_perm=pc, err=err,
                                  want_gain=False, W_perm_out=out)
+        elif which == "full_scores":
+            Xs = synth.make_activations(8192, Cc, 7, dev)
+            H = ctx.calib_gram(Xs)
+            err = torch.empty(nb, len(BITS), device=dev)
+            for _ in range(3):
+                ctx.block_scores_full(W, H, BITS, 128, 128, 128, err=err, want_gain=False)
         elif which == "pack":
             level = torch.randint(0, len(BITS), (nb,), device=dev, dtype=torch.uint8)
             for _ in range(3):
@@ -579,7 +585,7 @@ def main():
     ap.add_argument("--no-graphs", action="store_true", help="launch every library call eagerly")
     ap.add_argument("--only", default=None,
                     help="three calls of one library call on one input, then exit (for ncu captures): "
-                         "moments | gram | reorder_stats | scores | gather | pack")
+                         "moments | gram | full_scores | reorder_stats | scores | gather | pack")
     args = ap.parse_args()
     if args.only:
         run_only(args.only)

@@ -166,34 +166,6 @@ __device__ __forceinline__ void load_cols(const __nv_bfloat16* p, bool ok, uint3
 }
 
 // ---- packed fp32 pairs --------------------------------------------------------------------
-// sm_100a executes fma / add / mul on two fp32 values held in one 64-bit register.  The FP32
-// pipe does the same number of lane-operations per clock either way, but the packed form needs
-// half the issue slots, which leaves room for the integer, shuffle and load instructions.
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pk2(float a, float b) {
-    f32x2 r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
-    return r;
-}
-__device__ __forceinline__ void upk2(f32x2 v, float& a, float& b) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
-}
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
-    f32x2 d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
-    f32x2 d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
-    f32x2 d;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-
 // ---- block scores ------------------------------------------------------------------------
 // Every WARP is autonomous.  The matrix is cut into slabs of 16 rows x 128 columns (4 KB),
 // numbered tile by tile, chunk column by chunk column, top to bottom; the slabs are dealt to
