@@ -297,13 +297,14 @@ def kernel_rooflines(ctx, W, X, moments, dev, peak_gbs, sm_mhz):
          "peak": tpeak, "unit": "TFLOP/s", "frac": gram_flops / (t_gram * 1e-3) / 1e12 / tpeak,
          "peak_source": tkind, "ms_per_call": t_gram,
          "effective_tflops_of_full_product": 2.0 * Tg * Kg * Kg / (t_gram * 1e-3) / 1e12,
-         "note": f"one call of sb_calib_gram on the {Tg} x {Kg} MLP input; flops of the upper-triangular "
-                 "128 x 128 tiles it computes (the mirror image is copied)"},
+         "note": f"one call of sb_calib_gram on the {Tg} x {Kg} MLP input (CTA pairs, tcgen05.mma.cta_group::2 on "
+                 "256 x 256 tiles); flops of the upper-triangular 128 x 128 blocks (the mirror image is copied)"},
         {"kernel": "full_scores_kernel (tcgen05)", "bound": "tensor", "achieved": full_flops / (t_full * 1e-3) / 1e12,
          "peak": tpeak, "unit": "TFLOP/s", "frac": full_flops / (t_full * 1e-3) / 1e12 / tpeak,
          "peak_source": tkind, "ms_per_call": t_full,
          "note": "one call of sb_block_scores_full on a 14336 x 4096 matrix, 4 candidates; flops of the two "
-                 "128 x 128 x 128 contractions per block and candidate"},
+                 "128 x 128 x 128 contractions per block and candidate; the quantisation arithmetic in front of "
+                 "the tensor cores (binary64 code decisions) is what bounds it"},
         hbm("first_order_kernel", 4 * n, t_first,
             "one call of sb_first_order_scores, uniformly random levels (weights and gradient, 2 B each)"),
         hbm("reorder_stats_kernel (first-order form)", 4 * n, t_fstats,
