@@ -243,6 +243,26 @@ def pack_blocks(W, bits: Sequence[int], level, block_rows=128, block_cols=128, g
     return packed[:off[nb]].copy(), off, meta
 
 
+def dequant_gemm(X, packed, block_off, meta, level, R, Cc, bits: Sequence[int], block_rows=128,
+                 block_cols=128, group=128):
+    """Y[t][r] = sum_c X[t][c] (lo + scale q)[r][c] on the packed layout (Section 5.3) -> f64 [T][R]."""
+    X = _u16(X)
+    T = X.shape[0]
+    assert X.shape[1] == Cc
+    barr, L = _bits(bits)
+    packed = np.ascontiguousarray(packed, dtype=np.uint32)
+    block_off = np.ascontiguousarray(block_off, dtype=np.int64)
+    meta = np.ascontiguousarray(meta, dtype=np.float32)
+    level = np.ascontiguousarray(level, dtype=np.uint8)
+    Y = np.zeros((T, R), dtype=np.float64)
+    st = lib().sbo_dequant_gemm(_p(X), C.c_int64(T), C.c_int64(Cc), _p(packed), _p(block_off), _p(meta),
+                                _p(level), C.c_int64(R), C.c_int64(Cc), C.c_int(block_rows),
+                                C.c_int(block_cols), C.c_int(group), barr, C.c_int(L), _p(Y))
+    if st != OK:
+        raise ValueError(f"sbo_dequant_gemm status {st}")
+    return Y
+
+
 class StepReport(C.Structure):
     _fields_ = [("cap_bits", C.c_int64), ("used_in", C.c_int64), ("used_out", C.c_int64),
                 ("expansion", C.c_int32), ("moved", C.c_int32),

@@ -865,3 +865,46 @@ int sbo_pack_blocks(const uint16_t* W, int64_t R, int64_t C, int64_t ldw,
     free(v); free(code);
     return SBO_OK;
 }
+
+/* Fused dequantisation + matrix product on the packed format (Section 5.3, Table 4: the
+ * mixed-precision kernel dequantises tile by tile, one bitwidth per tile, and multiplies):
+ *     Y[t][r] = sum_c X[t][c] * What[r][c],   What[r][c] = lo[r][g(c)] + scale[r][g(c)] * q[r][c],
+ * q read back from the bit stream sbo_pack_blocks wrote (code k of a block in bits
+ * [k b, (k+1) b) of its little-endian word stream, block-row-major), scale and lo the fp32
+ * metadata of (row, group).  Rows and columns are those of the packed (permuted) layout.
+ * Plain definition in binary64: decode every code, form What, accumulate the dot products.
+ * X: bf16 [T][C] (ldx), Y: binary64 [T][R]. */
+int sbo_dequant_gemm(const uint16_t* X, int64_t T, int64_t ldx, const uint32_t* packed,
+                     const int64_t* block_off_words, const float* meta, const uint8_t* level,
+                     int64_t R, int64_t C, int br, int bc, int group, const int* bits, int L,
+                     double* Y) {
+    if (!check_bits(bits, L)) return SBO_ERR_INVALID;
+    if (br <= 0 || bc <= 0 || group <= 0 || R % br || C % bc || bc % group) return SBO_ERR_SHAPE;
+    const int64_t nbc = C / bc, ngc = C / group;
+    double* what = (double*)malloc(sizeof(double) * (size_t)C);
+    for (int64_t r = 0; r < R; ++r) {
+        const int64_t bi = r / br;
+        const int rr = (int)(r % br);
+        for (int64_t j = 0; j < C; ++j) {
+            const int64_t bj = j / bc;
+            const int64_t blk = bi * nbc + bj;
+            if (level[blk] >= L) { free(what); return SBO_ERR_INVALID; }
+            const int b = bits[level[blk]];
+            const uint32_t* in = packed + block_off_words[blk];
+            const int64_t e = (int64_t)rr * bc + (j % bc);       /* element index in the block */
+            const int64_t bit = e * b;
+            uint64_t word = in[bit / 32];
+            if ((bit % 32) + b > 32) word |= (uint64_t)in[bit / 32 + 1] << 32;
+            const uint32_t q = (uint32_t)((word >> (bit % 32)) & ((1u << b) - 1u));
+            const int64_t gi = r * ngc + j / group;
+            what[j] = (double)meta[2 * gi + 1] + (double)meta[2 * gi] * (double)q;
+        }
+        for (int64_t t = 0; t < T; ++t) {
+            double acc = 0.0;
+            for (int64_t j = 0; j < C; ++j) acc += sbo_bf16_to_f64(X[t * ldx + j]) * what[j];
+            Y[t * R + r] = acc;
+        }
+    }
+    free(what);
+    return SBO_OK;
+}
