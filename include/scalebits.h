@@ -170,6 +170,25 @@ sb_status sb_pack_blocks(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_t C, 
                          uint32_t* packed, int64_t packed_capacity_words,
                          int64_t* block_off_words, float* meta);
 
+/* Fused mixed-precision dequantisation + matrix product on the output of sb_pack_blocks
+ * (Section 5.3 and Table 4: dequantise tile by tile, one bitwidth per tile, and multiply):
+ *     Y[t][r] = sum_c X[t][c] * (lo[r][g(c)] + scale[r][g(c)] * q[r][c])
+ * in the packed (permuted) row and column order: X's columns are the packed columns, Y's
+ * columns the packed rows.  The contraction runs on the integer codes (exact in bf16) on the
+ * tensor cores with fp32 accumulation, one 128 x 128 block at a time, and scale and lo are
+ * applied per row and block in fp32; nothing else is rounded.
+ *   - X: device bf16 [T][C], leading dimension ldx >= C; T >= 1 (tokens are processed in
+ *     slices of 32; decode batches are the intended use).
+ *   - packed, block_off_words, meta, level, bits: as written by / given to sb_pack_blocks;
+ *     packed 16-byte aligned.  block_rows = block_cols = group = 128 is required.
+ *   - Y: device fp32 [T][R], leading dimension ldy >= R, overwritten.
+ * A pipeline wait that does not complete within 2 s latches SB_ERR_TIMEOUT.  Asynchronous. */
+sb_status sb_dequant_gemm(sb_ctx* ctx, const void* X_bf16, int64_t T, int64_t ldx,
+                          const uint32_t* packed, const int64_t* block_off_words, const float* meta,
+                          const uint8_t* level, int64_t R, int64_t C,
+                          int block_rows, int block_cols, int group, const int* bits, int n_bits,
+                          float* Y, int64_t ldy);
+
 /* Full calibration second-moment matrix on the tensor cores (Section 3.2: sb_calib_moments
  * returns the diagonal of this matrix; a sensitivity that keeps the cross terms between input
  * channels needs all of it):

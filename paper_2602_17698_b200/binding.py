@@ -25,7 +25,7 @@ EXPORTS = ["sb_create", "sb_destroy", "sb_sync", "sb_last_error", "sb_kernel_lau
            "sb_expand_segment_perm", "sb_block_scores", "sb_allocate_bits", "sb_pack_blocks",
            "sb_calib_moments_noalloc", "sb_first_order_scores", "sb_exchange_step",
            "sb_reorder_channels_first_order", "sb_calib_gram",
-           "sb_block_scores_full"]
+           "sb_block_scores_full", "sb_dequant_gemm"]
 
 
 class SbError(RuntimeError):
@@ -99,6 +99,8 @@ def lib() -> C.CDLL:
         L.sb_calib_gram.argtypes = [vp, vp, i64, i64, i64, vp, i32, f32]
         L.sb_block_scores_full.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp, i32, i32, i32,
                                            C.POINTER(C.c_int), i32, vp, vp, vp]
+        L.sb_dequant_gemm.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, i64, i64, i32, i32, i32,
+                                      C.POINTER(C.c_int), i32, vp, i64]
         L.sb_reorder_channels_first_order.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, i32, vp, vp, i32,
                                                       i64, i64, vp, vp]
         for name in EXPORTS:
@@ -337,6 +339,23 @@ class Context:
             block_rows, block_cols, group, barr, L, _ptr(level, torch.uint8), _ptr(packed),
             packed.numel(), _ptr(block_off, torch.int64), _ptr(meta, torch.float32)))
         return packed, block_off, meta
+
+
+    def dequant_gemm(self, X: torch.Tensor, packed: torch.Tensor, block_off: torch.Tensor, meta: torch.Tensor,
+                     level: torch.Tensor, R: int, Cc: int, bits: Sequence[int], block_rows: int = 128,
+                     block_cols: int = 128, group: int = 128, Y: Optional[torch.Tensor] = None):
+        """Y[t][r] = sum_c X[t][c] (lo + scale q)[r][c] on the output of pack_blocks -> fp32 [T][R]."""
+        T, Kx, ldx = _mat(X)
+        if Kx != Cc:
+            raise ValueError("X must have one column per packed column")
+        barr, L = _bits(bits)
+        if Y is None:
+            Y = torch.empty((T, R), dtype=torch.float32, device=X.device)
+        self._check(lib().sb_dequant_gemm(
+            self._h, _ptr(X), T, ldx, _ptr(packed), _ptr(block_off, torch.int64), _ptr(meta, torch.float32),
+            _ptr(level, torch.uint8), R, Cc, block_rows, block_cols, group, barr, L,
+            _ptr(Y, torch.float32), Y.stride(0)))
+        return Y
 
 
 def calib_moments_noalloc(X: torch.Tensor, sumsq: Optional[torch.Tensor] = None,

@@ -87,7 +87,7 @@ constexpr int SB_STATS_TILES = 8192;     // 128-wide tiles per axis a reorder ca
 constexpr int SB_MOMENT_CHUNKS = 4096;   // column chunks of 256 a moments call may have (K <= 1M)
 
 enum SbKernelId { SBK_MOMENTS = 1, SBK_STATS, SBK_SCORES, SBK_GATHER, SBK_ARGSORT, SBK_SCAN,
-                  SBK_SORT, SBK_ALLOC, SBK_PACK };
+                  SBK_SORT, SBK_ALLOC, SBK_PACK, SBK_GEMM };
 
 // ---- device helpers ----------------------------------------------------------------
 #ifdef __CUDACC__

@@ -165,4 +165,16 @@ def expected_channel_std(channels: int, seed: int, device="cpu") -> torch.Tensor
     return torch.exp(torch.randn((channels,), generator=g, device=device, dtype=torch.float32))
 
 
+def table4_levels(n_blocks: int, seed: int):
+    """Block levels of the mixed-precision kernel benchmark (Table 4): 40 % / 40 % / 20 % of the
+    blocks at the first / second / third candidate (2 / 4 / 8 bits: 4 bits on average), in a seeded
+    random arrangement.  numpy uint8 [n_blocks]."""
+    import numpy as np
+    n0 = (2 * n_blocks) // 5
+    n1 = (2 * n_blocks) // 5
+    lv = np.concatenate([np.zeros(n0, np.uint8), np.ones(n1, np.uint8), np.full(n_blocks - n0 - n1, 2, np.uint8)])
+    np.random.default_rng(seed).shuffle(lv)
+    return lv
+
+
 __all__ = [n for n in dir() if not n.startswith("_") and n not in ("math", "torch")]
