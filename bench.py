@@ -312,6 +312,69 @@ def kernel_rooflines(ctx, W, X, moments, dev, peak_gbs, sm_mhz):
     ]
 
 
+def dequant_gemm_times(ctx, dev, peak_gbs):
+    """sb_dequant_gemm on the workload of the paper's kernel table (Table 4): an 8192 x 8192 matrix,
+    16 and 32 tokens, all blocks at 4 bits and the 40 / 40 / 20 % mix of 2 / 4 / 8 bits (4 bits on
+    average).  Six packed copies in rotation (216 MB > L2), so every call streams its codes from
+    HBM; CUDA events on the context's stream around one CUDA graph of 12 calls."""
+    import torch
+    import numpy as np
+    from paper_2602_17698_b200 import synth
+    R = Cc = 8192
+    nb = (R // 128) * (Cc // 128)
+    bits = [2, 4, 8]
+    W = synth.make_weight(R, Cc, 4242, dev)
+    paper_us = {("int4", 16): 57.8, ("int4", 32): 65.0, ("mix", 16): 58.0, ("mix", 32): 65.9}
+    out = []
+    for kind in ("int4", "mix"):
+        sets = []
+        for k in range(6):
+            lv = np.ones(nb, np.uint8) if kind == "int4" else synth.table4_levels(nb, 100 + k)
+            level = torch.from_numpy(lv).to(dev)
+            packed, off, meta = ctx.pack_blocks(W, bits, level, 128, 128, 128)
+            ctx.sync()
+            words = int(off[-1].item())
+            sets.append((packed[:words + 4].clone(), off, meta, level, words))
+            del packed
+        for T in (16, 32):
+            X = synth.make_activations(T, Cc, 77 + T, dev)
+            Y = torch.empty((T, R), dtype=torch.float32, device=dev)
+            def call(i):
+                pk, off, meta, level, _ = sets[i % 6]
+                ctx.dequant_gemm(X, pk, off, meta, level, R, Cc, bits, Y=Y)
+            for i in range(6):
+                call(i)
+            ctx.stream.synchronize()
+            # the 12 calls as one CUDA graph: three short launches per call would otherwise be paced
+            # by the host
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=ctx.stream):
+                for i in range(12):
+                    call(i)
+            g.replay()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(ctx.stream):
+                a.record()
+                g.replay()
+                b.record()
+            b.synchronize()
+            ms = a.elapsed_time(b) / 12
+            del g
+            bytes_ = sets[0][4] * 4 + R * (Cc // 128) * 8 + T * Cc * 2 + T * R * 4
+            gbs = bytes_ / (ms * 1e-3) / 1e9
+            out.append({"kernel": "dequant_gemm_kernel (tcgen05) + dq_prepare_x_kernel + dq_reduce_kernel",
+                        "bound": "hbm", "achieved": gbs, "peak": peak_gbs, "unit": "GB/s", "frac": gbs / peak_gbs,
+                        "ms_per_call": ms, "us_per_call": ms * 1e3, "algorithmic_bytes": bytes_,
+                        "workload": f"8192 x 8192, {T} tokens, " + ("all blocks 4 bits" if kind == "int4"
+                                                                    else "40/40/20 % of 2/4/8 bits"),
+                        "paper_table_4_us": paper_us[(kind, T)],
+                        "note": "one call of sb_dequant_gemm (three launches); packed codes + scale / minimum "
+                                "metadata + activations read, outputs written; the paper's figure is its own "
+                                "kernel on its own GPU: context, not a comparison on equal hardware"})
+        del sets
+    return out
+
+
 def full_model_times(ctx, dev):
     """configs[2]: 32 layers of the 8B shape searched as ONE model (residual-stream permutation
     shared by all layers, one global allocation over N = 425,984 blocks per budget), budgets
@@ -487,6 +550,8 @@ def run_cuda(args):
                      "pack": w_bytes / (stage_ms["pack"] * 1e-3) / 1e9}
         sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
         kernels = kernel_rooflines(ctx, W, X, ws.moments, dev, peak, sm_mhz)
+        if world == 1:
+            kernels += dequant_gemm_times(ctx, dev, peak)
         full_model = None
         if world == 1 and not args.no_full_model:
             del hW, hX                                   # pinned copies of the layer, if any
@@ -561,6 +626,18 @@ def run_only(which: str):
             err = torch.empty(nb, len(BITS), device=dev)
             for _ in range(3):
                 ctx.block_scores_full(W, H, BITS, 128, 128, 128, err=err, want_gain=False)
+        elif which == "dequant_gemm":
+            import numpy as np
+            Rq = Cq = 8192
+            nbq = (Rq // 128) * (Cq // 128)
+            Wq = synth.make_weight(Rq, Cq, 4242, dev)
+            sets = []
+            for k in range(5):                           # 180 MB of packed copies: larger than L2
+                lv = torch.from_numpy(synth.table4_levels(nbq, 100 + k)).to(dev)
+                sets.append(ctx.pack_blocks(Wq, [2, 4, 8], lv, 128, 128, 128) + (lv,))
+            Xq = synth.make_activations(32, Cq, 109, dev)
+            for pk, off, meta, lv in sets:
+                ctx.dequant_gemm(Xq, pk, off, meta, lv, Rq, Cq, [2, 4, 8])
         elif which == "pack":
             level = torch.randint(0, len(BITS), (nb,), device=dev, dtype=torch.uint8)
             for _ in range(3):
@@ -586,7 +663,7 @@ def main():
     ap.add_argument("--no-graphs", action="store_true", help="launch every library call eagerly")
     ap.add_argument("--only", default=None,
                     help="three calls of one library call on one input, then exit (for ncu captures): "
-                         "moments | gram | full_scores | reorder_stats | scores | gather | pack")
+                         "moments | gram | full_scores | dequant_gemm | reorder_stats | scores | gather | pack")
     args = ap.parse_args()
     if args.only:
         run_only(args.only)

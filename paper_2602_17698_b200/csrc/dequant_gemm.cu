@@ -16,11 +16,11 @@
 // kernel first writes X in each of those column orders (and the per-block column sums of X).
 //
 // Grid: (R / 128 row tiles) x (S column segments), two CTAs per SM.  Per CTA:
-//   warps 4-7 (thread = weight row): cp.async of the row's own codes and of the block's slice
+//   warps 4-11 (thread = 32 columns of a weight row): cp.async of its own codes and of the block's slice
 //     of X (straight into the K-major 128-byte-swizzle operand layout) three blocks ahead;
 //     unpack half a block (64 columns) at a time into one of two shared-memory operand tiles,
 //     fence.proxy.async, mbarrier arrive;
-//   warp 8 (one thread): 4 tcgen05.mma (K = 16) per half block into one of two TMEM
+//   warp 12 (one thread): 4 tcgen05.mma (K = 16) per half block into one of two TMEM
 //     accumulators of N columns, tcgen05.commit to free operand tiles, X slices and to
 //     publish accumulators;
 //   warps 0-3 (thread = weight row = TMEM lane): tcgen05.ld of the block's accumulator,
@@ -41,12 +41,12 @@ constexpr int DQ_CODE_STAGE = 2048 * 8;     // bytes of codes of one block at 8 
 constexpr int DQ_A_BYTES = DQ_M * 128;      // one operand tile: 128 rows x 64 bf16
 constexpr int DQ_MAX_T = 32;
 constexpr int DQ_X_STAGE = DQ_MAX_T * DQ_KB * 2;        // X slice of a block: tokens x 128 bf16
-constexpr int DQ_CONV_WARPS = 4, DQ_EPI_WARPS = 4;
+constexpr int DQ_CONV_WARPS = 8, DQ_EPI_WARPS = 4;    // unpacking thread = 32 columns of a weight row
 constexpr int DQ_THREADS = (DQ_EPI_WARPS + DQ_CONV_WARPS + 1) * 32;
 constexpr int DQ_MAX_SEG_BLOCKS = 32;       // column blocks per segment (their column sums sit in shared memory)
 constexpr int DQ_ORDERS = 5;                // column orders of X: identity, b = 1, 2, 4, 8
 constexpr int DQ_SMEM = DQ_RING * (DQ_CODE_STAGE + DQ_X_STAGE) + 2 * DQ_A_BYTES +
-                        DQ_MAX_SEG_BLOCKS * DQ_MAX_T * 4 + 1024 /* alignment */ + 256 /* barriers */;
+                        DQ_MAX_SEG_BLOCKS * DQ_MAX_T * 4 + 1024 /* alignment */ + 512 /* barriers, block table */;
 constexpr unsigned long long DQ_WAIT_NS = 2000ull * 1000 * 1000;
 
 // candidate bitwidths, four bits each
@@ -164,32 +164,32 @@ __global__ void dq_prepare_x_kernel(const __nv_bfloat16* __restrict__ X, int64_t
 }
 
 // ---- unpacking ---------------------------------------------------------------------------------
-// One half row (64 codes = 2 B words) of b-bit codes, b in {1, 2, 4, 8}, from shared memory into
-// the operand tile: 8 chunks of 8 bf16.  `src` points at the row's codes (16 B bytes, 16-byte
-// chunks XOR-swizzled by `xr` over the row's B chunks so that neighbouring rows read different
-// banks), `dst` at the row's 128 bytes of the tile, `r7` = row & 7 (the tile's swizzle).
+// 32 codes (B words) of one weight row, b in {1, 2, 4, 8}, from shared memory into the operand
+// tile: 4 chunks of 8 bf16.  `src` points at the row's codes (16 B bytes; its 16-byte chunks are
+// XOR-swizzled by `xr` so that neighbouring rows read different banks), `qi` = which 32 codes of
+// the row (0..3), `dst` at the row's 128 bytes of the tile, `r7` = row & 7 (the tile's swizzle).
 template <int B>
-__device__ __forceinline__ void dq_unpack_half(const unsigned char* src, int half, int xr, unsigned char* dst, int r7) {
+__device__ __forceinline__ void dq_unpack32(const unsigned char* src, int qi, int xr, unsigned char* dst, int r7) {
     constexpr int N = 32 / B;                            // codes per word
-    constexpr int WORDS = 2 * B;                         // words per half row
     constexpr unsigned MASK = ((1u << B) - 1u) * 0x00010001u;
     const __nv_bfloat162 c128 = __float2bfloat162_rn(128.f);
-    uint32_t w[WORDS];
+    uint32_t w[B];
     if constexpr (B == 1) {
-        // the row is one 16-byte chunk: this half is 8 bytes of it
-        const uint2 v = *reinterpret_cast<const uint2*>(src + 8 * half);
+        w[0] = *reinterpret_cast<const uint32_t*>(src + 4 * qi);
+    } else if constexpr (B == 2) {
+        const uint2 v = *reinterpret_cast<const uint2*>(src + (((qi >> 1) ^ xr) << 4) + 8 * (qi & 1));
         w[0] = v.x; w[1] = v.y;
     } else {
 #pragma unroll
-        for (int k = 0; k < WORDS / 4; ++k) {
-            const int chunk = half * (WORDS / 4) + k;    // 16-byte chunk of the row
+        for (int k = 0; k < B / 4; ++k) {
+            const int chunk = qi * (B / 4) + k;          // 16-byte chunk of the row
             const uint4 v = *reinterpret_cast<const uint4*>(src + ((chunk ^ xr) << 4));
             w[4 * k] = v.x; w[4 * k + 1] = v.y; w[4 * k + 2] = v.z; w[4 * k + 3] = v.w;
         }
     }
-    uint32_t out[32];                                    // 64 bf16
+    uint32_t out[16];                                    // 32 bf16
 #pragma unroll
-    for (int m = 0; m < WORDS; ++m) {
+    for (int m = 0; m < B; ++m) {
 #pragma unroll
         for (int s = 0; s < N / 2; ++s) {
             const uint32_t v = (w[m] >> (B * s)) & MASK;
@@ -205,26 +205,27 @@ __device__ __forceinline__ void dq_unpack_half(const unsigned char* src, int hal
             out[(N / 2) * m + s] = bits;
         }
     }
+    const int c0 = 4 * (qi & 1);                         // chunk of the half-block tile
 #pragma unroll
-    for (int c = 0; c < 8; ++c)
-        *reinterpret_cast<uint4*>(dst + ((c ^ r7) << 4)) = make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
+    for (int c = 0; c < 4; ++c)
+        *reinterpret_cast<uint4*>(dst + (((c0 + c) ^ r7) << 4)) = make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
 }
 
 // any other bitwidth below 8: code k of the row at bit k b of its stream, columns in their own order
-__device__ __forceinline__ void dq_unpack_half_generic(const unsigned char* src, int b, int half, unsigned char* dst,
-                                                       int r7) {
+__device__ __forceinline__ void dq_unpack32_generic(const unsigned char* src, int b, int qi, unsigned char* dst, int r7) {
     const uint32_t* words = reinterpret_cast<const uint32_t*>(src);
     const uint32_t mask = (1u << b) - 1u;
     const __nv_bfloat162 c128 = __float2bfloat162_rn(128.f);
+    const int c0 = 4 * (qi & 1);
 #pragma unroll 1
-    for (int c = 0; c < 8; ++c) {
+    for (int c = 0; c < 4; ++c) {
         uint32_t o[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             uint32_t pair = 0;
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const int bit = (DQ_HALF * half + 8 * c + 2 * k + h) * b;
+                const int bit = (32 * qi + 8 * c + 2 * k + h) * b;
                 const int wi = bit >> 5;
                 // the row's stream is 4 b words long; the funnel shift may look one word past a code
                 // that ends at the stream's end, so that word is clamped to the last one
@@ -233,7 +234,7 @@ __device__ __forceinline__ void dq_unpack_half_generic(const unsigned char* src,
             }
             o[k] = u32(__hsub2(b162(pair | 0x43004300u), c128));
         }
-        *reinterpret_cast<uint4*>(dst + ((c ^ r7) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+        *reinterpret_cast<uint4*>(dst + (((c0 + c) ^ r7) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
     }
 }
 
@@ -270,6 +271,10 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
     unsigned long long* d_empty = d_full + 2;              // [2] drained -> MMA
     unsigned* tmem_slot = reinterpret_cast<unsigned*>(d_empty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    // per block of the segment: first word of its codes (blocks are below 2^32 words apart from the
+    // segment's first) and its bitwidth, so that the loop below has no dependent global loads
+    unsigned* blk_word = tmem_slot + 4;                 // [DQ_MAX_SEG_BLOCKS]
+    unsigned char* blk_bits = reinterpret_cast<unsigned char*>(blk_word + DQ_MAX_SEG_BLOCKS);   // [DQ_MAX_SEG_BLOCKS]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int TMEM_COLS = 2 * NT < 32 ? 32 : 2 * NT;
 
@@ -293,55 +298,72 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
                      "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // the segment's column sums of X
+    // the segment's column sums of X and its block table
     for (int i = threadIdx.x; i < nblk * NT; i += DQ_THREADS) xs[i] = a.xsum[(int64_t)j0 * NT + i];
+    const int64_t blk0 = (int64_t)bi * a.nbc + j0;
+    const int64_t word0 = a.block_off[blk0];
+    if (threadIdx.x < nblk) {
+        blk_word[threadIdx.x] = (unsigned)(a.block_off[blk0 + threadIdx.x] - word0);
+        blk_bits[threadIdx.x] = (unsigned char)dq_bits(a.bits, a.level[blk0 + threadIdx.x]);
+    }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const unsigned tmem_base = *tmem_slot;
 
     if (warp >= DQ_EPI_WARPS && warp < DQ_EPI_WARPS + DQ_CONV_WARPS) {
-        // ---- loaders / unpackers: thread = weight row r of the tile ---------------------------------
-        const int r = threadIdx.x - DQ_EPI_WARPS * 32;
+        // ---- loaders / unpackers: thread = 32 columns (quarter hq of the current half block) of
+        // weight row r of the tile ----------------------------------------------------------------------
+        const int ct = threadIdx.x - DQ_EPI_WARPS * 32;
+        const int r = ct & (DQ_M - 1), hq = ct >> 7;
         const int r7 = r & 7;
-        // cp.async of block jj of the segment into ring stage jj % DQ_RING: the row's codes and this
-        // thread's share of the X slice, the latter straight into the swizzled operand layout
+        // this thread's share of a block's X slice: 16-byte chunks ct, ct + 256, ... of the slice
+        // (token, chunk in the row), straight into the swizzled operand layout
+        unsigned xdst[NT / 16];
+        const __nv_bfloat16* xsrc[NT / 16];
+#pragma unroll
+        for (int i = 0; i < NT / 16; ++i) {
+            const int k = ct + 256 * i;
+            const int t = k >> 4, cc = k & 15;
+            const int panel = cc >> 3, c8 = cc & 7;      // K half, chunk inside its 128 bytes
+            xdst[i] = (unsigned)(panel * (NT * 128) + t * 128 + ((c8 ^ (t & 7)) << 4));
+            xsrc[i] = a.xp + (int64_t)t * a.C + (int64_t)j0 * DQ_KB + cc * 8;
+        }
+        // cp.async of block jj of the segment into ring stage jj % DQ_RING.  A thread copies the
+        // chunks of its row's codes that it will read itself (for b = 4, 8 those of its two
+        // quarters; otherwise the whole row, twice over with its partner), so waiting for its own
+        // copies is all the synchronisation the codes need.
         auto issue = [&](int jj) {
             const int st = jj % DQ_RING;
-            const int64_t blk = (int64_t)bi * a.nbc + j0 + jj;
-            const int b = dq_bits(a.bits, a.level[blk]);
-            const unsigned char* src = reinterpret_cast<const unsigned char*>(a.packed + a.block_off[blk]) + r * 16 * b;
+            const int b = blk_bits[jj];
+            const unsigned char* src = reinterpret_cast<const unsigned char*>(a.packed + word0 + blk_word[jj]) + r * 16 * b;
             const unsigned dstc = dq_smem_u32(code_ring + st * DQ_CODE_STAGE + r * 16 * b);
             // chunk swizzle over the row's b chunks (power-of-two b only): rows that share a bank
             // group get different chunk orders
             const int xr = (b == 2) ? ((r >> 2) & 1) : (b == 4) ? ((r >> 1) & 3) : (b == 8) ? r7 : 0;
-            for (int k = 0; k < b; ++k) dq_cp_async16(dstc + ((k ^ xr) << 4), src + (k << 4));
-            const __nv_bfloat16* xsrc = a.xp + (int64_t)dq_order(b) * NT * a.C + (int64_t)(j0 + jj) * DQ_KB;
+            if (b == 4) {
+                dq_cp_async16(dstc + ((hq ^ xr) << 4), src + (hq << 4));
+                dq_cp_async16(dstc + (((2 + hq) ^ xr) << 4), src + ((2 + hq) << 4));
+            } else if (b == 8) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int ch = (k >> 1) * 4 + 2 * hq + (k & 1);
+                    dq_cp_async16(dstc + ((ch ^ xr) << 4), src + (ch << 4));
+                }
+            } else {
+                for (int k = 0; k < b; ++k) dq_cp_async16(dstc + ((k ^ xr) << 4), src + (k << 4));
+            }
+            const int64_t xoff = (int64_t)dq_order(b) * NT * a.C + (int64_t)jj * DQ_KB;
             const unsigned dstx = dq_smem_u32(x_ring + st * DQ_X_STAGE);
 #pragma unroll
-            for (int i = 0; i < NT / 8; ++i) {
-                const int k = r + 128 * i;                   // 16-byte chunk of the slice: token, chunk in the row
-                const int t = k >> 4, cc = k & 15;
-                const int panel = cc >> 3, c8 = cc & 7;      // K half, chunk inside its 128 bytes
-                dq_cp_async16(dstx + panel * (NT * 128) + t * 128 + ((c8 ^ (t & 7)) << 4),
-                              xsrc + (int64_t)t * a.C + cc * 8);
-            }
+            for (int i = 0; i < NT / 16; ++i) dq_cp_async16(dstx + xdst[i], xsrc[i] + xoff);
         };
         bool ok = true;
         for (int jj = 0; jj < 2 && jj < nblk; ++jj) { issue(jj); dq_cp_commit(); }
         if (nblk < 2) dq_cp_commit();
         for (int j = 0; j < nblk && ok; ++j) {
-            // block j + 2 into the stage block j - 1 used: its X slice must have been consumed
-            if (j + 2 < nblk) {
-                if (j >= 1) ok = dq_mbar_wait(dq_smem_u32(x_empty + (j + 2) % DQ_RING), (unsigned)((j - 1) / DQ_RING) & 1u, abort_flag);
-                if (ok) issue(j + 2);
-            }
-            dq_cp_commit();                                   // (possibly empty) group: keeps the count uniform
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            dq_cp_wait<2>();                                  // block j has landed (this thread's copies)
-            const int64_t blk = (int64_t)bi * a.nbc + j0 + j;
-            const int b = dq_bits(a.bits, a.level[blk]);
+            dq_cp_wait<1>();                                  // block j has landed (this thread's copies)
+            const int b = blk_bits[j];
             const unsigned char* src = code_ring + (j % DQ_RING) * DQ_CODE_STAGE + r * 16 * b;
             const int xr = (b == 2) ? ((r >> 2) & 1) : (b == 4) ? ((r >> 1) & 3) : (b == 8) ? r7 : 0;
             for (int h = 0; h < 2 && ok; ++h) {
@@ -349,17 +371,28 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
                 ok = __all_sync(0xffffffffu, dq_mbar_wait(dq_smem_u32(a_empty + buf), ((unsigned)(u >> 1) & 1u) ^ 1u, abort_flag));
                 if (!ok) break;
                 unsigned char* dst = a_tiles + buf * DQ_A_BYTES + r * 128;
+                const int qi = 2 * h + hq;
                 switch (b) {                                  // uniform over the CTA
-                    case 1: dq_unpack_half<1>(src, h, xr, dst, r7); break;
-                    case 2: dq_unpack_half<2>(src, h, xr, dst, r7); break;
-                    case 4: dq_unpack_half<4>(src, h, xr, dst, r7); break;
-                    case 8: dq_unpack_half<8>(src, h, xr, dst, r7); break;
-                    default: dq_unpack_half_generic(src, b, h, dst, r7); break;
+                    case 1: dq_unpack32<1>(src, qi, xr, dst, r7); break;
+                    case 2: dq_unpack32<2>(src, qi, xr, dst, r7); break;
+                    case 4: dq_unpack32<4>(src, qi, xr, dst, r7); break;
+                    case 8: dq_unpack32<8>(src, qi, xr, dst, r7); break;
+                    default: dq_unpack32_generic(src, b, qi, dst, r7); break;
                 }
                 // the tensor cores read shared memory through the async proxy (the X slice of this
                 // block included: every thread's copies were waited for above)
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 dq_mbar_arrive(dq_smem_u32(a_full + buf));
+                if (h == 0) {
+                    // block j + 2 into the stage block j - 1 used: its X slice must have been consumed
+                    // (that contraction was issued before this half was unpacked)
+                    if (j + 2 < nblk) {
+                        if (j >= 1) ok = dq_mbar_wait(dq_smem_u32(x_empty + (j + 2) % DQ_RING), (unsigned)((j - 1) / DQ_RING) & 1u, abort_flag);
+                        if (ok) issue(j + 2);
+                    }
+                    dq_cp_commit();                           // (possibly empty) group: keeps the count uniform
+                    ok = __all_sync(0xffffffffu, ok);
+                }
             }
         }
         dq_cp_wait<0>();
