@@ -15,14 +15,20 @@
 // contraction does not care about the order of K as long as X uses the same one, so a small
 // kernel first writes X in each of those column orders (and the per-block column sums of X).
 //
+// The unpacked codes never touch shared memory: bf16 codes are four times the packed bytes at
+// 4 bits, and writing them to a shared-memory operand tile and reading them back by the tensor
+// cores made shared-memory bandwidth the bound.  They go from registers to TENSOR MEMORY
+// (tcgen05.st, thread = weight row = TMEM lane) and the contraction takes its A operand from
+// there; only the few-token slice of X is a shared-memory operand.
+//
 // Grid: (R / 128 row tiles) x (S column segments), two CTAs per SM.  Per CTA:
-//   warps 4-11 (thread = 32 columns of a weight row): cp.async of its own codes and of the block's slice
-//     of X (straight into the K-major 128-byte-swizzle operand layout) three blocks ahead;
-//     unpack half a block (64 columns) at a time into one of two shared-memory operand tiles,
-//     fence.proxy.async, mbarrier arrive;
-//   warp 12 (one thread): 4 tcgen05.mma (K = 16) per half block into one of two TMEM
-//     accumulators of N columns, tcgen05.commit to free operand tiles, X slices and to
-//     publish accumulators;
+//   warps 4-11 (thread = 2 x 32 columns of a weight row): cp.async of its own codes and of the
+//     block's slice of X (straight into the K-major 128-byte-swizzle operand layout) three blocks
+//     ahead; unpack the block into registers, tcgen05.st into one of two 64-column TMEM operand
+//     buffers, tcgen05.wait::st, fences, mbarrier arrive;
+//   warp 12 (one thread): 8 tcgen05.mma (K = 16, A from TMEM, B = X slice from shared memory) per
+//     block into one of two TMEM accumulators of N columns, tcgen05.commit to free the operand
+//     buffer and the X slice and to publish the accumulator;
 //   warps 0-3 (thread = weight row = TMEM lane): tcgen05.ld of the block's accumulator,
 //     y += scale * acc + lo * colsum(X) in fp32 registers; at the end the segment's partial
 //     sums go to scratch (or to Y when there is one segment) and a second kernel adds the
@@ -35,18 +41,18 @@ namespace {
 
 constexpr int DQ_M = 128;                   // weight rows per CTA = block rows
 constexpr int DQ_KB = 128;                  // block columns
-constexpr int DQ_HALF = 64;                 // columns per operand tile (one 128-byte swizzle atom)
-constexpr int DQ_RING = 3;                  // blocks in flight (codes + X slice)
+constexpr int DQ_RING = 4;                  // blocks in flight (codes + X slice)
 constexpr int DQ_CODE_STAGE = 2048 * 8;     // bytes of codes of one block at 8 bits
-constexpr int DQ_A_BYTES = DQ_M * 128;      // one operand tile: 128 rows x 64 bf16
+constexpr int DQ_A_COLS = DQ_KB / 2;         // TMEM columns of a block's codes: two bf16 per 32-bit column
 constexpr int DQ_MAX_T = 32;
 constexpr int DQ_X_STAGE = DQ_MAX_T * DQ_KB * 2;        // X slice of a block: tokens x 128 bf16
 constexpr int DQ_CONV_WARPS = 8, DQ_EPI_WARPS = 4;    // unpacking thread = 32 columns of a weight row
 constexpr int DQ_THREADS = (DQ_EPI_WARPS + DQ_CONV_WARPS + 1) * 32;
 constexpr int DQ_MAX_SEG_BLOCKS = 32;       // column blocks per segment (their column sums sit in shared memory)
 constexpr int DQ_ORDERS = 5;                // column orders of X: identity, b = 1, 2, 4, 8
-constexpr int DQ_SMEM = DQ_RING * (DQ_CODE_STAGE + DQ_X_STAGE) + 2 * DQ_A_BYTES +
-                        DQ_MAX_SEG_BLOCKS * DQ_MAX_T * 4 + 1024 /* alignment */ + 512 /* barriers, block table */;
+constexpr int DQ_SMEM = DQ_RING * (DQ_CODE_STAGE + DQ_X_STAGE) + DQ_MAX_SEG_BLOCKS * DQ_MAX_T * 4 +
+                        1024 /* alignment */ + 512 /* barriers, block table */;
+constexpr int DQ_TMEM_COLS = 256;           // accumulators in columns [0, 64), operand buffers at 64 and 128
 constexpr unsigned long long DQ_WAIT_NS = 2000ull * 1000 * 1000;
 
 // candidate bitwidths, four bits each
@@ -111,13 +117,22 @@ __device__ __forceinline__ unsigned long long dq_desc(unsigned addr) {
 __device__ __forceinline__ unsigned dq_idesc(int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(DQ_M >> 4) << 24);
 }
-__device__ __forceinline__ void dq_mma(unsigned tmem_d, unsigned long long a, unsigned long long b, unsigned idesc,
+// A (128 rows x 16 columns of bf16 = 8 TMEM columns, row = lane) from tensor memory, B from shared memory
+__device__ __forceinline__ void dq_mma(unsigned tmem_d, unsigned tmem_a, unsigned long long b, unsigned idesc,
                                        unsigned acc) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(a), "l"(b), "r"(idesc), "r"(acc)
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(b), "r"(idesc), "r"(acc)
+        : "memory");
+}
+__device__ __forceinline__ void dq_tmem_st16(unsigned taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
         : "memory");
 }
 __device__ __forceinline__ void dq_commit(unsigned bar) {
@@ -164,12 +179,11 @@ __global__ void dq_prepare_x_kernel(const __nv_bfloat16* __restrict__ X, int64_t
 }
 
 // ---- unpacking ---------------------------------------------------------------------------------
-// 32 codes (B words) of one weight row, b in {1, 2, 4, 8}, from shared memory into the operand
-// tile: 4 chunks of 8 bf16.  `src` points at the row's codes (16 B bytes; its 16-byte chunks are
-// XOR-swizzled by `xr` so that neighbouring rows read different banks), `qi` = which 32 codes of
-// the row (0..3), `dst` at the row's 128 bytes of the tile, `r7` = row & 7 (the tile's swizzle).
+// 32 codes (B words) of one weight row, b in {1, 2, 4, 8}, from shared memory into 16 registers of
+// bf16 pairs.  `src` points at the row's codes (16 B bytes; its 16-byte chunks are XOR-swizzled by
+// `xr` so that neighbouring rows read different banks), `qi` = which 32 codes of the row (0..3).
 template <int B>
-__device__ __forceinline__ void dq_unpack32(const unsigned char* src, int qi, int xr, unsigned char* dst, int r7) {
+__device__ __forceinline__ void dq_unpack32(const unsigned char* src, int qi, int xr, uint32_t (&out)[16]) {
     constexpr int N = 32 / B;                            // codes per word
     constexpr unsigned MASK = ((1u << B) - 1u) * 0x00010001u;
     const __nv_bfloat162 c128 = __float2bfloat162_rn(128.f);
@@ -187,7 +201,6 @@ __device__ __forceinline__ void dq_unpack32(const unsigned char* src, int qi, in
             w[4 * k] = v.x; w[4 * k + 1] = v.y; w[4 * k + 2] = v.z; w[4 * k + 3] = v.w;
         }
     }
-    uint32_t out[16];                                    // 32 bf16
 #pragma unroll
     for (int m = 0; m < B; ++m) {
 #pragma unroll
@@ -205,21 +218,15 @@ __device__ __forceinline__ void dq_unpack32(const unsigned char* src, int qi, in
             out[(N / 2) * m + s] = bits;
         }
     }
-    const int c0 = 4 * (qi & 1);                         // chunk of the half-block tile
-#pragma unroll
-    for (int c = 0; c < 4; ++c)
-        *reinterpret_cast<uint4*>(dst + (((c0 + c) ^ r7) << 4)) = make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
 }
 
 // any other bitwidth below 8: code k of the row at bit k b of its stream, columns in their own order
-__device__ __forceinline__ void dq_unpack32_generic(const unsigned char* src, int b, int qi, unsigned char* dst, int r7) {
+__device__ __forceinline__ void dq_unpack32_generic(const unsigned char* src, int b, int qi, uint32_t (&out)[16]) {
     const uint32_t* words = reinterpret_cast<const uint32_t*>(src);
     const uint32_t mask = (1u << b) - 1u;
     const __nv_bfloat162 c128 = __float2bfloat162_rn(128.f);
-    const int c0 = 4 * (qi & 1);
-#pragma unroll 1
+#pragma unroll
     for (int c = 0; c < 4; ++c) {
-        uint32_t o[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             uint32_t pair = 0;
@@ -232,9 +239,8 @@ __device__ __forceinline__ void dq_unpack32_generic(const unsigned char* src, in
                 const uint32_t w0 = words[wi], w1 = words[min(wi + 1, 4 * b - 1)];
                 pair |= (__funnelshift_r(w0, w1, bit & 31) & mask) << (16 * h);
             }
-            o[k] = u32(__hsub2(b162(pair | 0x43004300u), c128));
+            out[4 * c + k] = u32(__hsub2(b162(pair | 0x43004300u), c128));
         }
-        *reinterpret_cast<uint4*>(dst + (((c0 + c) ^ r7) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
     }
 }
 
@@ -259,13 +265,12 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
     extern __shared__ unsigned char dq_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(dq_smem_raw) + 1023) & ~uintptr_t(1023));
-    unsigned char* a_tiles = smem;                                        // 2 x 16 KB operand tiles (codes)
-    unsigned char* x_ring = a_tiles + 2 * DQ_A_BYTES;                     // DQ_RING x 8 KB slices of X
+    unsigned char* x_ring = smem;                                         // DQ_RING x 8 KB slices of X
     unsigned char* code_ring = x_ring + DQ_RING * DQ_X_STAGE;             // DQ_RING x 16 KB packed codes
     float* xs = reinterpret_cast<float*>(code_ring + DQ_RING * DQ_CODE_STAGE);   // [seg_blocks][NT] column sums
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(xs + DQ_MAX_SEG_BLOCKS * DQ_MAX_T);
-    unsigned long long* a_full = bars;              // [2] unpackers -> MMA
-    unsigned long long* a_empty = bars + 2;         // [2] MMA done reading -> unpackers
+    unsigned long long* a_full = bars;              // [2] unpackers (TMEM operand buffer written) -> MMA
+    unsigned long long* a_empty = bars + 2;         // [2] MMA done reading the buffer -> unpackers
     unsigned long long* x_empty = bars + 4;         // [DQ_RING] MMA done with the X slice -> loaders
     unsigned long long* d_full = bars + 4 + DQ_RING;       // [2] accumulator complete -> drain
     unsigned long long* d_empty = d_full + 2;              // [2] drained -> MMA
@@ -276,7 +281,8 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
     unsigned* blk_word = tmem_slot + 4;                 // [DQ_MAX_SEG_BLOCKS]
     unsigned char* blk_bits = reinterpret_cast<unsigned char*>(blk_word + DQ_MAX_SEG_BLOCKS);   // [DQ_MAX_SEG_BLOCKS]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr int TMEM_COLS = 2 * NT < 32 ? 32 : 2 * NT;
+    constexpr int TMEM_COLS = DQ_TMEM_COLS;
+    static_assert(2 * NT <= 64, "accumulators below the operand buffers");
 
     const int bi = blockIdx.x;                                  // row tile
     const int j0 = blockIdx.y * a.seg_blocks;                   // first column block of the segment
@@ -359,41 +365,50 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
             for (int i = 0; i < NT / 16; ++i) dq_cp_async16(dstx + xdst[i], xsrc[i] + xoff);
         };
         bool ok = true;
-        for (int jj = 0; jj < 2 && jj < nblk; ++jj) { issue(jj); dq_cp_commit(); }
-        if (nblk < 2) dq_cp_commit();
+        for (int jj = 0; jj < DQ_RING - 1; ++jj) {
+            if (jj < nblk) issue(jj);
+            dq_cp_commit();                                   // (possibly empty) group: keeps the count uniform
+        }
+        // TMEM lanes 32 (warp % 4) ... + 31 belong to this warp: lane = weight row
+        const unsigned a_lane = (unsigned)((r >> 5) * 32) << 16;
         for (int j = 0; j < nblk && ok; ++j) {
-            dq_cp_wait<1>();                                  // block j has landed (this thread's copies)
+            dq_cp_wait<DQ_RING - 2>();                        // block j has landed (this thread's copies)
             const int b = blk_bits[j];
             const unsigned char* src = code_ring + (j % DQ_RING) * DQ_CODE_STAGE + r * 16 * b;
             const int xr = (b == 2) ? ((r >> 2) & 1) : (b == 4) ? ((r >> 1) & 3) : (b == 8) ? r7 : 0;
-            for (int h = 0; h < 2 && ok; ++h) {
-                const int u = 2 * j + h, buf = u & 1;
-                ok = __all_sync(0xffffffffu, dq_mbar_wait(dq_smem_u32(a_empty + buf), ((unsigned)(u >> 1) & 1u) ^ 1u, abort_flag));
-                if (!ok) break;
-                unsigned char* dst = a_tiles + buf * DQ_A_BYTES + r * 128;
+            const int buf = j & 1;
+            ok = __all_sync(0xffffffffu, dq_mbar_wait(dq_smem_u32(a_empty + buf), ((unsigned)(j >> 1) & 1u) ^ 1u, abort_flag));
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            // the thread's two quarters of the row: columns 32 hq ... and 64 + 32 hq ... of the block
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
                 const int qi = 2 * h + hq;
+                uint32_t v[16];
                 switch (b) {                                  // uniform over the CTA
-                    case 1: dq_unpack32<1>(src, qi, xr, dst, r7); break;
-                    case 2: dq_unpack32<2>(src, qi, xr, dst, r7); break;
-                    case 4: dq_unpack32<4>(src, qi, xr, dst, r7); break;
-                    case 8: dq_unpack32<8>(src, qi, xr, dst, r7); break;
-                    default: dq_unpack32_generic(src, b, qi, dst, r7); break;
+                    case 1: dq_unpack32<1>(src, qi, xr, v); break;
+                    case 2: dq_unpack32<2>(src, qi, xr, v); break;
+                    case 4: dq_unpack32<4>(src, qi, xr, v); break;
+                    case 8: dq_unpack32<8>(src, qi, xr, v); break;
+                    default: dq_unpack32_generic(src, b, qi, v); break;
                 }
-                // the tensor cores read shared memory through the async proxy (the X slice of this
-                // block included: every thread's copies were waited for above)
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                dq_mbar_arrive(dq_smem_u32(a_full + buf));
-                if (h == 0) {
-                    // block j + 2 into the stage block j - 1 used: its X slice must have been consumed
-                    // (that contraction was issued before this half was unpacked)
-                    if (j + 2 < nblk) {
-                        if (j >= 1) ok = dq_mbar_wait(dq_smem_u32(x_empty + (j + 2) % DQ_RING), (unsigned)((j - 1) / DQ_RING) & 1u, abort_flag);
-                        if (ok) issue(j + 2);
-                    }
-                    dq_cp_commit();                           // (possibly empty) group: keeps the count uniform
-                    ok = __all_sync(0xffffffffu, ok);
-                }
+                dq_tmem_st16(tmem_base + a_lane + (unsigned)(64 + buf * DQ_A_COLS + 16 * qi), v);
             }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            // the tensor cores read the X slice through the async proxy (every thread's copies of this
+            // block were waited for above) and the operand buffer from TMEM
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            dq_mbar_arrive(dq_smem_u32(a_full + buf));
+            // block j + DQ_RING - 1 into the stage block j - 1 used: its X slice must have been consumed
+            // (that contraction was issued a whole block ago)
+            const int jn = j + DQ_RING - 1;
+            if (jn < nblk) {
+                if (j >= 1) ok = dq_mbar_wait(dq_smem_u32(x_empty + jn % DQ_RING), (unsigned)((j - 1) / DQ_RING) & 1u, abort_flag);
+                if (ok) issue(jn);
+            }
+            dq_cp_commit();
+            ok = __all_sync(0xffffffffu, ok);
         }
         dq_cp_wait<0>();
     } else if (warp == DQ_EPI_WARPS + DQ_CONV_WARPS) {
@@ -402,22 +417,18 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
             const unsigned idesc = dq_idesc(NT);
             bool ok = true;
             for (int j = 0; j < nblk && ok; ++j) {
-                const int ds_ = j & 1, st = j % DQ_RING;
-                ok = dq_mbar_wait(dq_smem_u32(d_empty + ds_), ((unsigned)(j >> 1) & 1u) ^ 1u, abort_flag);
-                for (int h = 0; h < 2 && ok; ++h) {
-                    const int u = 2 * j + h, buf = u & 1;
-                    ok = dq_mbar_wait(dq_smem_u32(a_full + buf), (unsigned)(u >> 1) & 1u, abort_flag);
-                    if (!ok) break;
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const unsigned at = dq_smem_u32(a_tiles + buf * DQ_A_BYTES);
-                    const unsigned xt = dq_smem_u32(x_ring + st * DQ_X_STAGE) + h * (NT * 128);
-#pragma unroll
-                    for (int ks = 0; ks < DQ_HALF / 16; ++ks)          // 16 columns = 32 bytes along K
-                        dq_mma(tmem_base + (unsigned)(ds_ * NT), dq_desc(at + ks * 32), dq_desc(xt + ks * 32), idesc,
-                               (h > 0 || ks > 0) ? 1u : 0u);
-                    dq_commit(dq_smem_u32(a_empty + buf));
-                }
+                const int ds_ = j & 1, st = j % DQ_RING, buf = j & 1;
+                ok = dq_mbar_wait(dq_smem_u32(d_empty + ds_), ((unsigned)(j >> 1) & 1u) ^ 1u, abort_flag) &&
+                     dq_mbar_wait(dq_smem_u32(a_full + buf), (unsigned)(j >> 1) & 1u, abort_flag);
                 if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const unsigned at = tmem_base + (unsigned)(64 + buf * DQ_A_COLS);
+                const unsigned xt = dq_smem_u32(x_ring + st * DQ_X_STAGE);
+#pragma unroll
+                for (int ks = 0; ks < DQ_KB / 16; ++ks)             // 16 columns: 8 TMEM columns of A, 32 bytes of X along K
+                    dq_mma(tmem_base + (unsigned)(ds_ * NT), at + ks * 8,
+                           dq_desc(xt + (ks >> 2) * (NT * 128) + (ks & 3) * 32), idesc, ks > 0 ? 1u : 0u);
+                dq_commit(dq_smem_u32(a_empty + buf));
                 dq_commit(dq_smem_u32(x_empty + st));
                 dq_commit(dq_smem_u32(d_full + ds_));
             }
