@@ -22,10 +22,13 @@
 // there; only the few-token slice of X is a shared-memory operand.
 //
 // Grid: (R / 128 row tiles) x (S column segments), two CTAs per SM.  Per CTA:
-//   warps 4-11 (thread = 2 x 32 columns of a weight row): cp.async of its own codes and of the
-//     block's slice of X (straight into the K-major 128-byte-swizzle operand layout) three blocks
-//     ahead; unpack the block into registers, tcgen05.st into one of two 64-column TMEM operand
-//     buffers, tcgen05.wait::st, fences, mbarrier arrive;
+//   warp 13 (one thread): per block two bulk copies (cp.async.bulk, mbarrier complete_tx) into a
+//     four-stage ring, three blocks ahead: the block's packed codes as they lie in memory, and its
+//     slice of X, which the preparation kernel has already laid out as the K-major
+//     128-byte-swizzle operand image;
+//   warps 4-11 (thread = 2 x 32 columns of a weight row): unpack the block into registers,
+//     tcgen05.st into one of two 64-column TMEM operand buffers, tcgen05.wait::st, fences,
+//     mbarrier arrives (operand ready; code stage free);
 //   warp 12 (one thread): 8 tcgen05.mma (K = 16, A from TMEM, B = X slice from shared memory) per
 //     block into one of two TMEM accumulators of N columns, tcgen05.commit to free the operand
 //     buffer and the X slice and to publish the accumulator;
@@ -47,7 +50,7 @@ constexpr int DQ_A_COLS = DQ_KB / 2;         // TMEM columns of a block's codes:
 constexpr int DQ_MAX_T = 32;
 constexpr int DQ_X_STAGE = DQ_MAX_T * DQ_KB * 2;        // X slice of a block: tokens x 128 bf16
 constexpr int DQ_CONV_WARPS = 8, DQ_EPI_WARPS = 4;    // unpacking thread = 32 columns of a weight row
-constexpr int DQ_THREADS = (DQ_EPI_WARPS + DQ_CONV_WARPS + 1) * 32;
+constexpr int DQ_THREADS = (DQ_EPI_WARPS + DQ_CONV_WARPS + 2) * 32;   // + MMA warp + loader warp
 constexpr int DQ_MAX_SEG_BLOCKS = 32;       // column blocks per segment (their column sums sit in shared memory)
 constexpr int DQ_ORDERS = 5;                // column orders of X: identity, b = 1, 2, 4, 8
 constexpr int DQ_SMEM = DQ_RING * (DQ_CODE_STAGE + DQ_X_STAGE) + DQ_MAX_SEG_BLOCKS * DQ_MAX_T * 4 +
@@ -96,11 +99,15 @@ __device__ __forceinline__ bool dq_mbar_wait(unsigned bar, unsigned parity, vola
         }
     }
 }
-__device__ __forceinline__ void dq_cp_async16(unsigned dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+__device__ __forceinline__ void dq_mbar_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void dq_cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void dq_cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// contiguous bytes (a multiple of 16, both addresses 16-byte aligned) into shared memory; the
+// bytes are counted on the mbarrier
+__device__ __forceinline__ void dq_bulk_load(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
 
 // K-major operand in the 128-byte-swizzle layout: rows of 128 bytes (64 bf16 along K), 8-row
 // groups 1024 bytes apart; the leading offset is not used by swizzled K-major layouts
@@ -154,8 +161,14 @@ __device__ __forceinline__ void dq_tmem_ld16(unsigned taddr, float (&v)[16]) {
 
 // ---- X in the column orders of the unpacking, and its per-block column sums ------------------
 // order o > 0 (codes of b bits, n = 32 / b per word): position n m + 2 s + h holds column
-// n m + s + (n / 2) h.  xp: [DQ_ORDERS][T][C] bf16, xsum: [C / 128][T] fp32.
-__global__ void dq_prepare_x_kernel(const __nv_bfloat16* __restrict__ X, int64_t ldx, int T, int64_t C,
+// n m + s + (n / 2) h.  xp: [DQ_ORDERS][C / 128] images of T x 128 bf16, each laid out as the
+// shared-memory operand (two K halves of T rows x 128 bytes, 16-byte chunks XOR-swizzled with the
+// row), so that one contiguous copy brings a block's slice in; xsum: [C / 128][T] fp32.
+__device__ __forceinline__ int dq_image_index(int T, int t, int p) {
+    const int panel = p >> 6, pp = p & 63;
+    return panel * (T * 64) + t * 64 + (((pp >> 3) ^ (t & 7)) << 3) + (pp & 7);
+}
+__global__ void dq_prepare_x_kernel(const __nv_bfloat16* __restrict__ X, int64_t ldx, int T, int64_t nbc,
                                     __nv_bfloat16* __restrict__ xp, float* __restrict__ xsum) {
     const int64_t jb = blockIdx.x;                       // column block
     const int t = blockIdx.y;
@@ -168,22 +181,22 @@ __global__ void dq_prepare_x_kernel(const __nv_bfloat16* __restrict__ X, int64_t
     if ((p & 31) == 0) ws[p >> 5] = s;
     __syncthreads();
     if (p == 0) xsum[jb * T + t] = (ws[0] + ws[1]) + (ws[2] + ws[3]);
-    __nv_bfloat16* out = xp + (int64_t)t * C + jb * DQ_KB + p;
+    const int64_t image = (int64_t)T * DQ_KB;
+    __nv_bfloat16* out = xp + jb * image + dq_image_index(T, t, p);
     out[0] = xrow[p];
 #pragma unroll
     for (int o = 1; o < DQ_ORDERS; ++o) {
         const int n = 32 >> (o - 1);                     // codes per word: 32, 16, 8, 4
         const int m = p / n, w = p % n, s2 = w >> 1, h = w & 1;
-        out[(int64_t)o * T * C] = xrow[n * m + s2 + (n >> 1) * h];
+        out[(int64_t)o * nbc * image] = xrow[n * m + s2 + (n >> 1) * h];
     }
 }
 
 // ---- unpacking ---------------------------------------------------------------------------------
 // 32 codes (B words) of one weight row, b in {1, 2, 4, 8}, from shared memory into 16 registers of
-// bf16 pairs.  `src` points at the row's codes (16 B bytes; its 16-byte chunks are XOR-swizzled by
-// `xr` so that neighbouring rows read different banks), `qi` = which 32 codes of the row (0..3).
+// bf16 pairs.  `src` points at the row's codes (16 B bytes), `qi` = which 32 codes of the row (0..3).
 template <int B>
-__device__ __forceinline__ void dq_unpack32(const unsigned char* src, int qi, int xr, uint32_t (&out)[16]) {
+__device__ __forceinline__ void dq_unpack32(const unsigned char* src, int qi, uint32_t (&out)[16]) {
     constexpr int N = 32 / B;                            // codes per word
     constexpr unsigned MASK = ((1u << B) - 1u) * 0x00010001u;
     const __nv_bfloat162 c128 = __float2bfloat162_rn(128.f);
@@ -191,13 +204,13 @@ __device__ __forceinline__ void dq_unpack32(const unsigned char* src, int qi, in
     if constexpr (B == 1) {
         w[0] = *reinterpret_cast<const uint32_t*>(src + 4 * qi);
     } else if constexpr (B == 2) {
-        const uint2 v = *reinterpret_cast<const uint2*>(src + (((qi >> 1) ^ xr) << 4) + 8 * (qi & 1));
+        const uint2 v = *reinterpret_cast<const uint2*>(src + 8 * qi);
         w[0] = v.x; w[1] = v.y;
     } else {
 #pragma unroll
         for (int k = 0; k < B / 4; ++k) {
             const int chunk = qi * (B / 4) + k;          // 16-byte chunk of the row
-            const uint4 v = *reinterpret_cast<const uint4*>(src + ((chunk ^ xr) << 4));
+            const uint4 v = *reinterpret_cast<const uint4*>(src + (chunk << 4));
             w[4 * k] = v.x; w[4 * k + 1] = v.y; w[4 * k + 2] = v.z; w[4 * k + 3] = v.w;
         }
     }
@@ -249,7 +262,7 @@ struct DqArgs {
     const int64_t* block_off;       // [nb + 1], words
     const float2* meta;             // [(r * nbc + j)] = (scale, lo), group == block width
     const uint8_t* level;           // [nb]
-    const __nv_bfloat16* xp;        // [DQ_ORDERS][T][C]
+    const __nv_bfloat16* xp;        // [DQ_ORDERS][nbc] operand images of T x 128
     const float* xsum;              // [nbc][T]
     float* out;                     // partial sums [S][T][R] (or Y when S == 1)
     int64_t out_t_stride;           // R for the partial sums, ldy for Y
@@ -271,10 +284,12 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(xs + DQ_MAX_SEG_BLOCKS * DQ_MAX_T);
     unsigned long long* a_full = bars;              // [2] unpackers (TMEM operand buffer written) -> MMA
     unsigned long long* a_empty = bars + 2;         // [2] MMA done reading the buffer -> unpackers
-    unsigned long long* x_empty = bars + 4;         // [DQ_RING] MMA done with the X slice -> loaders
+    unsigned long long* x_empty = bars + 4;         // [DQ_RING] MMA done with the X slice -> loader
     unsigned long long* d_full = bars + 4 + DQ_RING;       // [2] accumulator complete -> drain
     unsigned long long* d_empty = d_full + 2;              // [2] drained -> MMA
-    unsigned* tmem_slot = reinterpret_cast<unsigned*>(d_empty + 2);
+    unsigned long long* ld_full = d_empty + 2;             // [DQ_RING] both copies of a block landed
+    unsigned long long* code_empty = ld_full + DQ_RING;    // [DQ_RING] all unpackers have read the codes -> loader
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(code_empty + DQ_RING);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     // per block of the segment: first word of its codes (blocks are below 2^32 words apart from the
     // segment's first) and its bitwidth, so that the loop below has no dependent global loads
@@ -295,7 +310,11 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
             dq_mbar_init(dq_smem_u32(d_full + s), 1);
             dq_mbar_init(dq_smem_u32(d_empty + s), DQ_EPI_WARPS);
         }
-        for (int s = 0; s < DQ_RING; ++s) dq_mbar_init(dq_smem_u32(x_empty + s), 1);
+        for (int s = 0; s < DQ_RING; ++s) {
+            dq_mbar_init(dq_smem_u32(x_empty + s), 1);
+            dq_mbar_init(dq_smem_u32(ld_full + s), 1);
+            dq_mbar_init(dq_smem_u32(code_empty + s), DQ_CONV_WARPS * 32);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -318,99 +337,38 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
     const unsigned tmem_base = *tmem_slot;
 
     if (warp >= DQ_EPI_WARPS && warp < DQ_EPI_WARPS + DQ_CONV_WARPS) {
-        // ---- loaders / unpackers: thread = 32 columns (quarter hq of the current half block) of
-        // weight row r of the tile ----------------------------------------------------------------------
+        // ---- unpackers: thread = columns 32 hq ... and 64 + 32 hq ... of weight row r of the tile ------
         const int ct = threadIdx.x - DQ_EPI_WARPS * 32;
         const int r = ct & (DQ_M - 1), hq = ct >> 7;
-        const int r7 = r & 7;
-        // this thread's share of a block's X slice: 16-byte chunks ct, ct + 256, ... of the slice
-        // (token, chunk in the row), straight into the swizzled operand layout
-        unsigned xdst[NT / 16];
-        const __nv_bfloat16* xsrc[NT / 16];
-#pragma unroll
-        for (int i = 0; i < NT / 16; ++i) {
-            const int k = ct + 256 * i;
-            const int t = k >> 4, cc = k & 15;
-            const int panel = cc >> 3, c8 = cc & 7;      // K half, chunk inside its 128 bytes
-            xdst[i] = (unsigned)(panel * (NT * 128) + t * 128 + ((c8 ^ (t & 7)) << 4));
-            xsrc[i] = a.xp + (int64_t)t * a.C + (int64_t)j0 * DQ_KB + cc * 8;
-        }
-        // cp.async of block jj of the segment into ring stage jj % DQ_RING.  A thread copies the
-        // chunks of its row's codes that it will read itself (for b = 4, 8 those of its two
-        // quarters; otherwise the whole row, twice over with its partner), so waiting for its own
-        // copies is all the synchronisation the codes need.
-        auto issue = [&](int jj) {
-            const int st = jj % DQ_RING;
-            const int b = blk_bits[jj];
-            const unsigned char* src = reinterpret_cast<const unsigned char*>(a.packed + word0 + blk_word[jj]) + r * 16 * b;
-            const unsigned dstc = dq_smem_u32(code_ring + st * DQ_CODE_STAGE + r * 16 * b);
-            // chunk swizzle over the row's b chunks (power-of-two b only): rows that share a bank
-            // group get different chunk orders
-            const int xr = (b == 2) ? ((r >> 2) & 1) : (b == 4) ? ((r >> 1) & 3) : (b == 8) ? r7 : 0;
-            if (b == 4) {
-                dq_cp_async16(dstc + ((hq ^ xr) << 4), src + (hq << 4));
-                dq_cp_async16(dstc + (((2 + hq) ^ xr) << 4), src + ((2 + hq) << 4));
-            } else if (b == 8) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int ch = (k >> 1) * 4 + 2 * hq + (k & 1);
-                    dq_cp_async16(dstc + ((ch ^ xr) << 4), src + (ch << 4));
-                }
-            } else {
-                for (int k = 0; k < b; ++k) dq_cp_async16(dstc + ((k ^ xr) << 4), src + (k << 4));
-            }
-            const int64_t xoff = (int64_t)dq_order(b) * NT * a.C + (int64_t)jj * DQ_KB;
-            const unsigned dstx = dq_smem_u32(x_ring + st * DQ_X_STAGE);
-#pragma unroll
-            for (int i = 0; i < NT / 16; ++i) dq_cp_async16(dstx + xdst[i], xsrc[i] + xoff);
-        };
-        bool ok = true;
-        for (int jj = 0; jj < DQ_RING - 1; ++jj) {
-            if (jj < nblk) issue(jj);
-            dq_cp_commit();                                   // (possibly empty) group: keeps the count uniform
-        }
         // TMEM lanes 32 (warp % 4) ... + 31 belong to this warp: lane = weight row
         const unsigned a_lane = (unsigned)((r >> 5) * 32) << 16;
+        bool ok = true;
         for (int j = 0; j < nblk && ok; ++j) {
-            dq_cp_wait<DQ_RING - 2>();                        // block j has landed (this thread's copies)
+            const int st = j % DQ_RING, buf = j & 1;
             const int b = blk_bits[j];
-            const unsigned char* src = code_ring + (j % DQ_RING) * DQ_CODE_STAGE + r * 16 * b;
-            const int xr = (b == 2) ? ((r >> 2) & 1) : (b == 4) ? ((r >> 1) & 3) : (b == 8) ? r7 : 0;
-            const int buf = j & 1;
-            ok = __all_sync(0xffffffffu, dq_mbar_wait(dq_smem_u32(a_empty + buf), ((unsigned)(j >> 1) & 1u) ^ 1u, abort_flag));
+            ok = __all_sync(0xffffffffu, dq_mbar_wait(dq_smem_u32(ld_full + st), (unsigned)(j / DQ_RING) & 1u, abort_flag) &&
+                                         dq_mbar_wait(dq_smem_u32(a_empty + buf), ((unsigned)(j >> 1) & 1u) ^ 1u, abort_flag));
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            // the thread's two quarters of the row: columns 32 hq ... and 64 + 32 hq ... of the block
+            const unsigned char* src = code_ring + st * DQ_CODE_STAGE + r * 16 * b;
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int qi = 2 * h + hq;
                 uint32_t v[16];
                 switch (b) {                                  // uniform over the CTA
-                    case 1: dq_unpack32<1>(src, qi, xr, v); break;
-                    case 2: dq_unpack32<2>(src, qi, xr, v); break;
-                    case 4: dq_unpack32<4>(src, qi, xr, v); break;
-                    case 8: dq_unpack32<8>(src, qi, xr, v); break;
+                    case 1: dq_unpack32<1>(src, qi, v); break;
+                    case 2: dq_unpack32<2>(src, qi, v); break;
+                    case 4: dq_unpack32<4>(src, qi, v); break;
+                    case 8: dq_unpack32<8>(src, qi, v); break;
                     default: dq_unpack32_generic(src, b, qi, v); break;
                 }
                 dq_tmem_st16(tmem_base + a_lane + (unsigned)(64 + buf * DQ_A_COLS + 16 * qi), v);
             }
+            dq_mbar_arrive(dq_smem_u32(code_empty + st));     // the codes are in registers: the stage may be refilled
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-            // the tensor cores read the X slice through the async proxy (every thread's copies of this
-            // block were waited for above) and the operand buffer from TMEM
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             dq_mbar_arrive(dq_smem_u32(a_full + buf));
-            // block j + DQ_RING - 1 into the stage block j - 1 used: its X slice must have been consumed
-            // (that contraction was issued a whole block ago)
-            const int jn = j + DQ_RING - 1;
-            if (jn < nblk) {
-                if (j >= 1) ok = dq_mbar_wait(dq_smem_u32(x_empty + jn % DQ_RING), (unsigned)((j - 1) / DQ_RING) & 1u, abort_flag);
-                if (ok) issue(jn);
-            }
-            dq_cp_commit();
-            ok = __all_sync(0xffffffffu, ok);
         }
-        dq_cp_wait<0>();
     } else if (warp == DQ_EPI_WARPS + DQ_CONV_WARPS) {
         if (lane == 0) {
             // ---- MMA issue -----------------------------------------------------------------------------
@@ -419,6 +377,7 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
             for (int j = 0; j < nblk && ok; ++j) {
                 const int ds_ = j & 1, st = j % DQ_RING, buf = j & 1;
                 ok = dq_mbar_wait(dq_smem_u32(d_empty + ds_), ((unsigned)(j >> 1) & 1u) ^ 1u, abort_flag) &&
+                     dq_mbar_wait(dq_smem_u32(ld_full + st), (unsigned)(j / DQ_RING) & 1u, abort_flag) &&
                      dq_mbar_wait(dq_smem_u32(a_full + buf), (unsigned)(j >> 1) & 1u, abort_flag);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -431,6 +390,28 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
                 dq_commit(dq_smem_u32(a_empty + buf));
                 dq_commit(dq_smem_u32(x_empty + st));
                 dq_commit(dq_smem_u32(d_full + ds_));
+            }
+        }
+    } else if (warp == DQ_EPI_WARPS + DQ_CONV_WARPS + 1) {
+        if (lane == 0) {
+            // ---- loader: the codes of block j as they lie in memory and its slice of X (an operand
+            // image) into ring stage j % DQ_RING, as soon as the unpackers and the contraction of block
+            // j - DQ_RING have let go of it ----------------------------------------------------------------
+            bool ok = true;
+            const unsigned x_bytes = (unsigned)(NT * DQ_KB * 2);
+            for (int j = 0; j < nblk && ok; ++j) {
+                const int st = j % DQ_RING;
+                const unsigned ph = ((unsigned)(j / DQ_RING) & 1u) ^ 1u;
+                ok = dq_mbar_wait(dq_smem_u32(code_empty + st), ph, abort_flag) &&
+                     dq_mbar_wait(dq_smem_u32(x_empty + st), ph, abort_flag);
+                if (!ok) break;
+                const int b = blk_bits[j];
+                const unsigned code_bytes = (unsigned)(2048 * b);
+                const unsigned full = dq_smem_u32(ld_full + st);
+                dq_mbar_expect_tx(full, code_bytes + x_bytes);
+                dq_bulk_load(dq_smem_u32(code_ring + st * DQ_CODE_STAGE), a.packed + word0 + blk_word[j], code_bytes, full);
+                dq_bulk_load(dq_smem_u32(x_ring + st * DQ_X_STAGE),
+                             a.xp + ((int64_t)dq_order(b) * a.nbc + j0 + j) * (NT * DQ_KB), x_bytes, full);
             }
         }
     } else {
@@ -532,7 +513,7 @@ extern "C" sb_status sb_dequant_gemm(sb_ctx* ctx, const void* X, int64_t T, int6
             SB_CUDA(ctx, cudaMemsetAsync(xp, 0, (size_t)DQ_ORDERS * NT * C * 2, ctx->stream));
             SB_CUDA(ctx, cudaMemsetAsync(xsum, 0, (size_t)nbc * NT * 4, ctx->stream));
         }
-        dq_prepare_x_kernel<<<dim3((unsigned)nbc, (unsigned)Tn), 128, 0, ctx->stream>>>(Xs, ldx, NT, C, xp, xsum);
+        dq_prepare_x_kernel<<<dim3((unsigned)nbc, (unsigned)Tn), 128, 0, ctx->stream>>>(Xs, ldx, NT, nbc, xp, xsum);
         SB_LAUNCHED(ctx);
         DqArgs a{};
         a.packed = packed; a.block_off = block_off_words; a.meta = reinterpret_cast<const float2*>(meta);
