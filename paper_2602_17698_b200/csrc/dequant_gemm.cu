@@ -30,8 +30,8 @@
 //     tcgen05.st into one of two 64-column TMEM operand buffers, tcgen05.wait::st, fences,
 //     mbarrier arrives (operand ready; code stage free);
 //   warp 12 (one thread): 8 tcgen05.mma (K = 16, A from TMEM, B = X slice from shared memory) per
-//     block into one of two TMEM accumulators of N columns, tcgen05.commit to free the operand
-//     buffer and the X slice and to publish the accumulator;
+//     block into one of two TMEM accumulators of N columns, one tcgen05.commit per block, which
+//     frees the operand buffer and the X slice and publishes the accumulator;
 //   warps 0-3 (thread = weight row = TMEM lane): tcgen05.ld of the block's accumulator,
 //     y += scale * acc + lo * colsum(X) in fp32 registers; at the end the segment's partial
 //     sums go to scratch (or to Y when there is one segment) and a second kernel adds the
@@ -283,10 +283,11 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
     float* xs = reinterpret_cast<float*>(code_ring + DQ_RING * DQ_CODE_STAGE);   // [seg_blocks][NT] column sums
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(xs + DQ_MAX_SEG_BLOCKS * DQ_MAX_T);
     unsigned long long* a_full = bars;              // [2] unpackers (TMEM operand buffer written) -> MMA
-    unsigned long long* a_empty = bars + 2;         // [2] MMA done reading the buffer -> unpackers
-    unsigned long long* x_empty = bars + 4;         // [DQ_RING] MMA done with the X slice -> loader
-    unsigned long long* d_full = bars + 4 + DQ_RING;       // [2] accumulator complete -> drain
-    unsigned long long* d_empty = d_full + 2;              // [2] drained -> MMA
+    // [DQ_RING] the contraction of block j is complete (one commit per block, at j % DQ_RING): the
+    // drain may read its accumulator, the unpackers may rewrite the operand buffer two blocks
+    // later, the loader may refill the stage DQ_RING blocks later
+    unsigned long long* done = bars + 2;
+    unsigned long long* d_empty = done + DQ_RING;          // [2] drained -> MMA
     unsigned long long* ld_full = d_empty + 2;             // [DQ_RING] both copies of a block landed
     unsigned long long* code_empty = ld_full + DQ_RING;    // [DQ_RING] all unpackers have read the codes -> loader
     unsigned* tmem_slot = reinterpret_cast<unsigned*>(code_empty + DQ_RING);
@@ -306,12 +307,10 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
     if (threadIdx.x == 0) {
         for (int s = 0; s < 2; ++s) {
             dq_mbar_init(dq_smem_u32(a_full + s), DQ_CONV_WARPS * 32);
-            dq_mbar_init(dq_smem_u32(a_empty + s), 1);
-            dq_mbar_init(dq_smem_u32(d_full + s), 1);
             dq_mbar_init(dq_smem_u32(d_empty + s), DQ_EPI_WARPS);
         }
         for (int s = 0; s < DQ_RING; ++s) {
-            dq_mbar_init(dq_smem_u32(x_empty + s), 1);
+            dq_mbar_init(dq_smem_u32(done + s), 1);
             dq_mbar_init(dq_smem_u32(ld_full + s), 1);
             dq_mbar_init(dq_smem_u32(code_empty + s), DQ_CONV_WARPS * 32);
         }
@@ -346,8 +345,10 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
         for (int j = 0; j < nblk && ok; ++j) {
             const int st = j % DQ_RING, buf = j & 1;
             const int b = blk_bits[j];
+            // the block has landed, and the contraction of block j - 2 no longer reads the operand buffer
             ok = __all_sync(0xffffffffu, dq_mbar_wait(dq_smem_u32(ld_full + st), (unsigned)(j / DQ_RING) & 1u, abort_flag) &&
-                                         dq_mbar_wait(dq_smem_u32(a_empty + buf), ((unsigned)(j >> 1) & 1u) ^ 1u, abort_flag));
+                                         (j < 2 || dq_mbar_wait(dq_smem_u32(done + (j - 2) % DQ_RING),
+                                                                (unsigned)((j - 2) / DQ_RING) & 1u, abort_flag)));
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const unsigned char* src = code_ring + st * DQ_CODE_STAGE + r * 16 * b;
@@ -387,9 +388,7 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
                 for (int ks = 0; ks < DQ_KB / 16; ++ks)             // 16 columns: 8 TMEM columns of A, 32 bytes of X along K
                     dq_mma(tmem_base + (unsigned)(ds_ * NT), at + ks * 8,
                            dq_desc(xt + (ks >> 2) * (NT * 128) + (ks & 3) * 32), idesc, ks > 0 ? 1u : 0u);
-                dq_commit(dq_smem_u32(a_empty + buf));
-                dq_commit(dq_smem_u32(x_empty + st));
-                dq_commit(dq_smem_u32(d_full + ds_));
+                dq_commit(dq_smem_u32(done + st));
             }
         }
     } else if (warp == DQ_EPI_WARPS + DQ_CONV_WARPS + 1) {
@@ -401,9 +400,12 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
             const unsigned x_bytes = (unsigned)(NT * DQ_KB * 2);
             for (int j = 0; j < nblk && ok; ++j) {
                 const int st = j % DQ_RING;
-                const unsigned ph = ((unsigned)(j / DQ_RING) & 1u) ^ 1u;
-                ok = dq_mbar_wait(dq_smem_u32(code_empty + st), ph, abort_flag) &&
-                     dq_mbar_wait(dq_smem_u32(x_empty + st), ph, abort_flag);
+                // block j - DQ_RING used this stage: its codes have been read and its contraction is complete
+                if (j >= DQ_RING) {
+                    const unsigned ph = (unsigned)(j / DQ_RING - 1) & 1u;
+                    ok = dq_mbar_wait(dq_smem_u32(code_empty + st), ph, abort_flag) &&
+                         dq_mbar_wait(dq_smem_u32(done + st), ph, abort_flag);
+                }
                 if (!ok) break;
                 const int b = blk_bits[j];
                 const unsigned code_bytes = (unsigned)(2048 * b);
@@ -427,7 +429,7 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
             const float2 cur = sl;
             if (j + 1 < nblk) sl = a.meta[row * a.nbc + j0 + j + 1];
             const int ds_ = j & 1;
-            ok = __all_sync(0xffffffffu, dq_mbar_wait(dq_smem_u32(d_full + ds_), (unsigned)(j >> 1) & 1u, abort_flag));
+            ok = __all_sync(0xffffffffu, dq_mbar_wait(dq_smem_u32(done + j % DQ_RING), (unsigned)(j / DQ_RING) & 1u, abort_flag));
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
