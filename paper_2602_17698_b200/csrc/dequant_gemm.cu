@@ -27,7 +27,7 @@
 //     slice of X, which the preparation kernel has already laid out as the K-major
 //     128-byte-swizzle operand image;
 //   warps 4-11 (thread = 2 x 32 columns of a weight row): unpack the block into registers,
-//     tcgen05.st into one of two 64-column TMEM operand buffers, tcgen05.wait::st, fences,
+//     tcgen05.st into one of three 64-column TMEM operand buffers, tcgen05.wait::st, fences,
 //     mbarrier arrives (operand ready; code stage free);
 //   warp 12 (one thread): 8 tcgen05.mma (K = 16, A from TMEM, B = X slice from shared memory) per
 //     block into one of two TMEM accumulators of N columns, one tcgen05.commit per block, which
@@ -47,6 +47,7 @@ constexpr int DQ_KB = 128;                  // block columns
 constexpr int DQ_RING = 4;                  // blocks in flight (codes + X slice)
 constexpr int DQ_CODE_STAGE = 2048 * 8;     // bytes of codes of one block at 8 bits
 constexpr int DQ_A_COLS = DQ_KB / 2;         // TMEM columns of a block's codes: two bf16 per 32-bit column
+constexpr int DQ_ABUF = 3;                  // TMEM operand buffers: the unpackers run up to two blocks ahead of the contraction
 constexpr int DQ_MAX_T = 32;
 constexpr int DQ_X_STAGE = DQ_MAX_T * DQ_KB * 2;        // X slice of a block: tokens x 128 bf16
 constexpr int DQ_CONV_WARPS = 8, DQ_EPI_WARPS = 4;    // unpacking thread = 32 columns of a weight row
@@ -55,7 +56,7 @@ constexpr int DQ_MAX_SEG_BLOCKS = 32;       // column blocks per segment (their 
 constexpr int DQ_ORDERS = 5;                // column orders of X: identity, b = 1, 2, 4, 8
 constexpr int DQ_SMEM = DQ_RING * (DQ_CODE_STAGE + DQ_X_STAGE) + DQ_MAX_SEG_BLOCKS * DQ_MAX_T * 4 +
                         1024 /* alignment */ + 512 /* barriers, block table */;
-constexpr int DQ_TMEM_COLS = 256;           // accumulators in columns [0, 64), operand buffers at 64 and 128
+constexpr int DQ_TMEM_COLS = 256;           // accumulators in columns [0, 64), operand buffers at 64, 128 and 192
 constexpr unsigned long long DQ_WAIT_NS = 2000ull * 1000 * 1000;
 
 // candidate bitwidths, four bits each
@@ -282,11 +283,11 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
     unsigned char* code_ring = x_ring + DQ_RING * DQ_X_STAGE;             // DQ_RING x 16 KB packed codes
     float* xs = reinterpret_cast<float*>(code_ring + DQ_RING * DQ_CODE_STAGE);   // [seg_blocks][NT] column sums
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(xs + DQ_MAX_SEG_BLOCKS * DQ_MAX_T);
-    unsigned long long* a_full = bars;              // [2] unpackers (TMEM operand buffer written) -> MMA
+    unsigned long long* a_full = bars;              // [DQ_ABUF] unpackers (TMEM operand buffer written) -> MMA
     // [DQ_RING] the contraction of block j is complete (one commit per block, at j % DQ_RING): the
     // drain may read its accumulator, the unpackers may rewrite the operand buffer two blocks
     // later, the loader may refill the stage DQ_RING blocks later
-    unsigned long long* done = bars + 2;
+    unsigned long long* done = bars + DQ_ABUF;
     unsigned long long* d_empty = done + DQ_RING;          // [2] drained -> MMA
     unsigned long long* ld_full = d_empty + 2;             // [DQ_RING] both copies of a block landed
     unsigned long long* code_empty = ld_full + DQ_RING;    // [DQ_RING] all unpackers have read the codes -> loader
@@ -306,9 +307,9 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 2; ++s) {
-            dq_mbar_init(dq_smem_u32(a_full + s), DQ_CONV_WARPS * 32);
             dq_mbar_init(dq_smem_u32(d_empty + s), DQ_EPI_WARPS);
         }
+        for (int s = 0; s < DQ_ABUF; ++s) dq_mbar_init(dq_smem_u32(a_full + s), DQ_CONV_WARPS * 32);
         for (int s = 0; s < DQ_RING; ++s) {
             dq_mbar_init(dq_smem_u32(done + s), 1);
             dq_mbar_init(dq_smem_u32(ld_full + s), 1);
@@ -343,12 +344,12 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
         const unsigned a_lane = (unsigned)((r >> 5) * 32) << 16;
         bool ok = true;
         for (int j = 0; j < nblk && ok; ++j) {
-            const int st = j % DQ_RING, buf = j & 1;
+            const int st = j % DQ_RING, buf = j % DQ_ABUF;
             const int b = blk_bits[j];
-            // the block has landed, and the contraction of block j - 2 no longer reads the operand buffer
+            // the block has landed, and the contraction of block j - DQ_ABUF no longer reads the operand buffer
             ok = __all_sync(0xffffffffu, dq_mbar_wait(dq_smem_u32(ld_full + st), (unsigned)(j / DQ_RING) & 1u, abort_flag) &&
-                                         (j < 2 || dq_mbar_wait(dq_smem_u32(done + (j - 2) % DQ_RING),
-                                                                (unsigned)((j - 2) / DQ_RING) & 1u, abort_flag)));
+                                         (j < DQ_ABUF || dq_mbar_wait(dq_smem_u32(done + (j - DQ_ABUF) % DQ_RING),
+                                                                      (unsigned)((j - DQ_ABUF) / DQ_RING) & 1u, abort_flag)));
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const unsigned char* src = code_ring + st * DQ_CODE_STAGE + r * 16 * b;
@@ -376,10 +377,10 @@ __global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArg
             const unsigned idesc = dq_idesc(NT);
             bool ok = true;
             for (int j = 0; j < nblk && ok; ++j) {
-                const int ds_ = j & 1, st = j % DQ_RING, buf = j & 1;
+                const int ds_ = j & 1, st = j % DQ_RING, buf = j % DQ_ABUF;
                 ok = dq_mbar_wait(dq_smem_u32(d_empty + ds_), ((unsigned)(j >> 1) & 1u) ^ 1u, abort_flag) &&
                      dq_mbar_wait(dq_smem_u32(ld_full + st), (unsigned)(j / DQ_RING) & 1u, abort_flag) &&
-                     dq_mbar_wait(dq_smem_u32(a_full + buf), (unsigned)(j >> 1) & 1u, abort_flag);
+                     dq_mbar_wait(dq_smem_u32(a_full + buf), (unsigned)(j / DQ_ABUF) & 1u, abort_flag);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const unsigned at = tmem_base + (unsigned)(64 + buf * DQ_A_COLS);
