@@ -6,8 +6,8 @@
 //     Y[t][r] = sum over column blocks j of  scale[r][j] * (sum_c X[t][c] q[r][c]) + lo[r][j] * (sum_c X[t][c])
 // with one tcgen05 contraction (M = 128 weight rows, N = tokens, K = the block's 128 columns,
 // bf16 x bf16 -> fp32) per 128 x 128 block, scaled per row in the drain; nothing is rounded
-// but the fp32 accumulation.  The kernel is bound by reading the packed codes once from HBM
-// and by the unpacking arithmetic, so the unpacking is kept to about 1.4 operations per code:
+// but the fp32 accumulation.  The packed codes are read once from HBM; what costs time is
+// turning them into operands, so the unpacking is kept to about 1.4 operations per code:
 // for b in {1, 2, 4, 8} a 32-bit word of codes is split by ONE mask per pair,
 //     (w >> (b s)) & (2^b - 1) * 0x00010001     ->  codes s and s + 16 / b of the word as two 16-bit halves,
 // which OR 0x4300 turns into the bf16 pair (128 + q_lo, 128 + q_hi); subtracting 128 is exact.
