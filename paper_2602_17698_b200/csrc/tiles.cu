@@ -509,9 +509,11 @@ __global__ void scores_finish_kernel(const float* __restrict__ rec, ScoreGeom g,
 // are bit-identical -- and adds them to / stores them in the score vectors.
 // FIRST: the first-order form of the element sensitivity, |G_rj (W_rj - Q(W)_rj)| (Section 3.2
 // with p = 1), from a caller's gradient G; no column or row factors.
-template <bool ROWW, bool FINE, int TILE_ROWS, bool FIRST>
+// A tile is `tile_rows` (a multiple of 32) x 128; the host picks tile_rows so that the tiles fill
+// whole rounds of the CTA slots of the GPU.
+template <bool ROWW, bool FINE, bool FIRST>
 __global__ void __launch_bounds__(CTA_THREADS)
-reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, int64_t ldw,
+reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, int64_t ldw, int tile_rows,
                      const __nv_bfloat16* __restrict__ G, int64_t ldg,
                      const float* __restrict__ col_moment, const float* __restrict__ row_weight,
                      int group, float qmax, float inv_qmax,
@@ -520,13 +522,13 @@ reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, 
                      unsigned* __restrict__ done_row, unsigned* __restrict__ done_col,
                      SbDeviceState* dstate) {
     constexpr int CPL = 16, NW = 8, LANE_COLS = 8, ROW_SLOTS = 4;
-    constexpr int ITERS = TILE_ROWS / (CTA_WARPS * ROW_SLOTS);
+    const int ITERS = tile_rows / (CTA_WARPS * ROW_SLOTS);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int cl = lane % LANE_COLS, slot = lane / LANE_COLS;
     const int team = group / CPL > 0 ? group / CPL : 1;
     const int64_t col = (int64_t)blockIdx.x * TILE_COLS + cl * CPL;
     const bool col_ok = col < C;
-    const int64_t row0 = (int64_t)blockIdx.y * TILE_ROWS;
+    const int64_t row0 = (int64_t)blockIdx.y * tile_rows;
     const f32x2 magic2 = pk2(RNE_MAGIC, RNE_MAGIC), nmagic2 = pk2(-RNE_MAGIC, -RNE_MAGIC);
     f32x2 cw[NW], acc[NW];
 #pragma unroll
@@ -635,7 +637,7 @@ reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, 
     if (!last_row && !last_col) return;
     __threadfence();
     if (last_row) {
-        for (int rr = threadIdx.x; rr < TILE_ROWS; rr += CTA_THREADS) {
+        for (int rr = threadIdx.x; rr < tile_rows; rr += CTA_THREADS) {
             const int64_t r = row0 + rr;
             if (r < R) {
                 float s = 0.f;
@@ -855,8 +857,30 @@ static sb_status reorder_impl(sb_ctx* ctx, const void* W, const void* G, int64_t
             return sb_fail(ctx, SB_ERR_SHAPE, "reorder: group in {16,32,64,128} must divide C; ldw %% 8; 16-byte base");
     }
     const int tiles_c = (int)((C + 127) / 128);
-    // tall tiles (512 rows) amortise the per-CTA prologue and epilogue when they still fill the GPU
-    const int tile_rows = (R / 512) * tiles_c >= 2 * ctx->sm_count ? 512 : 128;
+    // Tile height: the CTAs run in rounds of `slots` (three or four fit an SM), so the time is about
+    // rounds x (tile_rows + a prologue / epilogue worth some 64 rows); take the height (a multiple of
+    // 32 rows) that minimises it.  A height that leaves a few tiles for an extra round costs a
+    // whole round: 512 rows on 14336 x 4096 made 896 tiles for 444 slots, three rounds instead of two.
+    // the instance that will run, for its occupancy
+    const bool fine = ref_bits >= 6;
+    const void* kern;
+    if (G) kern = fine ? (const void*)reorder_stats_kernel<false, true, true> : (const void*)reorder_stats_kernel<false, false, true>;
+    else if (row_weight) kern = fine ? (const void*)reorder_stats_kernel<true, true, false> : (const void*)reorder_stats_kernel<true, false, false>;
+    else kern = fine ? (const void*)reorder_stats_kernel<false, true, false> : (const void*)reorder_stats_kernel<false, false, false>;
+    int occ = 0;
+    SB_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, CTA_THREADS, 0));
+    if (occ < 1) occ = 1;
+    const long long slots = (long long)occ * ctx->sm_count;
+    int tile_rows = 128;
+    {
+        long long best = -1;
+        for (int h = 32; h <= 2048; h += 32) {
+            const long long n = (long long)((R + h - 1) / h) * tiles_c;
+            const long long rounds = (n + slots - 1) / slots;
+            const long long cost = rounds * (h + 64);
+            if (best < 0 || cost < best) { best = cost; tile_rows = h; }
+        }
+    }
     const int tiles_r = (int)((R + tile_rows - 1) / tile_rows);
     const int64_t maxK = R > C ? R : C;
     void* arena;
@@ -877,18 +901,15 @@ static sb_status reorder_impl(sb_ctx* ctx, const void* W, const void* G, int64_t
         float* cpart = col_score ? colpart : nullptr;
         unsigned* done_row = ctx->stats_done;
         unsigned* done_col = ctx->stats_done + SB_STATS_TILES;
-#define SB_STATS2(RW, FN, TR, FO)                                                                 \
-    reorder_stats_kernel<RW, FN, TR, FO><<<grid, CTA_THREADS, 0, ctx->stream>>>(                  \
-        Wb, R, C, ldw, Gb, ldg, col_moment, row_weight, group, qmax, 1.0f / qmax, rpart, cpart,  \
+#define SB_STATS(RW, FN, FO)                                                                      \
+    reorder_stats_kernel<RW, FN, FO><<<grid, CTA_THREADS, 0, ctx->stream>>>(                      \
+        Wb, R, C, ldw, tile_rows, Gb, ldg, col_moment, row_weight, group, qmax, 1.0f / qmax, rpart, cpart, \
         row_score, col_score, accumulate, done_row, done_col, ctx->dstate)
-#define SB_STATS(RW, FN, FO) do { if (tile_rows == 512) SB_STATS2(RW, FN, 512, FO); else SB_STATS2(RW, FN, 128, FO); } while (0)
-        const bool fine = ref_bits >= 6;
         auto* Gb = static_cast<const __nv_bfloat16*>(G);
         if (G) { if (fine) SB_STATS(false, true, true); else SB_STATS(false, false, true); }
         else if (row_weight) { if (fine) SB_STATS(true, true, false); else SB_STATS(true, false, false); }
         else { if (fine) SB_STATS(false, true, false); else SB_STATS(false, false, false); }
 #undef SB_STATS
-#undef SB_STATS2
         SB_LAUNCHED(ctx);
     }
     if (sort_rows) { st = argsort_axis(ctx, row_score, R, row_segment, row_perm, rank); if (st) return st; }
