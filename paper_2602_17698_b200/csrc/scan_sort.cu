@@ -1,7 +1,11 @@
 // Hand-written device-wide primitives: exclusive scans (decoupled look-back) and a stable
 // LSD radix sort of 64-bit keys with 32-bit payloads (8-bit digits: per-tile histogram,
 // one scan over the digit-major histogram, stable scatter).
+#include <cooperative_groups.h>
+
 #include "lookback.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -200,6 +204,138 @@ LookbackBuf sb_lookback(sb_ctx* ctx, unsigned tiles, sb_status* st) {
     return lb;
 }
 
+// ---- small and medium inputs: the whole sort in ONE launch of one thread-block cluster ----------
+// Up to CL_SORT_PER_CTA keys (with their payloads) per CTA live in shared memory, twice over; a
+// cluster of up to 16 CTAs holds 65536 keys, CTA c the keys [c m, (c + 1) m) of the current order.
+// The eight passes run back to back inside one launch instead of as eight launches with look-back
+// chains that cost about 11 us each whatever n is.  Per pass: every warp counts the digits of its
+// tiles of 32 consecutive keys into its own histogram (match_any: one leader per distinct digit
+// of a tile adds the group's size); after a cluster barrier every CTA reads all CTAs' digit totals
+// through distributed shared memory and derives, in the same order everywhere, the first output
+// position of each of its warps per digit; the warps walk their tiles again in order, ranking
+// inside a tile by the lanes below with the same digit, and store each key into the shared memory
+// of the CTA that owns its output position.  Stable, like the large sort, so both give the same
+// permutation.
+constexpr int CL_SORT_PER_CTA = 4096;
+constexpr int CL_SORT_MAX_CTAS = 16;
+constexpr int CL_SORT_THREADS = 1024;
+constexpr int CL_SORT_WARPS = CL_SORT_THREADS / 32;
+constexpr int CL_SORT_SMEM = 2 * CL_SORT_PER_CTA * 8 + 2 * CL_SORT_PER_CTA * 4 + CL_SORT_WARPS * RADIX * 4 +
+                             CL_SORT_WARPS * RADIX * 2 + 2 * RADIX * 4 + 256;
+
+__global__ void __launch_bounds__(CL_SORT_THREADS, 1)
+cluster_sort_kernel(unsigned long long* __restrict__ keys, unsigned* __restrict__ vals, int n, int m) {
+    cg::cluster_group cluster = cg::this_cluster();
+    extern __shared__ unsigned long long cs_smem[];
+    unsigned long long* kbase = cs_smem;                                          // two key buffers
+    unsigned* vbase = reinterpret_cast<unsigned*>(cs_smem + 2 * CL_SORT_PER_CTA); // two payload buffers
+    unsigned* wbase = vbase + 2 * CL_SORT_PER_CTA;                                // [warp][digit] next output position
+    unsigned short* hist = reinterpret_cast<unsigned short*>(wbase + CL_SORT_WARPS * RADIX);   // [warp][digit] counts
+    // [2][digit] this CTA's totals, alternating by pass: a skipped pass has no second barrier, so the
+    // next pass must not write where a slower CTA may still be reading
+    unsigned* ctot2 = reinterpret_cast<unsigned*>(hist + CL_SORT_WARPS * RADIX);
+    unsigned* wtot = ctot2 + 2 * RADIX;                                                // [8] scan scratch
+    const int G = (int)gridDim.x, c = (int)blockIdx.x;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    const int lo = min(n, c * m), n_loc = min(n, lo + m) - lo;
+    for (int i = tid; i < n_loc; i += CL_SORT_THREADS) { kbase[i] = keys[lo + i]; vbase[i] = vals[lo + i]; }
+    const int tiles = (n_loc + 31) / 32;
+    const int tpw = (tiles + CL_SORT_WARPS - 1) / CL_SORT_WARPS;
+    const int tile_lo = min(tiles, warp * tpw), tile_hi = min(tiles, tile_lo + tpw);
+    int cur = 0;
+    for (int pass = 0; pass < SORT_PASSES; ++pass) {
+        const int shift = 8 * pass;
+        unsigned* ctot = ctot2 + (pass & 1) * RADIX;
+        for (int i = tid; i < CL_SORT_WARPS * RADIX / 2; i += CL_SORT_THREADS)
+            reinterpret_cast<unsigned*>(hist)[i] = 0u;
+        __syncthreads();                                   // also: the load of the input is done
+        const unsigned long long* kin = kbase + cur * CL_SORT_PER_CTA;
+        unsigned short* myh = hist + warp * RADIX;
+        // (1) digit counts of this warp's tiles
+        for (int t = tile_lo; t < tile_hi; ++t) {
+            const int i = t * 32 + lane;
+            const bool live = i < n_loc;
+            const unsigned d = live ? (unsigned)(kin[i] >> shift) & 255u : 256u + lane;     // dead lanes match nobody
+            const unsigned peers = __match_any_sync(0xffffffffu, d);
+            if (live && (peers & lt_mask) == 0u) myh[d] += (unsigned short)__popc(peers);
+            __syncwarp();
+        }
+        __syncthreads();
+        if (tid < RADIX) {
+            unsigned t = 0;
+            for (int w = 0; w < CL_SORT_WARPS; ++w) t += hist[w * RADIX + tid];
+            ctot[tid] = t;
+        }
+        cluster.sync();                                    // every CTA's digit totals are published
+        // (2) first output position of this CTA per digit: all keys with smaller digits, then the
+        // lower CTAs' keys with this digit; then of each warp
+        bool same_digit = false;                           // all keys share this pass's digit
+        if (tid < RADIX) {
+            // all remote loads first: they are independent, and one at a time each would cost a full
+            // round trip through the cluster's shared-memory network
+            unsigned v[CL_SORT_MAX_CTAS];
+#pragma unroll
+            for (int cc = 0; cc < CL_SORT_MAX_CTAS; ++cc)
+                v[cc] = cc < G ? *cluster.map_shared_rank(ctot + tid, cc) : 0u;
+            unsigned all = 0, before = 0;
+#pragma unroll
+            for (int cc = 0; cc < CL_SORT_MAX_CTAS; ++cc) {
+                all += v[cc];
+                if (cc < c) before += v[cc];
+            }
+            same_digit = all == (unsigned)n;
+            unsigned incl = all;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned y = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += y;
+            }
+            if (lane == 31) wtot[warp] = incl;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            unsigned base = incl - all + before;
+            for (int w = 0; w < warp; ++w) base += wtot[w];
+            for (int w = 0; w < CL_SORT_WARPS; ++w) {
+                wbase[w * RADIX + tid] = base;
+                base += hist[w * RADIX + tid];
+            }
+        }
+        // A pass in which every key has the same digit (the top bytes of keys of one sign and a
+        // narrow range of magnitudes) moves nothing: every CTA sees that from the same totals and
+        // skips the scatter and its barrier.
+        if (__syncthreads_or(same_digit)) continue;
+        // (3) stable scatter: tiles in order, lanes in order inside a group of equal digits; the
+        // destination is the shared memory of the CTA that owns the output position
+        const unsigned* vin = vbase + cur * CL_SORT_PER_CTA;
+        unsigned long long* kout = kbase + (cur ^ 1) * CL_SORT_PER_CTA;
+        unsigned* vout = vbase + (cur ^ 1) * CL_SORT_PER_CTA;
+        unsigned* myb = wbase + warp * RADIX;
+        for (int t = tile_lo; t < tile_hi; ++t) {
+            const int i = t * 32 + lane;
+            const bool live = i < n_loc;
+            const unsigned long long key = live ? kin[i] : 0ull;
+            const unsigned d = live ? (unsigned)(key >> shift) & 255u : 256u + lane;
+            const unsigned peers = __match_any_sync(0xffffffffu, d);
+            unsigned pos = 0;
+            if (live) pos = myb[d] + __popc(peers & lt_mask);
+            __syncwarp();
+            if (live && (peers & lt_mask) == 0u) myb[d] += __popc(peers);
+            __syncwarp();
+            if (live) {
+                const unsigned dest = pos / (unsigned)m, idx = pos - dest * (unsigned)m;
+                *cluster.map_shared_rank(kout + idx, dest) = key;
+                *cluster.map_shared_rank(vout + idx, dest) = vin[i];
+            }
+        }
+        cur ^= 1;
+        cluster.sync();                // every CTA has received its keys; counters and totals may be reused
+    }
+    for (int i = tid; i < n_loc; i += CL_SORT_THREADS) {
+        keys[lo + i] = kbase[cur * CL_SORT_PER_CTA + i];
+        vals[lo + i] = vbase[cur * CL_SORT_PER_CTA + i];
+    }
+}
+
 template <typename T>
 static sb_status scan_launch(sb_ctx* ctx, const T* in, T* out, int64_t n, int write_total) {
     if (n <= 0) {
@@ -235,6 +371,36 @@ sb_status sb_radix_sort_u64(sb_ctx* ctx, unsigned long long* keys, unsigned long
                             unsigned* vals, unsigned* vals_tmp, int64_t n, void* scratch) {
     if (n <= 0) return SB_OK;
     if (n >= (1ll << 30)) return sb_fail(ctx, SB_ERR_SHAPE, "sort: more than 2^30 keys");
+    if (n <= (int64_t)CL_SORT_PER_CTA * CL_SORT_MAX_CTAS) {
+        // one launch of one cluster, everything in shared memory; sorted in place (the eight passes
+        // of the large path also end in `keys` / `vals`).  If the cluster cannot be placed, the
+        // large path below takes over.
+        int G = 1;
+        while ((int64_t)G * CL_SORT_PER_CTA < n) G *= 2;
+        const int m = (int)((n + G - 1) / G);
+        const void* kfn = reinterpret_cast<const void*>(cluster_sort_kernel);
+        if (!ctx->configured.count(kfn)) {                 // two attributes, once per context
+            SB_CUDA(ctx, cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, CL_SORT_SMEM));
+            SB_CUDA(ctx, cudaFuncSetAttribute(kfn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+            ctx->configured.insert(kfn);
+        }
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(G);
+        cfg.blockDim = dim3(CL_SORT_THREADS);
+        cfg.dynamicSmemBytes = CL_SORT_SMEM;
+        cfg.stream = ctx->stream;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = G; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        int nn = (int)n;
+        void* kargs[] = {&keys, &vals, &nn, (void*)&m};
+        if (cudaLaunchKernelExC(&cfg, kfn, kargs) == cudaSuccess) {
+            SB_LAUNCHED(ctx);
+            return SB_OK;
+        }
+        (void)cudaGetLastError();
+    }
     const int tiles = (int)((n + SORT_TILE - 1) / SORT_TILE);
     Carver cv(scratch);
     unsigned* ghist = cv.take<unsigned>(SORT_PASSES * RADIX);
