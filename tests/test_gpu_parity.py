@@ -291,7 +291,10 @@ def _check_alloc(ctx, table, bits, budget, mode, g0=0.05, gT=0.02, sizes=None, M
 
 @pytest.mark.parametrize("kind", ["convex", "ragged", "ties"])
 @pytest.mark.parametrize("N,bits", [(7, [2, 3, 4]), (300, [2, 3, 4, 8]), (5000, [1, 2, 3, 4, 5, 6, 8]),
-                                    (13312, [2, 3, 4, 8])])
+                                    (13312, [2, 3, 4, 8]),
+                                    # step lists of 7500, 65535 and 65538 keys: a two-CTA cluster sort, the
+                                    # largest one, and the first size of the multi-launch sort
+                                    (2500, [2, 3, 4, 8]), (21845, [2, 3, 4, 8]), (21846, [2, 3, 4, 8])])
 def test_allocate_scalebits(ctx, kind, N, bits):
     from paper_2602_17698_b200.binding import SB_ALLOC_SCALEBITS
     table = _tables(N, len(bits), N, kind)
