@@ -197,7 +197,7 @@ def block_scores(W, c, bits: Sequence[int], block_rows: int = 128, block_cols: i
     return err, gain[:, :L - 1]
 
 
-def _alloc(fn, err, bits, budget, block_elems, uniform_block_elems, extra=()):
+def _alloc(fn, err, bits, budget, block_elems, uniform_block_elems, extra=(), tail=()):
     err = _f64(err)
     N, L = err.shape
     barr, Lb = _bits(bits)
@@ -206,7 +206,7 @@ def _alloc(fn, err, bits, budget, block_elems, uniform_block_elems, extra=()):
     level = np.zeros(N, dtype=np.uint8)
     rep = AllocReport()
     st = fn(_p(err), C.c_int64(N), _p(be), C.c_int64(uniform_block_elems), barr, C.c_int(L),
-            C.c_double(budget), *extra, _p(level), C.byref(rep))
+            C.c_double(budget), *extra, _p(level), C.byref(rep), *tail)
     return int(st), level, rep.as_dict()
 
 
@@ -219,6 +219,19 @@ def allocate_scalebits(err, bits, budget, gamma0=0.05, gammaT=0.02, uniform_bloc
                        block_elems=None):
     return _alloc(lib().sbo_allocate_scalebits, err, bits, budget, block_elems, uniform_block_elems,
                   extra=(C.c_double(gamma0), C.c_double(gammaT)))
+
+
+def allocate_scalebits_trace(err, bits, budget, gamma0=0.05, gammaT=0.02, uniform_block_elems=128 * 128,
+                             block_elems=None, max_iters=64):
+    """allocate_scalebits plus the level vector after every iteration -> (status, level, report,
+    trace[iterations][N])."""
+    err = _f64(err)
+    N = err.shape[0]
+    trace = np.zeros((max_iters, N), dtype=np.uint8)
+    st, level, rep = _alloc(lib().sbo_allocate_scalebits_trace, err, bits, budget, block_elems,
+                            uniform_block_elems, extra=(C.c_double(gamma0), C.c_double(gammaT)),
+                            tail=(_p(trace), C.c_int64(max_iters)))
+    return st, level, rep, trace[:min(max_iters, rep["iterations"])]
 
 
 def pack_blocks(W, bits: Sequence[int], level, block_rows=128, block_cols=128, group=128,

@@ -504,9 +504,18 @@ static int cmp_key_asc(const void* pa, const void* pb) {
     if (x->key > y->key) return 1;
     return (x->i > y->i) - (x->i < y->i);
 }
-int sbo_allocate_scalebits(const double* err, int64_t N, const int64_t* block_elems,
+/* `trace` (optional, [trace_iters][N]): the level vector as it stands at the end of every
+ * iteration of the while loop (accepted, rejected or expansion), for the first trace_iters
+ * iterations.  Recording only: the arithmetic does not depend on it.                    */
+static int allocate_scalebits_core(const double* err, int64_t N, const int64_t* block_elems,
                            int64_t uniform, const int* bits, int L, double budget,
-                           double gamma0, double gammaT, uint8_t* level, sbo_alloc_report* rep) {
+                           double gamma0, double gammaT, uint8_t* level, sbo_alloc_report* rep,
+                           uint8_t* trace, int64_t trace_iters) {
+#define SBO_TRACE_ITERATION()                                                             \
+    do {                                                                                  \
+        if (trace && rep->iterations >= 1 && rep->iterations <= trace_iters)              \
+            memcpy(trace + (size_t)(rep->iterations - 1) * (size_t)N, level, (size_t)N);  \
+    } while (0)
     if (!check_bits(bits, L) || N <= 0) return SBO_ERR_INVALID;
     if (!(gamma0 > 0.0) || !(gammaT > 0.0) || gamma0 > 1.0 || gammaT > 1.0) return SBO_ERR_INVALID;
     memset(rep, 0, sizeof *rep);
@@ -531,6 +540,7 @@ int sbo_allocate_scalebits(const double* err, int64_t N, const int64_t* block_el
     uint8_t* inU0 = (uint8_t*)malloc((size_t)N);
     int status = SBO_OK;
     while (k >= kT) {
+        SBO_TRACE_ITERATION();                          /* the iteration that just ended */
         if (++rep->iterations > 4096) { status = SBO_ERR_NOCONVERGE; break; }
         /* refresh s_up / s_down at the current allocation */
         int64_t nup = 0;
@@ -606,10 +616,29 @@ int sbo_allocate_scalebits(const double* err, int64_t N, const int64_t* block_el
             rep->rejected++;
         }
     }
+    SBO_TRACE_ITERATION();
+#undef SBO_TRACE_ITERATION
     free(up); free(dn); free(inU0);
     rep->used_bits = used; rep->proxy_loss_final = loss;
     fill_report(rep, level, N);
     return status;
+}
+
+int sbo_allocate_scalebits(const double* err, int64_t N, const int64_t* block_elems,
+                           int64_t uniform, const int* bits, int L, double budget,
+                           double gamma0, double gammaT, uint8_t* level, sbo_alloc_report* rep) {
+    return allocate_scalebits_core(err, N, block_elems, uniform, bits, L, budget, gamma0, gammaT,
+                                   level, rep, NULL, 0);
+}
+
+/* The same search, also returning the level vector after each of the first trace_iters
+ * iterations (for checking a trajectory worked by hand from Algorithm 2's text).        */
+int sbo_allocate_scalebits_trace(const double* err, int64_t N, const int64_t* block_elems,
+                                 int64_t uniform, const int* bits, int L, double budget,
+                                 double gamma0, double gammaT, uint8_t* level,
+                                 sbo_alloc_report* rep, uint8_t* trace, int64_t trace_iters) {
+    return allocate_scalebits_core(err, N, block_elems, uniform, bits, L, budget, gamma0, gammaT,
+                                   level, rep, trace, trace_iters);
 }
 
 /* ---- first-order statistics of the current allocation (Appendix E.3) --------- */

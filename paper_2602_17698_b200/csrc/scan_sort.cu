@@ -330,6 +330,9 @@ cluster_sort_kernel(unsigned long long* __restrict__ keys, unsigned* __restrict_
         cur ^= 1;
         cluster.sync();                // every CTA has received its keys; counters and totals may be reused
     }
+    // A skipped last pass ends with remote reads of the peers' digit totals and no barrier after
+    // them: no CTA may exit (and give up its shared memory) while a peer can still be reading it.
+    cluster.sync();
     for (int i = tid; i < n_loc; i += CL_SORT_THREADS) {
         keys[lo + i] = kbase[cur * CL_SORT_PER_CTA + i];
         vals[lo + i] = vbase[cur * CL_SORT_PER_CTA + i];
