@@ -20,6 +20,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "moments_body.cuh"
 
 #define SB_NOALLOC_SCRATCH_FLOATS (1 << 20)
 #define SB_NOALLOC_MAX_K 65536
@@ -28,60 +29,14 @@ static __device__ __align__(256) float sb_noalloc_scratch[SB_NOALLOC_SCRATCH_FLO
 
 namespace {
 
-constexpr int NA_TX = 32, NA_TY = 8, NA_COLS = NA_TX * 8, NA_UNROLL = 8;
+constexpr int NA_TX = MOM_TX, NA_TY = MOM_TY, NA_COLS = MOM_COLS, NA_UNROLL = MOM_UNROLL;
 
-// grid.x = chunks of 256 columns, grid.y = row splits; partial[split][K]
+// grid.x = chunks of 256 columns, grid.y = row splits; partial[split][K]: the same reduction as
+// the regular entry point (every (split, column) it later reads is written first)
 __global__ void __launch_bounds__(NA_TX * NA_TY)
 noalloc_partial_kernel(const __nv_bfloat16* __restrict__ X, int64_t T, int64_t K, int64_t ldx,
                        int64_t rows_per_split, float* __restrict__ partial) {
-    const int tx = threadIdx.x, ty = threadIdx.y;
-    const int64_t col = (int64_t)blockIdx.x * NA_COLS + tx * 8;
-    const int64_t t0 = (int64_t)blockIdx.y * rows_per_split;
-    const int64_t t1 = min(T, t0 + rows_per_split);
-    float acc[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) acc[k] = 0.f;
-    if (col < K) {
-        const __nv_bfloat16* base = X + col;
-        int64_t t = t0 + ty;
-        for (; t + (NA_UNROLL - 1) * NA_TY < t1; t += NA_UNROLL * NA_TY) {
-            uint4 v[NA_UNROLL];
-#pragma unroll
-            for (int u = 0; u < NA_UNROLL; ++u) v[u] = ld_stream16(base + (t + u * NA_TY) * ldx);
-#pragma unroll
-            for (int u = 0; u < NA_UNROLL; ++u) {
-                const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float a = bf16lo(w[k]), b = bf16hi(w[k]);
-                    acc[2 * k] = fmaf(a, a, acc[2 * k]);
-                    acc[2 * k + 1] = fmaf(b, b, acc[2 * k + 1]);
-                }
-            }
-        }
-        for (; t < t1; t += NA_TY) {
-            const uint4 v = ld_stream16(base + t * ldx);
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float a = bf16lo(w[k]), b = bf16hi(w[k]);
-                acc[2 * k] = fmaf(a, a, acc[2 * k]);
-                acc[2 * k + 1] = fmaf(b, b, acc[2 * k + 1]);
-            }
-        }
-    }
-    __shared__ float red[NA_TY][NA_COLS + 8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) red[ty][tx * 8 + k] = acc[k];
-    __syncthreads();
-    const int c = ty * NA_TX + tx;
-    const int64_t gc = (int64_t)blockIdx.x * NA_COLS + c;
-    if (gc < K) {
-        float s = 0.f;
-#pragma unroll
-        for (int y = 0; y < NA_TY; ++y) s += red[y][c];
-        partial[(int64_t)blockIdx.y * K + gc] = s;      // every (split, column) is written
-    }
+    moments_split_partial(X, T, K, ldx, rows_per_split, partial);
 }
 
 __global__ void noalloc_finish_kernel(const float* __restrict__ partial, int splits, int64_t K,

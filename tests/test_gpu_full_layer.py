@@ -25,6 +25,7 @@ STRESS_BITS = [1, 2, 3, 4, 5, 6, 8]
     (STRESS_BITS, 64, 64, 64, 2.5, 4096),
     (STRESS_BITS, 256, 128, 128, 3.5, 4096),
     ([2, 3, 4], 128, 128, 64, 3.0, 4096),
+    (STRESS_BITS, 128, 128, 32, 2.75, 4096),          # seven candidates, four groups per block width
 ])
 def test_llama3_8b_layer_full_size_sampled_parity(bits, br, bc, g, budget, tokens):
     from paper_2602_17698_b200.binding import Context

@@ -44,6 +44,16 @@ def test_gram_matrix(ctx, T, K):
     assert np.allclose(np.diag(Hh), c.cpu().double().numpy(), rtol=2e-5)
 
 
+def test_gram_matrix_at_the_calibration_token_count(ctx):
+    """65536 tokens = 128 accumulator drains of 512 tokens each: the regime in which a single
+    tensor-core accumulator was seen to drift."""
+    T, K = 65536, 256
+    X = synth.make_activations(T, K, 77, DEV)
+    H = ctx.calib_gram(X)
+    ctx.sync()
+    _check(H.cpu().double().numpy(), sbo.calib_gram(X.cpu()))
+
+
 def test_gram_accumulate_strided_and_deterministic(ctx):
     T, K = 512, 256
     big = synth.make_activations(T, K + 64, 9, DEV)
@@ -86,6 +96,50 @@ def test_block_scores_with_the_full_second_moment_matrix(ctx, R, C, g, bits, per
     e2, _ = ctx.block_scores_full(W, H, bits, 128, 128, g, row_perm=pr, col_perm=pc)
     ctx.sync()
     assert torch.equal(err, e2)                       # deterministic
+
+
+@pytest.mark.parametrize("R,C,g,bits", [(2560, 2048, 128, [2, 3, 4, 8]),     # 320 blocks, 20 per block column
+                                        (640, 8192, 64, [2, 3, 4])])        # 320 blocks, 5 per block column
+def test_full_scores_when_a_cta_walks_several_blocks_and_block_columns(ctx, R, C, g, bits):
+    """More blocks than CTAs: every CTA walks a stretch of two or three blocks of the
+    column-major block sequence, most stretches of the second shape cross a block-column
+    boundary (a new H tile), and the operand ring carries over from block to block."""
+    from tests.helpers import REL
+    W = synth.make_weight(R, C, 71 + R, DEV)
+    X = synth.make_activations(1024, C, 73 + C, DEV)
+    H = ctx.calib_gram(X)
+    rng = np.random.default_rng(R + C)
+    pc = torch.from_numpy(rng.permutation(C).astype(np.int32)).to(DEV)
+    err, _ = ctx.block_scores_full(W, H, bits, 128, 128, g, col_perm=pc)
+    ctx.sync()
+    assert err.shape[0] == (R // 128) * (C // 128) > 2 * 148
+    ref = sbo.block_scores_full(W.cpu(), H.cpu().double().numpy(), bits, 128, 128, g,
+                                col_perm=pc.cpu().numpy())
+    got = err.cpu().double().numpy()
+    assert np.all(np.abs(got - ref) <= REL * np.abs(ref)), np.max(np.abs(got - ref) / np.abs(ref))
+
+
+def test_full_scores_sampled_blocks_of_a_layer_sized_matrix(ctx):
+    """The matrix bench.py times (14336 x 4096, four candidates, 3584 blocks on 148 CTAs):
+    sampled blocks against the oracle, which is fed the GPU's H and the block's own rows and
+    columns (a block's error depends on nothing else)."""
+    from tests.helpers import REL
+    R, C, g, bits = 14336, 4096, 128, [2, 3, 4, 8]
+    W = synth.make_weight(R, C, 81, DEV)
+    X = synth.make_activations(4096, C, 83, DEV)
+    H = ctx.calib_gram(X)
+    err, _ = ctx.block_scores_full(W, H, bits, 128, 128, g)
+    ctx.sync()
+    got = err.cpu().double().numpy()
+    rng = np.random.default_rng(5)
+    nbc = C // 128
+    picks = list(rng.choice(got.shape[0], 10, replace=False)) + [0, got.shape[0] - 1]
+    for blk in picks:
+        bi, bj = divmod(int(blk), nbc)
+        tile = W[bi * 128:(bi + 1) * 128, bj * 128:(bj + 1) * 128].contiguous().cpu()
+        Hjj = H[bj * 128:(bj + 1) * 128, bj * 128:(bj + 1) * 128].cpu().double().numpy()
+        ref = sbo.block_scores_full(tile, np.ascontiguousarray(Hjj), bits, 128, 128, g)
+        assert np.all(np.abs(got[blk:blk + 1] - ref) <= REL * np.abs(ref)), (blk, got[blk], ref)
 
 
 def test_full_scores_with_a_diagonal_matrix_equal_the_diagonal_path(ctx):

@@ -316,6 +316,23 @@ def test_allocate_greedy(ctx, kind, N, bits):
         _check_alloc(ctx, table, bits, budget, SB_ALLOC_GREEDY)
 
 
+def test_allocate_scalebits_walks_the_handworked_trajectories(ctx):
+    """The instances of tests/golden/alg2_handworked.txt (derived by hand from Algorithm 2's
+    text): final levels and every counter, straight against the file."""
+    from paper_2602_17698_b200.binding import SB_ALLOC_SCALEBITS
+    from tests.test_oracle_alg2_handworked import CASES
+    for case in CASES:
+        err = torch.tensor(case["table"], dtype=torch.float32, device=DEV)
+        be = torch.tensor(case["block_elems"], dtype=torch.int64, device=DEV)
+        level, rep = ctx.allocate_bits(err, case["bits"], case["budget"], SB_ALLOC_SCALEBITS,
+                                       case["gamma0"], case["gammaT"], uniform_block_elems=0, block_elems=be)
+        fin = case["final"]
+        assert level.cpu().tolist() == case["trace"][-1], case["name"]
+        for key in ("iterations", "expansions", "accepted", "rejected", "used_bits", "cap_bits"):
+            assert rep[key] == int(fin[key]), (case["name"], key, rep)
+        assert rep["proxy_loss_init"] == fin["loss_init"] and rep["proxy_loss_final"] == fin["loss_final"]
+
+
 def test_allocate_nonuniform_block_sizes(ctx):
     from paper_2602_17698_b200.binding import SB_ALLOC_GREEDY, SB_ALLOC_SCALEBITS
     rng = np.random.default_rng(4)
