@@ -8,37 +8,12 @@
 // column factor c_j multiplies the per-column accumulators once per tile instead of once
 // per element, and every candidate bitwidth is evaluated from the same registers.
 #include "common.cuh"
+#include "quant_common.cuh"
 
 namespace {
 
-constexpr int TILE_COLS = 128;
 constexpr int CTA_THREADS = 256;
 constexpr int CTA_WARPS = CTA_THREADS / 32;
-constexpr float RNE_MAGIC = 12582912.f;        // 1.5 * 2^23: fma(x, s, MAGIC) - MAGIC = rint(x*s)
-constexpr float MIN_RANGE = 7.52316385e-37f;   // 2^-120: below this a group counts as constant
-
-struct __align__(8) BitsArg {
-    float2 q2[8];        // (qmax, qmax), qmax = 2^b - 1, as a packed fp32 pair
-    float2 niq2[8];      // (-1/qmax, -1/qmax)
-    float qmax[8];
-    float inv_qmax[8];
-    int bits[8];
-};
-
-__device__ __forceinline__ float rcp_approx(float x) {
-    float r;
-    asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
-    return r;
-}
-
-// ---- asynchronous 16-byte copies global -> shared (L2 only, no register staging) -----------
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
-    const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // ---- permuted gather: out[r][j] = W[rp[r]][cp[j]] ---------------------------------------
 // A source row is staged in shared memory with coalesced asynchronous 16-byte copies (a ring of
@@ -163,342 +138,6 @@ __device__ __forceinline__ void load_cols(const __nv_bfloat16* p, bool ok, uint3
         uint4 x = ok ? __ldg(reinterpret_cast<const uint4*>(p + 8 * v)) : make_uint4(0, 0, 0, 0);
         w[4 * v] = x.x; w[4 * v + 1] = x.y; w[4 * v + 2] = x.z; w[4 * v + 3] = x.w;
     }
-}
-
-// ---- packed fp32 pairs --------------------------------------------------------------------
-// ---- block scores ------------------------------------------------------------------------
-// Every WARP is autonomous.  The matrix is cut into slabs of 16 rows x 128 columns (4 KB),
-// numbered tile by tile, chunk column by chunk column, top to bottom; the slabs are dealt to
-// the warps of the grid in contiguous, equally long ranges, so a warp streams down the chunk
-// columns of consecutive blocks.  It stages its slabs in its own shared-memory ring with
-// asynchronous 16-byte copies (three slabs per warp, two of them in flight) and synchronises
-// with nobody but itself, so the warps of an SM drift apart and the integer/shuffle phase of
-// one warp overlaps the FP32 phase of another.  Inside a warp the two phases of consecutive
-// steps overlap as well: the loop body first reads the NEXT step's rows from shared memory and
-// reduces their group min/max (shuffles, reciprocal), then evaluates all candidates on the
-// CURRENT step's registers, and the compiler interleaves the two instruction streams.
-//
-// A lane owns 8 consecutive columns of the chunk (16 lanes cover a row) and RPL rows per step,
-// so c_j multiplies the per-column accumulators once per chunk instead of once per element.
-// Everything inside the candidate loop is packed fp32 pairs (fma/add/mul.f32x2).  When the
-// warp leaves a chunk column (or its range ends) it writes the partial block errors of that
-// stretch as record (chunk number + warp number) -- unique, because either number only grows
-// along the slab sequence -- and a second tiny kernel adds the records of a block in order.
-//
-// NFINE = how many of the L candidates (the last ones: bits ascend) keep the grid step as a
-// two-float sum: with many levels q * scale carries the fp32 rounding of the step times q, a
-// bias shared by the whole group; the residual range - scale * qmax is exact in one FMA.
-// A row weight a_r multiplies the squared residual itself (one more multiply per pair and
-// candidate in the weighted instances): scaling v - lo by sqrt(a_r) instead would round an
-// otherwise exact difference and cost two digits of accuracy at 8 bits.
-constexpr int SLAB_ROWS = 16;
-constexpr int SLAB_BYTES = SLAB_ROWS * 256;
-constexpr int SC_THREADS = 512;                 // one CTA of 16 warps per SM
-constexpr int SC_WARPS = SC_THREADS / 32;
-constexpr int RING = 3;                         // slabs per warp: one being read, two in flight
-constexpr int SC_CPL = 8;                       // columns per lane
-constexpr int SC_NW = SC_CPL / 2;               // packed pairs per lane and row
-
-struct ScoreGeom {
-    int br, bc, group;
-    int chunks, tile_w, spb;       // 128-column chunks per tile; tile width; slabs per chunk column
-    int nsub, lanes_per_sub;       // blocks side by side in a chunk (bc < 128); lanes across one block
-    unsigned n_tile_cols, n_slabs, n_warps;
-};
-
-// owner of slab s when warp w takes slabs [n_slabs * w / n_warps, n_slabs * (w + 1) / n_warps)
-__device__ __forceinline__ unsigned slab_owner(unsigned s, unsigned n_slabs, unsigned n_warps) {
-    return (unsigned)((((unsigned long long)s + 1ull) * n_warps - 1ull) / n_slabs);
-}
-// warps between two owners may have an empty range (more warps than slabs): they write no record
-__device__ __forceinline__ bool slab_range_empty(unsigned w, unsigned n_slabs, unsigned n_warps) {
-    return (unsigned long long)n_slabs * w / n_warps == (unsigned long long)n_slabs * (w + 1) / n_warps;
-}
-
-struct SlabCursor { int sl, ch; unsigned bx, by; };
-
-template <int RPL>
-struct StepRegs {
-    uint32_t w[RPL][SC_NW];
-    float lo[RPL], rinv[RPL], range[RPL], ar[RPL];   // ar: row weight a_r (1 without weights)
-    unsigned q;          // chunk column (in slab-sequence order) the step belongs to
-    int col;             // first column of that chunk
-    int row;             // first row of the step (the lane's rows are row + slot + 2 i)
-    bool flush;          // last step of the warp's stretch of this chunk column
-};
-
-// The walk itself.  P supplies what is done with a step (P::burst) and with the end of a
-// stretch (P::flush), and keeps its accumulators in registers.
-template <class P>
-__global__ void __launch_bounds__(SC_THREADS, 1)
-slab_walk_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw,
-                 const int32_t* __restrict__ load_row_perm,   // rows gathered at load time
-                 const int32_t* __restrict__ a_perm,          // original row of permuted r
-                 const float* __restrict__ row_weight, ScoreGeom g, typename P::Args pa) {
-    constexpr int RPL = P::RPL;
-    constexpr int STEP_ROWS = 2 * RPL;              // rows per warp step
-    extern __shared__ __align__(16) unsigned char tile_smem[];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int cl = lane & 15, slot = lane >> 4;
-    const int team = g.group / SC_CPL;
-    const unsigned gw = blockIdx.x * SC_WARPS + warp;
-    const unsigned s_lo = (unsigned)((unsigned long long)g.n_slabs * gw / g.n_warps);
-    const unsigned s_hi = (unsigned)((unsigned long long)g.n_slabs * (gw + 1) / g.n_warps);
-    if (s_lo >= s_hi) return;                       // no barriers in this kernel
-    unsigned char* ring = tile_smem + (size_t)warp * (RING * SLAB_BYTES);
-
-    auto advance = [&](SlabCursor& c) {
-        if (++c.sl == g.spb) {
-            c.sl = 0;
-            if (++c.ch == g.chunks) {
-                c.ch = 0;
-                if (++c.bx == g.n_tile_cols) { c.bx = 0; ++c.by; }
-            }
-        }
-    };
-    SlabCursor rc;                                   // read cursor
-    unsigned r_q = s_lo / (unsigned)g.spb;           // chunk column of the read cursor
-    {
-        rc.sl = (int)(s_lo - r_q * (unsigned)g.spb);
-        const unsigned t = r_q / (unsigned)g.chunks;
-        rc.ch = (int)(r_q - t * (unsigned)g.chunks);
-        rc.by = t / g.n_tile_cols;
-        rc.bx = t - rc.by * g.n_tile_cols;
-    }
-    SlabCursor ic = rc;                              // issue cursor, RING - 1 slabs ahead
-    unsigned i_s = s_lo;
-    int i_stage = 0;
-    // stage the next slab of the range (an empty group past its end keeps the wait count fixed)
-    auto issue_next = [&]() {
-        if (i_s < s_hi) {
-            const int rows_here = min(SLAB_ROWS, g.br - ic.sl * SLAB_ROWS);
-            const int64_t row0 = (int64_t)ic.by * g.br + ic.sl * SLAB_ROWS;
-            const __nv_bfloat16* src = W + ((int64_t)ic.bx * g.tile_w + ic.ch * TILE_COLS + cl * SC_CPL);
-            unsigned char* dst = ring + i_stage * SLAB_BYTES + slot * 256 + cl * 16;
-            if (load_row_perm) {
-                const int32_t* rp = load_row_perm + row0;
-                for (int row = slot; row < rows_here; row += 2, dst += 512)
-                    cp_async16(dst, src + (int64_t)rp[row] * ldw);
-            } else {
-                src += (row0 + slot) * ldw;
-                if (rows_here == SLAB_ROWS) {
-#pragma unroll
-                    for (int i = 0; i < SLAB_ROWS / 2; ++i) cp_async16(dst + i * 512, src + (int64_t)(2 * i) * ldw);
-                } else {
-                    for (int row = slot; row < rows_here; row += 2, dst += 512, src += 2 * ldw)
-                        cp_async16(dst, src);
-                }
-            }
-            advance(ic);
-            ++i_s;
-        }
-        cp_async_commit();
-        i_stage = i_stage + 1 == RING ? 0 : i_stage + 1;
-    };
-
-    unsigned r_s = s_lo;
-    int r_stage = 0, r_step = 0, r_steps = 0;
-    bool more = true;                                // a step remains to be loaded
-    // the slab at the read cursor becomes readable; the stage left behind is refilled
-    auto enter_slab = [&]() {
-        __syncwarp();
-        issue_next();
-        cp_async_wait<RING - 1>();
-        __syncwarp();
-        r_steps = min(SLAB_ROWS, g.br - rc.sl * SLAB_ROWS) / STEP_ROWS;
-        r_step = 0;
-    };
-    // rows of the step at the read cursor -> registers, group min/max and reciprocal; advance
-    auto load_step = [&](StepRegs<RPL>& n) {
-        const unsigned char* src = ring + r_stage * SLAB_BYTES + (r_step * STEP_ROWS + slot) * 256 + cl * 16;
-#pragma unroll
-        for (int i = 0; i < RPL; ++i) {
-            const uint4 x = *reinterpret_cast<const uint4*>(src + i * 512);
-            n.w[i][0] = x.x; n.w[i][1] = x.y; n.w[i][2] = x.z; n.w[i][3] = x.w;
-        }
-        n.row = (int)(rc.by * (unsigned)g.br) + rc.sl * SLAB_ROWS + r_step * STEP_ROWS;
-#pragma unroll
-        for (int i = 0; i < RPL; ++i) {
-            float lo, hi;
-            group_minmax<SC_NW, P::FULLG ? 16 : 0>(n.w[i], team, lo, hi);
-            const float range = hi - lo;
-            const bool live = range >= MIN_RANGE;
-            const float rinv = rcp_approx(range);
-            float ar = 1.f;
-            if (P::ROWW) {
-                const int r = n.row + 2 * i + slot;
-                ar = row_weight[a_perm ? a_perm[r] : r];
-            }
-            n.lo[i] = lo;
-            n.rinv[i] = live ? rinv : 0.f;
-            n.range[i] = live ? range : 0.f;
-            n.ar[i] = ar;
-        }
-        n.q = r_q;
-        n.col = (int)(rc.bx * (unsigned)g.tile_w) + rc.ch * TILE_COLS;
-        n.flush = false;
-        if (++r_step == r_steps) {                   // the slab is in registers: move on
-            n.flush = rc.sl == g.spb - 1 || r_s + 1 == s_hi;
-            if (rc.sl == g.spb - 1) ++r_q;
-            advance(rc);
-            ++r_s;
-            r_stage = r_stage + 1 == RING ? 0 : r_stage + 1;
-            if (r_s < s_hi) enter_slab(); else more = false;
-        }
-    };
-
-    P p(pa, g, gw, cl, slot);
-#pragma unroll
-    for (int i = 0; i < RING - 1; ++i) issue_next();
-    enter_slab();
-    StepRegs<RPL> A, B;
-    load_step(A);
-    while (true) {
-        const bool haveB = more;
-        if (haveB) load_step(B);
-        p.burst(A);
-        if (A.flush) p.flush(A);
-        if (!haveB) break;
-        const bool haveA = more;
-        if (haveA) load_step(A);
-        p.burst(B);
-        if (B.flush) p.flush(B);
-        if (!haveA) break;
-    }
-    cp_async_wait<0>();
-}
-
-// v - lo of a lane's 8 columns as packed pairs (exact: both are bf16 values of one group)
-template <int RPL>
-__device__ __forceinline__ void centred_pairs(const StepRegs<RPL>& s, int i, f32x2 (&vm)[SC_NW]) {
-    const f32x2 nlo2 = pk2(-s.lo[i], -s.lo[i]);
-#pragma unroll
-    for (int k = 0; k < SC_NW; ++k) {
-        // low half through the byte permuter: the shift would take a slot of the FP32 pipe
-        const float v0 = __uint_as_float(__byte_perm(s.w[i][k], 0u, 0x1044));
-        vm[k] = add2(pk2(v0, bf16hi(s.w[i][k])), nlo2);
-    }
-}
-
-// Block scores: all L candidates per step, per-column accumulators, one record per stretch.
-template <int L_, int RPL_, int NFINE, bool FULLG_, bool ROWW_>
-struct ScorePolicy {
-    static constexpr int L = L_, RPL = RPL_;
-    static constexpr bool FULLG = FULLG_, ROWW = ROWW_;
-    struct Args {
-        const int32_t* c_perm;           // original column of permuted j
-        const float* col_moment;
-        BitsArg ba;
-        float* rec;
-    };
-    const Args& a;
-    const ScoreGeom& g;
-    const unsigned gw;
-    const int cl, slot;
-    f32x2 acc[SC_NW][L];
-    __device__ __forceinline__ ScorePolicy(const Args& a_, const ScoreGeom& g_, unsigned gw_, int cl_, int slot_)
-        : a(a_), g(g_), gw(gw_), cl(cl_), slot(slot_) {
-#pragma unroll
-        for (int k = 0; k < SC_NW; ++k)
-#pragma unroll
-            for (int l = 0; l < L; ++l) acc[k][l] = 0ull;
-    }
-    __device__ __forceinline__ void burst(const StepRegs<RPL>& s) {
-        const f32x2 magic2 = pk2(RNE_MAGIC, RNE_MAGIC), nmagic2 = pk2(-RNE_MAGIC, -RNE_MAGIC);
-#pragma unroll
-        for (int i = 0; i < RPL; ++i) {
-            const f32x2 rinv2 = pk2(s.rinv[i], s.rinv[i]), range2 = pk2(s.range[i], s.range[i]);
-            const f32x2 ar2 = pk2(s.ar[i], s.ar[i]);
-            f32x2 vm[SC_NW];
-            centred_pairs<RPL>(s, i, vm);
-#pragma unroll
-            for (int l = 0; l < L; ++l) {
-                const f32x2 q2 = *reinterpret_cast<const f32x2*>(&a.ba.q2[l]);
-                const f32x2 niq2 = *reinterpret_cast<const f32x2*>(&a.ba.niq2[l]);
-                const f32x2 inv2 = mul2(q2, rinv2);
-                const f32x2 ns2 = mul2(niq2, range2);                   // -(range / qmax)
-                if (l >= L - NFINE) {
-                    const f32x2 nslo2 = mul2(fma2(ns2, q2, range2), niq2);   // -(residual / qmax)
-#pragma unroll
-                    for (int k = 0; k < SC_NW; ++k) {
-                        const f32x2 qq = add2(fma2(vm[k], inv2, magic2), nmagic2);
-                        const f32x2 e = fma2(qq, nslo2, fma2(qq, ns2, vm[k]));
-                        acc[k][l] = fma2(ROWW ? mul2(e, ar2) : e, e, acc[k][l]);
-                    }
-                } else {
-#pragma unroll
-                    for (int k = 0; k < SC_NW; ++k) {
-                        const f32x2 qq = add2(fma2(vm[k], inv2, magic2), nmagic2);
-                        const f32x2 e = fma2(qq, ns2, vm[k]);
-                        acc[k][l] = fma2(ROWW ? mul2(e, ar2) : e, e, acc[k][l]);
-                    }
-                }
-            }
-        }
-    }
-    // column factors, lanes of the same block, record (chunk number + warp number)
-    __device__ __forceinline__ void flush(const StepRegs<RPL>& s) {
-        const int col = s.col + cl * SC_CPL;
-        f32x2 c2[SC_NW];
-#pragma unroll
-        for (int k = 0; k < SC_NW; ++k) {
-            const int j = col + 2 * k;
-            c2[k] = pk2(__ldg(a.col_moment + (a.c_perm ? a.c_perm[j] : j)),
-                        __ldg(a.col_moment + (a.c_perm ? a.c_perm[j + 1] : j + 1)));
-        }
-        float tot[L];
-#pragma unroll
-        for (int l = 0; l < L; ++l) {
-            f32x2 t2 = 0ull;
-#pragma unroll
-            for (int k = 0; k < SC_NW; ++k) { t2 = fma2(c2[k], acc[k][l], t2); acc[k][l] = 0ull; }
-            float a0, a1;
-            upk2(t2, a0, a1);
-            float v = a0 + a1;
-            for (int o = g.lanes_per_sub >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            v += __shfl_xor_sync(0xffffffffu, v, 16);
-            tot[l] = v;
-        }
-        if (slot == 0 && (cl % g.lanes_per_sub) == 0) {
-            float* dst = a.rec + ((size_t)(s.q + gw) * g.nsub + cl / g.lanes_per_sub) * L;
-#pragma unroll
-            for (int l = 0; l < L; ++l) dst[l] = tot[l];
-        }
-    }
-};
-
-// err[blk][l] = sum of the records of the block's chunk columns, in slab order; gains;
-// non-finite check
-__global__ void scores_finish_kernel(const float* __restrict__ rec, ScoreGeom g, int64_t n_blocks,
-                                     int64_t n_block_cols, int L, BitsArg ba, float M,
-                                     float* __restrict__ err, float* __restrict__ gain,
-                                     SbDeviceState* dstate) {
-    const int64_t blk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (blk >= n_blocks) return;
-    const unsigned by = (unsigned)(blk / n_block_cols), bxb = (unsigned)(blk - (int64_t)by * n_block_cols);
-    const unsigned bx = bxb / (unsigned)g.nsub, sb = bxb - bx * (unsigned)g.nsub;
-    const unsigned t = by * g.n_tile_cols + bx;
-    float e[8];
-    for (int l = 0; l < L; ++l) e[l] = 0.f;
-    for (int ch = 0; ch < g.chunks; ++ch) {
-        const unsigned q = t * (unsigned)g.chunks + (unsigned)ch;
-        const unsigned s0 = q * (unsigned)g.spb, s1 = s0 + (unsigned)g.spb - 1u;
-        const unsigned w0 = slab_owner(s0, g.n_slabs, g.n_warps), w1 = slab_owner(s1, g.n_slabs, g.n_warps);
-        for (unsigned w = w0; w <= w1; ++w) {
-            if (slab_range_empty(w, g.n_slabs, g.n_warps)) continue;
-            const float* src = rec + ((size_t)(q + w) * g.nsub + sb) * L;
-            for (int l = 0; l < L; ++l) e[l] += src[l];
-        }
-    }
-    bool finite = true;
-    for (int l = 0; l < L; ++l) {
-        err[blk * L + l] = e[l];
-        finite = finite && isfinite(e[l]);
-    }
-    if (!finite) sb_latch(dstate, SB_ERR_NONFINITE, SBK_SCORES);
-    if (gain)
-        for (int l = 0; l + 1 < L; ++l)
-            gain[blk * (L - 1) + l] = (e[l] - e[l + 1]) / ((float)(ba.bits[l + 1] - ba.bits[l]) * M);
 }
 
 // ---- reorder statistics --------------------------------------------------------------------
@@ -733,21 +372,6 @@ __global__ void expand_perm_kernel(int32_t* out, const int32_t* __restrict__ per
     for (int u = 0; u < reps; ++u) out[(h * reps + u) * seg + d] = (int32_t)((h * reps + u) * seg + local);
 }
 
-BitsArg make_bits(const int* bits, int n) {
-    BitsArg ba{};
-    for (int l = 0; l < 8; ++l) {
-        const int b = l < n ? bits[l] : 1;
-        ba.bits[l] = b;
-        ba.qmax[l] = (float)((1 << b) - 1);
-        ba.inv_qmax[l] = 1.0f / (float)((1 << b) - 1);
-        ba.q2[l] = make_float2(ba.qmax[l], ba.qmax[l]);
-        ba.niq2[l] = make_float2(-ba.inv_qmax[l], -ba.inv_qmax[l]);
-    }
-    return ba;
-}
-
-bool valid_group(int g) { return g == 16 || g == 32 || g == 64 || g == 128; }
-
 sb_status argsort_axis(sb_ctx* ctx, const float* score, int64_t K, int64_t seg, int32_t* perm, int* rank) {
     SB_CUDA(ctx, cudaMemsetAsync(rank, 0, sizeof(int) * K, ctx->stream));
     if (seg % 256 == 0) {
@@ -768,43 +392,6 @@ sb_status argsort_axis(sb_ctx* ctx, const float* score, int64_t K, int64_t seg, 
     rank_scatter_kernel<<<(unsigned)((K + 255) / 256), 256, 0, ctx->stream>>>(rank, K, seg, perm);
     SB_LAUNCHED(ctx);
     return SB_OK;
-}
-
-template <int L, int RPL, int NFINE, bool FULLG, bool ROWW>
-sb_status launch_scores_k(sb_ctx* ctx, const __nv_bfloat16* W, int64_t ldw, const int32_t* lrp,
-                          const int32_t* cperm, const int32_t* aperm, const float* cm, const float* rw,
-                          const ScoreGeom& g, const BitsArg& ba, int64_t n_blocks, int64_t nbc, int grid,
-                          float* err, float* gain, float* rec) {
-    const size_t smem = (size_t)SC_WARPS * RING * SLAB_BYTES;
-    using P = ScorePolicy<L, RPL, NFINE, FULLG, ROWW>;
-    auto kern = slab_walk_kernel<P>;
-    SB_FUNC_ATTR(ctx, kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    typename P::Args pa{cperm, cm, ba, rec};
-    kern<<<(unsigned)grid, SC_THREADS, smem, ctx->stream>>>(W, ldw, lrp, aperm, rw, g, pa);
-    SB_LAUNCHED(ctx);
-    scores_finish_kernel<<<(unsigned)((n_blocks + 255) / 256), 256, 0, ctx->stream>>>(
-        rec, g, n_blocks, nbc, L, ba, (float)g.br * (float)g.bc, err, gain, ctx->dstate);
-    SB_LAUNCHED(ctx);
-    return SB_OK;
-}
-
-// the common case (group = 128 columns, no row weights) gets its own instance with the
-// group reduction unrolled; everything else shares the general one
-template <int L, int RPL, int NFINE, typename... A>
-sb_status launch_scores_n(int group, const float* rw, A... args) {
-    if (group == 128 && !rw) return launch_scores_k<L, RPL, NFINE, true, false>(args...);
-    if (!rw) return launch_scores_k<L, RPL, NFINE, false, false>(args...);
-    return launch_scores_k<L, RPL, NFINE, false, true>(args...);
-}
-
-// candidates with >= 6 bits keep a two-float grid step; they are the last `nfine` of the list.
-// Compiled for 0..2 such candidates and for "all of them" (always correct, a little slower).
-template <int L, int RPL, typename... A>
-sb_status launch_scores(int nfine, A... args) {
-    if (nfine == 0) return launch_scores_n<L, RPL, 0>(args...);
-    if (nfine == 1 && L >= 1) return launch_scores_n<L, RPL, (L >= 1 ? 1 : L)>(args...);
-    if (nfine == 2 && L >= 2) return launch_scores_n<L, RPL, (L >= 2 ? 2 : L)>(args...);
-    return launch_scores_n<L, RPL, L>(args...);
 }
 
 }  // namespace
@@ -958,78 +545,6 @@ sb_status sb_expand_segment_perm(sb_ctx* ctx, int32_t* out, const int32_t* perm,
     expand_perm_kernel<<<(unsigned)((n_src + 255) / 256), 256, 0, ctx->stream>>>(out, perm, n_src, reps, seg);
     SB_LAUNCHED(ctx);
     return SB_OK;
-}
-
-sb_status sb_block_scores(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw,
-                          const int32_t* row_perm, const int32_t* col_perm, const float* col_moment,
-                          const float* row_weight, int br, int bc, int group, const int* bits,
-                          int n_bits, float* err, float* gain, void* W_perm_out) {
-    if (!ctx) return SB_ERR_INVALID;
-    if (!W || !col_moment || !err || R <= 0 || C <= 0) return sb_fail(ctx, SB_ERR_INVALID, "scores: null or empty");
-    if (!sb_check_bits(bits, n_bits)) return sb_fail(ctx, SB_ERR_INVALID, "scores: bits must be ascending in 1..8");
-    if (br <= 0 || bc <= 0 || br % 4 || R % br || C % bc || !valid_group(group) || bc % group ||
-        !(bc == 32 || bc == 64 || bc % 128 == 0) || ldw % 8 || ldw < C ||
-        (reinterpret_cast<uintptr_t>(W) & 15))
-        return sb_fail(ctx, SB_ERR_SHAPE, "scores: block %dx%d group %d does not tile %lldx%lld", br, bc,
-                       group, (long long)R, (long long)C);
-    SB_CUDA(ctx, cudaSetDevice(ctx->device));
-    const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(W);
-    int64_t ld = ldw;
-    const int32_t* load_rp = row_perm;
-    // geometry of the slab walk and the record buffer of the partial sums
-    ScoreGeom geo{};
-    geo.br = br; geo.bc = bc; geo.group = group;
-    geo.tile_w = bc >= TILE_COLS ? bc : TILE_COLS;
-    if (C % geo.tile_w) return sb_fail(ctx, SB_ERR_SHAPE, "scores: C must be a multiple of 128");
-    geo.chunks = geo.tile_w / TILE_COLS;
-    geo.spb = (br + SLAB_ROWS - 1) / SLAB_ROWS;
-    geo.nsub = bc >= TILE_COLS ? 1 : TILE_COLS / bc;
-    geo.lanes_per_sub = bc >= TILE_COLS ? TILE_COLS / SC_CPL : bc / SC_CPL;
-    geo.n_tile_cols = (unsigned)(C / geo.tile_w);
-    const int64_t n_chunk_cols = (R / br) * (int64_t)geo.n_tile_cols * geo.chunks;
-    const int64_t n_slabs = n_chunk_cols * geo.spb;
-    if (n_slabs >= (1ll << 31)) return sb_fail(ctx, SB_ERR_SHAPE, "scores: matrix too large");
-    geo.n_slabs = (unsigned)n_slabs;
-    int64_t grid = (n_slabs + SC_WARPS - 1) / SC_WARPS;       // persistent: one 16-warp CTA per SM
-    if (grid > ctx->sm_count) grid = ctx->sm_count;
-    geo.n_warps = (unsigned)(grid * SC_WARPS);
-    const int64_t nbc = C / bc, n_blocks = (R / br) * nbc;
-    const size_t rec_bytes = (size_t)(n_chunk_cols + geo.n_warps) * geo.nsub * n_bits * sizeof(float);
-    const bool need_copy = col_perm || W_perm_out;
-    void* arena;
-    sb_status sst = sb_scratch(ctx, Carver::need({rec_bytes, (need_copy && !W_perm_out) ? (size_t)R * C * 2 : 0}),
-                               &arena);
-    if (sst != SB_OK) return sst;
-    Carver cv(arena);
-    float* rec = cv.take<float>(rec_bytes / sizeof(float));
-    if (need_copy) {
-        void* dst = W_perm_out ? W_perm_out : static_cast<void*>(cv.take<unsigned char>((size_t)R * C * 2));
-        sb_status st = sb_gather_bf16(ctx, W, R, C, ldw, row_perm, col_perm, dst);
-        if (st != SB_OK) return st;
-        src = static_cast<const __nv_bfloat16*>(dst);
-        ld = C;
-        load_rp = nullptr;
-    }
-    const BitsArg ba = make_bits(bits, n_bits);
-    sb_status st = SB_OK;
-    int nfine = 0;
-    for (int l = 0; l < n_bits; ++l) nfine += bits[l] >= 6;
-    // up to four candidates: a lane takes two rows per step; more: one row (fewer accumulators)
-#define SB_SCORES(Lv, RPLv)                                                                        \
-    st = launch_scores<Lv, RPLv>(nfine, group, row_weight, ctx, src, ld, load_rp, col_perm, row_perm, \
-                                 col_moment, row_weight, geo, ba, n_blocks, nbc, (int)grid, err, gain, rec)
-    switch (n_bits) {
-        case 1: SB_SCORES(1, 2); break;
-        case 2: SB_SCORES(2, 2); break;
-        case 3: SB_SCORES(3, 2); break;
-        case 4: SB_SCORES(4, 2); break;
-        case 5: SB_SCORES(5, 1); break;
-        case 6: SB_SCORES(6, 1); break;
-        case 7: SB_SCORES(7, 1); break;
-        default: SB_SCORES(8, 1); break;
-    }
-#undef SB_SCORES
-    return st;
 }
 
 }  // extern "C"
