@@ -30,11 +30,12 @@ WORKLOAD = ("one Llama-3-8B-shaped decoder layer (q/o 4096x4096, k/v 1024x4096, 
             "down 4096x14336; 218,103,808 bf16 weights), 65536 calibration tokens per input, "
             "blocks 128x128, group 128, bits {2,3,4,8}, budget 2.5")
 
-# (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of the dominant kernel, from the
-# ncu capture summarised in profiles/moments_partial_kernel_65536x4096.md (541.04 MB moved for
-# 536.87 MB of activations); the kernel's traffic is proportional to T * K, so the ratio carries
-# over to the launches of the step
+# (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of the dominant kernel, from one
+# ncu capture of a 65536 x 4096 input (541.04 MB moved for 536.87 MB of activations); the kernel's
+# traffic is proportional to T * K, so the ratio carries over to the launches of the step
 NCU_TRAFFIC_RATIO = {"moments_partial_kernel": 1.0071}
+NOMINAL_HBM_GBS = 8000.0      # the B200's nominal HBM3e bandwidth: the figure the 70 % target is stated on
+STRESS_BITS = (1, 2, 3, 4, 5, 6, 8)
 
 
 def measured_peaks():
@@ -151,6 +152,31 @@ def time_oracle(steps: int, warmup: int):
     return n / dt, dt / steps, sbo.num_threads(), SAMPLE_TEXT
 
 
+def oracle_full_matrix():
+    """The oracle on ONE full-size matrix of the layer (q_proj, 4096 x 4096) with the full 65536-token
+    input: moments, reorder statistics and sorts, block scores, allocation, pack, as they stand."""
+    import numpy as np
+    from oracle import sbo
+    from paper_2602_17698_b200 import synth
+    shape = synth.LLAMA3_8B
+    l = next(x for x in shape.linears if x.name == "q_proj")
+    w = synth.make_weight(l.rows, l.cols, synth.tensor_seed(SEED, 0, l.tensor_id))
+    x = synth.make_activations(TOKENS, l.cols, synth.tensor_seed(SEED, 0, synth.ACT_TENSOR_ID[l.act]))
+    t0 = time.perf_counter()
+    c = sbo.calib_moments(x, 1.0 / x.shape[0])
+    t1 = time.perf_counter()
+    rs, cs = sbo.reorder_scores(w, c, ref_bits=2, group=128)
+    pr, pc = sbo.argsort_desc_segments(rs), sbo.argsort_desc_segments(cs)
+    err, _ = sbo.block_scores(w, c, BITS, 128, 128, 128, row_perm=pr, col_perm=pc)
+    st, level, _ = sbo.allocate_scalebits(err, BITS, BUDGET, 0.05, 0.02, 128 * 128)
+    assert st == sbo.OK
+    sbo.pack_blocks(w, BITS, level, 128, 128, 128, row_perm=pr, col_perm=pc)
+    t2 = time.perf_counter()
+    n = l.rows * l.cols
+    return {"matrix": "q_proj 4096 x 4096, 65536 tokens", "seconds_moments": t1 - t0,
+            "seconds_weight_stages": t2 - t1, "value": n / (t2 - t0), "unit": UNIT}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -201,12 +227,14 @@ def measured_tensor_peak():
     return 1590.0, "fallback"
 
 
-def kernel_rooflines(ctx, W, X, moments, dev, peak_gbs, sm_mhz):
+def kernel_rooflines(ctx, W, X, moments, dev, peak_gbs, sm_mhz, sm_count):
     """The other kernels of the path, one library call at a time on 14336 x 4096 matrices (three
     different ones in rotation, 352 MB > L2, so every call streams from HBM), CUDA events on the
     context's stream.  HBM-bound kernels against the measured copy bandwidth; the score kernel
-    against the FP32 pipe: 148 SMs x 128 lanes x SM clock lane-operations per second, with
-    4 L + 1 + (candidates of >= 6 bits) algorithmic lane-operations per weight."""
+    against the FP32 pipe: SMs x 128 lanes x SM clock lane-operations per second, with
+    4 L + 1 + (candidates of >= 6 bits) algorithmic lane-operations per weight.  The score kernel is
+    timed for the bit sets of every config ({2,3,4,8}, {2,3,4}, {1,2,3,4,5,6,8}) and for the block
+    shapes and group sizes at the corners of the stress sweep."""
     import torch
     mats = [W["gate_proj"], W["up_proj"], W["gate_proj"].clone()]
     c = moments["mlp_in"]
@@ -238,6 +266,14 @@ def kernel_rooflines(ctx, W, X, moments, dev, peak_gbs, sm_mhz):
 
     t_stats = timed(lambda m: ctx.reorder_channels(m, c, 2, 128, row_score=rs, col_score=cs))
     t_score = timed(lambda m: ctx.block_scores(m, c, BITS, 128, 128, 128, err=err, want_gain=False))
+    score_variants = []
+    for bits_v, br_v, bc_v, g_v in (((2, 3, 4), 128, 128, 128), (STRESS_BITS, 128, 128, 128),
+                                    (STRESS_BITS, 128, 128, 32), (STRESS_BITS, 32, 32, 32),
+                                    (STRESS_BITS, 64, 64, 64), (STRESS_BITS, 256, 128, 128)):
+        err_v = torch.empty((R // br_v) * (Cc // bc_v), len(bits_v), **f32)
+        t_v = timed(lambda m: ctx.block_scores(m, c, bits_v, br_v, bc_v, g_v, err=err_v, want_gain=False))
+        score_variants.append((bits_v, br_v, bc_v, g_v, t_v))
+        del err_v
     t_perm = timed(lambda m: ctx.block_scores(m, c, BITS, 128, 128, 128, row_perm=pr, col_perm=pc, err=err,
                                               want_gain=False, W_perm_out=out))
     t_pack = timed(lambda m: ctx.pack_blocks(m, BITS, level, 128, 128, 128, packed=packed, block_off=off,
@@ -276,19 +312,27 @@ def kernel_rooflines(ctx, W, X, moments, dev, peak_gbs, sm_mhz):
     def hbm(name, bytes_, ms, note):
         a = bytes_ / (ms * 1e-3) / 1e9
         return {"kernel": name, "bound": "hbm", "achieved": a, "peak": peak_gbs, "unit": "GB/s",
-                "frac": a / peak_gbs, "ms_per_call": ms, "algorithmic_bytes": bytes_, "note": note}
+                "frac": a / peak_gbs, "frac_nominal": a / NOMINAL_HBM_GBS, "ms_per_call": ms,
+                "algorithmic_bytes": bytes_, "note": note}
 
-    fine = sum(1 for b in BITS if b >= 6)
-    ops = 4 * len(BITS) + 1 + fine
-    alu_peak = 148 * 128 * sm_mhz * 1e6 / 1e12
-    a_ops = n * ops / (t_score * 1e-3) / 1e12
+    alu_peak = sm_count * 128 * sm_mhz * 1e6 / 1e12
+
+    def score_entry(bits_v, br_v, bc_v, g_v, ms):
+        ops = 4 * len(bits_v) + 1 + sum(1 for b in bits_v if b >= 6)
+        a_ops = n * ops / (ms * 1e-3) / 1e12
+        gbs = 2 * n / (ms * 1e-3) / 1e9
+        return {"kernel": "block_scores_kernel (+ scores_finish_kernel)", "bound": "alu", "achieved": a_ops,
+                "peak": alu_peak, "unit": "T fp32 lane-ops/s", "frac": a_ops / alu_peak, "ms_per_call": ms,
+                "bits": list(bits_v), "block": [br_v, bc_v], "group": g_v, "lane_ops_per_weight": ops,
+                "hbm_gbs": gbs, "hbm_frac": gbs / peak_gbs, "hbm_frac_nominal": gbs / NOMINAL_HBM_GBS,
+                "elements_per_s": n / (ms * 1e-3),
+                "note": f"one call of sb_block_scores without permutations; peak = {sm_count} SMs x 128 lanes "
+                        "x SM clock"}
+
     return [
         hbm("reorder_stats_kernel", 2 * n, t_stats, "one call of sb_reorder_channels (statistics only)"),
-        {"kernel": "slab_walk_kernel<ScorePolicy> (+ scores_finish_kernel)", "bound": "alu", "achieved": a_ops,
-         "peak": alu_peak, "unit": "T fp32 lane-ops/s", "frac": a_ops / alu_peak, "ms_per_call": t_score,
-         "lane_ops_per_weight": ops, "hbm_gbs": 2 * n / (t_score * 1e-3) / 1e9,
-         "hbm_frac": 2 * n / (t_score * 1e-3) / 1e9 / peak_gbs,
-         "note": "one call of sb_block_scores without permutations; peak = 148 SMs x 128 lanes x SM clock"},
+        score_entry(BITS, 128, 128, 128, t_score),
+    ] + [score_entry(*v) for v in score_variants] + [
         hbm("gather_cols_kernel", 4 * n, t_gather,
             "sb_block_scores with both permutations and W_perm_out minus the call without (2 B read + 2 B written)"),
         hbm("pack_offsets_small_kernel + pack_kernel", int(2 * n + n * avg_bits / 8 + n / 128 * 8), t_pack,
@@ -424,6 +468,133 @@ def full_model_times(ctx, dev):
                       "made twice and the faster one counted (it is eager and paced by the host)"}
 
 
+def small_layer_times(ctx, dev):
+    """configs[0]: one 2048 x 2048 layer, 8192 calibration tokens, blocks 128 x 128, bits {2,3,4},
+    budget 3.0, no coupling (rows and columns sorted freely): the whole path per call, CUDA events,
+    20 repetitions after 3 warm-up passes.  2048 x 2048 weights (8 MB) and 8192 x 2048 activations
+    (33.5 MB) fit in L2, so a buffer larger than L2 is written between repetitions."""
+    import torch
+    from paper_2602_17698_b200 import synth
+    R = Cc = 2048
+    T, bits, budget = 8192, (2, 3, 4), 3.0
+    W = synth.make_weight(R, Cc, synth.tensor_seed(SEED, 0, 1), dev)
+    X = synth.make_activations(T, Cc, synth.tensor_seed(SEED, 0, 2), dev)
+    f32 = dict(dtype=torch.float32, device=dev)
+    nb = (R // 128) * (Cc // 128)
+    c, rs, cs = torch.empty(Cc, **f32), torch.empty(R, **f32), torch.empty(Cc, **f32)
+    pr = torch.empty(R, dtype=torch.int32, device=dev)
+    pc = torch.empty(Cc, dtype=torch.int32, device=dev)
+    err, wp = torch.empty(nb, len(bits), **f32), torch.empty_like(W)
+    packed = torch.empty(R * Cc * max(bits) // 32, dtype=torch.int32, device=dev)
+    off, meta = torch.empty(nb + 1, dtype=torch.int64, device=dev), torch.empty((R * Cc // 128, 2), **f32)
+    flush = torch.empty(160 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    rep = {}
+
+    def once():
+        ctx.calib_moments(X, c)
+        ctx.reorder_channels(W, c, 3, 128, row_score=rs, col_score=cs, row_segment=R, col_segment=Cc,
+                             row_perm=pr, col_perm=pc)
+        ctx.block_scores(W, c, bits, 128, 128, 128, row_perm=pr, col_perm=pc, err=err, want_gain=False,
+                         W_perm_out=wp)
+        level, r = ctx.allocate_bits(err, bits, budget, uniform_block_elems=128 * 128)
+        ctx.pack_blocks(wp, bits, level, 128, 128, 128, packed=packed, block_off=off, meta=meta)
+        rep.update(r)
+
+    for _ in range(3):
+        once()
+    total = 0.0
+    reps = 20
+    for _ in range(reps):
+        flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        once()
+        b.record()
+        b.synchronize()
+        total += a.elapsed_time(b)
+    ms = total / reps
+    return {"workload": "configs[0]: W 2048 x 2048, X 8192 x 2048, blocks 128 x 128, bits {2,3,4}, group 128, "
+                        "budget 3.0, free row and column sort",
+            "ms_per_pass": ms, "elements_per_s": R * Cc / (ms * 1e-3), "allocation": dict(rep),
+            "timing": "CUDA events around the five library calls (eager launches, one host synchronisation in "
+                      "the allocation), mean of 20 passes, L2 flushed between passes"}
+
+
+def streamed_model_times(ctx, dev):
+    """configs[3]: 80 layers of the 70B shape (68.5 G weights, N = 4,177,920 blocks), bits {2,3,4},
+    budget 2.25.  Weights and activations are made again from their seeds in every sweep (the
+    model is never resident: 136.9 GB of weights); only moments, score vectors, permutations and
+    the table persist.  CUDA-event time of the library calls only."""
+    from paper_2602_17698_b200 import synth
+    from paper_2602_17698_b200.pipeline import SearchConfig, search_model
+    shape, n_layers, tokens, bits, budget = synth.LLAMA3_70B, 80, 16384, (2, 3, 4), 2.25
+    cfg = SearchConfig(bits=bits)
+    t0 = time.time()
+    res = search_model(ctx, shape, n_layers, cfg, (budget,),
+                       lambda layer: synth.make_layer_weights(shape, SEED, layer, dev),
+                       lambda layer: synth.make_layer_activations(shape, tokens, SEED, layer, dev), dev,
+                       keep_tables=False, keep_weights=False, alloc_repeats=2)
+    wall = time.time() - t0
+    ms = res.ms
+    r = res.reports[budget]
+    assert r["used_bits"] <= r["cap_bits"]
+    n_w = n_layers * shape.n_weights
+    return {"workload": f"configs[3]: {n_layers} layers of the 70B shape ({n_w} weights, {res.n_blocks} blocks), "
+                        f"{tokens} tokens per input, bits {list(bits)}, budget {budget}, streamed layer by layer",
+            "ms_library_calls_total": sum(ms.values()),
+            "ms": {"moments": ms["moments"], "reorder_stats": ms["stats@2"], "sort": ms["sort@2"],
+                   "scores": ms["scores@2"], "allocate": ms[f"allocate@{budget:g}"]},
+            "iterations": r["iterations"], "used_bits": r["used_bits"], "cap_bits": r["cap_bits"],
+            "scoring_elements_per_s": n_w / (ms["scores@2"] * 1e-3),
+            "wall_seconds_including_regeneration": wall,
+            "timing": "sum of CUDA-event times around the library calls; inside the timed calls: nothing but the "
+                      "library; outside: the synthetic layers (weights made twice, once per sweep; activations "
+                      "once) and their release"}
+
+
+def full_model_e2e(ctx, dev):
+    """configs[2] end to end for one budget: the weights of every layer come from pinned host memory
+    (13.96 GB, copied once, then resident for the second sweep), the activations of every layer are
+    copied from pinned host buffers as well (3.49 GB per layer; one set of host buffers serves all
+    layers, so the bytes are real and the values repeat), the levels go back to the host.  Wall
+    clock around the whole search after a device synchronisation on both sides."""
+    import torch
+    from paper_2602_17698_b200 import synth
+    from paper_2602_17698_b200.pipeline import SearchConfig, search_model
+    shape = synth.LLAMA3_8B
+    hW = []
+    for layer in range(FULL_MODEL_LAYERS):
+        W = synth.make_layer_weights(shape, SEED, layer, dev)
+        hW.append({n: torch.empty(w.shape, dtype=w.dtype, pin_memory=True).copy_(w) for n, w in W.items()})
+        del W
+    X0 = synth.make_layer_activations(shape, TOKENS, SEED, 0, dev)
+    hX = {n: torch.empty(x.shape, dtype=x.dtype, pin_memory=True).copy_(x) for n, x in X0.items()}
+    del X0
+    torch.cuda.synchronize()
+    h2d = sum(w.numel() * 2 for lw in hW for w in lw.values()) + FULL_MODEL_LAYERS * sum(x.numel() * 2 for x in hX.values())
+    budget = 2.5
+
+    def make_weights(layer):
+        return {n: w.to(dev, non_blocking=True) for n, w in hW[layer].items()}
+
+    def make_acts(layer):
+        return {n: x.to(dev, non_blocking=True) for n, x in hX.items()}
+
+    cfg = SearchConfig(bits=BITS)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    res = search_model(ctx, shape, FULL_MODEL_LAYERS, cfg, (budget,), make_weights, make_acts, dev,
+                       keep_tables=False)
+    level_h = res.levels[budget].cpu()
+    torch.cuda.synchronize()
+    sec = time.perf_counter() - t0
+    n_w = FULL_MODEL_LAYERS * shape.n_weights
+    return {"value": n_w / sec, "unit": UNIT, "seconds": sec, "h2d_bytes": h2d, "d2h_bytes": level_h.numel(),
+            "h2d_gbs": h2d / sec / 1e9,
+            "note": "configs[2], one budget (2.5), weights and activations from pinned host memory, levels back "
+                    "to the host; bound by the host-to-device copies"}
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -540,7 +711,8 @@ def run_cuda(args):
         achieved = mom_bytes / (stage_ms["moments"] * 1e-3) / 1e9
         traffic = NCU_TRAFFIC_RATIO["moments_partial_kernel"] * mom_bytes / mom_launches
         roofline = {"kernel": "moments_partial_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
-                    "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
+                    "unit": "GB/s", "frac": achieved / peak, "frac_nominal": achieved / NOMINAL_HBM_GBS,
+                    "peak_source": peak_kind + " copy bandwidth",
                     "traffic": traffic, "algorithmic_bytes_per_launch": mom_bytes / mom_launches,
                     "launches_per_step": mom_launches, "avg_launch_ms": stage_ms["moments"] / mom_launches}
         w_bytes = 2 * n_weights
@@ -549,31 +721,39 @@ def run_cuda(args):
                      "scores": w_bytes / (stage_ms["scores"] * 1e-3) / 1e9,
                      "pack": w_bytes / (stage_ms["pack"] * 1e-3) / 1e9}
         sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
-        kernels = kernel_rooflines(ctx, W, X, ws.moments, dev, peak, sm_mhz)
+        sm_count = torch.cuda.get_device_properties(local).multi_processor_count
+        kernels = kernel_rooflines(ctx, W, X, ws.moments, dev, peak, sm_mhz, sm_count)
         if world == 1:
             kernels += dequant_gemm_times(ctx, dev, peak)
-        full_model = None
+        full_model = small_layer = streamed = None
         if world == 1 and not args.no_full_model:
             del hW, hX                                   # pinned copies of the layer, if any
+            small_layer = small_layer_times(ctx, dev)
+            del W, X                                     # the layer's tensors: the models need the room
             full_model = full_model_times(ctx, dev)
+            full_model["e2e"] = full_model_e2e(ctx, dev)
+            streamed = streamed_model_times(ctx, dev)
         cpu = None
         if not args.no_cpu_baseline:
             v, sec, cores, sample = time_oracle(3, 0)
             cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
-                   "seconds": sec}
+                   "seconds": sec, "full_size_matrix": oracle_full_matrix()}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": WORKLOAD, "tokens": TOKENS, "bits": list(BITS), "budget": BUDGET,
                            "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                            "l2": "inputs (3.9 GB per step) larger than L2, no flush needed",
+                           "hbm_target": "fractions of the measured copy bandwidth (frac) and of the nominal "
+                                         "8000 GB/s (frac_nominal): the 70 % target is stated on the nominal figure",
                            "launch": "eager" if graphs is None else "one CUDA graph per stage (allocation eager)",
                            "allocation": res.report},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
                 "roofline": roofline, "cpu_baseline": cpu,
                 "stages_ms_per_step": stage_ms, "stages_algorithmic_gbs": stage_gbs,
                 "scoring_elements_per_s": n_weights / (stage_ms["scores"] * 1e-3),
-                "roofline_other_kernels": kernels, "full_model": full_model}
+                "roofline_other_kernels": kernels, "small_layer": small_layer, "full_model": full_model,
+                "streamed_model": streamed}
         print(json.dumps(line), flush=True)
     ctx.close()
     if world > 1:
