@@ -91,6 +91,16 @@ sb_status sb_reorder_channels(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_
                               int64_t row_segment, int64_t col_segment,
                               int32_t* row_perm, int32_t* col_perm);
 
+/* Appendix D (the residual-stream permutation also shuffles what is not quantised: the columns
+ * of the embedding and of the language-model head, the rows of anything that writes the stream):
+ * out[r][j] = W[row_perm[r]][col_perm[j]] for a bf16 matrix that is only moved, not scored.
+ * W [R][ldw] device, row-major, ldw >= C, C a multiple of 8, 16-byte aligned; row_perm [R] /
+ * col_perm [C] device (perm[new] = old) or NULL = identity; out [R][C] device, dense, must not
+ * overlap W.  Asynchronous on the context's stream.  SB_ERR_INVALID: null pointers;
+ * SB_ERR_SHAPE: alignment, or rows longer than 34133 columns.                                  */
+sb_status sb_permute_matrix(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_t C, int64_t ldw,
+                            const int32_t* row_perm, const int32_t* col_perm, void* out_bf16);
+
 /* Helpers for grouped-query attention (Appendix D: value / output projections are
  * reordered inside each head; query heads that read one value head share its order):
  *   fold:   dst[h*seg + d] += sum_{u<reps} src[(h*reps + u)*seg + d],  n_dst = len(dst)

@@ -22,7 +22,7 @@ SB_ACC_ROW, SB_ACC_COL = 1, 2
 
 EXPORTS = ["sb_create", "sb_destroy", "sb_sync", "sb_last_error", "sb_kernel_launches",
            "sb_calib_moments", "sb_reorder_channels", "sb_fold_segment_scores",
-           "sb_expand_segment_perm", "sb_block_scores", "sb_allocate_bits", "sb_pack_blocks",
+           "sb_expand_segment_perm", "sb_permute_matrix", "sb_block_scores", "sb_allocate_bits", "sb_pack_blocks",
            "sb_calib_moments_noalloc", "sb_first_order_scores", "sb_exchange_step",
            "sb_reorder_channels_first_order", "sb_calib_gram",
            "sb_block_scores_full", "sb_dequant_gemm"]
@@ -85,6 +85,7 @@ def lib() -> C.CDLL:
                                           i64, i64, vp, vp]
         L.sb_fold_segment_scores.argtypes = [vp, vp, vp, i64, i32, i64]
         L.sb_expand_segment_perm.argtypes = [vp, vp, vp, i64, i32, i64]
+        L.sb_permute_matrix.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
         L.sb_block_scores.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp, vp, i32, i32, i32,
                                       C.POINTER(C.c_int), i32, vp, vp, vp]
         L.sb_allocate_bits.argtypes = [vp, vp, i64, vp, i64, C.POINTER(C.c_int), i32, f64, i32,
@@ -218,6 +219,16 @@ class Context:
         assert out.numel() == perm.numel() * reps and out.dtype == torch.int32
         self._check(lib().sb_expand_segment_perm(self._h, _ptr(out), _ptr(perm, torch.int32),
                                                  perm.numel(), reps, seg))
+        return out
+
+    def permute_matrix(self, W: torch.Tensor, row_perm=None, col_perm=None, out=None) -> torch.Tensor:
+        """out[r][j] = W[row_perm[r]][col_perm[j]] (a matrix that is moved along with a channel
+        permutation but not scored: embedding, language-model head)."""
+        R, Cc, ldw = _mat(W)
+        if out is None:
+            out = torch.empty((R, Cc), dtype=torch.bfloat16, device=W.device)
+        self._check(lib().sb_permute_matrix(self._h, _ptr(W), R, Cc, ldw, _ptr(row_perm, torch.int32),
+                                            _ptr(col_perm, torch.int32), _ptr(out)))
         return out
 
     def block_scores(self, W: torch.Tensor, col_moment: torch.Tensor, bits: Sequence[int],

@@ -525,6 +525,16 @@ sb_status sb_reorder_channels_first_order(sb_ctx* ctx, const void* W, const void
                         accumulate, row_segment, col_segment, row_perm, col_perm);
 }
 
+sb_status sb_permute_matrix(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw,
+                            const int32_t* row_perm, const int32_t* col_perm, void* out) {
+    if (!ctx) return SB_ERR_INVALID;
+    if (!W || !out || R <= 0 || C <= 0) return sb_fail(ctx, SB_ERR_INVALID, "permute: null or empty");
+    if (C % 8 || ldw % 8 || ldw < C || (reinterpret_cast<uintptr_t>(W) & 15) || (reinterpret_cast<uintptr_t>(out) & 15))
+        return sb_fail(ctx, SB_ERR_SHAPE, "permute: C, ldw must be multiples of 8, both matrices 16-byte aligned");
+    SB_CUDA(ctx, cudaSetDevice(ctx->device));
+    return sb_gather_bf16(ctx, W, R, C, ldw, row_perm, col_perm, out);
+}
+
 sb_status sb_fold_segment_scores(sb_ctx* ctx, float* dst, const float* src, int64_t n_dst, int reps,
                                  int64_t seg) {
     if (!ctx) return SB_ERR_INVALID;
