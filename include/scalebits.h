@@ -58,6 +58,17 @@ sb_status sb_destroy(sb_ctx* ctx);
 sb_status sb_sync(sb_ctx* ctx);
 /* Static / context-owned string describing the last host-side error.                */
 const char* sb_last_error(const sb_ctx* ctx);
+
+/* Test hook for the one device-side wait of the path, the look-back of the chained scans
+ * (prefix sums of Algorithm 1's step costs and of the packed block sizes; the paper has no
+ * counterpart).  wait_ns: how long a tile may wait for a predecessor before it gives up, latches
+ * SB_ERR_TIMEOUT and lets the kernel return (negative: the default, 250 ms).  mute_tile: the tile
+ * of that index publishes nothing, like a predecessor that never arrives (negative: none).  With
+ * a muted tile the results of the call are undefined; the status is returned by sb_sync /
+ * sb_allocate_bits, which also clears it.  Synchronises the stream.  Use only with calls whose
+ * later kernels index by block id (SB_ALLOC_GREEDY with at most 65536 steps): a scan whose
+ * prefix feeds addresses (sb_pack_blocks, the multi-launch sort) must not run with a muted tile. */
+sb_status sb_debug_lookback(sb_ctx* ctx, int64_t wait_ns, int64_t mute_tile);
 /* Number of kernels this context has launched so far (for launch accounting).       */
 int64_t sb_kernel_launches(const sb_ctx* ctx);
 

@@ -20,7 +20,7 @@ SB_OK, SB_ERR_INVALID, SB_ERR_SHAPE, SB_ERR_BUDGET, SB_ERR_SCRATCH, SB_ERR_CUDA,
 SB_ALLOC_SCALEBITS, SB_ALLOC_GREEDY = 0, 1
 SB_ACC_ROW, SB_ACC_COL = 1, 2
 
-EXPORTS = ["sb_create", "sb_destroy", "sb_sync", "sb_last_error", "sb_kernel_launches",
+EXPORTS = ["sb_create", "sb_destroy", "sb_sync", "sb_last_error", "sb_kernel_launches", "sb_debug_lookback",
            "sb_calib_moments", "sb_reorder_channels", "sb_fold_segment_scores",
            "sb_expand_segment_perm", "sb_permute_matrix", "sb_block_scores", "sb_allocate_bits", "sb_pack_blocks",
            "sb_calib_moments_noalloc", "sb_first_order_scores", "sb_exchange_step",
@@ -76,6 +76,7 @@ def lib() -> C.CDLL:
         L.sb_create.argtypes = [C.POINTER(vp), i32, vp]
         L.sb_destroy.argtypes = [vp]
         L.sb_sync.argtypes = [vp]
+        L.sb_debug_lookback.argtypes = [vp, i64, i64]
         L.sb_last_error.argtypes = [vp]
         L.sb_last_error.restype = C.c_char_p
         L.sb_kernel_launches.argtypes = [vp]
@@ -220,6 +221,10 @@ class Context:
         self._check(lib().sb_expand_segment_perm(self._h, _ptr(out), _ptr(perm, torch.int32),
                                                  perm.numel(), reps, seg))
         return out
+
+    def debug_lookback(self, wait_ns: int = -1, mute_tile: int = -1):
+        """Test hook: the time limit of a look-back wait and a tile that publishes nothing."""
+        self._check(lib().sb_debug_lookback(self._h, int(wait_ns), int(mute_tile)))
 
     def permute_matrix(self, W: torch.Tensor, row_perm=None, col_perm=None, out=None) -> torch.Tensor:
         """out[r][j] = W[row_perm[r]][col_perm[j]] (a matrix that is moved along with a channel

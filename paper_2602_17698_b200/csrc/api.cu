@@ -69,14 +69,18 @@ sb_status sb_create(sb_ctx** out, int device, void* cuda_stream) {
         return SB_ERR_CUDA;
     }
     ctx->sm_count = prop.multiProcessorCount;
+    SbDeviceState init{};
+    init.lb_wait_ns = 250ull * 1000 * 1000;
+    init.lb_mute_tile = 0xffffffffu;
     if (cudaMalloc(&ctx->dstate, sizeof(SbDeviceState)) != cudaSuccess ||
-        cudaMemset(ctx->dstate, 0, sizeof(SbDeviceState)) != cudaSuccess ||
+        cudaMemcpy(ctx->dstate, &init, sizeof(SbDeviceState), cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMalloc(&ctx->moment_done, SB_MOMENT_CHUNKS * sizeof(unsigned)) != cudaSuccess ||
         cudaMemset(ctx->moment_done, 0, SB_MOMENT_CHUNKS * sizeof(unsigned)) != cudaSuccess ||
         cudaMalloc(&ctx->stats_done, 2 * SB_STATS_TILES * sizeof(unsigned)) != cudaSuccess ||
         cudaMemset(ctx->stats_done, 0, 2 * SB_STATS_TILES * sizeof(unsigned)) != cudaSuccess ||
         cudaMallocHost(&ctx->pinned, 4096) != cudaSuccess) {
-        delete ctx;
+        (void)cudaGetLastError();
+        sb_destroy(ctx);      // frees whatever was allocated before the failure
         return SB_ERR_CUDA;
     }
     ctx->pinned_bytes = 4096;
@@ -111,6 +115,17 @@ sb_status sb_sync(sb_ctx* ctx) {
         SB_CUDA(ctx, cudaMemsetAsync(ctx->dstate, 0, 2 * sizeof(int), ctx->stream));
         return sb_fail(ctx, st, "device-side status %d latched by kernel family %d", (int)st, where);
     }
+    return SB_OK;
+}
+
+sb_status sb_debug_lookback(sb_ctx* ctx, int64_t wait_ns, int64_t mute_tile) {
+    if (!ctx) return SB_ERR_INVALID;
+    SB_CUDA(ctx, cudaSetDevice(ctx->device));
+    const unsigned long long w = wait_ns < 0 ? 250ull * 1000 * 1000 : (unsigned long long)wait_ns;
+    const unsigned m = mute_tile < 0 ? 0xffffffffu : (unsigned)mute_tile;
+    SB_CUDA(ctx, cudaMemcpyAsync(&ctx->dstate->lb_wait_ns, &w, sizeof w, cudaMemcpyHostToDevice, ctx->stream));
+    SB_CUDA(ctx, cudaMemcpyAsync(&ctx->dstate->lb_mute_tile, &m, sizeof m, cudaMemcpyHostToDevice, ctx->stream));
+    SB_CUDA(ctx, cudaStreamSynchronize(ctx->stream));     // the two host words are on this stack
     return SB_OK;
 }
 

@@ -15,6 +15,9 @@ struct SbDeviceState {           // lives in device memory, one per context
     int where;                   // kernel id that latched it
     unsigned int ticket;         // dynamic tile ids of the look-back scans
     unsigned int pad;            // CTAs of the current look-back launch that have finished
+    unsigned long long lb_wait_ns;   // how long a look-back wait may last (default 250 ms)
+    unsigned int lb_mute_tile;       // test hook: this tile of a look-back launch publishes nothing
+    unsigned int pad2;               //   (0xffffffff: none)
 };
 
 struct sb_ctx {

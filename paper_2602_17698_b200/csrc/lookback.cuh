@@ -22,7 +22,7 @@ LookbackBuf sb_lookback(sb_ctx* ctx, unsigned tiles, sb_status* st);
 
 #ifdef __CUDACC__
 constexpr unsigned LB_AGG = 1u, LB_INC = 2u;
-constexpr unsigned long long LB_WAIT_NS = 250ull * 1000 * 1000;   // give up after 250 ms
+constexpr unsigned long long LB_WAIT_NS = 250ull * 1000 * 1000;   // default: give up after 250 ms
 __device__ __forceinline__ unsigned long long lb_now_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -117,19 +117,23 @@ __device__ __forceinline__ T lookback_prefix(T aggregate, unsigned tile, Lookbac
     T* incs = reinterpret_cast<T*>(lb.inc);
     if (threadIdx.x < 32) {
         const int lane = threadIdx.x;
+        // test hook (sb_debug_lookback): a muted tile behaves like a predecessor that never
+        // publishes, so that its successors' bounded waits can be seen to run out
+        const bool muted = tile == st->lb_mute_tile;
         if (tile == 0) {
             if (lane == 0) {
                 incs[0] = aggregate;
                 __threadfence();
-                st_release_u32(lb.flags, LB_INC);
+                if (!muted) st_release_u32(lb.flags, LB_INC);
                 prefix_sh = t_zero((T*)nullptr);
             }
         } else {
             if (lane == 0) {
                 aggs[tile] = aggregate;
                 __threadfence();
-                st_release_u32(lb.flags + tile, LB_AGG);
+                if (!muted) st_release_u32(lb.flags + tile, LB_AGG);
             }
+            const unsigned long long wait_ns = st->lb_wait_ns;
             T running = t_zero((T*)nullptr);
             int base = (int)tile - 1;
             bool timed_out = false;
@@ -146,7 +150,7 @@ __device__ __forceinline__ T lookback_prefix(T aggregate, unsigned tile, Lookbac
                         if ((++spins & 63) == 0) {
                             const unsigned long long now = lb_now_ns();
                             if (t_start == 0) t_start = now;
-                            else if (now - t_start > LB_WAIT_NS) { timed_out = true; break; }
+                            else if (now - t_start > wait_ns) { timed_out = true; break; }
                         }
                         __nanosleep(64);
                         f = ld_acquire_u32(lb.flags + t);
@@ -167,7 +171,7 @@ __device__ __forceinline__ T lookback_prefix(T aggregate, unsigned tile, Lookbac
             if (lane == 0) {
                 incs[tile] = t_add(running, aggregate);
                 __threadfence();
-                st_release_u32(lb.flags + tile, LB_INC);
+                if (!muted) st_release_u32(lb.flags + tile, LB_INC);
                 prefix_sh = running;
             }
         }

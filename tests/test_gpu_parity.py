@@ -333,6 +333,25 @@ def test_allocate_scalebits_walks_the_handworked_trajectories(ctx):
         assert rep["proxy_loss_init"] == fin["loss_init"] and rep["proxy_loss_final"] == fin["loss_final"]
 
 
+def test_lookback_wait_runs_out_and_the_context_stays_usable(ctx):
+    """The one device-side wait of the path (a scan tile waiting for its predecessor) is bounded:
+    with the test hook tile 0 of the cost prefix sum publishes nothing, tile 1 waits 1 ms, gives
+    up, latches SB_ERR_TIMEOUT and the kernel returns.  Nothing hangs or traps; the context works
+    afterwards."""
+    from paper_2602_17698_b200.binding import SB_ALLOC_GREEDY, SB_ERR_TIMEOUT, SbError
+    N, bits = 20000, [2, 3, 4, 8]                       # <= 60000 steps: one-launch sort, a scan of many tiles
+    table = _tables(N, len(bits), 5, "convex")
+    err = torch.from_numpy(table).to(DEV)
+    ctx.debug_lookback(wait_ns=1_000_000, mute_tile=0)
+    try:
+        with pytest.raises(SbError) as ei:
+            ctx.allocate_bits(err, bits, 2.5, SB_ALLOC_GREEDY)
+        assert ei.value.status == SB_ERR_TIMEOUT
+    finally:
+        ctx.debug_lookback()                            # defaults: 250 ms, no muted tile
+    _check_alloc(ctx, table, bits, 2.5, SB_ALLOC_GREEDY)    # exact again, the status was cleared
+
+
 def test_allocate_nonuniform_block_sizes(ctx):
     from paper_2602_17698_b200.binding import SB_ALLOC_GREEDY, SB_ALLOC_SCALEBITS
     rng = np.random.default_rng(4)
