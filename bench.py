@@ -822,6 +822,34 @@ def run_only(which: str):
             level = torch.randint(0, len(BITS), (nb,), device=dev, dtype=torch.uint8)
             for _ in range(3):
                 ctx.pack_blocks(W, BITS, level, 128, 128, 128)
+        elif which == "scores3":
+            err = torch.empty(nb, 3, device=dev)
+            for _ in range(3):
+                ctx.block_scores(W, c, (2, 3, 4), 128, 128, 128, err=err, want_gain=False)
+        elif which == "scores7":
+            err = torch.empty(nb, 7, device=dev)
+            for _ in range(3):
+                ctx.block_scores(W, c, STRESS_BITS, 128, 128, 128, err=err, want_gain=False)
+        elif which == "first_order":
+            G = (W.float() * 1e-2).to(torch.bfloat16)
+            level = torch.randint(0, len(BITS), (nb,), device=dev, dtype=torch.uint8)
+            for _ in range(3):
+                ctx.first_order_scores(W, G, BITS, level, 128, 128, 128, want_l1=False)
+        elif which == "sort":
+            score = torch.rand(R, device=dev)
+            perm = torch.empty(R, dtype=torch.int32, device=dev)
+            for _ in range(3):
+                ctx.reorder_channels(None, None, 2, 128, row_score=score, row_segment=R, row_perm=perm,
+                                     shape=(R, 128))
+        elif which in ("allocate", "allocate_model"):
+            # the layer's table (13,312 blocks: one cluster sort, the masked loop kernel) or the
+            # model's (425,984 blocks: multi-launch sort, cooperative loop kernel)
+            N = 13312 if which == "allocate" else 425984
+            table = (torch.rand(N, 1, device=dev) * 30 + 1) * (0.4 ** torch.arange(len(BITS), device=dev))[None, :] \
+                * (torch.rand(N, len(BITS), device=dev) * 1.3 + 0.5)
+            table = table.float().contiguous()
+            for _ in range(3):
+                ctx.allocate_bits(table, BITS, BUDGET)
         else:
             raise SystemExit(f"unknown stage {which}")
     ctx.sync()
@@ -843,7 +871,8 @@ def main():
     ap.add_argument("--no-graphs", action="store_true", help="launch every library call eagerly")
     ap.add_argument("--only", default=None,
                     help="three calls of one library call on one input, then exit (for ncu captures): "
-                         "moments | gram | full_scores | dequant_gemm | reorder_stats | scores | gather | pack")
+                         "moments | gram | full_scores | dequant_gemm | reorder_stats | scores | scores3 | scores7 | "
+                         "gather | pack | first_order | sort | allocate | allocate_model")
     args = ap.parse_args()
     if args.only:
         run_only(args.only)
