@@ -73,6 +73,7 @@ struct ScoreGeom {
     int nsub, lanes_per_sub;       // blocks side by side in a chunk (bc < 128); lanes across one block
     int gpc, rec_bytes;            // groups per 128-column chunk; bytes of one slab's records
     int ring;                      // slab slots per stream
+    int n_rows, n_cols;            // rows / columns of the matrix (the last slab / chunk may reach past them)
     unsigned n_tile_cols, n_slabs, n_warps;   // n_warps = warps of the grid
 };
 
@@ -80,7 +81,8 @@ struct ScoreArgs {
     const int32_t* c_perm;           // original column of permuted j
     const float* col_moment;
     BitsArg ba;
-    float* rec;
+    float* rec;                      // scores: partial block errors; statistics: partial column sums
+    float* rowpart;                  // statistics: [strip][row] partial row sums
 };
 
 // owner of slab s when stream w takes slabs [n_slabs * w / n_warps, n_slabs * (w + 1) / n_warps)
@@ -319,7 +321,7 @@ __device__ __forceinline__ void slab_records(unsigned slab, unsigned rec, int ro
                     float ar = 1.f;
                     if (ROWW) {
                         const int row = row0 + rr;
-                        ar = row_weight[a_perm ? a_perm[row] : row];
+                        ar = row < g.n_rows ? row_weight[a_perm ? a_perm[row] : row] : 0.f;
                     }
                     sts128(rec + (rr * g.gpc + grp) * 16, r.nlo, r.rinv, r.rng, ar);
                 }
@@ -342,7 +344,7 @@ __device__ __forceinline__ void slab_records_ragged(unsigned slab, unsigned rec,
         float ar = 1.f;
         if (ROWW) {
             const int row = row0 + rr;
-            ar = row_weight[a_perm ? a_perm[row] : row];
+            ar = row < g.n_rows ? row_weight[a_perm ? a_perm[row] : row] : 0.f;
         }
         if (use_pre(L, FULLG)) {
             if (cl == 0) pre_record<L, NFINE>(rec + rr * pre_stride(L, NFINE), r, ba, true, 0, L);
@@ -358,8 +360,13 @@ __device__ __forceinline__ void slab_records_ragged(unsigned slab, unsigned rec,
 }
 
 // ---- all candidates from registers, per-column accumulators ---------------------------------
-template <int L, int RPL, int NFINE, bool FULLG, bool ROWW>
+template <int L_, int RPL_, int NFINE_, bool FULLG_, bool ROWW_>
 struct Scorer {
+    static constexpr int L = L_, RPL = RPL_, NFINE = NFINE_;
+    static constexpr bool FULLG = FULLG_, ROWW = ROWW_;
+    static constexpr bool FULL_SLABS = false;      // a block's height need not be a multiple of 16
+    __device__ __forceinline__ void begin_column(int) {}
+    __device__ __forceinline__ void slab_done(int, unsigned) {}
     const ScoreArgs& a;
     const ScoreGeom& g;
     const unsigned gs;             // warp number in the grid
@@ -472,11 +479,130 @@ struct Scorer {
     }
 };
 
-template <int L, int RPL, int NFINE, bool FULLG, bool ROWW>
+// ---- reorder statistics on the same walk (Section 4.1: per-channel aggregates of the element
+// sensitivities a_r c_j (W - Q(W))^2 at the warm-start precision, on the ORIGINAL layout) ----------
+// One candidate.  The matrix is one block row as tall as the matrix, so a chunk column is a strip of
+// 128 columns from top to bottom.  Column sums: per-column accumulators over the warp's stretch of a
+// strip, written as a record of 128 partial sums at its end (c_j applied there).  Row sums: a lane's
+// 8 rows of a slab each get sum_j c_j e^2 over the lane's 8 columns; the 16 lanes of a row are reduced
+// for all 8 rows at once by the same transposed butterfly as the ranges, and the lane that ends up with
+// a row writes rowpart[strip][row].  A second kernel adds the partials in a fixed order: no float
+// atomics, reruns are bit-identical.
+template <int NFINE_, bool FULLG_, bool ROWW_>
+struct StatsScorer {
+    static constexpr int L = 1, RPL = 2, NFINE = NFINE_;
+    static constexpr bool FULLG = FULLG_, ROWW = ROWW_;
+    static constexpr bool PRE = use_pre(1, FULLG);
+    static constexpr bool FULL_SLABS = true;       // the strip is padded to whole slabs (zero rows add nothing)
+    const ScoreArgs& a;
+    const ScoreGeom& g;
+    const unsigned gs;
+    const int cl, slot2;
+    f32x2 colacc[SC_NW], c2[SC_NW];
+    float rowsum[8];
+    __device__ __forceinline__ StatsScorer(const ScoreArgs& a_, const ScoreGeom& g_, unsigned gs_, int cl_, int slot_)
+        : a(a_), g(g_), gs(gs_), cl(cl_), slot2(slot_) {
+#pragma unroll
+        for (int k = 0; k < SC_NW; ++k) colacc[k] = c2[k] = 0ull;
+    }
+    // column factors of the lane's 8 columns of the strip that starts at column col0
+    __device__ __forceinline__ void begin_column(int col0) {
+        const int col = col0 + cl * SC_CPL;
+#pragma unroll
+        for (int k = 0; k < SC_NW; ++k) {
+            const int j = col + 2 * k;
+            c2[k] = pk2(j < g.n_cols ? __ldg(a.col_moment + j) : 0.f, j + 1 < g.n_cols ? __ldg(a.col_moment + j + 1) : 0.f);
+        }
+    }
+    __device__ __forceinline__ void step(unsigned lane_slab, unsigned lane_rec, int rec_pitch, int r0) {
+        const f32x2 magic2 = pk2(RNE_MAGIC, RNE_MAGIC), nmagic2 = pk2(-RNE_MAGIC, -RNE_MAGIC);
+        uint4 x[RPL];
+#pragma unroll
+        for (int i = 0; i < RPL; ++i) x[i] = lds128(lane_slab + (r0 + 2 * i) * 256);
+#pragma unroll
+        for (int i = 0; i < RPL; ++i) {
+            f32x2 nlo2, inv2, ns2, nslo2 = 0ull, ar2 = 0ull;
+            if (PRE) {
+                const unsigned rec = lane_rec + (r0 + 2 * i) * pre_stride(1, NFINE);
+                nlo2 = lds64(rec);
+                lds128_pairs(rec + 16, inv2, ns2);
+                if (NFINE) nslo2 = lds64(rec + 32);
+            } else {
+                const float4 r = lds128f(lane_rec + (r0 + 2 * i) * rec_pitch);
+                const f32x2 q2 = *reinterpret_cast<const f32x2*>(&a.ba.q2[0]);
+                const f32x2 niq2 = *reinterpret_cast<const f32x2*>(&a.ba.niq2[0]);
+                const f32x2 range2 = pk2(r.z, r.z);
+                nlo2 = pk2(r.x, r.x);
+                inv2 = mul2(q2, pk2(r.y, r.y));
+                ns2 = mul2(niq2, range2);
+                if (NFINE) nslo2 = mul2(fma2(ns2, q2, range2), niq2);
+                ar2 = pk2(r.w, r.w);
+            }
+            const uint32_t w[SC_NW] = {x[i].x, x[i].y, x[i].z, x[i].w};
+            f32x2 rs2 = 0ull;
+#pragma unroll
+            for (int k = 0; k < SC_NW; ++k) {
+                const float v0 = __uint_as_float(__byte_perm(w[k], 0u, 0x1044));
+                const f32x2 vm = add2(pk2(v0, bf16hi(w[k])), nlo2);
+                const f32x2 qq = add2(fma2(vm, inv2, magic2), nmagic2);
+                const f32x2 e = NFINE ? fma2(qq, nslo2, fma2(qq, ns2, vm)) : fma2(qq, ns2, vm);
+                const f32x2 ea = ROWW ? mul2(e, ar2) : e;
+                colacc[k] = fma2(ea, e, colacc[k]);
+                rs2 = fma2(mul2(ea, c2[k]), e, rs2);
+            }
+            float s0, s1;
+            upk2(rs2, s0, s1);
+            rowsum[(r0 >> 1) + i] = s0 + s1;             // r0 is a compile-time constant in the unrolled slab
+        }
+    }
+    // the 8 rows of the lane: sums over the 16 lanes of the row, transposed; lane t of its half warp
+    // ends up with row slot2 + 2 (t >> 1)
+    __device__ __forceinline__ void slab_done(int row0, unsigned strip) {
+        const int t = cl;
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+            const int o = 8 >> k, h = 4 >> k;
+            const bool up = (t & o) != 0;
+            float got[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (i < h) got[i] = __shfl_xor_sync(0xffffffffu, up ? rowsum[i] : rowsum[i + h], o);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (i < h) rowsum[i] = (up ? rowsum[i + h] : rowsum[i]) + got[i];
+        }
+        const float tot = rowsum[0] + __shfl_xor_sync(0xffffffffu, rowsum[0], 1);
+        const int row = row0 + slot2 + 2 * (t >> 1);
+        if (a.rowpart && (t & 1) == 0 && row < g.n_rows) a.rowpart[(size_t)strip * g.br + row] = tot;
+    }
+    // the stretch's column sums: c_j, the two half warps (different rows, the same columns), one
+    // record of 128 floats
+    __device__ __forceinline__ void flush(unsigned q, int) {
+        float out[SC_CPL];
+#pragma unroll
+        for (int k = 0; k < SC_NW; ++k) {
+            const f32x2 t2 = mul2(colacc[k], c2[k]);
+            colacc[k] = 0ull;
+            float a0, a1;
+            upk2(t2, a0, a1);
+            out[2 * k] = a0 + __shfl_xor_sync(0xffffffffu, a0, 16);
+            out[2 * k + 1] = a1 + __shfl_xor_sync(0xffffffffu, a1, 16);
+        }
+        if (slot2 == 0 && a.rec) {
+            float4* dst = reinterpret_cast<float4*>(a.rec + (size_t)(q + gs) * TILE_COLS + cl * SC_CPL);
+            dst[0] = make_float4(out[0], out[1], out[2], out[3]);
+            dst[1] = make_float4(out[4], out[5], out[6], out[7]);
+        }
+    }
+};
+
+template <class P>
 __global__ void __launch_bounds__(SC_THREADS, 1)
 block_scores_kernel(const __grid_constant__ CUtensorMap wmap,     // the (permuted) weight matrix
                     const int32_t* __restrict__ a_perm,          // original row of permuted r
                     const float* __restrict__ row_weight, ScoreGeom g, ScoreArgs a, SbDeviceState* dstate) {
+    constexpr int L = P::L, RPL = P::RPL, NFINE = P::NFINE;
+    constexpr bool FULLG = P::FULLG, ROWW = P::ROWW;
     constexpr int STEP_ROWS = 2 * RPL;
     extern __shared__ unsigned char sc_smem_raw[];
     // TMA destinations want 128-byte alignment
@@ -498,7 +624,7 @@ block_scores_kernel(const __grid_constant__ CUtensorMap wmap,     // the (permut
     const unsigned smem_base = smem_u32(sc_smem) + SC_BAR_BYTES + (unsigned)stream * g.ring * slot_bytes;
     const int cl = lane & 15, slot2 = lane >> 4;
     const int team = g.group / SC_CPL;
-    Scorer<L, RPL, NFINE, FULLG, ROWW> sc(a, g, gs, cl, slot2);
+    P sc(a, g, gs, cl, slot2);
     const int rec_pitch = g.gpc * 16;                // bytes between the records of consecutive rows (general form)
     const unsigned lane_slab_off = (unsigned)(slot2 * 256 + cl * 16);
     const unsigned lane_rec_off =
@@ -527,18 +653,19 @@ block_scores_kernel(const __grid_constant__ CUtensorMap wmap,     // the (permut
     unsigned slot = 0, ph = 0;
     bool ok = true;
     unsigned k = 0;
+    sc.begin_column((int)(rc.bx * (unsigned)g.tile_w) + rc.ch * TILE_COLS);
     for (; k < n; ++k) {
         ok = __all_sync(0xffffffffu, mbar_wait(bar_addr(bars, stream, (int)slot), ph, abort_flag));
         if (!ok) break;
         const unsigned slab = smem_base + slot * slot_bytes;
         const int rows_here = min(SLAB_ROWS, g.br - rc.sl * SLAB_ROWS);
         const int row0 = (int)(rc.by * (unsigned)g.br) + rc.sl * SLAB_ROWS;
-        if (rows_here == SLAB_ROWS) {
+        if (P::FULL_SLABS || rows_here == SLAB_ROWS) {
             slab_records<L, NFINE, FULLG, ROWW>(slab, slab + SLAB_BYTES, row0, g, a.ba, team, cl, slot2, a_perm, row_weight);
             __syncwarp();                            // the records are written
 #pragma unroll
             for (int r0 = 0; r0 < SLAB_ROWS; r0 += STEP_ROWS) sc.step(slab + lane_slab_off, slab + lane_rec_off, rec_pitch, r0);
-        } else {
+        } else if constexpr (!P::FULL_SLABS) {
             slab_records_ragged<L, NFINE, FULLG, ROWW>(slab, slab + SLAB_BYTES, rows_here, row0, g, a.ba, team, cl, slot2,
                                                        a_perm, row_weight);
             __syncwarp();
@@ -546,11 +673,13 @@ block_scores_kernel(const __grid_constant__ CUtensorMap wmap,     // the (permut
         }
         __syncwarp();                                // every lane is done with the slot:
         if (issued < n) stage_next();                // refill it (i_slot == slot)
+        sc.slab_done(row0, r_q);
         const bool last_of_column = rc.sl == g.spb - 1;
         if (last_of_column || k + 1 == n)
             sc.flush(r_q, (int)(rc.bx * (unsigned)g.tile_w) + rc.ch * TILE_COLS);
         if (last_of_column) ++r_q;
         advance(rc, g);
+        if (last_of_column && k + 1 < n) sc.begin_column((int)(rc.bx * (unsigned)g.tile_w) + rc.ch * TILE_COLS);
         if (++slot == (unsigned)g.ring) { slot = 0; ph ^= 1u; }
     }
     if (!ok) {
@@ -605,9 +734,9 @@ sb_status launch_scores_k(sb_ctx* ctx, const CUtensorMap& wmap,
                           const ScoreGeom& g, const BitsArg& ba, int64_t n_blocks, int64_t nbc, int grid,
                           float* err, float* gain, float* rec) {
     const size_t smem = 128 + SC_BAR_BYTES + (size_t)SC_STREAMS * g.ring * (SLAB_BYTES + g.rec_bytes);
-    auto kern = block_scores_kernel<L, RPL, NFINE, FULLG, ROWW>;
+    auto kern = block_scores_kernel<Scorer<L, RPL, NFINE, FULLG, ROWW>>;
     SB_FUNC_ATTR(ctx, kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM_MAX);   // one instance serves several group sizes
-    ScoreArgs pa{cperm, cm, ba, rec};
+    ScoreArgs pa{cperm, cm, ba, rec, nullptr};
     kern<<<(unsigned)grid, SC_THREADS, smem, ctx->stream>>>(wmap, aperm, rw, g, pa, ctx->dstate);
     SB_LAUNCHED(ctx);
     scores_finish_kernel<<<(unsigned)((n_blocks + 255) / 256), 256, 0, ctx->stream>>>(
@@ -641,7 +770,137 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                   CUtensorMapFloatOOBfill);
 
+// a bf16 matrix as a 2-D tensor (columns innermost) in tiles of 128 columns x 16 rows; rows and
+// columns past the end read as zero
+sb_status weight_tile_map(sb_ctx* ctx, const __nv_bfloat16* W, int64_t R, int64_t C, int64_t ld, CUtensorMap* map) {
+    static EncodeTiledFn encode = nullptr;
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        SB_CUDA(ctx, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+        if (!fn || qres != cudaDriverEntryPointSuccess)
+            return sb_fail(ctx, SB_ERR_CUDA, "the driver does not export cuTensorMapEncodeTiled");
+        encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)C, (cuuint64_t)R};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)TILE_COLS, (cuuint32_t)SLAB_ROWS};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(W), dims, strides,
+                              box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return sb_fail(ctx, SB_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+    return SB_OK;
+}
+
+// row_score[r] (+)= sum over strips of rowpart[strip][r]; col_score[j] (+)= sum of the records of
+// strip j / 128 in slab order; accumulate: bit 0 rows, bit 1 columns.  A CTA is 32 outputs x 8
+// slices of the partial list: every thread's few loads are independent (one round trip to L2), the
+// slices are added in slice order (a fixed order: reruns are bit-identical).
+constexpr int SF_SLICES = 8;
+__global__ void __launch_bounds__(32 * SF_SLICES)
+stats_finish_kernel(const float* __restrict__ rec, const float* __restrict__ rowpart, ScoreGeom g,
+                    float* __restrict__ row_score, float* __restrict__ col_score, int accumulate,
+                    SbDeviceState* dstate) {
+    __shared__ float part[SF_SLICES][32];
+    const int x = threadIdx.x & 31, y = threadIdx.x >> 5;
+    // outputs: the rows padded to a multiple of 32, then the columns
+    const int64_t rows32 = ((int64_t)g.n_rows + 31) / 32 * 32;
+    const int64_t i = (int64_t)blockIdx.x * 32 + x;
+    const bool is_row = i < rows32;
+    const int64_t idx = is_row ? i : i - rows32;
+    const bool live = is_row ? (idx < g.n_rows && row_score != nullptr) : (idx < g.n_cols && col_score != nullptr);
+    float v = 0.f;
+    if (live) {
+        if (is_row) {
+            const float* src = rowpart + idx;
+            for (unsigned s = (unsigned)y; s < g.n_tile_cols; s += SF_SLICES) v += __ldg(src + (size_t)s * g.br);
+        } else {
+            const int j = (int)idx;
+            const unsigned q = (unsigned)j / TILE_COLS;
+            const unsigned s0 = q * (unsigned)g.spb, s1 = s0 + (unsigned)g.spb - 1u;
+            const unsigned w0 = slab_owner(s0, g.n_slabs, g.n_warps), w1 = slab_owner(s1, g.n_slabs, g.n_warps);
+            const float* src = rec + (size_t)q * TILE_COLS + (j - (int)q * TILE_COLS);
+            const bool gaps = g.n_warps > g.n_slabs;      // warps without slabs write no record
+            for (unsigned w = w0 + (unsigned)y; w <= w1; w += SF_SLICES)
+                if (!gaps || !slab_range_empty(w, g.n_slabs, g.n_warps)) v += __ldg(src + (size_t)w * TILE_COLS);
+        }
+    }
+    part[y][x] = v;
+    __syncthreads();
+    if (y == 0 && live) {
+        float t = 0.f;
+#pragma unroll
+        for (int k = 0; k < SF_SLICES; ++k) t += part[k][x];
+        if (is_row) row_score[idx] = (accumulate & 1) ? row_score[idx] + t : t;
+        else col_score[idx] = (accumulate & 2) ? col_score[idx] + t : t;
+        if (!isfinite(t)) sb_latch(dstate, SB_ERR_NONFINITE, SBK_STATS);
+    }
+}
+
+template <int NFINE, bool FULLG, bool ROWW>
+sb_status launch_stats(sb_ctx* ctx, const CUtensorMap& wmap, const float* rw, const ScoreGeom& g, const ScoreArgs& pa,
+                       int grid) {
+    const size_t smem = 128 + SC_BAR_BYTES + (size_t)SC_STREAMS * g.ring * (SLAB_BYTES + g.rec_bytes);
+    auto kern = block_scores_kernel<StatsScorer<NFINE, FULLG, ROWW>>;
+    SB_FUNC_ATTR(ctx, kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM_MAX);
+    kern<<<(unsigned)grid, SC_THREADS, smem, ctx->stream>>>(wmap, nullptr, rw, g, pa, ctx->dstate);
+    SB_LAUNCHED(ctx);
+    return SB_OK;
+}
+
 }  // namespace
+
+// Reorder statistics of one matrix on the slab walk (second-moment form).  Scratch (floats, from the
+// caller's arena): col_rec [sb_stats_col_rec_floats], rowpart [sb_stats_rowpart_floats].
+size_t sb_stats_col_rec_floats(int64_t C, int sm_count) {
+    return (size_t)((C + TILE_COLS - 1) / TILE_COLS + (int64_t)sm_count * SC_STREAMS) * TILE_COLS;
+}
+size_t sb_stats_rowpart_floats(int64_t R, int64_t C) {
+    return (size_t)((C + TILE_COLS - 1) / TILE_COLS) * (size_t)((R + SLAB_ROWS - 1) / SLAB_ROWS * SLAB_ROWS);
+}
+sb_status sb_reorder_stats_slab(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw,
+                                const float* col_moment, const float* row_weight, int ref_bits, int group,
+                                float* row_score, float* col_score, int accumulate, float* col_rec, float* rowpart) {
+    if (R >= (1ll << 30) || C >= (1ll << 30)) return sb_fail(ctx, SB_ERR_SHAPE, "reorder: matrix too large");
+    ScoreGeom geo{};
+    geo.br = (int)((R + SLAB_ROWS - 1) / SLAB_ROWS * SLAB_ROWS);     // one block row: strips of whole slabs
+    geo.bc = TILE_COLS; geo.group = group;
+    geo.tile_w = TILE_COLS; geo.chunks = 1;
+    geo.spb = geo.br / SLAB_ROWS;
+    geo.nsub = 1; geo.lanes_per_sub = TILE_COLS / SC_CPL;
+    geo.gpc = TILE_COLS / group;
+    const bool fullg = group == 128 && !row_weight;
+    const int nfine = ref_bits >= 6 ? 1 : 0;
+    geo.rec_bytes = use_pre(1, fullg) ? SLAB_ROWS * pre_stride(1, nfine) : SLAB_ROWS * geo.gpc * 16;
+    geo.ring = (SC_SMEM_MAX - SC_BAR_BYTES - 128) / (SC_STREAMS * (SLAB_BYTES + geo.rec_bytes));
+    if (geo.ring > MAX_RING) geo.ring = MAX_RING;
+    geo.n_rows = (int)R; geo.n_cols = (int)C;
+    geo.n_tile_cols = (unsigned)((C + TILE_COLS - 1) / TILE_COLS);
+    const int64_t n_slabs = (int64_t)geo.n_tile_cols * geo.spb;
+    if (n_slabs >= (1ll << 31)) return sb_fail(ctx, SB_ERR_SHAPE, "reorder: matrix too large");
+    geo.n_slabs = (unsigned)n_slabs;
+    int64_t grid = (n_slabs + SC_STREAMS - 1) / SC_STREAMS;
+    if (grid > ctx->sm_count) grid = ctx->sm_count;
+    geo.n_warps = (unsigned)(grid * SC_STREAMS);
+    CUtensorMap wmap;
+    sb_status st = weight_tile_map(ctx, static_cast<const __nv_bfloat16*>(W), R, C, ldw, &wmap);
+    if (st != SB_OK) return st;
+    const int one_bit[1] = {ref_bits};
+    ScoreArgs pa{nullptr, col_moment, make_bits(one_bit, 1), col_score ? col_rec : nullptr, row_score ? rowpart : nullptr};
+    if (row_weight) st = nfine ? launch_stats<1, false, true>(ctx, wmap, row_weight, geo, pa, (int)grid)
+                               : launch_stats<0, false, true>(ctx, wmap, row_weight, geo, pa, (int)grid);
+    else if (fullg) st = nfine ? launch_stats<1, true, false>(ctx, wmap, nullptr, geo, pa, (int)grid)
+                               : launch_stats<0, true, false>(ctx, wmap, nullptr, geo, pa, (int)grid);
+    else st = nfine ? launch_stats<1, false, false>(ctx, wmap, nullptr, geo, pa, (int)grid)
+                    : launch_stats<0, false, false>(ctx, wmap, nullptr, geo, pa, (int)grid);
+    if (st != SB_OK) return st;
+    const int64_t n = (R + 31) / 32 * 32 + C;
+    stats_finish_kernel<<<(unsigned)((n + 31) / 32), 32 * SF_SLICES, 0, ctx->stream>>>(col_rec, rowpart, geo, row_score,
+                                                                                       col_score, accumulate, ctx->dstate);
+    SB_LAUNCHED(ctx);
+    return SB_OK;
+}
 
 extern "C" sb_status sb_block_scores(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw,
                                      const int32_t* row_perm, const int32_t* col_perm, const float* col_moment,
@@ -678,6 +937,7 @@ extern "C" sb_status sb_block_scores(sb_ctx* ctx, const void* W, int64_t R, int6
                                            : SLAB_ROWS * geo.gpc * 16;
     geo.ring = (SC_SMEM_MAX - SC_BAR_BYTES - 128) / (SC_STREAMS * (SLAB_BYTES + geo.rec_bytes));
     if (geo.ring > MAX_RING) geo.ring = MAX_RING;
+    geo.n_rows = (int)R; geo.n_cols = (int)C;
     geo.n_tile_cols = (unsigned)(C / geo.tile_w);
     const int64_t n_chunk_cols = (R / br) * (int64_t)geo.n_tile_cols * geo.chunks;
     const int64_t n_slabs = n_chunk_cols * geo.spb;
@@ -702,26 +962,10 @@ extern "C" sb_status sb_block_scores(sb_ctx* ctx, const void* W, int64_t R, int6
         src = static_cast<const __nv_bfloat16*>(dst);
         ld = C;
     }
-    // the matrix as a 2-D tensor (columns innermost) in tiles of 128 columns x 16 rows
-    static EncodeTiledFn encode = nullptr;
-    if (!encode) {
-        void* fn = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        SB_CUDA(ctx, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
-        if (!fn || qres != cudaDriverEntryPointSuccess)
-            return sb_fail(ctx, SB_ERR_CUDA, "scores: the driver does not export cuTensorMapEncodeTiled");
-        encode = reinterpret_cast<EncodeTiledFn>(fn);
-    }
     CUtensorMap wmap;
     {
-        const cuuint64_t dims[2] = {(cuuint64_t)C, (cuuint64_t)R};
-        const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-        const cuuint32_t box[2] = {(cuuint32_t)TILE_COLS, (cuuint32_t)SLAB_ROWS};
-        const cuuint32_t estr[2] = {1, 1};
-        const CUresult r = encode(&wmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(src), dims,
-                                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return sb_fail(ctx, SB_ERR_CUDA, "scores: cuTensorMapEncodeTiled failed (%d)", (int)r);
+        sb_status mst = weight_tile_map(ctx, src, R, C, ld, &wmap);
+        if (mst != SB_OK) return mst;
     }
     const BitsArg ba = make_bits(bits, n_bits);
     sb_status st = SB_OK;

@@ -422,6 +422,13 @@ sb_status sb_gather_bf16(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64
     return SB_OK;
 }
 
+// the second-moment form runs on the slab walk of the score kernel (scores.cu)
+size_t sb_stats_col_rec_floats(int64_t C, int sm_count);
+size_t sb_stats_rowpart_floats(int64_t R, int64_t C);
+sb_status sb_reorder_stats_slab(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw,
+                                const float* col_moment, const float* row_weight, int ref_bits, int group,
+                                float* row_score, float* col_score, int accumulate, float* col_rec, float* rowpart);
+
 // both forms of the reorder statistics (G == NULL: second-moment form) and the sorts
 static sb_status reorder_impl(sb_ctx* ctx, const void* W, const void* G, int64_t R, int64_t C, int64_t ldw,
                               int64_t ldg, const float* col_moment, const float* row_weight, int ref_bits,
@@ -471,14 +478,21 @@ static sb_status reorder_impl(sb_ctx* ctx, const void* W, const void* G, int64_t
     const int tiles_r = (int)((R + tile_rows - 1) / tile_rows);
     const int64_t maxK = R > C ? R : C;
     void* arena;
+    const size_t slab_rec = sb_stats_col_rec_floats(C, ctx->sm_count), slab_rows = sb_stats_rowpart_floats(R, C);
     sb_status st = sb_scratch(ctx, Carver::need({(size_t)tiles_c * R * 4, (size_t)tiles_r * C * 4,
-                                                 (size_t)maxK * 4}), &arena);
+                                                 (size_t)maxK * 4, slab_rec * 4, slab_rows * 4}), &arena);
     if (st != SB_OK) return st;
     Carver cv(arena);
     float* rowpart = cv.take<float>((size_t)tiles_c * R);
     float* colpart = cv.take<float>((size_t)tiles_r * C);
     int* rank = cv.take<int>((size_t)maxK);
-    if (W && (row_score || col_score)) {
+    float* slab_col_rec = cv.take<float>(slab_rec);
+    float* slab_rowpart = cv.take<float>(slab_rows);
+    if (W && !G && (row_score || col_score)) {
+        st = sb_reorder_stats_slab(ctx, W, R, C, ldw, col_moment, row_weight, ref_bits, group, row_score, col_score,
+                                   accumulate, slab_col_rec, slab_rowpart);
+        if (st != SB_OK) return st;
+    } else if (W && (row_score || col_score)) {
         const float qmax = (float)((1 << ref_bits) - 1);
         if (tiles_r > SB_STATS_TILES || tiles_c > SB_STATS_TILES)
             return sb_fail(ctx, SB_ERR_SHAPE, "reorder: more than %d tiles on an axis", SB_STATS_TILES);
