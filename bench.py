@@ -330,7 +330,8 @@ def kernel_rooflines(ctx, W, X, moments, dev, peak_gbs, sm_mhz, sm_count):
                         "x SM clock"}
 
     return [
-        hbm("reorder_stats_kernel", 2 * n, t_stats, "one call of sb_reorder_channels (statistics only)"),
+        hbm("block_scores_kernel<StatsScorer> + stats_finish_kernel", 2 * n, t_stats,
+            "one call of sb_reorder_channels (statistics only): the score kernel's slab walk with one candidate"),
         score_entry(BITS, 128, 128, 128, t_score),
     ] + [score_entry(*v) for v in score_variants] + [
         hbm("gather_cols_kernel", 4 * n, t_gather,
@@ -794,6 +795,11 @@ def run_only(which: str):
             rs, cs = torch.empty(R, device=dev), torch.empty(Cc, device=dev)
             for _ in range(3):
                 ctx.reorder_channels(W, c, 2, 128, row_score=rs, col_score=cs)
+        elif which == "reorder_stats_first_order":
+            G = (W.float() * 1e-2).to(torch.bfloat16)
+            rs, cs = torch.empty(R, device=dev), torch.empty(Cc, device=dev)
+            for _ in range(3):
+                ctx.reorder_channels_first_order(W, G, 2, 128, row_score=rs, col_score=cs)
         elif which == "gather":
             pr, pc = torch.randperm(R, device=dev).int(), torch.randperm(Cc, device=dev).int()
             err, out = torch.empty(nb, len(BITS), device=dev), torch.empty_like(W)
@@ -871,7 +877,7 @@ def main():
     ap.add_argument("--no-graphs", action="store_true", help="launch every library call eagerly")
     ap.add_argument("--only", default=None,
                     help="three calls of one library call on one input, then exit (for ncu captures): "
-                         "moments | gram | full_scores | dequant_gemm | reorder_stats | scores | scores3 | scores7 | "
+                         "moments | gram | full_scores | dequant_gemm | reorder_stats | reorder_stats_first_order | scores | scores3 | scores7 | "
                          "gather | pack | first_order | sort | allocate | allocate_model")
     args = ap.parse_args()
     if args.only:
