@@ -352,7 +352,7 @@ def calib_gram(X, scale: Optional[float] = None) -> np.ndarray:
 
 
 def block_scores_full(W, H, bits: Sequence[int], block_rows=128, block_cols=128, group=128,
-                      row_perm=None, col_perm=None) -> np.ndarray:
+                      row_perm=None, col_perm=None, a=None) -> np.ndarray:
     """Block error table with the full second-moment matrix H [C, C] (original column order)."""
     W = _u16(W)
     R, Cc = W.shape
@@ -363,7 +363,7 @@ def block_scores_full(W, H, bits: Sequence[int], block_rows=128, block_cols=128,
     err = np.zeros((nb, L), dtype=np.float64)
     st = lib().sbo_block_scores_full(_p(W), C.c_int64(R), C.c_int64(Cc), C.c_int64(Cc), _p(rp), _p(cp),
                                      _p(H), C.c_int(block_rows), C.c_int(block_cols), C.c_int(group),
-                                     barr, C.c_int(L), _p(err))
+                                     barr, C.c_int(L), _p(err), _p(_f64(a, R)))
     if st != OK:
         raise ValueError(f"sbo_block_scores_full status {st}")
     return err

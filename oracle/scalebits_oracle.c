@@ -292,7 +292,8 @@ int sbo_block_scores(const uint16_t* W, int64_t R, int64_t C, int64_t ldw,
  * permuted column order.  With a diagonal H this is sbo_block_scores with c = diag(H).         */
 int sbo_block_scores_full(const uint16_t* W, int64_t R, int64_t C, int64_t ldw,
                           const int32_t* row_perm, const int32_t* col_perm, const double* H,
-                          int br, int bc, int group, const int* bits, int L, double* err) {
+                          int br, int bc, int group, const int* bits, int L, double* err,
+                          const double* row_weight /* [R] by original row, or NULL = 1 */) {
     if (!check_bits(bits, L)) return SBO_ERR_INVALID;
     if (br <= 0 || bc <= 0 || group <= 0 || R % br || C % bc || bc % group) return SBO_ERR_SHAPE;
     const int64_t nbr = R / br, nbc = C / bc;
@@ -327,7 +328,7 @@ int sbo_block_scores_full(const uint16_t* W, int64_t R, int64_t C, int64_t ldw,
                             const int64_t jbs = col_perm ? col_perm[jb] : jb;
                             s += H[jas * C + jbs] * d[b];
                         }
-                        e += d[a] * s;
+                        e += (row_weight ? row_weight[rs] : 1.0) * (d[a] * s);   /* a_r d_r H d_r^T */
                     }
                 }
                 err[blk * L + l] = e;

@@ -99,7 +99,7 @@ def lib() -> C.CDLL:
                                        vp, C.POINTER(StepReport)]
         L.sb_calib_moments_noalloc.argtypes = [vp, vp, i64, i64, i64, vp, i32, f32]
         L.sb_calib_gram.argtypes = [vp, vp, i64, i64, i64, vp, i32, f32]
-        L.sb_block_scores_full.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp, i32, i32, i32,
+        L.sb_block_scores_full.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp, vp, i32, i32, i32,
                                            C.POINTER(C.c_int), i32, vp, vp, vp]
         L.sb_dequant_gemm.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, i64, i64, i32, i32, i32,
                                       C.POINTER(C.c_int), i32, vp, i64]
@@ -256,8 +256,8 @@ class Context:
 
     def block_scores_full(self, W: torch.Tensor, H: torch.Tensor, bits: Sequence[int],
                           block_rows: int = 128, block_cols: int = 128, group: int = 128,
-                          row_perm=None, col_perm=None, err=None, gain=None, want_gain: bool = True,
-                          W_perm_out=None):
+                          row_perm=None, col_perm=None, row_weight=None, err=None, gain=None,
+                          want_gain: bool = True, W_perm_out=None):
         R, Cc, ldw = _mat(W)
         assert H.shape == (Cc, Cc) and H.is_contiguous()
         barr, L = _bits(bits)
@@ -268,8 +268,8 @@ class Context:
             gain = torch.empty((nb, L - 1), dtype=torch.float32, device=W.device)
         self._check(lib().sb_block_scores_full(
             self._h, _ptr(W), R, Cc, ldw, _ptr(row_perm, torch.int32), _ptr(col_perm, torch.int32),
-            _ptr(H, torch.float32), block_rows, block_cols, group, barr, L, _ptr(err, torch.float32),
-            _ptr(gain, torch.float32), _ptr(W_perm_out, torch.bfloat16)))
+            _ptr(H, torch.float32), _ptr(row_weight, torch.float32), block_rows, block_cols, group, barr, L,
+            _ptr(err, torch.float32), _ptr(gain, torch.float32), _ptr(W_perm_out, torch.bfloat16)))
         return err, gain
 
     def allocate_bits(self, err: torch.Tensor, bits: Sequence[int], budget: float,

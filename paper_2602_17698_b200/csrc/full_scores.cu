@@ -136,11 +136,17 @@ __global__ void gather_hblocks_kernel(const float* __restrict__ H, int64_t C, co
     }
 }
 
-template <int GROUP>
+// PLAIN: units of 128 rows and no row weights (both known at compile time: the common case keeps
+// its instruction stream)
+template <int GROUP, bool PLAIN>
 __global__ void __launch_bounds__(FS_THREADS, 1)
 full_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const float* __restrict__ hblk,
-                   FsBits fb, int L, int64_t n_blocks, int64_t n_block_cols,
+                   FsBits fb, int L, int64_t n_blocks, int64_t n_block_cols, int unit_rows,
+                   const float* __restrict__ row_weight, const int32_t* __restrict__ a_perm, float gain_elems,
                    float* __restrict__ err, float* __restrict__ gain, SbDeviceState* ds) {
+    // A work unit is `unit_rows` (64 or 128) rows x 128 columns; the contraction always runs over 128
+    // rows, the rows past unit_rows of a 64-row unit are written as zeros (they add nothing).
+    // n_blocks / n_block_cols count UNITS here; the host adds the two units of a 256-row block.
     // this CTA's blocks: a contiguous range of the COLUMN-major block sequence, so that consecutive
     // blocks share their columns J (and every thread keeps its entries of H'_JJ in registers)
     const int64_t n_block_rows = n_blocks / n_block_cols;
@@ -193,6 +199,9 @@ full_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const float
     // matrix, columns [32 cq, 32 cq + 32)
     const int j = (warp & 3) * 32 + lane, cq = warp >> 2;
 
+    if (PLAIN) unit_rows = FS_N;
+    const bool row_live = PLAIN || r < unit_rows;
+    float sa = 1.f;                                   // sqrt of the row weight: scales the row's residual
     uint32_t wv[16];
     float glo[NG], hreg[32];
     double dlo[NG], range64[NG];
@@ -217,7 +226,7 @@ full_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const float
         err[blk * L + l_f] = e;
         if (gain && l_f > 0)
             gain[blk * (L - 1) + l_f - 1] =
-                (e_prev - e) / ((float)(fs_bits(fb, l_f) - fs_bits(fb, l_f - 1)) * (float)(FS_N * FS_N));
+                (e_prev - e) / ((float)(fs_bits(fb, l_f) - fs_bits(fb, l_f - 1)) * gain_elems);
         e_prev = e;
         if (++l_f == L) {
             l_f = 0;
@@ -235,16 +244,20 @@ full_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const float
                 l = 0;
                 if (++bi_q == n_block_rows) { bi_q = 0; ++bj_q; }
                 --blocks_left;
-                const uint4* src = reinterpret_cast<const uint4*>(W + (bi_q * FS_N + r) * ldw + bj_q * FS_N + qd * 32);
+                const uint4* src = reinterpret_cast<const uint4*>(W + (bi_q * unit_rows + r) * ldw + bj_q * FS_N + qd * 32);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const uint4 x = __ldg(src + (c ^ cflip));
+                    const uint4 x = row_live ? __ldg(src + (c ^ cflip)) : make_uint4(0u, 0u, 0u, 0u);
                     wv[4 * c] = x.x; wv[4 * c + 1] = x.y; wv[4 * c + 2] = x.z; wv[4 * c + 3] = x.w;
                 }
-                if (blocks_left > 0) {                       // the next block's 64 bytes of this thread towards L2
+                if (!PLAIN && row_weight) {
+                    const int64_t row = bi_q * unit_rows + r;
+                    sa = row_live ? sqrtf(__ldg(row_weight + (a_perm ? a_perm[row] : row))) : 0.f;
+                }
+                if (blocks_left > 0 && row_live) {           // the next block's 64 bytes of this thread towards L2
                     const bool wrap = bi_q + 1 == n_block_rows;
                     const int64_t bi1 = wrap ? 0 : bi_q + 1, bj1 = wrap ? bj_q + 1 : bj_q;
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(W + (bi1 * FS_N + r) * ldw + bj1 * FS_N + qd * 32));
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(W + (bi1 * unit_rows + r) * ldw + bj1 * FS_N + qd * 32));
                 }
                 // group minimum and maximum per 8-column chunk (exact bf16 min / max)
                 float clo[4], chi[4];
@@ -314,13 +327,16 @@ full_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const float
                 for (int k = 0; k < 8; ++k) t8[k] = __dadd_rn(__dmul_rn(t8[k], inv64[g]), FS_MAGIC64);
                 // the fp32 part on packed pairs (half the issue slots)
                 const f32x2 ns2 = pk2(ns[g], ns[g]), ns_lo2 = pk2(ns_lo[g], ns_lo[g]), nlo2 = pk2(-glo[g], -glo[g]);
+                const f32x2 sa2 = pk2(sa, sa);
+                const bool weighted = !PLAIN && row_weight != nullptr;
                 const f32x2 nmagic2 = pk2(-8388608.f, -8388608.f), none2 = pk2(-1.f, -1.f);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     // exact int -> float: 2^23 + q as bits, minus 2^23
                     const f32x2 q2 = add2(pk2(__int_as_float(__double2loint(t8[2 * k])),
                                               __int_as_float(__double2loint(t8[2 * k + 1]))), nmagic2);
-                    const f32x2 e2 = fma2(q2, ns_lo2, fma2(q2, ns2, add2(pk2(w8[2 * k], w8[2 * k + 1]), nlo2)));
+                    f32x2 e2 = fma2(q2, ns_lo2, fma2(q2, ns2, add2(pk2(w8[2 * k], w8[2 * k + 1]), nlo2)));
+                    if (weighted) e2 = mul2(e2, sa2);
                     float e0, e1;
                     upk2(e2, e0, e1);
                     const __nv_bfloat162 hi2 = __floats2bfloat162_rn(e0, e1);
@@ -414,25 +430,46 @@ full_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const float
     if (threadIdx.x == 0 && *abort_flag) sb_latch(ds, SB_ERR_TIMEOUT, SBK_SCORES);
 }
 
+// blocks of 256 rows: err[blk][l] = the sum of the block's two 128-row units; gains
+__global__ void full_combine_kernel(const float* __restrict__ unit_err, int64_t n_blocks, int64_t nbc, int L,
+                                    FsBits fb, float gain_elems, float* __restrict__ err, float* __restrict__ gain) {
+    const int64_t blk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (blk >= n_blocks) return;
+    const int64_t bi = blk / nbc, bj = blk - bi * nbc;
+    const float* u0 = unit_err + ((2 * bi) * nbc + bj) * L;
+    const float* u1 = unit_err + ((2 * bi + 1) * nbc + bj) * L;
+    float prev = 0.f;
+    for (int l = 0; l < L; ++l) {
+        const float e = u0[l] + u1[l];
+        err[blk * L + l] = e;
+        if (gain && l > 0) gain[blk * (L - 1) + l - 1] = (prev - e) / ((float)(fs_bits(fb, l) - fs_bits(fb, l - 1)) * gain_elems);
+        prev = e;
+    }
+}
+
 }  // namespace
 
 extern "C" sb_status sb_block_scores_full(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64_t ldw,
                                           const int32_t* row_perm, const int32_t* col_perm, const float* H,
-                                          int br, int bc, int group, const int* bits, int n_bits, float* err,
-                                          float* gain, void* W_perm_out) {
+                                          const float* row_weight, int br, int bc, int group, const int* bits,
+                                          int n_bits, float* err, float* gain, void* W_perm_out) {
     if (!ctx) return SB_ERR_INVALID;
     if (!W || !H || !err || R <= 0 || C <= 0) return sb_fail(ctx, SB_ERR_INVALID, "full scores: null or empty");
     if (!sb_check_bits(bits, n_bits)) return sb_fail(ctx, SB_ERR_INVALID, "full scores: bits must be ascending in 1..8");
     const bool g_ok = group == 16 || group == 32 || group == 64 || group == 128;
-    if (br != FS_N || bc != FS_N || !g_ok || R % FS_N || C % FS_N || ldw % 8 || ldw < C ||
+    if (!(br == 64 || br == 128 || br == 256) || bc != FS_N || !g_ok || R % br || C % FS_N || ldw % 8 || ldw < C ||
         (reinterpret_cast<uintptr_t>(W) & 15))
-        return sb_fail(ctx, SB_ERR_SHAPE, "full scores: blocks of 128 x 128 tiling the matrix, group in {16,32,64,128}");
+        return sb_fail(ctx, SB_ERR_SHAPE, "full scores: blocks of 64, 128 or 256 rows x 128 columns tiling the matrix, "
+                                          "group in {16,32,64,128}");
     SB_CUDA(ctx, cudaSetDevice(ctx->device));
-    const int64_t nbc = C / FS_N, n_blocks = (R / FS_N) * nbc;
+    const int unit_rows = br < FS_N ? br : FS_N;                 // rows of one contraction
+    const int units_per_block = br / unit_rows;                  // 1, or 2 for 256-row blocks
+    const int64_t nbc = C / FS_N, n_units = (R / unit_rows) * nbc, n_blocks = (R / br) * nbc;
     const bool need_copy = row_perm || col_perm || W_perm_out;
     void* arena;
     sb_status st = sb_scratch(ctx, Carver::need({(size_t)nbc * FS_N * FS_N * 4,
-                                                 (need_copy && !W_perm_out) ? (size_t)R * C * 2 : 0}), &arena);
+                                                 (need_copy && !W_perm_out) ? (size_t)R * C * 2 : 0,
+                                                 units_per_block > 1 ? (size_t)n_units * n_bits * 4 : 0}), &arena);
     if (st != SB_OK) return st;
     Carver cv(arena);
     float* hblk = cv.take<float>((size_t)nbc * FS_N * FS_N);
@@ -445,17 +482,25 @@ extern "C" sb_status sb_block_scores_full(sb_ctx* ctx, const void* W, int64_t R,
         src = static_cast<const __nv_bfloat16*>(dst);
         ld = C;
     }
+    float* unit_err = units_per_block > 1 ? cv.take<float>((size_t)n_units * n_bits) : err;
     gather_hblocks_kernel<<<(unsigned)nbc, 256, 0, ctx->stream>>>(H, C, col_perm, hblk);
     SB_LAUNCHED(ctx);
     FsBits fb{};
     for (int l = 0; l < n_bits; ++l) fb.packed |= (unsigned)bits[l] << (4 * l);
-    const int64_t grid = n_blocks < ctx->sm_count ? n_blocks : ctx->sm_count;
+    const int64_t grid = n_units < ctx->sm_count ? n_units : ctx->sm_count;
+    const float gain_elems = (float)br * (float)FS_N;
+    float* kernel_gain = units_per_block > 1 ? nullptr : gain;
+    const bool plain = unit_rows == FS_N && !row_weight;
+#define FS_LAUNCH_P(G, P)                                                                                         \
+    do {                                                                                                          \
+        SB_FUNC_ATTR(ctx, (full_scores_kernel<G, P>), cudaFuncAttributeMaxDynamicSharedMemorySize, FS_SMEM);      \
+        full_scores_kernel<G, P><<<(unsigned)grid, FS_THREADS, FS_SMEM, ctx->stream>>>(                           \
+            src, ld, hblk, fb, n_bits, n_units, nbc, unit_rows, row_weight, row_perm, gain_elems, unit_err,       \
+            kernel_gain, ctx->dstate);                                                                            \
+    } while (0)
 #define FS_LAUNCH(G)                                                                                              \
     do {                                                                                                          \
-        SB_FUNC_ATTR(ctx, full_scores_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, FS_SMEM);           \
-        full_scores_kernel<G><<<(unsigned)grid, FS_THREADS, FS_SMEM, ctx->stream>>>(src, ld, hblk, fb, n_bits,    \
-                                                                                    n_blocks, nbc, err, gain,     \
-                                                                                    ctx->dstate);                 \
+        if (plain) FS_LAUNCH_P(G, true); else FS_LAUNCH_P(G, false);                                              \
     } while (0)
     switch (group) {
         case 16: FS_LAUNCH(16); break;
@@ -464,6 +509,12 @@ extern "C" sb_status sb_block_scores_full(sb_ctx* ctx, const void* W, int64_t R,
         default: FS_LAUNCH(128); break;
     }
 #undef FS_LAUNCH
+#undef FS_LAUNCH_P
     SB_LAUNCHED(ctx);
+    if (units_per_block > 1) {
+        full_combine_kernel<<<(unsigned)((n_blocks + 255) / 256), 256, 0, ctx->stream>>>(unit_err, n_blocks, nbc, n_bits, fb,
+                                                                                         gain_elems, err, gain);
+        SB_LAUNCHED(ctx);
+    }
     return SB_OK;
 }

@@ -258,3 +258,26 @@ def test_full_second_moment_block_scores_pins():
     Wp = W[torch.from_numpy(pr).long()][:, torch.from_numpy(pc).long()].contiguous()
     Hp = H[np.ix_(pc, pc)]
     assert np.allclose(e_perm, sbo.block_scores_full(Wp, Hp, bits, br, bc, g), rtol=1e-12)
+    # row weights a_r (the row factor of Section 3.2), indexed by ORIGINAL row: with a diagonal H the
+    # weighted form is the pinned weighted block table; with the rank-one H it is sum_r a_r (d_r . u)^2
+    # (rows of a block-row written out here); it is linear in a
+    a = rng.uniform(0.2, 3.0, size=R)
+    e_wd = sbo.block_scores_full(W, np.diag(c), bits, br, bc, g, a=a)
+    e_wref, _ = sbo.block_scores(W, c, bits, br, bc, g, a=a)
+    assert np.allclose(e_wd, e_wref, rtol=1e-12)
+    e_w1 = sbo.block_scores_full(W, np.outer(u, u), bits, br, bc, g, a=a)
+    for l, b in enumerate(bits):
+        D = np.empty_like(Wd)
+        for r in range(R):
+            for c0 in range(0, C, g):
+                _, vh, _, _ = sbo.quantize_group(Wd[r, c0:c0 + g], b)
+                D[r, c0:c0 + g] = Wd[r, c0:c0 + g] - vh
+        for blk in range((R // br) * (C // bc)):
+            bi, bj = divmod(blk, C // bc)
+            proj = D[bi * br:(bi + 1) * br, bj * bc:(bj + 1) * bc] @ u[bj * bc:(bj + 1) * bc]
+            assert e_w1[blk, l] == pytest.approx((a[bi * br:(bi + 1) * br] * proj ** 2).sum(), rel=1e-11)
+    assert np.allclose(sbo.block_scores_full(W, H, bits, br, bc, g, a=2.5 * a),
+                       2.5 * sbo.block_scores_full(W, H, bits, br, bc, g, a=a), rtol=1e-12)
+    # with a row permutation the weight follows the ORIGINAL row
+    e_wp = sbo.block_scores_full(W, H, bits, br, bc, g, row_perm=pr, col_perm=pc, a=a)
+    assert np.allclose(e_wp, sbo.block_scores_full(Wp, Hp, bits, br, bc, g, a=a[pr]), rtol=1e-12)
