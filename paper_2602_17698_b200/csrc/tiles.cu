@@ -140,21 +140,20 @@ __device__ __forceinline__ void load_cols(const __nv_bfloat16* p, bool ok, uint3
     }
 }
 
-// ---- reorder statistics --------------------------------------------------------------------
-// 128 x 128 tiles of the ORIGINAL layout, one candidate (ref_bits).  Every tile writes its
-// partial row sums rowpart[tile_col][r] and column sums colpart[tile_row][j]; the last tile of
-// a tile row (tile column) to finish adds the partials of that row strip (column strip) in
-// tile order -- a fixed order whichever CTA does it, and no floating-point atomics, so reruns
-// are bit-identical -- and adds them to / stores them in the score vectors.
-// FIRST: the first-order form of the element sensitivity, |G_rj (W_rj - Q(W)_rj)| (Section 3.2
-// with p = 1), from a caller's gradient G; no column or row factors.
-// A tile is `tile_rows` (a multiple of 32) x 128; the host picks tile_rows so that the tiles fill
-// whole rounds of the CTA slots of the GPU.
-template <bool ROWW, bool FINE, bool FIRST>
+// ---- reorder statistics, first-order form --------------------------------------------------
+// (The second-moment form runs on the score kernel's slab walk: scores.cu.)
+// Element sensitivity |G_rj (W_rj - Q(W)_rj)| (Section 3.2 with p = 1) from a caller's gradient G,
+// summed per channel (l1 aggregation, Section 4.1).  128 x 128 tiles of the ORIGINAL layout, one
+// candidate (ref_bits).  Every tile writes its partial row sums rowpart[tile_col][r] and column
+// sums colpart[tile_row][j]; the last tile of a tile row (tile column) to finish adds the partials
+// of that row strip (column strip) in tile order -- a fixed order whichever CTA does it, and no
+// floating-point atomics, so reruns are bit-identical -- and adds them to / stores them in the
+// score vectors.  A tile is `tile_rows` (a multiple of 32) x 128; the host picks tile_rows so that
+// the tiles fill whole rounds of the CTA slots of the GPU.
+template <bool FINE>
 __global__ void __launch_bounds__(CTA_THREADS)
 reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, int64_t ldw, int tile_rows,
                      const __nv_bfloat16* __restrict__ G, int64_t ldg,
-                     const float* __restrict__ col_moment, const float* __restrict__ row_weight,
                      int group, float qmax, float inv_qmax,
                      float* __restrict__ rowpart, float* __restrict__ colpart,
                      float* __restrict__ row_score, float* __restrict__ col_score, int accumulate,
@@ -169,37 +168,29 @@ reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, 
     const bool col_ok = col < C;
     const int64_t row0 = (int64_t)blockIdx.y * tile_rows;
     const f32x2 magic2 = pk2(RNE_MAGIC, RNE_MAGIC), nmagic2 = pk2(-RNE_MAGIC, -RNE_MAGIC);
-    f32x2 cw[NW], acc[NW];
+    f32x2 acc[NW];
 #pragma unroll
-    for (int k = 0; k < NW; ++k) {
-        if (FIRST) cw[k] = pk2(1.f, 1.f);
-        else cw[k] = col_ok ? pk2(col_moment[col + 2 * k], col_moment[col + 2 * k + 1]) : 0ull;
-        acc[k] = 0ull;
-    }
-    // the next step's two 16-byte loads are in flight while this step is evaluated
-    uint32_t wn[NW], gn[FIRST ? NW : 1];
+    for (int k = 0; k < NW; ++k) acc[k] = 0ull;
+    // the next step's 16-byte loads are in flight while this step is evaluated
+    uint32_t wn[NW], gn[NW];
     {
         const int64_t r = row0 + warp * ROW_SLOTS + slot;
         const bool ok = col_ok && r < R;
         load_cols<CPL>(W + (ok ? r * ldw + col : 0), ok, wn);
-        if constexpr (FIRST) load_cols<CPL>(G + (ok ? r * ldg + col : 0), ok, gn);
+        load_cols<CPL>(G + (ok ? r * ldg + col : 0), ok, gn);
     }
 #pragma unroll 2
     for (int it = 0; it < ITERS; ++it) {
         const int rr = it * (CTA_WARPS * ROW_SLOTS) + warp * ROW_SLOTS + slot;
         const int64_t r = row0 + rr;
-        uint32_t w[NW], gw[FIRST ? NW : 1];
+        uint32_t w[NW], gw[NW];
 #pragma unroll
-        for (int k = 0; k < NW; ++k) w[k] = wn[k];
-        if constexpr (FIRST) {
-#pragma unroll
-            for (int k = 0; k < NW; ++k) gw[k] = gn[k];
-        }
+        for (int k = 0; k < NW; ++k) { w[k] = wn[k]; gw[k] = gn[k]; }
         if (it + 1 < ITERS) {
             const int64_t rn = r + CTA_WARPS * ROW_SLOTS;
             const bool okn = col_ok && rn < R;
             load_cols<CPL>(W + (okn ? rn * ldw + col : 0), okn, wn);
-            if constexpr (FIRST) load_cols<CPL>(G + (okn ? rn * ldg + col : 0), okn, gn);
+            load_cols<CPL>(G + (okn ? rn * ldg + col : 0), okn, gn);
         }
         float lo, hi;
         group_minmax<NW>(w, team, lo, hi);
@@ -213,11 +204,6 @@ reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, 
             const float nscale_lo = -(fmaf(nscale, qmax, range) * inv_qmax);
             nslo2 = pk2(nscale_lo, nscale_lo);
         }
-        f32x2 ar2 = 0ull;
-        if (ROWW) {
-            const float ar = (r < R) ? row_weight[r] : 0.f;
-            ar2 = pk2(ar, ar);
-        }
         f32x2 rs2 = 0ull;
 #pragma unroll
         for (int k = 0; k < NW; ++k) {
@@ -225,16 +211,10 @@ reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, 
             const f32x2 qq = add2(fma2(vm, inv2, magic2), nmagic2);
             f32x2 e = fma2(qq, ns2, vm);
             if (FINE) e = fma2(qq, nslo2, e);
-            f32x2 e2;
-            if constexpr (FIRST) {
-                const f32x2 ge = mul2(pk2(bf16lo(gw[k]), bf16hi(gw[k])), e);
-                e2 = ge & 0x7fffffff7fffffffull;                // |g e| on both halves
-            } else {
-                e2 = mul2(e, e);
-            }
-            if (ROWW) e2 = mul2(e2, ar2);
+            const f32x2 ge = mul2(pk2(bf16lo(gw[k]), bf16hi(gw[k])), e);
+            const f32x2 e2 = ge & 0x7fffffff7fffffffull;        // |g e| on both halves
             acc[k] = add2(acc[k], e2);
-            rs2 = fma2(cw[k], e2, rs2);
+            rs2 = add2(rs2, e2);
         }
         float r0f, r1f;
         upk2(rs2, r0f, r1f);
@@ -247,11 +227,10 @@ reorder_stats_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int64_t C, 
     if (colpart) {
 #pragma unroll
         for (int k = 0; k < NW; ++k) {
-            float a0, a1, c0, c1;
+            float a0, a1;
             upk2(acc[k], a0, a1);
-            upk2(cw[k], c0, c1);
-            red[warp * ROW_SLOTS + slot][cl * CPL + 2 * k] = a0 * c0;
-            red[warp * ROW_SLOTS + slot][cl * CPL + 2 * k + 1] = a1 * c1;
+            red[warp * ROW_SLOTS + slot][cl * CPL + 2 * k] = a0;
+            red[warp * ROW_SLOTS + slot][cl * CPL + 2 * k + 1] = a1;
         }
         __syncthreads();
         if (threadIdx.x < TILE_COLS) {
@@ -457,10 +436,7 @@ static sb_status reorder_impl(sb_ctx* ctx, const void* W, const void* G, int64_t
     // whole round: 512 rows on 14336 x 4096 made 896 tiles for 444 slots, three rounds instead of two.
     // the instance that will run, for its occupancy
     const bool fine = ref_bits >= 6;
-    const void* kern;
-    if (G) kern = fine ? (const void*)reorder_stats_kernel<false, true, true> : (const void*)reorder_stats_kernel<false, false, true>;
-    else if (row_weight) kern = fine ? (const void*)reorder_stats_kernel<true, true, false> : (const void*)reorder_stats_kernel<true, false, false>;
-    else kern = fine ? (const void*)reorder_stats_kernel<false, true, false> : (const void*)reorder_stats_kernel<false, false, false>;
+    const void* kern = fine ? (const void*)reorder_stats_kernel<true> : (const void*)reorder_stats_kernel<false>;
     int occ = 0;
     SB_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, CTA_THREADS, 0));
     if (occ < 1) occ = 1;
@@ -502,15 +478,15 @@ static sb_status reorder_impl(sb_ctx* ctx, const void* W, const void* G, int64_t
         float* cpart = col_score ? colpart : nullptr;
         unsigned* done_row = ctx->stats_done;
         unsigned* done_col = ctx->stats_done + SB_STATS_TILES;
-#define SB_STATS(RW, FN, FO)                                                                      \
-    reorder_stats_kernel<RW, FN, FO><<<grid, CTA_THREADS, 0, ctx->stream>>>(                      \
-        Wb, R, C, ldw, tile_rows, Gb, ldg, col_moment, row_weight, group, qmax, 1.0f / qmax, rpart, cpart, \
-        row_score, col_score, accumulate, done_row, done_col, ctx->dstate)
         auto* Gb = static_cast<const __nv_bfloat16*>(G);
-        if (G) { if (fine) SB_STATS(false, true, true); else SB_STATS(false, false, true); }
-        else if (row_weight) { if (fine) SB_STATS(true, true, false); else SB_STATS(true, false, false); }
-        else { if (fine) SB_STATS(false, true, false); else SB_STATS(false, false, false); }
-#undef SB_STATS
+        if (fine)
+            reorder_stats_kernel<true><<<grid, CTA_THREADS, 0, ctx->stream>>>(
+                Wb, R, C, ldw, tile_rows, Gb, ldg, group, qmax, 1.0f / qmax, rpart, cpart, row_score, col_score,
+                accumulate, done_row, done_col, ctx->dstate);
+        else
+            reorder_stats_kernel<false><<<grid, CTA_THREADS, 0, ctx->stream>>>(
+                Wb, R, C, ldw, tile_rows, Gb, ldg, group, qmax, 1.0f / qmax, rpart, cpart, row_score, col_score,
+                accumulate, done_row, done_col, ctx->dstate);
         SB_LAUNCHED(ctx);
     }
     if (sort_rows) { st = argsort_axis(ctx, row_score, R, row_segment, row_perm, rank); if (st) return st; }
