@@ -71,6 +71,9 @@ const char* sb_last_error(const sb_ctx* ctx);
 sb_status sb_debug_lookback(sb_ctx* ctx, int64_t wait_ns, int64_t mute_tile);
 /* Number of kernels this context has launched so far (for launch accounting).       */
 int64_t sb_kernel_launches(const sb_ctx* ctx);
+/* 1 if the library was built with -DSB_CHECKED (data-dependent indices bounds-checked on the device,
+ * a failing one latched as SB_ERR_INVALID with the index in sb_last_error), else 0.           */
+int sb_checked_build(void);
 
 /* Calibration second moments -- the column factor |x_j| of the element sensitivity
  * (Section 3.2, the equation after Eq. 3), aggregated over tokens as a second moment:

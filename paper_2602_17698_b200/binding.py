@@ -13,7 +13,8 @@ from typing import Optional, Sequence
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libscalebits.so")
+# SCALEBITS_LIB selects another build of the same library (the bounds-checked one, for tests)
+LIB_PATH = os.environ.get("SCALEBITS_LIB") or os.path.join(_PKG, "libscalebits.so")
 
 SB_OK, SB_ERR_INVALID, SB_ERR_SHAPE, SB_ERR_BUDGET, SB_ERR_SCRATCH, SB_ERR_CUDA, \
     SB_ERR_NOCONVERGE, SB_ERR_NONFINITE, SB_ERR_TIMEOUT = range(9)
@@ -21,6 +22,7 @@ SB_ALLOC_SCALEBITS, SB_ALLOC_GREEDY = 0, 1
 SB_ACC_ROW, SB_ACC_COL = 1, 2
 
 EXPORTS = ["sb_create", "sb_destroy", "sb_sync", "sb_last_error", "sb_kernel_launches", "sb_debug_lookback",
+           "sb_checked_build",
            "sb_calib_moments", "sb_reorder_channels", "sb_fold_segment_scores",
            "sb_expand_segment_perm", "sb_permute_matrix", "sb_block_scores", "sb_allocate_bits", "sb_pack_blocks",
            "sb_calib_moments_noalloc", "sb_first_order_scores", "sb_exchange_step",
@@ -77,6 +79,7 @@ def lib() -> C.CDLL:
         L.sb_destroy.argtypes = [vp]
         L.sb_sync.argtypes = [vp]
         L.sb_debug_lookback.argtypes = [vp, i64, i64]
+        L.sb_checked_build.argtypes = []
         L.sb_last_error.argtypes = [vp]
         L.sb_last_error.restype = C.c_char_p
         L.sb_kernel_launches.argtypes = [vp]
@@ -372,6 +375,11 @@ class Context:
             _ptr(level, torch.uint8), R, Cc, block_rows, block_cols, group, barr, L,
             _ptr(Y, torch.float32), Y.stride(0)))
         return Y
+
+
+def checked_build() -> bool:
+    """True if the loaded library is the bounds-checked build (-DSB_CHECKED)."""
+    return bool(lib().sb_checked_build())
 
 
 def calib_moments_noalloc(X: torch.Tensor, sumsq: Optional[torch.Tensor] = None,

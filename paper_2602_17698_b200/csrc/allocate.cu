@@ -53,6 +53,7 @@ struct AllocArgs {
     // difference of that candidate, and the move marked for the apply step (stamp << 1 | down)
     unsigned long long* upsr; unsigned long long* upcum; double* upde; unsigned* mark;
     double* part;                                                      // partial sums
+    SbDeviceState* ds;                                                 // status word (bounds checks of the checked build)
 };
 
 __device__ __forceinline__ unsigned long long order_key64(double d) {
@@ -684,11 +685,11 @@ scalebits_loop_masked_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, c
             // the owner of a list entry knows the block and its new level: no loads
             for (unsigned m = um; m; m &= m - 1) {
                 const unsigned e = __ldg(up_ent + t_lo + (__ffs(m) - 1));
-                a.level[e >> 3] = (unsigned char)((e & 7u) + 1u);
+                if (SB_IN_BOUNDS(a.ds, SBK_ALLOC, e >> 3, a.N)) a.level[e >> 3] = (unsigned char)((e & 7u) + 1u);
             }
             for (unsigned m = dsel; m; m &= m - 1) {
                 const unsigned e = __ldg(dn_ent + t_lo + (__ffs(m) - 1));
-                a.level[e >> 3] = (unsigned char)(e & 7u);
+                if (SB_IN_BOUNDS(a.ds, SBK_ALLOC, e >> 3, a.N)) a.level[e >> 3] = (unsigned char)(e & 7u);
             }
         }
         if (expand && accept) { used += (long long)costU; loss -= dU; expansions += 1; }
@@ -755,6 +756,7 @@ __global__ void greedy_apply_kernel(AllocArgs a, const unsigned* __restrict__ li
     const unsigned e = list[p];
     const long long i = e / (unsigned)(a.L - 1);
     const int q = (int)(e % (unsigned)(a.L - 1)) + 1;
+    if (!SB_IN_BOUNDS(a.ds, SBK_ALLOC, i, a.N)) return;
     atomicMax(level32 + i, q);
     atomicAdd(steps, 1);
 }
@@ -868,7 +870,7 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
     a.err = err; a.block_elems = reinterpret_cast<const long long*>(block_elems);
     a.uniform = uniform_block_elems; a.N = N; a.L = L;
     for (int l = 0; l < 8; ++l) a.bits[l] = l < L ? bits[l] : 0;
-    a.level = level; a.st = dst;
+    a.level = level; a.st = dst; a.ds = ctx->dstate;
     a.upsr = upsr; a.upcum = upcum; a.upde = upde; a.mark = mark;
     a.part = part;
 

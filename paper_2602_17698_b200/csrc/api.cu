@@ -113,6 +113,10 @@ sb_status sb_sync(sb_ctx* ctx) {
         sb_status st = static_cast<sb_status>(h->status);
         int where = h->where;
         SB_CUDA(ctx, cudaMemsetAsync(ctx->dstate, 0, 2 * sizeof(int), ctx->stream));
+        SB_CUDA(ctx, cudaMemsetAsync(&ctx->dstate->bad_index, 0, 2 * sizeof(long long), ctx->stream));
+        if (h->bad_limit != 0)
+            return sb_fail(ctx, st, "device-side status %d latched by kernel family %d: index %lld outside [0, %lld)",
+                           (int)st, where, h->bad_index, h->bad_limit);
         return sb_fail(ctx, st, "device-side status %d latched by kernel family %d", (int)st, where);
     }
     return SB_OK;
@@ -132,5 +136,13 @@ sb_status sb_debug_lookback(sb_ctx* ctx, int64_t wait_ns, int64_t mute_tile) {
 const char* sb_last_error(const sb_ctx* ctx) { return ctx ? ctx->err : "null context"; }
 
 int64_t sb_kernel_launches(const sb_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int sb_checked_build(void) {
+#ifdef SB_CHECKED
+    return 1;
+#else
+    return 0;
+#endif
+}
 
 }  // extern "C"

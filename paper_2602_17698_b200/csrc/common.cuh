@@ -18,6 +18,7 @@ struct SbDeviceState {           // lives in device memory, one per context
     unsigned long long lb_wait_ns;   // how long a look-back wait may last (default 250 ms)
     unsigned int lb_mute_tile;       // test hook: this tile of a look-back launch publishes nothing
     unsigned int pad2;               //   (0xffffffff: none)
+    long long bad_index, bad_limit;  // checked build: the first index that failed its bounds check
 };
 
 struct sb_ctx {
@@ -97,6 +98,22 @@ enum SbKernelId { SBK_MOMENTS = 1, SBK_STATS, SBK_SCORES, SBK_GATHER, SBK_ARGSOR
 __device__ __forceinline__ void sb_latch(SbDeviceState* st, int status, int where) {
     if (atomicCAS(&st->status, 0, status) == 0) st->where = where;
 }
+
+// Checked build (-DSB_CHECKED, the stand-in for a memory checker): SB_IN_BOUNDS guards the
+// accesses whose index comes from data (permutations, sorted lists, prefix sums, record numbers).
+// A failing index is latched with the kernel family into the device state (SB_ERR_INVALID,
+// surfaced by sb_sync) and the access is skipped; nothing traps.  In the regular build the macro
+// is the constant true and costs nothing.
+#ifdef SB_CHECKED
+__device__ __forceinline__ bool sb_in_bounds(SbDeviceState* st, int where, long long idx, long long limit) {
+    if (idx >= 0 && idx < limit) return true;
+    if (atomicCAS(&st->status, 0, (int)SB_ERR_INVALID) == 0) { st->where = where; st->bad_index = idx; st->bad_limit = limit; }
+    return false;
+}
+#define SB_IN_BOUNDS(st, where, idx, limit) sb_in_bounds((st), (where), (long long)(idx), (long long)(limit))
+#else
+#define SB_IN_BOUNDS(st, where, idx, limit) true
+#endif
 
 // two bf16 packed in a 32-bit word -> two fp32 (exact)
 __device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }

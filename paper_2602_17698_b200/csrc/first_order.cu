@@ -126,6 +126,7 @@ struct StepArgs {
     const float* s_up; const float* s_down; const unsigned char* level; long long N;
     const long long* block_elems; long long uniform; int L; int bits[8];
     StepState* st;
+    SbDeviceState* ds;          // status word (bounds checks of the checked build)
 };
 
 __device__ __forceinline__ unsigned long long fo_order_key64(double d) {
@@ -260,13 +261,17 @@ step_apply_kernel(StepArgs a, const unsigned* __restrict__ vup, const unsigned* 
     if (st.moved && p < a.N) {
         if (p < st.n_up) {
             const long long i = vup[p];
-            level_out[i] = (unsigned char)(a.level[i] + 1);
-            su = (double)a.s_up[i];
+            if (SB_IN_BOUNDS(a.ds, SBK_ALLOC, i, a.N)) {
+                level_out[i] = (unsigned char)(a.level[i] + 1);
+                su = (double)a.s_up[i];
+            }
         }
         if (!st.expansion && flag[p] && (long long)dnrank[p] < st.h) {
             const long long i = vdn[p];
-            level_out[i] = (unsigned char)(a.level[i] - 1);
-            sd = (double)a.s_down[i];
+            if (SB_IN_BOUNDS(a.ds, SBK_ALLOC, i, a.N)) {
+                level_out[i] = (unsigned char)(a.level[i] - 1);
+                sd = (double)a.s_down[i];
+            }
         }
     }
     su = warp_sum(su); sd = warp_sum(sd);
@@ -393,7 +398,7 @@ sb_status sb_exchange_step(sb_ctx* ctx, const float* s_up, const float* s_down, 
     a.block_elems = reinterpret_cast<const long long*>(block_elems); a.uniform = uniform_block_elems;
     a.L = n_bits;
     for (int l = 0; l < 8; ++l) a.bits[l] = l < n_bits ? bits[l] : 0;
-    a.st = dst;
+    a.st = dst; a.ds = ctx->dstate;
     const unsigned g = (unsigned)((N + 255) / 256);
     step_keys_fo_kernel<<<g, 256, 0, ctx->stream>>>(a, kup, vup, kdn, vdn);
     SB_LAUNCHED(ctx);

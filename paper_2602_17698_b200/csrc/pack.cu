@@ -110,6 +110,9 @@ struct PackLane {
     unsigned* dst;               // first word of the lane in row row0 of its block
     unsigned row_words;          // words per block row
     bool meta_lane, odd_lane;
+    const unsigned* packed;      // the packed buffer and its capacity in words (checked build)
+    long long capacity;
+    SbDeviceState* ds;
 };
 
 // One (row, 16 columns) per lane and step: binary64 codes of the lane's 16 weights.
@@ -173,14 +176,18 @@ __device__ __forceinline__ void pack_rows(const PackLane& pl) {
             if (!pl.odd_lane) {
                 w[B >> 1] |= nb_low << 16;
 #pragma unroll
-                for (int i = 0; i <= (B >> 1); ++i) dst[i] = w[i];
+                for (int i = 0; i <= (B >> 1); ++i)
+                    if (SB_IN_BOUNDS(pl.ds, SBK_PACK, (dst - pl.packed) + i, pl.capacity)) dst[i] = w[i];
             } else {
 #pragma unroll
-                for (int i = 0; i < (B >> 1); ++i) dst[i] = (w[i] >> 16) | (w[i + 1] << 16);
+                for (int i = 0; i < (B >> 1); ++i)
+                    if (SB_IN_BOUNDS(pl.ds, SBK_PACK, (dst - pl.packed) + i, pl.capacity))
+                        dst[i] = (w[i] >> 16) | (w[i + 1] << 16);
             }
         } else {
 #pragma unroll
-            for (int i = 0; i < (B >> 1); ++i) dst[i] = w[i];
+            for (int i = 0; i < (B >> 1); ++i)
+                if (SB_IN_BOUNDS(pl.ds, SBK_PACK, (dst - pl.packed) + i, pl.capacity)) dst[i] = w[i];
         }
     }
 }
@@ -297,6 +304,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const int32_t* __r
     // word offset of this lane's bits inside its row piece; odd b: the odd lane starts 16 bits in
     const long long lane_word = s_base[pc] + (lp * 16 * b) / 32 + (((b & 1) && pl.odd_lane) ? 1 : 0);
     pl.dst = packed + lane_word;
+    pl.packed = packed; pl.capacity = capacity; pl.ds = ds;
 
     if (uniform && all_fit) {
         switch (b) {

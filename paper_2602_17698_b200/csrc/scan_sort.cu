@@ -168,8 +168,10 @@ onesweep_pass_kernel(const unsigned long long* __restrict__ keys_in, const unsig
         if (i < n) {
             const unsigned d = (unsigned)(key[k] >> shift) & 0xffu;
             const int64_t pos = (int64_t)basepos[d] + cnt[warp][d] + rank[k];
-            keys_out[pos] = key[k];
-            vals_out[pos] = val[k];
+            if (SB_IN_BOUNDS(st, SBK_SORT, pos, n)) {
+                keys_out[pos] = key[k];
+                vals_out[pos] = val[k];
+            }
         }
     }
 }
@@ -224,7 +226,8 @@ constexpr int CL_SORT_SMEM = 2 * CL_SORT_PER_CTA * 8 + 2 * CL_SORT_PER_CTA * 4 +
                              CL_SORT_WARPS * RADIX * 2 + 2 * RADIX * 4 + 256;
 
 __global__ void __launch_bounds__(CL_SORT_THREADS, 1)
-cluster_sort_kernel(unsigned long long* __restrict__ keys, unsigned* __restrict__ vals, int n, int m) {
+cluster_sort_kernel(unsigned long long* __restrict__ keys, unsigned* __restrict__ vals, int n, int m,
+                    SbDeviceState* ds) {
     cg::cluster_group cluster = cg::this_cluster();
     extern __shared__ unsigned long long cs_smem[];
     unsigned long long* kbase = cs_smem;                                          // two key buffers
@@ -323,8 +326,10 @@ cluster_sort_kernel(unsigned long long* __restrict__ keys, unsigned* __restrict_
             __syncwarp();
             if (live) {
                 const unsigned dest = pos / (unsigned)m, idx = pos - dest * (unsigned)m;
-                *cluster.map_shared_rank(kout + idx, dest) = key;
-                *cluster.map_shared_rank(vout + idx, dest) = vin[i];
+                if (SB_IN_BOUNDS(ds, SBK_SORT, pos, n)) {
+                    *cluster.map_shared_rank(kout + idx, dest) = key;
+                    *cluster.map_shared_rank(vout + idx, dest) = vin[i];
+                }
             }
         }
         cur ^= 1;
@@ -397,7 +402,8 @@ sb_status sb_radix_sort_u64(sb_ctx* ctx, unsigned long long* keys, unsigned long
         at[0].val.clusterDim.x = G; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
         cfg.attrs = at; cfg.numAttrs = 1;
         int nn = (int)n;
-        void* kargs[] = {&keys, &vals, &nn, (void*)&m};
+        SbDeviceState* ds = ctx->dstate;
+        void* kargs[] = {&keys, &vals, &nn, (void*)&m, &ds};
         if (cudaLaunchKernelExC(&cfg, kfn, kargs) == cudaSuccess) {
             SB_LAUNCHED(ctx);
             return SB_OK;

@@ -83,6 +83,8 @@ struct ScoreArgs {
     BitsArg ba;
     float* rec;                      // scores: partial block errors; statistics: partial column sums
     float* rowpart;                  // statistics: [strip][row] partial row sums
+    SbDeviceState* ds;               // status word; sizes of the two buffers in floats (checked build)
+    long long rec_limit, rowpart_limit;
 };
 
 // owner of slab s when stream w takes slabs [n_slabs * w / n_warps, n_slabs * (w + 1) / n_warps)
@@ -471,7 +473,8 @@ struct Scorer {
             v += __shfl_xor_sync(0xffffffffu, v, 16);
             tot[l] = v;
         }
-        if (slot2 == 0 && (cl % g.lanes_per_sub) == 0) {
+        if (slot2 == 0 && (cl % g.lanes_per_sub) == 0 &&
+            SB_IN_BOUNDS(a.ds, SBK_SCORES, ((long long)(q + gs) * g.nsub + cl / g.lanes_per_sub) * L + L - 1, a.rec_limit)) {
             float* dst = a.rec + ((size_t)(q + gs) * g.nsub + cl / g.lanes_per_sub) * L;
 #pragma unroll
             for (int l = 0; l < L; ++l) dst[l] = tot[l];
@@ -573,7 +576,9 @@ struct StatsScorer {
         }
         const float tot = rowsum[0] + __shfl_xor_sync(0xffffffffu, rowsum[0], 1);
         const int row = row0 + slot2 + 2 * (t >> 1);
-        if (a.rowpart && (t & 1) == 0 && row < g.n_rows) a.rowpart[(size_t)strip * g.br + row] = tot;
+        if (a.rowpart && (t & 1) == 0 && row < g.n_rows &&
+            SB_IN_BOUNDS(a.ds, SBK_STATS, (long long)strip * g.br + row, a.rowpart_limit))
+            a.rowpart[(size_t)strip * g.br + row] = tot;
     }
     // the stretch's column sums: c_j, the two half warps (different rows, the same columns), one
     // record of 128 floats
@@ -588,7 +593,8 @@ struct StatsScorer {
             out[2 * k] = a0 + __shfl_xor_sync(0xffffffffu, a0, 16);
             out[2 * k + 1] = a1 + __shfl_xor_sync(0xffffffffu, a1, 16);
         }
-        if (slot2 == 0 && a.rec) {
+        if (slot2 == 0 && a.rec &&
+            SB_IN_BOUNDS(a.ds, SBK_STATS, (long long)(q + gs) * TILE_COLS + cl * SC_CPL + SC_CPL - 1, a.rec_limit)) {
             float4* dst = reinterpret_cast<float4*>(a.rec + (size_t)(q + gs) * TILE_COLS + cl * SC_CPL);
             dst[0] = make_float4(out[0], out[1], out[2], out[3]);
             dst[1] = make_float4(out[4], out[5], out[6], out[7]);
@@ -732,11 +738,11 @@ template <int L, int RPL, int NFINE, bool FULLG, bool ROWW>
 sb_status launch_scores_k(sb_ctx* ctx, const CUtensorMap& wmap,
                           const int32_t* cperm, const int32_t* aperm, const float* cm, const float* rw,
                           const ScoreGeom& g, const BitsArg& ba, int64_t n_blocks, int64_t nbc, int grid,
-                          float* err, float* gain, float* rec) {
+                          float* err, float* gain, float* rec, long long rec_limit) {
     const size_t smem = 128 + SC_BAR_BYTES + (size_t)SC_STREAMS * g.ring * (SLAB_BYTES + g.rec_bytes);
     auto kern = block_scores_kernel<Scorer<L, RPL, NFINE, FULLG, ROWW>>;
     SB_FUNC_ATTR(ctx, kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM_MAX);   // one instance serves several group sizes
-    ScoreArgs pa{cperm, cm, ba, rec, nullptr};
+    ScoreArgs pa{cperm, cm, ba, rec, nullptr, ctx->dstate, rec_limit, 0};
     kern<<<(unsigned)grid, SC_THREADS, smem, ctx->stream>>>(wmap, aperm, rw, g, pa, ctx->dstate);
     SB_LAUNCHED(ctx);
     scores_finish_kernel<<<(unsigned)((n_blocks + 255) / 256), 256, 0, ctx->stream>>>(
@@ -887,7 +893,8 @@ sb_status sb_reorder_stats_slab(sb_ctx* ctx, const void* W, int64_t R, int64_t C
     sb_status st = weight_tile_map(ctx, static_cast<const __nv_bfloat16*>(W), R, C, ldw, &wmap);
     if (st != SB_OK) return st;
     const int one_bit[1] = {ref_bits};
-    ScoreArgs pa{nullptr, col_moment, make_bits(one_bit, 1), col_score ? col_rec : nullptr, row_score ? rowpart : nullptr};
+    ScoreArgs pa{nullptr, col_moment, make_bits(one_bit, 1), col_score ? col_rec : nullptr, row_score ? rowpart : nullptr,
+                 ctx->dstate, (long long)sb_stats_col_rec_floats(C, ctx->sm_count), (long long)sb_stats_rowpart_floats(R, C)};
     if (row_weight) st = nfine ? launch_stats<1, false, true>(ctx, wmap, row_weight, geo, pa, (int)grid)
                                : launch_stats<0, false, true>(ctx, wmap, row_weight, geo, pa, (int)grid);
     else if (fullg) st = nfine ? launch_stats<1, true, false>(ctx, wmap, nullptr, geo, pa, (int)grid)
@@ -972,7 +979,8 @@ extern "C" sb_status sb_block_scores(sb_ctx* ctx, const void* W, int64_t R, int6
     // up to four candidates: a lane takes two rows per step; more: one row (fewer accumulators)
 #define SB_SCORES(Lv, RPLv)                                                                        \
     st = launch_scores<Lv, RPLv>(nfine, group, row_weight, ctx, wmap, col_perm, row_perm, \
-                                 col_moment, row_weight, geo, ba, n_blocks, nbc, (int)grid, err, gain, rec)
+                                 col_moment, row_weight, geo, ba, n_blocks, nbc, (int)grid, err, gain, rec,        \
+                                 (long long)(rec_bytes / sizeof(float)))
     switch (n_bits) {
         case 1: SB_SCORES(1, 2); break;
         case 2: SB_SCORES(2, 2); break;

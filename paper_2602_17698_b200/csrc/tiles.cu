@@ -23,7 +23,7 @@ constexpr int GA_STAGES = 3;
 __global__ void __launch_bounds__(CTA_THREADS)
 gather_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int C, int64_t ldw,
               const int32_t* __restrict__ rp, const int32_t* __restrict__ cp,
-              __nv_bfloat16* __restrict__ out, int rows_per_cta) {
+              __nv_bfloat16* __restrict__ out, int rows_per_cta, SbDeviceState* ds) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const unsigned row_bytes = (unsigned)C * 2u;
     const int64_t r0 = (int64_t)blockIdx.x * rows_per_cta;
@@ -32,7 +32,9 @@ gather_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int C, int64_t ldw
     auto stage = [&](int rr, int st) {
         if (rr < nrows) {
             const int64_t r = r0 + rr;
-            const __nv_bfloat16* src = W + (rp ? (int64_t)rp[r] : r) * ldw;
+            int64_t rs = rp ? (int64_t)rp[r] : r;
+            if (!SB_IN_BOUNDS(ds, SBK_GATHER, rs, R)) rs = 0;          // a bad permutation entry reads row 0
+            const __nv_bfloat16* src = W + rs * ldw;
             unsigned char* dst = smem_raw + (unsigned)st * row_bytes;
             for (int j = j0; j < C; j += CTA_THREADS * 8) cp_async16(dst + 2 * j, src + j);
         }
@@ -50,8 +52,14 @@ gather_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int C, int64_t ldw
         for (int j = j0; j < C; j += CTA_THREADS * 8) {
             uint4 o;
             if (cp) {
-                const int4 p0 = __ldg(reinterpret_cast<const int4*>(cp + j));
-                const int4 p1 = __ldg(reinterpret_cast<const int4*>(cp + j + 4));
+                int4 p0 = __ldg(reinterpret_cast<const int4*>(cp + j));
+                int4 p1 = __ldg(reinterpret_cast<const int4*>(cp + j + 4));
+#ifdef SB_CHECKED
+                {
+                    int* pv[8] = {&p0.x, &p0.y, &p0.z, &p0.w, &p1.x, &p1.y, &p1.z, &p1.w};
+                    for (int k = 0; k < 8; ++k) if (!SB_IN_BOUNDS(ds, SBK_GATHER, *pv[k], C)) *pv[k] = 0;
+                }
+#endif
                 o.x = row[p0.x] | ((uint32_t)row[p0.y] << 16);
                 o.y = row[p0.z] | ((uint32_t)row[p0.w] << 16);
                 o.z = row[p1.x] | ((uint32_t)row[p1.y] << 16);
@@ -72,7 +80,7 @@ template <int NIT>
 __global__ void __launch_bounds__(CTA_THREADS)
 gather_cols_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int C, int64_t ldw,
                    const int32_t* __restrict__ rp, const int32_t* __restrict__ cp,
-                   __nv_bfloat16* __restrict__ out, int rows_per_cta) {
+                   __nv_bfloat16* __restrict__ out, int rows_per_cta, SbDeviceState* ds) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const unsigned row_bytes = (unsigned)C * 2u;
     const int64_t r0 = (int64_t)blockIdx.x * rows_per_cta;
@@ -86,6 +94,10 @@ gather_cols_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int C, int64_
         if (j < C) {
             p0 = __ldg(reinterpret_cast<const int4*>(cp + j));
             p1 = __ldg(reinterpret_cast<const int4*>(cp + j + 4));
+#ifdef SB_CHECKED
+            int* pv[8] = {&p0.x, &p0.y, &p0.z, &p0.w, &p1.x, &p1.y, &p1.z, &p1.w};
+            for (int k = 0; k < 8; ++k) if (!SB_IN_BOUNDS(ds, SBK_GATHER, *pv[k], C)) *pv[k] = 0;
+#endif
         }
         off2[it][0] = (uint32_t)(2 * p0.x) | ((uint32_t)(2 * p0.y) << 16);
         off2[it][1] = (uint32_t)(2 * p0.z) | ((uint32_t)(2 * p0.w) << 16);
@@ -95,7 +107,9 @@ gather_cols_kernel(const __nv_bfloat16* __restrict__ W, int64_t R, int C, int64_
     auto stage = [&](int rr, int st) {
         if (rr < nrows) {
             const int64_t r = r0 + rr;
-            const __nv_bfloat16* src = W + (rp ? (int64_t)rp[r] : r) * ldw;
+            int64_t rs = rp ? (int64_t)rp[r] : r;
+            if (!SB_IN_BOUNDS(ds, SBK_GATHER, rs, R)) rs = 0;          // a bad permutation entry reads row 0
+            const __nv_bfloat16* src = W + rs * ldw;
             unsigned char* dst = smem_raw + (unsigned)st * row_bytes;
             for (int j = j0; j < C; j += CTA_THREADS * 8) cp_async16(dst + 2 * j, src + j);
         }
@@ -390,12 +404,12 @@ sb_status sb_gather_bf16(sb_ctx* ctx, const void* W, int64_t R, int64_t C, int64
         SB_FUNC_ATTR(ctx, gather_cols_kernel<NIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
                      200 * 1024);                                                                    \
         gather_cols_kernel<NIT><<<grid, CTA_THREADS, smem, ctx->stream>>>(Wb, R, (int)C, ldw, rp, cp, ob, \
-                                                                          rows_per_cta);            \
+                                                                          rows_per_cta, ctx->dstate); \
     } while (0)
     if (cp && C <= 4096) SB_GATHER_COLS(2);
     else if (cp && C <= 8192) SB_GATHER_COLS(4);
     else if (cp && C <= 16384) SB_GATHER_COLS(8);
-    else gather_kernel<<<grid, CTA_THREADS, smem, ctx->stream>>>(Wb, R, (int)C, ldw, rp, cp, ob, rows_per_cta);
+    else gather_kernel<<<grid, CTA_THREADS, smem, ctx->stream>>>(Wb, R, (int)C, ldw, rp, cp, ob, rows_per_cta, ctx->dstate);
 #undef SB_GATHER_COLS
     SB_LAUNCHED(ctx);
     return SB_OK;
