@@ -4,66 +4,64 @@
 // for a few tokens t (decode batches) against a packed R x C matrix.  The codes are small
 // integers, exactly representable in bf16, so the contraction runs on the CODES:
 //     Y[t][r] = sum over column blocks j of  scale[r][j] * (sum_c X[t][c] q[r][c]) + lo[r][j] * (sum_c X[t][c])
-// with one tcgen05 contraction (M = 128 weight rows, N = tokens, K = the block's 128 columns,
-// bf16 x bf16 -> fp32) per 128 x 128 block, scaled per row in the drain; nothing is rounded
-// but the fp32 accumulation.  The packed codes are read once from HBM; what costs time is
-// turning them into operands, so the unpacking is kept to about 1.4 operations per code:
-// for b in {1, 2, 4, 8} a 32-bit word of codes is split by ONE mask per pair,
-//     (w >> (b s)) & (2^b - 1) * 0x00010001     ->  codes s and s + 16 / b of the word as two 16-bit halves,
-// which OR 0x4300 turns into the bf16 pair (128 + q_lo, 128 + q_hi); subtracting 128 is exact.
-// That visits the columns of a word in the order s, s + n/2, s + 1, ... (n = 32 / b); the
-// contraction does not care about the order of K as long as X uses the same one, so a small
-// kernel first writes X in each of those column orders (and the per-block column sums of X).
+// bf16 x bf16 -> fp32 per block, scaled per row when the block is done; nothing is rounded but
+// the fp32 accumulation.
 //
-// The unpacked codes never touch shared memory: bf16 codes are four times the packed bytes at
-// 4 bits, and writing them to a shared-memory operand tile and reading them back by the tensor
-// cores made shared-memory bandwidth the bound.  They go from registers to TENSOR MEMORY
-// (tcgen05.st, thread = weight row = TMEM lane) and the contraction takes its A operand from
-// there; only the few-token slice of X is a shared-memory operand.
+// The work is bound by the packed bytes (4 bits per weight on average against at most 32
+// tokens): what costs time is turning codes into tensor-core operands, so the design keeps that
+// path as short as it can be made.  A warp owns 16 weight rows of a block and feeds the tensor
+// cores from REGISTERS (mma.sync m16n8k16: weight rows on M, tokens on N): the unpacked codes are
+// the A fragment where the unpacking leaves them, with no trip through shared or tensor memory,
+// no second thread to hand them to and no accumulator to fetch back.  (A tcgen05 form of this
+// kernel, codes stored to tensor memory as the A operand of M = 128 instructions issued by one
+// thread, spent three times as many instructions per code on the hand-overs between its unpacking,
+// issuing and draining warps and ran at a third of the speed; the contraction itself is about a
+// microsecond of tensor work on any path.)
 //
-// Grid: (R / 128 row tiles) x (S column segments), two CTAs per SM.  Per CTA:
-//   warp 13 (one thread): per block two bulk copies (cp.async.bulk, mbarrier complete_tx) into a
-//     four-stage ring, three blocks ahead: the block's packed codes as they lie in memory, and its
-//     slice of X, which the preparation kernel has already laid out as the K-major
-//     128-byte-swizzle operand image;
-//   warps 4-11 (thread = 2 x 32 columns of a weight row): unpack the block into registers,
-//     tcgen05.st into one of three 64-column TMEM operand buffers, tcgen05.wait::st, fences,
-//     mbarrier arrives (operand ready; code stage free);
-//   warp 12 (one thread): 8 tcgen05.mma (K = 16, A from TMEM, B = X slice from shared memory) per
-//     block into one of two TMEM accumulators of N columns, one tcgen05.commit per block, which
-//     frees the operand buffer and the X slice and publishes the accumulator;
-//   warps 0-3 (thread = weight row = TMEM lane): tcgen05.ld of the block's accumulator,
-//     y += scale * acc + lo * colsum(X) in fp32 registers; at the end the segment's partial
-//     sums go to scratch (or to Y when there is one segment) and a second kernel adds the
-//     segments in order.
-// Every mbarrier wait is bounded; on a time-out the kernel latches SB_ERR_TIMEOUT and all
-// roles leave.
+// Unpacking, about one operation per code: lane (g, t) of a warp holds the 32 codes 32 t .. 32 t + 31
+// of rows g and g + 8.  For b in {1, 2, 4} a 32-bit word of codes is split by one shift and one
+// mask-and-or per PAIR,
+//     ((w >> (b s - (7 - b))) & MASK) | 0x43004300  ->  bf16 pair (128 + 2^(7-b) q_s, 128 + 2^(7-b) q_(s + 16/b)):
+// the code lands in the top bits of the bf16 mantissa under the exponent of 128.  The offset and
+// the power of two are taken out again when the block is scaled (they fold into scale and lo), so
+// no subtraction is spent per code.  Codes of 8 bits go through as two 4-bit fields each against
+// X and 16 X (a block of 256 columns to the tensor cores); 3, 5, 6 and 7 bits are cut out of the
+// bit stream one by one.  The contraction does not care in which order it visits the columns of
+// a block as long as X uses the same one, so a small kernel first writes X in the column order
+// each unpacking produces (and the per-block column sums of X).
+//
+// Grid: (R / block_rows row tiles) x (S column segments); block_rows / 16 contraction warps and a
+// loader warp per CTA, two (128-row blocks) or three (64-row blocks) CTAs per SM.  The loader
+// thread brings each block in with two bulk copies (cp.async.bulk, mbarrier complete_tx) into a
+// ring of three or four stages: the block's packed codes as they lie in memory, and its slice of
+// X, which the preparation kernel has laid out as the image ldmatrix reads without bank
+// conflicts.  Each warp: wait for the stage, read its rows' codes (one to seven loads), eight or
+// sixteen steps of {unpack four registers, ldmatrix the tokens' fragments, one mma.sync per eight
+// tokens}, release the stage, then y += scale' * acc + lo' * colsum(X) in fp32 registers.  The
+// segment's partial sums go to scratch (or to Y when there is one segment) and a second kernel
+// adds the segments in order.  Every mbarrier wait is bounded; on a time-out the kernel latches
+// SB_ERR_TIMEOUT and all roles leave.
 #include "common.cuh"
 
 namespace {
 
-constexpr int DQ_M = 128;                   // weight rows per CTA = block rows
-constexpr int DQ_KB = 128;                  // block columns
-constexpr int DQ_RING = 4;                  // blocks in flight (codes + X slice)
-constexpr int DQ_CODE_STAGE = 2048 * 8;     // bytes of codes of one block at 8 bits
-constexpr int DQ_A_COLS = DQ_KB / 2;         // TMEM columns of a block's codes: two bf16 per 32-bit column
-constexpr int DQ_ABUF = 3;                  // TMEM operand buffers: the unpackers run up to two blocks ahead of the contraction
-constexpr int DQ_MAX_T = 32;
-constexpr int DQ_X_STAGE = DQ_MAX_T * DQ_KB * 2;        // X slice of a block: tokens x 128 bf16
-constexpr int DQ_CONV_WARPS = 8, DQ_EPI_WARPS = 4;    // unpacking thread = 32 columns of a weight row
-constexpr int DQ_THREADS = (DQ_EPI_WARPS + DQ_CONV_WARPS + 2) * 32;   // + MMA warp + loader warp
+constexpr int DQ_KB = 128;                  // block columns = quantisation group
+constexpr int DQ_MAX_T = 32;                // tokens per pass
+#ifdef SB_EXP_C3
+constexpr int DQ_MAX_SEG_BLOCKS = 16;
+#else
 constexpr int DQ_MAX_SEG_BLOCKS = 32;       // column blocks per segment (their column sums sit in shared memory)
-constexpr int DQ_ORDERS = 5;                // column orders of X: identity, b = 1, 2, 4, 8
-constexpr int DQ_SMEM = DQ_RING * (DQ_CODE_STAGE + DQ_X_STAGE) + DQ_MAX_SEG_BLOCKS * DQ_MAX_T * 4 +
-                        1024 /* alignment */ + 512 /* barriers, block table */;
-constexpr int DQ_TMEM_COLS = 256;           // accumulators in columns [0, 64), operand buffers at 64, 128 and 192
+#endif
+constexpr int DQ_ORDERS = 5;                // column orders of X: one by one, b = 1, 2, 4, and 8 as two nibbles
 constexpr unsigned long long DQ_WAIT_NS = 2000ull * 1000 * 1000;
 
 // candidate bitwidths, four bits each
 struct DqBits { unsigned packed; };
 __device__ __forceinline__ int dq_bits(DqBits b, int l) { return (int)((b.packed >> (4 * l)) & 15u); }
-// column order of X that the unpacking of b-bit codes produces
+// column order of X that the unpacking of b-bit codes produces, and the columns its image has
 __host__ __device__ inline int dq_order(int b) { return b == 1 ? 1 : b == 2 ? 2 : b == 4 ? 3 : b == 8 ? 4 : 0; }
+// first element of order o's images: nbc images of NT x 128 per order
+__host__ __device__ inline int64_t dq_order_base(int o, int64_t nbc, int NT) { return (int64_t)o * nbc * NT * DQ_KB; }
 
 __device__ __forceinline__ unsigned dq_smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ unsigned long long dq_now_ns() {
@@ -77,28 +75,34 @@ __device__ __forceinline__ void dq_mbar_init(unsigned bar, unsigned count) {
 __device__ __forceinline__ void dq_mbar_arrive(unsigned bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ bool dq_mbar_try_wait(unsigned bar, unsigned parity) {
+// one try: the thread may sleep inside the instruction for up to hint_ns before it answers
+__device__ __forceinline__ bool dq_mbar_try_wait(unsigned bar, unsigned parity, unsigned hint_ns = 2000u) {
     unsigned ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool dq_mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
+__device__ __noinline__ bool dq_mbar_wait_slow(unsigned bar, unsigned parity, volatile int* abort_flag) {
     unsigned long long t0 = 0;
     for (unsigned spins = 0;; ++spins) {
         if (dq_mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if ((spins & 255u) == 255u) {
+        if ((spins & 15u) == 15u) {
             const unsigned long long now = dq_now_ns();
             if (t0 == 0) t0 = now;
             else if (now - t0 > DQ_WAIT_NS) { *abort_flag = 1; return false; }
         }
     }
+}
+// bounded wait: the first try is inline, the rest (with the clock and the abort flag) out of line
+__device__ __forceinline__ bool dq_mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
+    if (dq_mbar_try_wait(bar, parity)) return true;
+    return dq_mbar_wait_slow(bar, parity, abort_flag);
 }
 __device__ __forceinline__ void dq_mbar_expect_tx(unsigned bar, unsigned bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -109,162 +113,260 @@ __device__ __forceinline__ void dq_bulk_load(unsigned dst, const void* src, unsi
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+__device__ __forceinline__ uint32_t dq_lds32(unsigned addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint2 dq_lds64(unsigned addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint4 dq_lds128(unsigned addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+// four 8 x 8 matrices of 16-bit elements: lane L gives the address of row L % 8 of matrix L / 8
+// and receives elements 2 (L % 4), 2 (L % 4) + 1 of row L / 4 of each matrix
+__device__ __forceinline__ void dq_ldmatrix4(unsigned addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D (16 weight rows x 8 tokens, fp32) = or += A (16 x 16 codes, from registers) * B (16 x 8, X)
+__device__ __forceinline__ void dq_mma(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1, bool first) {
+    if (first) {
+        asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+            "{%10, %10, %10, %10};"
+            : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+            : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+    } else {
+        asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+            "{%0, %1, %2, %3};"
+            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+            : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    }
+}
 
-// K-major operand in the 128-byte-swizzle layout: rows of 128 bytes (64 bf16 along K), 8-row
-// groups 1024 bytes apart; the leading offset is not used by swizzled K-major layouts
-__device__ __forceinline__ unsigned long long dq_desc(unsigned addr) {
-    unsigned long long d = 0;
-    d |= (unsigned long long)((addr >> 4) & 0x3fffu);
-    d |= 1ull << 16;
-    d |= (unsigned long long)((1024 >> 4) & 0x3fff) << 32;
-    d |= 1ull << 46;
-    d |= 2ull << 61;
-    return d;
-}
-// fp32 accumulator, bf16 x bf16, both operands K-major, M = 128, N = n
-__device__ __forceinline__ unsigned dq_idesc(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(DQ_M >> 4) << 24);
-}
-// A (128 rows x 16 columns of bf16 = 8 TMEM columns, row = lane) from tensor memory, B from shared memory
-__device__ __forceinline__ void dq_mma(unsigned tmem_d, unsigned tmem_a, unsigned long long b, unsigned idesc,
-                                       unsigned acc) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "r"(tmem_a), "l"(b), "r"(idesc), "r"(acc)
-        : "memory");
-}
-__device__ __forceinline__ void dq_tmem_st16(unsigned taddr, const uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
-        : "memory");
-}
-__device__ __forceinline__ void dq_commit(unsigned bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void dq_tmem_ld16(unsigned taddr, float (&v)[16]) {
-    unsigned r[16];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int k = 0; k < 16; ++k) v[k] = __uint_as_float(r[k]);
+// ---- the column order of each unpacking ------------------------------------------------------
+// Position p of a block's image = 16 (step) + kappa, kappa = the column index inside one
+// m16n8k16: lane t of a quad holds kappa = 2 t, 2 t + 1 (first A register of a row, low and high
+// half) and 2 t + 8, 2 t + 9 (second register).  Register i = 2 step + (kappa >> 3) of lane t is
+// pair i of that lane's unpacking.  Returns the block column (0..127) that position p holds.
+__host__ __device__ inline int dq_source(int o, int p) {
+    const int step = p >> 4, kap = p & 15;
+    const int t = (kap & 7) >> 1, half = kap & 1, i = 2 * step + (kap >> 3);
+    int col;
+    if (o == 0) {
+        col = 32 * t + 2 * i + half;                       // codes cut out one by one: pair i = codes 2 i, 2 i + 1
+    } else if (o <= 3) {
+        const int b = 1 << (o - 1), n = 32 / b, hp = n / 2; // pair (m, s) of word m: fields s and s + n / 2
+        const int m = i / hp, s = i % hp;
+        col = 32 * t + n * m + s + hp * half;
+    } else {
+        // 8 bits: the lane's words are chunk t (codes 16 t ..) and chunk t + 4 (codes 64 + 16 t ..) of the row;
+        // pair i = bytes beta and beta + 2 of word i / 2 (beta = i % 2), whose low and high nibbles go
+        // through as two registers against the same columns of X
+        const int vw = i >> 1, beta = i & 1;
+        col = 16 * (vw < 4 ? t : t + 4) + 4 * (vw & 3) + beta + 2 * half;
+    }
+    return col;
 }
 
 // ---- X in the column orders of the unpacking, and its per-block column sums ------------------
-// order o > 0 (codes of b bits, n = 32 / b per word): position n m + 2 s + h holds column
-// n m + s + (n / 2) h.  xp: [DQ_ORDERS][C / 128] images of T x 128 bf16, each laid out as the
-// shared-memory operand (two K halves of T rows x 128 bytes, 16-byte chunks XOR-swizzled with the
-// row), so that one contiguous copy brings a block's slice in; xsum: [C / 128][T] fp32.
-__device__ __forceinline__ int dq_image_index(int T, int t, int p) {
-    const int panel = p >> 6, pp = p & 63;
-    return panel * (T * 64) + t * 64 + (((pp >> 3) ^ (t & 7)) << 3) + (pp & 7);
+// xp: per order and column block an image of NT rows (tokens) x 128 bf16, laid out as the
+// contraction warps read it: 16-byte chunks of a row XOR-swizzled with the token index so that
+// the eight rows of an ldmatrix hit different banks; one contiguous copy brings a block's slice
+// in.  xsum: [C / 128][NT] fp32.
+__device__ __forceinline__ int dq_image_index(int n, int p) {
+    return n * DQ_KB + ((((p >> 3) ^ (n & 7))) << 3) + (p & 7);
 }
-__global__ void dq_prepare_x_kernel(const __nv_bfloat16* __restrict__ X, int64_t ldx, int T, int64_t nbc,
-                                    __nv_bfloat16* __restrict__ xp, float* __restrict__ xsum) {
+__global__ void __launch_bounds__(DQ_KB)
+dq_prepare_x_kernel(const __nv_bfloat16* __restrict__ X, int64_t ldx, int NT, int64_t nbc,
+                    __nv_bfloat16* __restrict__ xp, float* __restrict__ xsum) {
     const int64_t jb = blockIdx.x;                       // column block
-    const int t = blockIdx.y;
-    const int p = threadIdx.x;                           // position inside the block, 0..127
-    const __nv_bfloat16* xrow = X + (int64_t)t * ldx + jb * DQ_KB;
-    const float v = __bfloat162float(xrow[p]);
+    const int n = blockIdx.y;                            // token
+    const int p = threadIdx.x;                           // position inside an image row, 0..127
+    const __nv_bfloat16* xrow = X + (int64_t)n * ldx + jb * DQ_KB;
     // column sum of the block in a fixed order: pairwise inside the warp, then the four warps
     __shared__ float ws[4];
-    const float s = warp_sum(v);
+    const float s = warp_sum(__bfloat162float(xrow[p]));
     if ((p & 31) == 0) ws[p >> 5] = s;
     __syncthreads();
-    if (p == 0) xsum[jb * T + t] = (ws[0] + ws[1]) + (ws[2] + ws[3]);
-    const int64_t image = (int64_t)T * DQ_KB;
-    __nv_bfloat16* out = xp + jb * image + dq_image_index(T, t, p);
-    out[0] = xrow[p];
+    if (p == 0) xsum[jb * NT + n] = (ws[0] + ws[1]) + (ws[2] + ws[3]);
+    const int64_t image = (int64_t)NT * DQ_KB;
 #pragma unroll
-    for (int o = 1; o < DQ_ORDERS; ++o) {
-        const int n = 32 >> (o - 1);                     // codes per word: 32, 16, 8, 4
-        const int m = p / n, w = p % n, s2 = w >> 1, h = w & 1;
-        out[(int64_t)o * nbc * image] = xrow[n * m + s2 + (n >> 1) * h];
-    }
+    for (int o = 0; o < DQ_ORDERS; ++o)
+        xp[dq_order_base(o, nbc, NT) + jb * image + dq_image_index(n, p)] = xrow[dq_source(o, p)];
 }
 
 // ---- unpacking ---------------------------------------------------------------------------------
-// 32 codes (B words) of one weight row, b in {1, 2, 4, 8}, from shared memory into 16 registers of
-// bf16 pairs.  `src` points at the row's codes (16 B bytes), `qi` = which 32 codes of the row (0..3).
+// Pair i of a row's codes held by this lane (w: the lane's words of the row) as two bf16
+// 128 + 2^(7-B) q in one register.
+// (x & mask) | c in one instruction; mask and c come in registers so that neither is split off
+__device__ __forceinline__ uint32_t dq_and_or(uint32_t x, uint32_t mask, uint32_t c) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(x), "r"(mask), "r"(c));
+    return d;
+}
 template <int B>
-__device__ __forceinline__ void dq_unpack32(const unsigned char* src, int qi, uint32_t (&out)[16]) {
-    constexpr int N = 32 / B;                            // codes per word
-    constexpr unsigned MASK = ((1u << B) - 1u) * 0x00010001u;
-    const __nv_bfloat162 c128 = __float2bfloat162_rn(128.f);
-    uint32_t w[B];
-    if constexpr (B == 1) {
-        w[0] = *reinterpret_cast<const uint32_t*>(src + 4 * qi);
+__device__ __forceinline__ uint32_t dq_pair(const uint32_t* w, int i, uint32_t mask, uint32_t c43) {
+    if constexpr (B == 1 || B == 2 || B == 4 || B == 8) {
+        // 8 bits: "pair" 2 i' + h is the low (h = 0) or high (h = 1) nibbles of bytes beta, beta + 2 of
+        // word i' / 2 (beta = i' % 2), i.e. nibbles s and s + 4 of the word with s = 2 beta + h: the same
+        // arithmetic as 4-bit fields, the caller passes 128's exponent for the low and 2048's for the high nibbles
+        constexpr int F = B == 8 ? 4 : B;                   // field width
+        constexpr int HP = 16 / F;                          // pairs per word
+        constexpr int P = 7 - F;                            // the field's lowest bit inside the bf16 mantissa
+        const int m = i / HP, s = i % HP;
+        const int sh = F * s - P;
+        const uint32_t v = sh >= 0 ? (w[m] >> (sh & 31)) : (w[m] << ((-sh) & 31));
+        return dq_and_or(v, mask, c43);
+    } else {
+        // codes 2 i and 2 i + 1 of the lane's 32, code k at bit k B of the lane's B words
+        constexpr int P = 7 - B;
+        constexpr uint32_t M1 = (1u << B) - 1u;
+        uint32_t out = 0x43004300u;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int bit = (2 * i + h) * B, wi = bit >> 5, off = bit & 31;
+            uint32_t e;
+            if (off + B <= 32) e = w[wi] >> off;
+            else e = __funnelshift_r(w[wi], w[wi + 1], off);
+            out |= (e & M1) << (P + 16 * h);
+        }
+        return out;
+    }
+}
+// the mask of dq_pair's fields for B bits, kept in a register across the block
+template <int B>
+__device__ __forceinline__ uint32_t dq_pair_mask() {
+    constexpr int F = B == 8 ? 4 : B;
+    constexpr int P = 7 - F;
+    return (((1u << F) - 1u) << P) * 0x00010001u;
+}
+
+// The lane's words of one weight row.  rowaddr: shared address of the row's codes (16 B bytes);
+// t: the lane's place in its quad.
+template <int B>
+__device__ __forceinline__ void dq_load_row(unsigned rowaddr, int t, uint32_t* w) {
+    if constexpr (B == 8) {
+        const uint4 a = dq_lds128(rowaddr + 16 * t), b = dq_lds128(rowaddr + 64 + 16 * t);
+        w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w; w[4] = b.x; w[5] = b.y; w[6] = b.z; w[7] = b.w;
+    } else if constexpr (B == 4) {
+        const uint4 a = dq_lds128(rowaddr + 16 * t);
+        w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w;
     } else if constexpr (B == 2) {
-        const uint2 v = *reinterpret_cast<const uint2*>(src + 8 * qi);
-        w[0] = v.x; w[1] = v.y;
+        const uint2 a = dq_lds64(rowaddr + 8 * t);
+        w[0] = a.x; w[1] = a.y;
     } else {
 #pragma unroll
-        for (int k = 0; k < B / 4; ++k) {
-            const int chunk = qi * (B / 4) + k;          // 16-byte chunk of the row
-            const uint4 v = *reinterpret_cast<const uint4*>(src + (chunk << 4));
-            w[4 * k] = v.x; w[4 * k + 1] = v.y; w[4 * k + 2] = v.z; w[4 * k + 3] = v.w;
-        }
-    }
-#pragma unroll
-    for (int m = 0; m < B; ++m) {
-#pragma unroll
-        for (int s = 0; s < N / 2; ++s) {
-            const uint32_t v = (w[m] >> (B * s)) & MASK;
-            uint32_t bits;
-            if constexpr (B < 8) {
-                bits = u32(__hsub2(b162(v | 0x43004300u), c128));
-            } else {
-                // 8 significant bits: the low seven through the exponent trick, the top one added
-                const __nv_bfloat162 lo7 = __hsub2(b162((v & 0x007f007fu) | 0x43004300u), c128);
-                const uint32_t top = ((v >> 7) & 0x00010001u) * 0x4300u;     // 128.0 or 0 per half
-                bits = u32(__hadd2(lo7, b162(top)));
-            }
-            out[(N / 2) * m + s] = bits;
-        }
+        for (int k = 0; k < B; ++k) w[k] = dq_lds32(rowaddr + 4 * B * t + 4 * k);
     }
 }
 
-// any other bitwidth below 8: code k of the row at bit k b of its stream, columns in their own order
-__device__ __forceinline__ void dq_unpack32_generic(const unsigned char* src, int b, int qi, uint32_t (&out)[16]) {
-    const uint32_t* words = reinterpret_cast<const uint32_t*>(src);
-    const uint32_t mask = (1u << b) - 1u;
-    const __nv_bfloat162 c128 = __float2bfloat162_rn(128.f);
+// One block for one warp: acc[nt][.] = sum over the block's columns of codes x X for the warp's
+// 16 rows and tokens 8 nt .. 8 nt + 7.  codes: shared address of the warp's first row in the
+// stage; xlane: the lane's ldmatrix row address(es) in the stage's image, before the step is
+// XOR-ed in.
+template <int B, int NT>
+__device__ __forceinline__ void dq_block(unsigned codes, const unsigned (&xlane)[2], int g, int t,
+                                         unsigned empty_bar, int lane, float2 c0, float2 c1, unsigned xs_addr,
+                                         float (&y)[NT / 8][4]) {
+    float acc[NT / 8][4];
+    constexpr int VW = B == 8 ? 8 : B;
+    constexpr int STEPS = 8;
+    constexpr int SUB = B == 8 ? 2 : 1;         // 8 bits: low and high nibbles against the same columns of X
+    uint32_t w0[VW], w1[VW];
+    dq_load_row<B>(codes + (unsigned)(g * 16 * B), t, w0);
+    dq_load_row<B>(codes + (unsigned)((g + 8) * 16 * B), t, w1);
+    // the constants of the unpacking live in registers (an immediate would split the operation in
+    // two): the field mask and the exponent under which the field sits, 128 (x 16 for high nibbles)
+    uint32_t mask = dq_pair_mask<B>(), c43 = 0x43004300u, c45 = 0x45004500u;
+    asm volatile("" : "+r"(mask), "+r"(c43), "+r"(c45));
+    // registers 2 ks and 2 ks + 1 of step ks (8 bits: of its low, then of its high nibbles)
+    auto a_regs = [&](int ks, int sub, uint32_t (&a)[4]) {
+        const int i0 = SUB * (2 * ks) + sub, i1 = SUB * (2 * ks + 1) + sub;
+        const uint32_t c = sub ? c45 : c43;
+        a[0] = dq_pair<B>(w0, i0, mask, c);
+        a[1] = dq_pair<B>(w1, i0, mask, c);
+        a[2] = dq_pair<B>(w0, i1, mask, c);
+        a[3] = dq_pair<B>(w1, i1, mask, c);
+    };
+    if constexpr (NT == 8) {
+        // one ldmatrix brings the fragments of two steps; the next pair of steps is fetched a pair ahead
+        uint32_t bf[2][4];
+        dq_ldmatrix4(xlane[0], bf[0]);
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+        for (int ks = 0; ks < STEPS; ++ks) {
+            if ((ks & 1) == 0 && ks + 2 < STEPS) dq_ldmatrix4(xlane[0] ^ (unsigned)((ks + 2) << 5), bf[((ks >> 1) + 1) & 1]);
+            const uint32_t(&cur)[4] = bf[(ks >> 1) & 1];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            uint32_t pair = 0;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int bit = (32 * qi + 8 * c + 2 * k + h) * b;
-                const int wi = bit >> 5;
-                // the row's stream is 4 b words long; the funnel shift may look one word past a code
-                // that ends at the stream's end, so that word is clamped to the last one
-                const uint32_t w0 = words[wi], w1 = words[min(wi + 1, 4 * b - 1)];
-                pair |= (__funnelshift_r(w0, w1, bit & 31) & mask) << (16 * h);
+            for (int sub = 0; sub < SUB; ++sub) {
+                uint32_t a[4];
+                a_regs(ks, sub, a);
+                dq_mma(acc[0], a, cur[2 * (ks & 1)], cur[2 * (ks & 1) + 1], ks == 0 && sub == 0);
             }
-            out[4 * c + k] = u32(__hsub2(b162(pair | 0x43004300u), c128));
+        }
+    } else {
+        // the tokens' fragments of step ks + 1 are fetched before the products of step ks are issued
+        constexpr int NQ = NT / 16;
+        uint32_t bf[2][NQ][4];
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) dq_ldmatrix4(xlane[q], bf[0][q]);
+#pragma unroll
+        for (int ks = 0; ks < STEPS; ++ks) {
+            if (ks + 1 < STEPS) {
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) dq_ldmatrix4(xlane[q] ^ (unsigned)((ks + 1) << 5), bf[(ks + 1) & 1][q]);
+            }
+#pragma unroll
+            for (int sub = 0; sub < SUB; ++sub) {
+                uint32_t a[4];
+                a_regs(ks, sub, a);
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    dq_mma(acc[2 * q], a, bf[ks & 1][q][0], bf[ks & 1][q][1], ks == 0 && sub == 0);
+                    dq_mma(acc[2 * q + 1], a, bf[ks & 1][q][2], bf[ks & 1][q][3], ks == 0 && sub == 0);
+                }
+            }
         }
     }
+    __syncwarp();
+    if (lane == 0) dq_mbar_arrive(empty_bar);            // codes and image are in registers
+    // codes went in as 128 + 2^P q (P = 7 - B; 8 bits: two nibbles with P = 3 against X and 16 X,
+    // offset 128 * 17): sum_c x q = (acc - OFF colsum) / 2^P, folded into the row's scale and minimum
+    constexpr float INV = B == 8 ? 0.125f : 1.f / (float)(1 << (7 - B));
+    constexpr float OFF = B == 8 ? 2176.f : 128.f;
+    const float s0 = c0.x * INV, s1 = c1.x * INV;
+    const float l0 = fmaf(-s0, OFF, c0.y), l1 = fmaf(-s1, OFF, c1.y);
+#pragma unroll
+    for (int nt = 0; nt < NT / 8; ++nt) {
+        const uint2 cu = dq_lds64(xs_addr + 32 * nt);
+        const float cx = __uint_as_float(cu.x), cy = __uint_as_float(cu.y);
+        y[nt][0] = fmaf(s0, acc[nt][0], fmaf(l0, cx, y[nt][0]));
+        y[nt][1] = fmaf(s0, acc[nt][1], fmaf(l0, cy, y[nt][1]));
+        y[nt][2] = fmaf(s1, acc[nt][2], fmaf(l1, cx, y[nt][2]));
+        y[nt][3] = fmaf(s1, acc[nt][3], fmaf(l1, cy, y[nt][3]));
+    }
 }
+
+#ifdef SB_EXP_TL
+__device__ long long dq_tl[9][40][4];
+__device__ unsigned long long dq_cta[512][4];
+#define DQ_TL(w, j, k) do { if (blockIdx.x == 3 && blockIdx.y == 1 && lane == 0 && (j) < 40) dq_tl[w][j][k] = clock64(); } while (0)
+#else
+#define DQ_TL(w, j, k) do { } while (0)
+#endif
 
 struct DqArgs {
     const uint32_t* packed;
     const int64_t* block_off;       // [nb + 1], words
     const float2* meta;             // [(r * nbc + j)] = (scale, lo), group == block width
     const uint8_t* level;           // [nb]
-    const __nv_bfloat16* xp;        // [DQ_ORDERS][nbc] operand images of T x 128
-    const float* xsum;              // [nbc][T]
+    const __nv_bfloat16* xp;        // per order, per column block: image of NT x 128 (256 for 8 bits)
+    const float* xsum;              // [nbc][NT]
     float* out;                     // partial sums [S][T][R] (or Y when S == 1)
     int64_t out_t_stride;           // R for the partial sums, ldy for Y
     int64_t out_seg_stride;
@@ -274,190 +376,169 @@ struct DqArgs {
     SbDeviceState* ds;
 };
 
-template <int NT>
-__global__ void __launch_bounds__(DQ_THREADS, 2) dequant_gemm_kernel(const DqArgs a) {
+template <int NT, int WARPS> struct DqShape {
+    static constexpr int ROWS = 16 * WARPS;                         // block rows
+    static constexpr int X_STAGE = NT * DQ_KB * 2;                  // an image: NT x 128 bf16
+    static constexpr int CODE_STAGE = ROWS * 16 * 8;                // a block's codes at 8 bits
+    static constexpr int STAGE = X_STAGE + CODE_STAGE;
+#ifdef SB_EXP_C3
+    static constexpr int RING = 3;
+#else
+    static constexpr int RING = 4;
+#endif
+    static constexpr int THREADS = (WARPS + 1) * 32;                // + loader warp
+    static constexpr int SMEM = RING * STAGE + DQ_MAX_SEG_BLOCKS * NT * 4 + 256 /* alignment */ +
+                                256 /* barriers, block table */;
+    // resident CTAs per SM by shared memory (227 KB, 1 KB reserved per CTA), at most four
+    static constexpr int FIT = (227 * 1024) / (SMEM + 1024);
+    static constexpr int CTAS_PER_SM = FIT > 4 ? 4 : FIT;
+};
+
+template <int NT, int WARPS>
+__global__ void __launch_bounds__(DqShape<NT, WARPS>::THREADS, DqShape<NT, WARPS>::CTAS_PER_SM)
+dequant_gemm_kernel(const DqArgs a) {
+    using S = DqShape<NT, WARPS>;
+    constexpr int RING = S::RING;
     extern __shared__ unsigned char dq_smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>(
-        (reinterpret_cast<uintptr_t>(dq_smem_raw) + 1023) & ~uintptr_t(1023));
-    unsigned char* x_ring = smem;                                         // DQ_RING x 8 KB slices of X
-    unsigned char* code_ring = x_ring + DQ_RING * DQ_X_STAGE;             // DQ_RING x 16 KB packed codes
-    float* xs = reinterpret_cast<float*>(code_ring + DQ_RING * DQ_CODE_STAGE);   // [seg_blocks][NT] column sums
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(xs + DQ_MAX_SEG_BLOCKS * DQ_MAX_T);
-    unsigned long long* a_full = bars;              // [DQ_ABUF] unpackers (TMEM operand buffer written) -> MMA
-    // [DQ_RING] the contraction of block j is complete (one commit per block, at j % DQ_RING): the
-    // drain may read its accumulator, the unpackers may rewrite the operand buffer two blocks
-    // later, the loader may refill the stage DQ_RING blocks later
-    unsigned long long* done = bars + DQ_ABUF;
-    unsigned long long* d_empty = done + DQ_RING;          // [2] drained -> MMA
-    unsigned long long* ld_full = d_empty + 2;             // [DQ_RING] both copies of a block landed
-    unsigned long long* code_empty = ld_full + DQ_RING;    // [DQ_RING] all unpackers have read the codes -> loader
-    unsigned* tmem_slot = reinterpret_cast<unsigned*>(code_empty + DQ_RING);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    // stage s: the block's image of X (256-byte aligned in the shared window: the swizzle is an XOR
+    // on the address bits below a row's 256 bytes), then its codes
+    unsigned char* smem = dq_smem_raw + ((256u - (dq_smem_u32(dq_smem_raw) & 255u)) & 255u);
+    float* xs = reinterpret_cast<float*>(smem + RING * S::STAGE);           // [seg_blocks][NT] column sums
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(xs + DQ_MAX_SEG_BLOCKS * NT);
+    unsigned long long* full = bars;                    // [RING] both copies of a block landed
+    unsigned long long* empty = bars + RING;            // [RING] every contraction warp has read the stage
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + RING);
     // per block of the segment: first word of its codes (blocks are below 2^32 words apart from the
     // segment's first) and its bitwidth, so that the loop below has no dependent global loads
-    unsigned* blk_word = tmem_slot + 4;                 // [DQ_MAX_SEG_BLOCKS]
-    unsigned char* blk_bits = reinterpret_cast<unsigned char*>(blk_word + DQ_MAX_SEG_BLOCKS);   // [DQ_MAX_SEG_BLOCKS]
+    unsigned* blk_word = reinterpret_cast<unsigned*>(const_cast<int*>(abort_flag) + 4);   // [DQ_MAX_SEG_BLOCKS]
+    unsigned char* blk_bits = reinterpret_cast<unsigned char*>(blk_word + DQ_MAX_SEG_BLOCKS);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr int TMEM_COLS = DQ_TMEM_COLS;
-    static_assert(2 * NT <= 64, "accumulators below the operand buffers");
+#ifdef SB_EXP_TL
+    if (threadIdx.x == 0) {
+        unsigned smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        dq_cta[blockIdx.y * gridDim.x + blockIdx.x][0] = dq_now_ns();
+        dq_cta[blockIdx.y * gridDim.x + blockIdx.x][2] = smid;
+    }
+#endif
 
     const int bi = blockIdx.x;                                  // row tile
     const int j0 = blockIdx.y * a.seg_blocks;                   // first column block of the segment
     const int nblk = min(a.seg_blocks, a.nbc - j0);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < 2; ++s) {
-            dq_mbar_init(dq_smem_u32(d_empty + s), DQ_EPI_WARPS);
-        }
-        for (int s = 0; s < DQ_ABUF; ++s) dq_mbar_init(dq_smem_u32(a_full + s), DQ_CONV_WARPS * 32);
-        for (int s = 0; s < DQ_RING; ++s) {
-            dq_mbar_init(dq_smem_u32(done + s), 1);
-            dq_mbar_init(dq_smem_u32(ld_full + s), 1);
-            dq_mbar_init(dq_smem_u32(code_empty + s), DQ_CONV_WARPS * 32);
+        for (int s = 0; s < RING; ++s) {
+            dq_mbar_init(dq_smem_u32(full + s), 1);
+            dq_mbar_init(dq_smem_u32(empty + s), WARPS);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == DQ_EPI_WARPS + DQ_CONV_WARPS) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dq_smem_u32(tmem_slot)),
-                     "r"(TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
     // the segment's column sums of X and its block table
-    for (int i = threadIdx.x; i < nblk * NT; i += DQ_THREADS) xs[i] = a.xsum[(int64_t)j0 * NT + i];
+    for (int i = threadIdx.x; i < nblk * NT; i += S::THREADS) xs[i] = a.xsum[(int64_t)j0 * NT + i];
     const int64_t blk0 = (int64_t)bi * a.nbc + j0;
     const int64_t word0 = a.block_off[blk0];
     if (threadIdx.x < nblk) {
         blk_word[threadIdx.x] = (unsigned)(a.block_off[blk0 + threadIdx.x] - word0);
         blk_bits[threadIdx.x] = (unsigned char)dq_bits(a.bits, a.level[blk0 + threadIdx.x]);
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const unsigned tmem_base = *tmem_slot;
 
-    if (warp >= DQ_EPI_WARPS && warp < DQ_EPI_WARPS + DQ_CONV_WARPS) {
-        // ---- unpackers: thread = columns 32 hq ... and 64 + 32 hq ... of weight row r of the tile ------
-        const int ct = threadIdx.x - DQ_EPI_WARPS * 32;
-        const int r = ct & (DQ_M - 1), hq = ct >> 7;
-        // TMEM lanes 32 (warp % 4) ... + 31 belong to this warp: lane = weight row
-        const unsigned a_lane = (unsigned)((r >> 5) * 32) << 16;
-        bool ok = true;
-        for (int j = 0; j < nblk && ok; ++j) {
-            const int st = j % DQ_RING, buf = j % DQ_ABUF;
-            const int b = blk_bits[j];
-            // the block has landed, and the contraction of block j - DQ_ABUF no longer reads the operand buffer
-            ok = __all_sync(0xffffffffu, dq_mbar_wait(dq_smem_u32(ld_full + st), (unsigned)(j / DQ_RING) & 1u, abort_flag) &&
-                                         (j < DQ_ABUF || dq_mbar_wait(dq_smem_u32(done + (j - DQ_ABUF) % DQ_RING),
-                                                                      (unsigned)((j - DQ_ABUF) / DQ_RING) & 1u, abort_flag)));
-            if (!ok) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const unsigned char* src = code_ring + st * DQ_CODE_STAGE + r * 16 * b;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int qi = 2 * h + hq;
-                uint32_t v[16];
-                switch (b) {                                  // uniform over the CTA
-                    case 1: dq_unpack32<1>(src, qi, v); break;
-                    case 2: dq_unpack32<2>(src, qi, v); break;
-                    case 4: dq_unpack32<4>(src, qi, v); break;
-                    case 8: dq_unpack32<8>(src, qi, v); break;
-                    default: dq_unpack32_generic(src, b, qi, v); break;
-                }
-                dq_tmem_st16(tmem_base + a_lane + (unsigned)(64 + buf * DQ_A_COLS + 16 * qi), v);
-            }
-            dq_mbar_arrive(dq_smem_u32(code_empty + st));     // the codes are in registers: the stage may be refilled
-            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            dq_mbar_arrive(dq_smem_u32(a_full + buf));
-        }
-    } else if (warp == DQ_EPI_WARPS + DQ_CONV_WARPS) {
+    if (warp == WARPS) {
         if (lane == 0) {
-            // ---- MMA issue -----------------------------------------------------------------------------
-            const unsigned idesc = dq_idesc(NT);
+            // ---- loader: the codes of block j as they lie in memory and its slice of X (an image in
+            // the order of the block's bitwidth) into ring stage j % RING, as soon as every
+            // contraction warp has let go of block j - RING -------------------------------------------
             bool ok = true;
             for (int j = 0; j < nblk && ok; ++j) {
-                const int ds_ = j & 1, st = j % DQ_RING, buf = j % DQ_ABUF;
-                ok = dq_mbar_wait(dq_smem_u32(d_empty + ds_), ((unsigned)(j >> 1) & 1u) ^ 1u, abort_flag) &&
-                     dq_mbar_wait(dq_smem_u32(ld_full + st), (unsigned)(j / DQ_RING) & 1u, abort_flag) &&
-                     dq_mbar_wait(dq_smem_u32(a_full + buf), (unsigned)(j / DQ_ABUF) & 1u, abort_flag);
+                const int st = j % RING;
+                DQ_TL(WARPS, j, 0);
+                if (j >= RING) ok = dq_mbar_wait(dq_smem_u32(empty + st), (unsigned)(j / RING - 1) & 1u, abort_flag);
                 if (!ok) break;
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const unsigned at = tmem_base + (unsigned)(64 + buf * DQ_A_COLS);
-                const unsigned xt = dq_smem_u32(x_ring + st * DQ_X_STAGE);
-#pragma unroll
-                for (int ks = 0; ks < DQ_KB / 16; ++ks)             // 16 columns: 8 TMEM columns of A, 32 bytes of X along K
-                    dq_mma(tmem_base + (unsigned)(ds_ * NT), at + ks * 8,
-                           dq_desc(xt + (ks >> 2) * (NT * 128) + (ks & 3) * 32), idesc, ks > 0 ? 1u : 0u);
-                dq_commit(dq_smem_u32(done + st));
-            }
-        }
-    } else if (warp == DQ_EPI_WARPS + DQ_CONV_WARPS + 1) {
-        if (lane == 0) {
-            // ---- loader: the codes of block j as they lie in memory and its slice of X (an operand
-            // image) into ring stage j % DQ_RING, as soon as the unpackers and the contraction of block
-            // j - DQ_RING have let go of it ----------------------------------------------------------------
-            bool ok = true;
-            const unsigned x_bytes = (unsigned)(NT * DQ_KB * 2);
-            for (int j = 0; j < nblk && ok; ++j) {
-                const int st = j % DQ_RING;
-                // block j - DQ_RING used this stage: its codes have been read and its contraction is complete
-                if (j >= DQ_RING) {
-                    const unsigned ph = (unsigned)(j / DQ_RING - 1) & 1u;
-                    ok = dq_mbar_wait(dq_smem_u32(code_empty + st), ph, abort_flag) &&
-                         dq_mbar_wait(dq_smem_u32(done + st), ph, abort_flag);
-                }
-                if (!ok) break;
+                DQ_TL(WARPS, j, 1);
                 const int b = blk_bits[j];
-                const unsigned code_bytes = (unsigned)(2048 * b);
-                const unsigned full = dq_smem_u32(ld_full + st);
-                dq_mbar_expect_tx(full, code_bytes + x_bytes);
-                dq_bulk_load(dq_smem_u32(code_ring + st * DQ_CODE_STAGE), a.packed + word0 + blk_word[j], code_bytes, full);
-                dq_bulk_load(dq_smem_u32(x_ring + st * DQ_X_STAGE),
-                             a.xp + ((int64_t)dq_order(b) * a.nbc + j0 + j) * (NT * DQ_KB), x_bytes, full);
+                const int o = dq_order(b);
+                const unsigned code_bytes = (unsigned)(S::ROWS * 16 * b);
+                const unsigned x_bytes = (unsigned)(NT * DQ_KB * 2);
+                const unsigned bar = dq_smem_u32(full + st);
+                unsigned char* stage = smem + st * S::STAGE;
+                dq_mbar_expect_tx(bar, code_bytes + x_bytes);
+                dq_bulk_load(dq_smem_u32(stage + S::X_STAGE), a.packed + word0 + blk_word[j], code_bytes, bar);
+                dq_bulk_load(dq_smem_u32(stage),
+                             a.xp + dq_order_base(o, a.nbc, NT) + (int64_t)(j0 + j) * (NT * DQ_KB),
+                             x_bytes, bar);
             }
         }
     } else {
-        // ---- drain: thread = weight row = TMEM lane -----------------------------------------------------
-        const int r = threadIdx.x;
-        const int64_t row = (int64_t)bi * DQ_M + r;
-        float y[NT];
+        // ---- contraction warps: 16 weight rows each -----------------------------------------------------
+        const int g = lane >> 2, t = lane & 3;
+        const int64_t row_lo = (int64_t)bi * S::ROWS + warp * 16 + g;        // and row_lo + 8
+        // the lane's ldmatrix row inside an image, without the stage and the row pitch (which depends
+        // on the block's order): matrix mi = lane / 8, row r8 = lane % 8
+        const int mi = lane >> 3, r8 = lane & 7;
+        float y[NT / 8][4];
 #pragma unroll
-        for (int t = 0; t < NT; ++t) y[t] = 0.f;
+        for (int nt = 0; nt < NT / 8; ++nt) y[nt][0] = y[nt][1] = y[nt][2] = y[nt][3] = 0.f;
         bool ok = true;
-        float2 sl = a.meta[row * a.nbc + j0];
+        float2 m0 = a.meta[row_lo * a.nbc + j0], m1 = a.meta[(row_lo + 8) * a.nbc + j0];
         for (int j = 0; j < nblk && ok; ++j) {
-            const float2 cur = sl;
-            if (j + 1 < nblk) sl = a.meta[row * a.nbc + j0 + j + 1];
-            const int ds_ = j & 1;
-            ok = __all_sync(0xffffffffu, dq_mbar_wait(dq_smem_u32(done + j % DQ_RING), (unsigned)(j / DQ_RING) & 1u, abort_flag));
-            if (!ok) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll
-            for (int c0 = 0; c0 < NT; c0 += 16) {
-                float d[16];
-                dq_tmem_ld16(tmem_base + ((unsigned)(warp * 32) << 16) + (unsigned)(ds_ * NT + c0), d);
-#pragma unroll
-                for (int k = 0; k < 16; ++k)
-                    y[c0 + k] = fmaf(cur.x, d[k], fmaf(cur.y, xs[j * NT + c0 + k], y[c0 + k]));
+            const float2 c0 = m0, c1 = m1;
+            if (j + 1 < nblk) {
+                m0 = a.meta[row_lo * a.nbc + j0 + j + 1];
+                m1 = a.meta[(row_lo + 8) * a.nbc + j0 + j + 1];
             }
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) dq_mbar_arrive(dq_smem_u32(d_empty + ds_));
+            const int st = j % RING;
+            DQ_TL(warp, j, 0);
+            ok = dq_mbar_wait(dq_smem_u32(full + st), (unsigned)(j / RING) & 1u, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            DQ_TL(warp, j, 1);
+            if (!ok) break;
+            const int b = blk_bits[j];                       // uniform over the CTA
+            const unsigned stage = dq_smem_u32(smem + st * S::STAGE);
+            const unsigned codes = stage + S::X_STAGE + (unsigned)(warp * 16 * 16 * b);
+            constexpr unsigned pitch = 2u * DQ_KB;                          // bytes of an image row
+            unsigned xlane[2];
+            if constexpr (NT == 8) {
+                // matrices: (step, low half), (step, high half), (step + 1, low), (step + 1, high) of tokens 0..7
+                xlane[0] = (stage + (unsigned)r8 * pitch + (unsigned)((((mi & 1) ^ r8) << 4))) ^ (unsigned)((mi >> 1) << 5);
+                xlane[1] = 0;
+            } else {
+                // matrices: tokens 16 q + 8 (mi / 2) .., low (mi even) or high (mi odd) half of the step
+#pragma unroll
+                for (int q = 0; q < 2; ++q)
+                    xlane[q] = stage + (unsigned)(16 * q + 8 * (mi >> 1) + r8) * pitch + (unsigned)(((mi & 1) ^ r8) << 4);
+            }
+            const unsigned eb = dq_smem_u32(empty + st);
+            const unsigned xa = dq_smem_u32(xs + j * NT + 2 * t);
+            switch (b) {
+                case 1: dq_block<1, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
+                case 2: dq_block<2, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
+                case 3: dq_block<3, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
+                case 4: dq_block<4, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
+                case 5: dq_block<5, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
+                case 6: dq_block<6, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
+                case 7: dq_block<7, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
+                default: dq_block<8, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
+            }
+            DQ_TL(warp, j, 2);
         }
         if (ok) {
-            float* out = a.out + (int64_t)blockIdx.y * a.out_seg_stride + row;
+            float* out = a.out + (int64_t)blockIdx.y * a.out_seg_stride;
 #pragma unroll
-            for (int t = 0; t < NT; ++t) {
-                if (!isfinite(y[t])) sb_latch(a.ds, SB_ERR_NONFINITE, SBK_GEMM);
-                if (t < a.T) out[(int64_t)t * a.out_t_stride] = y[t];
+            for (int nt = 0; nt < NT / 8; ++nt) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int tok = 8 * nt + 2 * t + (e & 1);
+                    if (!isfinite(y[nt][e])) sb_latch(a.ds, SB_ERR_NONFINITE, SBK_GEMM);
+                    if (tok < a.T) out[(int64_t)tok * a.out_t_stride + row_lo + 8 * (e >> 1)] = y[nt][e];
+                }
             }
         }
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (warp == DQ_EPI_WARPS + DQ_CONV_WARPS)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+#ifdef SB_EXP_TL
+    if (threadIdx.x == 0) dq_cta[blockIdx.y * gridDim.x + blockIdx.x][1] = dq_now_ns();
+#endif
     if (threadIdx.x == 0 && *abort_flag) sb_latch(a.ds, SB_ERR_TIMEOUT, SBK_GEMM);
 }
 
@@ -472,7 +553,27 @@ __global__ void dq_reduce_kernel(const float* __restrict__ part, int S, int T, i
     Y[(int64_t)t * ldy + r] = acc;
 }
 
+// resident CTAs per SM of the instance that serves (tokens padded to NT, block rows)
+int dq_ctas_per_sm(int NT, int br) {
+    if (br == 128) return NT == 8 ? DqShape<8, 8>::CTAS_PER_SM : NT == 16 ? DqShape<16, 8>::CTAS_PER_SM : DqShape<32, 8>::CTAS_PER_SM;
+    return NT == 8 ? DqShape<8, 4>::CTAS_PER_SM : NT == 16 ? DqShape<16, 4>::CTAS_PER_SM : DqShape<32, 4>::CTAS_PER_SM;
+}
+
+template <int NT, int WARPS>
+sb_status dq_launch(sb_ctx* ctx, const DqArgs& a, dim3 grid) {
+    using S = DqShape<NT, WARPS>;
+    SB_FUNC_ATTR(ctx, (dequant_gemm_kernel<NT, WARPS>), cudaFuncAttributeMaxDynamicSharedMemorySize, S::SMEM);
+    dequant_gemm_kernel<NT, WARPS><<<grid, S::THREADS, S::SMEM, ctx->stream>>>(a);
+    SB_LAUNCHED(ctx);
+    return SB_OK;
+}
+
 }  // namespace
+
+#ifdef SB_EXP_TL
+extern "C" int sb_dq_timeline(long long* dst) { return (int)cudaMemcpyFromSymbol(dst, dq_tl, sizeof(dq_tl)); }
+extern "C" int sb_dq_ctas(unsigned long long* dst) { return (int)cudaMemcpyFromSymbol(dst, dq_cta, sizeof(dq_cta)); }
+#endif
 
 extern "C" sb_status sb_dequant_gemm(sb_ctx* ctx, const void* X, int64_t T, int64_t ldx, const uint32_t* packed,
                                      const int64_t* block_off_words, const float* meta, const uint8_t* level,
@@ -482,15 +583,17 @@ extern "C" sb_status sb_dequant_gemm(sb_ctx* ctx, const void* X, int64_t T, int6
     if (!X || !packed || !block_off_words || !meta || !level || !Y || T <= 0 || R <= 0 || C <= 0)
         return sb_fail(ctx, SB_ERR_INVALID, "dequant gemm: null or empty");
     if (!sb_check_bits(bits, n_bits)) return sb_fail(ctx, SB_ERR_INVALID, "dequant gemm: bits must be ascending in 1..8");
-    if (br != DQ_M || bc != DQ_KB || group != DQ_KB || R % DQ_M || C % DQ_KB || ldx < C || ldy < R ||
+    if ((br != 64 && br != 128) || bc != DQ_KB || group != DQ_KB || R % br || C % DQ_KB || ldx < C || ldy < R ||
         (reinterpret_cast<uintptr_t>(packed) & 15))
-        return sb_fail(ctx, SB_ERR_SHAPE, "dequant gemm: blocks of 128 x 128 with group 128 tiling the matrix, 16-byte aligned codes");
+        return sb_fail(ctx, SB_ERR_SHAPE,
+                       "dequant gemm: blocks of 64 x 128 or 128 x 128 with group 128 tiling the matrix, 16-byte aligned codes");
     if (R >= (1ll << 31) || C >= (1ll << 31)) return sb_fail(ctx, SB_ERR_SHAPE, "dequant gemm: R and C must fit 31 bits");
     SB_CUDA(ctx, cudaSetDevice(ctx->device));
     const int nbc = (int)(C / DQ_KB);
-    const int64_t nbr = R / DQ_M;
-    // column segments: enough CTAs for two per SM, at most DQ_MAX_SEG_BLOCKS blocks each
-    int S = (int)((2 * (int64_t)ctx->sm_count) / nbr);
+    const int64_t nbr = R / br;
+    // column segments: enough CTAs to fill every SM's slots once, at most DQ_MAX_SEG_BLOCKS blocks each
+    const int NT0 = T <= 8 ? 8 : T <= 16 ? 16 : 32;            // the first (largest) slice decides the segments
+    int S = (int)((dq_ctas_per_sm(NT0, br) * (int64_t)ctx->sm_count) / nbr);
     if (S < 1) S = 1;
     if (S > nbc) S = nbc;
     int seg_blocks = (nbc + S - 1) / S;
@@ -499,24 +602,25 @@ extern "C" sb_status sb_dequant_gemm(sb_ctx* ctx, const void* X, int64_t T, int6
     if (S > 65535) return sb_fail(ctx, SB_ERR_SHAPE, "dequant gemm: too many column segments");
     DqBits db{};
     for (int l = 0; l < n_bits; ++l) db.packed |= (unsigned)bits[l] << (4 * l);
-    // tokens in slices of at most DQ_MAX_T (padded to 16 or 32 with zero rows)
+    // tokens in slices of at most DQ_MAX_T (padded to 8, 16 or 32 with zero rows)
     for (int64_t t0 = 0; t0 < T; t0 += DQ_MAX_T) {
         const int Tn = (int)((T - t0) < DQ_MAX_T ? (T - t0) : DQ_MAX_T);
-        const int NT = Tn <= 16 ? 16 : 32;
+        const int NT = Tn <= 8 ? 8 : Tn <= 16 ? 16 : 32;
+        const size_t image_elems = (size_t)DQ_ORDERS * NT * C;
         void* arena;
-        sb_status st = sb_scratch(ctx, Carver::need({(size_t)DQ_ORDERS * NT * C * 2, (size_t)nbc * NT * 4,
+        sb_status st = sb_scratch(ctx, Carver::need({image_elems * 2, (size_t)nbc * NT * 4,
                                                      S > 1 ? (size_t)S * Tn * R * 4 : 0}), &arena);
         if (st != SB_OK) return st;
         Carver cv(arena);
-        __nv_bfloat16* xp = cv.take<__nv_bfloat16>((size_t)DQ_ORDERS * NT * C);
+        __nv_bfloat16* xp = cv.take<__nv_bfloat16>(image_elems);
         float* xsum = cv.take<float>((size_t)nbc * NT);
         float* part = S > 1 ? cv.take<float>((size_t)S * Tn * R) : nullptr;
         const __nv_bfloat16* Xs = static_cast<const __nv_bfloat16*>(X) + t0 * ldx;
         if (Tn < NT) {      // zero rows for the padding tokens
-            SB_CUDA(ctx, cudaMemsetAsync(xp, 0, (size_t)DQ_ORDERS * NT * C * 2, ctx->stream));
+            SB_CUDA(ctx, cudaMemsetAsync(xp, 0, image_elems * 2, ctx->stream));
             SB_CUDA(ctx, cudaMemsetAsync(xsum, 0, (size_t)nbc * NT * 4, ctx->stream));
         }
-        dq_prepare_x_kernel<<<dim3((unsigned)nbc, (unsigned)Tn), 128, 0, ctx->stream>>>(Xs, ldx, NT, nbc, xp, xsum);
+        dq_prepare_x_kernel<<<dim3((unsigned)nbc, (unsigned)Tn), DQ_KB, 0, ctx->stream>>>(Xs, ldx, NT, nbc, xp, xsum);
         SB_LAUNCHED(ctx);
         DqArgs a{};
         a.packed = packed; a.block_off = block_off_words; a.meta = reinterpret_cast<const float2*>(meta);
@@ -526,14 +630,14 @@ extern "C" sb_status sb_dequant_gemm(sb_ctx* ctx, const void* X, int64_t T, int6
         a.out_seg_stride = S > 1 ? (int64_t)Tn * R : 0;
         a.R = R; a.C = C; a.nbc = nbc; a.seg_blocks = seg_blocks; a.T = Tn; a.bits = db; a.ds = ctx->dstate;
         const dim3 grid((unsigned)nbr, (unsigned)S);
-        if (NT == 16) {
-            SB_FUNC_ATTR(ctx, dequant_gemm_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM);
-            dequant_gemm_kernel<16><<<grid, DQ_THREADS, DQ_SMEM, ctx->stream>>>(a);
+        if (br == 128) {
+            st = NT == 8 ? dq_launch<8, 8>(ctx, a, grid) : NT == 16 ? dq_launch<16, 8>(ctx, a, grid)
+                                                                    : dq_launch<32, 8>(ctx, a, grid);
         } else {
-            SB_FUNC_ATTR(ctx, dequant_gemm_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM);
-            dequant_gemm_kernel<32><<<grid, DQ_THREADS, DQ_SMEM, ctx->stream>>>(a);
+            st = NT == 8 ? dq_launch<8, 4>(ctx, a, grid) : NT == 16 ? dq_launch<16, 4>(ctx, a, grid)
+                                                                    : dq_launch<32, 4>(ctx, a, grid);
         }
-        SB_LAUNCHED(ctx);
+        if (st != SB_OK) return st;
         if (S > 1) {
             dq_reduce_kernel<<<dim3((unsigned)((R + 255) / 256), (unsigned)Tn), 256, 0, ctx->stream>>>(part, S, Tn, R,
                                                                                                        Y + t0 * ldy, ldy);

@@ -21,27 +21,27 @@ def ctx():
     c.close()
 
 
-def _tolerance(X, meta, level, bits, R, Cc):
+def _tolerance(X, meta, level, bits, R, Cc, br=128):
     """The kernel contracts the integer codes exactly (bf16 x bf16 products are exact in fp32) and
     rounds only in fp32 sums: the tensor cores' accumulation over a block, scale * acc + lo * colsum
     per block, and the sum over blocks.  Each is within a few 2^-24 of the magnitudes it adds, which
     are bounded by sum_j (sum_{c in j} |x_c|) (|lo_rj| + scale_rj qmax_j): 2e-6 of that bound."""
     nbc = Cc // 128
-    qmax = np.array([2 ** bits[l] - 1 for l in level], dtype=np.float64).reshape(R // 128, nbc)
-    qmax = np.repeat(qmax, 128, axis=0)                                   # [R][nbc]
+    qmax = np.array([2 ** bits[l] - 1 for l in level], dtype=np.float64).reshape(R // br, nbc)
+    qmax = np.repeat(qmax, br, axis=0)                                    # [R][nbc]
     m = meta.reshape(R, nbc, 2).astype(np.float64)
     bound_w = np.abs(m[:, :, 1]) + m[:, :, 0] * qmax                      # [R][nbc]
     xabs = X.double().abs().reshape(X.shape[0], nbc, 128).sum(-1).numpy() # [T][nbc]
     return 2e-6 * xabs @ bound_w.T + 1e-30
 
 
-def _run(ctx, R, Cc, T, bits, seed, ldx=None, ldy=None):
+def _run(ctx, R, Cc, T, bits, seed, ldx=None, ldy=None, br=128):
     W = synth.make_weight(R, Cc, 300 + seed)
     X = synth.make_activations(T, Cc, 400 + seed)
     rng = np.random.default_rng(seed)
-    level = rng.integers(0, len(bits), (R // 128) * (Cc // 128)).astype(np.uint8)
-    packed, off, meta = sbo.pack_blocks(W, bits, level, 128, 128, 128)
-    ref = sbo.dequant_gemm(X, packed, off, meta, level, R, Cc, bits, 128, 128, 128)
+    level = rng.integers(0, len(bits), (R // br) * (Cc // 128)).astype(np.uint8)
+    packed, off, meta = sbo.pack_blocks(W, bits, level, br, 128, 128)
+    ref = sbo.dequant_gemm(X, packed, off, meta, level, R, Cc, bits, br, 128, 128)
     Xg = X.to(DEV)
     if ldx:
         buf = torch.zeros(T, ldx, dtype=torch.bfloat16, device=DEV)
@@ -51,10 +51,11 @@ def _run(ctx, R, Cc, T, bits, seed, ldx=None, ldy=None):
     if ldy:
         Y = torch.full((T, ldy), float("nan"), dtype=torch.float32, device=DEV)[:, :R]
     out = ctx.dequant_gemm(Xg, torch.from_numpy(packed.view(np.int32)).to(DEV), torch.from_numpy(off).to(DEV),
-                           torch.from_numpy(meta).to(DEV), torch.from_numpy(level).to(DEV), R, Cc, bits, Y=Y)
+                           torch.from_numpy(meta).to(DEV), torch.from_numpy(level).to(DEV), R, Cc, bits,
+                           block_rows=br, Y=Y)
     ctx.sync()
     got = out.cpu().double().numpy()
-    tol = _tolerance(X, meta, level, bits, R, Cc)
+    tol = _tolerance(X, meta, level, bits, R, Cc, br)
     err = np.abs(got - ref)
     assert np.all(err <= tol), (float((err / tol).max()), np.unravel_index((err / tol).argmax(), err.shape))
     return got, ref
@@ -66,14 +67,21 @@ def test_table_4_mix_of_2_4_8_bits(ctx, R, Cc, T):
     _run(ctx, R, Cc, T, [2, 4, 8], seed=R + Cc + T)
 
 
-@pytest.mark.parametrize("T", [1, 5, 17, 40, 64])
+@pytest.mark.parametrize("T", [1, 5, 8, 9, 17, 40, 64])
 def test_any_number_of_tokens(ctx, T):
-    """Padding to 16 or 32 tokens, and slices of 32."""
+    """Padding to 8, 16 or 32 tokens, and slices of 32."""
     _run(ctx, 256, 512, T, [2, 4, 8], seed=T)
 
 
+@pytest.mark.parametrize("R,Cc,T,bits", [(64, 128, 16, [4]), (192, 384, 32, [2, 4, 8]), (448, 1024, 7, [2, 4, 8]),
+                                         (1024, 2048, 32, [1, 2, 3, 4, 5, 6, 7, 8])])
+def test_blocks_of_64_rows(ctx, R, Cc, T, bits):
+    """The paper's own partition (Section 5 "Implementation": 64 x 128 blocks, group 128)."""
+    _run(ctx, R, Cc, T, bits, seed=R + T, br=64)
+
+
 def test_every_bitwidth(ctx):
-    """1, 2, 4, 8 through the mask-per-pair unpacking, 3, 5, 6, 7 through the generic one."""
+    """1, 2, 4 through the mask-per-pair unpacking, 8 as two nibbles, 3, 5, 6, 7 cut out code by code."""
     _run(ctx, 512, 1024, 16, [1, 2, 3, 4, 5, 6, 7, 8], seed=11)
     for b in range(1, 9):
         _run(ctx, 128, 256, 16, [b], seed=20 + b)
