@@ -407,13 +407,13 @@ def dequant_gemm_times(ctx, dev, peak_gbs):
             del g
             bytes_ = sets[0][4] * 4 + R * (Cc // 128) * 8 + T * Cc * 2 + T * R * 4
             gbs = bytes_ / (ms * 1e-3) / 1e9
-            out.append({"kernel": "dequant_gemm_kernel (tcgen05) + dq_prepare_x_kernel + dq_reduce_kernel",
+            out.append({"kernel": "dq_prepare_x_kernel + dequant_gemm_kernel (register-fragment tensor-core products, segments added inside a cluster)",
                         "bound": "hbm", "achieved": gbs, "peak": peak_gbs, "unit": "GB/s", "frac": gbs / peak_gbs,
                         "ms_per_call": ms, "us_per_call": ms * 1e3, "algorithmic_bytes": bytes_,
                         "workload": f"8192 x 8192, {T} tokens, " + ("all blocks 4 bits" if kind == "int4"
                                                                     else "40/40/20 % of 2/4/8 bits"),
                         "paper_table_4_us": paper_us[(kind, T)],
-                        "note": "one call of sb_dequant_gemm (three launches); packed codes + scale / minimum "
+                        "note": "one call of sb_dequant_gemm (two launches); packed codes + scale / minimum "
                                 "metadata + activations read, outputs written; the paper's figure is its own "
                                 "kernel on its own GPU: context, not a comparison on equal hardware"})
         del sets

@@ -199,12 +199,13 @@ sb_status sb_pack_blocks(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_t C, 
  *     Y[t][r] = sum_c X[t][c] * (lo[r][g(c)] + scale[r][g(c)] * q[r][c])
  * in the packed (permuted) row and column order: X's columns are the packed columns, Y's
  * columns the packed rows.  The contraction runs on the integer codes (exact in bf16) on the
- * tensor cores with fp32 accumulation, one 128 x 128 block at a time, and scale and lo are
- * applied per row and block in fp32; nothing else is rounded.
+ * tensor cores with fp32 accumulation, one block at a time, and scale and lo are applied per
+ * row and block in fp32; nothing else is rounded.
  *   - X: device bf16 [T][C], leading dimension ldx >= C; T >= 1 (tokens are processed in
- *     slices of 32; decode batches are the intended use).
+ *     slices of 32, padded to 8, 16 or 32; decode batches are the intended use).
  *   - packed, block_off_words, meta, level, bits: as written by / given to sb_pack_blocks;
- *     packed 16-byte aligned.  block_rows = block_cols = group = 128 is required.
+ *     packed 16-byte aligned.  Blocks of 64 x 128 (the paper's partition, Section 5
+ *     "Implementation") or 128 x 128 with group = 128 are required.
  *   - Y: device fp32 [T][R], leading dimension ldy >= R, overwritten.
  * A pipeline wait that does not complete within 2 s latches SB_ERR_TIMEOUT.  Asynchronous. */
 sb_status sb_dequant_gemm(sb_ctx* ctx, const void* X_bf16, int64_t T, int64_t ldx,

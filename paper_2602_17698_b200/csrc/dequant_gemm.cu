@@ -7,52 +7,57 @@
 // bf16 x bf16 -> fp32 per block, scaled per row when the block is done; nothing is rounded but
 // the fp32 accumulation.
 //
-// The work is bound by the packed bytes (4 bits per weight on average against at most 32
-// tokens): what costs time is turning codes into tensor-core operands, so the design keeps that
-// path as short as it can be made.  A warp owns 16 weight rows of a block and feeds the tensor
-// cores from REGISTERS (mma.sync m16n8k16: weight rows on M, tokens on N): the unpacked codes are
-// the A fragment where the unpacking leaves them, with no trip through shared or tensor memory,
-// no second thread to hand them to and no accumulator to fetch back.  (A tcgen05 form of this
-// kernel, codes stored to tensor memory as the A operand of M = 128 instructions issued by one
-// thread, spent three times as many instructions per code on the hand-overs between its unpacking,
-// issuing and draining warps and ran at a third of the speed; the contraction itself is about a
-// microsecond of tensor work on any path.)
+// A decode batch is at most 32 tokens against 4 bits per weight on average: the packed bytes
+// are what must move, and what costs time is turning codes into tensor-core operands.  A warp
+// owns 32 weight rows of a block and feeds the tensor cores from REGISTERS (mma.sync m16n8k16:
+// weight rows on M, tokens on N): the unpacked codes are the A fragment where the unpacking
+// leaves them, with no trip through shared or tensor memory, no second thread to hand them to
+// and no accumulator to fetch back.  (A tcgen05 form of this kernel -- codes stored to tensor
+// memory as the A operand of M = 128, N = tokens instructions issued by one thread -- needed the
+// same number of instructions per code for the hand-overs between its unpacking, issuing and
+// draining warps and was bound by those chains; with so few tokens the contraction is a
+// microsecond or two of tensor work on either path.)
 //
-// Unpacking, about one operation per code: lane (g, t) of a warp holds the 32 codes 32 t .. 32 t + 31
-// of rows g and g + 8.  For b in {1, 2, 4} a 32-bit word of codes is split by one shift and one
-// mask-and-or per PAIR,
+// Unpacking, one shift and one three-input logic operation per PAIR of codes: lane (g, t) of a
+// warp holds the 32 codes 32 t .. 32 t + 31 of rows g and g + 8 of each of its 16-row tiles.
+// For b in {1, 2, 4} a 32-bit word of codes gives
 //     ((w >> (b s - (7 - b))) & MASK) | 0x43004300  ->  bf16 pair (128 + 2^(7-b) q_s, 128 + 2^(7-b) q_(s + 16/b)):
 // the code lands in the top bits of the bf16 mantissa under the exponent of 128.  The offset and
 // the power of two are taken out again when the block is scaled (they fold into scale and lo), so
-// no subtraction is spent per code.  Codes of 8 bits go through as two 4-bit fields each against
-// X and 16 X (a block of 256 columns to the tensor cores); 3, 5, 6 and 7 bits are cut out of the
-// bit stream one by one.  The contraction does not care in which order it visits the columns of
-// a block as long as X uses the same one, so a small kernel first writes X in the column order
-// each unpacking produces (and the per-block column sums of X).
+// no subtraction is spent per code.  Codes of 8 bits go through as their two nibbles, the low one
+// under the exponent of 128 and the high one under the exponent of 2048 (sixteen times the
+// weight), both against the same fragment of X; 3, 5, 6 and 7 bits are cut out of the bit stream
+// one by one.  The contraction does not care in which order it visits the columns of a block as
+// long as X uses the same one, so a small kernel first writes X in the column order each
+// unpacking produces (and the per-block column sums of X).
 //
-// Grid: (R / block_rows row tiles) x (S column segments); block_rows / 16 contraction warps and a
-// loader warp per CTA, two (128-row blocks) or three (64-row blocks) CTAs per SM.  The loader
-// thread brings each block in with two bulk copies (cp.async.bulk, mbarrier complete_tx) into a
-// ring of three or four stages: the block's packed codes as they lie in memory, and its slice of
-// X, which the preparation kernel has laid out as the image ldmatrix reads without bank
-// conflicts.  Each warp: wait for the stage, read its rows' codes (one to seven loads), eight or
-// sixteen steps of {unpack four registers, ldmatrix the tokens' fragments, one mma.sync per eight
-// tokens}, release the stage, then y += scale' * acc + lo' * colsum(X) in fp32 registers.  The
-// segment's partial sums go to scratch (or to Y when there is one segment) and a second kernel
-// adds the segments in order.  Every mbarrier wait is bounded; on a time-out the kernel latches
-// SB_ERR_TIMEOUT and all roles leave.
+// Grid: (R / block_rows row tiles) x (S column segments); block_rows / 32 contraction warps and
+// a loader warp per CTA, two CTAs per SM for 128-row blocks.  The loader warp brings each block
+// into a ring in shared memory whose entries are as large as their block (image of X, codes at
+// their own bitwidth, the rows' scale and minimum): lane 0 issues two bulk copies (cp.async.bulk,
+// mbarrier complete_tx) for the block's packed codes as they lie in memory and for its slice of X
+// as the image ldmatrix reads without bank conflicts, all lanes fetch the rows' (scale, minimum)
+// with 8-byte asynchronous copies counted on the same barrier.  Each contraction warp: wait for
+// the block, read its rows' codes, eight steps of {ldmatrix the next step's tokens, unpack four
+// registers per tile, one mma.sync per tile and eight tokens}, release the entry, then
+// y += scale' * acc + lo' * colsum(X) in fp32 registers.  With 2 to 8 segments the segments of a
+// row tile are the CTAs of one cluster and are added in segment order through distributed shared
+// memory; with more, partial sums go to scratch and a second kernel adds them in order.  Every
+// mbarrier wait is bounded; on a time-out the kernel latches SB_ERR_TIMEOUT and all roles leave.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
 constexpr int DQ_KB = 128;                  // block columns = quantisation group
 constexpr int DQ_MAX_T = 32;                // tokens per pass
-#ifdef SB_EXP_C3
-constexpr int DQ_MAX_SEG_BLOCKS = 16;
-#else
-constexpr int DQ_MAX_SEG_BLOCKS = 32;       // column blocks per segment (their column sums sit in shared memory)
-#endif
-constexpr int DQ_ORDERS = 5;                // column orders of X: one by one, b = 1, 2, 4, and 8 as two nibbles
+constexpr int DQ_MAX_SEG_BLOCKS = 16;       // column blocks per segment (their column sums sit in shared memory)
+constexpr int DQ_MT = 2;                    // tiles of 16 rows per contraction warp
+constexpr int DQ_MAX_CTAS = 4;              // resident CTAs per SM the launch bounds ask for at most
+constexpr int DQ_ORDERS = 5;                // column orders of X: one by one, b = 1, 2, 4, and 8 as byte pairs
 constexpr unsigned long long DQ_WAIT_NS = 2000ull * 1000 * 1000;
 
 // candidate bitwidths, four bits each
@@ -266,33 +271,37 @@ __device__ __forceinline__ void dq_load_row(unsigned rowaddr, int t, uint32_t* w
     }
 }
 
-// One block for one warp: acc[nt][.] = sum over the block's columns of codes x X for the warp's
-// 16 rows and tokens 8 nt .. 8 nt + 7.  codes: shared address of the warp's first row in the
-// stage; xlane: the lane's ldmatrix row address(es) in the stage's image, before the step is
-// XOR-ed in.
-template <int B, int NT>
+// One block for one warp: acc[m][nt][.] = sum over the block's columns of codes x X for the warp's
+// 16 MT rows (MT tiles of 16) and tokens 8 nt .. 8 nt + 7; every fragment of X that is fetched
+// serves all MT tiles.  codes: shared address of the warp's first row in the stage; xlane: the
+// lane's ldmatrix row address(es) in the stage's image, before the step is XOR-ed in; meta[m][h]:
+// (scale, minimum) of row 16 m + 8 h + g.
+template <int B, int NT, int MT>
 __device__ __forceinline__ void dq_block(unsigned codes, const unsigned (&xlane)[2], int g, int t,
-                                         unsigned empty_bar, int lane, float2 c0, float2 c1, unsigned xs_addr,
-                                         float (&y)[NT / 8][4]) {
-    float acc[NT / 8][4];
+                                         unsigned empty_bar, int lane, const float2 (&meta)[MT][2], unsigned xs_addr,
+                                         float (&y)[MT][NT / 8][4]) {
+    float acc[MT][NT / 8][4];
     constexpr int VW = B == 8 ? 8 : B;
     constexpr int STEPS = 8;
     constexpr int SUB = B == 8 ? 2 : 1;         // 8 bits: low and high nibbles against the same columns of X
-    uint32_t w0[VW], w1[VW];
-    dq_load_row<B>(codes + (unsigned)(g * 16 * B), t, w0);
-    dq_load_row<B>(codes + (unsigned)((g + 8) * 16 * B), t, w1);
+    uint32_t w[MT][2][VW];
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+        dq_load_row<B>(codes + (unsigned)((16 * m + g) * 16 * B), t, w[m][0]);
+        dq_load_row<B>(codes + (unsigned)((16 * m + g + 8) * 16 * B), t, w[m][1]);
+    }
     // the constants of the unpacking live in registers (an immediate would split the operation in
     // two): the field mask and the exponent under which the field sits, 128 (x 16 for high nibbles)
     uint32_t mask = dq_pair_mask<B>(), c43 = 0x43004300u, c45 = 0x45004500u;
     asm volatile("" : "+r"(mask), "+r"(c43), "+r"(c45));
     // registers 2 ks and 2 ks + 1 of step ks (8 bits: of its low, then of its high nibbles)
-    auto a_regs = [&](int ks, int sub, uint32_t (&a)[4]) {
+    auto a_regs = [&](int m, int ks, int sub, uint32_t (&a)[4]) {
         const int i0 = SUB * (2 * ks) + sub, i1 = SUB * (2 * ks + 1) + sub;
         const uint32_t c = sub ? c45 : c43;
-        a[0] = dq_pair<B>(w0, i0, mask, c);
-        a[1] = dq_pair<B>(w1, i0, mask, c);
-        a[2] = dq_pair<B>(w0, i1, mask, c);
-        a[3] = dq_pair<B>(w1, i1, mask, c);
+        a[0] = dq_pair<B>(w[m][0], i0, mask, c);
+        a[1] = dq_pair<B>(w[m][1], i0, mask, c);
+        a[2] = dq_pair<B>(w[m][0], i1, mask, c);
+        a[3] = dq_pair<B>(w[m][1], i1, mask, c);
     };
     if constexpr (NT == 8) {
         // one ldmatrix brings the fragments of two steps; the next pair of steps is fetched a pair ahead
@@ -304,9 +313,12 @@ __device__ __forceinline__ void dq_block(unsigned codes, const unsigned (&xlane)
             const uint32_t(&cur)[4] = bf[(ks >> 1) & 1];
 #pragma unroll
             for (int sub = 0; sub < SUB; ++sub) {
-                uint32_t a[4];
-                a_regs(ks, sub, a);
-                dq_mma(acc[0], a, cur[2 * (ks & 1)], cur[2 * (ks & 1) + 1], ks == 0 && sub == 0);
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    uint32_t a[4];
+                    a_regs(m, ks, sub, a);
+                    dq_mma(acc[m][0], a, cur[2 * (ks & 1)], cur[2 * (ks & 1) + 1], ks == 0 && sub == 0);
+                }
             }
         }
     } else {
@@ -323,112 +335,113 @@ __device__ __forceinline__ void dq_block(unsigned codes, const unsigned (&xlane)
             }
 #pragma unroll
             for (int sub = 0; sub < SUB; ++sub) {
-                uint32_t a[4];
-                a_regs(ks, sub, a);
 #pragma unroll
-                for (int q = 0; q < NQ; ++q) {
-                    dq_mma(acc[2 * q], a, bf[ks & 1][q][0], bf[ks & 1][q][1], ks == 0 && sub == 0);
-                    dq_mma(acc[2 * q + 1], a, bf[ks & 1][q][2], bf[ks & 1][q][3], ks == 0 && sub == 0);
+                for (int m = 0; m < MT; ++m) {
+                    uint32_t a[4];
+                    a_regs(m, ks, sub, a);
+#pragma unroll
+                    for (int q = 0; q < NQ; ++q) {
+                        dq_mma(acc[m][2 * q], a, bf[ks & 1][q][0], bf[ks & 1][q][1], ks == 0 && sub == 0);
+                        dq_mma(acc[m][2 * q + 1], a, bf[ks & 1][q][2], bf[ks & 1][q][3], ks == 0 && sub == 0);
+                    }
                 }
             }
         }
     }
     __syncwarp();
     if (lane == 0) dq_mbar_arrive(empty_bar);            // codes and image are in registers
-    // codes went in as 128 + 2^P q (P = 7 - B; 8 bits: two nibbles with P = 3 against X and 16 X,
-    // offset 128 * 17): sum_c x q = (acc - OFF colsum) / 2^P, folded into the row's scale and minimum
+    // codes went in as 128 + 2^P q (P = 7 - B; 8 bits: low nibbles as 128 + 8 n, high nibbles as
+    // 2048 + 128 n, offset 128 * 17): sum_c x q = (acc - OFF colsum) / 2^P, folded into the row's
+    // scale and minimum
     constexpr float INV = B == 8 ? 0.125f : 1.f / (float)(1 << (7 - B));
     constexpr float OFF = B == 8 ? 2176.f : 128.f;
-    const float s0 = c0.x * INV, s1 = c1.x * INV;
-    const float l0 = fmaf(-s0, OFF, c0.y), l1 = fmaf(-s1, OFF, c1.y);
+    float sc[MT][2], lo[MT][2];
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            sc[m][h] = meta[m][h].x * INV;
+            lo[m][h] = fmaf(-sc[m][h], OFF, meta[m][h].y);
+        }
+    }
 #pragma unroll
     for (int nt = 0; nt < NT / 8; ++nt) {
         const uint2 cu = dq_lds64(xs_addr + 32 * nt);
         const float cx = __uint_as_float(cu.x), cy = __uint_as_float(cu.y);
-        y[nt][0] = fmaf(s0, acc[nt][0], fmaf(l0, cx, y[nt][0]));
-        y[nt][1] = fmaf(s0, acc[nt][1], fmaf(l0, cy, y[nt][1]));
-        y[nt][2] = fmaf(s1, acc[nt][2], fmaf(l1, cx, y[nt][2]));
-        y[nt][3] = fmaf(s1, acc[nt][3], fmaf(l1, cy, y[nt][3]));
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            y[m][nt][0] = fmaf(sc[m][0], acc[m][nt][0], fmaf(lo[m][0], cx, y[m][nt][0]));
+            y[m][nt][1] = fmaf(sc[m][0], acc[m][nt][1], fmaf(lo[m][0], cy, y[m][nt][1]));
+            y[m][nt][2] = fmaf(sc[m][1], acc[m][nt][2], fmaf(lo[m][1], cx, y[m][nt][2]));
+            y[m][nt][3] = fmaf(sc[m][1], acc[m][nt][3], fmaf(lo[m][1], cy, y[m][nt][3]));
+        }
     }
 }
-
-#ifdef SB_EXP_TL
-__device__ long long dq_tl[9][40][4];
-__device__ unsigned long long dq_cta[512][4];
-#define DQ_TL(w, j, k) do { if (blockIdx.x == 3 && blockIdx.y == 1 && lane == 0 && (j) < 40) dq_tl[w][j][k] = clock64(); } while (0)
-#else
-#define DQ_TL(w, j, k) do { } while (0)
-#endif
 
 struct DqArgs {
     const uint32_t* packed;
     const int64_t* block_off;       // [nb + 1], words
     const float2* meta;             // [(r * nbc + j)] = (scale, lo), group == block width
     const uint8_t* level;           // [nb]
-    const __nv_bfloat16* xp;        // per order, per column block: image of NT x 128 (256 for 8 bits)
+    const __nv_bfloat16* xp;        // per order, per column block: image of NT x 128
     const float* xsum;              // [nbc][NT]
     float* out;                     // partial sums [S][T][R] (or Y when S == 1)
     int64_t out_t_stride;           // R for the partial sums, ldy for Y
     int64_t out_seg_stride;
     int64_t R, C;
     int nbc, seg_blocks, T;
+    int cluster_sum;                // the segments of a row tile are one cluster: summed through shared memory, out = Y
     DqBits bits;
     SbDeviceState* ds;
 };
 
-template <int NT, int WARPS> struct DqShape {
-    static constexpr int ROWS = 16 * WARPS;                         // block rows
-    static constexpr int X_STAGE = NT * DQ_KB * 2;                  // an image: NT x 128 bf16
-    static constexpr int CODE_STAGE = ROWS * 16 * 8;                // a block's codes at 8 bits
-    static constexpr int STAGE = X_STAGE + CODE_STAGE;
-#ifdef SB_EXP_C3
-    static constexpr int RING = 3;
-#else
-    static constexpr int RING = 4;
-#endif
+// WARPS contraction warps of MT tiles of 16 rows each.  A block's entry in the CTA's ring is its
+// image of X, its codes at their own bitwidth and its rows' (scale, minimum): entries are as large
+// as their block, so that low-bit blocks leave room for more blocks in flight.
+template <int NT, int WARPS, int MT> struct DqShape {
+    static constexpr int ROWS = 16 * MT * WARPS;                    // block rows
+    static constexpr int X_BYTES = NT * DQ_KB * 2;                  // an image: NT x 128 bf16
+    static constexpr int META_BYTES = ROWS * 8;                     // (scale, minimum) of the block's rows
+    static constexpr int RING_BYTES = WARPS >= 4 ? 104 * 1024 : 46 * 1024;
     static constexpr int THREADS = (WARPS + 1) * 32;                // + loader warp
-    static constexpr int SMEM = RING * STAGE + DQ_MAX_SEG_BLOCKS * NT * 4 + 256 /* alignment */ +
-                                256 /* barriers, block table */;
-    // resident CTAs per SM by shared memory (227 KB, 1 KB reserved per CTA), at most four
+    static constexpr int SMEM = RING_BYTES + DQ_MAX_SEG_BLOCKS * NT * 4 + 256 /* alignment */ +
+                                512 /* barriers, block table */;
+    // resident CTAs per SM by shared memory (227 KB, 1 KB reserved per CTA), at most DQ_MAX_CTAS
     static constexpr int FIT = (227 * 1024) / (SMEM + 1024);
-    static constexpr int CTAS_PER_SM = FIT > 4 ? 4 : FIT;
+    static constexpr int CTAS_PER_SM = FIT > DQ_MAX_CTAS ? DQ_MAX_CTAS : FIT;
+    __host__ __device__ static constexpr int entry_bytes(int b) { return X_BYTES + ROWS * 16 * b + META_BYTES; }
+    static_assert(X_BYTES + ROWS * 16 * 8 + META_BYTES <= RING_BYTES, "the largest entry fits the ring");
 };
 
-template <int NT, int WARPS>
-__global__ void __launch_bounds__(DqShape<NT, WARPS>::THREADS, DqShape<NT, WARPS>::CTAS_PER_SM)
+template <int NT, int WARPS, int MT>
+__global__ void __launch_bounds__(DqShape<NT, WARPS, MT>::THREADS, DqShape<NT, WARPS, MT>::CTAS_PER_SM)
 dequant_gemm_kernel(const DqArgs a) {
-    using S = DqShape<NT, WARPS>;
-    constexpr int RING = S::RING;
+    using S = DqShape<NT, WARPS, MT>;
     extern __shared__ unsigned char dq_smem_raw[];
-    // stage s: the block's image of X (256-byte aligned in the shared window: the swizzle is an XOR
-    // on the address bits below a row's 256 bytes), then its codes
+    // the ring (256-byte aligned in the shared window: entries are multiples of 256 bytes and start
+    // with the image, whose swizzle is an XOR on the address bits below a row's 256 bytes)
     unsigned char* smem = dq_smem_raw + ((256u - (dq_smem_u32(dq_smem_raw) & 255u)) & 255u);
-    float* xs = reinterpret_cast<float*>(smem + RING * S::STAGE);           // [seg_blocks][NT] column sums
+    float* xs = reinterpret_cast<float*>(smem + S::RING_BYTES);             // [seg_blocks][NT] column sums
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(xs + DQ_MAX_SEG_BLOCKS * NT);
-    unsigned long long* full = bars;                    // [RING] both copies of a block landed
-    unsigned long long* empty = bars + RING;            // [RING] every contraction warp has read the stage
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + RING);
+    // one pair of barriers per block of the segment, each used once
+    unsigned long long* full = bars;                        // [j] the block's copies have landed
+    unsigned long long* empty = bars + DQ_MAX_SEG_BLOCKS;   // [j] every contraction warp has read the block
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + DQ_MAX_SEG_BLOCKS);
     // per block of the segment: first word of its codes (blocks are below 2^32 words apart from the
-    // segment's first) and its bitwidth, so that the loop below has no dependent global loads
+    // segment's first), where its entry starts in the ring (written by the loader before the
+    // block's barrier is armed) and its bitwidth
     unsigned* blk_word = reinterpret_cast<unsigned*>(const_cast<int*>(abort_flag) + 4);   // [DQ_MAX_SEG_BLOCKS]
-    unsigned char* blk_bits = reinterpret_cast<unsigned char*>(blk_word + DQ_MAX_SEG_BLOCKS);
+    unsigned* blk_at = blk_word + DQ_MAX_SEG_BLOCKS;
+    unsigned char* blk_bits = reinterpret_cast<unsigned char*>(blk_at + DQ_MAX_SEG_BLOCKS);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-#ifdef SB_EXP_TL
-    if (threadIdx.x == 0) {
-        unsigned smid;
-        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-        dq_cta[blockIdx.y * gridDim.x + blockIdx.x][0] = dq_now_ns();
-        dq_cta[blockIdx.y * gridDim.x + blockIdx.x][2] = smid;
-    }
-#endif
 
     const int bi = blockIdx.x;                                  // row tile
     const int j0 = blockIdx.y * a.seg_blocks;                   // first column block of the segment
     const int nblk = min(a.seg_blocks, a.nbc - j0);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < RING; ++s) {
-            dq_mbar_init(dq_smem_u32(full + s), 1);
+        for (int s = 0; s < nblk; ++s) {
+            dq_mbar_init(dq_smem_u32(full + s), 1 + 32);       // the bulk copies' expect_tx and the loader lanes' row copies
             dq_mbar_init(dq_smem_u32(empty + s), WARPS);
         }
         *abort_flag = 0;
@@ -443,102 +456,173 @@ dequant_gemm_kernel(const DqArgs a) {
         blk_bits[threadIdx.x] = (unsigned char)dq_bits(a.bits, a.level[blk0 + threadIdx.x]);
     }
     __syncthreads();
+    const float2* mbase = a.meta + ((int64_t)bi * S::ROWS) * a.nbc + j0;
+    // what the loader does for block j
+    auto load_codes_meta = [&](int j, unsigned at) {
+        const unsigned bar = dq_smem_u32(full + j);
+        const unsigned code_bytes = (unsigned)(S::ROWS * 16 * blk_bits[j]);
+        if (lane == 0) {
+            blk_at[j] = at;
+            dq_mbar_expect_tx(bar, code_bytes + (unsigned)S::X_BYTES);
+            dq_bulk_load(dq_smem_u32(smem + at + S::X_BYTES), a.packed + word0 + blk_word[j], code_bytes, bar);
+        }
+        const unsigned mdst = dq_smem_u32(smem + at + S::X_BYTES) + code_bytes;
+#pragma unroll
+        for (int r = lane; r < S::ROWS; r += 32)
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(mdst + 8u * r), "l"(mbase + (int64_t)r * a.nbc + j)
+                         : "memory");
+        // counted on the block's barrier when this lane's copies have landed
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+    };
+    auto load_image = [&](int j, unsigned at) {
+        if (lane == 0)
+            dq_bulk_load(dq_smem_u32(smem + at),
+                         a.xp + dq_order_base(dq_order(blk_bits[j]), a.nbc, NT) + (int64_t)(j0 + j) * (NT * DQ_KB),
+                         (unsigned)S::X_BYTES, dq_smem_u32(full + j));
+    };
+    // The ring: entries in order of the blocks, each where the one before it ends, back to the
+    // start when the end is reached; `head` = where the next entry goes, `tail` = the oldest block
+    // not yet known to be released (its entry is the first thing `head` would run into).
+    unsigned head = 0;
+    int tail = 0, jl = 0;
+    bool lok = true;
+    // place block j: returns its offset, waiting for older blocks to be released where it must
+    auto place = [&](int j, bool may_wait, unsigned& at) -> bool {
+        const unsigned sz = (unsigned)S::entry_bytes(blk_bits[j]);
+        for (;;) {
+            if (tail == j) { head = 0; break; }                          // nothing in flight: start over
+            const unsigned ta = blk_at[tail];
+            if (head > ta) {                                             // in flight: [ta, head)
+                if (head + sz <= (unsigned)S::RING_BYTES) break;
+                if (sz <= ta) { head = 0; break; }
+            } else if (head + sz <= ta) {                                // in flight: [ta, end) and [0, head)
+                break;
+            }
+            if (!may_wait) return false;
+            lok = dq_mbar_wait(dq_smem_u32(empty + tail), 0u, abort_flag);
+            lok = __all_sync(0xffffffffu, lok);
+            if (!lok) return false;
+            ++tail;
+        }
+        at = head;
+        head += sz;
+        return true;
+    };
 
     if (warp == WARPS) {
-        if (lane == 0) {
-            // ---- loader: the codes of block j as they lie in memory and its slice of X (an image in
-            // the order of the block's bitwidth) into ring stage j % RING, as soon as every
-            // contraction warp has let go of block j - RING -------------------------------------------
-            bool ok = true;
-            for (int j = 0; j < nblk && ok; ++j) {
-                const int st = j % RING;
-                DQ_TL(WARPS, j, 0);
-                if (j >= RING) ok = dq_mbar_wait(dq_smem_u32(empty + st), (unsigned)(j / RING - 1) & 1u, abort_flag);
-                if (!ok) break;
-                DQ_TL(WARPS, j, 1);
-                const int b = blk_bits[j];
-                const int o = dq_order(b);
-                const unsigned code_bytes = (unsigned)(S::ROWS * 16 * b);
-                const unsigned x_bytes = (unsigned)(NT * DQ_KB * 2);
-                const unsigned bar = dq_smem_u32(full + st);
-                unsigned char* stage = smem + st * S::STAGE;
-                dq_mbar_expect_tx(bar, code_bytes + x_bytes);
-                dq_bulk_load(dq_smem_u32(stage + S::X_STAGE), a.packed + word0 + blk_word[j], code_bytes, bar);
-                dq_bulk_load(dq_smem_u32(stage),
-                             a.xp + dq_order_base(o, a.nbc, NT) + (int64_t)(j0 + j) * (NT * DQ_KB),
-                             x_bytes, bar);
-            }
+        // ---- loader warp: the codes of block j as they lie in memory and its slice of X (an image in
+        // the order of the block's bitwidth) by two bulk copies of lane 0, the rows' (scale, minimum) by
+        // 8-byte asynchronous copies of all lanes, into the ring as soon as the blocks whose entries are
+        // in the way have been let go of by every contraction warp ------------------------------------
+        for (jl = 0; jl < nblk && lok; ++jl) {
+            unsigned at;
+            if (!place(jl, true, at)) break;
+            __syncwarp();
+            load_codes_meta(jl, at);
+            load_image(jl, at);
+            __syncwarp();
         }
     } else {
-        // ---- contraction warps: 16 weight rows each -----------------------------------------------------
+        // ---- contraction warps: 16 MT weight rows each --------------------------------------------------
         const int g = lane >> 2, t = lane & 3;
-        const int64_t row_lo = (int64_t)bi * S::ROWS + warp * 16 + g;        // and row_lo + 8
-        // the lane's ldmatrix row inside an image, without the stage and the row pitch (which depends
-        // on the block's order): matrix mi = lane / 8, row r8 = lane % 8
+        const int64_t row_lo = (int64_t)bi * S::ROWS + warp * (16 * MT) + g;   // rows row_lo + 16 m + 8 h
+        // the lane's ldmatrix row inside an image, without the stage: matrix mi = lane / 8, row r8 = lane % 8
         const int mi = lane >> 3, r8 = lane & 7;
-        float y[NT / 8][4];
+        constexpr unsigned pitch = 2u * DQ_KB;                          // bytes of an image row
+        unsigned xoff[2];
+        if constexpr (NT == 8) {
+            // matrices: (step, low half), (step, high half), (step + 1, low), (step + 1, high) of tokens 0..7
+            xoff[0] = ((unsigned)r8 * pitch + (unsigned)((((mi & 1) ^ r8) << 4))) ^ (unsigned)((mi >> 1) << 5);
+            xoff[1] = 0;
+        } else {
+            // matrices: tokens 16 q + 8 (mi / 2) .., low (mi even) or high (mi odd) half of the step
 #pragma unroll
-        for (int nt = 0; nt < NT / 8; ++nt) y[nt][0] = y[nt][1] = y[nt][2] = y[nt][3] = 0.f;
+            for (int q = 0; q < 2; ++q)
+                xoff[q] = (unsigned)(16 * q + 8 * (mi >> 1) + r8) * pitch + (unsigned)(((mi & 1) ^ r8) << 4);
+        }
+        float y[MT][NT / 8][4];
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+#pragma unroll
+            for (int nt = 0; nt < NT / 8; ++nt) y[m][nt][0] = y[m][nt][1] = y[m][nt][2] = y[m][nt][3] = 0.f;
         bool ok = true;
-        float2 m0 = a.meta[row_lo * a.nbc + j0], m1 = a.meta[(row_lo + 8) * a.nbc + j0];
         for (int j = 0; j < nblk && ok; ++j) {
-            const float2 c0 = m0, c1 = m1;
-            if (j + 1 < nblk) {
-                m0 = a.meta[row_lo * a.nbc + j0 + j + 1];
-                m1 = a.meta[(row_lo + 8) * a.nbc + j0 + j + 1];
-            }
-            const int st = j % RING;
-            DQ_TL(warp, j, 0);
-            ok = dq_mbar_wait(dq_smem_u32(full + st), (unsigned)(j / RING) & 1u, abort_flag);
+            ok = dq_mbar_wait(dq_smem_u32(full + j), 0u, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
-            DQ_TL(warp, j, 1);
             if (!ok) break;
             const int b = blk_bits[j];                       // uniform over the CTA
-            const unsigned stage = dq_smem_u32(smem + st * S::STAGE);
-            const unsigned codes = stage + S::X_STAGE + (unsigned)(warp * 16 * 16 * b);
-            constexpr unsigned pitch = 2u * DQ_KB;                          // bytes of an image row
-            unsigned xlane[2];
-            if constexpr (NT == 8) {
-                // matrices: (step, low half), (step, high half), (step + 1, low), (step + 1, high) of tokens 0..7
-                xlane[0] = (stage + (unsigned)r8 * pitch + (unsigned)((((mi & 1) ^ r8) << 4))) ^ (unsigned)((mi >> 1) << 5);
-                xlane[1] = 0;
-            } else {
-                // matrices: tokens 16 q + 8 (mi / 2) .., low (mi even) or high (mi odd) half of the step
-#pragma unroll
-                for (int q = 0; q < 2; ++q)
-                    xlane[q] = stage + (unsigned)(16 * q + 8 * (mi >> 1) + r8) * pitch + (unsigned)(((mi & 1) ^ r8) << 4);
-            }
-            const unsigned eb = dq_smem_u32(empty + st);
+            const unsigned stage = dq_smem_u32(smem) + blk_at[j];
+            const unsigned codes = stage + S::X_BYTES + (unsigned)(warp * (16 * MT) * 16 * b);
+            const unsigned metas = stage + S::X_BYTES + (unsigned)(S::ROWS * 16 * b);
+            const unsigned xlane[2] = {stage + xoff[0], stage + xoff[1]};
+            const unsigned eb = dq_smem_u32(empty + j);
             const unsigned xa = dq_smem_u32(xs + j * NT + 2 * t);
+            // (scale, minimum) of rows 16 m + 8 h + g of the warp
+            float2 cur[MT][2];
+#pragma unroll
+            for (int m = 0; m < MT; ++m)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint2 v = dq_lds64(metas + 8u * (unsigned)(warp * (16 * MT) + 16 * m + 8 * h + g));
+                    cur[m][h] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
+                }
             switch (b) {
-                case 1: dq_block<1, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
-                case 2: dq_block<2, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
-                case 3: dq_block<3, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
-                case 4: dq_block<4, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
-                case 5: dq_block<5, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
-                case 6: dq_block<6, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
-                case 7: dq_block<7, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
-                default: dq_block<8, NT>(codes, xlane, g, t, eb, lane, c0, c1, xa, y); break;
+                case 1: dq_block<1, NT, MT>(codes, xlane, g, t, eb, lane, cur, xa, y); break;
+                case 2: dq_block<2, NT, MT>(codes, xlane, g, t, eb, lane, cur, xa, y); break;
+                case 3: dq_block<3, NT, MT>(codes, xlane, g, t, eb, lane, cur, xa, y); break;
+                case 4: dq_block<4, NT, MT>(codes, xlane, g, t, eb, lane, cur, xa, y); break;
+                case 5: dq_block<5, NT, MT>(codes, xlane, g, t, eb, lane, cur, xa, y); break;
+                case 6: dq_block<6, NT, MT>(codes, xlane, g, t, eb, lane, cur, xa, y); break;
+                case 7: dq_block<7, NT, MT>(codes, xlane, g, t, eb, lane, cur, xa, y); break;
+                default: dq_block<8, NT, MT>(codes, xlane, g, t, eb, lane, cur, xa, y); break;
             }
-            DQ_TL(warp, j, 2);
         }
-        if (ok) {
+        if (a.cluster_sum) {
+            // all of the CTA's warps are past their last block before the ring's memory is reused
+            asm volatile("bar.sync 1, %0;" ::"r"(WARPS * 32) : "memory");
+            float* ysm = reinterpret_cast<float*>(smem);                 // [NT][ROWS] partial sums of the segment
+#pragma unroll
+            for (int m = 0; m < MT; ++m)
+#pragma unroll
+                for (int nt = 0; nt < NT / 8; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        ysm[(8 * nt + 2 * t + (e & 1)) * S::ROWS + warp * (16 * MT) + 16 * m + 8 * (e >> 1) + g] =
+                            ok ? y[m][nt][e] : 0.f;
+        } else if (ok) {
             float* out = a.out + (int64_t)blockIdx.y * a.out_seg_stride;
 #pragma unroll
-            for (int nt = 0; nt < NT / 8; ++nt) {
+            for (int m = 0; m < MT; ++m) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int tok = 8 * nt + 2 * t + (e & 1);
-                    if (!isfinite(y[nt][e])) sb_latch(a.ds, SB_ERR_NONFINITE, SBK_GEMM);
-                    if (tok < a.T) out[(int64_t)tok * a.out_t_stride + row_lo + 8 * (e >> 1)] = y[nt][e];
+                for (int nt = 0; nt < NT / 8; ++nt) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int tok = 8 * nt + 2 * t + (e & 1);
+                        if (!isfinite(y[m][nt][e])) sb_latch(a.ds, SB_ERR_NONFINITE, SBK_GEMM);
+                        if (tok < a.T) out[(int64_t)tok * a.out_t_stride + row_lo + 16 * m + 8 * (e >> 1)] = y[m][nt][e];
+                    }
                 }
             }
         }
     }
+    if (a.cluster_sum) {
+        // the segments of this row tile are the CTAs of one cluster, rank = segment: every CTA adds a
+        // slice of the tile's outputs over all segments, in segment order, out of their shared memory
+        cg::cluster_group cluster = cg::this_cluster();
+        cluster.sync();
+        const float* ysm = reinterpret_cast<const float*>(smem);
+        const int nseg = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+        const int total = a.T * S::ROWS, chunk = (total + nseg - 1) / nseg;
+        const int end = min(total, (rank + 1) * chunk);
+        for (int idx = rank * chunk + (int)threadIdx.x; idx < end; idx += S::THREADS) {
+            float acc = 0.f;
+            for (int sgm = 0; sgm < nseg; ++sgm) acc += *cluster.map_shared_rank(ysm + idx, sgm);
+            if (!isfinite(acc)) sb_latch(a.ds, SB_ERR_NONFINITE, SBK_GEMM);
+            a.out[(int64_t)(idx / S::ROWS) * a.out_t_stride + (int64_t)bi * S::ROWS + idx % S::ROWS] = acc;
+        }
+        cluster.sync();                     // nobody leaves while its shared memory may still be read
+    }
     __syncthreads();
-#ifdef SB_EXP_TL
-    if (threadIdx.x == 0) dq_cta[blockIdx.y * gridDim.x + blockIdx.x][1] = dq_now_ns();
-#endif
     if (threadIdx.x == 0 && *abort_flag) sb_latch(a.ds, SB_ERR_TIMEOUT, SBK_GEMM);
 }
 
@@ -553,27 +637,42 @@ __global__ void dq_reduce_kernel(const float* __restrict__ part, int S, int T, i
     Y[(int64_t)t * ldy + r] = acc;
 }
 
-// resident CTAs per SM of the instance that serves (tokens padded to NT, block rows)
-int dq_ctas_per_sm(int NT, int br) {
-    if (br == 128) return NT == 8 ? DqShape<8, 8>::CTAS_PER_SM : NT == 16 ? DqShape<16, 8>::CTAS_PER_SM : DqShape<32, 8>::CTAS_PER_SM;
-    return NT == 8 ? DqShape<8, 4>::CTAS_PER_SM : NT == 16 ? DqShape<16, 4>::CTAS_PER_SM : DqShape<32, 4>::CTAS_PER_SM;
-}
-
 template <int NT, int WARPS>
 sb_status dq_launch(sb_ctx* ctx, const DqArgs& a, dim3 grid) {
-    using S = DqShape<NT, WARPS>;
-    SB_FUNC_ATTR(ctx, (dequant_gemm_kernel<NT, WARPS>), cudaFuncAttributeMaxDynamicSharedMemorySize, S::SMEM);
-    dequant_gemm_kernel<NT, WARPS><<<grid, S::THREADS, S::SMEM, ctx->stream>>>(a);
+    using S = DqShape<NT, WARPS, DQ_MT>;
+    SB_FUNC_ATTR(ctx, (dequant_gemm_kernel<NT, WARPS, DQ_MT>), cudaFuncAttributeMaxDynamicSharedMemorySize, S::SMEM);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(S::THREADS);
+    cfg.dynamicSmemBytes = S::SMEM;
+    cfg.stream = ctx->stream;
+    cudaLaunchAttribute attr[1];
+    cfg.numAttrs = 0;
+    if (a.cluster_sum) {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 1;
+        attr[0].val.clusterDim.y = grid.y;
+        attr[0].val.clusterDim.z = 1;
+        cfg.numAttrs = 1;
+    }
+    cfg.attrs = attr;
+    SB_CUDA(ctx, cudaLaunchKernelEx(&cfg, dequant_gemm_kernel<NT, WARPS, DQ_MT>, a));
     SB_LAUNCHED(ctx);
     return SB_OK;
+}
+// contraction warps of a CTA for blocks of br rows; resident CTAs per SM of the instance that
+// serves (tokens padded to NT, block rows)
+constexpr int dq_warps(int br) { return br / (16 * DQ_MT); }
+int dq_ctas_per_sm(int NT, int br) {
+    if (br == 128)
+        return NT == 8 ? DqShape<8, dq_warps(128), DQ_MT>::CTAS_PER_SM
+                       : NT == 16 ? DqShape<16, dq_warps(128), DQ_MT>::CTAS_PER_SM : DqShape<32, dq_warps(128), DQ_MT>::CTAS_PER_SM;
+    return NT == 8 ? DqShape<8, dq_warps(64), DQ_MT>::CTAS_PER_SM
+                   : NT == 16 ? DqShape<16, dq_warps(64), DQ_MT>::CTAS_PER_SM : DqShape<32, dq_warps(64), DQ_MT>::CTAS_PER_SM;
 }
 
 }  // namespace
 
-#ifdef SB_EXP_TL
-extern "C" int sb_dq_timeline(long long* dst) { return (int)cudaMemcpyFromSymbol(dst, dq_tl, sizeof(dq_tl)); }
-extern "C" int sb_dq_ctas(unsigned long long* dst) { return (int)cudaMemcpyFromSymbol(dst, dq_cta, sizeof(dq_cta)); }
-#endif
 
 extern "C" sb_status sb_dequant_gemm(sb_ctx* ctx, const void* X, int64_t T, int64_t ldx, const uint32_t* packed,
                                      const int64_t* block_off_words, const float* meta, const uint8_t* level,
@@ -602,6 +701,10 @@ extern "C" sb_status sb_dequant_gemm(sb_ctx* ctx, const void* X, int64_t T, int6
     if (S > 65535) return sb_fail(ctx, SB_ERR_SHAPE, "dequant gemm: too many column segments");
     DqBits db{};
     for (int l = 0; l < n_bits; ++l) db.packed |= (unsigned)bits[l] << (4 * l);
+    // how the segments of a row tile are added: as one (portable) cluster through shared memory, or by
+    // a second kernel over partial sums in scratch
+    const bool cluster_sum = S >= 2 && S <= 8;
+    const bool two_pass = S > 1 && !cluster_sum;
     // tokens in slices of at most DQ_MAX_T (padded to 8, 16 or 32 with zero rows)
     for (int64_t t0 = 0; t0 < T; t0 += DQ_MAX_T) {
         const int Tn = (int)((T - t0) < DQ_MAX_T ? (T - t0) : DQ_MAX_T);
@@ -609,12 +712,12 @@ extern "C" sb_status sb_dequant_gemm(sb_ctx* ctx, const void* X, int64_t T, int6
         const size_t image_elems = (size_t)DQ_ORDERS * NT * C;
         void* arena;
         sb_status st = sb_scratch(ctx, Carver::need({image_elems * 2, (size_t)nbc * NT * 4,
-                                                     S > 1 ? (size_t)S * Tn * R * 4 : 0}), &arena);
+                                                     two_pass ? (size_t)S * Tn * R * 4 : 0}), &arena);
         if (st != SB_OK) return st;
         Carver cv(arena);
         __nv_bfloat16* xp = cv.take<__nv_bfloat16>(image_elems);
         float* xsum = cv.take<float>((size_t)nbc * NT);
-        float* part = S > 1 ? cv.take<float>((size_t)S * Tn * R) : nullptr;
+        float* part = two_pass ? cv.take<float>((size_t)S * Tn * R) : nullptr;
         const __nv_bfloat16* Xs = static_cast<const __nv_bfloat16*>(X) + t0 * ldx;
         if (Tn < NT) {      // zero rows for the padding tokens
             SB_CUDA(ctx, cudaMemsetAsync(xp, 0, image_elems * 2, ctx->stream));
@@ -625,20 +728,23 @@ extern "C" sb_status sb_dequant_gemm(sb_ctx* ctx, const void* X, int64_t T, int6
         DqArgs a{};
         a.packed = packed; a.block_off = block_off_words; a.meta = reinterpret_cast<const float2*>(meta);
         a.level = level; a.xp = xp; a.xsum = xsum;
-        a.out = S > 1 ? part : Y + t0 * ldy;
-        a.out_t_stride = S > 1 ? R : ldy;
-        a.out_seg_stride = S > 1 ? (int64_t)Tn * R : 0;
+        a.cluster_sum = cluster_sum ? 1 : 0;
+        a.out = two_pass ? part : Y + t0 * ldy;
+        a.out_t_stride = two_pass ? R : ldy;
+        a.out_seg_stride = two_pass ? (int64_t)Tn * R : 0;
         a.R = R; a.C = C; a.nbc = nbc; a.seg_blocks = seg_blocks; a.T = Tn; a.bits = db; a.ds = ctx->dstate;
         const dim3 grid((unsigned)nbr, (unsigned)S);
         if (br == 128) {
-            st = NT == 8 ? dq_launch<8, 8>(ctx, a, grid) : NT == 16 ? dq_launch<16, 8>(ctx, a, grid)
-                                                                    : dq_launch<32, 8>(ctx, a, grid);
+            constexpr int W = dq_warps(128);
+            st = NT == 8 ? dq_launch<8, W>(ctx, a, grid) : NT == 16 ? dq_launch<16, W>(ctx, a, grid)
+                                                                    : dq_launch<32, W>(ctx, a, grid);
         } else {
-            st = NT == 8 ? dq_launch<8, 4>(ctx, a, grid) : NT == 16 ? dq_launch<16, 4>(ctx, a, grid)
-                                                                    : dq_launch<32, 4>(ctx, a, grid);
+            constexpr int W = dq_warps(64);
+            st = NT == 8 ? dq_launch<8, W>(ctx, a, grid) : NT == 16 ? dq_launch<16, W>(ctx, a, grid)
+                                                                    : dq_launch<32, W>(ctx, a, grid);
         }
         if (st != SB_OK) return st;
-        if (S > 1) {
+        if (two_pass) {
             dq_reduce_kernel<<<dim3((unsigned)((R + 255) / 256), (unsigned)Tn), 256, 0, ctx->stream>>>(part, S, Tn, R,
                                                                                                        Y + t0 * ldy, ldy);
             SB_LAUNCHED(ctx);
