@@ -228,17 +228,18 @@ sb_status sb_calib_gram(sb_ctx* ctx, const void* X_bf16, int64_t T, int64_t K, i
 /* Block error table with the full second-moment matrix (Section 3.2 with the cross terms
  * between input channels kept), on the permuted layout W' = W[row_perm][:, col_perm]:
  *     err[i][l]  = sum over rows r of block i of  d_r H'_JJ d_r^T,
- *                  d_r = (W' - Q_{b_l}(W'))[r, J],  J = the block's 128 columns,
+ *                  d_r = (W' - Q_{b_l}(W'))[r, J],  J = the block's columns,
  *                  H'_JJ[a][b] = H[col_perm[J0 + a]][col_perm[J0 + b]]
- *     gain[i][l] = (err[i][l] - err[i][l+1]) / ((b_{l+1} - b_l) * 128 * 128)
+ *     gain[i][l] = (err[i][l] - err[i][l+1]) / ((b_{l+1} - b_l) * block_rows * block_cols)
  * H: device fp32 [C][C] in the ORIGINAL column order (sb_calib_gram); symmetric.  With a
  * diagonal H this is sb_block_scores with col_moment = diag(H).  row_weight: [R] device fp32
  * by ORIGINAL row (non-negative) or NULL = 1: err sums a_r d_r H'_JJ d_r^T.  Blocks are 64, 128
- * or 256 rows x 128 columns (block_cols = 128 is required; 64 x 128 is the paper's default
- * partition, Section 5 "Implementation"), group in {16,32,64,128}; gain divides by
- * block_rows * 128.  The 128 x 128 Gram matrix of every (128-row unit, candidate) residual is a
+ * or 256 rows x 64 or 128 columns (64 x 128 is the paper's default partition, Section 5
+ * "Implementation"; C must be a multiple of 128), group in {16,32,64,128} and at most the block
+ * width.  The 128 x 128 Gram matrix of every (128 rows x 128 columns, candidate) residual is a
  * tensor-core contraction of two bf16 terms of the residual (relative error about 2^-16); a
- * 64-row block contracts 64 zero rows along, a 256-row block is the sum of two units.  err, gain
+ * 64-row block contracts 64 zero rows along, a 256-row block is the sum of two units, two
+ * 64-column blocks side by side take the two diagonal quadrants of one Gram matrix.  err, gain
  * (or NULL) and W_perm_out (or NULL) as in sb_block_scores.  A pipeline wait that does not
  * complete within 2 s latches SB_ERR_TIMEOUT.  Asynchronous.                                  */
 sb_status sb_block_scores_full(sb_ctx* ctx, const void* W_bf16, int64_t R, int64_t C, int64_t ldw,

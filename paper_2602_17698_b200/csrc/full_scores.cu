@@ -142,7 +142,7 @@ template <int GROUP, bool PLAIN>
 __global__ void __launch_bounds__(FS_THREADS, 1)
 full_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const float* __restrict__ hblk,
                    FsBits fb, int L, int64_t n_blocks, int64_t n_block_cols, int unit_rows,
-                   const float* __restrict__ row_weight, const int32_t* __restrict__ a_perm, float gain_elems,
+                   const float* __restrict__ row_weight, const int32_t* __restrict__ a_perm, float gain_elems, int halves,
                    float* __restrict__ err, float* __restrict__ gain, SbDeviceState* ds) {
     // A work unit is `unit_rows` (64 or 128) rows x 128 columns; the contraction always runs over 128
     // rows, the rows past unit_rows of a 64-row unit are written as zeros (they add nothing).
@@ -223,7 +223,16 @@ full_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const float
         for (int q4 = 0; q4 < 4; ++q4) e += (rr[4 * q4] + rr[4 * q4 + 1]) + (rr[4 * q4 + 2] + rr[4 * q4 + 3]);
         const int64_t blk = bi_f * n_block_cols + bj_f;
         if (!isfinite(e)) sb_latch(ds, SB_ERR_NONFINITE, SBK_SCORES);
-        err[blk * L + l_f] = e;
+        if (!PLAIN && halves == 2) {
+            // blocks of 64 columns: the unit holds two of them side by side; each takes the diagonal
+            // quadrant of the 128 x 128 Gram matrix that belongs to its own columns (warps 0, 1, 4, 5 hold
+            // rows and columns 0..63, warps 10, 11, 14, 15 rows and columns 64..127), the cross
+            // quadrants belong to no block
+            err[(blk * 2) * L + l_f] = (rr[0] + rr[1]) + (rr[4] + rr[5]);
+            err[(blk * 2 + 1) * L + l_f] = (rr[10] + rr[11]) + (rr[14] + rr[15]);
+        } else {
+            err[blk * L + l_f] = e;
+        }
         if (gain && l_f > 0)
             gain[blk * (L - 1) + l_f - 1] =
                 (e_prev - e) / ((float)(fs_bits(fb, l_f) - fs_bits(fb, l_f - 1)) * gain_elems);
@@ -430,17 +439,21 @@ full_scores_kernel(const __nv_bfloat16* __restrict__ W, int64_t ldw, const float
     if (threadIdx.x == 0 && *abort_flag) sb_latch(ds, SB_ERR_TIMEOUT, SBK_SCORES);
 }
 
-// blocks of 256 rows: err[blk][l] = the sum of the block's two 128-row units; gains
-__global__ void full_combine_kernel(const float* __restrict__ unit_err, int64_t n_blocks, int64_t nbc, int L,
-                                    FsBits fb, float gain_elems, float* __restrict__ err, float* __restrict__ gain) {
+// blocks that are not one contraction unit: err[blk][l] = the sum over the block's units (two for
+// 256-row blocks) of the unit's entry for the block's half (two halves per unit for 64-column
+// blocks); gains
+__global__ void full_combine_kernel(const float* __restrict__ unit_err, int64_t n_blocks, int64_t nbc_blocks,
+                                    int64_t nbc_units, int units_per_block, int halves, int L, FsBits fb,
+                                    float gain_elems, float* __restrict__ err, float* __restrict__ gain) {
     const int64_t blk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (blk >= n_blocks) return;
-    const int64_t bi = blk / nbc, bj = blk - bi * nbc;
-    const float* u0 = unit_err + ((2 * bi) * nbc + bj) * L;
-    const float* u1 = unit_err + ((2 * bi + 1) * nbc + bj) * L;
+    const int64_t bi = blk / nbc_blocks, bjb = blk - bi * nbc_blocks;
+    const int64_t bj = bjb / halves, half = bjb - bj * halves;
     float prev = 0.f;
     for (int l = 0; l < L; ++l) {
-        const float e = u0[l] + u1[l];
+        float e = 0.f;
+        for (int u = 0; u < units_per_block; ++u)
+            e += unit_err[(((bi * units_per_block + u) * nbc_units + bj) * halves + half) * L + l];
         err[blk * L + l] = e;
         if (gain && l > 0) gain[blk * (L - 1) + l - 1] = (prev - e) / ((float)(fs_bits(fb, l) - fs_bits(fb, l - 1)) * gain_elems);
         prev = e;
@@ -457,19 +470,21 @@ extern "C" sb_status sb_block_scores_full(sb_ctx* ctx, const void* W, int64_t R,
     if (!W || !H || !err || R <= 0 || C <= 0) return sb_fail(ctx, SB_ERR_INVALID, "full scores: null or empty");
     if (!sb_check_bits(bits, n_bits)) return sb_fail(ctx, SB_ERR_INVALID, "full scores: bits must be ascending in 1..8");
     const bool g_ok = group == 16 || group == 32 || group == 64 || group == 128;
-    if (!(br == 64 || br == 128 || br == 256) || bc != FS_N || !g_ok || R % br || C % FS_N || ldw % 8 || ldw < C ||
-        (reinterpret_cast<uintptr_t>(W) & 15))
-        return sb_fail(ctx, SB_ERR_SHAPE, "full scores: blocks of 64, 128 or 256 rows x 128 columns tiling the matrix, "
-                                          "group in {16,32,64,128}");
+    if (!(br == 64 || br == 128 || br == 256) || !(bc == 64 || bc == FS_N) || !g_ok || group > bc || R % br || C % FS_N ||
+        ldw % 8 || ldw < C || (reinterpret_cast<uintptr_t>(W) & 15))
+        return sb_fail(ctx, SB_ERR_SHAPE, "full scores: blocks of 64, 128 or 256 rows x 64 or 128 columns tiling the "
+                                          "matrix (C a multiple of 128), group in {16,32,64,128} and at most the block width");
     SB_CUDA(ctx, cudaSetDevice(ctx->device));
     const int unit_rows = br < FS_N ? br : FS_N;                 // rows of one contraction
     const int units_per_block = br / unit_rows;                  // 1, or 2 for 256-row blocks
-    const int64_t nbc = C / FS_N, n_units = (R / unit_rows) * nbc, n_blocks = (R / br) * nbc;
+    const int halves = FS_N / bc;                                // 64-column blocks: two side by side in a unit
+    const int64_t nbc = C / FS_N, n_units = (R / unit_rows) * nbc, n_blocks = (R / br) * (C / bc);
+    const bool combine = units_per_block > 1 || halves > 1;
     const bool need_copy = row_perm || col_perm || W_perm_out;
     void* arena;
     sb_status st = sb_scratch(ctx, Carver::need({(size_t)nbc * FS_N * FS_N * 4,
                                                  (need_copy && !W_perm_out) ? (size_t)R * C * 2 : 0,
-                                                 units_per_block > 1 ? (size_t)n_units * n_bits * 4 : 0}), &arena);
+                                                 combine ? (size_t)n_units * halves * n_bits * 4 : 0}), &arena);
     if (st != SB_OK) return st;
     Carver cv(arena);
     float* hblk = cv.take<float>((size_t)nbc * FS_N * FS_N);
@@ -482,20 +497,20 @@ extern "C" sb_status sb_block_scores_full(sb_ctx* ctx, const void* W, int64_t R,
         src = static_cast<const __nv_bfloat16*>(dst);
         ld = C;
     }
-    float* unit_err = units_per_block > 1 ? cv.take<float>((size_t)n_units * n_bits) : err;
+    float* unit_err = combine ? cv.take<float>((size_t)n_units * halves * n_bits) : err;
     gather_hblocks_kernel<<<(unsigned)nbc, 256, 0, ctx->stream>>>(H, C, col_perm, hblk);
     SB_LAUNCHED(ctx);
     FsBits fb{};
     for (int l = 0; l < n_bits; ++l) fb.packed |= (unsigned)bits[l] << (4 * l);
     const int64_t grid = n_units < ctx->sm_count ? n_units : ctx->sm_count;
-    const float gain_elems = (float)br * (float)FS_N;
-    float* kernel_gain = units_per_block > 1 ? nullptr : gain;
-    const bool plain = unit_rows == FS_N && !row_weight;
+    const float gain_elems = (float)br * (float)bc;
+    float* kernel_gain = combine ? nullptr : gain;
+    const bool plain = unit_rows == FS_N && !row_weight && halves == 1;
 #define FS_LAUNCH_P(G, P)                                                                                         \
     do {                                                                                                          \
         SB_FUNC_ATTR(ctx, (full_scores_kernel<G, P>), cudaFuncAttributeMaxDynamicSharedMemorySize, FS_SMEM);      \
         full_scores_kernel<G, P><<<(unsigned)grid, FS_THREADS, FS_SMEM, ctx->stream>>>(                           \
-            src, ld, hblk, fb, n_bits, n_units, nbc, unit_rows, row_weight, row_perm, gain_elems, unit_err,       \
+            src, ld, hblk, fb, n_bits, n_units, nbc, unit_rows, row_weight, row_perm, gain_elems, halves, unit_err, \
             kernel_gain, ctx->dstate);                                                                            \
     } while (0)
 #define FS_LAUNCH(G)                                                                                              \
@@ -511,9 +526,9 @@ extern "C" sb_status sb_block_scores_full(sb_ctx* ctx, const void* W, int64_t R,
 #undef FS_LAUNCH
 #undef FS_LAUNCH_P
     SB_LAUNCHED(ctx);
-    if (units_per_block > 1) {
-        full_combine_kernel<<<(unsigned)((n_blocks + 255) / 256), 256, 0, ctx->stream>>>(unit_err, n_blocks, nbc, n_bits, fb,
-                                                                                         gain_elems, err, gain);
+    if (combine) {
+        full_combine_kernel<<<(unsigned)((n_blocks + 255) / 256), 256, 0, ctx->stream>>>(
+            unit_err, n_blocks, C / bc, nbc, units_per_block, halves, n_bits, fb, gain_elems, err, gain);
         SB_LAUNCHED(ctx);
     }
     return SB_OK;

@@ -142,14 +142,18 @@ def test_full_scores_sampled_blocks_of_a_layer_sized_matrix(ctx):
         assert np.all(np.abs(got[blk:blk + 1] - ref) <= REL * np.abs(ref)), (blk, got[blk], ref)
 
 
-@pytest.mark.parametrize("R,C,br,g,bits,weights,perm", [
-    (512, 384, 64, 128, [2, 3, 4, 8], False, False),     # the paper's default partition, 64 x 128
-    (1024, 256, 64, 32, [2, 3, 4], True, True),
-    (1024, 384, 256, 64, [2, 3, 4, 8], False, True),     # 256 x 128: two contraction units per block
-    (512, 256, 256, 128, [3, 4], True, False),
-    (512, 512, 128, 128, [2, 3, 4, 8], True, True),      # row weights on the 128 x 128 form
+@pytest.mark.parametrize("R,C,br,bc,g,bits,weights,perm", [
+    (512, 384, 64, 128, 128, [2, 3, 4, 8], False, False),     # the paper's default partition, 64 x 128
+    (1024, 256, 64, 128, 32, [2, 3, 4], True, True),
+    (1024, 384, 256, 128, 64, [2, 3, 4, 8], False, True),     # 256 x 128: two contraction units per block
+    (512, 256, 256, 128, 128, [3, 4], True, False),
+    (512, 512, 128, 128, 128, [2, 3, 4, 8], True, True),      # row weights on the 128 x 128 form
+    (512, 384, 64, 64, 64, [2, 3, 4, 8], False, False),       # 64-column blocks: two side by side in a unit
+    (512, 256, 128, 64, 32, [2, 3, 4], True, True),
+    (1024, 384, 256, 64, 64, [2, 4, 8], False, True),
+    (1280, 4096, 64, 64, 16, [3, 4], True, False),            # more units than CTAs
 ])
-def test_full_scores_block_heights_and_row_weights(ctx, R, C, br, g, bits, weights, perm):
+def test_full_scores_block_shapes_and_row_weights(ctx, R, C, br, bc, g, bits, weights, perm):
     from tests.helpers import REL
     W = synth.make_weight(R, C, 91 + R + br, DEV)
     X = synth.make_activations(1024, C, 93 + C, DEV)
@@ -158,19 +162,19 @@ def test_full_scores_block_heights_and_row_weights(ctx, R, C, br, g, bits, weigh
     pr = torch.from_numpy(rng.permutation(R).astype(np.int32)).to(DEV) if perm else None
     pc = torch.from_numpy(rng.permutation(C).astype(np.int32)).to(DEV) if perm else None
     a = (torch.rand(R, device=DEV) * 3 + 0.1) if weights else None
-    err, gain = ctx.block_scores_full(W, H, bits, br, 128, g, row_perm=pr, col_perm=pc, row_weight=a)
+    err, gain = ctx.block_scores_full(W, H, bits, br, bc, g, row_perm=pr, col_perm=pc, row_weight=a)
     ctx.sync()
-    ref = sbo.block_scores_full(W.cpu(), H.cpu().double().numpy(), bits, br, 128, g,
+    ref = sbo.block_scores_full(W.cpu(), H.cpu().double().numpy(), bits, br, bc, g,
                                 row_perm=None if pr is None else pr.cpu().numpy(),
                                 col_perm=None if pc is None else pc.cpu().numpy(),
                                 a=None if a is None else a.cpu().double().numpy())
     got = err.cpu().double().numpy()
-    assert got.shape == ref.shape == ((R // br) * (C // 128), len(bits))
+    assert got.shape == ref.shape == ((R // br) * (C // bc), len(bits))
     assert np.all(np.abs(got - ref) <= REL * np.abs(ref)), np.max(np.abs(got - ref) / np.abs(ref))
-    gref = (ref[:, :-1] - ref[:, 1:]) / (np.diff(bits)[None, :] * br * 128)
-    tol = REL * (np.abs(ref[:, :-1]) + np.abs(ref[:, 1:])) / (np.diff(bits)[None, :] * br * 128)
+    gref = (ref[:, :-1] - ref[:, 1:]) / (np.diff(bits)[None, :] * br * bc)
+    tol = REL * (np.abs(ref[:, :-1]) + np.abs(ref[:, 1:])) / (np.diff(bits)[None, :] * br * bc)
     assert np.all(np.abs(gain.cpu().double().numpy() - gref) <= tol)
-    e2, _ = ctx.block_scores_full(W, H, bits, br, 128, g, row_perm=pr, col_perm=pc, row_weight=a)
+    e2, _ = ctx.block_scores_full(W, H, bits, br, bc, g, row_perm=pr, col_perm=pc, row_weight=a)
     ctx.sync()
     assert torch.equal(err, e2)                       # deterministic
 
