@@ -614,9 +614,17 @@ dequant_gemm_kernel(const DqArgs a) {
         const int nseg = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
         const int total = a.T * S::ROWS, chunk = (total + nseg - 1) / nseg;
         const int end = min(total, (rank + 1) * chunk);
+        // the remote reads of an output are issued together (up to 8 segments), then added in order
+        const float* seg[8];
+#pragma unroll
+        for (int sgm = 0; sgm < 8; ++sgm) seg[sgm] = cluster.map_shared_rank(ysm, sgm < nseg ? sgm : 0);
         for (int idx = rank * chunk + (int)threadIdx.x; idx < end; idx += S::THREADS) {
+            float v[8];
+#pragma unroll
+            for (int sgm = 0; sgm < 8; ++sgm) v[sgm] = sgm < nseg ? seg[sgm][idx] : 0.f;
             float acc = 0.f;
-            for (int sgm = 0; sgm < nseg; ++sgm) acc += *cluster.map_shared_rank(ysm + idx, sgm);
+#pragma unroll
+            for (int sgm = 0; sgm < 8; ++sgm) acc += v[sgm];
             if (!isfinite(acc)) sb_latch(a.ds, SB_ERR_NONFINITE, SBK_GEMM);
             a.out[(int64_t)(idx / S::ROWS) * a.out_t_stride + (int64_t)bi * S::ROWS + idx % S::ROWS] = acc;
         }
