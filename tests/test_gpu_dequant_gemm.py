@@ -98,6 +98,15 @@ def test_many_column_segments_and_a_ragged_last_one(ctx):
     _run(ctx, 128, 128 * 70, 16, [4], seed=8)
 
 
+@pytest.mark.parametrize("R,Cc,T,br", [(4096, 1024, 32, 128),      # 32 row tiles x 8 segments of one block: clusters of 8
+                                        (8192, 1024, 16, 64),       # 128 row tiles of 64 rows x 4 segments
+                                        (2048, 2560, 8, 128)])      # 16 x 18 CTAs: 20 blocks in segments of 2, partial sums
+def test_segments_added_inside_a_cluster_and_by_the_second_kernel(ctx, R, Cc, T, br):
+    """With 2 to 8 column segments the segments of a row tile are one cluster and are added through
+    shared memory; with more they go through partial sums and a second kernel."""
+    _run(ctx, R, Cc, T, [2, 4, 8], seed=R + Cc + br, br=br)
+
+
 def test_deterministic(ctx):
     a, _ = _run(ctx, 256, 1024, 32, [2, 4, 8], seed=3)
     b, _ = _run(ctx, 256, 1024, 32, [2, 4, 8], seed=3)
