@@ -33,6 +33,7 @@ struct sb_ctx {
     void* pinned = nullptr;      // small pinned host buffer for read-backs
     size_t pinned_bytes = 0;
     unsigned int* moment_done = nullptr;   // per column chunk: row splits finished (zero between calls)
+    int moments_ctas_per_sm = 0;           // resident CTAs per SM of the moments kernel (asked once)
     unsigned int* stats_done = nullptr;    // per tile row / tile column: tiles finished (zero between calls)
     void* lb_mem = nullptr;      // look-back descriptors (context-owned, never in the arena)
     unsigned int lb_max_tiles = 0;
