@@ -668,9 +668,47 @@ sb_status dq_launch(sb_ctx* ctx, const DqArgs& a, dim3 grid) {
     SB_LAUNCHED(ctx);
     return SB_OK;
 }
+// Can a cluster of `segments` CTAs of this instance be resident at all (it can on a whole B200; a
+// partition with fewer SMs per GPC may not hold one)?  Asked from the occupancy calculator.
+template <int NT, int WARPS>
+bool dq_cluster_fits(sb_ctx* ctx, int segments) {
+    using S = DqShape<NT, WARPS, DQ_MT>;
+    const void* f = reinterpret_cast<const void*>(dequant_gemm_kernel<NT, WARPS, DQ_MT>);
+    if (!ctx->configured.count(f)) {
+        if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, S::SMEM) != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
+        ctx->configured.insert(f);
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(1, (unsigned)segments);
+    cfg.blockDim = dim3(S::THREADS);
+    cfg.dynamicSmemBytes = S::SMEM;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = (unsigned)segments;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, dequant_gemm_kernel<NT, WARPS, DQ_MT>, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return n >= 1;
+}
 // contraction warps of a CTA for blocks of br rows; resident CTAs per SM of the instance that
 // serves (tokens padded to NT, block rows)
 constexpr int dq_warps(int br) { return br / (16 * DQ_MT); }
+bool dq_cluster_ok(sb_ctx* ctx, int NT, int br, int segments) {
+    if (br == 128)
+        return NT == 8 ? dq_cluster_fits<8, dq_warps(128)>(ctx, segments)
+                       : NT == 16 ? dq_cluster_fits<16, dq_warps(128)>(ctx, segments) : dq_cluster_fits<32, dq_warps(128)>(ctx, segments);
+    return NT == 8 ? dq_cluster_fits<8, dq_warps(64)>(ctx, segments)
+                   : NT == 16 ? dq_cluster_fits<16, dq_warps(64)>(ctx, segments) : dq_cluster_fits<32, dq_warps(64)>(ctx, segments);
+}
 int dq_ctas_per_sm(int NT, int br) {
     if (br == 128)
         return NT == 8 ? DqShape<8, dq_warps(128), DQ_MT>::CTAS_PER_SM
@@ -711,7 +749,7 @@ extern "C" sb_status sb_dequant_gemm(sb_ctx* ctx, const void* X, int64_t T, int6
     for (int l = 0; l < n_bits; ++l) db.packed |= (unsigned)bits[l] << (4 * l);
     // how the segments of a row tile are added: as one (portable) cluster through shared memory, or by
     // a second kernel over partial sums in scratch
-    const bool cluster_sum = S >= 2 && S <= 8;
+    const bool cluster_sum = S >= 2 && S <= 8 && dq_cluster_ok(ctx, NT0, br, S);
     const bool two_pass = S > 1 && !cluster_sum;
     // tokens in slices of at most DQ_MAX_T (padded to 8, 16 or 32 with zero rows)
     for (int64_t t0 = 0; t0 < T; t0 += DQ_MAX_T) {
