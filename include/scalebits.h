@@ -321,8 +321,9 @@ sb_status sb_exchange_step(sb_ctx* ctx, const float* s_up, const float* s_down, 
  *     cudaStream_t (NULL = default stream).  Work is enqueued, not waited for.
  *   - K <= 65536; larger K returns SB_ERR_SCRATCH (and says so on stderr): split the columns
  *     across calls or use sb_calib_moments.  Other argument errors as in sb_calib_moments.
- *   - The first call on each device looks up the array's device address; make that first
- *     call before any stream capture begins.
+ *   - The first call on each device looks up the array's device address and asks the occupancy
+ *     calculator how many CTAs of the kernel are resident per SM (the grid is one wave of them);
+ *     neither allocates.  Make that first call before any stream capture begins.
  *   - All calls share the array and it keeps the previous call's contents.  Every partial
  *     that a call reads it has written first, so nothing needs clearing; but two calls whose
  *     kernels overlap on the GPU (e.g. on different streams) race on it and must be ordered

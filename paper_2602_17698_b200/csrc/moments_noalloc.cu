@@ -54,7 +54,7 @@ __global__ void noalloc_finish_kernel(const float* __restrict__ partial, int spl
 // with that device current.
 std::mutex g_mu;
 float* g_scratch_ptr[64] = {nullptr};
-int g_sm_count[64] = {0};
+int g_sm_count[64] = {0};          // resident CTAs of the partial-sum kernel per device (SMs x CTAs per SM)
 
 sb_status scratch_for_current_device(float** out, int* sm_count) {
     int dev = -1;
@@ -76,11 +76,18 @@ sb_status scratch_for_current_device(float** out, int* sm_count) {
         int sms = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
             sms = 148;
-        g_sm_count[dev] = sms;
+        // one wave of resident CTAs (a host-side calculation: nothing is allocated)
+        int occ = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, noalloc_partial_kernel, NA_TX * NA_TY, 0) != cudaSuccess ||
+            occ <= 0) {
+            (void)cudaGetLastError();
+            occ = 6;
+        }
+        g_sm_count[dev] = sms * occ;
         g_scratch_ptr[dev] = p;
     }
     *out = g_scratch_ptr[dev];
-    *sm_count = g_sm_count[dev];
+    *sm_count = g_sm_count[dev];               // resident CTAs of the partial-sum kernel on this device
     return SB_OK;
 }
 
@@ -103,13 +110,13 @@ extern "C" sb_status sb_calib_moments_noalloc(void* cuda_stream, const void* X, 
         return SB_ERR_SCRATCH;
     }
     float* partial = nullptr;
-    int sms = 148;
+    int sms = 148 * 6;                              // resident CTAs of the partial-sum kernel
     sb_status st = scratch_for_current_device(&partial, &sms);
     if (st != SB_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int col_chunks = (int)((K + NA_COLS - 1) / NA_COLS);
     const int64_t min_rows = NA_TY * NA_UNROLL;
-    int splits = (sms * 8 + col_chunks - 1) / col_chunks;
+    int splits = sms / col_chunks;                  // sms: resident CTAs; the grid is one wave of them
     const int max_splits = (int)(SB_NOALLOC_SCRATCH_FLOATS / K);       // >= 16 by the K limit
     if (splits > max_splits) splits = max_splits;
     if ((int64_t)splits * min_rows > T) splits = (int)((T + min_rows - 1) / min_rows);
