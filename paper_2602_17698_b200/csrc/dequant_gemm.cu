@@ -439,23 +439,32 @@ dequant_gemm_kernel(const DqArgs a) {
     const int j0 = blockIdx.y * a.seg_blocks;                   // first column block of the segment
     const int nblk = min(a.seg_blocks, a.nbc - j0);
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < nblk; ++s) {
-            dq_mbar_init(dq_smem_u32(full + s), 1 + 32);       // the bulk copies' expect_tx and the loader lanes' row copies
-            dq_mbar_init(dq_smem_u32(empty + s), WARPS);
-        }
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    // the segment's column sums of X and its block table
-    for (int i = threadIdx.x; i < nblk * NT; i += S::THREADS) xs[i] = a.xsum[(int64_t)j0 * NT + i];
+    // Set-up is the loader warp's: it arms the barriers, reads the segment's block table (one load of
+    // the offsets, one of the levels) and starts the first copies without waiting for the other
+    // warps, which meanwhile fetch the segment's column sums of X; they meet it at a named barrier on
+    // which the loader only arrives.
     const int64_t blk0 = (int64_t)bi * a.nbc + j0;
-    const int64_t word0 = a.block_off[blk0];
-    if (threadIdx.x < nblk) {
-        blk_word[threadIdx.x] = (unsigned)(a.block_off[blk0 + threadIdx.x] - word0);
-        blk_bits[threadIdx.x] = (unsigned char)dq_bits(a.bits, a.level[blk0 + threadIdx.x]);
+    int64_t word0 = 0;
+    if (warp == WARPS) {
+        if (lane < nblk) {
+            dq_mbar_init(dq_smem_u32(full + lane), 1 + 32);     // the bulk copies' expect_tx and the loader lanes' row copies
+            dq_mbar_init(dq_smem_u32(empty + lane), WARPS);
+        }
+        if (lane == 0) *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const int64_t off = lane <= nblk ? a.block_off[blk0 + lane] : 0;
+        const int lv = lane < nblk ? (int)a.level[blk0 + lane] : 0;
+        word0 = __shfl_sync(0xffffffffu, off, 0);
+        if (lane < nblk) {
+            blk_word[lane] = (unsigned)(off - word0);
+            blk_bits[lane] = (unsigned char)dq_bits(a.bits, lv);
+        }
+        __syncwarp();
+        asm volatile("bar.arrive 2, %0;" ::"r"(S::THREADS) : "memory");
+    } else {
+        for (int i = threadIdx.x; i < nblk * NT; i += WARPS * 32) xs[i] = a.xsum[(int64_t)j0 * NT + i];
+        asm volatile("bar.sync 2, %0;" ::"r"(S::THREADS) : "memory");
     }
-    __syncthreads();
     const float2* mbase = a.meta + ((int64_t)bi * S::ROWS) * a.nbc + j0;
     // what the loader does for block j
     auto load_codes_meta = [&](int j, unsigned at) {
@@ -464,7 +473,7 @@ dequant_gemm_kernel(const DqArgs a) {
         if (lane == 0) {
             blk_at[j] = at;
             dq_mbar_expect_tx(bar, code_bytes + (unsigned)S::X_BYTES);
-            dq_bulk_load(dq_smem_u32(smem + at + S::X_BYTES), a.packed + word0 + blk_word[j], code_bytes, bar);
+            dq_bulk_load(dq_smem_u32(smem + at + S::X_BYTES), a.packed + word0 + blk_word[j], code_bytes, bar);   // word0: the loader's
         }
         const unsigned mdst = dq_smem_u32(smem + at + S::X_BYTES) + code_bytes;
 #pragma unroll
