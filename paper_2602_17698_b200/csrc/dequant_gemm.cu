@@ -627,15 +627,26 @@ dequant_gemm_kernel(const DqArgs a) {
         const float* seg[8];
 #pragma unroll
         for (int sgm = 0; sgm < 8; ++sgm) seg[sgm] = cluster.map_shared_rank(ysm, sgm < nseg ? sgm : 0);
-        for (int idx = rank * chunk + (int)threadIdx.x; idx < end; idx += S::THREADS) {
-            float v[8];
+        // four outputs per thread at a time, so that up to 32 remote reads are in flight
+        constexpr int OU = 4;
+        for (int base = rank * chunk + (int)threadIdx.x; base < end; base += OU * S::THREADS) {
+            float v[OU][8];
 #pragma unroll
-            for (int sgm = 0; sgm < 8; ++sgm) v[sgm] = sgm < nseg ? seg[sgm][idx] : 0.f;
-            float acc = 0.f;
+            for (int u = 0; u < OU; ++u) {
+                const int idx = base + u * S::THREADS;
 #pragma unroll
-            for (int sgm = 0; sgm < 8; ++sgm) acc += v[sgm];
-            if (!isfinite(acc)) sb_latch(a.ds, SB_ERR_NONFINITE, SBK_GEMM);
-            a.out[(int64_t)(idx / S::ROWS) * a.out_t_stride + (int64_t)bi * S::ROWS + idx % S::ROWS] = acc;
+                for (int sgm = 0; sgm < 8; ++sgm) v[u][sgm] = (sgm < nseg && idx < end) ? seg[sgm][idx] : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < OU; ++u) {
+                const int idx = base + u * S::THREADS;
+                float acc = 0.f;
+#pragma unroll
+                for (int sgm = 0; sgm < 8; ++sgm) acc += v[u][sgm];
+                if (!isfinite(acc)) sb_latch(a.ds, SB_ERR_NONFINITE, SBK_GEMM);
+                if (idx < end)
+                    a.out[(int64_t)(idx / S::ROWS) * a.out_t_stride + (int64_t)bi * S::ROWS + idx % S::ROWS] = acc;
+            }
         }
         cluster.sync();                     // nobody leaves while its shared memory may still be read
     }
