@@ -420,7 +420,7 @@ def dequant_gemm_times(ctx, dev, peak_gbs):
     return out
 
 
-def full_model_times(ctx, dev):
+def full_model_times(ctx, dev, ctx2=None):
     """configs[2]: 32 layers of the 8B shape searched as ONE model (residual-stream permutation
     shared by all layers, one global allocation over N = 425,984 blocks per budget), budgets
     2.0 ... 4.0.  Returns the CUDA-event time of the library calls only (the synthetic layers
@@ -442,9 +442,9 @@ def full_model_times(ctx, dev):
     cfg = SearchConfig(bits=BITS)
     # untimed warm-up on four layers: grows the library's scratch arena to its steady-state size
     # and loads the kernels that only large tables use (the cooperative form of the loop kernel)
-    search_model(ctx, shape, 4, cfg, (2.25,), make_weights, make_acts, dev, keep_tables=False)
+    search_model(ctx, shape, 4, cfg, (2.25,), make_weights, make_acts, dev, keep_tables=False, ctx2=ctx2)
     res = search_model(ctx, shape, FULL_MODEL_LAYERS, cfg, FULL_MODEL_BUDGETS, make_weights, make_acts, dev,
-                       keep_tables=False, alloc_repeats=2)
+                       keep_tables=False, alloc_repeats=2, ctx2=ctx2)
     ms = res.ms
     sweeps = sorted({int(k.split("@")[1]) for k in ms if k.startswith("stats@")})
     first = FULL_MODEL_BUDGETS[0]
@@ -521,7 +521,7 @@ def small_layer_times(ctx, dev):
                       "the allocation), mean of 20 passes, L2 flushed between passes"}
 
 
-def streamed_model_times(ctx, dev):
+def streamed_model_times(ctx, dev, ctx2=None):
     """configs[3]: 80 layers of the 70B shape (68.5 G weights, N = 4,177,920 blocks), bits {2,3,4},
     budget 2.25.  Weights and activations are made again from their seeds in every sweep (the
     model is never resident: 136.9 GB of weights); only moments, score vectors, permutations and
@@ -534,7 +534,7 @@ def streamed_model_times(ctx, dev):
     res = search_model(ctx, shape, n_layers, cfg, (budget,),
                        lambda layer: synth.make_layer_weights(shape, SEED, layer, dev),
                        lambda layer: synth.make_layer_activations(shape, tokens, SEED, layer, dev), dev,
-                       keep_tables=False, keep_weights=False, alloc_repeats=2)
+                       keep_tables=False, keep_weights=False, alloc_repeats=2, ctx2=ctx2)
     wall = time.time() - t0
     ms = res.ms
     r = res.reports[budget]
@@ -553,7 +553,7 @@ def streamed_model_times(ctx, dev):
                       "once) and their release"}
 
 
-def full_model_e2e(ctx, dev):
+def full_model_e2e(ctx, dev, ctx2=None):
     """configs[2] end to end for one budget: the weights of every layer come from pinned host memory
     (13.96 GB, copied once, then resident for the second sweep), the activations of every layer are
     copied from pinned host buffers as well (3.49 GB per layer; one set of host buffers serves all
@@ -585,7 +585,7 @@ def full_model_e2e(ctx, dev):
     torch.cuda.synchronize()
     t0 = time.perf_counter()
     res = search_model(ctx, shape, FULL_MODEL_LAYERS, cfg, (budget,), make_weights, make_acts, dev,
-                       keep_tables=False)
+                       keep_tables=False, ctx2=ctx2)
     level_h = res.levels[budget].cpu()
     torch.cuda.synchronize()
     sec = time.perf_counter() - t0
@@ -624,8 +624,11 @@ def run_cuda(args):
     torch.cuda.synchronize()
     torch.cuda.set_stream(stream)
     ctx = Context()
+    # a second context on a stream of its own: the stages whose matrices are independent (block
+    # scores, pack) deal them to the two contexts in turn (pipeline.search_layer)
+    ctx2 = None if args.one_stream else Context(stream=torch.cuda.Stream(device=dev))
     ws = LayerWorkspace(shape, cfg, dev)
-    graphs = None if args.no_graphs else StageGraphs(ctx)
+    graphs = None if args.no_graphs else StageGraphs(ctx, ctx2)
     n_weights = shape.n_weights
     in_bytes = sum(w.numel() * 2 for w in W.values()) + sum(x.numel() * 2 for x in X.values())
 
@@ -635,7 +638,7 @@ def run_cuda(args):
         torch.cuda.synchronize()
 
     def step(timers=None):
-        return search_layer(ctx, W, X, ws, timers=timers, graphs=graphs)
+        return search_layer(ctx, W, X, ws, timers=timers, graphs=graphs, ctx2=ctx2)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -647,7 +650,11 @@ def run_cuda(args):
         sampler.start()
         time.sleep(0.15)
     timers = {s: [] for s in STAGES}
-    l0 = ctx.kernel_launches() + (graphs.replayed_kernels if graphs else 0)
+    def launched():
+        return (ctx.kernel_launches() + (ctx2.kernel_launches() if ctx2 is not None else 0)
+                + (graphs.replayed_kernels if graphs else 0))
+
+    l0 = launched()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     t_wall0 = time.time()
@@ -657,7 +664,7 @@ def run_cuda(args):
     e1.record()
     barrier()
     t_wall1 = time.time()
-    launches = ctx.kernel_launches() + (graphs.replayed_kernels if graphs else 0) - l0
+    launches = launched() - l0
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
     ms = max_over_ranks(ms, world, dev)
@@ -731,9 +738,9 @@ def run_cuda(args):
             del hW, hX                                   # pinned copies of the layer, if any
             small_layer = small_layer_times(ctx, dev)
             del W, X                                     # the layer's tensors: the models need the room
-            full_model = full_model_times(ctx, dev)
-            full_model["e2e"] = full_model_e2e(ctx, dev)
-            streamed = streamed_model_times(ctx, dev)
+            full_model = full_model_times(ctx, dev, ctx2)
+            full_model["e2e"] = full_model_e2e(ctx, dev, ctx2)
+            streamed = streamed_model_times(ctx, dev, ctx2)
         cpu = None
         if not args.no_cpu_baseline:
             v, sec, cores, sample = time_oracle(3, 0)
@@ -747,7 +754,8 @@ def run_cuda(args):
                            "l2": "inputs (3.9 GB per step) larger than L2, no flush needed",
                            "hbm_target": "fractions of the measured copy bandwidth (frac) and of the nominal "
                                          "8000 GB/s (frac_nominal): the 70 % target is stated on the nominal figure",
-                           "launch": "eager" if graphs is None else "one CUDA graph per stage (allocation eager)",
+                           "launch": ("eager" if graphs is None else "one CUDA graph per stage (allocation eager)")
+                                     + ("" if ctx2 is None else "; block scores and pack dealt to two streams"),
                            "allocation": res.report},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
                 "roofline": roofline, "cpu_baseline": cpu,
@@ -756,6 +764,9 @@ def run_cuda(args):
                 "roofline_other_kernels": kernels, "small_layer": small_layer, "full_model": full_model,
                 "streamed_model": streamed}
         print(json.dumps(line), flush=True)
+    if ctx2 is not None:
+        ctx2.sync()
+        ctx2.close()
     ctx.close()
     if world > 1:
         dist.barrier()              # rank 0 may still have been timing its extra legs
@@ -875,6 +886,8 @@ def main():
     ap.add_argument("--no-full-model", action="store_true",
                     help="skip the 32-layer global-allocation timing (single GPU only)")
     ap.add_argument("--no-graphs", action="store_true", help="launch every library call eagerly")
+    ap.add_argument("--one-stream", action="store_true",
+                    help="one context only (no dealing of independent matrices to a second stream)")
     ap.add_argument("--only", default=None,
                     help="three calls of one library call on one input, then exit (for ncu captures): "
                          "moments | gram | full_scores | dequant_gemm | reorder_stats | reorder_stats_first_order | scores | scores3 | scores7 | "

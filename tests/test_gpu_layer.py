@@ -85,3 +85,40 @@ def test_tiny_layer_stagewise(bits, budget, br, bc, g):
         total_words += int(ooff[-1])
     assert total_words * 32 == res.report["used_bits"]          # exact budget accounting
     ctx.close()
+
+
+def test_two_contexts_give_the_same_layer_result():
+    """search_layer with a second context (block scores and pack dealt to two streams, eager and
+    from CUDA graphs) against the one-context run: every output identical."""
+    from paper_2602_17698_b200.binding import Context
+    from paper_2602_17698_b200.pipeline import LayerWorkspace, SearchConfig, StageGraphs, search_layer
+    torch.cuda.set_device(0)
+    shape = synth.LLAMA_TINY
+    cfg = SearchConfig(bits=[2, 3, 4, 8], budget=2.75)
+    W = synth.make_layer_weights(shape, 5, 0, DEV)
+    X = synth.make_layer_activations(shape, 1024, 5, 0, DEV)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s1):
+        ctx = Context()
+        ctx2 = Context(stream=s2)
+        ws_a, ws_b, ws_c = (LayerWorkspace(shape, cfg, DEV) for _ in range(3))
+        ref = search_layer(ctx, W, X, ws_a)
+        ctx.sync()
+        eager = search_layer(ctx, W, X, ws_b, ctx2=ctx2)
+        ctx.sync(); ctx2.sync()
+        graphs = StageGraphs(ctx, ctx2)
+        search_layer(ctx, W, X, ws_c, graphs=graphs, ctx2=ctx2)           # captures
+        replay = search_layer(ctx, W, X, ws_c, graphs=graphs, ctx2=ctx2)  # replays
+        ctx.sync(); ctx2.sync()
+    torch.cuda.synchronize()
+    assert ctx2.kernel_launches() > 0
+    for got in (eager, replay):
+        assert torch.equal(got.err, ref.err) and torch.equal(got.level, ref.level)
+        assert got.report == ref.report
+        for name in ref.packed:
+            for a, b in zip(got.packed[name], ref.packed[name]):
+                n = int(ref.packed[name][1][-1].item()) if a.dtype == torch.int32 else a.numel()
+                assert torch.equal(a.reshape(-1)[:n], b.reshape(-1)[:n]), name
+    ctx2.close()
+    ctx.close()

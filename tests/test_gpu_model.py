@@ -242,3 +242,37 @@ def test_llama3_70b_streamed_allocation_matches_oracle():
         assert rep["used_bits"] == orep["used_bits"]
         assert rep["iterations"] == orep["iterations"]
     ctx.close()
+
+
+def test_second_context_gives_the_same_model_result():
+    """The block-score calls of a layer's matrices dealt to two contexts on two streams: tables,
+    permutations, levels and reports are those of the one-context run, bit for bit."""
+    from paper_2602_17698_b200.binding import Context
+    from paper_2602_17698_b200.pipeline import SearchConfig, search_model
+    torch.cuda.set_device(0)
+    shape, n_layers, tokens = synth.LLAMA_TINY, 3, 384
+    budgets = [2.5, 3.25]
+    cfg = SearchConfig(bits=[2, 3, 4, 8])
+
+    def make_weights(layer):
+        return synth.make_layer_weights(shape, 5, layer, DEV)
+
+    def make_acts(layer):
+        return synth.make_layer_activations(shape, tokens, 5, layer, DEV)
+
+    ctx = Context()
+    ctx2 = Context(stream=torch.cuda.Stream(device=DEV))
+    one = search_model(ctx, shape, n_layers, cfg, budgets, make_weights, make_acts, DEV)
+    two = search_model(ctx, shape, n_layers, cfg, budgets, make_weights, make_acts, DEV, ctx2=ctx2)
+    torch.cuda.synchronize()
+    assert sorted(one.tables) == sorted(two.tables)
+    for rb in one.tables:
+        assert torch.equal(one.tables[rb], two.tables[rb]), rb
+        for k in one.perms[rb]:
+            assert torch.equal(one.perms[rb][k], two.perms[rb][k]), (rb, k)
+    for b in budgets:
+        assert torch.equal(one.levels[b], two.levels[b]), b
+        for k in ("used_bits", "iterations", "cap_bits"):
+            assert one.reports[b][k] == two.reports[b][k], (b, k)
+    ctx2.close()
+    ctx.close()
