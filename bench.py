@@ -628,7 +628,9 @@ def run_cuda(args):
     # scores, pack) deal them to the two contexts in turn (pipeline.search_layer)
     ctx2 = None if args.one_stream else Context(stream=torch.cuda.Stream(device=dev))
     ws = LayerWorkspace(shape, cfg, dev)
-    graphs = None if args.no_graphs else StageGraphs(ctx, ctx2)
+    # the timed step is ONE CUDA graph (moments ... pack, the allocation in its enqueue-only form);
+    # a second pass below replays one graph per stage for the per-stage times
+    graphs = None if args.no_graphs else StageGraphs(ctx, ctx2, whole=not args.stage_graphs)
     n_weights = shape.n_weights
     in_bytes = sum(w.numel() * 2 for w in W.values()) + sum(x.numel() * 2 for x in X.values())
 
@@ -671,6 +673,26 @@ def run_cuda(args):
     ms_per_step = ms / args.steps
     value = job_throughput(n_weights, world, ms_per_step)
 
+    res.read_report()
+    ctx.sync()                                       # device-side status of everything replayed so far
+    if ctx2 is not None:
+        ctx2.sync()
+    stagewise_ms = None
+    if graphs is not None and graphs.whole:
+        # per-stage times: the same steps again, one graph per stage with events between the stages
+        # (the allocation eager and synchronous); this pass also times the roofline kernel
+        timers = {s: [] for s in STAGES}
+        stage_graphs = StageGraphs(ctx, ctx2)
+        for _ in range(3):
+            search_layer(ctx, W, X, ws, graphs=stage_graphs, ctx2=ctx2)
+        barrier()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for _ in range(args.steps):
+            search_layer(ctx, W, X, ws, timers=timers, graphs=stage_graphs, ctx2=ctx2)
+        s1.record()
+        barrier()
+        stagewise_ms = s0.elapsed_time(s1) / args.steps
     stage_ms = {s: sum(a.elapsed_time(b) for a, b in timers[s]) / args.steps for s in STAGES}
     stage_launch_ms = {s: (sum(a.elapsed_time(b) for a, b in timers[s]) / max(len(timers[s]), 1))
                        for s in STAGES}
@@ -754,12 +776,19 @@ def run_cuda(args):
                            "l2": "inputs (3.9 GB per step) larger than L2, no flush needed",
                            "hbm_target": "fractions of the measured copy bandwidth (frac) and of the nominal "
                                          "8000 GB/s (frac_nominal): the 70 % target is stated on the nominal figure",
-                           "launch": ("eager" if graphs is None else "one CUDA graph per stage (allocation eager)")
+                           "launch": ("eager" if graphs is None else
+                                      "one CUDA graph per step (allocation enqueued, report left on the device)"
+                                      if graphs.whole else "one CUDA graph per stage (allocation eager)")
                                      + ("" if ctx2 is None else "; block scores and pack dealt to two streams"),
-                           "allocation": res.report},
+                           "allocation": res.read_report()},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
                 "roofline": roofline, "cpu_baseline": cpu,
                 "stages_ms_per_step": stage_ms, "stages_algorithmic_gbs": stage_gbs,
+                "stages_timing": ("CUDA events between the stages of the timed steps" if stagewise_ms is None else
+                                  "a second timed pass of the same steps with one CUDA graph per stage, events "
+                                  "between the stages and the synchronous allocation: %.4f ms per step; the "
+                                  "roofline kernel's launch time is taken there" % stagewise_ms),
+                "ms_per_step_stagewise": stagewise_ms,
                 "scoring_elements_per_s": n_weights / (stage_ms["scores"] * 1e-3),
                 "roofline_other_kernels": kernels, "small_layer": small_layer, "full_model": full_model,
                 "streamed_model": streamed}
@@ -886,6 +915,9 @@ def main():
     ap.add_argument("--no-full-model", action="store_true",
                     help="skip the 32-layer global-allocation timing (single GPU only)")
     ap.add_argument("--no-graphs", action="store_true", help="launch every library call eagerly")
+    ap.add_argument("--stage-graphs", action="store_true",
+                    help="time the step as one CUDA graph per stage with an eager, synchronous allocation "
+                         "instead of one graph for the whole step")
     ap.add_argument("--one-stream", action="store_true",
                     help="one context only (no dealing of independent matrices to a second stream)")
     ap.add_argument("--only", default=None,

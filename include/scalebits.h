@@ -176,6 +176,20 @@ sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
                            int mode, double gamma0, double gammaT,
                            uint8_t* level, sb_alloc_report* report);
 
+/* The same allocation (Algorithm 2 / Algorithm 1, same kernels, same results) without the
+ * host round trip: everything is enqueued on the context's stream and the call returns, so
+ * it can be captured in a CUDA graph between sb_block_scores and sb_pack_blocks.
+ * report_dev: DEVICE struct, written in stream order after `level`; copy it back after a
+ * synchronisation.  What the synchronous form reports after reading the device -- a lowest
+ * candidate that does not fit the budget in greedy mode (SB_ERR_BUDGET; `level` is then all
+ * zero), the iteration cap (SB_ERR_NOCONVERGE) -- is latched in the device status word and
+ * returned by the next sb_sync.  Errors in the arguments are returned at once, as above.   */
+sb_status sb_allocate_bits_async(sb_ctx* ctx, const float* err, int64_t N,
+                                 const int64_t* block_elems, int64_t uniform_block_elems,
+                                 const int* bits, int n_bits, double budget_avg_bits,
+                                 int mode, double gamma0, double gammaT,
+                                 uint8_t* level, sb_alloc_report* report_dev);
+
 /* Pack (Section 5.3: one bitwidth per tile).  Quantise each block of W' at
  * bits[level[block]] with the same quantizer, evaluated in IEEE binary64 so that the
  * integer codes are reproducible: lo = min, range = max - min, inv = qmax / range,

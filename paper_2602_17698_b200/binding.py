@@ -24,7 +24,8 @@ SB_ACC_ROW, SB_ACC_COL = 1, 2
 EXPORTS = ["sb_create", "sb_destroy", "sb_sync", "sb_last_error", "sb_kernel_launches", "sb_debug_lookback",
            "sb_checked_build",
            "sb_calib_moments", "sb_reorder_channels", "sb_fold_segment_scores",
-           "sb_expand_segment_perm", "sb_permute_matrix", "sb_block_scores", "sb_allocate_bits", "sb_pack_blocks",
+           "sb_expand_segment_perm", "sb_permute_matrix", "sb_block_scores", "sb_allocate_bits", "sb_allocate_bits_async",
+           "sb_pack_blocks",
            "sb_calib_moments_noalloc", "sb_first_order_scores", "sb_exchange_step",
            "sb_reorder_channels_first_order", "sb_calib_gram",
            "sb_block_scores_full", "sb_dequant_gemm"]
@@ -94,6 +95,8 @@ def lib() -> C.CDLL:
                                       C.POINTER(C.c_int), i32, vp, vp, vp]
         L.sb_allocate_bits.argtypes = [vp, vp, i64, vp, i64, C.POINTER(C.c_int), i32, f64, i32,
                                        f64, f64, vp, C.POINTER(AllocReport)]
+        L.sb_allocate_bits_async.argtypes = [vp, vp, i64, vp, i64, C.POINTER(C.c_int), i32, f64, i32,
+                                             f64, f64, vp, vp]
         L.sb_pack_blocks.argtypes = [vp, vp, i64, i64, i64, vp, vp, i32, i32, i32,
                                      C.POINTER(C.c_int), i32, vp, vp, i64, vp, vp]
         L.sb_first_order_scores.argtypes = [vp, vp, vp, i64, i64, i64, i64, vp, vp, i32, i32, i32,
@@ -289,6 +292,35 @@ class Context:
                                     float(gamma0), float(gammaT), _ptr(level, torch.uint8), C.byref(rep))
         self._check(st)
         return level, rep.as_dict()
+
+    def allocate_bits_async(self, err: torch.Tensor, bits: Sequence[int], budget: float,
+                            mode: int = SB_ALLOC_SCALEBITS, gamma0: float = 0.05, gammaT: float = 0.02,
+                            uniform_block_elems: int = 128 * 128, block_elems=None, level=None,
+                            report=None):
+        """The allocation enqueued only (no host round trip; can be captured in a CUDA graph).
+        Returns (level, report): `report` is a uint8 device tensor holding the report struct;
+        `read_report(report)` decodes it after a synchronisation."""
+        N, L = err.shape
+        barr, Lb = _bits(bits)
+        assert L == Lb and err.is_contiguous()
+        if level is None:
+            level = torch.empty(N, dtype=torch.uint8, device=err.device)
+        if report is None:
+            report = torch.zeros(C.sizeof(AllocReport), dtype=torch.uint8, device=err.device)
+        assert report.dtype == torch.uint8 and report.numel() >= C.sizeof(AllocReport) and report.is_contiguous()
+        st = lib().sb_allocate_bits_async(self._h, _ptr(err, torch.float32), N, _ptr(block_elems, torch.int64),
+                                          int(uniform_block_elems), barr, L, float(budget), int(mode),
+                                          float(gamma0), float(gammaT), _ptr(level, torch.uint8),
+                                          _ptr(report, torch.uint8))
+        self._check(st)
+        return level, report
+
+    @staticmethod
+    def read_report(report: torch.Tensor) -> dict:
+        """Decodes the device report of `allocate_bits_async` (copies it to the host: the
+        stream that wrote it must have been synchronised, or be the current one)."""
+        raw = bytes(report.cpu().numpy().tobytes()[:C.sizeof(AllocReport)])
+        return AllocReport.from_buffer_copy(raw).as_dict()
 
     def reorder_channels_first_order(self, W: torch.Tensor, G: torch.Tensor, ref_bits: int, group: int,
                                      row_score=None, col_score=None, accumulate_row: bool = False,

@@ -42,6 +42,7 @@ struct AllocState {
     double dU, dD;
     unsigned done_down, done_decide, done_apply, done_eval;   // last-CTA tickets
     long long hist[8];
+    long long used_init;            // bits of the warm start (greedy: of the lowest candidate)
 };
 
 struct AllocArgs {
@@ -170,6 +171,42 @@ __global__ void init_finish_kernel(AllocArgs a, int nparts) {
     for (int p = 0; p < nparts; ++p) s += a.part[p];
     a.st->loss = s;
     a.st->loss_init = s;
+    a.st->used_init = a.st->used;
+}
+// The loop state before the first kernel reads it, computed where it is used so that the call
+// needs no host round trip: cap = floor(budget * total weights), k = floor(gamma0 N) and
+// kT = floor(gammaT N), both at least 1 (the same binary64 operations the host would do).
+__global__ void init_state_kernel(AllocState* st, const unsigned long long* total_dev, long long total_host,
+                                  double budget, double gamma0, double gammaT, long long N, int scalebits) {
+    AllocState z{};
+    const long long total = total_dev ? (long long)*total_dev : total_host;
+    z.cap = (long long)floor(budget * (double)total);
+    if (scalebits) {
+        long long k = (long long)floor(gamma0 * (double)N); if (k < 1) k = 1;
+        long long kT = (long long)floor(gammaT * (double)N); if (kT < 1) kT = 1;
+        if (k < kT) k = kT;
+        z.k = k; z.kT = kT;
+    }
+    *st = z;
+}
+// The report in the caller's device memory; conditions the loop found are latched for sb_sync.
+__global__ void report_kernel(AllocArgs a, const int* greedy_steps, int greedy, sb_alloc_report* rep) {
+    const AllocState s = *a.st;
+    sb_alloc_report r{};
+    r.cap_bits = s.cap;
+    r.used_bits = s.used;
+    r.proxy_loss_init = s.loss_init;
+    r.proxy_loss_final = s.loss;
+    if (greedy) {
+        r.iterations = greedy_steps ? *greedy_steps : 0;
+        r.accepted = r.iterations;
+        if (s.used_init > s.cap) sb_latch(a.ds, SB_ERR_BUDGET, SBK_ALLOC);   // the lowest candidate must fit
+    } else {
+        r.iterations = s.iter; r.accepted = s.accepted; r.rejected = s.rejected; r.expansions = s.expansions;
+        if (s.status != 0) sb_latch(a.ds, s.status, SBK_ALLOC);              // iteration cap reached
+    }
+    for (int l = 0; l < 8; ++l) r.level_hist[l] = s.hist[l];
+    *rep = r;
 }
 
 // ---- the Algorithm 2 loop, one persistent kernel ----------------------------------------------
@@ -794,13 +831,15 @@ __global__ void __launch_bounds__(BT) eval_kernel(AllocArgs a, double* part, int
 
 }  // namespace
 
-extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
-                                      const int64_t* block_elems, int64_t uniform_block_elems,
-                                      const int* bits, int n_bits, double budget, int mode,
-                                      double gamma0, double gammaT, uint8_t* level,
-                                      sb_alloc_report* report) {
+// Everything of an allocation call in stream order, no host round trip (so the call can be part
+// of a captured CUDA graph); the report goes to device memory.
+static sb_status allocate_enqueue(sb_ctx* ctx, const float* err, int64_t N,
+                                  const int64_t* block_elems, int64_t uniform_block_elems,
+                                  const int* bits, int n_bits, double budget, int mode,
+                                  double gamma0, double gammaT, uint8_t* level,
+                                  sb_alloc_report* report_dev, bool own_report) {
     if (!ctx) return SB_ERR_INVALID;
-    if (!err || !level || !report || N <= 0) return sb_fail(ctx, SB_ERR_INVALID, "allocate: null or empty");
+    if (!err || !level || (!report_dev && !own_report) || N <= 0) return sb_fail(ctx, SB_ERR_INVALID, "allocate: null or empty");
     if (!sb_check_bits(bits, n_bits)) return sb_fail(ctx, SB_ERR_INVALID, "allocate: bits must be ascending in 1..8");
     if (!block_elems && uniform_block_elems <= 0) return sb_fail(ctx, SB_ERR_INVALID, "allocate: block size");
     if (mode != SB_ALLOC_SCALEBITS && mode != SB_ALLOC_GREEDY) return sb_fail(ctx, SB_ERR_INVALID, "allocate: mode");
@@ -811,10 +850,14 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
     const long long nsteps = (long long)N * (L - 1);
     if (nsteps >= (1ll << 32) || N >= (1ll << 29) - 1)
         return sb_fail(ctx, SB_ERR_SHAPE, "allocate: N must be below 2^29 and N * (n_bits - 1) below 2^32");
+    int l0 = 0;
+    if (mode == SB_ALLOC_SCALEBITS) {
+        l0 = -1;
+        for (int l = 0; l < L; ++l) if ((double)bits[l] <= budget) l0 = l;
+        if (l0 < 0) return sb_fail(ctx, SB_ERR_BUDGET, "allocate: budget %.4f below the smallest candidate %d", budget, bits[0]);
+    }
     SB_CUDA(ctx, cudaSetDevice(ctx->device));
-    memset(report, 0, sizeof *report);
 
-    // total weights -> cap.  Uniform blocks: closed form; else a device sum via the scan.
     const int nblkB = (int)((N + BT - 1) / BT);
     const long long ntiles = (nsteps + ATILE - 1) / ATILE;
     const size_t nparts = (size_t)(nblkB > ntiles ? nblkB : ntiles) + 8;
@@ -826,7 +869,7 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
                                                    (size_t)N * 8, (size_t)N * 8, (size_t)N * 8,
                                                    (size_t)N * 4, nparts * 8,
                                                    nparts * 8, sort_bytes, (size_t)(N + 1) * 8,
-                                                   (size_t)LOOP_MAX_CTAS * 128}), &arena);
+                                                   (size_t)LOOP_MAX_CTAS * 128, sizeof(sb_alloc_report)}), &arena);
     if (stt != SB_OK) return stt;
     Carver cv(arena);
     AllocState* dst = cv.take<AllocState>(1);
@@ -851,20 +894,16 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
     double* loop_d = cv.take<double>(2 * LOOP_MAX_CTAS);
     unsigned long long* loop_u64 = cv.take<unsigned long long>(2 * LOOP_MAX_CTAS);
     unsigned* loop_u32 = cv.take<unsigned>(2 * LOOP_MAX_CTAS);
+    sb_alloc_report* own_rep = cv.take<sb_alloc_report>(1);
+    if (own_report) report_dev = own_rep;
 
-    long long total_elems = 0;
-    AllocState* hst = static_cast<AllocState*>(ctx->pinned);
+    // total weights -> cap.  Uniform blocks: closed form; else a device sum via the scan.
+    const unsigned long long* total_dev = nullptr;
     if (block_elems) {
         stt = sb_scan_exclusive_u64(ctx, reinterpret_cast<const unsigned long long*>(block_elems), totals, N);
         if (stt != SB_OK) return stt;
-        SB_CUDA(ctx, cudaMemcpyAsync(hst, totals + N, 8, cudaMemcpyDeviceToHost, ctx->stream));
-        SB_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
-        total_elems = *reinterpret_cast<long long*>(hst);
-    } else {
-        total_elems = (long long)N * uniform_block_elems;
+        total_dev = totals + N;
     }
-    const long long cap = (long long)floor(budget * (double)total_elems);
-    report->cap_bits = cap;
 
     AllocArgs a{};
     a.err = err; a.block_elems = reinterpret_cast<const long long*>(block_elems);
@@ -874,40 +913,18 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
     a.upsr = upsr; a.upcum = upcum; a.upde = upde; a.mark = mark;
     a.part = part;
 
-    int l0 = 0;
-    AllocState init{};
-    init.cap = cap;
-    if (mode == SB_ALLOC_SCALEBITS) {
-        l0 = -1;
-        for (int l = 0; l < L; ++l) if ((double)bits[l] <= budget) l0 = l;
-        if (l0 < 0) return sb_fail(ctx, SB_ERR_BUDGET, "allocate: budget %.4f below the smallest candidate %d", budget, bits[0]);
-        long long k = (long long)floor(gamma0 * (double)N); if (k < 1) k = 1;
-        long long kT = (long long)floor(gammaT * (double)N); if (kT < 1) kT = 1;
-        if (k < kT) k = kT;
-        init.k = k; init.kT = kT;
-    }
-    memcpy(hst, &init, sizeof init);
-    SB_CUDA(ctx, cudaMemcpyAsync(dst, hst, sizeof init, cudaMemcpyHostToDevice, ctx->stream));
+    init_state_kernel<<<1, 1, 0, ctx->stream>>>(dst, total_dev, (long long)N * uniform_block_elems, budget,
+                                                gamma0, gammaT, (long long)N, mode == SB_ALLOC_SCALEBITS);
+    SB_LAUNCHED(ctx);
     init_levels_kernel<<<nblkB, BT, 0, ctx->stream>>>(a, l0, 1);
     SB_LAUNCHED(ctx);
     init_finish_kernel<<<1, 1, 0, ctx->stream>>>(a, nblkB);
     SB_LAUNCHED(ctx);
 
-    auto read_state = [&](AllocState* out) -> sb_status {
-        SB_CUDA(ctx, cudaMemcpyAsync(hst, dst, sizeof(AllocState), cudaMemcpyDeviceToHost, ctx->stream));
-        SB_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
-        *out = *hst;
-        return SB_OK;
-    };
-
-    AllocState fin{};
+    const int* greedy_steps = nullptr;
     if (mode == SB_ALLOC_GREEDY) {
-        // the lowest candidate must fit
-        stt = read_state(&fin);
-        if (stt != SB_OK) return stt;
-        report->proxy_loss_init = fin.loss_init;
-        report->used_bits = fin.used;
-        if (fin.used > cap) return sb_fail(ctx, SB_ERR_BUDGET, "allocate: budget below the smallest candidate");
+        // a lowest candidate that does not fit leaves no slack: no step is applied, and the
+        // report kernel latches SB_ERR_BUDGET
         if (nsteps > 0) {
             int* level32 = reinterpret_cast<int*>(upsr);
             int* steps = reinterpret_cast<int*>(mark);
@@ -926,19 +943,13 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
             SB_LAUNCHED(ctx);
             level_from32_kernel<<<nblkB, BT, 0, ctx->stream>>>(a, level32);
             SB_LAUNCHED(ctx);
-            SB_CUDA(ctx, cudaMemcpyAsync(reinterpret_cast<int*>(hst) + 512, steps, sizeof(int),
-                                         cudaMemcpyDeviceToHost, ctx->stream));
+            greedy_steps = steps;
         }
         // recompute used / loss / histogram from the final levels
         SB_CUDA(ctx, cudaMemsetAsync(&dst->used, 0, sizeof(long long), ctx->stream));
         eval_kernel<<<nblkB, BT, 0, ctx->stream>>>(a, part2, 1);
         SB_LAUNCHED(ctx);
-        stt = read_state(&fin);
-        if (stt != SB_OK) return stt;
-        report->iterations = nsteps > 0 ? reinterpret_cast<int*>(hst)[512] : 0;
-        report->accepted = report->iterations;
     } else {
-        report->proxy_loss_init = 0.0;
         if (nsteps > 0) {
             const unsigned g = (unsigned)((nsteps + 255) / 256);
             step_keys_kernel<<<g, 256, 0, ctx->stream>>>(a, kA, vA);
@@ -1019,22 +1030,40 @@ extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
         // single candidate (or finished): histogram of the final levels
         eval_kernel<<<nblkB, BT, 0, ctx->stream>>>(a, part2, 0);
         SB_LAUNCHED(ctx);
-        stt = read_state(&fin);
-        if (stt != SB_OK) return stt;
-        report->proxy_loss_init = fin.loss_init;
     }
-    report->used_bits = fin.used;
-    report->proxy_loss_final = fin.loss;
-    if (mode == SB_ALLOC_SCALEBITS) {
-        report->iterations = fin.iter;
-        report->accepted = fin.accepted;
-        report->rejected = fin.rejected;
-        report->expansions = fin.expansions;
+    report_kernel<<<1, 1, 0, ctx->stream>>>(a, greedy_steps, mode == SB_ALLOC_GREEDY, report_dev);
+    SB_LAUNCHED(ctx);
+    if (own_report) {
+        SB_CUDA(ctx, cudaMemcpyAsync(ctx->pinned, report_dev, sizeof(sb_alloc_report), cudaMemcpyDeviceToHost,
+                                     ctx->stream));
     }
-    for (int l = 0; l < 8; ++l) report->level_hist[l] = fin.hist[l];
-    // device status (look-back timeouts, non-finite inputs latched earlier)
-    sb_status dev = sb_sync(ctx);
-    if (dev != SB_OK) return dev;
-    if (fin.status != 0) return sb_fail(ctx, (sb_status)fin.status, "allocate: iteration cap reached");
     return SB_OK;
+}
+
+extern "C" sb_status sb_allocate_bits_async(sb_ctx* ctx, const float* err, int64_t N,
+                                            const int64_t* block_elems, int64_t uniform_block_elems,
+                                            const int* bits, int n_bits, double budget, int mode,
+                                            double gamma0, double gammaT, uint8_t* level,
+                                            sb_alloc_report* report_dev) {
+    if (ctx && !report_dev) return sb_fail(ctx, SB_ERR_INVALID, "allocate: null report");
+    return allocate_enqueue(ctx, err, N, block_elems, uniform_block_elems, bits, n_bits, budget, mode,
+                            gamma0, gammaT, level, report_dev, false);
+}
+
+extern "C" sb_status sb_allocate_bits(sb_ctx* ctx, const float* err, int64_t N,
+                                      const int64_t* block_elems, int64_t uniform_block_elems,
+                                      const int* bits, int n_bits, double budget, int mode,
+                                      double gamma0, double gammaT, uint8_t* level,
+                                      sb_alloc_report* report) {
+    if (!ctx) return SB_ERR_INVALID;
+    if (!report) return sb_fail(ctx, SB_ERR_INVALID, "allocate: null or empty");
+    memset(report, 0, sizeof *report);
+    sb_status stt = allocate_enqueue(ctx, err, N, block_elems, uniform_block_elems, bits, n_bits, budget, mode,
+                                     gamma0, gammaT, level, nullptr, true);
+    if (stt != SB_OK) return stt;
+    SB_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    memcpy(report, ctx->pinned, sizeof *report);
+    // device status (look-back timeouts, non-finite inputs latched earlier, a budget below the
+    // smallest candidate in greedy mode, the iteration cap)
+    return sb_sync(ctx);
 }

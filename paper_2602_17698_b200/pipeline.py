@@ -62,7 +62,15 @@ class LayerResult:
     n_blocks: int
     level: Optional[torch.Tensor] = None
     report: Optional[dict] = None
+    report_dev: Optional[torch.Tensor] = None        # the report on the device (whole-step graphs)
     packed: Dict[str, tuple] = field(default_factory=dict)
+
+    def read_report(self) -> dict:
+        """The allocation's report; after a whole-step graph it is still on the device and is
+        copied here (the caller has synchronised, or is on the stream that wrote it)."""
+        if self.report is None and self.report_dev is not None:
+            self.report = Context.read_report(self.report_dev)
+        return self.report
 
     def row_perm(self, name):
         return self.perms[COUPLING[name][0]] if COUPLING[name][0] else None
@@ -98,6 +106,7 @@ class LayerWorkspace:
         self.err = torch.empty((n, L), **f32)
         self.gain = torch.empty((n, max(L - 1, 1)), **f32)   # [N, L-1] per-bit marginal gains
         self.level = torch.empty(n, dtype=torch.uint8, device=device)
+        self.report_dev = torch.zeros(128, dtype=torch.uint8, device=device)   # sb_alloc_report
         self.w_perm = ({lin.name: torch.empty((lin.rows, lin.cols), dtype=torch.bfloat16, device=device)
                         for lin in shape.linears} if keep_permuted else None)
         self.packed = {}
@@ -124,7 +133,7 @@ class _Timed:
     def __exit__(self, *exc):
         if self.timers is not None:
             self.b.record()
-            self.timers[self.stage].append((self.a, self.b))
+            self.timers.setdefault(self.stage, []).append((self.a, self.b))
 
 
 class StageGraphs:
@@ -132,14 +141,19 @@ class StageGraphs:
 
     Every pointer a stage uses is fixed (the workspace and the input tensors), so the stage's
     library calls can be captured once on the context's stream and replayed: the kernels then
-    run back to back without per-call host overhead.  The allocation stays eager (it reads its
-    report back to the host).  The context must live on a non-default stream.
+    run back to back without per-call host overhead.  With `whole=False` there is one graph per
+    stage and the allocation stays eager (it reads its report back to the host); with `whole=True`
+    `search_layer` captures the whole step, moments to pack, as ONE graph with the allocation in
+    its enqueue-only form (the report stays on the device), so that a step is one launch and
+    nothing waits for the host.  The context must live on a non-default stream.
     """
 
-    def __init__(self, ctx: Context, ctx2: Optional[Context] = None):
+    def __init__(self, ctx: Context, ctx2: Optional[Context] = None, whole: bool = False):
         # ctx2: the second context of a two-stream search_layer; its launches are captured (and
         # counted) with the first one's
         self.ctx, self.ctx2, self.graphs, self.kernels = ctx, ctx2, {}, {}
+        self.whole = whole
+        self.results = {}                  # what the captured function returned, per graph
         self.replayed_kernels = 0          # kernels launched through graph replays so far
 
     def _launches(self) -> int:
@@ -153,22 +167,26 @@ class StageGraphs:
             g = torch.cuda.CUDAGraph()
             n0 = self._launches()
             with torch.cuda.graph(g, stream=self.ctx.stream):
-                fn()
+                self.results[stage] = fn()
             self.kernels[stage] = self._launches() - n0
             self.graphs[stage] = g
         g.replay()
         self.replayed_kernels += self.kernels[stage]
+        return self.results[stage]
 
 
 def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str, torch.Tensor],
                  ws: LayerWorkspace, allocate: bool = True, pack: bool = True,
                  timers: Optional[dict] = None, graphs: Optional[StageGraphs] = None,
-                 ctx2: Optional[Context] = None) -> LayerResult:
+                 ctx2: Optional[Context] = None, _inside_whole: bool = False) -> LayerResult:
     """moments -> reorder statistics -> permutations -> block scores -> allocation -> pack.
 
     `timers`, if given, maps the stage names moments / reorder_stats / sort / scores /
     allocate / pack to lists that receive one (start, end) CUDA event pair per stage.
-    `graphs`, if given, replays each stage from a CUDA graph captured on first use.
+    `graphs`, if given, replays each stage from a CUDA graph captured on first use, or the whole
+    step from one graph (`StageGraphs(whole=True)`: `timers` then receives one pair under "step",
+    the report stays on the device until `LayerResult.read_report()`, and device-side conditions
+    are reported by the caller's next `ctx.sync()`).
     `ctx2`, if given, is a second context on another stream: the stages whose matrices are
     independent of one another (block scores, pack) deal the matrices to the two contexts in turn,
     forked from and joined back to the first context's stream, so that the ramp and the tail of one
@@ -177,9 +195,19 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
     scored and packed by the same kernels on its own.  The reorder statistics stay on one stream:
     the matrices of a coupled channel set add into one buffer in a fixed order.
     """
+    whole = graphs is not None and graphs.whole
+    if whole and not _inside_whole:
+        # the whole step as one graph: the body below runs under capture with direct calls and the
+        # enqueue-only allocation; replays return the same result object (all of it lives in `ws`)
+        with _Timed(timers, "step"):
+            res = graphs.run("step", lambda: search_layer(ctx, weights, acts, ws, allocate, pack, None,
+                                                          graphs, ctx2, _inside_whole=True))
+        res.report = None                          # decoded on demand from the device copy
+        return res
+
     def stage(name, fn):
         with _Timed(timers, name):
-            if graphs is not None:
+            if graphs is not None and not whole:
                 graphs.run(name, fn)
             else:
                 fn()
@@ -275,11 +303,16 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
         return res
 
     # a5: one global allocation over all blocks of the layer
-    with _Timed(timers, "allocate"):
-        res.level, res.report = ctx.allocate_bits(
+    if whole:
+        res.level, res.report_dev = ctx.allocate_bits_async(
             ws.err, cfg.bits, cfg.budget, cfg.mode, cfg.gamma0, cfg.gammaT,
-            uniform_block_elems=cfg.block_rows * cfg.block_cols, level=ws.level)
-    if ctx2 is not None:
+            uniform_block_elems=cfg.block_rows * cfg.block_cols, level=ws.level, report=ws.report_dev)
+    else:
+        with _Timed(timers, "allocate"):
+            res.level, res.report = ctx.allocate_bits(
+                ws.err, cfg.bits, cfg.budget, cfg.mode, cfg.gamma0, cfg.gammaT,
+                uniform_block_elems=cfg.block_rows * cfg.block_cols, level=ws.level)
+    if ctx2 is not None and not whole:
         # the allocation has just synchronised with the host and checked the first context's device
         # status; the second context's (its share of the score kernels) is read here.  What its pack
         # kernels latch is seen at the next call, or by the caller's own ctx2.sync().

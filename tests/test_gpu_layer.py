@@ -122,3 +122,43 @@ def test_two_contexts_give_the_same_layer_result():
                 assert torch.equal(a.reshape(-1)[:n], b.reshape(-1)[:n]), name
     ctx2.close()
     ctx.close()
+
+
+def test_whole_step_graph_gives_the_same_layer_result():
+    """The step as ONE CUDA graph (allocation enqueued, report on the device) against the eager
+    step with the synchronous allocation: identical levels, report and packed words, on one
+    context and on two."""
+    from paper_2602_17698_b200.binding import Context
+    from paper_2602_17698_b200.pipeline import LayerWorkspace, SearchConfig, StageGraphs, search_layer
+    torch.cuda.set_device(0)
+    shape = synth.LLAMA_TINY
+    cfg = SearchConfig(bits=[2, 3, 4, 8], budget=2.75)
+    W = synth.make_layer_weights(shape, 21, 0, DEV)
+    X = synth.make_layer_activations(shape, 640, 21, 0, DEV)
+    stream = torch.cuda.Stream(device=DEV)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        ctx = Context()
+        ctx2 = Context(stream=torch.cuda.Stream(device=DEV))
+        ws_ref = LayerWorkspace(shape, cfg, DEV)
+        ref = search_layer(ctx, W, X, ws_ref)
+        torch.cuda.synchronize()
+        for second in (None, ctx2):
+            ws = LayerWorkspace(shape, cfg, DEV)
+            graphs = StageGraphs(ctx, second, whole=True)
+            for _ in range(3):                                   # eager + capture + replay, then two replays
+                got = search_layer(ctx, W, X, ws, graphs=graphs, ctx2=second)
+            ctx.sync()
+            if second is not None:
+                second.sync()
+            assert got.report is None and got.read_report() == ref.report
+            assert torch.equal(got.level, ref.level)
+            assert torch.equal(ws.err, ws_ref.err)
+            for name in ref.packed:
+                off = ref.packed[name][1]
+                n = int(off[-1].item())
+                assert torch.equal(got.packed[name][1], off), name
+                assert torch.equal(got.packed[name][0][:n], ref.packed[name][0][:n]), name
+                assert torch.equal(got.packed[name][2], ref.packed[name][2]), name
+        ctx2.close()
+        ctx.close()

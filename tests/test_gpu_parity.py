@@ -352,6 +352,57 @@ def test_lookback_wait_runs_out_and_the_context_stays_usable(ctx):
     _check_alloc(ctx, table, bits, 2.5, SB_ALLOC_GREEDY)    # exact again, the status was cleared
 
 
+def test_allocate_enqueue_only_form_and_its_latched_errors(ctx):
+    """sb_allocate_bits_async: same levels and report as the synchronous call (which is checked
+    against the oracle above), eager and replayed from a CUDA graph; a greedy budget below the
+    smallest candidate is latched and comes back from the next sync."""
+    from paper_2602_17698_b200.binding import (Context, SB_ALLOC_GREEDY, SB_ALLOC_SCALEBITS, SB_ERR_BUDGET,
+                                               SbError)
+    rng = np.random.default_rng(8)
+    N, bits = 3000, [2, 3, 4, 8]
+    table = _tables(N, 4, 78, "ragged")
+    err = torch.from_numpy(table).to(DEV)
+    sizes = torch.from_numpy(rng.choice([1024, 4096, 16384], size=N).astype(np.int64)).to(DEV)
+    for mode in (SB_ALLOC_SCALEBITS, SB_ALLOC_GREEDY):
+        for be in (None, sizes):
+            lv_ref, rep_ref = ctx.allocate_bits(err, bits, 2.6, mode, block_elems=be)
+            lv, rep = ctx.allocate_bits_async(err, bits, 2.6, mode, block_elems=be)
+            n0 = ctx.kernel_launches()
+            ctx.sync()
+            assert ctx.kernel_launches() == n0
+            assert torch.equal(lv, lv_ref) and Context.read_report(rep) == rep_ref
+    # captured once, replayed on a changed table: the graph holds no value of the first run
+    s = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s):
+        c2 = Context()
+        e2 = err.clone()
+        lv, rep = c2.allocate_bits_async(e2, bits, 2.6)          # eager once: scratch growth
+        c2.sync()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            c2.allocate_bits_async(e2, bits, 2.6, level=lv, report=rep)
+        table2 = _tables(N, 4, 79, "convex")
+        e2.copy_(torch.from_numpy(table2).to(DEV))
+        g.replay()
+        c2.sync()
+        lv_ref, rep_ref = c2.allocate_bits(e2, bits, 2.6)
+        assert torch.equal(lv, lv_ref) and Context.read_report(rep) == rep_ref
+        c2.close()
+    torch.cuda.synchronize()
+    _check_alloc(ctx, table2, bits, 2.6, SB_ALLOC_SCALEBITS)
+    # greedy below the smallest candidate: the synchronous call and the next sync report it
+    with pytest.raises(SbError) as ei:
+        ctx.allocate_bits(err, bits, 1.5, SB_ALLOC_GREEDY)
+    assert ei.value.status == SB_ERR_BUDGET
+    lv, rep = ctx.allocate_bits_async(err, bits, 1.5, SB_ALLOC_GREEDY)
+    with pytest.raises(SbError) as ei:
+        ctx.sync()
+    assert ei.value.status == SB_ERR_BUDGET
+    assert int(lv.max().item()) == 0                            # no step was applied
+    ctx.sync()                                                  # the latch is cleared
+
+
 def test_allocate_nonuniform_block_sizes(ctx):
     from paper_2602_17698_b200.binding import SB_ALLOC_GREEDY, SB_ALLOC_SCALEBITS
     rng = np.random.default_rng(4)
