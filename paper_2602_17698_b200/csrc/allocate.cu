@@ -84,6 +84,22 @@ __device__ __forceinline__ double cta_sum(double v) {
     return s;
 }
 
+// The same sums (fixed tree, so every CTA that adds the same values gets the same bits) for two
+// doubles per thread, result in EVERY thread, one CTA barrier: the buffer alternates with `flip`,
+// and a buffer is written again only after the barrier of the call in between.
+template <int NT>
+__device__ __forceinline__ void cta_sum2_all(double& u, double& d, unsigned& flip) {
+    __shared__ double sh[2][2][NT / 32];
+    u = warp_sum(u); d = warp_sum(d);
+    if ((threadIdx.x & 31) == 0) { sh[flip][0][threadIdx.x >> 5] = u; sh[flip][1][threadIdx.x >> 5] = d; }
+    __syncthreads();
+    double su = 0.0, sd = 0.0;
+#pragma unroll
+    for (int w = 0; w < NT / 32; ++w) { su += sh[flip][0][w]; sd += sh[flip][1][w]; }
+    u = su; d = sd;
+    flip ^= 1u;
+}
+
 // true in exactly one CTA: the last one to get here.  All writes and atomics of every CTA
 // made before the call are visible to it afterwards.
 __device__ __forceinline__ bool cta_is_last(unsigned* counter) {
@@ -300,7 +316,7 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, const do
     long long k = s0.k, used = s0.used;
     double loss = s0.loss;
     int iter = 0, accepted = 0, rejected = 0, expansions = 0, status = 0;
-    unsigned flip = 0;
+    unsigned flip = 0, flip2 = 0;
 
     // bit difference of the step l -> l + 1 in nibble l (a table in registers, not in local memory)
     unsigned dbits = 0;
@@ -465,15 +481,13 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, const do
         }
 
         // ---- totals (same order in every CTA), decision, apply, replicated state update -----------
-        __shared__ double sh_dU, sh_dD;
-        if (tid == 0) {
-            double u = 0.0, dsum = 0.0;
-            for (int j = 0; j < G; ++j) u += __ldcg(w.dU + j);
-            if (!expand) for (int j = 0; j < G; ++j) dsum += __ldcg(w.dD + j);
-            sh_dU = u; sh_dD = dsum;
-        }
+        // every thread fetches the totals of its CTAs at once (one L2 round trip, not one per CTA);
+        // the sums over CTAs follow a fixed tree
+        double dU = 0.0, dD = 0.0;
         unsigned long long tot[4] = {0ull, 0ull, 0ull, 0ull};       // costU (max), nU, freed, nD
         for (int j = tid; j < G; j += LT) {
+            dU += __ldcg(w.dU + j);
+            if (!expand) dD += __ldcg(w.dD + j);
             const unsigned long long cu = __ldcg(w.costU + j);
             if (cu > tot[0]) tot[0] = cu;
             tot[1] += __ldcg(w.nU + j);
@@ -482,7 +496,7 @@ scalebits_loop_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, const do
         cta_allreduce<LT, 4, 2 | (0 << 2) | (0 << 4) | (0 << 6)>(tot, flip);
         const unsigned long long costU = tot[0], freed = tot[2];
         const unsigned nU = (unsigned)tot[1], nD = (unsigned)tot[3];
-        const double dU = sh_dU, dD = sh_dD;
+        cta_sum2_all<LT>(dU, dD, flip2);
         const bool accept = expand ? (nU > 0) : (nU > 0 && nD > 0 && dU > dD);
         if (accept) {
             for (long long i = (long long)c * LT + tid; i < a.N; i += (long long)G * LT) {
@@ -518,6 +532,7 @@ scalebits_loop_masked_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, c
         if (CLUSTER) cg::this_cluster().sync();
         else cg::this_grid().sync();
     };
+    constexpr int MLC = 8;             // list entries in flight per thread: one round for the layer-sized lists
     const int G = gridDim.x, c = blockIdx.x, tid = threadIdx.x;
     const long long per_cta = (ne + G - 1) / G;
     const long long ipt = (per_cta + LT - 1) / LT;                    // entries per thread, <= 32
@@ -531,7 +546,7 @@ scalebits_loop_masked_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, c
     long long k = s0.k, used = s0.used;
     double loss = s0.loss;
     int iter = 0, accepted = 0, rejected = 0, expansions = 0, status = 0;
-    unsigned flip = 0;
+    unsigned flip = 0, flip2 = 0;
 
     unsigned dbits = 0;
 #pragma unroll
@@ -554,14 +569,14 @@ scalebits_loop_masked_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, c
         unsigned cm = 0;
         CntCost mine{0ull, 0u, 0u};
         unsigned long long my_first = 0;
-        for (int b0 = 0; b0 < n_mine; b0 += LC) {
-            unsigned e[LC]; int lv[LC];
+        for (int b0 = 0; b0 < n_mine; b0 += MLC) {
+            unsigned e[MLC]; int lv[MLC];
 #pragma unroll
-            for (int j = 0; j < LC; ++j) e[j] = b0 + j < n_mine ? __ldg(up_ent + t_lo + b0 + j) : ENT_NONE;
+            for (int j = 0; j < MLC; ++j) e[j] = b0 + j < n_mine ? __ldg(up_ent + t_lo + b0 + j) : ENT_NONE;
 #pragma unroll
-            for (int j = 0; j < LC; ++j) lv[j] = e[j] != ENT_NONE ? (int)__ldcg(a.level + (e[j] >> 3)) : -1;
+            for (int j = 0; j < MLC; ++j) lv[j] = e[j] != ENT_NONE ? (int)__ldcg(a.level + (e[j] >> 3)) : -1;
 #pragma unroll
-            for (int j = 0; j < LC; ++j) {
+            for (int j = 0; j < MLC; ++j) {
                 if (lv[j] == (int)(e[j] & 7u)) {
                     const unsigned long long cost = cost_of(e[j]);
                     if (mine.cnt == 0) my_first = cost;
@@ -620,6 +635,13 @@ scalebits_loop_masked_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, c
             }
         }
         if (expand) {
+            // an expansion is accepted whenever U is not empty, and U is known here: the owner of a
+            // list entry writes the block's new level now, so the barrier below also publishes the
+            // levels and the iteration needs no third one
+            for (unsigned m = um; m; m &= m - 1) {
+                const unsigned e = __ldg(up_ent + t_lo + (__ffs(m) - 1));
+                if (SB_IN_BOUNDS(a.ds, SBK_ALLOC, e >> 3, a.N)) a.level[e >> 3] = (unsigned char)((e & 7u) + 1u);
+            }
             const double d = cta_sum<LT>(dU_mine);
             unsigned long long r2[2] = {costU_mine, nU_mine};
             cta_allreduce<LT, 2, 2 | (0 << 2)>(r2, flip);
@@ -632,12 +654,12 @@ scalebits_loop_masked_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, c
             // ---- down-count: the step ends at the block's level, the block is not in the up set ----
             unsigned dcm = 0;
             CntCost dm{0ull, 0u, 0u};
-            for (int b0 = 0; b0 < n_mine; b0 += LC) {
-                unsigned e[LC]; int lv[LC]; unsigned long long sr[LC];
+            for (int b0 = 0; b0 < n_mine; b0 += MLC) {
+                unsigned e[MLC]; int lv[MLC]; unsigned long long sr[MLC];
 #pragma unroll
-                for (int j = 0; j < LC; ++j) e[j] = b0 + j < n_mine ? __ldg(dn_ent + t_lo + b0 + j) : ENT_NONE;
+                for (int j = 0; j < MLC; ++j) e[j] = b0 + j < n_mine ? __ldg(dn_ent + t_lo + b0 + j) : ENT_NONE;
 #pragma unroll
-                for (int j = 0; j < LC; ++j) {
+                for (int j = 0; j < MLC; ++j) {
                     lv[j] = -1; sr[j] = 0ull;
                     if (e[j] != ENT_NONE) {
                         lv[j] = (int)__ldcg(a.level + (e[j] >> 3));
@@ -645,7 +667,7 @@ scalebits_loop_masked_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, c
                     }
                 }
 #pragma unroll
-                for (int j = 0; j < LC; ++j) {
+                for (int j = 0; j < MLC; ++j) {
                     if (lv[j] != (int)(e[j] & 7u) + 1) continue;
                     if ((unsigned)(sr[j] >> 32) == stamp && (long long)(unsigned)sr[j] < h) continue;
                     dm.cnt += 1; dm.cost += cost_of(e[j]);
@@ -699,15 +721,13 @@ scalebits_loop_masked_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, c
         }
 
         // ---- totals (same order in every CTA), decision, apply, replicated state update -----------
-        __shared__ double sh_dU, sh_dD;
-        if (tid == 0) {
-            double u = 0.0, dsum = 0.0;
-            for (int j = 0; j < G; ++j) u += __ldcg(w.dU + j);
-            if (!expand) for (int j = 0; j < G; ++j) dsum += __ldcg(w.dD + j);
-            sh_dU = u; sh_dD = dsum;
-        }
+        // every thread fetches the totals of its CTAs at once (one L2 round trip, not one per CTA);
+        // the sums over CTAs follow a fixed tree
+        double dU = 0.0, dD = 0.0;
         unsigned long long tot[4] = {0ull, 0ull, 0ull, 0ull};       // costU (max), nU, freed, nD
         for (int j = tid; j < G; j += LT) {
+            dU += __ldcg(w.dU + j);
+            if (!expand) dD += __ldcg(w.dD + j);
             const unsigned long long cu = __ldcg(w.costU + j);
             if (cu > tot[0]) tot[0] = cu;
             tot[1] += __ldcg(w.nU + j);
@@ -716,9 +736,9 @@ scalebits_loop_masked_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, c
         cta_allreduce<LT, 4, 2 | (0 << 2) | (0 << 4) | (0 << 6)>(tot, flip);
         const unsigned long long costU = tot[0], freed = tot[2];
         const unsigned nU = (unsigned)tot[1], nD = (unsigned)tot[3];
-        const double dU = sh_dU, dD = sh_dD;
+        cta_sum2_all<LT>(dU, dD, flip2);
         const bool accept = expand ? (nU > 0) : (nU > 0 && nD > 0 && dU > dD);
-        if (accept) {
+        if (accept && !expand) {
             // the owner of a list entry knows the block and its new level: no loads
             for (unsigned m = um; m; m &= m - 1) {
                 const unsigned e = __ldg(up_ent + t_lo + (__ffs(m) - 1));
@@ -733,7 +753,7 @@ scalebits_loop_masked_kernel(AllocArgs a, const unsigned* __restrict__ up_ent, c
         else if (accept) { used += (long long)costU - (long long)freed; loss += dD - dU; accepted += 1; }
         else { k /= 2; rejected += 1; }
         iter += 1;
-        phase_barrier();                                  // the new levels are visible to the next up-count
+        if (!expand) phase_barrier();                     // the new levels are visible to the next up-count
     }
     if (c == 0 && tid == 0) {
         AllocState* st = a.st;
