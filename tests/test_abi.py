@@ -76,3 +76,35 @@ def test_product_code_never_imports_the_oracle():
                 text = open(os.path.join(dirpath, fn)).read()
                 assert not re.search(r"^\s*(from|import)\s+oracle\b", text, flags=re.M), fn
                 assert "libsbo" not in text and "scalebits_oracle" not in text, fn
+
+
+def test_report_structs_of_the_binding_match_the_header(tmp_path):
+    """The two report structs are laid out by a C compiler from the header and by ctypes from the
+    binding's field lists: same size and same offset for every field, and a report decoded from
+    raw bytes (as `read_report` does for the device copy) returns the values that were stored."""
+    import subprocess
+    from paper_2602_17698_b200 import binding
+    src = tmp_path / "layout.c"
+    fields = {"sb_alloc_report": [f for f, _ in binding.AllocReport._fields_],
+              "sb_step_report": [f for f, _ in binding.StepReport._fields_]}
+    lines = ['#include <stddef.h>', '#include <stdio.h>', '#include "scalebits.h"', "int main(void) {"]
+    for struct, names in fields.items():
+        lines.append(f'  printf("{struct} %zu", sizeof({struct}));')
+        for f in names:
+            lines.append(f'  printf(" %zu", offsetof({struct}, {f}));')
+        lines.append('  printf("\\n");')
+    lines += ["  return 0;", "}"]
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split("\n")
+    for line, (struct, names), cls in zip(out, fields.items(), (binding.AllocReport, binding.StepReport)):
+        got = line.split()
+        assert got[0] == struct and int(got[1]) == ctypes.sizeof(cls), line
+        assert [int(x) for x in got[2:]] == [getattr(cls, f).offset for f in names], line
+    rep = binding.AllocReport(cap_bits=1 << 40, used_bits=(1 << 40) - 5, iterations=13, accepted=1, rejected=2,
+                              expansions=10, proxy_loss_init=2.5, proxy_loss_final=0.125)
+    for i in range(8):
+        rep.level_hist[i] = 100 + i
+    raw = torch.frombuffer(bytearray(bytes(rep)) + bytearray(16), dtype=torch.uint8)   # a larger buffer, as the workspace's
+    assert binding.Context.read_report(raw) == rep.as_dict()
