@@ -178,7 +178,7 @@ class StageGraphs:
 def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str, torch.Tensor],
                  ws: LayerWorkspace, allocate: bool = True, pack: bool = True,
                  timers: Optional[dict] = None, graphs: Optional[StageGraphs] = None,
-                 ctx2: Optional[Context] = None, _inside_whole: bool = False) -> LayerResult:
+                 ctx2: Optional[Context] = None) -> LayerResult:
     """moments -> reorder statistics -> permutations -> block scores -> allocation -> pack.
 
     `timers`, if given, maps the stage names moments / reorder_stats / sort / scores /
@@ -190,24 +190,28 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
     `ctx2`, if given, is a second context on another stream: the stages whose matrices are
     independent of one another (block scores, pack) deal the matrices to the two contexts in turn,
     forked from and joined back to the first context's stream, so that the ramp and the tail of one
-    matrix's kernels run beside the next matrix's (measured on the 8B layer: scores 0.43 -> 0.38 ms,
-    pack 0.22 -> 0.19 ms).  Every output is the same as with one context: each matrix is still
+    matrix's kernels run beside the next matrix's (measured on the 8B layer: scores 0.40 -> 0.35 ms,
+    pack 0.21 -> 0.17 ms).  Every output is the same as with one context: each matrix is still
     scored and packed by the same kernels on its own.  The reorder statistics stay on one stream:
     the matrices of a coupled channel set add into one buffer in a fixed order.
     """
-    whole = graphs is not None and graphs.whole
-    if whole and not _inside_whole:
-        # the whole step as one graph: the body below runs under capture with direct calls and the
+    if graphs is not None and graphs.whole:
+        # the whole step as one graph: the stages run under capture with direct calls and the
         # enqueue-only allocation; replays return the same result object (all of it lives in `ws`)
         with _Timed(timers, "step"):
-            res = graphs.run("step", lambda: search_layer(ctx, weights, acts, ws, allocate, pack, None,
-                                                          graphs, ctx2, _inside_whole=True))
+            res = graphs.run("step", lambda: _layer_stages(ctx, weights, acts, ws, allocate, pack, None, None,
+                                                           ctx2, enqueue_only=True))
         res.report = None                          # decoded on demand from the device copy
         return res
+    return _layer_stages(ctx, weights, acts, ws, allocate, pack, timers, graphs, ctx2, enqueue_only=False)
 
+
+def _layer_stages(ctx, weights, acts, ws, allocate, pack, timers, graphs, ctx2, enqueue_only) -> LayerResult:
+    """The stages of `search_layer`, each eager or from its own graph; `enqueue_only` takes the
+    allocation without the host round trip (its report stays in `ws.report_dev`)."""
     def stage(name, fn):
         with _Timed(timers, name):
-            if graphs is not None and not whole:
+            if graphs is not None:
                 graphs.run(name, fn)
             else:
                 fn()
@@ -303,7 +307,7 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
         return res
 
     # a5: one global allocation over all blocks of the layer
-    if whole:
+    if enqueue_only:
         res.level, res.report_dev = ctx.allocate_bits_async(
             ws.err, cfg.bits, cfg.budget, cfg.mode, cfg.gamma0, cfg.gammaT,
             uniform_block_elems=cfg.block_rows * cfg.block_cols, level=ws.level, report=ws.report_dev)
@@ -312,7 +316,7 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
             res.level, res.report = ctx.allocate_bits(
                 ws.err, cfg.bits, cfg.budget, cfg.mode, cfg.gamma0, cfg.gammaT,
                 uniform_block_elems=cfg.block_rows * cfg.block_cols, level=ws.level)
-    if ctx2 is not None and not whole:
+    if ctx2 is not None and not enqueue_only:
         # the allocation has just synchronised with the host and checked the first context's device
         # status; the second context's (its share of the score kernels) is read here.  What its pack
         # kernels latch is seen at the next call, or by the caller's own ctx2.sync().
