@@ -199,7 +199,7 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
         # the whole step as one graph: the stages run under capture with direct calls and the
         # enqueue-only allocation; replays return the same result object (all of it lives in `ws`)
         with _Timed(timers, "step"):
-            res = graphs.run("step", lambda: _layer_stages(ctx, weights, acts, ws, allocate, pack, None, None,
+            res = graphs.run(f"step:{int(allocate)}{int(pack)}", lambda: _layer_stages(ctx, weights, acts, ws, allocate, pack, None, None,
                                                            ctx2, enqueue_only=True))
         res.report = None                          # decoded on demand from the device copy
         return res
