@@ -371,6 +371,15 @@ def test_allocate_enqueue_only_form_and_its_latched_errors(ctx):
             ctx.sync()
             assert ctx.kernel_launches() == n0
             assert torch.equal(lv, lv_ref) and Context.read_report(rep) == rep_ref
+    # degenerate tables: a single candidate (no steps at all), a single block
+    for tab, bb, budget in ((table[:, :1].copy(), [4], 4.0), (table[:1].copy(), bits, 3.0)):
+        e1 = torch.from_numpy(tab).to(DEV)
+        for mode in (SB_ALLOC_SCALEBITS, SB_ALLOC_GREEDY):
+            lv_ref, rep_ref = ctx.allocate_bits(e1, bb, budget, mode)
+            lv, rep = ctx.allocate_bits_async(e1, bb, budget, mode)
+            ctx.sync()
+            assert torch.equal(lv, lv_ref) and Context.read_report(rep) == rep_ref
+            assert rep_ref["used_bits"] <= rep_ref["cap_bits"]
     # captured once, replayed on a changed table: the graph holds no value of the first run
     s = torch.cuda.Stream()
     torch.cuda.synchronize()
