@@ -624,9 +624,10 @@ def run_cuda(args):
     torch.cuda.synchronize()
     torch.cuda.set_stream(stream)
     ctx = Context()
-    # a second context on a stream of its own: the stages whose matrices are independent (block
-    # scores, pack) deal them to the two contexts in turn (pipeline.search_layer)
-    ctx2 = None if args.one_stream else Context(stream=torch.cuda.Stream(device=dev))
+    # more contexts, each on a stream of its own: the stages whose matrices are independent (block
+    # scores, pack) deal them to the contexts in turn (pipeline.search_layer)
+    n_extra = 0 if args.one_stream else max(args.streams, 1) - 1
+    ctx2 = [Context(stream=torch.cuda.Stream(device=dev)) for _ in range(n_extra)] or None
     ws = LayerWorkspace(shape, cfg, dev)
     # the timed step is ONE CUDA graph (moments ... pack, the allocation in its enqueue-only form);
     # a second pass below replays one graph per stage for the per-stage times
@@ -653,7 +654,7 @@ def run_cuda(args):
         time.sleep(0.15)
     timers = {s: [] for s in STAGES}
     def launched():
-        return (ctx.kernel_launches() + (ctx2.kernel_launches() if ctx2 is not None else 0)
+        return (ctx.kernel_launches() + sum(c.kernel_launches() for c in ctx2 or [])
                 + (graphs.replayed_kernels if graphs else 0))
 
     l0 = launched()
@@ -675,8 +676,8 @@ def run_cuda(args):
 
     res.read_report()
     ctx.sync()                                       # device-side status of everything replayed so far
-    if ctx2 is not None:
-        ctx2.sync()
+    for c in ctx2 or []:
+        c.sync()
     stagewise_ms = None
     if graphs is not None and graphs.whole:
         # per-stage times: the same steps again, one graph per stage with events between the stages
@@ -779,7 +780,9 @@ def run_cuda(args):
                            "launch": ("eager" if graphs is None else
                                       "one CUDA graph per step (allocation enqueued, report left on the device)"
                                       if graphs.whole else "one CUDA graph per stage (allocation eager)")
-                                     + ("" if ctx2 is None else "; block scores and pack dealt to two streams"),
+                                     + ("" if ctx2 is None else
+                                        "; the matrices of the block-score and pack stages dealt to %d streams"
+                                        % (len(ctx2) + 1)),
                            "allocation": res.read_report()},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
                 "roofline": roofline, "cpu_baseline": cpu,
@@ -793,9 +796,9 @@ def run_cuda(args):
                 "roofline_other_kernels": kernels, "small_layer": small_layer, "full_model": full_model,
                 "streamed_model": streamed}
         print(json.dumps(line), flush=True)
-    if ctx2 is not None:
-        ctx2.sync()
-        ctx2.close()
+    for c in ctx2 or []:
+        c.sync()
+        c.close()
     ctx.close()
     if world > 1:
         dist.barrier()              # rank 0 may still have been timing its extra legs
@@ -918,6 +921,9 @@ def main():
     ap.add_argument("--stage-graphs", action="store_true",
                     help="time the step as one CUDA graph per stage with an eager, synchronous allocation "
                          "instead of one graph for the whole step")
+    ap.add_argument("--streams", type=int, default=7,
+                    help="contexts (streams) the independent matrices of the block-score and pack stages are "
+                         "dealt to (default 7: one per matrix of the layer)")
     ap.add_argument("--one-stream", action="store_true",
                     help="one context only (no dealing of independent matrices to a second stream)")
     ap.add_argument("--only", default=None,

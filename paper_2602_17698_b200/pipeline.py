@@ -136,6 +136,15 @@ class _Timed:
             self.timers.setdefault(self.stage, []).append((self.a, self.b))
 
 
+def contexts_of(ctx: Context, ctx2) -> list:
+    """[ctx] plus the extra contexts: `ctx2` is None, one Context or a sequence of them."""
+    if ctx2 is None:
+        return [ctx]
+    if isinstance(ctx2, Context):
+        return [ctx, ctx2]
+    return [ctx] + list(ctx2)
+
+
 class StageGraphs:
     """CUDA graphs of the stages of one (workspace, weights, activations) binding.
 
@@ -148,8 +157,8 @@ class StageGraphs:
     nothing waits for the host.  The context must live on a non-default stream.
     """
 
-    def __init__(self, ctx: Context, ctx2: Optional[Context] = None, whole: bool = False):
-        # ctx2: the second context of a two-stream search_layer; its launches are captured (and
+    def __init__(self, ctx: Context, ctx2=None, whole: bool = False):
+        # ctx2: the extra context(s) of a multi-stream search_layer; their launches are captured (and
         # counted) with the first one's
         self.ctx, self.ctx2, self.graphs, self.kernels = ctx, ctx2, {}, {}
         self.whole = whole
@@ -157,7 +166,7 @@ class StageGraphs:
         self.replayed_kernels = 0          # kernels launched through graph replays so far
 
     def _launches(self) -> int:
-        return self.ctx.kernel_launches() + (self.ctx2.kernel_launches() if self.ctx2 is not None else 0)
+        return sum(c.kernel_launches() for c in contexts_of(self.ctx, self.ctx2))
 
     def run(self, stage: str, fn):
         g = self.graphs.get(stage)
@@ -175,10 +184,29 @@ class StageGraphs:
         return self.results[stage]
 
 
+def _dealt(cxs, names, fn):
+    """fn(context, name) for every name, the names dealt to the contexts in turn; the extra
+    contexts' streams fork from the first one's and join it again (graph edges under capture)."""
+    if len(cxs) == 1:
+        for n in names:
+            fn(cxs[0], n)
+        return
+    fork = torch.cuda.Event()
+    fork.record(cxs[0].stream)
+    for c in cxs[1:]:
+        c.stream.wait_event(fork)
+    for i, n in enumerate(names):
+        fn(cxs[i % len(cxs)], n)
+    for c in cxs[1:]:
+        join = torch.cuda.Event()
+        join.record(c.stream)
+        cxs[0].stream.wait_event(join)
+
+
 def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str, torch.Tensor],
                  ws: LayerWorkspace, allocate: bool = True, pack: bool = True,
                  timers: Optional[dict] = None, graphs: Optional[StageGraphs] = None,
-                 ctx2: Optional[Context] = None) -> LayerResult:
+                 ctx2=None) -> LayerResult:
     """moments -> reorder statistics -> permutations -> block scores -> allocation -> pack.
 
     `timers`, if given, maps the stage names moments / reorder_stats / sort / scores /
@@ -187,13 +215,14 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
     step from one graph (`StageGraphs(whole=True)`: `timers` then receives one pair under "step",
     the report stays on the device until `LayerResult.read_report()`, and device-side conditions
     are reported by the caller's next `ctx.sync()`).
-    `ctx2`, if given, is a second context on another stream: the stages whose matrices are
-    independent of one another (block scores, pack) deal the matrices to the two contexts in turn,
-    forked from and joined back to the first context's stream, so that the ramp and the tail of one
-    matrix's kernels run beside the next matrix's (measured on the 8B layer: scores 0.40 -> 0.35 ms,
-    pack 0.21 -> 0.17 ms).  Every output is the same as with one context: each matrix is still
-    scored and packed by the same kernels on its own.  The reorder statistics stay on one stream:
-    the matrices of a coupled channel set add into one buffer in a fixed order.
+    `ctx2`, if given, is one more context, or a sequence of them, each on a stream of its own: the
+    stages whose matrices are independent of one another (block scores, pack) deal the matrices to
+    the contexts in turn, forked from and joined back to the first context's stream, so that the
+    kernels of different matrices run beside one another (measured on the 8B layer, one / two /
+    seven contexts: scores 0.40 / 0.35 / 0.32 ms, pack 0.21 / 0.17 / 0.14 ms).  Every output is the
+    same as with one context: each matrix is still scored and packed by the same kernels on its
+    own.  The reorder statistics stay on one stream: the matrices of a coupled channel set add
+    into one buffer in a fixed order.
     """
     if graphs is not None and graphs.whole:
         # the whole step as one graph: the stages run under capture with direct calls and the
@@ -217,19 +246,8 @@ def _layer_stages(ctx, weights, acts, ws, allocate, pack, timers, graphs, ctx2, 
                 fn()
 
     def dealt(names, fn):
-        """fn(context, name) for every name: on ctx alone, or in turn on ctx and ctx2."""
-        if ctx2 is None:
-            for n in names:
-                fn(ctx, n)
-            return
-        fork = torch.cuda.Event()
-        fork.record(ctx.stream)
-        ctx2.stream.wait_event(fork)
-        for i, n in enumerate(names):
-            fn(ctx if i % 2 == 0 else ctx2, n)
-        join = torch.cuda.Event()
-        join.record(ctx2.stream)
-        ctx.stream.wait_event(join)
+        """fn(context, name) for every name: on ctx alone, or in turn on ctx and the extra contexts."""
+        _dealt(contexts_of(ctx, ctx2), names, fn)
 
     shape, cfg = ws.shape, ws.cfg
     lin = {l.name: l for l in shape.linears}
@@ -316,11 +334,12 @@ def _layer_stages(ctx, weights, acts, ws, allocate, pack, timers, graphs, ctx2, 
             res.level, res.report = ctx.allocate_bits(
                 ws.err, cfg.bits, cfg.budget, cfg.mode, cfg.gamma0, cfg.gammaT,
                 uniform_block_elems=cfg.block_rows * cfg.block_cols, level=ws.level)
-    if ctx2 is not None and not enqueue_only:
+    if not enqueue_only:
         # the allocation has just synchronised with the host and checked the first context's device
-        # status; the second context's (its share of the score kernels) is read here.  What its pack
-        # kernels latch is seen at the next call, or by the caller's own ctx2.sync().
-        ctx2.sync()
+        # status; the extra contexts' (their share of the score kernels) is read here.  What their
+        # pack kernels latch is seen at the next call, or by the caller's own sync() of them.
+        for c in contexts_of(ctx, ctx2)[1:]:
+            c.sync()
     if not pack:
         return res
 
@@ -391,7 +410,7 @@ class _Clock:
 def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConfig,
                  budgets: Sequence[float], make_weights, make_acts, device,
                  keep_tables: bool = True, keep_weights: bool = True,
-                 alloc_repeats: int = 1, ctx2: Optional[Context] = None) -> ModelResult:
+                 alloc_repeats: int = 1, ctx2=None) -> ModelResult:
     """Two sweeps over a model of `n_layers` identical decoder layers, then one global
     allocation per budget (Eq. 1 over ALL blocks of the model).
 
@@ -408,8 +427,8 @@ def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConf
     timed (`ModelResult.ms`, keys moments / stats@b / sort@b / scores@b / allocate@budget).
     The allocation is eager and paced by the host; `alloc_repeats` > 1 repeats each (deterministic)
     allocation call and keeps the fastest time, so that a host hiccup does not pass for GPU time.
-    `ctx2`, if given, is a second context on another stream: the block-score calls of a layer's
-    matrices are dealt to the two contexts in turn (as in `search_layer`).
+    `ctx2`, if given, is one more context or a sequence of them, each on a stream of its own: the
+    block-score calls of a layer's matrices are dealt to the contexts in turn (as in `search_layer`).
     """
     f32 = dict(dtype=torch.float32, device=device)
     i32 = dict(dtype=torch.int32, device=device)
@@ -508,22 +527,16 @@ def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConf
             for layer in range(n_layers):
                 W, m = layer_weights(layer), res.moments[layer]
                 with clock(f"scores@{rb}"):
-                    if ctx2 is not None:
-                        fork = torch.cuda.Event()
-                        fork.record(ctx.stream)
-                        ctx2.stream.wait_event(fork)
-                    for i, (nm, l) in enumerate(lin.items()):
+                    def score_one(cx, nm):
+                        l = lin[nm]
                         nb = (l.rows // cfg.block_rows) * (l.cols // cfg.block_cols)
                         s = block_start[(layer, nm)]
                         rp, cp = COUPLING[nm]
-                        cx = ctx2 if (ctx2 is not None and i % 2 == 1) else ctx
                         cx.block_scores(W[nm], m[l.act], cfg.bits, cfg.block_rows, cfg.block_cols, g,
                                         row_perm=perm_of(rp, layer), col_perm=perm_of(cp, layer),
                                         err=err[s:s + nb], want_gain=False)
-                    if ctx2 is not None:
-                        join = torch.cuda.Event()
-                        join.record(ctx2.stream)
-                        ctx.stream.wait_event(join)
+
+                    _dealt(contexts_of(ctx, ctx2), list(lin), score_one)
             # a5: one global allocation per budget of the group
             for b in bs:
                 for r in range(max(1, alloc_repeats)):
@@ -536,8 +549,8 @@ def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConf
                 res.perms[rb] = perms
                 res.scores[rb] = {"hidden": hid, "intermediate": mid, "v_heads": vo, "o_cols": ocol}
         ctx.stream.synchronize()
-        if ctx2 is not None:
-            ctx2.sync()                            # device status of the second context's score kernels
+        for c in contexts_of(ctx, ctx2)[1:]:
+            c.sync()                               # device status of the extra contexts' score kernels
     prev_stream.synchronize()
     totals = clock.totals()
     res.ms = {k: v for k, v in totals.items() if "#" not in k}

@@ -1,6 +1,6 @@
 """The benchmark's workload at full size (one Llama-3-8B-shaped layer, 65536 tokens) in the
 launch configuration bench.py times (non-default stream, the whole step as one CUDA graph with
-the enqueue-only allocation, block scores and pack shared between two contexts), and the
+the enqueue-only allocation, block scores and pack shared between seven contexts), and the
 corners of the stress sweep (block shapes, group sizes, seven candidates) on the same layer,
 checked on sampled outputs the oracle can compute one by one, plus the exact stages
 (permutations given scores, levels given the table, budget accounting)."""
@@ -40,13 +40,14 @@ def test_llama3_8b_layer_full_size_sampled_parity(bits, br, bc, g, budget, token
     torch.cuda.synchronize()
     with torch.cuda.stream(stream):
         ctx = Context()
-        ctx2 = Context(stream=torch.cuda.Stream())
+        ctx2 = [Context(stream=torch.cuda.Stream()) for _ in range(6)]       # seven streams, as bench.py
         ws = LayerWorkspace(shape, cfg, DEV)
         graphs = StageGraphs(ctx, ctx2, whole=True)
         search_layer(ctx, W, X, ws, graphs=graphs, ctx2=ctx2)            # eager once, captures, replays
         res = search_layer(ctx, W, X, ws, graphs=graphs, ctx2=ctx2)      # replays
         ctx.sync()
-        ctx2.sync()
+        for c in ctx2:
+            c.sync()
         res.read_report()
     torch.cuda.synchronize()
     rng = np.random.default_rng(0)
@@ -126,5 +127,6 @@ def test_llama3_8b_layer_full_size_sampled_parity(bits, br, bc, g, budget, token
             assert np.array_equal(got_meta.view(np.uint32).reshape(-1),
                                   ometa.view(np.uint32).reshape(-1)), f"meta {name} block {blk}"
     assert total_words * 32 == res.report["used_bits"]
-    ctx2.close()
+    for c in ctx2:
+        c.close()
     ctx.close()

@@ -143,14 +143,16 @@ def test_whole_step_graph_gives_the_same_layer_result():
         ws_ref = LayerWorkspace(shape, cfg, DEV)
         ref = search_layer(ctx, W, X, ws_ref)
         torch.cuda.synchronize()
-        for second in (None, ctx2):
+        more = [Context(stream=torch.cuda.Stream(device=DEV)) for _ in range(6)]
+        for second in (None, ctx2, more):                        # one, two and seven streams
             ws = LayerWorkspace(shape, cfg, DEV)
             graphs = StageGraphs(ctx, second, whole=True)
             for _ in range(3):                                   # eager + capture + replay, then two replays
                 got = search_layer(ctx, W, X, ws, graphs=graphs, ctx2=second)
             ctx.sync()
-            if second is not None:
-                second.sync()
+            for c in ([] if second is None else [second] if second is ctx2 else second):
+                c.sync()
+                assert c.kernel_launches() > 0
             assert got.report is None and got.read_report() == ref.report
             assert torch.equal(got.level, ref.level)
             assert torch.equal(ws.err, ws_ref.err)
@@ -160,5 +162,7 @@ def test_whole_step_graph_gives_the_same_layer_result():
                 assert torch.equal(got.packed[name][1], off), name
                 assert torch.equal(got.packed[name][0][:n], ref.packed[name][0][:n]), name
                 assert torch.equal(got.packed[name][2], ref.packed[name][2]), name
+        for c in more:
+            c.close()
         ctx2.close()
         ctx.close()

@@ -264,15 +264,20 @@ def test_second_context_gives_the_same_model_result():
     ctx2 = Context(stream=torch.cuda.Stream(device=DEV))
     one = search_model(ctx, shape, n_layers, cfg, budgets, make_weights, make_acts, DEV)
     two = search_model(ctx, shape, n_layers, cfg, budgets, make_weights, make_acts, DEV, ctx2=ctx2)
+    more = [ctx2] + [Context(stream=torch.cuda.Stream(device=DEV)) for _ in range(5)]
+    seven = search_model(ctx, shape, n_layers, cfg, budgets, make_weights, make_acts, DEV, ctx2=more)
     torch.cuda.synchronize()
-    assert sorted(one.tables) == sorted(two.tables)
-    for rb in one.tables:
-        assert torch.equal(one.tables[rb], two.tables[rb]), rb
-        for k in one.perms[rb]:
-            assert torch.equal(one.perms[rb][k], two.perms[rb][k]), (rb, k)
-    for b in budgets:
-        assert torch.equal(one.levels[b], two.levels[b]), b
-        for k in ("used_bits", "iterations", "cap_bits"):
-            assert one.reports[b][k] == two.reports[b][k], (b, k)
-    ctx2.close()
+    for other in (two, seven):
+        assert sorted(one.tables) == sorted(other.tables)
+        for rb in one.tables:
+            assert torch.equal(one.tables[rb], other.tables[rb]), rb
+            for k in one.perms[rb]:
+                assert torch.equal(one.perms[rb][k], other.perms[rb][k]), (rb, k)
+        for b in budgets:
+            assert torch.equal(one.levels[b], other.levels[b]), b
+            for k in ("used_bits", "iterations", "cap_bits"):
+                assert one.reports[b][k] == other.reports[b][k], (b, k)
+    for c in more:
+        assert c.kernel_launches() > 0
+        c.close()
     ctx.close()
