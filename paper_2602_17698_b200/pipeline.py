@@ -218,7 +218,8 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
     `ctx2`, if given, is one more context, or a sequence of them, each on a stream of its own: the
     stages whose matrices are independent of one another (block scores, pack) deal the matrices to
     the contexts in turn, forked from and joined back to the first context's stream, so that the
-    kernels of different matrices run beside one another (measured on the 8B layer, one / two /
+    kernels of different matrices run beside one another (the moments of the distinct inputs and
+    the sorts of the three channel sets are dealt the same way) (measured on the 8B layer, one / two /
     seven contexts: scores 0.40 / 0.35 / 0.32 ms, pack 0.21 / 0.17 / 0.14 ms).  Every output is the
     same as with one context: each matrix is still scored and packed by the same kernels on its
     own.  The reorder statistics stay on one stream: the matrices of a coupled channel set add
@@ -258,8 +259,7 @@ def _layer_stages(ctx, weights, acts, ws, allocate, pack, timers, graphs, ctx2, 
 
     # a1: calibration second moments, one per distinct linear input
     def do_moments():
-        for name, X in acts.items():
-            ctx.calib_moments(X, ws.moments[name])
+        dealt(list(acts), lambda cx, name: cx.calib_moments(acts[name], ws.moments[name]))
 
     stage("moments", do_moments)
     c = {n: ws.moments[l.act] for n, l in lin.items()}
@@ -283,16 +283,24 @@ def _layer_stages(ctx, weights, acts, ws, allocate, pack, timers, graphs, ctx2, 
                 ctx.reorder_channels(W[name], c[name], rb, g, **kw)
 
         # a3: one sort per coupled channel set ("sort only" calls: W = NULL)
+        # the three channel sets are sorted independently of one another: three chains of calls
+        def sort_hidden(cx):
+            cx.reorder_channels(None, None, rb, g, row_score=ws.hid_score, row_segment=shape.hidden,
+                                row_perm=ws.p_hid, shape=(shape.hidden, g))
+
+        def sort_intermediate(cx):
+            cx.reorder_channels(None, None, rb, g, row_score=ws.mid_score,
+                                row_segment=shape.intermediate, row_perm=ws.p_mid,
+                                shape=(shape.intermediate, g))
+
+        def sort_heads(cx):
+            cx.fold_segment_scores(ws.vo_score, ws.o_col_score, reps, hd)
+            cx.reorder_channels(None, None, rb, g, row_score=ws.vo_score, row_segment=hd,
+                                row_perm=ws.p_v, shape=(ws.vo_score.numel(), g))
+            cx.expand_segment_perm(ws.p_v, reps, hd, out=ws.p_o)
+
         def do_sort():
-            ctx.fold_segment_scores(ws.vo_score, ws.o_col_score, reps, hd)
-            ctx.reorder_channels(None, None, rb, g, row_score=ws.hid_score, row_segment=shape.hidden,
-                                 row_perm=ws.p_hid, shape=(shape.hidden, g))
-            ctx.reorder_channels(None, None, rb, g, row_score=ws.mid_score,
-                                 row_segment=shape.intermediate, row_perm=ws.p_mid,
-                                 shape=(shape.intermediate, g))
-            ctx.reorder_channels(None, None, rb, g, row_score=ws.vo_score, row_segment=hd,
-                                 row_perm=ws.p_v, shape=(ws.vo_score.numel(), g))
-            ctx.expand_segment_perm(ws.p_v, reps, hd, out=ws.p_o)
+            dealt([sort_intermediate, sort_hidden, sort_heads], lambda cx, chain: chain(cx))
 
         stage("reorder_stats", do_stats)
         stage("sort", do_sort)
@@ -455,8 +463,7 @@ def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConf
             X = make_acts(layer)
             m = {name: torch.empty(k, **f32) for name, k in shape.act_dims.items()}
             with clock("moments"):
-                for name, x in X.items():
-                    ctx.calib_moments(x, m[name])
+                _dealt(contexts_of(ctx, ctx2), list(X), lambda cx, name: cx.calib_moments(X[name], m[name]))
             ctx.stream.synchronize()               # X is dropped: its memory must not be reused early
             del X
             res.moments.append(m)
@@ -501,16 +508,28 @@ def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConf
             p_o = [torch.empty(qd, **i32) for _ in range(n_layers)]
             with clock(f"sort@{rb}"):
                 if cfg.reorder:
-                    ctx.reorder_channels(None, None, rb, g, row_score=hid, row_segment=shape.hidden,
-                                         row_perm=p_hid, shape=(shape.hidden, g))
+                    # independent chains of calls: the residual stream once, two channel sets per layer
+                    def sort_hidden(cx):
+                        cx.reorder_channels(None, None, rb, g, row_score=hid, row_segment=shape.hidden,
+                                            row_perm=p_hid, shape=(shape.hidden, g))
+
+                    def sort_intermediate(layer):
+                        return lambda cx: cx.reorder_channels(
+                            None, None, rb, g, row_score=mid[layer], row_segment=shape.intermediate,
+                            row_perm=p_mid[layer], shape=(shape.intermediate, g))
+
+                    def sort_heads(layer):
+                        def chain(cx):
+                            cx.fold_segment_scores(vo[layer], ocol[layer], reps, hd)
+                            cx.reorder_channels(None, None, rb, g, row_score=vo[layer], row_segment=hd,
+                                                row_perm=p_v[layer], shape=(kv, g))
+                            cx.expand_segment_perm(p_v[layer], reps, hd, out=p_o[layer])
+                        return chain
+
+                    chains = [sort_hidden]
                     for layer in range(n_layers):
-                        ctx.fold_segment_scores(vo[layer], ocol[layer], reps, hd)
-                        ctx.reorder_channels(None, None, rb, g, row_score=mid[layer],
-                                             row_segment=shape.intermediate, row_perm=p_mid[layer],
-                                             shape=(shape.intermediate, g))
-                        ctx.reorder_channels(None, None, rb, g, row_score=vo[layer], row_segment=hd,
-                                             row_perm=p_v[layer], shape=(kv, g))
-                        ctx.expand_segment_perm(p_v[layer], reps, hd, out=p_o[layer])
+                        chains += [sort_intermediate(layer), sort_heads(layer)]
+                    _dealt(contexts_of(ctx, ctx2), chains, lambda cx, chain: chain(cx))
             perms = {"hidden": p_hid if cfg.reorder else None}
             for layer in range(n_layers):
                 perms[("intermediate", layer)] = p_mid[layer] if cfg.reorder else None
