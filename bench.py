@@ -745,7 +745,11 @@ def run_cuda(args):
                     "unit": "GB/s", "frac": achieved / peak, "frac_nominal": achieved / NOMINAL_HBM_GBS,
                     "peak_source": peak_kind + " copy bandwidth",
                     "traffic": traffic, "algorithmic_bytes_per_launch": mom_bytes / mom_launches,
-                    "launches_per_step": mom_launches, "avg_launch_ms": stage_ms["moments"] / mom_launches}
+                    "launches_per_step": mom_launches, "avg_launch_ms": stage_ms["moments"] / mom_launches,
+                    "timing": "CUDA events around the stage's %d launches (one per distinct input%s): stage bytes / "
+                              "stage time" % (mom_launches, "" if ctx2 is None else
+                                              ", dealt to %d streams, so consecutive launches overlap at their "
+                                              "ends" % min(len(ctx2) + 1, mom_launches))}
         w_bytes = 2 * n_weights
         stage_gbs = {"moments": achieved,
                      "reorder_stats": w_bytes / (stage_ms["reorder_stats"] * 1e-3) / 1e9,
