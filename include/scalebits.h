@@ -124,6 +124,17 @@ sb_status sb_fold_segment_scores(sb_ctx* ctx, float* dst, const float* src, int6
 sb_status sb_expand_segment_perm(sb_ctx* ctx, int32_t* out, const int32_t* perm, int64_t n_src,
                                  int reps, int64_t seg);
 
+/* Score vectors of the matrices of one coupled channel set (Appendix D), each written by an
+ * sb_reorder_channels call of its own -- possibly on another context's stream, so that the
+ * calls overlap -- added in a fixed order:
+ *   dst[i] = (accumulate ? dst[i] : 0) + src[0][i] + src[1][i] + ... + src[n_src-1][i],
+ * left to right in fp32, which is the order (and the result, bit for bit) of the same calls
+ * accumulating into dst one after the other.  src: HOST array of 1..8 device pointers to
+ * fp32 [n] (read during the call); dst: device fp32 [n].  The caller orders this call after
+ * the calls that wrote the sources (stream order, or an event).                          */
+sb_status sb_sum_scores(sb_ctx* ctx, float* dst, const float* const* src, int n_src, int64_t n,
+                        int accumulate);
+
 /* Block scores -- the hot loop (block partition: Section 4.1; marginal gains of one
  * precision step: Section 4.2, Eq. 6).  On the permuted layout
  * W'[r][j] = W[row_perm[r]][col_perm[j]], for every block i of block_rows x block_cols

@@ -24,7 +24,7 @@ SB_ACC_ROW, SB_ACC_COL = 1, 2
 EXPORTS = ["sb_create", "sb_destroy", "sb_sync", "sb_last_error", "sb_kernel_launches", "sb_debug_lookback",
            "sb_checked_build",
            "sb_calib_moments", "sb_reorder_channels", "sb_fold_segment_scores",
-           "sb_expand_segment_perm", "sb_permute_matrix", "sb_block_scores", "sb_allocate_bits", "sb_allocate_bits_async",
+           "sb_expand_segment_perm", "sb_sum_scores", "sb_permute_matrix", "sb_block_scores", "sb_allocate_bits", "sb_allocate_bits_async",
            "sb_pack_blocks",
            "sb_calib_moments_noalloc", "sb_first_order_scores", "sb_exchange_step",
            "sb_reorder_channels_first_order", "sb_calib_gram",
@@ -90,6 +90,7 @@ def lib() -> C.CDLL:
                                           i64, i64, vp, vp]
         L.sb_fold_segment_scores.argtypes = [vp, vp, vp, i64, i32, i64]
         L.sb_expand_segment_perm.argtypes = [vp, vp, vp, i64, i32, i64]
+        L.sb_sum_scores.argtypes = [vp, vp, C.POINTER(C.c_void_p), i32, i64, i32]
         L.sb_permute_matrix.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
         L.sb_block_scores.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp, vp, i32, i32, i32,
                                       C.POINTER(C.c_int), i32, vp, vp, vp]
@@ -219,6 +220,15 @@ class Context:
         assert dst.numel() * reps == src.numel()
         self._check(lib().sb_fold_segment_scores(self._h, _ptr(dst, torch.float32),
                                                  _ptr(src, torch.float32), dst.numel(), reps, seg))
+
+    def sum_scores(self, dst: torch.Tensor, srcs: Sequence[torch.Tensor], accumulate: bool = False):
+        """dst = (dst +) srcs[0] + srcs[1] + ... left to right in fp32 (the score vectors of the
+        matrices of a coupled channel set, in the order a one-stream accumulation would take)."""
+        n = dst.numel()
+        assert 1 <= len(srcs) <= 8 and all(t.numel() == n and t.is_contiguous() for t in srcs)
+        arr = (C.c_void_p * len(srcs))(*[_ptr(t, torch.float32).value for t in srcs])
+        self._check(lib().sb_sum_scores(self._h, _ptr(dst, torch.float32), arr, len(srcs), n, int(accumulate)))
+        return dst
 
     def expand_segment_perm(self, perm: torch.Tensor, reps: int, seg: int, out=None) -> torch.Tensor:
         if out is None:

@@ -347,6 +347,23 @@ __global__ void rank_scatter_kernel(const int* __restrict__ rank, int64_t K, int
     perm[i / seg * seg + rank[i]] = (int32_t)i;
 }
 
+// dst[i] = (dst[i] +) src[0][i] + src[1][i] + ... in that order: the score vectors of the matrices
+// of a coupled channel set, each written by a call of its own (possibly on a stream of its own),
+// added in the order the one-stream accumulation would have taken.
+constexpr int SB_SUM_MAX_SRC = 8;
+struct SumSources { const float* p[SB_SUM_MAX_SRC]; };
+__global__ void sum_scores_kernel(float* __restrict__ dst, SumSources ss, int n_src, int64_t n, int accumulate) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float v[SB_SUM_MAX_SRC];
+#pragma unroll
+    for (int k = 0; k < SB_SUM_MAX_SRC; ++k) v[k] = k < n_src ? __ldg(ss.p[k] + i) : 0.f;
+    float s = accumulate ? __fadd_rn(dst[i], v[0]) : v[0];
+#pragma unroll
+    for (int k = 1; k < SB_SUM_MAX_SRC; ++k) if (k < n_src) s = __fadd_rn(s, v[k]);
+    dst[i] = s;
+}
+
 __global__ void fold_scores_kernel(float* dst, const float* __restrict__ src, int64_t n_dst,
                                    int reps, int64_t seg) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -546,6 +563,21 @@ sb_status sb_fold_segment_scores(sb_ctx* ctx, float* dst, const float* src, int6
         return sb_fail(ctx, SB_ERR_INVALID, "fold: bad arguments");
     SB_CUDA(ctx, cudaSetDevice(ctx->device));
     fold_scores_kernel<<<(unsigned)((n_dst + 255) / 256), 256, 0, ctx->stream>>>(dst, src, n_dst, reps, seg);
+    SB_LAUNCHED(ctx);
+    return SB_OK;
+}
+
+sb_status sb_sum_scores(sb_ctx* ctx, float* dst, const float* const* src, int n_src, int64_t n, int accumulate) {
+    if (!ctx) return SB_ERR_INVALID;
+    if (!dst || !src || n <= 0 || n_src < 1 || n_src > SB_SUM_MAX_SRC)
+        return sb_fail(ctx, SB_ERR_INVALID, "sum: bad arguments (1 .. %d sources)", SB_SUM_MAX_SRC);
+    SumSources ss{};
+    for (int k = 0; k < n_src; ++k) {
+        if (!src[k]) return sb_fail(ctx, SB_ERR_INVALID, "sum: source %d is NULL", k);
+        ss.p[k] = src[k];
+    }
+    SB_CUDA(ctx, cudaSetDevice(ctx->device));
+    sum_scores_kernel<<<(unsigned)((n + 255) / 256), 256, 0, ctx->stream>>>(dst, ss, n_src, n, accumulate);
     SB_LAUNCHED(ctx);
     return SB_OK;
 }

@@ -79,6 +79,44 @@ class LayerResult:
         return self.perms[COUPLING[name][1]] if COUPLING[name][1] else None
 
 
+# Reorder statistics (Appendix D): which coupled score vector a matrix's row / column sums belong
+# to, in the order in which the sums of a set are added.  "vo" and "o_cols" have one writer each.
+STAT_SETS = {
+    "q_proj": (None, "hidden"), "k_proj": (None, "hidden"), "v_proj": ("vo", "hidden"),
+    "o_proj": ("hidden", "o_cols"), "gate_proj": ("intermediate", "hidden"),
+    "up_proj": ("intermediate", "hidden"), "down_proj": ("hidden", "intermediate"),
+}
+
+
+def stat_part_buffers(shape: LayerShape, device) -> Dict[str, list]:
+    """One private fp32 vector per (matrix, axis) that feeds a shared score vector:
+    {"hidden": [(matrix, axis, buffer), ...], "intermediate": [...]} in adding order."""
+    size = {"hidden": shape.hidden, "intermediate": shape.intermediate}
+    parts = {"hidden": [], "intermediate": []}
+    for name, (row_set, col_set) in STAT_SETS.items():
+        for axis, key in (("row", row_set), ("col", col_set)):
+            if key in parts:
+                parts[key].append((name, axis, torch.empty(size[key], dtype=torch.float32, device=device)))
+    return parts
+
+
+def layer_statistics(cxs, W, c, rb, g, parts, vo_score, o_col_score, hid_score, mid_score, accumulate_hidden=False):
+    """a2 for one layer: every matrix's statistics by a call of its own (dealt to the contexts
+    `cxs`), then the shared vectors as fixed-order sums of the matrices' parts on cxs[0]:
+    bit for bit what the calls would give accumulating into the shared vectors one by one."""
+    own = {(name, axis): buf for key in parts for name, axis, buf in parts[key]}
+    own[("v_proj", "row")] = vo_score
+    own[("o_proj", "col")] = o_col_score
+
+    def one(cx, name):
+        cx.reorder_channels(W[name], c[name], rb, g, row_score=own.get((name, "row")),
+                            col_score=own.get((name, "col")))
+
+    _dealt(cxs, list(STAT_SETS), one)
+    cxs[0].sum_scores(hid_score, [buf for _, _, buf in parts["hidden"]], accumulate=accumulate_hidden)
+    cxs[0].sum_scores(mid_score, [buf for _, _, buf in parts["intermediate"]])
+
+
 class LayerWorkspace:
     """Device buffers for one layer, allocated once so a timed step allocates nothing."""
 
@@ -94,6 +132,8 @@ class LayerWorkspace:
         self.mid_score = torch.empty(shape.intermediate, **f32)
         self.vo_score = torch.empty(kv, **f32)
         self.o_col_score = torch.empty(qd, **f32)
+        # reorder statistics of each matrix on its own (added per coupled set in a fixed order)
+        self.stat_parts = stat_part_buffers(shape, device)
         self.p_hid = torch.empty(shape.hidden, **i32)
         self.p_mid = torch.empty(shape.intermediate, **i32)
         self.p_v = torch.empty(kv, **i32)
@@ -218,19 +258,20 @@ def search_layer(ctx: Context, weights: Dict[str, torch.Tensor], acts: Dict[str,
     `ctx2`, if given, is one more context, or a sequence of them, each on a stream of its own: the
     stages whose matrices are independent of one another (block scores, pack) deal the matrices to
     the contexts in turn, forked from and joined back to the first context's stream, so that the
-    kernels of different matrices run beside one another (the moments of the distinct inputs and
-    the sorts of the three channel sets are dealt the same way) (measured on the 8B layer, one / two /
-    seven contexts: scores 0.40 / 0.35 / 0.32 ms, pack 0.21 / 0.17 / 0.14 ms).  Every output is the
-    same as with one context: each matrix is still scored and packed by the same kernels on its
-    own.  The reorder statistics stay on one stream: the matrices of a coupled channel set add
-    into one buffer in a fixed order.
+    kernels of different matrices run beside one another (measured on the 8B layer, one / two /
+    seven contexts: scores 0.40 / 0.35 / 0.32 ms, pack 0.21 / 0.17 / 0.14 ms).  The moments of the
+    distinct inputs, the sorts of the three channel sets and the reorder statistics of the seven
+    matrices are dealt the same way; the statistics of a coupled channel set are written per
+    matrix and added afterwards in a fixed order (`layer_statistics`).  Every output is the same
+    as with one context, bit for bit: each call runs the same kernels on its own data.
     """
     if graphs is not None and graphs.whole:
         # the whole step as one graph: the stages run under capture with direct calls and the
         # enqueue-only allocation; replays return the same result object (all of it lives in `ws`)
         with _Timed(timers, "step"):
-            res = graphs.run(f"step:{int(allocate)}{int(pack)}", lambda: _layer_stages(ctx, weights, acts, ws, allocate, pack, None, None,
-                                                           ctx2, enqueue_only=True))
+            res = graphs.run(f"step:{int(allocate)}{int(pack)}",
+                             lambda: _layer_stages(ctx, weights, acts, ws, allocate, pack, None, None, ctx2,
+                                                   enqueue_only=True))
         res.report = None                          # decoded on demand from the device copy
         return res
     return _layer_stages(ctx, weights, acts, ws, allocate, pack, timers, graphs, ctx2, enqueue_only=False)
@@ -266,23 +307,11 @@ def _layer_stages(ctx, weights, acts, ws, allocate, pack, timers, graphs, ctx2, 
 
     perms = {"hidden": None, "intermediate": None, "v_heads": None, "o_heads": None}
     if cfg.reorder:
-        # a2: reorder statistics, accumulated into the buffer of each coupled channel set
-        stats = [
-            ("q_proj", dict(col_score=ws.hid_score)),
-            ("k_proj", dict(col_score=ws.hid_score, accumulate_col=True)),
-            ("v_proj", dict(row_score=ws.vo_score, col_score=ws.hid_score, accumulate_col=True)),
-            ("o_proj", dict(row_score=ws.hid_score, col_score=ws.o_col_score, accumulate_row=True)),
-            ("gate_proj", dict(row_score=ws.mid_score, col_score=ws.hid_score, accumulate_col=True)),
-            ("up_proj", dict(row_score=ws.mid_score, col_score=ws.hid_score, accumulate_row=True,
-                             accumulate_col=True)),
-            ("down_proj", dict(row_score=ws.hid_score, col_score=ws.mid_score, accumulate_row=True,
-                               accumulate_col=True)),
-        ]
+        # a2: reorder statistics, one call per matrix, added per coupled channel set in a fixed order
         def do_stats():
-            for name, kw in stats:
-                ctx.reorder_channels(W[name], c[name], rb, g, **kw)
+            layer_statistics(contexts_of(ctx, ctx2), W, c, rb, g, ws.stat_parts, ws.vo_score, ws.o_col_score,
+                             ws.hid_score, ws.mid_score)
 
-        # a3: one sort per coupled channel set ("sort only" calls: W = NULL)
         # the three channel sets are sorted independently of one another: three chains of calls
         def sort_hidden(cx):
             cx.reorder_channels(None, None, rb, g, row_score=ws.hid_score, row_segment=shape.hidden,
@@ -436,7 +465,8 @@ def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConf
     The allocation is eager and paced by the host; `alloc_repeats` > 1 repeats each (deterministic)
     allocation call and keeps the fastest time, so that a host hiccup does not pass for GPU time.
     `ctx2`, if given, is one more context or a sequence of them, each on a stream of its own: the
-    block-score calls of a layer's matrices are dealt to the contexts in turn (as in `search_layer`).
+    independent calls of a layer (moments, statistics, sorts, block scores) are dealt to the
+    contexts in turn (as in `search_layer`).
     """
     f32 = dict(dtype=torch.float32, device=device)
     i32 = dict(dtype=torch.int32, device=device)
@@ -483,24 +513,15 @@ def search_model(ctx: Context, shape: LayerShape, n_layers: int, cfg: SearchConf
             mid = [torch.empty(shape.intermediate, **f32) for _ in range(n_layers)]
             vo = [torch.empty(kv, **f32) for _ in range(n_layers)]
             ocol = [torch.empty(qd, **f32) for _ in range(n_layers)]
+            stat_parts = stat_part_buffers(shape, device)
             # sweep 1: a2, hidden scores accumulated over all layers
             for layer in range(n_layers):
                 W, m = layer_weights(layer), res.moments[layer]
                 c = {nm: m[l.act] for nm, l in lin.items()}
                 first = layer == 0
                 with clock(f"stats@{rb}"):
-                    ctx.reorder_channels(W["q_proj"], c["q_proj"], rb, g, col_score=hid, accumulate_col=not first)
-                    ctx.reorder_channels(W["k_proj"], c["k_proj"], rb, g, col_score=hid, accumulate_col=True)
-                    ctx.reorder_channels(W["v_proj"], c["v_proj"], rb, g, row_score=vo[layer], col_score=hid,
-                                         accumulate_col=True)
-                    ctx.reorder_channels(W["o_proj"], c["o_proj"], rb, g, row_score=hid, col_score=ocol[layer],
-                                         accumulate_row=True)
-                    ctx.reorder_channels(W["gate_proj"], c["gate_proj"], rb, g, row_score=mid[layer],
-                                         col_score=hid, accumulate_col=True)
-                    ctx.reorder_channels(W["up_proj"], c["up_proj"], rb, g, row_score=mid[layer], col_score=hid,
-                                         accumulate_row=True, accumulate_col=True)
-                    ctx.reorder_channels(W["down_proj"], c["down_proj"], rb, g, row_score=hid,
-                                         col_score=mid[layer], accumulate_row=True, accumulate_col=True)
+                    layer_statistics(contexts_of(ctx, ctx2), W, c, rb, g, stat_parts, vo[layer], ocol[layer],
+                                     hid, mid[layer], accumulate_hidden=not first)
             # a3: one sort of the residual stream, per-layer sorts of the other sets
             p_hid = torch.empty(shape.hidden, **i32)
             p_mid = [torch.empty(shape.intermediate, **i32) for _ in range(n_layers)]

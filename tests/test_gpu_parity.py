@@ -493,3 +493,27 @@ def test_pack_capacity_is_enforced(ctx):
     with pytest.raises(SbError) as ei:
         ctx.sync()
     assert ei.value.status == SB_ERR_SCRATCH
+
+
+def test_sum_scores_adds_left_to_right(ctx):
+    """sb_sum_scores: fp32 adds in source order, with and without the destination as first term
+    (bit-exact against the same adds in numpy float32)."""
+    from paper_2602_17698_b200.binding import SbError, SB_ERR_INVALID
+    rng = np.random.default_rng(3)
+    n = 5000
+    srcs = [(rng.standard_normal(n) * 10.0 ** rng.integers(-3, 4)).astype(np.float32) for _ in range(8)]
+    d0 = rng.standard_normal(n).astype(np.float32)
+    for k in (1, 3, 8):
+        for acc in (False, True):
+            want = d0.copy() if acc else np.zeros(n, np.float32)
+            start = 0
+            if not acc:
+                want = srcs[0].copy(); start = 1
+            for s_ in srcs[start:k]:
+                want = (want + s_).astype(np.float32)
+            dst = torch.from_numpy(d0.copy()).to(DEV)
+            ctx.sum_scores(dst, [torch.from_numpy(s_).to(DEV) for s_ in srcs[:k]], accumulate=acc)
+            ctx.sync()
+            assert np.array_equal(dst.cpu().numpy().view(np.uint32), want.view(np.uint32)), (k, acc)
+    with pytest.raises(AssertionError):
+        ctx.sum_scores(dst, [])
