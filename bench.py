@@ -929,7 +929,7 @@ def main():
                     help="contexts (streams) the independent matrices of the block-score and pack stages are "
                          "dealt to (default 7: one per matrix of the layer)")
     ap.add_argument("--one-stream", action="store_true",
-                    help="one context only (no dealing of independent matrices to a second stream)")
+                    help="one context only (no dealing of a stage's independent calls to extra streams)")
     ap.add_argument("--only", default=None,
                     help="three calls of one library call on one input, then exit (for ncu captures): "
                          "moments | gram | full_scores | dequant_gemm | reorder_stats | reorder_stats_first_order | scores | scores3 | scores7 | "

@@ -88,7 +88,7 @@ def test_tiny_layer_stagewise(bits, budget, br, bc, g):
 
 
 def test_two_contexts_give_the_same_layer_result():
-    """search_layer with a second context (block scores and pack dealt to two streams, eager and
+    """search_layer with a second context (the independent calls of the stages dealt to two streams, eager and
     from CUDA graphs) against the one-context run: every output identical."""
     from paper_2602_17698_b200.binding import Context
     from paper_2602_17698_b200.pipeline import LayerWorkspace, SearchConfig, StageGraphs, search_layer

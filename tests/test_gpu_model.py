@@ -245,7 +245,7 @@ def test_llama3_70b_streamed_allocation_matches_oracle():
 
 
 def test_second_context_gives_the_same_model_result():
-    """The block-score calls of a layer's matrices dealt to two contexts on two streams: tables,
+    """The independent calls of a layer dealt to two and to seven contexts on streams of their own: tables,
     permutations, levels and reports are those of the one-context run, bit for bit."""
     from paper_2602_17698_b200.binding import Context
     from paper_2602_17698_b200.pipeline import SearchConfig, search_model
