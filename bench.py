@@ -709,17 +709,30 @@ def run_cuda(args):
                     for n in ws.packed}
         d2h = h_level.numel() + sum(t.numel() * t.element_size() for tup in h_packed.values() for t in tup)
 
+        # The results leave on a stream of their own, so that the read-back of one step (232 MB)
+        # runs while the inputs of the next step arrive (PCIe carries both directions at once);
+        # a step's kernels wait until the previous step's results have left their buffers.
+        out_stream = torch.cuda.Stream(device=dev)
+        results_left = [None]
+
         def e2e_step():
             for n in W:
                 W[n].copy_(hW[n], non_blocking=True)
             for n in X:
                 X[n].copy_(hX[n], non_blocking=True)
+            if results_left[0] is not None:
+                stream.wait_event(results_left[0])
             r = step()
-            h_level.copy_(r.level, non_blocking=True)
-            for n, tup in r.packed.items():
-                for dst, src in zip(h_packed[n], tup):
-                    dst.copy_(src, non_blocking=True)
-            torch.cuda.synchronize()
+            computed = torch.cuda.Event()
+            computed.record(stream)
+            out_stream.wait_event(computed)
+            with torch.cuda.stream(out_stream):
+                h_level.copy_(r.level, non_blocking=True)
+                for n, tup in r.packed.items():
+                    for dst, src in zip(h_packed[n], tup):
+                        dst.copy_(src, non_blocking=True)
+                results_left[0] = torch.cuda.Event()
+                results_left[0].record(out_stream)
 
         e2e_steps = max(1, min(args.steps, args.e2e_steps))
         e2e_step()
@@ -728,6 +741,7 @@ def run_cuda(args):
         a.record()
         for _ in range(e2e_steps):
             e2e_step()
+        stream.wait_event(results_left[0])           # the last step's results are on the host
         b.record()
         barrier()
         e2e_ms = max_over_ranks(a.elapsed_time(b), world, dev) / e2e_steps
